@@ -1,0 +1,500 @@
+// Host side of the C ABI: validation, handles, table upload, argument checks, kernel dispatch.
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "guide_internal.cuh"
+
+namespace guide {
+
+static thread_local std::string g_err;
+
+int fail(int code, const char *fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_err = buf;
+    return code;
+}
+
+int cuda_fail(cudaError_t e, const char *what) {
+    return fail(GUIDE_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+int num_sms() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    return n;
+}
+
+// ---- 64-bit overflow proof for the integer FLOP / byte counts --------------------------------
+
+typedef unsigned __int128 u128;
+static const u128 LIMIT = (u128)1 << 63;   // one bit of margin below wrap-around
+
+struct Maxima { u128 T, E, A, C, R; };
+
+static bool counts_fit(const guide_model &m, uint32_t t_max, const Maxima &x) {
+    const u128 H = m.hidden, I = m.ffn, V = m.vocab, nh = m.n_heads, ab = m.a_bytes, wb = m.w_bytes,
+               kvb = m.kv_bytes, Dkv = (u128)m.n_kv_heads * (m.hidden / m.n_heads), g = m.gated;
+    const u128 T = x.T, E = x.E, A = x.A, C = x.C, R = x.R;
+    const u128 big = H > I ? H : I;
+    const u128 terms[] = {
+        4 * T * big, 3 * T * H * ab, 2 * T * H * big, R * H * big * wb + T * big * ab + T * H * ab,
+        2 * T * H * Dkv, R * H * Dkv * wb + T * Dkv * kvb, (2 + g) * T * I * ab,
+        2 * H * A, T * H * ab + C * Dkv * kvb + nh * A * ab, 5 * nh * A, 2 * nh * A * ab,
+        2 * E * H * V, R * H * V * wb + E * V * ab, E * H * ab,
+        R * 2 * t_max, (u128)2 * t_max * T * H * ab,
+    };
+    for (u128 v : terms)
+        if (v >= LIMIT) return false;
+    return true;
+}
+
+static u128 weight_bytes(const guide_model &m) {
+    const u128 H = m.hidden, I = m.ffn, V = m.vocab, Dkv = (u128)m.n_kv_heads * (m.hidden / m.n_heads);
+    return ((u128)m.n_layers * (2 * H * H + 2 * H * Dkv + (2 + (u128)m.gated) * H * I) + 2 * V * H) * m.w_bytes;
+}
+
+static int check_closed_form_overflow(const guide_space &s) {
+    for (size_t mi = 0; mi < s.models.size(); mi++) {
+        const guide_model &m = s.models[mi];
+        const u128 b = s.max_batch;
+        for (const guide_len_pair &p : s.pairs) {
+            const u128 lin = p.lin, n = p.lout - 1;
+            Maxima pre{b * lin, b, b * lin * lin, b * lin, 1};
+            Maxima dec{b * n, b * n, b * (n * lin + n * (n + 1) / 2), b * (n * lin + n * (n + 1) / 2), n};
+            if (!counts_fit(m, s.max_tp, pre) || !counts_fit(m, s.max_tp, dec))
+                return fail(GUIDE_ERR_OVERFLOW,
+                            "model %zu with batch %u and lengths (%u, %u) overflows a 64-bit FLOP/byte count",
+                            mi, s.max_batch, p.lin, p.lout);
+            if (b * (1 + n) >= LIMIT) return fail(GUIDE_ERR_OVERFLOW, "request-iteration count overflows");
+        }
+    }
+    return GUIDE_OK;
+}
+
+static int check_trace_overflow(const guide_space &s, const guide_trace &t) {
+    const u128 q = std::max<uint64_t>(t.max_tokens, t.n_zero ? (uint64_t)s.max_lin + s.max_lout : 0);
+    const u128 b = s.max_batch;
+    for (size_t mi = 0; mi < s.models.size(); mi++) {
+        Maxima pre{b * q, b, b * q * q, b * q, 1};
+        Maxima dec{b, b, b * q, b * q, 1};
+        if (!counts_fit(s.models[mi], s.max_tp, pre) || !counts_fit(s.models[mi], s.max_tp, dec))
+            return fail(GUIDE_ERR_OVERFLOW, "model %zu overflows a 64-bit FLOP/byte count on this trace", mi);
+    }
+    return GUIDE_OK;
+}
+
+// ---- device tables ------------------------------------------------------------------------------
+
+// Derived per-model quantities and the reciprocal rates of every hardware x framework pair.
+__global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *gh, u32 n_h, const guide_fw *gf,
+                               u32 n_f, DModel *dm, DRate *dr) {
+    const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n_m) {
+        const guide_model m = gm[i];
+        DModel d;
+        d.N = m.n_layers; d.H = m.hidden; d.nh = m.n_heads; d.nkv = m.n_kv_heads; d.I = m.ffn; d.V = m.vocab;
+        d.g = m.gated; d.wb = m.w_bytes; d.ab = m.a_bytes; d.kvb = m.kv_bytes;
+        d.Dkv = m.n_kv_heads * (m.hidden / m.n_heads);
+        d.pad = 0;
+        const u64 H = d.H, Dkv = d.Dkv, I = d.I, V = d.V;
+        const u64 per_layer = 2 * H * H + 2 * H * Dkv + (2 + (u64)d.g) * H * I;
+        d.wbytes = ((u64)d.N * per_layer + 2 * V * H) * d.wb;
+        d.kv2 = 2 * (u64)d.N * Dkv * d.kvb;
+        dm[i] = d;
+    }
+    if (i < n_h * n_f) {
+        const guide_hw h = gh[i / n_f];
+        const guide_fw f = gf[i % n_f];
+        DRate r;
+        for (int k = 0; k < 3; k++) {
+            r.inv_c[k] = 1.0 / (h.peak_flops * f.e_c[k]);
+            r.inv_m[k] = 1.0 / (h.mem_bw * f.e_m[k]);
+        }
+        r.inv_comm = 1.0 / (h.comm_bw * f.e_comm);
+        r.clat = h.comm_lat;
+        r.tovh = f.t_ovh;
+        r.price = h.price_per_hr;
+        r.usable = h.mem_bytes - (h.mem_bytes / 1000) * f.reserve_permille;
+        r.flash = f.flash;
+        r.kv_block = f.kv_block;
+        dr[i] = r;
+    }
+}
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+int space_on_device(guide_space *s, DSpace *out) {
+    int dev = 0;
+    GUIDE_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(s->mu);
+    for (const DeviceTables &d : s->dev)
+        if (d.device == dev) { *out = d.view; return GUIDE_OK; }
+
+    const size_t n_m = s->models.size(), n_h = s->hw.size(), n_f = s->fw.size();
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t o_gm = take(n_m * sizeof(guide_model)), o_gh = take(n_h * sizeof(guide_hw)),
+                 o_gf = take(n_f * sizeof(guide_fw)), o_dm = take(n_m * sizeof(DModel)),
+                 o_dr = take(n_h * n_f * sizeof(DRate)), o_b = take(s->batch.size() * 4),
+                 o_t = take(s->tp.size() * 4), o_p = take(s->pairs.size() * 8);
+    char *blob = nullptr;
+    GUIDE_CUDA(cudaMalloc(&blob, off));
+    cudaError_t e = cudaSuccess;
+    auto put = [&](size_t o, const void *src, size_t bytes) {
+        if (e == cudaSuccess) e = cudaMemcpy(blob + o, src, bytes, cudaMemcpyHostToDevice);
+    };
+    put(o_gm, s->models.data(), n_m * sizeof(guide_model));
+    put(o_gh, s->hw.data(), n_h * sizeof(guide_hw));
+    put(o_gf, s->fw.data(), n_f * sizeof(guide_fw));
+    put(o_b, s->batch.data(), s->batch.size() * 4);
+    put(o_t, s->tp.data(), s->tp.size() * 4);
+    put(o_p, s->pairs.data(), s->pairs.size() * 8);
+    if (e == cudaSuccess) {
+        const u32 n = (u32)std::max(n_m, n_h * n_f);
+        k_build_tables<<<(n + 127) / 128, 128>>>((const guide_model *)(blob + o_gm), (u32)n_m,
+                                                 (const guide_hw *)(blob + o_gh), (u32)n_h,
+                                                 (const guide_fw *)(blob + o_gf), (u32)n_f,
+                                                 (DModel *)(blob + o_dm), (DRate *)(blob + o_dr));
+        e = cudaGetLastError();
+        if (e == cudaSuccess) e = cudaStreamSynchronize(0);
+    }
+    if (e != cudaSuccess) { cudaFree(blob); return cuda_fail(e, "uploading the space tables"); }
+    DeviceTables d;
+    d.device = dev;
+    d.blob = blob;
+    d.view.models = (const DModel *)(blob + o_dm);
+    d.view.rates = (const DRate *)(blob + o_dr);
+    d.view.batch = (const u32 *)(blob + o_b);
+    d.view.tp = (const u32 *)(blob + o_t);
+    d.view.pairs = (const uint2 *)(blob + o_p);
+    d.view.n_m = (u32)n_m; d.view.n_h = (u32)n_h; d.view.n_f = (u32)n_f;
+    d.view.n_b = (u32)s->batch.size(); d.view.n_t = (u32)s->tp.size(); d.view.n_l = (u32)s->pairs.size();
+    s->dev.push_back(d);
+    *out = d.view;
+    return GUIDE_OK;
+}
+
+int trace_on_device(guide_trace *t, DTrace *out) {
+    int dev = 0;
+    GUIDE_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(t->mu);
+    for (const DeviceTrace &d : t->dev)
+        if (d.device == dev) { *out = d.view; return GUIDE_OK; }
+    const size_t n = t->arrival.size();
+    const size_t o_a = 0, o_i = align_up(n * 8, 256), o_o = o_i + align_up(n * 4, 256), total = o_o + align_up(n * 4, 256);
+    char *blob = nullptr;
+    GUIDE_CUDA(cudaMalloc(&blob, total));
+    cudaError_t e = cudaMemcpy(blob + o_a, t->arrival.data(), n * 8, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(blob + o_i, t->in_len.data(), n * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(blob + o_o, t->out_len.data(), n * 4, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) { cudaFree(blob); return cuda_fail(e, "uploading the trace"); }
+    DeviceTrace d;
+    d.device = dev;
+    d.blob = blob;
+    d.view.arrival = (const double *)(blob + o_a);
+    d.view.in_len = (const u32 *)(blob + o_i);
+    d.view.out_len = (const u32 *)(blob + o_o);
+    d.view.n = (u32)n;
+    d.view.max_tokens = t->max_tokens;
+    d.view.any_zero = t->n_zero ? 1 : 0;
+    d.view.sum_out = t->sum_out;
+    d.view.n_zero = t->n_zero;
+    t->dev.push_back(d);
+    *out = d.view;
+    return GUIDE_OK;
+}
+
+static bool pow2(uint32_t v) { return v && !(v & (v - 1)); }
+
+static int resolve_range(const guide_space *s, const guide_sim_opts *o, Range *r) {
+    r->first = o ? o->first : 0;
+    r->count = o ? o->count : 0;
+    if (r->first > s->size) return fail(GUIDE_ERR_INVALID, "first (%llu) is past the end of the space", (unsigned long long)r->first);
+    if (r->count == 0) r->count = s->size - r->first;
+    if (r->count > s->size - r->first) return fail(GUIDE_ERR_INVALID, "range runs past the end of the space");
+    if (o && (o->time_model < 0 || o->time_model > 1 || o->tp_model < 0 || o->tp_model > 1))
+        return fail(GUIDE_ERR_INVALID, "unknown time_model or tp_model");
+    return GUIDE_OK;
+}
+
+static int check_workspace(const void *ws, size_t have, size_t need) {
+    if (need == 0) return GUIDE_OK;
+    if (!ws) return fail(GUIDE_ERR_WORKSPACE, "workspace is NULL, %zu bytes needed", need);
+    if ((uintptr_t)ws % 256) return fail(GUIDE_ERR_WORKSPACE, "workspace must be 256-byte aligned");
+    if (have < need) return fail(GUIDE_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", have, need);
+    return GUIDE_OK;
+}
+
+static const double *metric_array(const guide_outputs &o, int key) {
+    switch (key) {
+    case GUIDE_LATENCY: return o.latency;
+    case GUIDE_TTFT: return o.ttft;
+    case GUIDE_TTFT_P99: return o.ttft_p99;
+    case GUIDE_TPOT: return o.tpot;
+    case GUIDE_THROUGHPUT: return o.thr_decode;
+    case GUIDE_COST_PER_HR: return o.cost_per_hr;
+    case GUIDE_COST_PER_TOKEN: return o.cost_per_token;
+    }
+    return nullptr;
+}
+
+static int check_selection_args(const guide_space *space, const guide_trace *trace, const guide_outputs *outputs,
+                                const guide_constraints *cons, const int *keys, int n_keys) {
+    if (!space || !cons) return fail(GUIDE_ERR_INVALID, "space and constraints are required");
+    for (int i = 0; i < n_keys; i++)
+        if (keys[i] < GUIDE_LATENCY || keys[i] > GUIDE_COST_PER_TOKEN) return fail(GUIDE_ERR_INVALID, "unknown metric %d", keys[i]);
+    if (cons->ttft_stat < GUIDE_STAT_MEAN || cons->ttft_stat > GUIDE_STAT_P99) return fail(GUIDE_ERR_INVALID, "unknown ttft_stat");
+    if (std::isnan(cons->max_ttft) || std::isnan(cons->max_latency) || std::isnan(cons->max_cost_per_hr) ||
+        std::isnan(cons->min_throughput))
+        return fail(GUIDE_ERR_INVALID, "a constraint is NaN");
+    if (!outputs) {
+        if (trace) return fail(GUIDE_ERR_UNSUPPORTED, "fused selection evaluates the closed form only: run guide_simulate on the trace and pass its outputs");
+        return GUIDE_OK;
+    }
+    if (!outputs->status) return fail(GUIDE_ERR_INVALID, "materialised selection needs outputs->status");
+    for (int i = 0; i < n_keys; i++)
+        if (!metric_array(*outputs, keys[i])) return fail(GUIDE_ERR_INVALID, "the array of metric %d is NULL", keys[i]);
+    const double *ttft = cons->ttft_stat == GUIDE_STAT_MEAN ? outputs->ttft
+                         : cons->ttft_stat == GUIDE_STAT_P50 ? outputs->ttft_p50 : outputs->ttft_p99;
+    if (cons->max_ttft < INFINITY && !ttft) return fail(GUIDE_ERR_INVALID, "max_ttft is set but its array is NULL");
+    if (cons->max_latency < INFINITY && !outputs->latency) return fail(GUIDE_ERR_INVALID, "max_latency is set but latency is NULL");
+    if (cons->max_cost_per_hr < INFINITY && !outputs->cost_per_hr) return fail(GUIDE_ERR_INVALID, "max_cost_per_hr is set but cost_per_hr is NULL");
+    if (cons->min_throughput > 0.0 && !outputs->thr_decode) return fail(GUIDE_ERR_INVALID, "min_throughput is set but thr_decode is NULL");
+    return GUIDE_OK;
+}
+
+}  // namespace guide
+
+using namespace guide;
+
+extern "C" {
+
+const char *guide_last_error(void) { return g_err.c_str(); }
+
+int guide_space_create(const guide_space_desc *d, guide_space **out) {
+    if (!d || !out) return fail(GUIDE_ERR_INVALID, "desc and out are required");
+    *out = nullptr;
+    if (!d->models || !d->hw || !d->fw || !d->batch || !d->tp || !d->pairs)
+        return fail(GUIDE_ERR_INVALID, "an axis pointer is NULL");
+    if (!d->n_models || !d->n_hw || !d->n_fw || !d->n_batch || !d->n_tp || !d->n_pairs)
+        return fail(GUIDE_ERR_INVALID, "an axis is empty");
+    if (d->n_models > 4096 || (uint64_t)d->n_hw * d->n_fw > 65536)
+        return fail(GUIDE_ERR_INVALID, "too many models (max 4096) or hardware x framework pairs (max 65536)");
+    guide_space *s = new (std::nothrow) guide_space;
+    if (!s) return fail(GUIDE_ERR_INVALID, "out of host memory");
+    s->models.assign(d->models, d->models + d->n_models);
+    s->hw.assign(d->hw, d->hw + d->n_hw);
+    s->fw.assign(d->fw, d->fw + d->n_fw);
+    s->batch.assign(d->batch, d->batch + d->n_batch);
+    s->tp.assign(d->tp, d->tp + d->n_tp);
+    s->pairs.assign(d->pairs, d->pairs + d->n_pairs);
+    int rc = GUIDE_OK;
+    for (uint32_t v : s->tp) {
+        if (!pow2(v) || v > 1024) { rc = fail(GUIDE_ERR_UNSUPPORTED, "TP degree %u is not a power of two in 1..1024", v); break; }
+        s->max_tp = std::max(s->max_tp, v);
+    }
+    for (uint32_t v : s->batch) {
+        if (rc) break;
+        if (!v) rc = fail(GUIDE_ERR_INVALID, "batch size 0");
+        s->max_batch = std::max(s->max_batch, v);
+    }
+    for (const guide_len_pair &p : s->pairs) {
+        if (rc) break;
+        if (!p.lin || !p.lout) rc = fail(GUIDE_ERR_INVALID, "a length pair has a zero length");
+        s->max_lin = std::max(s->max_lin, p.lin);
+        s->max_lout = std::max(s->max_lout, p.lout);
+    }
+    for (size_t i = 0; i < s->models.size() && !rc; i++) {
+        const guide_model &m = s->models[i];
+        if (!m.n_layers || !m.hidden || !m.n_heads || !m.n_kv_heads || !m.ffn || !m.vocab || !m.w_bytes ||
+            !m.a_bytes || !m.kv_bytes || m.gated > 1)
+            rc = fail(GUIDE_ERR_INVALID, "model %zu has a zero size or gated > 1", i);
+        else if (m.hidden % m.n_heads)
+            rc = fail(GUIDE_ERR_INVALID, "model %zu: hidden is not a multiple of n_heads", i);
+        else if (2ull * m.n_layers * m.n_kv_heads * (m.hidden / m.n_heads) * m.kv_bytes < s->max_tp)
+            rc = fail(GUIDE_ERR_INVALID, "model %zu: KV bytes per token per GPU would round to zero", i);
+        else if (weight_bytes(m) >= LIMIT)
+            rc = fail(GUIDE_ERR_OVERFLOW, "model %zu: weight bytes overflow", i);
+    }
+    for (size_t i = 0; i < s->hw.size() && !rc; i++) {
+        const guide_hw &h = s->hw[i];
+        if (!(h.peak_flops > 0) || !(h.mem_bw > 0) || !(h.comm_bw > 0) || !(h.comm_lat >= 0) ||
+            !(h.price_per_hr >= 0) || !std::isfinite(h.peak_flops + h.mem_bw + h.comm_bw + h.comm_lat + h.price_per_hr))
+            rc = fail(GUIDE_ERR_INVALID, "hardware profile %zu has a non-positive or non-finite rate", i);
+    }
+    for (size_t i = 0; i < s->fw.size() && !rc; i++) {
+        const guide_fw &f = s->fw[i];
+        bool ok = f.kv_block >= 1 && f.reserve_permille <= 1000 && f.flash <= 1 && f.e_comm > 0 && f.t_ovh >= 0 &&
+                  std::isfinite(f.e_comm + f.t_ovh);
+        for (int k = 0; k < 3; k++) ok = ok && f.e_c[k] > 0 && f.e_m[k] > 0 && std::isfinite(f.e_c[k] + f.e_m[k]);
+        if (!ok) rc = fail(GUIDE_ERR_INVALID, "framework profile %zu has a bad efficiency, kv_block or reserve", i);
+        else if (f.policy != GUIDE_POLICY_PREFILL_FIRST) rc = fail(GUIDE_ERR_UNSUPPORTED, "framework profile %zu: unknown policy", i);
+    }
+    if (!rc) {
+        u128 n = (u128)d->n_models * d->n_hw * d->n_fw * d->n_batch * d->n_tp * d->n_pairs;
+        if (n >= ((u128)1 << 48)) rc = fail(GUIDE_ERR_OVERFLOW, "the space has 2^48 configs or more");
+        s->size = (uint64_t)n;
+    }
+    if (!rc) {
+        // capacity arithmetic: (lin+lout rounded to blocks) x KV bytes per token
+        u128 worst = ((u128)s->max_lin + s->max_lout + 0xFFFFFFFFull);
+        for (const guide_model &m : s->models)
+            if (worst * (2ull * m.n_layers * m.n_kv_heads * (m.hidden / m.n_heads) * m.kv_bytes) >= LIMIT)
+                rc = fail(GUIDE_ERR_OVERFLOW, "KV bytes of one request overflow");
+    }
+    if (!rc) rc = check_closed_form_overflow(*s);
+    if (rc) { delete s; return rc; }
+    *out = s;
+    return GUIDE_OK;
+}
+
+void guide_space_destroy(guide_space *s) {
+    if (!s) return;
+    int cur = 0;
+    const bool have = cudaGetDevice(&cur) == cudaSuccess;
+    for (DeviceTables &d : s->dev) {
+        if (have && cudaSetDevice(d.device) == cudaSuccess) cudaFree(d.blob);
+    }
+    if (have && !s->dev.empty()) cudaSetDevice(cur);
+    delete s;
+}
+
+uint64_t guide_space_size(const guide_space *s) { return s ? s->size : 0; }
+
+int guide_space_decode(const guide_space *s, uint64_t idx, guide_config *o) {
+    if (!s || !o) return fail(GUIDE_ERR_INVALID, "space and out are required");
+    if (idx >= s->size) return fail(GUIDE_ERR_INVALID, "index %llu is outside the space", (unsigned long long)idx);
+    o->pair_pos = (uint32_t)(idx % s->pairs.size()); idx /= s->pairs.size();
+    o->tp_pos = (uint32_t)(idx % s->tp.size()); idx /= s->tp.size();
+    o->batch_pos = (uint32_t)(idx % s->batch.size()); idx /= s->batch.size();
+    o->fw = (uint32_t)(idx % s->fw.size()); idx /= s->fw.size();
+    o->hw = (uint32_t)(idx % s->hw.size()); idx /= s->hw.size();
+    o->model = (uint32_t)idx;
+    o->batch = s->batch[o->batch_pos];
+    o->tp = s->tp[o->tp_pos];
+    o->lin = s->pairs[o->pair_pos].lin;
+    o->lout = s->pairs[o->pair_pos].lout;
+    return GUIDE_OK;
+}
+
+int guide_trace_load(const double *arrival, const uint32_t *in_len, const uint32_t *out_len, uint64_t n,
+                     guide_trace **out) {
+    if (!out) return fail(GUIDE_ERR_INVALID, "out is required");
+    *out = nullptr;
+    if (!arrival || !in_len || !out_len) return fail(GUIDE_ERR_INVALID, "a trace array is NULL");
+    if (n == 0 || n > 65536) return fail(GUIDE_ERR_INVALID, "n_req must be in 1..65536");
+    guide_trace *t = new (std::nothrow) guide_trace;
+    if (!t) return fail(GUIDE_ERR_INVALID, "out of host memory");
+    t->arrival.assign(arrival, arrival + n);
+    t->in_len.assign(in_len, in_len + n);
+    t->out_len.assign(out_len, out_len + n);
+    int rc = GUIDE_OK;
+    for (uint64_t i = 0; i < n && !rc; i++) {
+        if (!(arrival[i] >= 0) || !std::isfinite(arrival[i])) rc = fail(GUIDE_ERR_INVALID, "arrival[%llu] is negative or not finite", (unsigned long long)i);
+        else if (i && arrival[i] < arrival[i - 1]) rc = fail(GUIDE_ERR_INVALID, "arrivals must be non-decreasing (entry %llu)", (unsigned long long)i);
+        else if (in_len[i] && !out_len[i]) rc = fail(GUIDE_ERR_INVALID, "request %llu has an input length but no output length", (unsigned long long)i);
+        else if (in_len[i] > (1u << 24) || out_len[i] > (1u << 24)) rc = fail(GUIDE_ERR_INVALID, "request %llu is longer than 2^24 tokens", (unsigned long long)i);
+        if (in_len[i]) {
+            t->max_in = std::max(t->max_in, in_len[i]);
+            t->max_out = std::max(t->max_out, out_len[i]);
+            t->max_tokens = std::max(t->max_tokens, in_len[i] + out_len[i]);
+            t->sum_out += out_len[i];
+        } else t->n_zero++;
+    }
+    if (rc) { delete t; return rc; }
+    *out = t;
+    return GUIDE_OK;
+}
+
+void guide_trace_destroy(guide_trace *t) {
+    if (!t) return;
+    int cur = 0;
+    const bool have = cudaGetDevice(&cur) == cudaSuccess;
+    for (DeviceTrace &d : t->dev)
+        if (have && cudaSetDevice(d.device) == cudaSuccess) cudaFree(d.blob);
+    if (have && !t->dev.empty()) cudaSetDevice(cur);
+    delete t;
+}
+
+uint64_t guide_trace_size(const guide_trace *t) { return t ? t->arrival.size() : 0; }
+
+size_t guide_workspace_bytes(const guide_space *space, const guide_trace *trace, const guide_sim_opts *) {
+    if (!space || !trace) return 0;
+    return trace_workspace_bytes((u32)trace->arrival.size());
+}
+
+int guide_simulate(const guide_space *space_c, const guide_trace *trace_c, const guide_sim_opts *opts,
+                   const guide_outputs *out, void *ws, size_t ws_bytes, void *stream) {
+    guide_space *space = const_cast<guide_space *>(space_c);
+    guide_trace *trace = const_cast<guide_trace *>(trace_c);
+    if (!space || !out) return fail(GUIDE_ERR_INVALID, "space and out are required");
+    Range r;
+    int rc = resolve_range(space, opts, &r);
+    if (rc) return rc;
+    const int time_model = opts ? opts->time_model : GUIDE_TIME_MAX, tp_model = opts ? opts->tp_model : GUIDE_TP_EXPLICIT;
+    if (!trace && (out->req_ttft || out->req_tpot))
+        return fail(GUIDE_ERR_INVALID, "per-request outputs need a trace");
+    if (trace) {
+        if (space->max_batch > GUIDE_TRACE_MAX_BATCH)
+            return fail(GUIDE_ERR_UNSUPPORTED, "the trace kernel keeps at most %u requests resident; the batch axis goes to %u",
+                        GUIDE_TRACE_MAX_BATCH, space->max_batch);
+        if ((rc = check_trace_overflow(*space, *trace))) return rc;
+        if ((rc = check_workspace(ws, ws_bytes, trace_workspace_bytes((u32)trace->arrival.size())))) return rc;
+    }
+    if (r.count == 0) return GUIDE_OK;
+    DSpace ds;
+    if ((rc = space_on_device(space, &ds))) return rc;
+    if (!trace) return launch_closed_form(ds, r, time_model, tp_model, *out, (cudaStream_t)stream);
+    DTrace dt;
+    if ((rc = trace_on_device(trace, &dt))) return rc;
+    return launch_trace_sim(ds, dt, r, time_model, tp_model, opts ? opts->max_iters : 0, *out, ws, ws_bytes,
+                            (cudaStream_t)stream);
+}
+
+size_t guide_select_workspace_bytes(const guide_space *, uint32_t k) {
+    return (k == 0 || k > GUIDE_TOPK_MAX) ? 0 : topk_workspace_bytes(k);
+}
+size_t guide_pareto_workspace_bytes(const guide_space *) { return pareto_workspace_bytes(); }
+
+int guide_select_topk(const guide_space *space_c, const guide_trace *trace, const guide_outputs *outputs,
+                      const guide_sim_opts *opts, const guide_constraints *cons, int key, uint32_t k,
+                      uint64_t *idx_out, double *key_out, uint32_t *count_out, void *ws, size_t ws_bytes,
+                      void *stream) {
+    guide_space *space = const_cast<guide_space *>(space_c);
+    int rc = check_selection_args(space, trace, outputs, cons, &key, 1);
+    if (rc) return rc;
+    if (k == 0 || k > GUIDE_TOPK_MAX) return fail(GUIDE_ERR_INVALID, "k must be in 1..%u", GUIDE_TOPK_MAX);
+    if (!idx_out || !key_out || !count_out) return fail(GUIDE_ERR_INVALID, "an output pointer is NULL");
+    Range r;
+    if ((rc = resolve_range(space, opts, &r))) return rc;
+    if ((rc = check_workspace(ws, ws_bytes, topk_workspace_bytes(k)))) return rc;
+    DSpace ds;
+    if ((rc = space_on_device(space, &ds))) return rc;
+    return launch_topk(ds, r, outputs, opts ? opts->time_model : 0, opts ? opts->tp_model : 0, *cons, key, k,
+                       (u64 *)idx_out, key_out, count_out, ws, (cudaStream_t)stream);
+}
+
+int guide_pareto(const guide_space *space_c, const guide_trace *trace, const guide_outputs *outputs,
+                 const guide_sim_opts *opts, const guide_constraints *cons, int xm, int ym, uint64_t *idx_out,
+                 uint32_t cap, uint32_t *count_out, void *ws, size_t ws_bytes, void *stream) {
+    guide_space *space = const_cast<guide_space *>(space_c);
+    const int keys[2] = {xm, ym};
+    int rc = check_selection_args(space, trace, outputs, cons, keys, 2);
+    if (rc) return rc;
+    if (!count_out || (cap && !idx_out)) return fail(GUIDE_ERR_INVALID, "an output pointer is NULL");
+    Range r;
+    if ((rc = resolve_range(space, opts, &r))) return rc;
+    if ((rc = check_workspace(ws, ws_bytes, pareto_workspace_bytes()))) return rc;
+    DSpace ds;
+    if ((rc = space_on_device(space, &ds))) return rc;
+    return launch_pareto(ds, r, outputs, opts ? opts->time_model : 0, opts ? opts->tp_model : 0, *cons, xm, ym,
+                         (u64 *)idx_out, cap, count_out, ws, (cudaStream_t)stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,85 @@
+// Library-internal declarations: handles, device views, launch entry points of each kernel file.
+#pragma once
+#include <cstdarg>
+#include <cstdio>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "../../include/guide.h"
+#include "model.cuh"
+
+namespace guide {
+
+int fail(int code, const char *fmt, ...);          // records the message, returns code
+int cuda_fail(cudaError_t e, const char *what);
+
+#define GUIDE_CUDA(call)                                            \
+    do {                                                            \
+        cudaError_t e__ = (call);                                   \
+        if (e__ != cudaSuccess) return guide::cuda_fail(e__, #call); \
+    } while (0)
+
+struct DeviceTables {
+    int device = -1;
+    void *blob = nullptr;
+    DSpace view{};
+};
+
+struct DeviceTrace {
+    int device = -1;
+    void *blob = nullptr;
+    DTrace view{};
+};
+
+}  // namespace guide
+
+struct guide_space {
+    std::vector<guide_model> models;
+    std::vector<guide_hw> hw;
+    std::vector<guide_fw> fw;
+    std::vector<uint32_t> batch, tp;
+    std::vector<guide_len_pair> pairs;
+    uint64_t size = 0;
+    uint32_t max_batch = 0, max_tp = 0, max_lin = 0, max_lout = 0;
+    std::mutex mu;
+    std::vector<guide::DeviceTables> dev;
+};
+
+struct guide_trace {
+    std::vector<double> arrival;
+    std::vector<uint32_t> in_len, out_len;
+    uint32_t max_in = 0, max_out = 0, max_tokens = 0, n_zero = 0;
+    uint64_t sum_out = 0;
+    std::mutex mu;
+    std::vector<guide::DeviceTrace> dev;
+};
+
+namespace guide {
+
+// device views for the current device (uploads on first use)
+int space_on_device(guide_space *s, DSpace *out);
+int trace_on_device(guide_trace *t, DTrace *out);
+
+struct Range { u64 first, count; };
+
+// closed_form.cu
+int launch_closed_form(const DSpace &s, Range r, int time_model, int tp_model, const guide_outputs &o,
+                       cudaStream_t st);
+// trace_sim.cu
+size_t trace_workspace_bytes(u32 n_req);
+int launch_trace_sim(const DSpace &s, const DTrace &t, Range r, int time_model, int tp_model, u64 max_iters,
+                     const guide_outputs &o, void *ws, size_t ws_bytes, cudaStream_t st);
+// select.cu
+size_t topk_workspace_bytes(u32 k);
+size_t pareto_workspace_bytes();
+int launch_topk(const DSpace &s, Range r, const guide_outputs *mat, int time_model, int tp_model,
+                const guide_constraints &c, int key, u32 k, u64 *idx_out, double *key_out, u32 *count_out,
+                void *ws, cudaStream_t st);
+int launch_pareto(const DSpace &s, Range r, const guide_outputs *mat, int time_model, int tp_model,
+                  const guide_constraints &c, int xm, int ym, u64 *idx_out, u32 cap, u32 *count_out,
+                  void *ws, cudaStream_t st);
+
+int num_sms();
+
+}  // namespace guide

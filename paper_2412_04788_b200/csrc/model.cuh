@@ -1,0 +1,304 @@
+// Device-side performance model: task table, roofline, stage time, memory check.
+//
+// Everything here is written so that the same values come out regardless of how a kernel
+// arranges its loops: integer FLOP/byte counts are exact 64-bit integers, converted to double
+// once, combined in one fixed order, and the file is compiled with -fmad=false so no
+// multiply-add is ever fused.  Scaling by a power of two (the tensor-parallel degree, the
+// task multiplicities 2 and 1+g) is exact in binary64 and commutes with rounding, which is
+// what lets a kernel fold those factors into a cached table without changing a bit.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace guide {
+
+typedef unsigned long long u64;
+typedef unsigned int u32;
+
+enum { CLS_LINEAR = 0, CLS_ATTN = 1, CLS_ELEM = 2 };
+
+// per-model table entry (built on the device by k_build_tables)
+struct DModel {
+    u32 N, H, nh, nkv, I, V, g, wb, ab, kvb;
+    u32 Dkv;      // n_kv * (H / n_h)
+    u32 pad;
+    u64 wbytes;   // all weights in bytes: (N (2H^2 + 2 H Dkv + (2+g) H I) + 2 V H) * w_b
+    u64 kv2;      // KV bytes per token over all GPUs: 2 N Dkv kv_b   (Sec. 3.3.1 with H -> Dkv)
+};
+
+// per (hardware, framework) entry: reciprocal rates (product first, then one reciprocal)
+struct DRate {
+    double inv_c[3], inv_m[3], inv_comm, clat, tovh, price;
+    u64 usable;   // MEM - (MEM/1000) * reserve_permille
+    u32 flash, kv_block;
+};
+
+struct DSpace {
+    const DModel *models;
+    const DRate *rates;          // [n_h * n_f]
+    const u32 *batch, *tp;
+    const uint2 *pairs;          // (lin, lout)
+    u32 n_m, n_h, n_f, n_b, n_t, n_l;
+};
+
+struct DTrace {
+    const double *arrival;
+    const u32 *in_len, *out_len;
+    u32 n;
+    u32 max_tokens;              // max over requests of in+out (0-length requests excluded)
+    u32 any_zero;                // some request takes the config's lengths
+    u64 sum_out;                 // sum of out_len over requests with explicit lengths
+    u32 n_zero;                  // number of requests taking the config's lengths
+};
+
+struct Cfg { u32 m, h, f, b, t, l; };
+
+__device__ __forceinline__ Cfg decode_index(const DSpace &s, u64 idx) {
+    Cfg c;
+    c.l = (u32)(idx % s.n_l); idx /= s.n_l;
+    c.t = (u32)(idx % s.n_t); idx /= s.n_t;
+    c.b = (u32)(idx % s.n_b); idx /= s.n_b;
+    c.f = (u32)(idx % s.n_f); idx /= s.n_f;
+    c.h = (u32)(idx % s.n_h); idx /= s.n_h;
+    c.m = (u32)idx;
+    return c;
+}
+
+// ---- task table --------------------------------------------------------------------------------
+// Compute load F and data size B of every distinct task of one layer, for a stage with T new
+// tokens, E sequences emitting a token, A = sum(query x context), C = sum(context), R repeats.
+// Values are per GPU (sharded part / t + replicated part) with the task multiplicity folded in.
+// o_proj has the same F and B as q_proj, and sv the same as qk, so each pair shares an entry.
+struct TaskTab {
+    double F1, B1;      // norm x2 (ELEM)
+    double F2, B2;      // q_proj, o_proj (LINEAR)
+    double F3, B3;      // k_proj + v_proj (LINEAR)
+    double F5, B5;      // residual x2 (ELEM)
+    double F6, B6;      // up (+ gate) (LINEAR)
+    double F7, B7;      // activation (ELEM)
+    double F8, B8;      // down (LINEAR)
+    double F9, B9;      // qk = sv (ATTN), B9 with FlashAttention
+    double B9x;         // ... without: + score matrix
+    double F10, B10x;   // softmax (ATTN); with FlashAttention its B is 0
+    double F13, B13;    // lm_head (LINEAR), once per stage
+    double hops, cbytes; // all-reduce: latency hops R*2(t-1), bytes 2(t-1) M / t
+    double Rd;
+};
+
+__device__ __forceinline__ double cvt(u64 x) { return __ull2double_rn(x); }
+
+// sharded / t + replicated, one rounding in the add
+__device__ __forceinline__ double per_gpu(u64 sh, u64 rp, double inv_t) { return cvt(sh) * inv_t + cvt(rp); }
+
+// The part of the table that does not depend on A or C (everything but attention).
+__device__ __forceinline__ void build_fixed_tasks(const DModel &m, u32 t, u64 T, u64 E, u64 R, TaskTab &k) {
+    const double inv_t = 1.0 / (double)t;      // t is a power of two: exact
+    const u64 H = m.H, I = m.I, Dkv = m.Dkv, V = m.V, ab = m.ab, wb = m.wb, kvb = m.kvb;
+    const u64 TH = T * H, THa = TH * ab, TI = T * I, TIa = TI * ab;
+    k.F1 = 2.0 * cvt(4 * TH);
+    k.B1 = 2.0 * cvt(2 * THa);
+    k.F2 = cvt(2 * TH * H) * inv_t;
+    k.B2 = per_gpu(R * (H * H * wb) + THa, THa, inv_t);
+    k.F3 = 2.0 * (cvt(2 * TH * Dkv) * inv_t);
+    k.B3 = 2.0 * per_gpu(R * (H * Dkv * wb) + T * Dkv * kvb, THa, inv_t);
+    k.F5 = 2.0 * cvt(TH);
+    k.B5 = 2.0 * cvt(3 * THa);
+    const double mult6 = (double)(1 + m.g);
+    k.F6 = mult6 * (cvt(2 * TH * I) * inv_t);
+    k.B6 = mult6 * per_gpu(R * (H * I * wb) + TIa, THa, inv_t);
+    k.F7 = cvt(4 * TI) * inv_t;
+    k.B7 = cvt((2 + m.g) * TIa) * inv_t;
+    k.F8 = cvt(2 * TI * H) * inv_t;
+    k.B8 = per_gpu(R * (I * H * wb) + TIa, THa, inv_t);
+    k.F13 = cvt(2 * (E * H) * V) * inv_t;
+    k.B13 = per_gpu(R * (H * V * wb) + E * V * ab, E * H * ab, inv_t);
+    k.Rd = cvt(R);
+    if (t > 1) {
+        k.hops = cvt(R * (u64)(2 * (t - 1)));
+        k.cbytes = cvt((u64)(2 * (t - 1)) * THa) * inv_t;
+    } else {
+        k.hops = 0.0; k.cbytes = 0.0;
+    }
+}
+
+// Attention entries: query x context work A, KV read of C context tokens, score matrix X.
+__device__ __forceinline__ void build_attn_tasks(const DModel &m, u32 t, u64 T, u64 A, u64 C, TaskTab &k) {
+    const double inv_t = 1.0 / (double)t;
+    const u64 THa = T * m.H * m.ab;
+    const u64 kv_read = C * m.Dkv * m.kvb;
+    const u64 X = (u64)m.nh * A * m.ab;
+    k.F9 = cvt(2 * m.H * A) * inv_t;
+    k.B9 = cvt(THa + kv_read) * inv_t;
+    k.B9x = cvt(THa + kv_read + X) * inv_t;
+    k.F10 = cvt(5 * (u64)m.nh * A) * inv_t;
+    k.B10x = cvt(2 * X) * inv_t;
+}
+
+template <int TIME_SUM>
+__device__ __forceinline__ double task_time(double F, double B, double ic, double im) {
+    const double tc = F * ic;          // compute time (Sec. 3.5.1)
+    const double tm = B * im;          // read/write time
+    return TIME_SUM ? tc + tm : fmax(tc, tm);   // Sec. 3.5.1 literal sum, or the roofline of Sec. 3.4.2
+}
+
+// Sum of the eight non-attention layer tasks in their fixed order.
+template <int TIME_SUM>
+__device__ __forceinline__ double eval_fixed(const TaskTab &k, const DRate &r) {
+    const double icL = r.inv_c[CLS_LINEAR], imL = r.inv_m[CLS_LINEAR];
+    const double icE = r.inv_c[CLS_ELEM], imE = r.inv_m[CLS_ELEM];
+    const double t2 = task_time<TIME_SUM>(k.F2, k.B2, icL, imL);
+    double s = task_time<TIME_SUM>(k.F1, k.B1, icE, imE);
+    s = s + t2;
+    s = s + task_time<TIME_SUM>(k.F3, k.B3, icL, imL);
+    s = s + t2;
+    s = s + task_time<TIME_SUM>(k.F5, k.B5, icE, imE);
+    s = s + task_time<TIME_SUM>(k.F6, k.B6, icL, imL);
+    s = s + task_time<TIME_SUM>(k.F7, k.B7, icE, imE);
+    s = s + task_time<TIME_SUM>(k.F8, k.B8, icL, imL);
+    return s;
+}
+
+template <int TIME_SUM>
+__device__ __forceinline__ double eval_attn(const TaskTab &k, const DRate &r) {
+    const double ic = r.inv_c[CLS_ATTN], im = r.inv_m[CLS_ATTN];
+    const double t9 = task_time<TIME_SUM>(k.F9, r.flash ? k.B9 : k.B9x, ic, im);
+    const double t10 = task_time<TIME_SUM>(k.F10, r.flash ? 0.0 : k.B10x, ic, im);
+    return (t9 + t10) + t9;
+}
+
+__device__ __forceinline__ double eval_comm(const TaskTab &k, const DRate &r) {
+    // two ring all-reduces per layer; both terms are exactly 0 when t == 1
+    return 2.0 * (k.hops * r.clat + k.cbytes * r.inv_comm);
+}
+
+template <int TIME_SUM>
+__device__ __forceinline__ double eval_head(const TaskTab &k, const DRate &r) {
+    return task_time<TIME_SUM>(k.F13, k.B13, r.inv_c[CLS_LINEAR], r.inv_m[CLS_LINEAR]);
+}
+
+// T_phase = R t_ovh + (N ((S_fix + S_att) + S_comm) + t_head), then the optional log2 rule.
+__device__ __forceinline__ double combine_phase(double s_fix, double s_att, double s_comm, double t_head,
+                                                double Rd, double Nd, double tovh, double log2_factor) {
+    const double layer = (s_fix + s_att) + s_comm;
+    double tp = Rd * tovh + (Nd * layer + t_head);
+    if (log2_factor != 1.0) tp = tp * log2_factor;   // x1.0 would be exact anyway
+    return tp;
+}
+
+template <int TIME_SUM>
+__device__ __forceinline__ double eval_phase(const TaskTab &k, const DRate &r, double Nd, double log2_factor) {
+    return combine_phase(eval_fixed<TIME_SUM>(k, r), eval_attn<TIME_SUM>(k, r), eval_comm(k, r),
+                         eval_head<TIME_SUM>(k, r), k.Rd, Nd, r.tovh, log2_factor);
+}
+
+// (1 + log2 t) / t for the throughput rule of Sec. 3.2; 1.0 when the explicit TP model is used.
+__device__ __forceinline__ double log2_rule_factor(u32 t, int tp_model) {
+    if (tp_model == 0) return 1.0;
+    const u32 lg = 31 - __clz(t);
+    return (double)(1 + lg) / (double)t;
+}
+
+// ---- memory model (Sec. 3.2 Step 1, Sec. 3.3.1) ---------------------------------------------
+
+// floor(num / den) for den >= 1, by one double division plus a correction when both fit 2^53
+__device__ __forceinline__ u64 floor_div(u64 num, u64 den) {
+    if ((num | den) >> 53) return num / den;
+    u64 q = __double2ull_rz(__ull2double_rn(num) / __ull2double_rn(den));
+    // the rounded quotient is within 1 of the true one
+    if (q * den > num) q--;
+    else if ((q + 1) * den <= num) q++;
+    return q;
+}
+
+struct MemInfo { u64 w_gpu, kv_tok; u32 log2t; };
+
+__device__ __forceinline__ MemInfo mem_info(const DModel &m, u32 t) {
+    MemInfo mi;
+    mi.log2t = 31 - __clz(t);
+    mi.w_gpu = (m.wbytes + (u64)(t - 1)) >> mi.log2t;   // ceil(W w_b / t)
+    mi.kv_tok = m.kv2 >> mi.log2t;
+    return mi;
+}
+
+__device__ __forceinline__ u32 clamp_u32(u64 v) { return v > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)v; }
+
+// ---- one config in closed form -------------------------------------------------------------------
+
+struct Metrics {
+    double latency, ttft, tpot, thr, cost_hr, cost_tok;
+    u64 n_iters, n_req_iters;
+    u32 bmax;
+    u32 status;
+};
+
+__device__ __forceinline__ void set_infeasible(Metrics &o) {
+    const double inf = __longlong_as_double(0x7FF0000000000000LL);
+    o.latency = inf; o.ttft = inf; o.tpot = inf; o.thr = 0.0; o.cost_hr = inf; o.cost_tok = inf;
+    o.n_iters = 0; o.n_req_iters = 0;
+}
+
+// status and B_max of a closed-form config
+__device__ __forceinline__ u32 closed_form_feasibility(const DModel &m, const DRate &r, const MemInfo &mi, u32 t,
+                                                       u32 b, u32 lin, u32 lout, u32 &bmax_out) {
+    const u64 S = (u64)lin + lout;
+    const u64 s_blk = r.kv_block == 1 ? S : ((S + r.kv_block - 1) / r.kv_block) * r.kv_block;
+    const u64 bmax = r.usable > mi.w_gpu ? floor_div(r.usable - mi.w_gpu, s_blk * mi.kv_tok) : 0;
+    u32 st = 0;
+    if (r.usable <= mi.w_gpu) st |= 1;
+    if ((u64)b > bmax) st |= 2;
+    if ((m.nh & (t - 1)) != 0 || (m.nkv & (t - 1)) != 0) st |= 4;   // t is a power of two
+    bmax_out = clamp_u32(bmax);
+    return st;
+}
+
+// final metrics from the two stage times (Sec. 3.2: TTFT = prefill time, throughput; Sec. 5.1)
+__device__ __forceinline__ void closed_form_metrics(double t_pre, double t_dec, u32 b, u32 n, u32 t, double price,
+                                                    Metrics &o) {
+    const double inf = __longlong_as_double(0x7FF0000000000000LL);
+    o.ttft = t_pre;
+    o.latency = t_pre + t_dec;
+    o.cost_hr = price * (double)t;
+    if (n > 0) {
+        o.tpot = t_dec / (double)n;
+        o.thr = cvt((u64)b * n) / t_dec;
+        o.cost_tok = (o.cost_hr / 3600.0) / o.thr;
+    } else {
+        o.tpot = 0.0; o.thr = 0.0; o.cost_tok = inf;
+    }
+    o.n_iters = 1 + (u64)n;
+    o.n_req_iters = (u64)b * (1 + (u64)n);
+}
+
+// Whole closed-form evaluation of one config, nothing cached (used where configs arrive in
+// arbitrary order; the tiled kernels hoist the table building out of the hardware x framework loop).
+template <int TIME_SUM>
+__device__ __forceinline__ void closed_form_eval(const DSpace &s, const Cfg &c, int tp_model, Metrics &o) {
+    const DModel m = s.models[c.m];
+    const DRate &r = s.rates[c.h * s.n_f + c.f];
+    const u32 t = s.tp[c.t], b = s.batch[c.b];
+    const uint2 pr = s.pairs[c.l];
+    const u32 lin = pr.x, lout = pr.y;
+    const MemInfo mi = mem_info(m, t);
+    o.status = closed_form_feasibility(m, r, mi, t, b, lin, lout, o.bmax);
+    if (o.status) { set_infeasible(o); return; }
+    const u32 tt = tp_model ? 1u : t;
+    const double lf = log2_rule_factor(t, tp_model);
+    const double Nd = (double)m.N;
+    TaskTab k;
+    const u64 Tp = (u64)b * lin;
+    build_fixed_tasks(m, tt, Tp, b, 1, k);
+    build_attn_tasks(m, tt, Tp, Tp * lin, Tp, k);
+    const double t_pre = eval_phase<TIME_SUM>(k, r, Nd, lf);
+    const u32 n = lout - 1;
+    double t_dec = 0.0;
+    if (n > 0) {
+        const u64 Td = (u64)b * n;
+        const u64 ctx = (u64)b * ((u64)n * lin + ((u64)n * (n + 1)) / 2);
+        build_fixed_tasks(m, tt, Td, Td, n, k);
+        build_attn_tasks(m, tt, Td, ctx, ctx, k);
+        t_dec = eval_phase<TIME_SUM>(k, r, Nd, lf);
+    }
+    closed_form_metrics(t_pre, t_dec, b, n, t, r.price, o);
+}
+
+}  // namespace guide

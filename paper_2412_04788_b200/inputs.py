@@ -230,20 +230,22 @@ def make_trace(seed: int, n: int, rate: float, lengths: bool,
 # the five workloads
 # ----------------------------------------------------------------------------------------------
 
-def workload(k: int, scale: float = 1.0):
+def workload(k: int, scale: float = 1.0, trace_scale: float | None = None):
     """Workload k in 1..5 -> dict(space, trace or None, constraints, topk, name).
 
-    `scale` < 1 shrinks the hardware axis (and the trace) for quick parity cases while keeping
-    every other axis, value law and seed; scale = 1 is the full-size workload.
+    `scale` < 1 shrinks the hardware axis and `trace_scale` (default: = scale) the trace, for
+    quick parity cases that keep every other axis, value law and seed; 1 is the full size.
     """
     seed = SEED_BASE + k
+    if trace_scale is None:
+        trace_scale = scale
     if k == 1:
         models = models_from_shapes([SHAPES_8[2]])
         hw, mem = seeded_hw(seed, 4, mem_gb=[24, 48, 80, 192])
         fw_f, fw_i = seeded_fw(seed, 1)
         space = _space(models, hw, mem, fw_f, fw_i, [1, 2, 4, 8, 16, 32, 64], [1, 2, 4],
                        pairs_grid([128, 512, 2048], [128, 512]))
-        trace = make_trace(seed, max(8, int(256 * scale)), 4.0, lengths=False)
+        trace = make_trace(seed, max(8, int(256 * trace_scale)), 4.0, lengths=False)
         cons = {"max_ttft": 0.5, "ttft_stat": "p99"}
         return {"name": "C1", "space": space, "trace": trace, "constraints": cons,
                 "topk": {"key": "cost_per_token", "k": 8}}
@@ -262,7 +264,7 @@ def workload(k: int, scale: float = 1.0):
         hw, mem = seeded_hw(seed, n_hw, mem_gb=[192] * n_hw)
         fw_f, fw_i = seeded_fw(seed, 4)
         space = _space(models, hw, mem, fw_f, fw_i, BATCHES_16, [1, 2, 4, 8], [(1, 1)])
-        trace = make_trace(seed, max(8, int(4096 * scale)), 16.0, lengths=True)
+        trace = make_trace(seed, max(8, int(4096 * trace_scale)), 16.0, lengths=True)
         return {"name": "C3", "space": space, "trace": trace, "constraints": {},
                 "topk": {"key": "ttft_p99", "k": 8}}
     if k == 4:
@@ -271,7 +273,7 @@ def workload(k: int, scale: float = 1.0):
         hw, mem = seeded_hw(seed, n_hw, mem_range=(16, 192))
         fw_f, fw_i = seeded_fw(seed, 4)
         space = _space(models, hw, mem, fw_f, fw_i, BATCHES_16, [1, 2, 4, 8], [(1, 1)])
-        trace = make_trace(seed, max(8, int(1024 * scale)), 32.0, lengths=True)
+        trace = make_trace(seed, max(8, int(1024 * trace_scale)), 32.0, lengths=True)
         return {"name": "C4", "space": space, "trace": trace, "constraints": {},
                 "topk": {"key": "ttft_p99", "k": 8}}
     if k == 5:

@@ -1,0 +1,102 @@
+"""GPU parity, trace-driven continuous batching: warp-per-config kernel against the oracle."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2412_04788_b200 import guide, inputs as I
+from gpu_util import assert_parity, bit_mismatches, run_simulate, run_topk
+
+pytestmark = pytest.mark.gpu
+
+SMALL = [4, 256, 8, 4, 512, 1000, 1, 2, 2, 2]
+
+
+def toy_space(golden, mem, kv_block, batch):
+    return I._space(np.array([golden["model"]]), np.array([golden["hw"]]), np.array([mem]), np.array([[1.0] * 7 + [0.0]]),
+                    np.array([[1, kv_block, 0, 0]]), list(batch), [1], [(4, 3)])
+
+
+def test_hand_worked_timelines(golden):
+    for tl in golden["timelines"]:
+        sp = toy_space(golden, tl["mem"], tl["kv_block"], [tl["max_batch"]])
+        n = len(tl["arrival"])
+        tr = {"arrival": np.array(tl["arrival"]), "in_len": np.zeros(n, np.uint32), "out_len": np.zeros(n, np.uint32)}
+        got, *_ = run_simulate(sp, tr, per_request=True)
+        assert got["status"][0] == 0
+        for k in ("latency", "ttft", "ttft_p50", "ttft_p99", "tpot"):
+            assert got[k][0] == tl[k], (tl["name"], k)
+        assert got["req_ttft"][0].tolist() == tl["req_ttft"] and got["req_tpot"][0].tolist() == tl["req_tpot"]
+        assert got["thr_decode"][0] == tl["dec_tok"] / tl["dec_time"]
+        assert got["n_iters"][0] == tl["n_iters"] and got["n_req_iters"][0] == tl["n_req_iters"]
+
+
+def test_workload1_full(golden):
+    """504 configs x the 256-request trace, lengths taken from each config; every output incl. the
+    per-request ones; then the top-8 by cost per token under the 500 ms p99-TTFT objective."""
+    w = I.workload(1)
+    want = oracle.simulate(w["space"], w["trace"], per_request=True)
+    got, out_dev, sp, tr = run_simulate(w["space"], w["trace"], per_request=True)
+    assert_parity(got, want, fields=guide.F64_OUTPUTS + ("req_ttft", "req_tpot"))
+    assert sum(bit_mismatches(got, want, guide.F64_OUTPUTS + ("req_ttft", "req_tpot")).values()) == 0
+    assert (want["status"] == 0).sum() > 100
+    for key in ("cost_per_token", "cost_per_hr"):
+        idx, val, cnt = run_topk(sp, out_dev, w["constraints"], key, 8, tr=tr)
+        w_idx, w_val, w_cnt = oracle.select_topk(want, w["constraints"], key, 8)
+        assert cnt == w_cnt and np.array_equal(idx, w_idx)
+        assert np.array_equal(val.view(np.uint64), w_val.view(np.uint64))
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_memory_pressure_small(seed):
+    """Tiny model and memories, 4-token blocks: preemption and recompute happen in most configs."""
+    n = 96
+    tr = {"arrival": I.poisson_arrivals(seed, n, 3000.0), "in_len": I.randint(seed, 81, n, 1, 60).astype(np.uint32),
+          "out_len": I.randint(seed, 82, n, 1, 40).astype(np.uint32)}
+    hw, _ = I.seeded_hw(seed, 6, mem_gb=[1] * 6)
+    w_bytes, kv_tok = oracle.weight_bytes_per_gpu(SMALL, 1), oracle.kv_bytes_per_token(SMALL, 1)
+    mem = np.array([w_bytes + nb * 4 * kv_tok + 7 for nb in (20, 25, 26, 40, 90, 5000)], dtype=np.uint64)
+    fw_f, fw_i = I.seeded_fw(seed, 2, kv_block=4, reserve_permille=0)
+    sp = I._space(np.array([SMALL]), hw, mem, fw_f, fw_i, [1, 2, 5, 17, 64, 256], [1, 2, 4], [(1, 1)])
+    want = oracle.simulate(sp, tr, per_request=True)
+    got, *_ = run_simulate(sp, tr, per_request=True)
+    assert_parity(got, want, fields=guide.F64_OUTPUTS + ("req_ttft", "req_tpot"))
+    assert sum(bit_mismatches(got, want, guide.F64_OUTPUTS + ("req_ttft", "req_tpot")).values()) == 0
+    assert want["n_preempt"].sum() > 0
+    assert (want["status"] == guide.ST_KV).any() and (want["status"] == 0).any()
+
+
+@pytest.mark.parametrize("k", [3, 4])
+def test_workloads_3_and_4_reduced(k):
+    """Workloads 3 and 4 with a shortened trace and one hardware profile in eight: same axes,
+    laws and seeds, sized so the oracle takes seconds."""
+    w = I.workload(k, scale=1 / 32 if k == 3 else 1 / 64, trace_scale=1 / 8 if k == 3 else 1 / 4)
+    want = oracle.simulate(w["space"], w["trace"], per_request=(k == 3))
+    got, *_ = run_simulate(w["space"], w["trace"], per_request=(k == 3))
+    fields = guide.F64_OUTPUTS + (("req_ttft", "req_tpot") if k == 3 else ())
+    assert_parity(got, want, fields=fields)
+    assert sum(bit_mismatches(got, want, fields).values()) == 0
+    assert (want["status"] == 0).sum() > 50
+
+
+def test_iteration_cap_and_models(golden):
+    sp = toy_space(golden, 10**6, 1, [1])
+    tr = {"arrival": np.array([0.0, 1.0]), "in_len": np.zeros(2, np.uint32), "out_len": np.zeros(2, np.uint32)}
+    got, *_ = run_simulate(sp, tr, max_iters=5)
+    assert got["status"][0] == guide.ST_ITER and np.isinf(got["latency"][0])
+    got, *_ = run_simulate(sp, tr, max_iters=6)
+    assert got["status"][0] == 0
+    w = I.workload(1, scale=1.0, trace_scale=0.25)
+    for tm, tpm in ((1, 0), (0, 1)):
+        want = oracle.simulate(w["space"], w["trace"], time_model=tm, tp_model=tpm)
+        got, *_ = run_simulate(w["space"], w["trace"], time_model=tm, tp_model=tpm)
+        assert_parity(got, want)
+        assert sum(bit_mismatches(got, want).values()) == 0
+
+
+def test_run_to_run_identical():
+    """The same launch twice gives the same bits (no dependence on scheduling order)."""
+    w = I.workload(4, scale=1 / 64, trace_scale=1 / 4)
+    a, *_ = run_simulate(w["space"], w["trace"])
+    b, *_ = run_simulate(w["space"], w["trace"])
+    for k in guide.F64_OUTPUTS:
+        assert np.array_equal(a[k].view(np.uint64), b[k].view(np.uint64))
