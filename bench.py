@@ -1,0 +1,415 @@
+#!/usr/bin/env python
+"""Benchmark of the deployment-space evaluator.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--extras LIST]
+
+A step is one pass of the whole closed-form path over the 983,040-config grid (workload 2):
+guide_simulate (memory check, task list, roofline, metrics -> 6 fp64 arrays + mask + B_max),
+guide_select_topk (constraint filter + top-8 by cost per token) and guide_pareto (latency vs $/h),
+with the space tables already resident on the device.  `value` is configs per second over the K
+timed steps; L2 is flushed between steps (outputs are smaller than L2).  The trace-driven
+workloads (1, 3, 4) and the 16.7M-config sweep (5) are timed once each afterwards and reported
+under "workloads" with configs/s and simulated request-iterations/s.
+
+With N > 1 (launched by torchrun) every rank evaluates a grid of the same size over its own slice
+of an N-times longer hardware axis (weak scaling); the only exchange is an all-gather of each
+rank's top-k candidates before a final merge.
+
+--impl reference times the CPU oracle (the repo's slow, plain restatement of the method) on the
+host cores on the same workload and metric.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+BYTES_SIM = 6 * 8 + 1 + 4          # six fp64 metrics + status + bmax written per config
+BYTES_TOPK = 1 + 8                 # status + key read per config
+BYTES_PARETO = 1 + 8 + 8           # status + two metrics read per config
+SIM_FIELDS = ("latency", "ttft", "tpot", "thr_decode", "cost_per_hr", "cost_per_token", "status", "bmax")
+TRACE_FIELDS = ("latency", "ttft", "ttft_p50", "ttft_p99", "tpot", "thr_decode", "cost_per_hr", "cost_per_token",
+                "status", "bmax", "n_iters", "n_req_iters")
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons through NVML while the timed region runs (read only)."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.stop_flag, self.max_mhz = index, [], set(), False, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {nv.nvmlClocksEventReasonSwPowerCap: "sw_power_cap", nv.nvmlClocksEventReasonHwSlowdown: "hw_slowdown",
+                 nv.nvmlClocksEventReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                 nv.nvmlClocksEventReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                 nv.nvmlClocksEventReasonHwPowerBrakeSlowdown: "hw_power_brake"}
+        while not self.stop_flag:
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def summary(self):
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+def table_bytes(space):
+    return (len(space["models"]) * 40 + len(space["hw"]) * 48 + len(space["fw_f"]) * 80 + len(space["batch"]) * 4 +
+            len(space["tp"]) * 4 + len(space["pairs"]) * 8)
+
+
+# ---------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands
+# ---------------------------------------------------------------------------------------------------
+
+def oracle_step(oracle, w):
+    out = oracle.simulate(w["space"])
+    oracle.select_topk(out, w["constraints"], w["topk"]["key"], w["topk"]["k"])
+    oracle.pareto(out, w["constraints"], "latency", "cost_per_hr")
+    return out
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2412_04788_b200 import inputs
+    w = inputs.workload(2)
+    n = inputs.space_size(w["space"])
+    for _ in range(args.warmup):
+        oracle_step(oracle, w)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(oracle, w)
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    cores = oracle.threads()
+    line = {"impl": "reference", "metric": "configs/sec", "value": value, "unit": "configs/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "C2 closed-form grid, 983040 configs: simulate + top-8 + Pareto"},
+            "cpu_baseline": {"value": value, "unit": "configs/s", "cores": cores, "kind": "oracle",
+                             "sample": f"the whole workload, {args.steps} passes"},
+            "e2e": {"value": value, "unit": "configs/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------------------------------
+
+class ClosedFormPath:
+    """Device buffers and the three calls of one step on a closed-form space."""
+
+    def __init__(self, guide, torch, space_np, cons, key, k):
+        self.guide, self.torch = guide, torch
+        self.sp = guide.Space(space_np)
+        self.n = self.sp.size
+        self.cons, self.key, self.k = cons, key, k
+        self.out = guide.alloc_outputs(self.n, fields=SIM_FIELDS)
+        self.idx = torch.empty(k, dtype=torch.int64, device="cuda")
+        self.val = torch.empty(k, dtype=torch.float64, device="cuda")
+        self.cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+        self.fidx = torch.empty(guide.PARETO_MAX, dtype=torch.int64, device="cuda")
+        self.fcnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+        self.ws_k = torch.empty(guide.guide_select_workspace_bytes(self.sp, k), dtype=torch.uint8, device="cuda")
+        self.ws_p = torch.empty(guide.guide_pareto_workspace_bytes(self.sp), dtype=torch.uint8, device="cuda")
+
+    def simulate(self):
+        self.guide.guide_simulate(self.sp, None, self.out)
+
+    def topk(self, fused=False):
+        self.guide.guide_select_topk(self.sp, None, None if fused else self.out, self.cons, self.key, self.k,
+                                     self.idx, self.val, self.cnt, self.ws_k)
+
+    def pareto(self, fused=False):
+        self.guide.guide_pareto(self.sp, None, None if fused else self.out, self.cons, "latency", "cost_per_hr",
+                                self.fidx, self.fcnt, self.ws_p)
+
+
+def time_call(torch, fn, reps=3, warm=1, flush=None):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(reps):
+        if flush is not None:
+            flush.zero_()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    return min(ts), sorted(ts)[len(ts) // 2]
+
+
+def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full):
+    """Workloads 1, 3, 4, 5, each timed on its own: best of a few launches, CUDA events."""
+    res = {}
+    for k in which:
+        if k in (1, 3, 4):
+            scale = 1.0 if (full or k == 1) else (1 / 8 if k == 3 else 1 / 16)
+            w = inputs.workload(k, scale=scale, trace_scale=1.0)
+            sp, tr = guide.Space(w["space"]), guide.Trace(w["trace"])
+            n = sp.size
+            out = guide.alloc_outputs(n, tr.n, fields=TRACE_FIELDS, per_request=(k != 4))
+            ws = torch.empty(guide.guide_workspace_bytes(sp, tr), dtype=torch.uint8, device="cuda")
+            best, med = time_call(torch, lambda: guide.guide_simulate(sp, tr, out, workspace=ws), reps=2, warm=1)
+            iters = int(out["n_iters"].sum().item())
+            req_iters = int(out["n_req_iters"].sum().item())
+            feasible = int((out["status"] == 0).sum().item())
+            res[f"C{k}"] = {"configs": n, "requests": tr.n, "feasible": feasible, "ms": best,
+                            "configs_per_s": n / best * 1e3, "iters_per_s": iters / best * 1e3,
+                            "request_iters_per_s": req_iters / best * 1e3, "request_iters": req_iters,
+                            "hardware_axis_fraction": scale, "kernel_launches": 1}
+            del out, ws
+        elif k == 5:
+            w = inputs.workload(5)
+            p = ClosedFormPath(guide, torch, w["space"], w["constraints"], w["topk"]["key"], w["topk"]["k"])
+            n = p.n
+            t_sim = time_call(torch, p.simulate, flush=flush)[0]
+            t_kf = time_call(torch, lambda: p.topk(True), flush=flush)[0]
+            t_pf = time_call(torch, lambda: p.pareto(True), flush=flush)[0]
+            t_km = time_call(torch, lambda: p.topk(False), flush=flush)[0]
+            t_pm = time_call(torch, lambda: p.pareto(False), flush=flush)[0]
+            res["C5"] = {"configs": n, "front": int(p.fcnt.item()), "found": int(p.cnt.item()),
+                         "fused_ms": {"topk": t_kf, "pareto": t_pf}, "fused_configs_per_s": n / (t_kf + t_pf) * 1e3,
+                         "materialised_ms": {"simulate": t_sim, "topk": t_km, "pareto": t_pm},
+                         "materialised_configs_per_s": n / (t_sim + t_km + t_pm) * 1e3,
+                         "simulate_write_gbs": BYTES_SIM * n / t_sim / 1e6,
+                         "simulate_frac_of_hbm": BYTES_SIM * n / t_sim / 1e6 / hbm_peak, "kernel_launches": 5}
+            del p
+        torch.cuda.empty_cache()
+    return res
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2412_04788_b200 import build, guide, inputs, sharding
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if rank == 0:
+        build.build()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device: the library has no CPU fallback"
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    guide.lib()
+
+    hbm_peak, peak_kind = measured_peaks()
+    # workload 2; with N ranks the hardware axis is N times longer and each rank takes one slice
+    w = inputs.workload(2, scale=float(world))
+    global_space = w["space"]
+    local_space, hw_off = sharding.shard_space(global_space, rank, world) if world > 1 else (global_space, 0)
+    k, key, cons = w["topk"]["k"], w["topk"]["key"], w["constraints"]
+    path = ClosedFormPath(guide, torch, local_space, cons, key, k)
+    n_local = path.n
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+
+    def exchange():
+        """all-gather of the k local candidates, then the same kernel merges them"""
+        gidx = sharding.local_to_global(path.idx, local_space, global_space, hw_off)
+        all_idx = sharding.all_gather_concat(gidx)
+        all_val = sharding.all_gather_concat(path.val)
+        order = sharding.order_for_merge(all_idx)
+        all_idx, all_val = all_idx[order], all_val[order]
+        m = all_idx.numel()
+        gathered = {"status": (all_idx < 0).to(torch.uint8), "cost_per_token": all_val.contiguous()}
+        guide.guide_select_topk(path.sp, None, gathered, {}, key, k, path.idx, path.val, path.cnt, path.ws_k, count=m)
+        return all_idx
+
+    def step(events=None):
+        if events:
+            events[0].record()
+        path.simulate()
+        if events:
+            events[1].record()
+        path.topk()
+        if events:
+            events[2].record()
+        path.pareto()
+        if world > 1:
+            exchange()
+        if events:
+            events[3].record()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    wall0 = time.perf_counter()
+    for i in range(args.steps):
+        flush.zero_()                     # outputs (52 MB) fit in L2: evict them between steps
+        step(evs[i])
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - wall0
+    sampler.stop_flag = True
+    sampler.join()
+    t_sim = sum(e[0].elapsed_time(e[1]) for e in evs)
+    t_topk = sum(e[1].elapsed_time(e[2]) for e in evs)
+    t_par = sum(e[2].elapsed_time(e[3]) for e in evs)
+    total_ms = t_sim + t_topk + t_par
+    if world > 1:
+        tt = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+        dist.barrier()
+    n_total = n_local * world
+    value = n_total * args.steps / (total_ms * 1e-3)
+
+    # ---- end to end through the C ABI with host buffers: build the space from host arrays, run the
+    # step, bring every output back to pinned host memory ----
+    host = {f: torch.empty_like(t, device="cpu").pin_memory() for f, t in path.out.items()}
+    host_idx, host_val = torch.empty(k, dtype=torch.int64).pin_memory(), torch.empty(k, dtype=torch.float64).pin_memory()
+    host_front = torch.empty(guide.PARETO_MAX, dtype=torch.int64).pin_memory()
+    e2e_steps = min(args.steps, 20)
+
+    def e2e_step():
+        sp = guide.Space(local_space)                      # host tables -> validated -> uploaded on first use
+        guide.guide_simulate(sp, None, path.out)
+        guide.guide_select_topk(sp, None, path.out, cons, key, k, path.idx, path.val, path.cnt, path.ws_k)
+        guide.guide_pareto(sp, None, path.out, cons, "latency", "cost_per_hr", path.fidx, path.fcnt, path.ws_p)
+        for f, t in path.out.items():
+            host[f].copy_(t, non_blocking=True)
+        host_idx.copy_(path.idx, non_blocking=True)
+        host_val.copy_(path.val, non_blocking=True)
+        host_front.copy_(path.fidx, non_blocking=True)
+        torch.cuda.synchronize()
+        sp.close()
+
+    for _ in range(3):
+        e2e_step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e2e_dt = time.perf_counter() - t0
+    if world > 1:
+        tt = torch.tensor([e2e_dt], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_dt = float(tt.item())
+    e2e_value = n_total * e2e_steps / e2e_dt
+    d2h = BYTES_SIM * n_local + k * 16 + guide.PARETO_MAX * 8
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel of the step ----
+    per = {"guide_simulate (k_closed_form_tiled)": (t_sim / args.steps, BYTES_SIM),
+           "guide_select_topk (k_topk)": (t_topk / args.steps, BYTES_TOPK),
+           "guide_pareto (k_pareto)": (t_par / args.steps, BYTES_PARETO)}
+    dom = max(per, key=lambda name: per[name][0])
+    dom_ms, dom_bytes = per[dom]
+    achieved = dom_bytes * n_local / (dom_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+                "frac": achieved / hbm_peak, "traffic": None, "peak_kind": f"of {peak_kind}",
+                "bytes_per_config": dom_bytes,
+                "per_kernel_ms": {name: v[0] for name, v in per.items()},
+                "per_kernel_gbs": {name: v[1] * n_local / (v[0] * 1e-3) / 1e9 for name, v in per.items()}}
+
+    # ---- the oracle on the host cores, same workload ----
+    cpu = None
+    if world == 1 and not args.no_cpu:
+        import oracle
+        oracle_step(oracle, w)
+        reps, t0 = 0, time.perf_counter()
+        while reps < 5 or time.perf_counter() - t0 < 2.0:
+            oracle_step(oracle, w)
+            reps += 1
+        dt = time.perf_counter() - t0
+        cpu = {"value": n_local * reps / dt, "unit": "configs/s", "cores": oracle.threads(), "kind": "oracle",
+               "sample": f"the whole 983040-config workload (simulate + top-{k} + Pareto), {reps} passes"}
+
+    extras = {}
+    if world == 1 and args.extras:
+        which = [int(x) for x in args.extras.split(",") if x]
+        extras = extra_workloads(guide, torch, inputs, which, flush, hbm_peak, args.full)
+
+    launches_per_step = 3 + (1 if world > 1 else 0)
+    line = {"metric": "configs/sec", "value": value, "unit": "configs/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "C2 closed-form grid: 8 models x 16 hw x 3 fw x 10 batch x 4 TP x 64 length pairs "
+                                   f"= {n_local} configs per GPU; simulate + top-{k} by cost/token + Pareto(latency, $/h)",
+                       "l2": "256 MB buffer written between timed steps", "timing": "CUDA events per step, summed"},
+            "clocks": sampler.summary(),
+            "e2e": {"value": e2e_value, "unit": "configs/s", "h2d_bytes_per_step": table_bytes(local_space),
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu, "workloads": extras,
+            "wall_s_timed_region": wall}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--extras", default="1,3,4,5", help="other workloads to time after the main loop ('' = none)")
+    ap.add_argument("--full", action="store_true", help="run workloads 3 and 4 on their whole hardware axis")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
