@@ -232,6 +232,38 @@ int guide_pareto(const guide_space *space, const guide_trace *trace, const guide
                  uint64_t *idx_out_dev, uint32_t cap, uint32_t *count_out_dev,
                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* Top-k over materialised metrics for callers that must not allocate device memory.  (The paper
+ * has no counterpart: this is a packaging variant of guide_select_topk, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a serving loop whose memory
+ * pool was sized up front and must not grow, in a plug-in whose host application owns every
+ * allocation, or after start-up in a process that has promised a fixed device footprint.  Such a
+ * caller cannot supply the workspace guide_select_topk asks for.  Here the per-block partial
+ * results live in a fixed array compiled into the library (about 257 KB of device memory on every
+ * GPU that loads the library, held until the process exits), and the call makes no cudaMalloc,
+ * cudaFree or other allocating call.
+ *
+ * It selects among count configs whose metrics were written by guide_simulate: entry j of each
+ * array belongs to config first + j.  outputs: host struct of DEVICE pointers; status, the key's
+ * array and the array of every enabled bound must be non-NULL.  idx_out_dev[k], key_out_dev[k],
+ * count_out_dev[1]: device, caller-owned.  Results, order, tie-break and unused slots are exactly
+ * those of guide_select_topk.
+ *
+ * Limits: 1 <= k <= GUIDE_NOALLOC_TOPK_MAX and 1 <= count <= GUIDE_NOALLOC_COUNT_MAX; anything
+ * larger returns GUIDE_ERR_UNSUPPORTED with a message naming the limit.
+ *
+ * The first call on each device looks up the array's device address (no allocation, but a
+ * one-time set-up step): make that first call before starting any stream capture.  All calls on a
+ * device share the one array, which keeps the previous call's contents; the call clears the part
+ * that must start at zero on the given stream.  Two calls whose kernels could overlap on the GPU
+ * (different streams, or different threads, without ordering between them) race on it: order them. */
+#define GUIDE_NOALLOC_TOPK_MAX 64u
+#define GUIDE_NOALLOC_COUNT_MAX (1ull << 40)
+int guide_select_topk_noalloc(const guide_outputs *outputs, uint64_t first, uint64_t count,
+                              const guide_constraints *cons, int key, uint32_t k,
+                              uint64_t *idx_out_dev, double *key_out_dev, uint32_t *count_out_dev,
+                              void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

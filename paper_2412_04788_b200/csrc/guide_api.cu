@@ -497,4 +497,33 @@ int guide_pareto(const guide_space *space_c, const guide_trace *trace, const gui
                          (u64 *)idx_out, cap, count_out, ws, (cudaStream_t)stream);
 }
 
+int guide_select_topk_noalloc(const guide_outputs *outputs, uint64_t first, uint64_t count,
+                              const guide_constraints *cons, int key, uint32_t k, uint64_t *idx_out,
+                              double *key_out, uint32_t *count_out, void *stream) {
+    if (!outputs || !cons) return fail(GUIDE_ERR_INVALID, "outputs and constraints are required");
+    if (k == 0) return fail(GUIDE_ERR_INVALID, "k must be at least 1");
+    if (k > GUIDE_NOALLOC_TOPK_MAX)
+        return fail(GUIDE_ERR_UNSUPPORTED, "k = %u is above GUIDE_NOALLOC_TOPK_MAX (%u): the built-in scratch array cannot hold it; "
+                    "use guide_select_topk with a workspace", k, GUIDE_NOALLOC_TOPK_MAX);
+    if (count == 0 || count > GUIDE_NOALLOC_COUNT_MAX)
+        return fail(GUIDE_ERR_UNSUPPORTED, "count must be in 1..%llu for the no-allocation variant", (unsigned long long)GUIDE_NOALLOC_COUNT_MAX);
+    if (first > UINT64_MAX - count) return fail(GUIDE_ERR_INVALID, "first + count overflows");
+    if (!idx_out || !key_out || !count_out) return fail(GUIDE_ERR_INVALID, "an output pointer is NULL");
+    if (key < GUIDE_LATENCY || key > GUIDE_COST_PER_TOKEN) return fail(GUIDE_ERR_INVALID, "unknown metric %d", key);
+    if (cons->ttft_stat < GUIDE_STAT_MEAN || cons->ttft_stat > GUIDE_STAT_P99) return fail(GUIDE_ERR_INVALID, "unknown ttft_stat");
+    if (std::isnan(cons->max_ttft) || std::isnan(cons->max_latency) || std::isnan(cons->max_cost_per_hr) ||
+        std::isnan(cons->min_throughput))
+        return fail(GUIDE_ERR_INVALID, "a constraint is NaN");
+    if (!outputs->status) return fail(GUIDE_ERR_INVALID, "outputs->status is required");
+    if (!metric_array(*outputs, key)) return fail(GUIDE_ERR_INVALID, "the array of metric %d is NULL", key);
+    const double *ttft = cons->ttft_stat == GUIDE_STAT_MEAN ? outputs->ttft
+                         : cons->ttft_stat == GUIDE_STAT_P50 ? outputs->ttft_p50 : outputs->ttft_p99;
+    if (cons->max_ttft < INFINITY && !ttft) return fail(GUIDE_ERR_INVALID, "max_ttft is set but its array is NULL");
+    if (cons->max_latency < INFINITY && !outputs->latency) return fail(GUIDE_ERR_INVALID, "max_latency is set but latency is NULL");
+    if (cons->max_cost_per_hr < INFINITY && !outputs->cost_per_hr) return fail(GUIDE_ERR_INVALID, "max_cost_per_hr is set but cost_per_hr is NULL");
+    if (cons->min_throughput > 0.0 && !outputs->thr_decode) return fail(GUIDE_ERR_INVALID, "min_throughput is set but thr_decode is NULL");
+    Range r{first, count};
+    return launch_topk_noalloc(r, *outputs, *cons, key, k, (u64 *)idx_out, key_out, count_out, (cudaStream_t)stream);
+}
+
 }  // extern "C"

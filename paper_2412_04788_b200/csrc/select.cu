@@ -452,4 +452,51 @@ int launch_pareto(const DSpace &s, Range r, const guide_outputs *mat, int time_m
     return run_pareto(src, r, idx_out, cap, count_out, ws, st);
 }
 
+// ---- top-k over materialised metrics with library-owned scratch ----------------------------------
+//
+// Same kernel as launch_topk, but the per-block partial results live in a fixed device array that
+// is part of the library image instead of a caller-supplied workspace, for callers that are not
+// allowed to allocate device memory.  The array bounds k and the grid; every call reuses it.
+
+static constexpr u32 NOALLOC_BLOCKS = 256;                     // grid cap of this variant
+static constexpr size_t NOALLOC_SCRATCH_BYTES = 256 + (size_t)NOALLOC_BLOCKS * GUIDE_NOALLOC_TOPK_MAX * sizeof(KI);
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
+
+// Device address of the scratch array on the current device.  The array's name is only a handle
+// on the host, so the address is asked for once per device and cached.
+static int noalloc_scratch_address(unsigned char **out) {
+    static std::mutex mu;
+    static unsigned char *cached[64] = {};
+    int dev = 0;
+    GUIDE_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return fail(GUIDE_ERR_UNSUPPORTED, "device ordinal %d is outside 0..63", dev);
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cached[dev]) {
+        void *p = nullptr;
+        GUIDE_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        if (!p) return fail(GUIDE_ERR_CUDA, "the scratch array has no device address");
+        cached[dev] = (unsigned char *)p;
+    }
+    *out = cached[dev];
+    return GUIDE_OK;
+}
+
+int launch_topk_noalloc(Range r, const guide_outputs &mat, const guide_constraints &c, int key, u32 k,
+                        u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st) {
+    unsigned char *scratch = nullptr;
+    const int rc = noalloc_scratch_address(&scratch);
+    if (rc) return rc;
+    MatSource src{mat, make_cons(c), key, -1};
+    const u32 cap = topk_cap(k);
+    const u32 grid = std::min<u32>(grid_for(r.count, 4), NOALLOC_BLOCKS);
+    // the array still holds the previous call's ticket and candidates: the ticket must restart at 0,
+    // the candidate slots are all rewritten by the blocks of this launch before they are read
+    GUIDE_CUDA(cudaMemsetAsync(scratch, 0, 256, st));
+    k_topk<MatSource><<<grid, SEL_THREADS, cap * sizeof(KI), st>>>(src, r, k, cap, (u32 *)scratch, (KI *)(scratch + 256),
+                                                                   key == GUIDE_THROUGHPUT, idx_out, key_out, count_out);
+    GUIDE_CUDA(cudaGetLastError());
+    return GUIDE_OK;
+}
+
 }  // namespace guide

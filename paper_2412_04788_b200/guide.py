@@ -23,13 +23,15 @@ METRICS = {"latency": 0, "ttft": 1, "ttft_p99": 2, "tpot": 3, "throughput": 4, "
            "cost_per_token": 6}
 TTFT_STATS = {"mean": 0, "p50": 1, "p99": 2}
 TOPK_MAX, PARETO_MAX, TRACE_MAX_BATCH = 1024, 2048, 256
+NOALLOC_TOPK_MAX = 64
 
 F64_OUTPUTS = ("latency", "ttft", "ttft_p50", "ttft_p99", "tpot", "thr_decode", "cost_per_hr", "cost_per_token")
 ALL_OUTPUTS = F64_OUTPUTS + ("status", "bmax", "n_iters", "n_req_iters")
 
 EXPORTS = ("guide_last_error", "guide_space_create", "guide_space_destroy", "guide_space_size", "guide_space_decode",
            "guide_trace_load", "guide_trace_destroy", "guide_trace_size", "guide_workspace_bytes", "guide_simulate",
-           "guide_select_workspace_bytes", "guide_pareto_workspace_bytes", "guide_select_topk", "guide_pareto")
+           "guide_select_workspace_bytes", "guide_pareto_workspace_bytes", "guide_select_topk", "guide_pareto",
+           "guide_select_topk_noalloc")
 
 
 class GuideError(RuntimeError):
@@ -117,6 +119,8 @@ def lib():
                                         C.c_void_p, C.c_size_t, C.c_void_p]
         L.guide_pareto.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Outputs), C.POINTER(SimOpts), C.POINTER(Constraints),
                                    C.c_int, C.c_int, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.guide_select_topk_noalloc.argtypes = [C.POINTER(Outputs), C.c_uint64, C.c_uint64, C.POINTER(Constraints), C.c_int,
+                                                C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -276,3 +280,16 @@ def guide_pareto(space: Space, trace: Trace | None, out: dict | None, cons: dict
                               C.byref(opts), C.byref(cs), METRICS[x], METRICS[y], _ptr(idx_out), idx_out.numel(),
                               _ptr(count_out), _ptr(workspace), workspace.numel() if workspace is not None else 0,
                               _stream_ptr(stream)))
+
+
+def guide_select_topk_noalloc(out: dict, cons: dict | None, key: str, k: int, idx_out, key_out, count_out,
+                              first=0, count=0, stream=None):
+    """Top-k over materialised metrics without any workspace: for callers that may not allocate
+    device memory.  The partial results go to a fixed array inside the library (k <= 64); calls
+    that could overlap on the GPU must be ordered by the caller.  `out` holds the metric arrays
+    written by guide_simulate; `count` defaults to the length of out["status"]."""
+    o = _outputs_struct(out)
+    cs = _cons(cons)
+    n = count or out["status"].numel()
+    _check(lib().guide_select_topk_noalloc(C.byref(o), first, n, C.byref(cs), METRICS[key], k, _ptr(idx_out),
+                                           _ptr(key_out), _ptr(count_out), _stream_ptr(stream)))
