@@ -182,12 +182,14 @@ def time_call(torch, fn, reps=3, warm=1, flush=None):
     return min(ts), sorted(ts)[len(ts) // 2]
 
 
-def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full):
+def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full, fraction=None):
     """Workloads 1, 3, 4, 5, each timed on its own: best of a few launches, CUDA events."""
     res = {}
     for k in which:
         if k in (1, 3, 4):
             scale = 1.0 if (full or k == 1) else (1 / 8 if k == 3 else 1 / 16)
+            if fraction and k != 1:
+                scale = fraction
             w = inputs.workload(k, scale=scale, trace_scale=1.0)
             sp, tr = guide.Space(w["space"]), guide.Trace(w["trace"])
             n = sp.size
@@ -375,7 +377,7 @@ def run_ours(args):
     extras = {}
     if world == 1 and args.extras:
         which = [int(x) for x in args.extras.split(",") if x]
-        extras = extra_workloads(guide, torch, inputs, which, flush, hbm_peak, args.full)
+        extras = extra_workloads(guide, torch, inputs, which, flush, hbm_peak, args.full, args.trace_fraction)
 
     launches_per_step = 3 + (1 if world > 1 else 0)
     line = {"metric": "configs/sec", "value": value, "unit": "configs/s", "n_gpus": world, "steps": args.steps,
@@ -404,6 +406,8 @@ def main():
     ap.add_argument("--extras", default="1,3,4,5", help="other workloads to time after the main loop ('' = none)")
     ap.add_argument("--full", action="store_true", help="run workloads 3 and 4 on their whole hardware axis")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
+    ap.add_argument("--trace-fraction", type=float, default=None,
+                    help="fraction of the hardware axis of workloads 3 and 4 (small cases for profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -2,13 +2,26 @@
 // prompt-priority scheduling and fixed-granularity paged KV of the vLLM-like framework model,
 // Sec. 2.3.2 / 2.4.1 / 2.4.2).
 //
-// A warp owns one config at a time and pulls the next one from a global counter, so configs
-// whose schedules are long do not hold back a whole block.  The clock, counters and the
-// iteration time are warp-uniform; the resident requests live in per-warp shared-memory slots,
-// kept in ascending request order, which the 32 lanes scan together.  Per-request results that
-// must outlive residency (tokens generated so far, first-token time, time per output token) sit
-// in a per-warp slice of the workspace.  The request trace itself is the same for every config
-// and is read through the read-only path, so it stays cache resident.
+// A warp owns one config at a time and pulls the next one from a global counter, smallest
+// max-batch first (those schedules have the most iterations), so long schedules start early and
+// do not hold back a whole block.  The clock, counters and the iteration time are warp-uniform.
+//
+// Between events a decode iteration costs O(1): nothing per request is touched.
+//   - Resident requests live in per-warp shared-memory slots in ascending request order and store
+//     invariants, not running values: with D = decode iterations done so far, a slot keeps
+//     base = cache - D and fin = D + tokens still to generate, both constant while it is resident.
+//   - The number of requests whose last KV block is full comes from a histogram of
+//     (cache - D) mod block; the next completion is a countdown; the summed context grows by the
+//     running count each step.
+//   - The attention tasks are re-evaluated every iteration from the summed context; everything
+//     that depends only on the running count is cached until that count changes.  When every
+//     integer FLOP/byte count of the config stays below 2^53 the counts are carried as doubles
+//     (products and sums of integers below 2^53 are exact in binary64), which removes the
+//     integer-to-double conversions from the loop without changing a bit.
+// Events (admission, prompt pass, completion, eviction) scan the slots with all 32 lanes.
+// Per-request results that outlive residency (tokens generated so far, first-token time, time per
+// output token) sit in a per-warp slice of the workspace.  The request trace is the same for every
+// config and is read through the read-only path, so it stays cache resident.
 #include "guide_internal.cuh"
 
 namespace guide {
@@ -17,8 +30,10 @@ static constexpr u32 SIM_WARPS_PER_BLOCK = 8;
 static constexpr u32 SIM_THREADS = SIM_WARPS_PER_BLOCK * 32;
 static constexpr u32 SIM_MAX_WARPS = 6144;        // workspace is sized for this many resident warps
 static constexpr u32 SLOTS = GUIDE_TRACE_MAX_BATCH;
-static constexpr u32 F_NEEDS_PREFILL = 0x80000000u, F_FIRST = 0x40000000u, REM_MASK = 0x3FFFFFFFu;
+static constexpr u32 HIST = 64;                   // block sizes up to this use the phase histogram
+static constexpr u32 M_PHASE = 0x3F, M_FIRST = 0x40, M_NEEDS_PREFILL = 0x80;
 static constexpr u32 GEN_DONE = 0x80000000u;
+static constexpr u32 NO_COMPLETION = 0xFFFFFFFFu;
 
 static u32 pow2_at_least(u32 v) { u32 p = 1; while (p < v) p <<= 1; return p; }
 
@@ -34,23 +49,39 @@ __device__ __forceinline__ u64 warp_sum(u64 v) {
     for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
     return v;
 }
+__device__ __forceinline__ u32 warp_min(u32 v) {
+    for (int d = 16; d > 0; d >>= 1) v = min(v, __shfl_xor_sync(0xFFFFFFFFu, v, d));
+    return v;
+}
 __device__ __forceinline__ u32 ceil_div32(u32 a, u32 b) { return (a + b - 1) / b; }
 
-// time of a decode iteration's fixed part, cached while the number of running sequences stays
-struct DecodeCache {
-    u32 n;              // running count the cache was built for (0 = empty)
-    double s_fix, s_comm, t_head;
-    u64 THa;            // n * H * a_b
+struct SlotArrays {
+    u32 req[SLOTS];     // request index
+    u32 base[SLOTS];    // resident: cache - D (mod 2^32); waiting for its prompt pass: prompt + recompute tokens
+    u32 fin[SLOTS];     // resident: D at which it completes; waiting for its prompt pass: tokens still to emit
+    u32 hist[HIST];     // residents per (cache - D) mod block
+    unsigned char meta[SLOTS];   // phase (6 bits) | first-ever prompt pass | waiting for its prompt pass
 };
 
+// The work order visits the batch axis slowest when the whole space is simulated, so configs with
+// a small max batch (the long schedules) are started first.
+__device__ __forceinline__ u64 work_to_index(const DSpace &s, u64 w, bool reorder) {
+    if (!reorder) return w;
+    const u64 tl = (u64)s.n_t * s.n_l;
+    const u64 per_b = (u64)s.n_m * s.n_h * s.n_f * tl;
+    const u64 b = w / per_b, rest = w % per_b;
+    const u64 mhf = rest / tl, x = rest % tl;
+    return (mhf * s.n_b + b) * tl + x;
+}
+
 template <int TIME_SUM>
-__global__ void __launch_bounds__(SIM_THREADS)
+__global__ void __launch_bounds__(SIM_THREADS, 2)
 k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide_outputs o, u32 *counter,
-            unsigned char *scratch, size_t per_warp, u32 gen_bytes, u32 first_bytes) {
-    __shared__ u32 sh_slots[SIM_WARPS_PER_BLOCK][3][SLOTS];
+            unsigned char *scratch, size_t per_warp, u32 gen_bytes, u32 first_bytes, int reorder) {
+    __shared__ SlotArrays sh[SIM_WARPS_PER_BLOCK];
     const u32 lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const u32 warp_global = blockIdx.x * SIM_WARPS_PER_BLOCK + wib;
-    u32 *s_req = sh_slots[wib][0], *s_cache = sh_slots[wib][1], *s_rem = sh_slots[wib][2];
+    SlotArrays &sl = sh[wib];
     unsigned char *mine = scratch + (size_t)warp_global * per_warp;
     u32 *gen = (u32 *)mine;
     double *first = (double *)(mine + gen_bytes);
@@ -60,11 +91,13 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
     const u32 lt_mask = (1u << lane) - 1;
 
     for (;;) {
-        u64 j = 0;
-        if (lane == 0) j = atomicAdd(counter, 1u);
-        j = __shfl_sync(0xFFFFFFFFu, j, 0);
-        if (j >= r.count) break;
-        const Cfg c = decode_index(s, r.first + j);
+        u64 w = 0;
+        if (lane == 0) w = atomicAdd(counter, 1u);
+        w = __shfl_sync(0xFFFFFFFFu, w, 0);
+        if (w >= r.count) break;
+        const u64 idx = reorder ? work_to_index(s, w, true) : r.first + w;
+        const u64 j = idx - r.first;
+        const Cfg c = decode_index(s, idx);
         const DModel m = s.models[c.m];
         const DRate rt = s.rates[c.h * s.n_f + c.f];
         const u32 t = s.tp[c.t], b = s.batch[c.b];
@@ -73,6 +106,8 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         const MemInfo mi = mem_info(m, t);
         const u32 tt = tp_model ? 1u : t;
         const double lf = log2_rule_factor(t, tp_model), Nd = (double)m.N;
+        const double inv_tt = 1.0 / (double)tt;
+        const double icA = rt.inv_c[CLS_ATTN], imA = rt.inv_m[CLS_ATTN];
 
         // ---- what fits (Sec. 3.2 Step 1) ----
         const u64 blocks_total = rt.usable > mi.w_gpu ? floor_div(rt.usable - mi.w_gpu, (u64)blk * mi.kv_tok) : 0;
@@ -84,173 +119,239 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         if ((m.nh & (t - 1)) != 0 || (m.nkv & (t - 1)) != 0) st |= GUIDE_ST_HEADS;
         const u32 fit = clamp_u32(blocks_total / worst);
 
-        double clock = 0.0, dec_time = 0.0;
+        // ---- constants of the per-iteration attention terms ----
+        // Largest summed context this config can see: every resident at its full length plus one.
+        const u64 ctx_max = (u64)b * ((u64)longest + 1);
+        const u64 lim53 = 1ull << 53;
+        const u64 xw = rt.flash ? 0ull : (u64)m.nh * m.ab;                 // score-matrix bytes per unit of A
+        const bool exact53 = 2 * (u64)m.H * ctx_max < lim53 && 5 * (u64)m.nh * ctx_max < lim53 &&
+                             (u64)b * m.H * m.ab + ctx_max * ((u64)m.Dkv * m.kvb + xw) < lim53 && 2 * xw * ctx_max < lim53;
+        const double c_f9 = (double)(2 * (u64)m.H) * inv_tt;               // F9  = ctx * 2H / t
+        const double c_kv = (double)((u64)m.Dkv * m.kvb) * inv_tt;         // KV read per context token / t
+        const double c_x = (double)xw * inv_tt;                            // score bytes per context token / t
+        const double c_f10 = (double)(5 * (u64)m.nh) * inv_tt;             // F10 = ctx * 5 n_h / t
+        const double c_b10 = (double)(2 * xw) * inv_tt;                    // B10 = ctx * 2 n_h a_b / t (0 with flash)
+
+        double clock = 0.0, dec_time = 0.0, csum_d = 0.0;   // csum_d mirrors csum when exact53
         u64 dec_tok = 0, n_iters = 0, n_req_iters = 0, free_blocks = blocks_total, csum = 0;
         u32 next = 0, high_water = 0, nrun = 0, n_new = 0;
+        u32 D = 0, Dmod = 0, min_rem = NO_COMPLETION;
+        const bool use_hist = blk > 1 && blk <= HIST;
         const u64 max_iters = max_iters_opt ? max_iters_opt : 64 * (tr.sum_out + (u64)tr.n_zero * Lout) + 4 * (u64)n;
-        DecodeCache dc;
-        dc.n = 0;
+        // cached while the running count stays the same
+        u32 dc_n = 0;
+        double dc_fix = 0.0, dc_comm = 0.0, dc_head = 0.0, dc_tha = 0.0, dc_nd = 0.0;
+        u64 dc_tha_i = 0;
+        // the head of the waiting queue: its arrival time and the blocks it needs
+        double arr_next = 0.0;
+        u32 need_next = 0;
+        auto refresh_head = [&]() {
+            while (next < high_water && (gen[next] & GEN_DONE)) next++;
+            if (next < n) {
+                arr_next = __ldg(tr.arrival + next);
+                const u32 g = next < high_water ? gen[next] : 0u;       // tokens kept from before an eviction
+                const u32 in = __ldg(tr.in_len + next);
+                need_next = ceil_div32((in ? in : Lin) + g, blk);
+            } else {
+                arr_next = inf; need_next = 0;
+            }
+        };
+        if (!st) {
+            for (u32 i = lane; i < HIST; i += 32) sl.hist[i] = 0;
+            refresh_head();
+            __syncwarp();
+        }
 
         while (!st) {
             // ---- 1. admit in arrival order, no overtaking ----
-            for (;;) {
-                while (next < high_water && (gen[next] & GEN_DONE)) next++;
-                if (next >= n || nrun >= b) break;
-                if (!(__ldg(tr.arrival + next) <= clock)) break;
-                const u32 g = next < high_water ? gen[next] : 0u;     // tokens kept from before an eviction
-                u32 in = __ldg(tr.in_len + next), out = __ldg(tr.out_len + next);
-                if (in == 0) { in = Lin; out = Lout; }
-                const u32 q = in + g;                                  // prompt + tokens to recompute
-                const u32 need = ceil_div32(q, blk);
-                if (need > free_blocks) break;
-                free_blocks -= need;
-                if (lane == 0) {
-                    s_req[nrun] = next;
-                    s_cache[nrun] = q;
-                    s_rem[nrun] = (out - g) | F_NEEDS_PREFILL | (g == 0 ? F_FIRST : 0u);
-                }
-                nrun++; n_new++; next++;
-                if (next > high_water) high_water = next;
+            if (nrun < b && arr_next <= clock && need_next <= free_blocks) {
+                do {
+                    const u32 g = next < high_water ? gen[next] : 0u;
+                    u32 in = __ldg(tr.in_len + next), out = __ldg(tr.out_len + next);
+                    if (in == 0) { in = Lin; out = Lout; }
+                    free_blocks -= need_next;
+                    if (lane == 0) {
+                        sl.req[nrun] = next;
+                        sl.base[nrun] = in + g;                           // prompt + tokens to recompute
+                        sl.fin[nrun] = out - g;
+                        sl.meta[nrun] = (unsigned char)(M_NEEDS_PREFILL | (g == 0 ? M_FIRST : 0u));
+                    }
+                    nrun++; n_new++; next++;
+                    if (next > high_water) high_water = next;
+                    refresh_head();
+                } while (nrun < b && arr_next <= clock && need_next <= free_blocks);
+                __syncwarp();
             }
-            __syncwarp();
             // ---- 2. nothing to run: finished, or jump to the next arrival ----
             if (nrun == 0) {
                 if (next >= n) break;
-                const double a = __ldg(tr.arrival + next);
-                if (a > clock) { clock = a; continue; }
+                if (arr_next > clock) { clock = arr_next; continue; }
                 st |= GUIDE_ST_ITER;                                   // cannot happen when each request fits alone
                 break;
             }
             if (n_iters >= max_iters) { st |= GUIDE_ST_ITER; break; }
             // ---- 3. build the iteration: prompts first, everything else stalls ----
             double t_iter;
-            u32 participants;
-            bool any_done = false;
+            bool any_done;
             if (n_new > 0) {
                 u64 T = 0, A = 0;
                 for (u32 base = 0; base < nrun; base += 32) {
                     const u32 k = base + lane;
-                    if (k < nrun && (s_rem[k] & F_NEEDS_PREFILL)) {
-                        const u64 q = s_cache[k];
+                    if (k < nrun && (sl.meta[k] & M_NEEDS_PREFILL)) {
+                        const u64 q = sl.base[k];
                         T += q; A += q * q;
                     }
                 }
                 T = warp_sum(T); A = warp_sum(A);
-                TaskTab kt;
-                build_fixed_tasks(m, tt, T, n_new, 1, kt);
-                build_attn_tasks(m, tt, T, A, T, kt);
-                t_iter = eval_phase<TIME_SUM>(kt, rt, Nd, lf);
+                {
+                    TaskTab kt;
+                    build_fixed_tasks(m, tt, T, n_new, 1, kt);
+                    build_attn_tasks(m, tt, T, A, T, kt);
+                    t_iter = eval_phase<TIME_SUM>(kt, rt, Nd, lf);
+                }
                 const double after = clock + t_iter;
+                u32 local_min = NO_COMPLETION;
                 for (u32 base = 0; base < nrun; base += 32) {
                     const u32 k = base + lane;
                     if (k < nrun) {
-                        const u32 rem = s_rem[k];
-                        if (rem & F_NEEDS_PREFILL) {
-                            if (rem & F_FIRST) first[s_req[k]] = after;    // first token of this request
-                            const u32 left = (rem & REM_MASK) - 1;
-                            s_rem[k] = left;
-                            any_done |= left == 0;
+                        const u32 mt = sl.meta[k];
+                        if (mt & M_NEEDS_PREFILL) {
+                            if (mt & M_FIRST) first[sl.req[k]] = after;    // first token of this request
+                            const u32 q = sl.base[k], left = sl.fin[k] - 1;
+                            u32 ph = 0;
+                            if (use_hist) {
+                                ph = (q % blk + blk - Dmod) % blk;          // (cache - D) mod block
+                                atomicAdd(&sl.hist[ph], 1u);
+                            }
+                            sl.base[k] = q - D;
+                            sl.fin[k] = D + left;
+                            sl.meta[k] = (unsigned char)ph;
+                            local_min = min(local_min, left);
                         }
                     }
                 }
+                __syncwarp();
+                min_rem = min(min_rem, warp_min(local_min));
+                any_done = min_rem == 0;
                 csum += T;
-                participants = n_new;
+                csum_d = (double)(long long)csum;
+                n_req_iters += n_new;
                 n_new = 0;
             } else {
                 // every sequence whose last block is full needs one more block
-                u32 needed = 0;
-                for (u32 base = 0; base < nrun; base += 32) {
-                    const u32 k = base + lane;
-                    needed += __popc(__ballot_sync(0xFFFFFFFFu, k < nrun && s_cache[k] % blk == 0));
+                u32 needed;
+                if (blk == 1) needed = nrun;
+                else if (use_hist) needed = sl.hist[Dmod == 0 ? 0 : blk - Dmod];
+                else {
+                    needed = 0;
+                    for (u32 base = 0; base < nrun; base += 32) {
+                        const u32 k = base + lane;
+                        needed += __popc(__ballot_sync(0xFFFFFFFFu, k < nrun && (sl.base[k] + D) % blk == 0));
+                    }
                 }
                 if (needed > free_blocks) {
                     while (needed > free_blocks) {                     // evict the youngest, recompute later
                         const u32 v = nrun - 1;
-                        const u32 cv = s_cache[v], rq = s_req[v], rem = s_rem[v] & REM_MASK;
+                        const u32 cv = sl.base[v] + D, rq = sl.req[v], rem = sl.fin[v] - D, ph = sl.meta[v] & M_PHASE;
                         free_blocks += ceil_div32(cv, blk);
                         if (cv % blk == 0) needed--;
                         csum -= cv;
-                        u32 out = __ldg(tr.in_len + rq) ? __ldg(tr.out_len + rq) : Lout;
-                        if (lane == 0) gen[rq] = out - rem;
+                        const u32 out = __ldg(tr.in_len + rq) ? __ldg(tr.out_len + rq) : Lout;
+                        __syncwarp();
+                        if (lane == 0) {
+                            gen[rq] = out - rem;
+                            if (use_hist) sl.hist[ph] -= 1;
+                        }
                         nrun--;
                         next = rq;
                     }
                     __syncwarp();
+                    refresh_head();
+                    csum_d = (double)(long long)csum;
                 }
                 free_blocks -= needed;
-                const u64 ctx = csum + nrun;                           // cached tokens + the new one, summed
-                if (dc.n != nrun) {
+                if (dc_n != nrun) {
                     TaskTab kt;
                     build_fixed_tasks(m, tt, nrun, nrun, 1, kt);
-                    dc.n = nrun;
-                    dc.s_fix = eval_fixed<TIME_SUM>(kt, rt);
-                    dc.s_comm = eval_comm(kt, rt);
-                    dc.t_head = eval_head<TIME_SUM>(kt, rt);
-                    dc.THa = (u64)nrun * m.H * m.ab;
+                    dc_n = nrun;
+                    dc_fix = eval_fixed<TIME_SUM>(kt, rt);
+                    dc_comm = eval_comm(kt, rt);
+                    dc_head = eval_head<TIME_SUM>(kt, rt);
+                    dc_tha_i = (u64)nrun * m.H * m.ab;
+                    dc_tha = (double)dc_tha_i * inv_tt;
+                    dc_nd = (double)nrun;
                 }
-                {
-                    const double inv_t = 1.0 / (double)tt;
-                    const u64 X = rt.flash ? 0ull : (u64)m.nh * ctx * m.ab;
-                    const double F9 = cvt(2 * (u64)m.H * ctx) * inv_t;
-                    const double B9 = cvt(dc.THa + ctx * m.Dkv * m.kvb + X) * inv_t;
-                    const double F10 = cvt(5 * (u64)m.nh * ctx) * inv_t;
-                    const double B10 = cvt(2 * X) * inv_t;
-                    const double ic = rt.inv_c[CLS_ATTN], im = rt.inv_m[CLS_ATTN];
-                    const double t9 = task_time<TIME_SUM>(F9, B9, ic, im);
-                    const double t10 = task_time<TIME_SUM>(F10, B10, ic, im);
-                    const double s_att = (t9 + t10) + t9;
-                    t_iter = combine_phase(dc.s_fix, s_att, dc.s_comm, dc.t_head, 1.0, Nd, rt.tovh, lf);
+                const u64 ctx = csum + nrun;                           // cached tokens + the new one, summed
+                double F9, B9, F10, B10;
+                if (exact53) {
+                    const double cd = csum_d + dc_nd;                  // exact: integers below 2^53
+                    csum_d = cd;                                       // the new token joins every cache
+                    F9 = cd * c_f9;
+                    B9 = dc_tha + cd * c_kv;
+                    F10 = cd * c_f10;
+                    if (!rt.flash) { B9 = B9 + cd * c_x; }
+                    B10 = cd * c_b10;
+                } else {
+                    const u64 X = xw * ctx;
+                    F9 = cvt(2 * (u64)m.H * ctx) * inv_tt;
+                    B9 = cvt(dc_tha_i + ctx * m.Dkv * m.kvb + X) * inv_tt;
+                    F10 = cvt(5 * (u64)m.nh * ctx) * inv_tt;
+                    B10 = cvt(2 * X) * inv_tt;
                 }
-                for (u32 base = 0; base < nrun; base += 32) {
-                    const u32 k = base + lane;
-                    if (k < nrun) {
-                        s_cache[k] += 1;
-                        const u32 left = s_rem[k] - 1;
-                        s_rem[k] = left;
-                        any_done |= left == 0;
-                    }
-                }
+                const double t9 = task_time<TIME_SUM>(F9, B9, icA, imA);
+                const double t10 = task_time<TIME_SUM>(F10, B10, icA, imA);
+                const double s_att = (t9 + t10) + t9;
+                t_iter = combine_phase(dc_fix, s_att, dc_comm, dc_head, 1.0, Nd, rt.tovh, lf);
+                D++;
+                Dmod = Dmod + 1 == blk ? 0 : Dmod + 1;
                 csum += nrun;
                 dec_time = dec_time + t_iter;
                 dec_tok += nrun;
-                participants = nrun;
+                n_req_iters += nrun;
+                min_rem--;
+                any_done = min_rem == 0;
             }
             // ---- 4. advance the clock ----
             clock = clock + t_iter;
             n_iters++;
-            n_req_iters += participants;
             // ---- 5. retire finished sequences, keep the rest in order ----
-            if (__any_sync(0xFFFFFFFFu, any_done)) {
+            if (any_done) {
                 __syncwarp();
-                u32 kept = 0;
+                u32 kept = 0, local_min = NO_COMPLETION;
                 u64 freed = 0, gone = 0;
                 const u32 n_before = nrun;
                 for (u32 base = 0; base < n_before; base += 32) {
                     const u32 k = base + lane;
                     const bool valid = k < n_before;
-                    u32 rq = 0, cv = 0, rem = 1;
-                    if (valid) { rq = s_req[k]; cv = s_cache[k]; rem = s_rem[k]; }
+                    u32 rq = 0, bs = 0, fn = 0, mt = 0;
+                    if (valid) { rq = sl.req[k]; bs = sl.base[k]; fn = sl.fin[k]; mt = sl.meta[k]; }
+                    const u32 rem = fn - D;
                     const bool done = valid && rem == 0;
                     if (done) {
+                        const u32 cv = bs + D;
                         gen[rq] = GEN_DONE;
                         const u32 out = __ldg(tr.in_len + rq) ? __ldg(tr.out_len + rq) : Lout;
                         tpot[rq] = out > 1 ? (clock - first[rq]) / (double)(out - 1) : 0.0;
                         freed += ceil_div32(cv, blk);
                         gone += cv;
+                        if (use_hist) atomicSub(&sl.hist[mt & M_PHASE], 1u);
                     }
                     const bool keep = valid && !done;
+                    if (keep) local_min = min(local_min, rem);
                     const u32 ballot = __ballot_sync(0xFFFFFFFFu, keep);
                     __syncwarp();
                     if (keep) {
                         const u32 d = kept + __popc(ballot & lt_mask);
-                        s_req[d] = rq; s_cache[d] = cv; s_rem[d] = rem;
+                        sl.req[d] = rq; sl.base[d] = bs; sl.fin[d] = fn; sl.meta[d] = (unsigned char)mt;
                     }
                     kept += __popc(ballot);
                     __syncwarp();
                 }
                 free_blocks += warp_sum(freed);
                 csum -= warp_sum(gone);
+                min_rem = warp_min(local_min);
                 nrun = kept;
+                csum_d = (double)(long long)csum;
             }
         }
 
@@ -336,23 +437,34 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
     }
 }
 
-int launch_trace_sim(const DSpace &s, const DTrace &t, Range r, int time_model, int tp_model, u64 max_iters,
-                     const guide_outputs &o, void *ws, size_t, cudaStream_t st) {
+template <int TIME_SUM>
+static int launch_one(const DSpace &s, const DTrace &t, Range r, int tp_model, u64 max_iters, const guide_outputs &o,
+                      void *ws, cudaStream_t st) {
     const size_t pw = per_warp_bytes(t.n);
     const u32 gen_bytes = (u32)(((size_t)t.n * 4 + 255) / 256 * 256);
     const u32 first_bytes = (u32)(((size_t)t.n * 8 + 255) / 256 * 256);
     // resident warps: as many as the SMs hold, never more than the workspace was sized for
-    u32 blocks = (u32)num_sms() * 4;
+    int per_sm = 0;
+    GUIDE_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_trace_sim<TIME_SUM>, SIM_THREADS, 0));
+    if (per_sm < 1) per_sm = 1;
+    u32 blocks = (u32)num_sms() * (u32)per_sm;
     blocks = std::min<u32>(blocks, SIM_MAX_WARPS / SIM_WARPS_PER_BLOCK);
     blocks = (u32)std::min<u64>(blocks, (r.count + SIM_WARPS_PER_BLOCK - 1) / SIM_WARPS_PER_BLOCK);
+    const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
+    const int reorder = r.first == 0 && r.count == total;
     GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
     unsigned char *scratch = (unsigned char *)ws + 256;
-    if (time_model)
-        k_trace_sim<1><<<blocks, SIM_THREADS, 0, st>>>(s, t, r, tp_model, max_iters, o, (u32 *)ws, scratch, pw, gen_bytes, first_bytes);
-    else
-        k_trace_sim<0><<<blocks, SIM_THREADS, 0, st>>>(s, t, r, tp_model, max_iters, o, (u32 *)ws, scratch, pw, gen_bytes, first_bytes);
+    k_trace_sim<TIME_SUM><<<blocks, SIM_THREADS, 0, st>>>(s, t, r, tp_model, max_iters, o, (u32 *)ws, scratch, pw,
+                                                         gen_bytes, first_bytes, reorder);
     GUIDE_CUDA(cudaGetLastError());
     return GUIDE_OK;
+}
+
+int launch_trace_sim(const DSpace &s, const DTrace &t, Range r, int time_model, int tp_model, u64 max_iters,
+                     const guide_outputs &o, void *ws, size_t, cudaStream_t st) {
+    if (r.count > 0xFFFFFFF0ull) return fail(GUIDE_ERR_UNSUPPORTED, "at most 2^32 - 16 configs per trace launch");
+    return time_model ? launch_one<1>(s, t, r, tp_model, max_iters, o, ws, st)
+                      : launch_one<0>(s, t, r, tp_model, max_iters, o, ws, st);
 }
 
 }  // namespace guide
