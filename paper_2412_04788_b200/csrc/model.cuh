@@ -138,7 +138,7 @@ template <int TIME_SUM>
 __device__ __forceinline__ double task_time(double F, double B, double ic, double im) {
     const double tc = F * ic;          // compute time (Sec. 3.5.1)
     const double tm = B * im;          // read/write time
-    return TIME_SUM ? tc + tm : fmax(tc, tm);   // Sec. 3.5.1 literal sum, or the roofline of Sec. 3.4.2
+    return TIME_SUM ? tc + tm : (tc > tm ? tc : tm);   // Sec. 3.5.1 literal sum, or the roofline of Sec. 3.4.2
 }
 
 // Sum of the eight non-attention layer tasks in their fixed order.

@@ -55,6 +55,20 @@ __device__ __forceinline__ u32 warp_min(u32 v) {
 }
 __device__ __forceinline__ u32 ceil_div32(u32 a, u32 b) { return (a + b - 1) / b; }
 
+// Time of one decode iteration from the summed context (as an exact double), when every integer
+// count of the config is below 2^53: the same products and sums as the integer form, in doubles.
+// B9 = (T H a_b + ctx (Dkv kv_b + score bytes)) / t is a sum of exact terms, so its association
+// does not matter; with FlashAttention the score constants are 0 and t10's memory time is 0.
+template <int TIME_SUM>
+__device__ __forceinline__ double decode_time(double ctxd, double c_f9, double tha, double c_kvx, double c_f10, double c_b10,
+                                              double ic, double im, double fix, double comm, double head, double Nd,
+                                              double tovh, double lf) {
+    const double t9 = task_time<TIME_SUM>(ctxd * c_f9, tha + ctxd * c_kvx, ic, im);
+    const double t10 = task_time<TIME_SUM>(ctxd * c_f10, ctxd * c_b10, ic, im);
+    const double s_att = (t9 + t10) + t9;
+    return combine_phase(fix, s_att, comm, head, 1.0, Nd, tovh, lf);
+}
+
 struct SlotArrays {
     u32 req[SLOTS];     // request index
     u32 base[SLOTS];    // resident: cache - D (mod 2^32); waiting for its prompt pass: prompt + recompute tokens
@@ -127,8 +141,7 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         const bool exact53 = 2 * (u64)m.H * ctx_max < lim53 && 5 * (u64)m.nh * ctx_max < lim53 &&
                              (u64)b * m.H * m.ab + ctx_max * ((u64)m.Dkv * m.kvb + xw) < lim53 && 2 * xw * ctx_max < lim53;
         const double c_f9 = (double)(2 * (u64)m.H) * inv_tt;               // F9  = ctx * 2H / t
-        const double c_kv = (double)((u64)m.Dkv * m.kvb) * inv_tt;         // KV read per context token / t
-        const double c_x = (double)xw * inv_tt;                            // score bytes per context token / t
+        const double c_kvx = (double)((u64)m.Dkv * m.kvb + xw) * inv_tt;   // KV read + score bytes per context token / t
         const double c_f10 = (double)(5 * (u64)m.nh) * inv_tt;             // F10 = ctx * 5 n_h / t
         const double c_b10 = (double)(2 * xw) * inv_tt;                    // B10 = ctx * 2 n_h a_b / t (0 with flash)
 
@@ -137,6 +150,7 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         u32 next = 0, high_water = 0, nrun = 0, n_new = 0;
         u32 D = 0, Dmod = 0, min_rem = NO_COMPLETION;
         const bool use_hist = blk > 1 && blk <= HIST;
+        const bool burst_ok = exact53 && (blk == 1 || use_hist);
         const u64 max_iters = max_iters_opt ? max_iters_opt : 64 * (tr.sum_out + (u64)tr.n_zero * Lout) + 4 * (u64)n;
         // cached while the running count stays the same
         u32 dc_n = 0;
@@ -190,8 +204,7 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                 break;
             }
             if (n_iters >= max_iters) { st |= GUIDE_ST_ITER; break; }
-            // ---- 3. build the iteration: prompts first, everything else stalls ----
-            double t_iter;
+            // ---- 3./4. build the iteration (prompts first, everything else stalls) and advance the clock ----
             bool any_done;
             if (n_new > 0) {
                 u64 T = 0, A = 0;
@@ -203,6 +216,7 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                     }
                 }
                 T = warp_sum(T); A = warp_sum(A);
+                double t_iter;
                 {
                     TaskTab kt;
                     build_fixed_tasks(m, tt, T, n_new, 1, kt);
@@ -237,6 +251,8 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                 csum_d = (double)(long long)csum;
                 n_req_iters += n_new;
                 n_new = 0;
+                clock = after;
+                n_iters++;
             } else {
                 // every sequence whose last block is full needs one more block
                 u32 needed;
@@ -281,39 +297,69 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                     dc_tha = (double)dc_tha_i * inv_tt;
                     dc_nd = (double)nrun;
                 }
-                const u64 ctx = csum + nrun;                           // cached tokens + the new one, summed
-                double F9, B9, F10, B10;
-                if (exact53) {
-                    const double cd = csum_d + dc_nd;                  // exact: integers below 2^53
-                    csum_d = cd;                                       // the new token joins every cache
-                    F9 = cd * c_f9;
-                    B9 = dc_tha + cd * c_kv;
-                    F10 = cd * c_f10;
-                    if (!rt.flash) { B9 = B9 + cd * c_x; }
-                    B10 = cd * c_b10;
+                if (burst_ok) {
+                    // A run of decode iterations up to the next event.  Nothing per request is
+                    // touched; integer counters are settled once after the run.  The next
+                    // iteration's time is computed before the clock-dependent exit test so the two
+                    // dependency chains overlap.
+                    const u64 cap_left = max_iters - n_iters;
+                    const u32 steps_max = (u32)min((u64)min_rem, cap_left);
+                    const u32 fb0 = (u32)min(free_blocks, (u64)0xFFFFFFFFu);
+                    u32 fb = fb0, it = 0;
+                    u32 hidx = Dmod + 1 == blk ? 0 : blk - (Dmod + 1);     // histogram bin of the next iteration's needers
+                    const bool room = nrun < b;
+                    const double nd = dc_nd, tha = dc_tha, fix = dc_fix, comm = dc_comm, head = dc_head, tovh = rt.tovh;
+                    double cd = csum_d;
+                    double ctxd = cd + nd;
+                    double tcur = decode_time<TIME_SUM>(ctxd, c_f9, tha, c_kvx, c_f10, c_b10, icA, imA, fix, comm, head, Nd,
+                                                        tovh, lf);
+                    for (;;) {
+                        clock = clock + tcur;
+                        dec_time = dec_time + tcur;
+                        cd = ctxd;
+                        it++;
+                        ctxd = cd + nd;
+                        const double tnext = decode_time<TIME_SUM>(ctxd, c_f9, tha, c_kvx, c_f10, c_b10, icA, imA, fix, comm,
+                                                                   head, Nd, tovh, lf);
+                        if (it == steps_max) break;                               // a completion (or the cap) follows
+                        const u32 need2 = blk == 1 ? nrun : sl.hist[hidx];
+                        if (need2 > fb) break;                                    // eviction needed
+                        if (room && arr_next <= clock && need_next <= fb) break;  // the queue head can come in
+                        fb -= need2;
+                        hidx = hidx == 0 ? blk - 1 : hidx - 1;
+                        tcur = tnext;
+                    }
+                    const u64 tok = (u64)it * nrun;
+                    D += it;
+                    Dmod = (Dmod + it) % blk;
+                    csum += tok; csum_d = cd;
+                    dec_tok += tok; n_req_iters += tok; n_iters += it;
+                    min_rem -= it;
+                    free_blocks -= fb0 - fb;
+                    any_done = min_rem == 0;
                 } else {
+                    const u64 ctx = csum + nrun;                       // cached tokens + the new one, summed
                     const u64 X = xw * ctx;
-                    F9 = cvt(2 * (u64)m.H * ctx) * inv_tt;
-                    B9 = cvt(dc_tha_i + ctx * m.Dkv * m.kvb + X) * inv_tt;
-                    F10 = cvt(5 * (u64)m.nh * ctx) * inv_tt;
-                    B10 = cvt(2 * X) * inv_tt;
+                    const double F9 = cvt(2 * (u64)m.H * ctx) * inv_tt;
+                    const double B9 = cvt(dc_tha_i + ctx * m.Dkv * m.kvb + X) * inv_tt;
+                    const double F10 = cvt(5 * (u64)m.nh * ctx) * inv_tt;
+                    const double B10 = cvt(2 * X) * inv_tt;
+                    const double t9 = task_time<TIME_SUM>(F9, B9, icA, imA);
+                    const double t10 = task_time<TIME_SUM>(F10, B10, icA, imA);
+                    const double s_att = (t9 + t10) + t9;
+                    const double t_iter = combine_phase(dc_fix, s_att, dc_comm, dc_head, 1.0, Nd, rt.tovh, lf);
+                    D++;
+                    Dmod = Dmod + 1 == blk ? 0 : Dmod + 1;
+                    csum += nrun;
+                    dec_time = dec_time + t_iter;
+                    dec_tok += nrun;
+                    n_req_iters += nrun;
+                    n_iters++;
+                    min_rem--;
+                    any_done = min_rem == 0;
+                    clock = clock + t_iter;
                 }
-                const double t9 = task_time<TIME_SUM>(F9, B9, icA, imA);
-                const double t10 = task_time<TIME_SUM>(F10, B10, icA, imA);
-                const double s_att = (t9 + t10) + t9;
-                t_iter = combine_phase(dc_fix, s_att, dc_comm, dc_head, 1.0, Nd, rt.tovh, lf);
-                D++;
-                Dmod = Dmod + 1 == blk ? 0 : Dmod + 1;
-                csum += nrun;
-                dec_time = dec_time + t_iter;
-                dec_tok += nrun;
-                n_req_iters += nrun;
-                min_rem--;
-                any_done = min_rem == 0;
             }
-            // ---- 4. advance the clock ----
-            clock = clock + t_iter;
-            n_iters++;
             // ---- 5. retire finished sequences, keep the rest in order ----
             if (any_done) {
                 __syncwarp();
