@@ -30,92 +30,31 @@ __global__ void __launch_bounds__(256) k_closed_form_flat(DSpace s, Range r, int
     store_metrics(o, j, m);
 }
 
-// Tiled evaluation.  The integer task table of a config depends on (model, batch, TP, lengths)
-// only, and within one (model, batch) the (TP, length) positions are the fastest-running part of
-// the config index.  A thread therefore owns one (model, batch, TP, length) point, builds both
-// stage tables once, and walks a chunk of the hardware x framework pairs, which are the only
-// things the roofline evaluation needs beyond the table.  A warp's 32 threads hold 32
-// consecutive config indices for every pair, so each store instruction writes one 256-byte run.
+// Tiled evaluation (see tiled.cuh): every valid config's metrics are stored.
 template <int TIME_SUM>
-__global__ void __launch_bounds__(256) k_closed_form_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk,
-                                                           u32 tiles_per_mb, guide_outputs o) {
-    const u32 n_tl = s.n_t * s.n_l;
-    const u32 n_hf = s.n_h * s.n_f;
-    // blockIdx.x -> (model, batch, tile of the (TP, length) plane); blockIdx.y -> chunk of pairs
-    const u32 tile = blockIdx.x % tiles_per_mb;
-    const u32 mb = blockIdx.x / tiles_per_mb;
-    const u32 bpos = mb % s.n_b, mpos = mb / s.n_b;
-    const u32 tl = tile * blockDim.x + threadIdx.x;
-    if (tl >= n_tl) return;
-    const u32 tpos = tl / s.n_l, lpos = tl % s.n_l;
-    const u32 hf0 = blockIdx.y * hf_chunk;
-    const u32 hf1 = min(hf0 + hf_chunk, n_hf);
-
-    const DModel m = s.models[mpos];
-    const u32 t = s.tp[tpos], b = s.batch[bpos];
-    const uint2 pr = s.pairs[lpos];
-    const u32 lin = pr.x, lout = pr.y, n = lout - 1;
-    const MemInfo mi = mem_info(m, t);
-    const u32 tt = tp_model ? 1u : t;
-    const double lf = log2_rule_factor(t, tp_model);
-    const double Nd = (double)m.N;
-
-    TaskTab kp, kd;
-    const u64 Tp = (u64)b * lin;
-    build_fixed_tasks(m, tt, Tp, b, 1, kp);
-    build_attn_tasks(m, tt, Tp, Tp * lin, Tp, kp);
-    if (n > 0) {
-        const u64 Td = (u64)b * n;
-        const u64 ctx = (u64)b * ((u64)n * lin + ((u64)n * (n + 1)) / 2);
-        build_fixed_tasks(m, tt, Td, Td, n, kd);
-        build_attn_tasks(m, tt, Td, ctx, ctx, kd);
-    }
-    // index of this thread's config for pair (h, f): ((((m n_h + h) n_f + f) n_b + b) n_t n_l) + tl
-    const u64 stride_hf = (u64)s.n_b * n_tl;
-    const u64 base = ((u64)mpos * n_hf) * stride_hf + (u64)bpos * n_tl + tl;
-
-    for (u32 hf = hf0; hf < hf1; hf++) {
-        const u64 idx = base + (u64)hf * stride_hf;
-        if (idx < r.first || idx - r.first >= r.count) continue;
-        const DRate rt = s.rates[hf];
-        Metrics out;
-        out.status = closed_form_feasibility(m, rt, mi, t, b, lin, lout, out.bmax);
-        if (out.status) set_infeasible(out);
-        else {
-            const double t_pre = eval_phase<TIME_SUM>(kp, rt, Nd, lf);
-            const double t_dec = n > 0 ? eval_phase<TIME_SUM>(kd, rt, Nd, lf) : 0.0;
-            closed_form_metrics(t_pre, t_dec, b, n, t, rt.price, out);
-        }
-        store_metrics(o, idx - r.first, out);
-    }
+__global__ void __launch_bounds__(256, 2) k_closed_form_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk,
+                                                              u32 tiles_per_mb, guide_outputs o) {
+    tiled_visit<TIME_SUM>(s, r, tp_model, hf_chunk, tiles_per_mb, [&](bool valid, u64 idx, const Metrics &m) {
+        if (valid) store_metrics(o, idx - r.first, m);
+    });
 }
 
 int launch_closed_form(const DSpace &s, Range r, int time_model, int tp_model, const guide_outputs &o,
                        cudaStream_t st) {
-    const u32 n_tl = s.n_t * s.n_l, n_hf = s.n_h * s.n_f;
-    const u64 total = (u64)s.n_m * n_hf * s.n_b * n_tl;
+    const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
     // The tiled kernel pays off when a (TP, length) plane fills warps and the range is (most of)
     // the space; slivers of the space go through the flat kernel.
-    const bool tiled = n_tl >= 32 && r.count * 2 >= total;
+    TileGeom g;
+    const bool tiled = r.count * 2 >= total && tiled_geometry(s, (u64)num_sms() * 16, 1ull << 30, &g);
     if (!tiled) {
         const u64 blocks = (r.count + 255) / 256;
         if (blocks > 0x7FFFFFFFull) return fail(GUIDE_ERR_UNSUPPORTED, "range too large for one launch");
         if (time_model) k_closed_form_flat<1><<<(u32)blocks, 256, 0, st>>>(s, r, tp_model, o);
         else k_closed_form_flat<0><<<(u32)blocks, 256, 0, st>>>(s, r, tp_model, o);
     } else {
-        const u32 threads = n_tl >= 256 ? 256 : ((n_tl + 31) / 32) * 32;
-        const u32 tiles = (n_tl + threads - 1) / threads;
-        const u64 gx = (u64)s.n_m * s.n_b * tiles;
-        // Split the pair loop so the grid has a few waves of blocks; longer chunks amortise the
-        // table building over more configs.
-        const u64 want_blocks = (u64)num_sms() * 16;
-        u32 splits = (u32)std::min<u64>(n_hf, std::max<u64>(1, (want_blocks + gx - 1) / gx));
-        u32 chunk = (n_hf + splits - 1) / splits;
-        splits = (n_hf + chunk - 1) / chunk;
-        if (gx > 0x7FFFFFFFull || splits > 65535) return fail(GUIDE_ERR_UNSUPPORTED, "space too large for one launch");
-        const dim3 grid((u32)gx, splits);
-        if (time_model) k_closed_form_tiled<1><<<grid, threads, 0, st>>>(s, r, tp_model, chunk, tiles, o);
-        else k_closed_form_tiled<0><<<grid, threads, 0, st>>>(s, r, tp_model, chunk, tiles, o);
+        const dim3 grid(g.gx, g.splits);
+        if (time_model) k_closed_form_tiled<1><<<grid, g.threads, 0, st>>>(s, r, tp_model, g.hf_chunk, g.tiles_per_mb, o);
+        else k_closed_form_tiled<0><<<grid, g.threads, 0, st>>>(s, r, tp_model, g.hf_chunk, g.tiles_per_mb, o);
     }
     GUIDE_CUDA(cudaGetLastError());
     return GUIDE_OK;

@@ -8,6 +8,7 @@
 
 #include "../../include/guide.h"
 #include "model.cuh"
+#include "tiled.cuh"
 
 namespace guide {
 
@@ -60,8 +61,6 @@ namespace guide {
 // device views for the current device (uploads on first use)
 int space_on_device(guide_space *s, DSpace *out);
 int trace_on_device(guide_trace *t, DTrace *out);
-
-struct Range { u64 first, count; };
 
 // closed_form.cu
 int launch_closed_form(const DSpace &s, Range r, int time_model, int tp_model, const guide_outputs &o,

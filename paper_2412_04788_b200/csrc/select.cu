@@ -2,11 +2,17 @@
 //
 // Both reductions are streaming: a block walks its share of the configs, drops on the spot
 // whatever its current partial result already beats (a threshold for top-k, the block's current
-// front for Pareto), appends the few survivors to a shared-memory buffer and, when that fills,
-// sorts the buffer and rebuilds the partial result.  Block results go to the workspace; the block
-// that finishes last streams them through the same routine to produce the global answer.
+// front for Pareto) and appends the few survivors to a shared-memory buffer with one atomic and
+// no barrier.  Every few rounds the block meets at a checkpoint and, if the buffer could overflow
+// before the next one, sorts it and rebuilds the partial result.  Block results go to the
+// workspace.  Top-k lists are merged by a second, fully parallel kernel that ranks every surviving
+// candidate against all lists; Pareto fronts are folded by the block that finishes last.
 // Every comparison is on the total order (value, config index), so the answer does not depend on
 // how configs are spread over blocks or in which order they are appended.
+//
+// The metrics come either from materialised arrays or, fused, from the closed-form evaluation
+// itself, walked in the tiled order of tiled.cuh so the integer task tables are built once per
+// (model, batch, TP, length) point.
 #include "guide_internal.cuh"
 
 namespace guide {
@@ -14,6 +20,8 @@ namespace guide {
 static constexpr u32 SEL_THREADS = 256;
 static constexpr u32 SEL_MAX_BLOCKS = 1024;
 static constexpr u32 PARETO_CAP = 4096;          // shared-memory items per block
+static constexpr u32 TOPK_CAP = 2048;            // shared-memory candidates per block
+static constexpr u32 CHECK_EVERY = 4;            // appends per thread between two checkpoints
 static constexpr u64 KEY_MAX = ~0ull;
 
 // order-preserving map double -> u64 (after -0.0 -> +0.0)
@@ -48,6 +56,7 @@ __device__ __forceinline__ double pick_metric(int key, double latency, double tt
 
 // materialised arrays written by guide_simulate
 struct MatSource {
+    static constexpr int ITEMS = 4;     // loads of four configs are in flight before the first barrier
     guide_outputs o;
     Cons c;
     int m0, m1;
@@ -62,25 +71,28 @@ struct MatSource {
         default: return __ldg(o.cost_per_token + j);
         }
     }
+    // No data-dependent early exit: every load of a config (and of the other configs a thread
+    // fetches in the same round) can be in flight at once.  Branches are on launch constants only.
     __device__ __forceinline__ bool get(u64 j, u64, double &a, double &b) const {
-        if (__ldg(o.status + j)) return false;
         const double inf = __longlong_as_double(0x7FF0000000000000LL);
+        bool ok = __ldg(o.status + j) == 0;
         if (c.max_ttft < inf) {
             const double *p = c.ttft_stat == GUIDE_STAT_MEAN ? o.ttft : c.ttft_stat == GUIDE_STAT_P50 ? o.ttft_p50 : o.ttft_p99;
-            if (!(__ldg(p + j) <= c.max_ttft)) return false;
+            ok &= __ldg(p + j) <= c.max_ttft;
         }
-        if (c.max_latency < inf && !(__ldg(o.latency + j) <= c.max_latency)) return false;
-        if (c.max_cost_hr < inf && !(__ldg(o.cost_per_hr + j) <= c.max_cost_hr)) return false;
-        if (c.min_thr > 0.0 && !(__ldg(o.thr_decode + j) >= c.min_thr)) return false;
+        if (c.max_latency < inf) ok &= __ldg(o.latency + j) <= c.max_latency;
+        if (c.max_cost_hr < inf) ok &= __ldg(o.cost_per_hr + j) <= c.max_cost_hr;
+        if (c.min_thr > 0.0) ok &= __ldg(o.thr_decode + j) >= c.min_thr;
         a = metric(m0, j);
         b = m1 >= 0 ? metric(m1, j) : 0.0;
-        return true;
+        return ok;
     }
 };
 
 // closed form evaluated on the fly: nothing is written to memory
 template <int TIME_SUM>
 struct FusedSource {
+    static constexpr int ITEMS = 1;     // evaluation is register heavy: one config at a time
     DSpace s;
     Cons c;
     int m0, m1, tp_model;
@@ -132,15 +144,15 @@ __device__ void block_bitonic_sort(T *buf, u32 P, Less less) {
 // ---- top-k accumulator -------------------------------------------------------------------------------
 
 struct TopKAcc {
-    KI *buf;          // shared, cap entries
+    KI *buf;          // shared, TOPK_CAP entries
     u32 *cnt;         // shared append cursor
-    u32 cap, k;
-    u32 c;            // mirror of *cnt, identical in every thread
+    u32 k;
+    u32 c;            // buffered count at the last checkpoint, identical in every thread
     bool has_thr;
     KI thr;
 
-    __device__ void init(KI *b, u32 *cn, u32 cap_, u32 k_) {
-        buf = b; cnt = cn; cap = cap_; k = k_; c = 0; has_thr = false; thr.key = KEY_MAX; thr.idx = KEY_MAX;
+    __device__ void init(KI *b, u32 *cn, u32 k_) {
+        buf = b; cnt = cn; k = k_; c = 0; has_thr = false; thr.key = KEY_MAX; thr.idx = KEY_MAX;
         if (threadIdx.x == 0) *cnt = 0;
         __syncthreads();
     }
@@ -155,12 +167,27 @@ struct TopKAcc {
         if (threadIdx.x == 0) *cnt = c;
         __syncthreads();
     }
-    // collective: every thread of the block calls it once per tile
-    __device__ void push(bool ok, KI it) {
-        const bool take = ok && (!has_thr || ki_less(it, thr));
-        if (take) buf[atomicAdd(cnt, 1)] = it;
-        c += __syncthreads_count(take);        // same count in every thread
-        if (c + blockDim.x > cap) compact();
+    // No barrier.  Between two checkpoints a thread may offer at most CHECK_EVERY items; the
+    // checkpoint keeps c + CHECK_EVERY * blockDim <= TOPK_CAP, so the slot is always in range.
+    __device__ __forceinline__ void offer(bool ok, const KI &it) {
+        if (ok && (!has_thr || ki_less(it, thr))) buf[atomicAdd(cnt, 1)] = it;
+    }
+    // collective.  Compacts when the buffer could overflow before the next checkpoint, and early
+    // while that is cheap: as soon as k candidates exist (first threshold), then whenever about k
+    // more have slipped under the stale threshold.  Small sorts cost little; a fresh threshold
+    // keeps almost everything out.
+    __device__ void checkpoint() {
+        __syncthreads();
+        c = *cnt;
+        __syncthreads();                       // nobody appends before everyone has read the count
+        const u32 early = has_thr ? 2 * k + blockDim.x : k;
+        if (c + CHECK_EVERY * blockDim.x > TOPK_CAP || c >= early) compact();
+    }
+    __device__ void finish() {
+        __syncthreads();
+        c = *cnt;
+        __syncthreads();
+        compact();
     }
 };
 
@@ -246,132 +273,312 @@ struct ParetoAcc {
         if (threadIdx.x == 0) *cnt = out;
         __syncthreads();
     }
-    __device__ void push(bool ok, P3 it) {
-        const bool take = ok && !beaten(it);
-        if (take) buf[atomicAdd(cnt, 1)] = it;
-        c += __syncthreads_count(take);
-        if (c + blockDim.x > PARETO_CAP) merge();
+    // no barrier; at most CHECK_EVERY offers per thread between checkpoints
+    __device__ __forceinline__ void offer(bool ok, const P3 &it) {
+        if (ok && !beaten(it)) buf[atomicAdd(cnt, 1)] = it;
+    }
+    __device__ void checkpoint() {
+        __syncthreads();
+        c = *cnt;
+        __syncthreads();
+        // merge when the buffer could overflow before the next checkpoint, as soon as there is
+        // anything while no front exists yet (until then nothing is filtered), and whenever a
+        // block's worth of points has slipped past the stale front
+        if (c + CHECK_EVERY * blockDim.x > PARETO_CAP || (nf == 0 && c > 0) || c >= nf + blockDim.x) merge();
+    }
+    __device__ void finish() {
+        __syncthreads();
+        c = *cnt;
+        __syncthreads();
+        merge();
     }
 };
 
-// ---- kernels ----------------------------------------------------------------------------------------
+// constraint filter and metric choice on freshly evaluated closed-form metrics
+__device__ __forceinline__ bool fused_pick(const Metrics &m, const Cons &c, int m0, int m1, double &a, double &b) {
+    if (m.status) return false;
+    if (!(m.ttft <= c.max_ttft) || !(m.latency <= c.max_latency) || !(m.cost_hr <= c.max_cost_hr) || !(m.thr >= c.min_thr))
+        return false;
+    a = pick_metric(m0, m.latency, m.ttft, m.ttft, m.tpot, m.thr, m.cost_hr, m.cost_tok);
+    b = m1 >= 0 ? pick_metric(m1, m.latency, m.ttft, m.ttft, m.tpot, m.thr, m.cost_hr, m.cost_tok) : 0.0;
+    return true;
+}
 
-// workspace: [0] ticket, then per block k candidates
+// ---- top-k kernels -----------------------------------------------------------------------------------
+
+// a block's sorted candidates and their number go to the workspace
+__device__ __forceinline__ void topk_store(TopKAcc &acc, u32 block, u32 k, u32 *counts, KI *lists) {
+    acc.finish();
+    KI *mine = lists + (size_t)block * k;
+    for (u32 i = threadIdx.x; i < acc.c; i += blockDim.x) mine[i] = acc.buf[i];
+    if (threadIdx.x == 0) counts[block] = acc.c;
+}
+
 template <class Src>
-__global__ void __launch_bounds__(SEL_THREADS) k_topk(Src src, Range r, u32 k, u32 cap, u32 *ticket, KI *partial,
-                                                      int negate_out, u64 *idx_out, double *key_out, u32 *count_out) {
+__global__ void __launch_bounds__(SEL_THREADS) k_topk_scan(Src src, Range r, u32 k, u32 *counts, KI *lists) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    KI *buf = (KI *)smem_raw;
     __shared__ u32 cnt;
-    __shared__ u32 last_flag;
     TopKAcc acc;
-    acc.init(buf, &cnt, cap, k);
-    const u64 tiles = (r.count + blockDim.x - 1) / blockDim.x;
+    acc.init((KI *)smem_raw, &cnt, k);
+    constexpr int ITEMS = Src::ITEMS;
+    constexpr u32 ROUNDS = CHECK_EVERY / ITEMS;          // tiles between checkpoints
+    const u64 span = (u64)ITEMS * blockDim.x;
+    const u64 tiles = (r.count + span - 1) / span;
+    u32 since = 0;
     for (u64 tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-        const u64 j = tile * blockDim.x + threadIdx.x;
-        double a = 0.0, b;
-        const bool ok = j < r.count && src.get(j, r.first + j, a, b);
-        KI it;
-        it.key = enc(a); it.idx = r.first + j;
-        acc.push(ok, it);
-    }
-    acc.compact();
-    KI *mine = partial + (size_t)blockIdx.x * k;
-    for (u32 i = threadIdx.x; i < k; i += blockDim.x) {
-        KI v; v.key = KEY_MAX; v.idx = KEY_MAX;
-        if (i < acc.c) v = buf[i];
-        mine[i] = v;
-    }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) last_flag = (atomicAdd(ticket, 1) == gridDim.x - 1);
-    __syncthreads();
-    if (!last_flag) return;
-    __threadfence();
-    // the last block folds every block's candidates
-    acc.init(buf, &cnt, cap, k);
-    const u64 total = (u64)gridDim.x * k;
-    for (u64 base = 0; base < total; base += blockDim.x) {
-        const u64 i = base + threadIdx.x;
-        KI it; it.key = KEY_MAX; it.idx = KEY_MAX;
-        if (i < total) {      // written by other blocks: read through L2
-            const ulonglong2 v = __ldcg(reinterpret_cast<const ulonglong2 *>(partial) + i);
-            it.key = v.x; it.idx = v.y;
+        bool ok[ITEMS];
+        KI it[ITEMS];
+#pragma unroll
+        for (int u = 0; u < ITEMS; u++) {
+            const u64 j = tile * span + (u64)u * blockDim.x + threadIdx.x;
+            const u64 jc = j < r.count ? j : r.count - 1;          // keep the loads in range
+            double a = 0.0, b;
+            ok[u] = src.get(jc, r.first + jc, a, b) && j < r.count;
+            it[u].key = enc(a); it[u].idx = r.first + j;
         }
-        acc.push(i < total && it.idx != KEY_MAX, it);
+        if (tile == blockIdx.x) {
+            // first round: one offer per checkpoint, so the first threshold comes from a small sort
+#pragma unroll
+            for (int u = 0; u < ITEMS; u++) { acc.offer(ok[u], it[u]); acc.checkpoint(); }
+            continue;
+        }
+#pragma unroll
+        for (int u = 0; u < ITEMS; u++) acc.offer(ok[u], it[u]);
+        if (++since == ROUNDS) { acc.checkpoint(); since = 0; }
     }
-    acc.compact();
-    for (u32 i = threadIdx.x; i < k; i += blockDim.x) {
-        if (i < acc.c) {
-            const double v = dec(buf[i].key);
-            idx_out[i] = buf[i].idx;
-            key_out[i] = negate_out ? 0.0 - v : v;
-        } else {
+    topk_store(acc, blockIdx.x, k, counts, lists);
+}
+
+template <int TIME_SUM>
+__global__ void __launch_bounds__(SEL_THREADS, 2)
+k_topk_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, Cons c, int key, u32 k, u32 *counts, KI *lists) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ u32 cnt;
+    TopKAcc acc;
+    acc.init((KI *)smem_raw, &cnt, k);
+    u32 since = CHECK_EVERY - 1;          // the first offer is followed by a checkpoint: early threshold
+    tiled_visit<TIME_SUM>(s, r, tp_model, hf_chunk, tiles_per_mb, [&](bool valid, u64 idx, const Metrics &m) {
+        double a = 0.0, b;
+        const bool ok = valid && fused_pick(m, c, key, -1, a, b);
+        KI it;
+        it.key = enc(a); it.idx = idx;
+        acc.offer(ok, it);
+        if (++since == CHECK_EVERY) { acc.checkpoint(); since = 0; }
+    });
+    topk_store(acc, blockIdx.y * gridDim.x + blockIdx.x, k, counts, lists);
+}
+
+// Merge of the per-block lists.  One warp per candidate: its rank in the union is its position in
+// its own list plus, for every other list, the number of entries smaller than it (binary search,
+// the lanes sharing out the lists; entries are unique because config indices are).  Candidates
+// above the smallest k-th entry of any full list cannot be among the k smallest and are skipped.
+// Ranks below k are distinct, so every output slot has one writer.
+__global__ void __launch_bounds__(SEL_THREADS) k_topk_merge(u32 nblk, u32 k, const u32 *counts, const KI *lists,
+                                                            int negate_out, u64 *idx_out, double *key_out, u32 *count_out) {
+    __shared__ KI s_best[SEL_THREADS / 32];
+    __shared__ u32 s_tot[SEL_THREADS / 32];
+    KI best; best.key = KEY_MAX; best.idx = KEY_MAX;
+    u32 tot = 0;
+    for (u32 b = threadIdx.x; b < nblk; b += blockDim.x) {
+        const u32 cb = counts[b];
+        tot += min(cb, k);          // saturating: only min(total, k) matters
+        if (cb >= k) {
+            const KI e = lists[(size_t)b * k + k - 1];
+            if (ki_less(e, best)) best = e;
+        }
+    }
+    for (int d = 16; d > 0; d >>= 1) {
+        KI o;
+        o.key = __shfl_xor_sync(0xFFFFFFFFu, best.key, d);
+        o.idx = __shfl_xor_sync(0xFFFFFFFFu, best.idx, d);
+        if (ki_less(o, best)) best = o;
+        const u32 t2 = __shfl_xor_sync(0xFFFFFFFFu, tot, d);
+        tot = min(tot + t2, k);
+    }
+    if ((threadIdx.x & 31) == 0) { s_best[threadIdx.x >> 5] = best; s_tot[threadIdx.x >> 5] = tot; }
+    __syncthreads();
+    best = s_best[0]; tot = s_tot[0];
+    for (u32 w = 1; w < SEL_THREADS / 32; w++) {
+        if (ki_less(s_best[w], best)) best = s_best[w];
+        tot = min(tot + s_tot[w], k);
+    }
+    const u32 found = min(tot, k);
+    if (blockIdx.x == 0) {
+        if (threadIdx.x == 0) *count_out = found;
+        for (u32 i = found + threadIdx.x; i < k; i += blockDim.x) {
             idx_out[i] = KEY_MAX;
             key_out[i] = __longlong_as_double(0x7FF0000000000000LL);
         }
     }
-    if (threadIdx.x == 0) *count_out = acc.c;
+    // candidates, one warp each: the lanes split the lists
+    const u32 lane = threadIdx.x & 31;
+    const u64 n_warps = (u64)gridDim.x * (blockDim.x >> 5);
+    const u64 n_cand = (u64)nblk * k;
+    for (u64 g = (u64)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); g < n_cand; g += n_warps) {
+        const u32 b = (u32)(g / k), p = (u32)(g % k);
+        if (p >= counts[b]) continue;
+        const KI me = lists[g];
+        if (ki_less(best, me)) continue;
+        u32 part = 0;
+        for (u32 b2 = lane; b2 < nblk; b2 += 32) {
+            if (b2 == b) continue;
+            const u32 cb = counts[b2];
+            if (cb == 0) continue;
+            const KI *L = lists + (size_t)b2 * k;
+            if (!ki_less(L[0], me)) continue;              // nothing smaller in that list
+            u32 lo = 1, hi = cb;                           // number of entries smaller than me
+            while (lo < hi) {
+                const u32 mid = (lo + hi) >> 1;
+                if (ki_less(L[mid], me)) lo = mid + 1; else hi = mid;
+            }
+            part += lo;
+        }
+        for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, d);
+        const u32 rank = p + part;
+        if (lane == 0 && rank < k) {
+            const double v = dec(me.key);
+            idx_out[rank] = me.idx;
+            key_out[rank] = negate_out ? 0.0 - v : v;
+        }
+    }
 }
 
-// workspace: ticket, per-block front sizes and overflow flags, per-block fronts
-template <class Src>
-__global__ void __launch_bounds__(SEL_THREADS) k_pareto(Src src, Range r, u32 *ticket, u32 *sizes, P3 *partial,
-                                                        u64 *idx_out, u32 out_cap, u32 *count_out) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    P3 *buf = (P3 *)smem_raw;
-    __shared__ u32 cnt;
+// ---- Pareto kernels --------------------------------------------------------------------------------
+
+// Store this block's front; the block that arrives last folds all fronts into the answer.  A prefix
+// sum over the front sizes turns them into one flat list, so the number of collective steps
+// depends on the number of points, not on the number of blocks.
+__device__ void pareto_store_and_fold(ParetoAcc &acc, u32 block, u32 nblk, u32 *ticket, u32 *sizes, P3 *partial,
+                                      u64 *idx_out, u32 out_cap, u32 *count_out) {
     __shared__ u32 last_flag;
-    __shared__ __align__(8) u32 scratch[64];
-    ParetoAcc acc;
-    acc.init(buf, &cnt, scratch);
-    const u64 tiles = (r.count + blockDim.x - 1) / blockDim.x;
-    for (u64 tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-        const u64 j = tile * blockDim.x + threadIdx.x;
-        double a = 0.0, b = 0.0;
-        const bool ok = j < r.count && src.get(j, r.first + j, a, b);
-        P3 it;
-        it.x = enc(a); it.y = enc(b); it.idx = r.first + j;
-        acc.push(ok, it);
-    }
-    acc.merge();
-    P3 *mine = partial + (size_t)blockIdx.x * GUIDE_PARETO_MAX;
-    for (u32 i = threadIdx.x; i < acc.nf; i += blockDim.x) mine[i] = buf[i];
-    if (threadIdx.x == 0) sizes[blockIdx.x] = acc.nf | (acc.overflow ? 0x80000000u : 0u);
+    __shared__ u32 pre[SEL_MAX_BLOCKS + 1];
+    __shared__ u32 wsum[SEL_THREADS / 32];
+    acc.finish();
+    P3 *mine = partial + (size_t)block * GUIDE_PARETO_MAX;
+    for (u32 i = threadIdx.x; i < acc.nf; i += blockDim.x) mine[i] = acc.buf[i];
+    if (threadIdx.x == 0) sizes[block] = acc.nf | (acc.overflow ? 0x80000000u : 0u);
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) last_flag = (atomicAdd(ticket, 1) == gridDim.x - 1);
+    if (threadIdx.x == 0) last_flag = (atomicAdd(ticket, 1) == nblk - 1);
     __syncthreads();
     if (!last_flag) return;
     __threadfence();
-    acc.init(buf, &cnt, scratch);
-    bool overflow = false;
-    for (u32 blk = 0; blk < gridDim.x; blk++) {
-        const u32 sz = __ldcg(sizes + blk);
-        overflow |= (sz >> 31) != 0;
-        const u32 n = sz & 0x7FFFFFFFu;
-        const P3 *theirs = partial + (size_t)blk * GUIDE_PARETO_MAX;
-        for (u32 base = 0; base < n; base += blockDim.x) {
-            const u32 i = base + threadIdx.x;
-            P3 it; it.x = KEY_MAX; it.y = KEY_MAX; it.idx = KEY_MAX;
-            if (i < n) {      // written by other blocks: read through L2
-                const u64 *w = reinterpret_cast<const u64 *>(theirs + i);
-                it.x = __ldcg(w); it.y = __ldcg(w + 1); it.idx = __ldcg(w + 2);
-            }
-            acc.push(i < n, it);
-        }
+    // exclusive prefix sum of the front sizes (up to SEL_MAX_BLOCKS of them) with any block size
+    const u32 per = (SEL_MAX_BLOCKS + blockDim.x - 1) / blockDim.x;
+    u32 local = 0;
+    bool ovf = false;
+    for (u32 u = 0; u < per; u++) {
+        const u32 bi = threadIdx.x * per + u;
+        const u32 sz = bi < nblk ? __ldcg(sizes + bi) : 0u;
+        ovf |= (sz >> 31) != 0;
+        local += sz & 0x7FFFFFFFu;
     }
-    acc.merge();
+    u32 incl = local;
+    const u32 lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (u32 d = 1; d < 32; d <<= 1) {
+        const u32 v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= d) incl += v;
+    }
+    if (lane == 31) wsum[warp] = incl;
+    bool overflow = __syncthreads_or(ovf) != 0;
+    u32 run = incl - local;
+    for (u32 w2 = 0; w2 < warp; w2++) run += wsum[w2];
+    for (u32 u = 0; u < per; u++) {
+        const u32 bi = threadIdx.x * per + u;
+        if (bi < SEL_MAX_BLOCKS) pre[bi] = run;
+        run += bi < nblk ? (__ldcg(sizes + bi) & 0x7FFFFFFFu) : 0u;
+    }
+    if (threadIdx.x == blockDim.x - 1) pre[SEL_MAX_BLOCKS] = run;
+    acc.init(acc.buf, acc.cnt, acc.scratch);            // includes a barrier: pre[] is complete
+    const u32 total = pre[SEL_MAX_BLOCKS];
+    u32 since = 0;
+    for (u32 base = 0; base < total; base += blockDim.x) {
+        const u32 i = base + threadIdx.x;
+        P3 it; it.x = KEY_MAX; it.y = KEY_MAX; it.idx = KEY_MAX;
+        if (i < total) {
+            u32 lo = 0, hi = SEL_MAX_BLOCKS;            // last block index whose offset is <= i
+            while (lo < hi) {
+                const u32 mid = (lo + hi + 1) >> 1;
+                if (pre[mid] <= i) lo = mid; else hi = mid - 1;
+            }
+            // written by other blocks: read through L2
+            const u64 *w = reinterpret_cast<const u64 *>(partial + (size_t)lo * GUIDE_PARETO_MAX + (i - pre[lo]));
+            it.x = __ldcg(w); it.y = __ldcg(w + 1); it.idx = __ldcg(w + 2);
+        }
+        acc.offer(i < total, it);
+        if (++since == CHECK_EVERY) { acc.checkpoint(); since = 0; }
+    }
+    acc.finish();
     overflow |= acc.overflow;
-    for (u32 i = threadIdx.x; i < acc.nf && i < out_cap; i += blockDim.x) idx_out[i] = buf[i].idx;
+    for (u32 i = threadIdx.x; i < acc.nf && i < out_cap; i += blockDim.x) idx_out[i] = acc.buf[i].idx;
     if (threadIdx.x == 0) *count_out = overflow ? 0xFFFFFFFFu : acc.nf;
+}
+
+template <class Src>
+__global__ void __launch_bounds__(SEL_THREADS) k_pareto_scan(Src src, Range r, u32 *ticket, u32 *sizes, P3 *partial,
+                                                             u64 *idx_out, u32 out_cap, u32 *count_out) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ u32 cnt;
+    __shared__ __align__(8) u32 scratch[64];
+    ParetoAcc acc;
+    acc.init((P3 *)smem_raw, &cnt, scratch);
+    constexpr int ITEMS = Src::ITEMS;
+    constexpr u32 ROUNDS = CHECK_EVERY / ITEMS;
+    const u64 span = (u64)ITEMS * blockDim.x;
+    const u64 tiles = (r.count + span - 1) / span;
+    u32 since = 0;
+    for (u64 tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+        bool ok[ITEMS];
+        P3 it[ITEMS];
+#pragma unroll
+        for (int u = 0; u < ITEMS; u++) {
+            const u64 j = tile * span + (u64)u * blockDim.x + threadIdx.x;
+            const u64 jc = j < r.count ? j : r.count - 1;          // keep the loads in range
+            double a = 0.0, b = 0.0;
+            ok[u] = src.get(jc, r.first + jc, a, b) && j < r.count;
+            it[u].x = enc(a); it[u].y = enc(b); it[u].idx = r.first + j;
+        }
+        if (tile == blockIdx.x) {
+            // first round: one offer per checkpoint, so the first front comes from a small sort
+#pragma unroll
+            for (int u = 0; u < ITEMS; u++) { acc.offer(ok[u], it[u]); acc.checkpoint(); }
+            continue;
+        }
+#pragma unroll
+        for (int u = 0; u < ITEMS; u++) acc.offer(ok[u], it[u]);
+        if (++since == ROUNDS) { acc.checkpoint(); since = 0; }
+    }
+    pareto_store_and_fold(acc, blockIdx.x, gridDim.x, ticket, sizes, partial, idx_out, out_cap, count_out);
+}
+
+template <int TIME_SUM>
+__global__ void __launch_bounds__(SEL_THREADS, 2)
+k_pareto_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, Cons c, int xm, int ym, u32 *ticket,
+               u32 *sizes, P3 *partial, u64 *idx_out, u32 out_cap, u32 *count_out) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ u32 cnt;
+    __shared__ __align__(8) u32 scratch[64];
+    ParetoAcc acc;
+    acc.init((P3 *)smem_raw, &cnt, scratch);
+    u32 since = CHECK_EVERY - 1;          // the first offer is followed by a checkpoint: early front
+    tiled_visit<TIME_SUM>(s, r, tp_model, hf_chunk, tiles_per_mb, [&](bool valid, u64 idx, const Metrics &m) {
+        double a = 0.0, b = 0.0;
+        const bool ok = valid && fused_pick(m, c, xm, ym, a, b);
+        P3 it;
+        it.x = enc(a); it.y = enc(b); it.idx = idx;
+        acc.offer(ok, it);
+        if (++since == CHECK_EVERY) { acc.checkpoint(); since = 0; }
+    });
+    pareto_store_and_fold(acc, blockIdx.y * gridDim.x + blockIdx.x, gridDim.x * gridDim.y, ticket, sizes, partial, idx_out,
+                          out_cap, count_out);
 }
 
 // ---- host side -----------------------------------------------------------------------------------------
 
-static u32 topk_cap(u32 k) { return k <= 256 ? 512u : 2048u; }
+// top-k workspace: 256 B header | counts u32[max_blocks] | lists KI[max_blocks][k]
+static size_t topk_lists_offset(u32 max_blocks) { return 256 + ((size_t)max_blocks * 4 + 255) / 256 * 256; }
 
-size_t topk_workspace_bytes(u32 k) { return 256 + (size_t)SEL_MAX_BLOCKS * k * sizeof(KI); }
+size_t topk_workspace_bytes(u32 k) { return topk_lists_offset(SEL_MAX_BLOCKS) + (size_t)SEL_MAX_BLOCKS * k * sizeof(KI); }
 size_t pareto_workspace_bytes() {
     return 256 + (size_t)SEL_MAX_BLOCKS * sizeof(u32) + (size_t)SEL_MAX_BLOCKS * GUIDE_PARETO_MAX * sizeof(P3);
 }
@@ -383,58 +590,108 @@ static Cons make_cons(const guide_constraints &c) {
     return k;
 }
 
-static u32 grid_for(u64 count, u32 blocks_per_sm) {
-    const u64 tiles = (count + SEL_THREADS - 1) / SEL_THREADS;
-    u64 g = std::min<u64>((u64)num_sms() * blocks_per_sm, SEL_MAX_BLOCKS);
+static u32 grid_for(u64 count, u32 items, u32 blocks_per_sm, u32 max_blocks) {
+    const u64 tiles = (count + (u64)SEL_THREADS * items - 1) / ((u64)SEL_THREADS * items);
+    u64 g = std::min<u64>((u64)num_sms() * blocks_per_sm, max_blocks);
     g = std::min<u64>(g, std::max<u64>(tiles, 1));
     return (u32)g;
 }
 
-template <class Src>
-static int run_topk(const Src &src, Range r, u32 k, int negate, u64 *idx_out, double *key_out, u32 *count_out,
-                    void *ws, cudaStream_t st) {
-    const u32 cap = topk_cap(k);
-    const u32 grid = grid_for(r.count, 4);
-    GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
-    k_topk<Src><<<grid, SEL_THREADS, cap * sizeof(KI), st>>>(src, r, k, cap, (u32 *)ws, (KI *)((char *)ws + 256), negate,
-                                                             idx_out, key_out, count_out);
+// can the fused selection walk the space in tiled order (grid bounded by the workspace's block count)?
+static bool fused_tiled(const DSpace &s, Range r, TileGeom *g) {
+    const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
+    return r.count * 2 >= total && tiled_geometry(s, SEL_MAX_BLOCKS, SEL_MAX_BLOCKS, g);
+}
+
+template <class K>
+static int allow_smem(K kernel, size_t bytes) {
+    GUIDE_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    return GUIDE_OK;
+}
+
+static int run_topk_merge(u32 nblk, u32 k, int negate, u32 *counts, KI *lists, u64 *idx_out, double *key_out,
+                          u32 *count_out, cudaStream_t st) {
+    const u64 cand = (u64)nblk * k;                      // one warp per candidate, a few candidates per warp
+    const u64 want = (cand + (SEL_THREADS / 32) * 4 - 1) / ((SEL_THREADS / 32) * 4);
+    const u32 grid = (u32)std::min<u64>(std::max<u64>(want, 1), (u64)num_sms() * 8);
+    k_topk_merge<<<grid, SEL_THREADS, 0, st>>>(nblk, k, counts, lists, negate,
+                                                                                       idx_out, key_out, count_out);
     GUIDE_CUDA(cudaGetLastError());
     return GUIDE_OK;
 }
 
 template <class Src>
-static int run_pareto(const Src &src, Range r, u64 *idx_out, u32 cap, u32 *count_out, void *ws, cudaStream_t st) {
-    const size_t smem = (size_t)PARETO_CAP * sizeof(P3);
-    static bool configured[64] = {};      // per kernel instantiation and device
-    int dev = 0;
-    GUIDE_CUDA(cudaGetDevice(&dev));
-    if (dev >= 64 || !configured[dev]) {
-        GUIDE_CUDA(cudaFuncSetAttribute(k_pareto<Src>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        if (dev < 64) configured[dev] = true;
-    }
-    const u32 grid = grid_for(r.count, 2);
-    GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
-    u32 *sizes = (u32 *)((char *)ws + 256);
-    P3 *partial = (P3 *)((char *)ws + 256 + (size_t)SEL_MAX_BLOCKS * sizeof(u32));
-    k_pareto<Src><<<grid, SEL_THREADS, smem, st>>>(src, r, (u32 *)ws, sizes, partial, idx_out, cap, count_out);
+static int run_topk_scan(const Src &src, Range r, u32 k, int negate, u32 max_blocks, unsigned char *ws, u64 *idx_out,
+                         double *key_out, u32 *count_out, cudaStream_t st) {
+    u32 *counts = (u32 *)(ws + 256);
+    KI *lists = (KI *)(ws + topk_lists_offset(max_blocks));
+    const u32 grid = grid_for(r.count, Src::ITEMS, 4, max_blocks);
+    k_topk_scan<Src><<<grid, SEL_THREADS, TOPK_CAP * sizeof(KI), st>>>(src, r, k, counts, lists);
     GUIDE_CUDA(cudaGetLastError());
-    return GUIDE_OK;
+    return run_topk_merge(grid, k, negate, counts, lists, idx_out, key_out, count_out, st);
+}
+
+template <int TIME_SUM>
+static int run_topk_tiled(const DSpace &s, Range r, const TileGeom &g, int tp_model, const Cons &c, int key, u32 k,
+                          unsigned char *ws, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st) {
+    u32 *counts = (u32 *)(ws + 256);
+    KI *lists = (KI *)(ws + topk_lists_offset(SEL_MAX_BLOCKS));
+    const dim3 grid(g.gx, g.splits);
+    k_topk_tiled<TIME_SUM><<<grid, g.threads, TOPK_CAP * sizeof(KI), st>>>(s, r, tp_model, g.hf_chunk, g.tiles_per_mb, c,
+                                                                          key, k, counts, lists);
+    GUIDE_CUDA(cudaGetLastError());
+    return run_topk_merge(g.gx * g.splits, k, key == GUIDE_THROUGHPUT, counts, lists, idx_out, key_out, count_out, st);
 }
 
 int launch_topk(const DSpace &s, Range r, const guide_outputs *mat, int time_model, int tp_model,
                 const guide_constraints &c, int key, u32 k, u64 *idx_out, double *key_out, u32 *count_out,
                 void *ws, cudaStream_t st) {
     const int negate = key == GUIDE_THROUGHPUT;
+    unsigned char *w = (unsigned char *)ws;
     if (mat) {
         MatSource src{*mat, make_cons(c), key, -1};
-        return run_topk(src, r, k, negate, idx_out, key_out, count_out, ws, st);
+        return run_topk_scan(src, r, k, negate, SEL_MAX_BLOCKS, w, idx_out, key_out, count_out, st);
     }
+    TileGeom g;
+    if (fused_tiled(s, r, &g))
+        return time_model ? run_topk_tiled<1>(s, r, g, tp_model, make_cons(c), key, k, w, idx_out, key_out, count_out, st)
+                          : run_topk_tiled<0>(s, r, g, tp_model, make_cons(c), key, k, w, idx_out, key_out, count_out, st);
     if (time_model) {
         FusedSource<1> src{s, make_cons(c), key, -1, tp_model};
-        return run_topk(src, r, k, negate, idx_out, key_out, count_out, ws, st);
+        return run_topk_scan(src, r, k, negate, SEL_MAX_BLOCKS, w, idx_out, key_out, count_out, st);
     }
     FusedSource<0> src{s, make_cons(c), key, -1, tp_model};
-    return run_topk(src, r, k, negate, idx_out, key_out, count_out, ws, st);
+    return run_topk_scan(src, r, k, negate, SEL_MAX_BLOCKS, w, idx_out, key_out, count_out, st);
+}
+
+template <class Src>
+static int run_pareto_scan(const Src &src, Range r, u64 *idx_out, u32 cap, u32 *count_out, void *ws, cudaStream_t st) {
+    const size_t smem = (size_t)PARETO_CAP * sizeof(P3);
+    int rc = allow_smem(k_pareto_scan<Src>, smem);
+    if (rc) return rc;
+    const u32 grid = grid_for(r.count, Src::ITEMS, 2, SEL_MAX_BLOCKS);
+    GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
+    u32 *sizes = (u32 *)((char *)ws + 256);
+    P3 *partial = (P3 *)((char *)ws + 256 + (size_t)SEL_MAX_BLOCKS * sizeof(u32));
+    k_pareto_scan<Src><<<grid, SEL_THREADS, smem, st>>>(src, r, (u32 *)ws, sizes, partial, idx_out, cap, count_out);
+    GUIDE_CUDA(cudaGetLastError());
+    return GUIDE_OK;
+}
+
+template <int TIME_SUM>
+static int run_pareto_tiled(const DSpace &s, Range r, const TileGeom &g, int tp_model, const Cons &c, int xm, int ym,
+                            u64 *idx_out, u32 cap, u32 *count_out, void *ws, cudaStream_t st) {
+    const size_t smem = (size_t)PARETO_CAP * sizeof(P3);
+    int rc = allow_smem(k_pareto_tiled<TIME_SUM>, smem);
+    if (rc) return rc;
+    GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
+    u32 *sizes = (u32 *)((char *)ws + 256);
+    P3 *partial = (P3 *)((char *)ws + 256 + (size_t)SEL_MAX_BLOCKS * sizeof(u32));
+    const dim3 grid(g.gx, g.splits);
+    k_pareto_tiled<TIME_SUM><<<grid, g.threads, smem, st>>>(s, r, tp_model, g.hf_chunk, g.tiles_per_mb, c, xm, ym,
+                                                           (u32 *)ws, sizes, partial, idx_out, cap, count_out);
+    GUIDE_CUDA(cudaGetLastError());
+    return GUIDE_OK;
 }
 
 int launch_pareto(const DSpace &s, Range r, const guide_outputs *mat, int time_model, int tp_model,
@@ -442,24 +699,28 @@ int launch_pareto(const DSpace &s, Range r, const guide_outputs *mat, int time_m
                   cudaStream_t st) {
     if (mat) {
         MatSource src{*mat, make_cons(c), xm, ym};
-        return run_pareto(src, r, idx_out, cap, count_out, ws, st);
+        return run_pareto_scan(src, r, idx_out, cap, count_out, ws, st);
     }
+    TileGeom g;
+    if (fused_tiled(s, r, &g))
+        return time_model ? run_pareto_tiled<1>(s, r, g, tp_model, make_cons(c), xm, ym, idx_out, cap, count_out, ws, st)
+                          : run_pareto_tiled<0>(s, r, g, tp_model, make_cons(c), xm, ym, idx_out, cap, count_out, ws, st);
     if (time_model) {
         FusedSource<1> src{s, make_cons(c), xm, ym, tp_model};
-        return run_pareto(src, r, idx_out, cap, count_out, ws, st);
+        return run_pareto_scan(src, r, idx_out, cap, count_out, ws, st);
     }
     FusedSource<0> src{s, make_cons(c), xm, ym, tp_model};
-    return run_pareto(src, r, idx_out, cap, count_out, ws, st);
+    return run_pareto_scan(src, r, idx_out, cap, count_out, ws, st);
 }
 
 // ---- top-k over materialised metrics with library-owned scratch ----------------------------------
 //
-// Same kernel as launch_topk, but the per-block partial results live in a fixed device array that
+// Same kernels as launch_topk, but the per-block candidate lists live in a fixed device array that
 // is part of the library image instead of a caller-supplied workspace, for callers that are not
 // allowed to allocate device memory.  The array bounds k and the grid; every call reuses it.
 
 static constexpr u32 NOALLOC_BLOCKS = 256;                     // grid cap of this variant
-static constexpr size_t NOALLOC_SCRATCH_BYTES = 256 + (size_t)NOALLOC_BLOCKS * GUIDE_NOALLOC_TOPK_MAX * sizeof(KI);
+static constexpr size_t NOALLOC_SCRATCH_BYTES = 256 + (size_t)NOALLOC_BLOCKS * 4 + (size_t)NOALLOC_BLOCKS * GUIDE_NOALLOC_TOPK_MAX * sizeof(KI);
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
 
@@ -487,16 +748,12 @@ int launch_topk_noalloc(Range r, const guide_outputs &mat, const guide_constrain
     unsigned char *scratch = nullptr;
     const int rc = noalloc_scratch_address(&scratch);
     if (rc) return rc;
+    static_assert(256 + NOALLOC_BLOCKS * 4 == 1280, "list offset below assumes a 256-byte multiple");
     MatSource src{mat, make_cons(c), key, -1};
-    const u32 cap = topk_cap(k);
-    const u32 grid = std::min<u32>(grid_for(r.count, 4), NOALLOC_BLOCKS);
-    // the array still holds the previous call's ticket and candidates: the ticket must restart at 0,
-    // the candidate slots are all rewritten by the blocks of this launch before they are read
-    GUIDE_CUDA(cudaMemsetAsync(scratch, 0, 256, st));
-    k_topk<MatSource><<<grid, SEL_THREADS, cap * sizeof(KI), st>>>(src, r, k, cap, (u32 *)scratch, (KI *)(scratch + 256),
-                                                                   key == GUIDE_THROUGHPUT, idx_out, key_out, count_out);
-    GUIDE_CUDA(cudaGetLastError());
-    return GUIDE_OK;
+    // The array still holds the previous call's counts and lists.  Nothing has to start at zero:
+    // every block of this launch writes its count and its list before the merge kernel, which
+    // follows on the same stream, reads them, and the merge reads only this launch's blocks.
+    return run_topk_scan(src, r, k, key == GUIDE_THROUGHPUT, NOALLOC_BLOCKS, scratch, idx_out, key_out, count_out, st);
 }
 
 }  // namespace guide

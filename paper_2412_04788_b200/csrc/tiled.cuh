@@ -1,0 +1,108 @@
+// Tiled walk over a closed-form space, shared by the evaluation kernel and the fused selection
+// kernels.
+//
+// The integer task table of a config depends on (model, batch, TP, lengths) only, and within one
+// (model, batch) the (TP, length) positions are the fastest-running part of the config index.  A
+// thread therefore owns one (model, batch, TP, length) point, builds both stage tables once, and
+// walks a chunk of the hardware x framework pairs, which are the only things the roofline
+// evaluation needs beyond the table.  A warp's 32 threads hold 32 consecutive config indices for
+// every pair, so whatever is stored per config goes out as 256-byte runs.
+#pragma once
+#include "model.cuh"
+
+namespace guide {
+
+struct Range { u64 first, count; };
+
+struct TileGeom {
+    u32 threads;        // block size (multiple of 32, <= 256)
+    u32 tiles_per_mb;   // blocks along the (TP, length) plane of one (model, batch)
+    u32 gx;             // n_models * n_batch * tiles_per_mb
+    u32 splits;         // chunks of the hardware x framework axis (grid.y)
+    u32 hf_chunk;       // pairs per chunk
+};
+
+// emit(valid, idx, metrics) is called by every thread of the block exactly hf_chunk times, valid or
+// not, so emit may contain block-wide barriers.
+template <int TIME_SUM, class Emit>
+__device__ __forceinline__ void tiled_visit(const DSpace &s, const Range &r, int tp_model, u32 hf_chunk,
+                                            u32 tiles_per_mb, Emit &&emit) {
+    const u32 n_tl = s.n_t * s.n_l;
+    const u32 n_hf = s.n_h * s.n_f;
+    // blockIdx.x -> (model, batch, tile of the (TP, length) plane); blockIdx.y -> chunk of pairs
+    const u32 tile = blockIdx.x % tiles_per_mb;
+    const u32 mb = blockIdx.x / tiles_per_mb;
+    const u32 bpos = mb % s.n_b, mpos = mb / s.n_b;
+    const u32 tl_raw = tile * blockDim.x + threadIdx.x;
+    const bool active = tl_raw < n_tl;
+    const u32 tl = active ? tl_raw : n_tl - 1;
+    const u32 tpos = tl / s.n_l, lpos = tl % s.n_l;
+    const u32 hf0 = blockIdx.y * hf_chunk;
+
+    const DModel m = s.models[mpos];
+    const u32 t = s.tp[tpos], b = s.batch[bpos];
+    const uint2 pr = s.pairs[lpos];
+    const u32 lin = pr.x, lout = pr.y, n = lout - 1;
+    const MemInfo mi = mem_info(m, t);
+    const u32 tt = tp_model ? 1u : t;
+    const double lf = log2_rule_factor(t, tp_model);
+    const double Nd = (double)m.N;
+
+    TaskTab kp, kd;
+    const u64 Tp = (u64)b * lin;
+    build_fixed_tasks(m, tt, Tp, b, 1, kp);
+    build_attn_tasks(m, tt, Tp, Tp * lin, Tp, kp);
+    {
+        const u32 nn = n > 0 ? n : 1;          // a table is built either way; unused when n == 0
+        const u64 Td = (u64)b * nn;
+        const u64 ctx = (u64)b * ((u64)nn * lin + ((u64)nn * (nn + 1)) / 2);
+        build_fixed_tasks(m, tt, Td, Td, nn, kd);
+        build_attn_tasks(m, tt, Td, ctx, ctx, kd);
+    }
+    // index of this thread's config for pair (h, f): ((((m n_h + h) n_f + f) n_b + b) n_t n_l) + tl
+    const u64 stride_hf = (u64)s.n_b * n_tl;
+    const u64 base = ((u64)mpos * n_hf) * stride_hf + (u64)bpos * n_tl + tl;
+
+    for (u32 i = 0; i < hf_chunk; i++) {
+        const u32 hf = hf0 + i;
+        const u64 idx = base + (u64)hf * stride_hf;
+        const bool valid = active && hf < n_hf && idx >= r.first && idx - r.first < r.count;
+        Metrics out;
+        if (valid) {
+            const DRate rt = s.rates[hf];
+            out.status = closed_form_feasibility(m, rt, mi, t, b, lin, lout, out.bmax);
+            if (out.status) set_infeasible(out);
+            else {
+                const double t_pre = eval_phase<TIME_SUM>(kp, rt, Nd, lf);
+                const double t_dec = n > 0 ? eval_phase<TIME_SUM>(kd, rt, Nd, lf) : 0.0;
+                closed_form_metrics(t_pre, t_dec, b, n, t, rt.price, out);
+            }
+        } else {
+            out.status = 0xFF;
+        }
+        emit(valid, idx, out);
+    }
+}
+
+// Host side: block and grid shape.  want_blocks steers how finely the pair axis is split (longer
+// chunks amortise the table building over more configs); max_blocks bounds the whole grid.
+// Returns false when the space does not suit the tiled walk.
+inline bool tiled_geometry(const DSpace &s, u64 want_blocks, u64 max_blocks, TileGeom *g) {
+    const u32 n_tl = s.n_t * s.n_l, n_hf = s.n_h * s.n_f;
+    if (n_tl < 32) return false;
+    g->threads = n_tl >= 256 ? 256 : ((n_tl + 31) / 32) * 32;
+    g->tiles_per_mb = (n_tl + g->threads - 1) / g->threads;
+    const u64 gx = (u64)s.n_m * s.n_b * g->tiles_per_mb;
+    if (gx > 0x7FFFFFFFull || gx > max_blocks) return false;
+    u64 splits = (want_blocks + gx - 1) / gx;
+    if (splits < 1) splits = 1;
+    if (splits > n_hf) splits = n_hf;
+    if (gx * splits > max_blocks) splits = max_blocks / gx;
+    if (splits > 65535) splits = 65535;
+    g->hf_chunk = (u32)((n_hf + splits - 1) / splits);
+    g->splits = (n_hf + g->hf_chunk - 1) / g->hf_chunk;
+    g->gx = (u32)gx;
+    return true;
+}
+
+}  // namespace guide
