@@ -20,8 +20,8 @@ namespace guide {
 static constexpr u32 SEL_THREADS = 256;
 static constexpr u32 SEL_MAX_BLOCKS = 1024;
 static constexpr u32 PARETO_CAP = 4096;          // shared-memory items per block
-static constexpr u32 TOPK_CAP = 2048;            // shared-memory candidates per block
-static constexpr u32 CHECK_EVERY = 4;            // appends per thread between two checkpoints
+static constexpr u32 TOPK_CAP = 4096;            // shared-memory candidates per block
+static constexpr u32 MAX_BUDGET = 16;            // most appends per thread between two checkpoints
 static constexpr u64 KEY_MAX = ~0ull;
 
 // order-preserving map double -> u64 (after -0.0 -> +0.0)
@@ -148,11 +148,14 @@ struct TopKAcc {
     u32 *cnt;         // shared append cursor
     u32 k;
     u32 c;            // buffered count at the last checkpoint, identical in every thread
+    u32 budget;       // appends each thread may still make before the next checkpoint
+    u32 ramp;         // checkpoint spacing: 1, 2, 4, ... MAX_BUDGET appends per thread
     bool has_thr;
     KI thr;
 
     __device__ void init(KI *b, u32 *cn, u32 k_) {
         buf = b; cnt = cn; k = k_; c = 0; has_thr = false; thr.key = KEY_MAX; thr.idx = KEY_MAX;
+        budget = 1; ramp = 1;
         if (threadIdx.x == 0) *cnt = 0;
         __syncthreads();
     }
@@ -167,21 +170,25 @@ struct TopKAcc {
         if (threadIdx.x == 0) *cnt = c;
         __syncthreads();
     }
-    // No barrier.  Between two checkpoints a thread may offer at most CHECK_EVERY items; the
-    // checkpoint keeps c + CHECK_EVERY * blockDim <= TOPK_CAP, so the slot is always in range.
-    __device__ __forceinline__ void offer(bool ok, const KI &it) {
-        if (ok && (!has_thr || ki_less(it, thr))) buf[atomicAdd(cnt, 1)] = it;
-    }
-    // collective.  Compacts when the buffer could overflow before the next checkpoint, and early
+    // Collective.  Compacts when the buffer could overflow before the next checkpoint, and early
     // while that is cheap: as soon as k candidates exist (first threshold), then whenever about k
-    // more have slipped under the stale threshold.  Small sorts cost little; a fresh threshold
-    // keeps almost everything out.
+    // more have slipped under the stale threshold.  Checkpoints start one append apart, so the
+    // first threshold comes from a small sort, and thin out to MAX_BUDGET appends apart.
     __device__ void checkpoint() {
         __syncthreads();
         c = *cnt;
         __syncthreads();                       // nobody appends before everyone has read the count
+        if (ramp < MAX_BUDGET) ramp *= 2;
         const u32 early = has_thr ? 2 * k + blockDim.x : k;
-        if (c + CHECK_EVERY * blockDim.x > TOPK_CAP || c >= early) compact();
+        if (c >= early || c + ramp * blockDim.x > TOPK_CAP) compact();
+        budget = min(ramp, (TOPK_CAP - c) / blockDim.x);
+    }
+    // Collective in the sense that every thread of the block calls it the same number of times; a
+    // barrier happens only when the budget runs out.  The slot is always in range because the
+    // checkpoint leaves room for budget * blockDim appends.
+    __device__ __forceinline__ void push(bool ok, const KI &it) {
+        if (ok && (!has_thr || ki_less(it, thr))) buf[atomicAdd(cnt, 1)] = it;
+        if (--budget == 0) checkpoint();
     }
     __device__ void finish() {
         __syncthreads();
@@ -198,10 +205,13 @@ struct ParetoAcc {
     u32 *cnt;
     u32 *scratch;     // shared, 2 * 32 words
     u32 nf, c;
+    u32 budget, ramp;
     bool overflow;
+    bool lazy;        // folding fronts: incoming points are mostly keepers, merge only when the buffer fills
 
-    __device__ void init(P3 *b, u32 *cn, u32 *sc) {
-        buf = b; cnt = cn; scratch = sc; nf = 0; c = 0; overflow = false;
+    __device__ void init(P3 *b, u32 *cn, u32 *sc, bool lazy_ = false) {
+        buf = b; cnt = cn; scratch = sc; nf = 0; c = 0; overflow = false; lazy = lazy_;
+        budget = lazy_ ? (PARETO_CAP / 2) / blockDim.x : 1; ramp = lazy_ ? MAX_BUDGET : 1;
         if (threadIdx.x == 0) *cnt = 0;
         __syncthreads();
     }
@@ -273,18 +283,22 @@ struct ParetoAcc {
         if (threadIdx.x == 0) *cnt = out;
         __syncthreads();
     }
-    // no barrier; at most CHECK_EVERY offers per thread between checkpoints
-    __device__ __forceinline__ void offer(bool ok, const P3 &it) {
-        if (ok && !beaten(it)) buf[atomicAdd(cnt, 1)] = it;
-    }
+    // Collective.  Merges when the buffer could overflow before the next checkpoint and, unless
+    // lazy, as soon as there is anything while no front exists yet (until then nothing is
+    // filtered) and whenever a block's worth of points has slipped past the stale front.
     __device__ void checkpoint() {
         __syncthreads();
         c = *cnt;
         __syncthreads();
-        // merge when the buffer could overflow before the next checkpoint, as soon as there is
-        // anything while no front exists yet (until then nothing is filtered), and whenever a
-        // block's worth of points has slipped past the stale front
-        if (c + CHECK_EVERY * blockDim.x > PARETO_CAP || (nf == 0 && c > 0) || c >= nf + blockDim.x) merge();
+        if (ramp < MAX_BUDGET) ramp *= 2;
+        const bool early = !lazy && ((nf == 0 && c > 0) || c >= nf + blockDim.x);
+        if (early || c + ramp * blockDim.x > PARETO_CAP) merge();
+        budget = min(ramp, (PARETO_CAP - c) / blockDim.x);
+    }
+    // every thread of the block calls it the same number of times; a barrier only when the budget runs out
+    __device__ __forceinline__ void push(bool ok, const P3 &it) {
+        if (ok && !beaten(it)) buf[atomicAdd(cnt, 1)] = it;
+        if (--budget == 0) checkpoint();
     }
     __device__ void finish() {
         __syncthreads();
@@ -321,10 +335,8 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_scan(Src src, Range r, u32
     TopKAcc acc;
     acc.init((KI *)smem_raw, &cnt, k);
     constexpr int ITEMS = Src::ITEMS;
-    constexpr u32 ROUNDS = CHECK_EVERY / ITEMS;          // tiles between checkpoints
     const u64 span = (u64)ITEMS * blockDim.x;
     const u64 tiles = (r.count + span - 1) / span;
-    u32 since = 0;
     for (u64 tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
         bool ok[ITEMS];
         KI it[ITEMS];
@@ -336,15 +348,8 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_scan(Src src, Range r, u32
             ok[u] = src.get(jc, r.first + jc, a, b) && j < r.count;
             it[u].key = enc(a); it[u].idx = r.first + j;
         }
-        if (tile == blockIdx.x) {
-            // first round: one offer per checkpoint, so the first threshold comes from a small sort
 #pragma unroll
-            for (int u = 0; u < ITEMS; u++) { acc.offer(ok[u], it[u]); acc.checkpoint(); }
-            continue;
-        }
-#pragma unroll
-        for (int u = 0; u < ITEMS; u++) acc.offer(ok[u], it[u]);
-        if (++since == ROUNDS) { acc.checkpoint(); since = 0; }
+        for (int u = 0; u < ITEMS; u++) acc.push(ok[u], it[u]);
     }
     topk_store(acc, blockIdx.x, k, counts, lists);
 }
@@ -356,14 +361,12 @@ k_topk_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, Co
     __shared__ u32 cnt;
     TopKAcc acc;
     acc.init((KI *)smem_raw, &cnt, k);
-    u32 since = CHECK_EVERY - 1;          // the first offer is followed by a checkpoint: early threshold
     tiled_visit<TIME_SUM>(s, r, tp_model, hf_chunk, tiles_per_mb, [&](bool valid, u64 idx, const Metrics &m) {
         double a = 0.0, b;
         const bool ok = valid && fused_pick(m, c, key, -1, a, b);
         KI it;
         it.key = enc(a); it.idx = idx;
-        acc.offer(ok, it);
-        if (++since == CHECK_EVERY) { acc.checkpoint(); since = 0; }
+        acc.push(ok, it);
     });
     topk_store(acc, blockIdx.y * gridDim.x + blockIdx.x, k, counts, lists);
 }
@@ -489,9 +492,8 @@ __device__ void pareto_store_and_fold(ParetoAcc &acc, u32 block, u32 nblk, u32 *
         run += bi < nblk ? (__ldcg(sizes + bi) & 0x7FFFFFFFu) : 0u;
     }
     if (threadIdx.x == blockDim.x - 1) pre[SEL_MAX_BLOCKS] = run;
-    acc.init(acc.buf, acc.cnt, acc.scratch);            // includes a barrier: pre[] is complete
+    acc.init(acc.buf, acc.cnt, acc.scratch, true);      // includes a barrier: pre[] is complete
     const u32 total = pre[SEL_MAX_BLOCKS];
-    u32 since = 0;
     for (u32 base = 0; base < total; base += blockDim.x) {
         const u32 i = base + threadIdx.x;
         P3 it; it.x = KEY_MAX; it.y = KEY_MAX; it.idx = KEY_MAX;
@@ -505,8 +507,7 @@ __device__ void pareto_store_and_fold(ParetoAcc &acc, u32 block, u32 nblk, u32 *
             const u64 *w = reinterpret_cast<const u64 *>(partial + (size_t)lo * GUIDE_PARETO_MAX + (i - pre[lo]));
             it.x = __ldcg(w); it.y = __ldcg(w + 1); it.idx = __ldcg(w + 2);
         }
-        acc.offer(i < total, it);
-        if (++since == CHECK_EVERY) { acc.checkpoint(); since = 0; }
+        acc.push(i < total, it);
     }
     acc.finish();
     overflow |= acc.overflow;
@@ -523,10 +524,8 @@ __global__ void __launch_bounds__(SEL_THREADS) k_pareto_scan(Src src, Range r, u
     ParetoAcc acc;
     acc.init((P3 *)smem_raw, &cnt, scratch);
     constexpr int ITEMS = Src::ITEMS;
-    constexpr u32 ROUNDS = CHECK_EVERY / ITEMS;
     const u64 span = (u64)ITEMS * blockDim.x;
     const u64 tiles = (r.count + span - 1) / span;
-    u32 since = 0;
     for (u64 tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
         bool ok[ITEMS];
         P3 it[ITEMS];
@@ -538,15 +537,8 @@ __global__ void __launch_bounds__(SEL_THREADS) k_pareto_scan(Src src, Range r, u
             ok[u] = src.get(jc, r.first + jc, a, b) && j < r.count;
             it[u].x = enc(a); it[u].y = enc(b); it[u].idx = r.first + j;
         }
-        if (tile == blockIdx.x) {
-            // first round: one offer per checkpoint, so the first front comes from a small sort
 #pragma unroll
-            for (int u = 0; u < ITEMS; u++) { acc.offer(ok[u], it[u]); acc.checkpoint(); }
-            continue;
-        }
-#pragma unroll
-        for (int u = 0; u < ITEMS; u++) acc.offer(ok[u], it[u]);
-        if (++since == ROUNDS) { acc.checkpoint(); since = 0; }
+        for (int u = 0; u < ITEMS; u++) acc.push(ok[u], it[u]);
     }
     pareto_store_and_fold(acc, blockIdx.x, gridDim.x, ticket, sizes, partial, idx_out, out_cap, count_out);
 }
@@ -560,14 +552,12 @@ k_pareto_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, 
     __shared__ __align__(8) u32 scratch[64];
     ParetoAcc acc;
     acc.init((P3 *)smem_raw, &cnt, scratch);
-    u32 since = CHECK_EVERY - 1;          // the first offer is followed by a checkpoint: early front
     tiled_visit<TIME_SUM>(s, r, tp_model, hf_chunk, tiles_per_mb, [&](bool valid, u64 idx, const Metrics &m) {
         double a = 0.0, b = 0.0;
         const bool ok = valid && fused_pick(m, c, xm, ym, a, b);
         P3 it;
         it.x = enc(a); it.y = enc(b); it.idx = idx;
-        acc.offer(ok, it);
-        if (++since == CHECK_EVERY) { acc.checkpoint(); since = 0; }
+        acc.push(ok, it);
     });
     pareto_store_and_fold(acc, blockIdx.y * gridDim.x + blockIdx.x, gridDim.x * gridDim.y, ticket, sizes, partial, idx_out,
                           out_cap, count_out);
@@ -591,9 +581,11 @@ static Cons make_cons(const guide_constraints &c) {
 }
 
 static u32 grid_for(u64 count, u32 items, u32 blocks_per_sm, u32 max_blocks) {
+    // every block has fixed costs (first sorts, final sort, its list in the merge): give each at
+    // least eight rounds of tiles
     const u64 tiles = (count + (u64)SEL_THREADS * items - 1) / ((u64)SEL_THREADS * items);
     u64 g = std::min<u64>((u64)num_sms() * blocks_per_sm, max_blocks);
-    g = std::min<u64>(g, std::max<u64>(tiles, 1));
+    g = std::min<u64>(g, std::max<u64>(tiles / 8, 1));
     return (u32)g;
 }
 
@@ -625,7 +617,9 @@ static int run_topk_scan(const Src &src, Range r, u32 k, int negate, u32 max_blo
                          double *key_out, u32 *count_out, cudaStream_t st) {
     u32 *counts = (u32 *)(ws + 256);
     KI *lists = (KI *)(ws + topk_lists_offset(max_blocks));
-    const u32 grid = grid_for(r.count, Src::ITEMS, 4, max_blocks);
+    const int rc = allow_smem(k_topk_scan<Src>, TOPK_CAP * sizeof(KI));
+    if (rc) return rc;
+    const u32 grid = grid_for(r.count, Src::ITEMS, 3, max_blocks);
     k_topk_scan<Src><<<grid, SEL_THREADS, TOPK_CAP * sizeof(KI), st>>>(src, r, k, counts, lists);
     GUIDE_CUDA(cudaGetLastError());
     return run_topk_merge(grid, k, negate, counts, lists, idx_out, key_out, count_out, st);
@@ -636,6 +630,8 @@ static int run_topk_tiled(const DSpace &s, Range r, const TileGeom &g, int tp_mo
                           unsigned char *ws, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st) {
     u32 *counts = (u32 *)(ws + 256);
     KI *lists = (KI *)(ws + topk_lists_offset(SEL_MAX_BLOCKS));
+    const int rc = allow_smem(k_topk_tiled<TIME_SUM>, TOPK_CAP * sizeof(KI));
+    if (rc) return rc;
     const dim3 grid(g.gx, g.splits);
     k_topk_tiled<TIME_SUM><<<grid, g.threads, TOPK_CAP * sizeof(KI), st>>>(s, r, tp_model, g.hf_chunk, g.tiles_per_mb, c,
                                                                           key, k, counts, lists);
