@@ -93,7 +93,8 @@ static int check_trace_overflow(const guide_space &s, const guide_trace &t) {
 
 // Derived per-model quantities and the reciprocal rates of every hardware x framework pair.
 __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *gh, u32 n_h, const guide_fw *gf,
-                               u32 n_f, DModel *dm, DRate *dr) {
+                               u32 n_f, const u32 *tp, u32 n_t, DModel *dm, DRate *dr, double *cost_hr,
+                               double *cost_sec) {
     const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n_m) {
         const guide_model m = gm[i];
@@ -124,6 +125,11 @@ __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *g
         r.flash = f.flash;
         r.kv_block = f.kv_block;
         dr[i] = r;
+        for (u32 k = 0; k < n_t; k++) {
+            const double c = h.price_per_hr * (double)tp[k];
+            cost_hr[i * n_t + k] = c;
+            cost_sec[i * n_t + k] = c / 3600.0;
+        }
     }
 }
 
@@ -142,7 +148,8 @@ int space_on_device(guide_space *s, DSpace *out) {
     const size_t o_gm = take(n_m * sizeof(guide_model)), o_gh = take(n_h * sizeof(guide_hw)),
                  o_gf = take(n_f * sizeof(guide_fw)), o_dm = take(n_m * sizeof(DModel)),
                  o_dr = take(n_h * n_f * sizeof(DRate)), o_b = take(s->batch.size() * 4),
-                 o_t = take(s->tp.size() * 4), o_p = take(s->pairs.size() * 8);
+                 o_t = take(s->tp.size() * 4), o_p = take(s->pairs.size() * 8),
+                 o_ch = take(n_h * n_f * s->tp.size() * 8), o_cs = take(n_h * n_f * s->tp.size() * 8);
     char *blob = nullptr;
     GUIDE_CUDA(cudaMalloc(&blob, off));
     cudaError_t e = cudaSuccess;
@@ -160,7 +167,9 @@ int space_on_device(guide_space *s, DSpace *out) {
         k_build_tables<<<(n + 127) / 128, 128>>>((const guide_model *)(blob + o_gm), (u32)n_m,
                                                  (const guide_hw *)(blob + o_gh), (u32)n_h,
                                                  (const guide_fw *)(blob + o_gf), (u32)n_f,
-                                                 (DModel *)(blob + o_dm), (DRate *)(blob + o_dr));
+                                                 (const u32 *)(blob + o_t), (u32)s->tp.size(),
+                                                 (DModel *)(blob + o_dm), (DRate *)(blob + o_dr),
+                                                 (double *)(blob + o_ch), (double *)(blob + o_cs));
         e = cudaGetLastError();
         if (e == cudaSuccess) e = cudaStreamSynchronize(0);
     }
@@ -173,6 +182,8 @@ int space_on_device(guide_space *s, DSpace *out) {
     d.view.batch = (const u32 *)(blob + o_b);
     d.view.tp = (const u32 *)(blob + o_t);
     d.view.pairs = (const uint2 *)(blob + o_p);
+    d.view.cost_hr = (const double *)(blob + o_ch);
+    d.view.cost_sec = (const double *)(blob + o_cs);
     d.view.n_m = (u32)n_m; d.view.n_h = (u32)n_h; d.view.n_f = (u32)n_f;
     d.view.n_b = (u32)s->batch.size(); d.view.n_t = (u32)s->tp.size(); d.view.n_l = (u32)s->pairs.size();
     s->dev.push_back(d);

@@ -38,6 +38,8 @@ struct DSpace {
     const DRate *rates;          // [n_h * n_f]
     const u32 *batch, *tp;
     const uint2 *pairs;          // (lin, lout)
+    const double *cost_hr;       // [n_h * n_f][n_t]: price x TP degree
+    const double *cost_sec;      // [n_h * n_f][n_t]: (price x TP degree) / 3600
     u32 n_m, n_h, n_f, n_b, n_t, n_l;
 };
 
@@ -210,7 +212,50 @@ __device__ __forceinline__ u64 floor_div(u64 num, u64 den) {
     return q;
 }
 
+__device__ __forceinline__ u32 clamp_u32(u64 v) { return v > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)v; }
+
+// floor(num / den) with a precomputed reciprocal inv = 1 / (double)den, for num, den < 2^52:
+// the product is within one unit of the quotient, two integer checks make it exact.
+__device__ __forceinline__ u64 floor_div_recip(u64 num, u64 den, double inv) {
+    u64 q = __double2ull_rz(__ull2double_rn(num) * inv);
+    if (q * den > num) q--;
+    else if ((q + 1) * den <= num) q++;
+    return q;
+}
+
 struct MemInfo { u64 w_gpu, kv_tok; u32 log2t; };
+
+// KV bytes of one request of S tokens under a block size, and the reciprocal used to divide by it;
+// depends on the thread's (model, TP, lengths) and on the framework's block size only, so a loop
+// over hardware x framework pairs recomputes it just when the block size changes.
+struct ReqBytes {
+    u64 bytes;        // ceil(S / block) * block * kv_tok
+    double inv;       // 1 / bytes, valid when small is set
+    u32 block;        // block size this was computed for (0 = not yet)
+    bool small;       // bytes < 2^52: the reciprocal path is exact
+};
+__device__ __forceinline__ void req_bytes_for(ReqBytes &q, u32 block, u64 S, u64 kv_tok) {
+    const u64 s_blk = block == 1 ? S : ((S + block - 1) / block) * block;
+    q.bytes = s_blk * kv_tok;
+    q.small = (q.bytes >> 52) == 0;
+    q.inv = 1.0 / __ull2double_rn(q.bytes);
+    q.block = block;
+}
+// status and B_max with the request bytes already known
+__device__ __forceinline__ u32 feasibility_cached(const DModel &m, u64 usable, const MemInfo &mi, u32 t, u32 b,
+                                                  const ReqBytes &q, u32 &bmax_out) {
+    u64 bmax = 0;
+    if (usable > mi.w_gpu) {
+        const u64 avail = usable - mi.w_gpu;
+        bmax = (q.small && (avail >> 52) == 0) ? floor_div_recip(avail, q.bytes, q.inv) : avail / q.bytes;
+    }
+    u32 st = 0;
+    if (usable <= mi.w_gpu) st |= 1;
+    if ((u64)b > bmax) st |= 2;
+    if ((m.nh & (t - 1)) != 0 || (m.nkv & (t - 1)) != 0) st |= 4;   // t is a power of two
+    bmax_out = clamp_u32(bmax);
+    return st;
+}
 
 __device__ __forceinline__ MemInfo mem_info(const DModel &m, u32 t) {
     MemInfo mi;
@@ -220,7 +265,6 @@ __device__ __forceinline__ MemInfo mem_info(const DModel &m, u32 t) {
     return mi;
 }
 
-__device__ __forceinline__ u32 clamp_u32(u64 v) { return v > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)v; }
 
 // ---- one config in closed form -------------------------------------------------------------------
 
@@ -252,16 +296,16 @@ __device__ __forceinline__ u32 closed_form_feasibility(const DModel &m, const DR
 }
 
 // final metrics from the two stage times (Sec. 3.2: TTFT = prefill time, throughput; Sec. 5.1)
-__device__ __forceinline__ void closed_form_metrics(double t_pre, double t_dec, u32 b, u32 n, u32 t, double price,
-                                                    Metrics &o) {
+__device__ __forceinline__ void closed_form_metrics(double t_pre, double t_dec, u32 b, u32 n, double cost_hr,
+                                                    double cost_sec, Metrics &o) {
     const double inf = __longlong_as_double(0x7FF0000000000000LL);
     o.ttft = t_pre;
     o.latency = t_pre + t_dec;
-    o.cost_hr = price * (double)t;
+    o.cost_hr = cost_hr;                 // price x TP degree
     if (n > 0) {
         o.tpot = t_dec / (double)n;
         o.thr = cvt((u64)b * n) / t_dec;
-        o.cost_tok = (o.cost_hr / 3600.0) / o.thr;
+        o.cost_tok = cost_sec / o.thr;   // (cost_hr / 3600) / throughput
     } else {
         o.tpot = 0.0; o.thr = 0.0; o.cost_tok = inf;
     }
@@ -298,7 +342,8 @@ __device__ __forceinline__ void closed_form_eval(const DSpace &s, const Cfg &c, 
         build_attn_tasks(m, tt, Td, ctx, ctx, k);
         t_dec = eval_phase<TIME_SUM>(k, r, Nd, lf);
     }
-    closed_form_metrics(t_pre, t_dec, b, n, t, r.price, o);
+    const u32 ci = (c.h * s.n_f + c.f) * s.n_t + c.t;
+    closed_form_metrics(t_pre, t_dec, b, n, s.cost_hr[ci], s.cost_sec[ci], o);
 }
 
 }  // namespace guide

@@ -63,19 +63,40 @@ __device__ __forceinline__ void tiled_visit(const DSpace &s, const Range &r, int
     const u64 stride_hf = (u64)s.n_b * n_tl;
     const u64 base = ((u64)mpos * n_hf) * stride_hf + (u64)bpos * n_tl + tl;
 
+    ReqBytes rq;
+    rq.block = 0; rq.bytes = 1; rq.inv = 1.0; rq.small = false;
+    const u64 S = (u64)lin + lout;
+    const double nd = (double)n;
+    const double tok = cvt((u64)b * n);
+
     for (u32 i = 0; i < hf_chunk; i++) {
         const u32 hf = hf0 + i;
         const u64 idx = base + (u64)hf * stride_hf;
         const bool valid = active && hf < n_hf && idx >= r.first && idx - r.first < r.count;
         Metrics out;
         if (valid) {
-            const DRate rt = s.rates[hf];
-            out.status = closed_form_feasibility(m, rt, mi, t, b, lin, lout, out.bmax);
+            const DRate &rt = s.rates[hf];
+            const u32 block = rt.kv_block;
+            if (block != rq.block) req_bytes_for(rq, block, S, mi.kv_tok);
+            out.status = feasibility_cached(m, rt.usable, mi, t, b, rq, out.bmax);
             if (out.status) set_infeasible(out);
             else {
+                const double inf = __longlong_as_double(0x7FF0000000000000LL);
                 const double t_pre = eval_phase<TIME_SUM>(kp, rt, Nd, lf);
                 const double t_dec = n > 0 ? eval_phase<TIME_SUM>(kd, rt, Nd, lf) : 0.0;
-                closed_form_metrics(t_pre, t_dec, b, n, t, rt.price, out);
+                const u32 ci = hf * s.n_t + tpos;
+                out.ttft = t_pre;
+                out.latency = t_pre + t_dec;
+                out.cost_hr = s.cost_hr[ci];
+                if (n > 0) {
+                    out.tpot = t_dec / nd;
+                    out.thr = tok / t_dec;
+                    out.cost_tok = s.cost_sec[ci] / out.thr;
+                } else {
+                    out.tpot = 0.0; out.thr = 0.0; out.cost_tok = inf;
+                }
+                out.n_iters = 1 + (u64)n;
+                out.n_req_iters = (u64)b * (1 + (u64)n);
             }
         } else {
             out.status = 0xFF;
