@@ -254,10 +254,10 @@ int guide_pareto(const guide_space *space, const guide_trace *trace, const guide
  *
  * The first call on each device looks up the array's device address (no allocation, but a
  * one-time set-up step): make that first call before starting any stream capture.  All calls on a
- * device share the one array, which keeps the previous call's contents; nothing in it has to start
- * at zero, because a call's kernels write every word before they read it.  Two calls whose kernels
- * could overlap on the GPU (different streams, or different threads, without ordering between
- * them) race on it: order them. */
+ * device share the one array, which keeps the previous call's contents; the call resets, on the
+ * given stream, the one word that has to start from a known value, and its kernels write every
+ * other word before they read it.  Two calls whose kernels could overlap on the GPU (different
+ * streams, or different threads, without ordering between them) race on it: order them. */
 #define GUIDE_NOALLOC_TOPK_MAX 64u
 #define GUIDE_NOALLOC_COUNT_MAX (1ull << 40)
 int guide_select_topk_noalloc(const guide_outputs *outputs, uint64_t first, uint64_t count,

@@ -198,6 +198,111 @@ struct TopKAcc {
     }
 };
 
+// ---- per-warp top-k accumulator (k <= TOPK_WARP_K) -------------------------------------------------
+//
+// No block barrier on the hot path.  Each warp owns a segment of shared memory with its own sorted
+// candidates and its own threshold; takers of a round are placed by ballot, and when the segment
+// fills (or about k entries have slipped under a stale threshold) the warp sorts it alone.  A warp
+// that holds k candidates publishes its k-th key to a grid-wide word (atomicMin); every warp drops
+// anything above that word at once, so once a few warps have found good candidates the rest of
+// the grid hardly appends at all.  The word only bounds keys (strictly larger keys are dropped),
+// ties on the key are still decided by the index in the exact per-warp test.
+
+static constexpr u32 TOPK_WARP_K = 128;
+
+__host__ __device__ inline u32 warp_seg_cap(u32 k) {
+    u32 need = 2 * k + 64, p = 128;
+    while (p < need) p <<= 1;
+    return p;
+}
+
+struct WarpTopK {
+    KI *seg;          // this warp's segment, cap entries
+    u64 *gptr;        // grid-wide upper bound on the k-th key
+    u64 gthr;         // cached copy
+    u32 cap, k, fill, tick;
+    bool has_thr;
+    KI thr;
+
+    __device__ void init(KI *smem, u32 k_, u64 *gptr_) {
+        k = k_; cap = warp_seg_cap(k_);
+        seg = smem + (size_t)(threadIdx.x >> 5) * cap;
+        gptr = gptr_; gthr = __ldcg(gptr_);
+        fill = 0; tick = 0; has_thr = false; thr.key = KEY_MAX; thr.idx = KEY_MAX;
+    }
+    __device__ void compact() {
+        const u32 lane = threadIdx.x & 31;
+        const u32 P = next_pow2(fill);
+        for (u32 i = fill + lane; i < P; i += 32) { seg[i].key = KEY_MAX; seg[i].idx = KEY_MAX; }
+        __syncwarp();
+        for (u32 size = 2; size <= P; size <<= 1) {
+            for (u32 stride = size >> 1; stride > 0; stride >>= 1) {
+                for (u32 i = lane; i < (P >> 1); i += 32) {
+                    const u32 lo = ((i & ~(stride - 1)) << 1) | (i & (stride - 1));
+                    const u32 hi = lo + stride;
+                    const bool up = (lo & size) == 0;
+                    const KI a = seg[lo], b = seg[hi];
+                    if (ki_less(b, a) == up) { seg[lo] = b; seg[hi] = a; }
+                }
+                __syncwarp();
+            }
+        }
+        if (fill >= k) {
+            fill = k; has_thr = true; thr = seg[k - 1];
+            if (lane == 0) atomicMin((unsigned long long *)gptr, (unsigned long long)thr.key);
+            if (thr.key < gthr) gthr = thr.key;
+        }
+        __syncwarp();
+    }
+    // all 32 lanes of the warp call it together
+    __device__ __forceinline__ void push(bool ok, const KI &it) {
+        if ((++tick & 15u) == 0) { const u64 g = __ldcg(gptr); if (g < gthr) gthr = g; }
+        const bool take = ok && it.key <= gthr && (!has_thr || ki_less(it, thr));
+        const u32 ballot = __ballot_sync(0xFFFFFFFFu, take);
+        if (ballot) {
+            if (take) seg[fill + __popc(ballot & ((1u << (threadIdx.x & 31)) - 1))] = it;
+            fill += __popc(ballot);
+            __syncwarp();
+            const u32 early = has_thr ? 2 * k + 32 : k;
+            if (fill + 32 > cap || fill >= early) compact();
+        }
+    }
+};
+
+// the block's warps pool their candidates, one sort, the k smallest go to the workspace
+__device__ void warp_topk_store(WarpTopK &w, KI *smem, u32 block, u32 k, u32 *counts, KI *lists) {
+    __shared__ u32 wfill[SEL_THREADS / 32];
+    const u32 lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    if (w.fill > 0) w.compact();                   // sorted, at most k left
+    KI mine[TOPK_WARP_K / 32];
+#pragma unroll
+    for (u32 q = 0; q < TOPK_WARP_K / 32; q++) {
+        const u32 i = q * 32 + lane;
+        if (i < w.fill) mine[q] = w.seg[i];
+    }
+    if (lane == 0) wfill[warp] = w.fill;
+    __syncthreads();                               // every segment has been read into registers
+    u32 off = 0, total = 0;
+    for (u32 x = 0; x < n_warps; x++) {
+        if (x < warp) off += wfill[x];
+        total += wfill[x];
+    }
+#pragma unroll
+    for (u32 q = 0; q < TOPK_WARP_K / 32; q++) {
+        const u32 i = q * 32 + lane;
+        if (i < w.fill) smem[off + i] = mine[q];
+    }
+    const u32 P = next_pow2(total);
+    __syncthreads();
+    for (u32 i = total + threadIdx.x; i < P; i += blockDim.x) { smem[i].key = KEY_MAX; smem[i].idx = KEY_MAX; }
+    __syncthreads();
+    block_bitonic_sort(smem, P, ki_less);
+    const u32 c = min(total, k);
+    KI *dst = lists + (size_t)block * k;
+    for (u32 i = threadIdx.x; i < c; i += blockDim.x) dst[i] = smem[i];
+    if (threadIdx.x == 0) counts[block] = c;
+}
+
 // ---- Pareto accumulator ----------------------------------------------------------------------------
 
 struct ParetoAcc {
@@ -328,12 +433,24 @@ __device__ __forceinline__ void topk_store(TopKAcc &acc, u32 block, u32 k, u32 *
     if (threadIdx.x == 0) counts[block] = acc.c;
 }
 
-template <class Src>
-__global__ void __launch_bounds__(SEL_THREADS) k_topk_scan(Src src, Range r, u32 k, u32 *counts, KI *lists) {
+// WARP: per-warp accumulators (no barrier while scanning); otherwise one accumulator per block.
+template <bool WARP> struct TopKPick { typedef TopKAcc type; };
+template <> struct TopKPick<true> { typedef WarpTopK type; };
+__device__ __forceinline__ void topk_begin(TopKAcc &acc, KI *smem, u32 *cnt, u32 k, u64 *) { acc.init(smem, cnt, k); }
+__device__ __forceinline__ void topk_begin(WarpTopK &acc, KI *smem, u32 *, u32 k, u64 *gthr) { acc.init(smem, k, gthr); }
+__device__ __forceinline__ void topk_end(TopKAcc &acc, KI *, u32 block, u32 k, u32 *counts, KI *lists) {
+    topk_store(acc, block, k, counts, lists);
+}
+__device__ __forceinline__ void topk_end(WarpTopK &acc, KI *smem, u32 block, u32 k, u32 *counts, KI *lists) {
+    warp_topk_store(acc, smem, block, k, counts, lists);
+}
+
+template <class Src, bool WARP>
+__global__ void __launch_bounds__(SEL_THREADS) k_topk_scan(Src src, Range r, u32 k, u32 *counts, KI *lists, u64 *gthr) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ u32 cnt;
-    TopKAcc acc;
-    acc.init((KI *)smem_raw, &cnt, k);
+    typename TopKPick<WARP>::type acc;
+    topk_begin(acc, (KI *)smem_raw, &cnt, k, gthr);
     constexpr int ITEMS = Src::ITEMS;
     const u64 span = (u64)ITEMS * blockDim.x;
     const u64 tiles = (r.count + span - 1) / span;
@@ -351,16 +468,17 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_scan(Src src, Range r, u32
 #pragma unroll
         for (int u = 0; u < ITEMS; u++) acc.push(ok[u], it[u]);
     }
-    topk_store(acc, blockIdx.x, k, counts, lists);
+    topk_end(acc, (KI *)smem_raw, blockIdx.x, k, counts, lists);
 }
 
-template <int TIME_SUM>
+template <int TIME_SUM, bool WARP>
 __global__ void __launch_bounds__(SEL_THREADS, 2)
-k_topk_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, Cons c, int key, u32 k, u32 *counts, KI *lists) {
+k_topk_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, Cons c, int key, u32 k, u32 *counts, KI *lists,
+             u64 *gthr) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ u32 cnt;
-    TopKAcc acc;
-    acc.init((KI *)smem_raw, &cnt, k);
+    typename TopKPick<WARP>::type acc;
+    topk_begin(acc, (KI *)smem_raw, &cnt, k, gthr);
     tiled_visit<TIME_SUM>(s, r, tp_model, hf_chunk, tiles_per_mb, [&](bool valid, u64 idx, const Metrics &m) {
         double a = 0.0, b;
         const bool ok = valid && fused_pick(m, c, key, -1, a, b);
@@ -368,7 +486,7 @@ k_topk_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, Co
         it.key = enc(a); it.idx = idx;
         acc.push(ok, it);
     });
-    topk_store(acc, blockIdx.y * gridDim.x + blockIdx.x, k, counts, lists);
+    topk_end(acc, (KI *)smem_raw, blockIdx.y * gridDim.x + blockIdx.x, k, counts, lists);
 }
 
 // Merge of the per-block lists.  One warp per candidate: its rank in the union is its position in
@@ -612,31 +730,57 @@ static int run_topk_merge(u32 nblk, u32 k, int negate, u32 *counts, KI *lists, u
     return GUIDE_OK;
 }
 
+// The first 256 bytes of a top-k workspace hold the grid-wide key bound of the per-warp mode; it
+// has to start at all-ones.
+static int topk_reset_bound(unsigned char *ws, cudaStream_t st) {
+    GUIDE_CUDA(cudaMemsetAsync(ws, 0xFF, 256, st));
+    return GUIDE_OK;
+}
+
+template <class Src, bool WARP>
+static int run_topk_scan_mode(const Src &src, Range r, u32 k, int negate, u32 max_blocks, unsigned char *ws, u64 *idx_out,
+                              double *key_out, u32 *count_out, cudaStream_t st) {
+    u32 *counts = (u32 *)(ws + 256);
+    KI *lists = (KI *)(ws + topk_lists_offset(max_blocks));
+    const size_t smem = WARP ? (size_t)(SEL_THREADS / 32) * warp_seg_cap(k) * sizeof(KI) : (size_t)TOPK_CAP * sizeof(KI);
+    int rc = allow_smem(k_topk_scan<Src, WARP>, smem);
+    if (rc) return rc;
+    if ((rc = topk_reset_bound(ws, st))) return rc;
+    const u32 grid = grid_for(r.count, Src::ITEMS, WARP ? 4 : 3, max_blocks);
+    k_topk_scan<Src, WARP><<<grid, SEL_THREADS, smem, st>>>(src, r, k, counts, lists, (u64 *)ws);
+    GUIDE_CUDA(cudaGetLastError());
+    return run_topk_merge(grid, k, negate, counts, lists, idx_out, key_out, count_out, st);
+}
+
 template <class Src>
 static int run_topk_scan(const Src &src, Range r, u32 k, int negate, u32 max_blocks, unsigned char *ws, u64 *idx_out,
                          double *key_out, u32 *count_out, cudaStream_t st) {
+    return k <= TOPK_WARP_K ? run_topk_scan_mode<Src, true>(src, r, k, negate, max_blocks, ws, idx_out, key_out, count_out, st)
+                            : run_topk_scan_mode<Src, false>(src, r, k, negate, max_blocks, ws, idx_out, key_out, count_out, st);
+}
+
+template <int TIME_SUM, bool WARP>
+static int run_topk_tiled_mode(const DSpace &s, Range r, const TileGeom &g, int tp_model, const Cons &c, int key, u32 k,
+                               unsigned char *ws, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st) {
     u32 *counts = (u32 *)(ws + 256);
-    KI *lists = (KI *)(ws + topk_lists_offset(max_blocks));
-    const int rc = allow_smem(k_topk_scan<Src>, TOPK_CAP * sizeof(KI));
+    KI *lists = (KI *)(ws + topk_lists_offset(SEL_MAX_BLOCKS));
+    const size_t smem = WARP ? (size_t)(SEL_THREADS / 32) * warp_seg_cap(k) * sizeof(KI) : (size_t)TOPK_CAP * sizeof(KI);
+    int rc = allow_smem(k_topk_tiled<TIME_SUM, WARP>, smem);
     if (rc) return rc;
-    const u32 grid = grid_for(r.count, Src::ITEMS, 3, max_blocks);
-    k_topk_scan<Src><<<grid, SEL_THREADS, TOPK_CAP * sizeof(KI), st>>>(src, r, k, counts, lists);
+    if ((rc = topk_reset_bound(ws, st))) return rc;
+    const dim3 grid(g.gx, g.splits);
+    k_topk_tiled<TIME_SUM, WARP><<<grid, g.threads, smem, st>>>(s, r, tp_model, g.hf_chunk, g.tiles_per_mb, c, key, k,
+                                                               counts, lists, (u64 *)ws);
     GUIDE_CUDA(cudaGetLastError());
-    return run_topk_merge(grid, k, negate, counts, lists, idx_out, key_out, count_out, st);
+    return run_topk_merge(g.gx * g.splits, k, key == GUIDE_THROUGHPUT, counts, lists, idx_out, key_out, count_out, st);
 }
 
 template <int TIME_SUM>
 static int run_topk_tiled(const DSpace &s, Range r, const TileGeom &g, int tp_model, const Cons &c, int key, u32 k,
                           unsigned char *ws, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st) {
-    u32 *counts = (u32 *)(ws + 256);
-    KI *lists = (KI *)(ws + topk_lists_offset(SEL_MAX_BLOCKS));
-    const int rc = allow_smem(k_topk_tiled<TIME_SUM>, TOPK_CAP * sizeof(KI));
-    if (rc) return rc;
-    const dim3 grid(g.gx, g.splits);
-    k_topk_tiled<TIME_SUM><<<grid, g.threads, TOPK_CAP * sizeof(KI), st>>>(s, r, tp_model, g.hf_chunk, g.tiles_per_mb, c,
-                                                                          key, k, counts, lists);
-    GUIDE_CUDA(cudaGetLastError());
-    return run_topk_merge(g.gx * g.splits, k, key == GUIDE_THROUGHPUT, counts, lists, idx_out, key_out, count_out, st);
+    return k <= TOPK_WARP_K
+               ? run_topk_tiled_mode<TIME_SUM, true>(s, r, g, tp_model, c, key, k, ws, idx_out, key_out, count_out, st)
+               : run_topk_tiled_mode<TIME_SUM, false>(s, r, g, tp_model, c, key, k, ws, idx_out, key_out, count_out, st);
 }
 
 int launch_topk(const DSpace &s, Range r, const guide_outputs *mat, int time_model, int tp_model,
@@ -746,9 +890,10 @@ int launch_topk_noalloc(Range r, const guide_outputs &mat, const guide_constrain
     if (rc) return rc;
     static_assert(256 + NOALLOC_BLOCKS * 4 == 1280, "list offset below assumes a 256-byte multiple");
     MatSource src{mat, make_cons(c), key, -1};
-    // The array still holds the previous call's counts and lists.  Nothing has to start at zero:
-    // every block of this launch writes its count and its list before the merge kernel, which
-    // follows on the same stream, reads them, and the merge reads only this launch's blocks.
+    // The array still holds the previous call's bound, counts and lists.  The bound word is reset
+    // on this stream before the scan; counts and lists need no clearing: every block of this
+    // launch writes its own before the merge kernel, which follows on the same stream and reads
+    // only this launch's blocks.
     return run_topk_scan(src, r, k, key == GUIDE_THROUGHPUT, NOALLOC_BLOCKS, scratch, idx_out, key_out, count_out, st);
 }
 
