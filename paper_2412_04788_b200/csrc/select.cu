@@ -56,10 +56,73 @@ __device__ __forceinline__ double pick_metric(int key, double latency, double tt
 
 // materialised arrays written by guide_simulate
 struct MatSource {
-    static constexpr int ITEMS = 4;     // loads of four configs are in flight before the first barrier
+    static constexpr int ITEMS = 4;     // a thread fetches four consecutive configs per round
+    static constexpr bool CONSEC = true;
     guide_outputs o;
     Cons c;
     int m0, m1;
+    int vec;                            // every array in use is 16-byte aligned (status: 4-byte)
+    __device__ __forceinline__ const double *metric_ptr(int key) const {
+        switch (key) {
+        case GUIDE_LATENCY: return o.latency;
+        case GUIDE_TTFT: return o.ttft;
+        case GUIDE_TTFT_P99: return o.ttft_p99;
+        case GUIDE_TPOT: return o.tpot;
+        case GUIDE_THROUGHPUT: return o.thr_decode;
+        case GUIDE_COST_PER_HR: return o.cost_per_hr;
+        default: return o.cost_per_token;
+        }
+    }
+    static __device__ __forceinline__ void load4(const double *p, u64 j0, double v[4]) {
+        const double2 lo = __ldg(reinterpret_cast<const double2 *>(p + j0));
+        const double2 hi = __ldg(reinterpret_cast<const double2 *>(p + j0 + 2));
+        v[0] = lo.x; v[1] = lo.y; v[2] = hi.x; v[3] = hi.y;
+    }
+    // Four consecutive configs j0..j0+3 (j0 a multiple of 4, all in range, vec set): one 4-byte
+    // status load and two 16-byte loads per array in use.
+    __device__ __forceinline__ void get4(u64 j0, bool ok[4], double a[4], double b[4]) const {
+        const double inf = __longlong_as_double(0x7FF0000000000000LL);
+        const u32 st = __ldg(reinterpret_cast<const u32 *>(o.status + j0));
+        double v[4];
+#pragma unroll
+        for (int u = 0; u < 4; u++) ok[u] = ((st >> (8 * u)) & 0xFFu) == 0;
+        if (c.max_ttft < inf) {
+            const double *p = c.ttft_stat == GUIDE_STAT_MEAN ? o.ttft : c.ttft_stat == GUIDE_STAT_P50 ? o.ttft_p50 : o.ttft_p99;
+            load4(p, j0, v);
+#pragma unroll
+            for (int u = 0; u < 4; u++) ok[u] &= v[u] <= c.max_ttft;
+        }
+        if (c.max_latency < inf) {
+            load4(o.latency, j0, v);
+#pragma unroll
+            for (int u = 0; u < 4; u++) ok[u] &= v[u] <= c.max_latency;
+        }
+        if (c.max_cost_hr < inf) {
+            load4(o.cost_per_hr, j0, v);
+#pragma unroll
+            for (int u = 0; u < 4; u++) ok[u] &= v[u] <= c.max_cost_hr;
+        }
+        if (c.min_thr > 0.0) {
+            load4(o.thr_decode, j0, v);
+#pragma unroll
+            for (int u = 0; u < 4; u++) ok[u] &= v[u] >= c.min_thr;
+        }
+        load4(metric_ptr(m0), j0, a);
+        if (m0 == GUIDE_THROUGHPUT) {
+#pragma unroll
+            for (int u = 0; u < 4; u++) a[u] = 0.0 - a[u];
+        }
+        if (m1 >= 0) {
+            load4(metric_ptr(m1), j0, b);
+            if (m1 == GUIDE_THROUGHPUT) {
+#pragma unroll
+                for (int u = 0; u < 4; u++) b[u] = 0.0 - b[u];
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < 4; u++) b[u] = 0.0;
+        }
+    }
     __device__ __forceinline__ double metric(int key, u64 j) const {
         switch (key) {
         case GUIDE_LATENCY: return __ldg(o.latency + j);
@@ -93,6 +156,9 @@ struct MatSource {
 template <int TIME_SUM>
 struct FusedSource {
     static constexpr int ITEMS = 1;     // evaluation is register heavy: one config at a time
+    static constexpr bool CONSEC = false;
+    __device__ __forceinline__ void get4(u64, bool *, double *, double *) const {}
+    static constexpr int vec = 0;
     DSpace s;
     Cons c;
     int m0, m1, tp_model;
@@ -108,6 +174,30 @@ struct FusedSource {
         return true;
     }
 };
+
+// One round of a scan: ITEMS configs per thread.  Sources with CONSEC give a thread consecutive
+// configs (vector loads when aligned and in range); otherwise thread t takes t, t + blockDim, ...
+template <class Src>
+__device__ __forceinline__ void fetch_round(const Src &src, const Range &r, u64 tile, bool ok[Src::ITEMS],
+                                            double a[Src::ITEMS], double b[Src::ITEMS], u64 jj[Src::ITEMS]) {
+    constexpr int ITEMS = Src::ITEMS;
+    const u64 span = (u64)ITEMS * blockDim.x;
+    if (Src::CONSEC) {
+        const u64 j0 = tile * span + (u64)ITEMS * threadIdx.x;
+#pragma unroll
+        for (int u = 0; u < ITEMS; u++) jj[u] = j0 + u;
+        if (src.vec && j0 + ITEMS <= r.count) { src.get4(j0, ok, a, b); return; }
+    } else {
+#pragma unroll
+        for (int u = 0; u < ITEMS; u++) jj[u] = tile * span + (u64)u * blockDim.x + threadIdx.x;
+    }
+#pragma unroll
+    for (int u = 0; u < ITEMS; u++) {
+        const u64 jc = jj[u] < r.count ? jj[u] : r.count - 1;      // keep the loads in range
+        a[u] = 0.0; b[u] = 0.0;
+        ok[u] = src.get(jc, r.first + jc, a[u], b[u]) && jj[u] < r.count;
+    }
+}
 
 // ---- block-wide helpers ---------------------------------------------------------------------------
 
@@ -254,9 +344,14 @@ struct WarpTopK {
         }
         __syncwarp();
     }
+    // largest key that can still matter to this warp
+    __device__ __forceinline__ u64 bound() const { return has_thr && thr.key < gthr ? thr.key : gthr; }
+    __device__ __forceinline__ void refresh() {
+        if ((++tick & 15u) == 0) { const u64 g = __ldcg(gptr); if (g < gthr) gthr = g; }
+    }
     // all 32 lanes of the warp call it together
     __device__ __forceinline__ void push(bool ok, const KI &it) {
-        if ((++tick & 15u) == 0) { const u64 g = __ldcg(gptr); if (g < gthr) gthr = g; }
+        refresh();
         const bool take = ok && it.key <= gthr && (!has_thr || ki_less(it, thr));
         const u32 ballot = __ballot_sync(0xFFFFFFFFu, take);
         if (ballot) {
@@ -311,12 +406,15 @@ struct ParetoAcc {
     u32 *scratch;     // shared, 2 * 32 words
     u32 nf, c;
     u32 budget, ramp;
+    u64 kx[4], ky[4];  // a few front points kept in registers: most configs are beaten by one of them
     bool overflow;
     bool lazy;        // folding fronts: incoming points are mostly keepers, merge only when the buffer fills
 
     __device__ void init(P3 *b, u32 *cn, u32 *sc, bool lazy_ = false) {
         buf = b; cnt = cn; scratch = sc; nf = 0; c = 0; overflow = false; lazy = lazy_;
         budget = lazy_ ? (PARETO_CAP / 2) / blockDim.x : 1; ramp = lazy_ ? MAX_BUDGET : 1;
+#pragma unroll
+        for (int i = 0; i < 4; i++) { kx[i] = KEY_MAX; ky[i] = KEY_MAX; }
         if (threadIdx.x == 0) *cnt = 0;
         __syncthreads();
     }
@@ -387,6 +485,19 @@ struct ParetoAcc {
         nf = out; c = out;
         if (threadIdx.x == 0) *cnt = out;
         __syncthreads();
+        // refresh the register copies: four points spread over the front
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            if (nf > 0) { const P3 p = buf[(nf * (2 * i + 1)) / 8]; kx[i] = p.x; ky[i] = p.y; }
+            else { kx[i] = KEY_MAX; ky[i] = KEY_MAX; }
+        }
+    }
+    // strictly dominated by one of the register points (equal points are left to the exact test)
+    __device__ __forceinline__ bool killed(const P3 &it) const {
+        bool k = false;
+#pragma unroll
+        for (int i = 0; i < 4; i++) k |= (kx[i] <= it.x && ky[i] <= it.y) && (kx[i] < it.x || ky[i] < it.y);
+        return k;
     }
     // Collective.  Merges when the buffer could overflow before the next checkpoint and, unless
     // lazy, as soon as there is anything while no front exists yet (until then nothing is
@@ -402,7 +513,7 @@ struct ParetoAcc {
     }
     // every thread of the block calls it the same number of times; a barrier only when the budget runs out
     __device__ __forceinline__ void push(bool ok, const P3 &it) {
-        if (ok && !beaten(it)) buf[atomicAdd(cnt, 1)] = it;
+        if (ok && !killed(it) && !beaten(it)) buf[atomicAdd(cnt, 1)] = it;
         if (--budget == 0) checkpoint();
     }
     __device__ void finish() {
@@ -436,6 +547,13 @@ __device__ __forceinline__ void topk_store(TopKAcc &acc, u32 block, u32 k, u32 *
 // WARP: per-warp accumulators (no barrier while scanning); otherwise one accumulator per block.
 template <bool WARP> struct TopKPick { typedef TopKAcc type; };
 template <> struct TopKPick<true> { typedef WarpTopK type; };
+// cheap necessary condition for an item to be taken (exact for neither: push decides)
+__device__ __forceinline__ bool topk_maybe(const TopKAcc &, u64) { return true; }
+__device__ __forceinline__ bool topk_maybe(const WarpTopK &acc, u64 key) { return key <= acc.bound(); }
+// may a whole warp skip its pushes when no lane has a candidate?  Only the per-warp mode: the
+// block accumulator counts pushes towards its checkpoints.
+__device__ __forceinline__ bool topk_can_skip(const TopKAcc &) { return false; }
+__device__ __forceinline__ bool topk_can_skip(WarpTopK &acc) { acc.refresh(); return true; }
 __device__ __forceinline__ void topk_begin(TopKAcc &acc, KI *smem, u32 *cnt, u32 k, u64 *) { acc.init(smem, cnt, k); }
 __device__ __forceinline__ void topk_begin(WarpTopK &acc, KI *smem, u32 *, u32 k, u64 *gthr) { acc.init(smem, k, gthr); }
 __device__ __forceinline__ void topk_end(TopKAcc &acc, KI *, u32 block, u32 k, u32 *counts, KI *lists) {
@@ -456,15 +574,19 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_scan(Src src, Range r, u32
     const u64 tiles = (r.count + span - 1) / span;
     for (u64 tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
         bool ok[ITEMS];
+        double a[ITEMS], b[ITEMS];
+        u64 jj[ITEMS];
         KI it[ITEMS];
+        fetch_round(src, r, tile, ok, a, b, jj);
+        bool any = false;
 #pragma unroll
         for (int u = 0; u < ITEMS; u++) {
-            const u64 j = tile * span + (u64)u * blockDim.x + threadIdx.x;
-            const u64 jc = j < r.count ? j : r.count - 1;          // keep the loads in range
-            double a = 0.0, b;
-            ok[u] = src.get(jc, r.first + jc, a, b) && j < r.count;
-            it[u].key = enc(a); it[u].idx = r.first + j;
+            it[u].key = enc(a[u]); it[u].idx = r.first + jj[u];
+            ok[u] = ok[u] && topk_maybe(acc, it[u].key);
+            any |= ok[u];
         }
+        // almost always nobody in the warp has a candidate: one vote instead of ITEMS pushes
+        if (topk_can_skip(acc) && !__any_sync(0xFFFFFFFFu, any)) continue;
 #pragma unroll
         for (int u = 0; u < ITEMS; u++) acc.push(ok[u], it[u]);
     }
@@ -646,17 +768,15 @@ __global__ void __launch_bounds__(SEL_THREADS) k_pareto_scan(Src src, Range r, u
     const u64 tiles = (r.count + span - 1) / span;
     for (u64 tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
         bool ok[ITEMS];
-        P3 it[ITEMS];
+        double a[ITEMS], b[ITEMS];
+        u64 jj[ITEMS];
+        fetch_round(src, r, tile, ok, a, b, jj);
 #pragma unroll
         for (int u = 0; u < ITEMS; u++) {
-            const u64 j = tile * span + (u64)u * blockDim.x + threadIdx.x;
-            const u64 jc = j < r.count ? j : r.count - 1;          // keep the loads in range
-            double a = 0.0, b = 0.0;
-            ok[u] = src.get(jc, r.first + jc, a, b) && j < r.count;
-            it[u].x = enc(a); it[u].y = enc(b); it[u].idx = r.first + j;
+            P3 it;
+            it.x = enc(a[u]); it.y = enc(b[u]); it.idx = r.first + jj[u];
+            acc.push(ok[u], it);
         }
-#pragma unroll
-        for (int u = 0; u < ITEMS; u++) acc.push(ok[u], it[u]);
     }
     pareto_store_and_fold(acc, blockIdx.x, gridDim.x, ticket, sizes, partial, idx_out, out_cap, count_out);
 }
@@ -689,6 +809,16 @@ static size_t topk_lists_offset(u32 max_blocks) { return 256 + ((size_t)max_bloc
 size_t topk_workspace_bytes(u32 k) { return topk_lists_offset(SEL_MAX_BLOCKS) + (size_t)SEL_MAX_BLOCKS * k * sizeof(KI); }
 size_t pareto_workspace_bytes() {
     return 256 + (size_t)SEL_MAX_BLOCKS * sizeof(u32) + (size_t)SEL_MAX_BLOCKS * GUIDE_PARETO_MAX * sizeof(P3);
+}
+
+// Are all arrays a scan over materialised metrics will touch aligned for 16-byte loads?
+static int mat_vec_ok(const guide_outputs &o, const guide_constraints &c, int m0, int m1) {
+    auto al = [](const void *p, uintptr_t a) { return ((uintptr_t)p % a) == 0; };
+    const double *arrs[] = {o.latency, o.ttft, o.ttft_p50, o.ttft_p99, o.tpot, o.thr_decode, o.cost_per_hr, o.cost_per_token};
+    (void)c; (void)m0; (void)m1;
+    for (const double *p : arrs)
+        if (p && !al(p, 16)) return 0;
+    return al(o.status, 4) ? 1 : 0;
 }
 
 static Cons make_cons(const guide_constraints &c) {
@@ -789,7 +919,7 @@ int launch_topk(const DSpace &s, Range r, const guide_outputs *mat, int time_mod
     const int negate = key == GUIDE_THROUGHPUT;
     unsigned char *w = (unsigned char *)ws;
     if (mat) {
-        MatSource src{*mat, make_cons(c), key, -1};
+        MatSource src{*mat, make_cons(c), key, -1, mat_vec_ok(*mat, c, key, -1)};
         return run_topk_scan(src, r, k, negate, SEL_MAX_BLOCKS, w, idx_out, key_out, count_out, st);
     }
     TileGeom g;
@@ -838,7 +968,7 @@ int launch_pareto(const DSpace &s, Range r, const guide_outputs *mat, int time_m
                   const guide_constraints &c, int xm, int ym, u64 *idx_out, u32 cap, u32 *count_out, void *ws,
                   cudaStream_t st) {
     if (mat) {
-        MatSource src{*mat, make_cons(c), xm, ym};
+        MatSource src{*mat, make_cons(c), xm, ym, mat_vec_ok(*mat, c, xm, ym)};
         return run_pareto_scan(src, r, idx_out, cap, count_out, ws, st);
     }
     TileGeom g;
@@ -889,7 +1019,7 @@ int launch_topk_noalloc(Range r, const guide_outputs &mat, const guide_constrain
     const int rc = noalloc_scratch_address(&scratch);
     if (rc) return rc;
     static_assert(256 + NOALLOC_BLOCKS * 4 == 1280, "list offset below assumes a 256-byte multiple");
-    MatSource src{mat, make_cons(c), key, -1};
+    MatSource src{mat, make_cons(c), key, -1, mat_vec_ok(mat, c, key, -1)};
     // The array still holds the previous call's bound, counts and lists.  The bound word is reset
     // on this stream before the scan; counts and lists need no clearing: every block of this
     // launch writes its own before the merge kernel, which follows on the same stream and reads

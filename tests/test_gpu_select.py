@@ -94,6 +94,16 @@ def test_pareto_materialised_and_fused(c2_small):
 
 def test_selection_on_a_sub_range(c2_small):
     w, want, out_dev, sp = c2_small
+    # an odd offset: the arrays handed over are not 16-byte aligned, so the scalar loads are used
+    f1, c1 = 1001, 40003
+    sub1 = {k: v[f1:f1 + c1] for k, v in want.items()}
+    dev1 = {k: v[f1:f1 + c1] for k, v in out_dev.items()}
+    idx, val, cnt = run_topk(sp, dev1, {"max_latency": 5.0}, "cost_per_token", 32, first=f1, count=c1)
+    w_idx, w_val, w_cnt = oracle.select_topk(sub1, {"max_latency": 5.0}, "cost_per_token", 32, first=f1)
+    assert cnt == w_cnt and np.array_equal(idx, w_idx)
+    fidx, fcnt = run_pareto(sp, dev1, {}, "latency", "cost_per_token", first=f1, count=c1)
+    w_f, w_n = oracle.pareto(sub1, {}, "latency", "cost_per_token", first=f1)
+    assert fcnt == w_n and np.array_equal(fidx, w_f)
     first, count = 1000, 50001
     sub = {k: v[first:first + count] for k, v in want.items()}
     sub_dev = {k: v[first:first + count] for k, v in out_dev.items()}
