@@ -3,13 +3,14 @@
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--extras LIST]
 
-A step is one pass of the whole closed-form path over the 983,040-config grid (workload 2):
+A step is one pass of the whole closed-form path over the 16,777,216-config sweep (workload 5):
 guide_simulate (memory check, task list, roofline, metrics -> 6 fp64 arrays + mask + B_max),
-guide_select_topk (constraint filter + top-8 by cost per token) and guide_pareto (latency vs $/h),
+guide_select_topk (constraint filter + top-64 by cost per token) and guide_pareto (latency vs $/h),
 with the space tables already resident on the device.  `value` is configs per second over the K
-timed steps; L2 is flushed between steps (outputs are smaller than L2).  The trace-driven
-workloads (1, 3, 4) and the 16.7M-config sweep (5) are timed once each afterwards and reported
-under "workloads" with configs/s and simulated request-iterations/s.
+timed steps; the 0.89 GB of outputs a step writes and reads back exceed L2 several times over, so
+no flush is needed between steps.  The trace-driven workloads (1, 3, 4), the 983,040-config grid
+(2) and the fused (nothing materialised) selection on workload 5 are timed once each afterwards
+and reported under "workloads" with configs/s and simulated request-iterations/s.
 
 With N > 1 (launched by torchrun) every rank evaluates a grid of the same size over its own slice
 of an N-times longer hardware axis (weak scaling); the only exchange is an all-gather of each
@@ -34,8 +35,6 @@ if ROOT not in sys.path:
 import numpy as np
 
 BYTES_SIM = 6 * 8 + 1 + 4          # six fp64 metrics + status + bmax written per config
-BYTES_TOPK = 1 + 8                 # status + key read per config
-BYTES_PARETO = 1 + 8 + 8           # status + two metrics read per config
 SIM_FIELDS = ("latency", "ttft", "tpot", "thr_decode", "cost_per_hr", "cost_per_token", "status", "bmax")
 TRACE_FIELDS = ("latency", "ttft", "ttft_p50", "ttft_p99", "tpot", "thr_decode", "cost_per_hr", "cost_per_token",
                 "status", "bmax", "n_iters", "n_req_iters")
@@ -111,7 +110,7 @@ def run_reference(args):
         return
     import oracle
     from paper_2412_04788_b200 import inputs
-    w = inputs.workload(2)
+    w = inputs.workload(5)
     n = inputs.space_size(w["space"])
     for _ in range(args.warmup):
         oracle_step(oracle, w)
@@ -124,7 +123,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": "configs/sec", "value": value, "unit": "configs/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "C2 closed-form grid, 983040 configs: simulate + top-8 + Pareto"},
+            "config": {"workload": "C5 closed-form sweep, 16777216 configs: simulate + top-64 + Pareto"},
             "cpu_baseline": {"value": value, "unit": "configs/s", "cores": cores, "kind": "oracle",
                              "sample": f"the whole workload, {args.steps} passes"},
             "e2e": {"value": value, "unit": "configs/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -215,21 +214,23 @@ def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full, fraction
                             "request_iters_per_s": req_iters / best * 1e3, "request_iters": req_iters,
                             "hardware_axis_fraction": scale, "kernel_launches": 1, **extra}
             del out, ws
-        elif k == 5:
-            w = inputs.workload(5)
+        elif k in (2, 5):
+            w = inputs.workload(k, scale=fraction if (fraction and k == 5) else 1.0)
             p = ClosedFormPath(guide, torch, w["space"], w["constraints"], w["topk"]["key"], w["topk"]["k"])
             n = p.n
-            t_sim = time_call(torch, p.simulate, flush=flush)[0]
-            t_kf = time_call(torch, lambda: p.topk(True), flush=flush)[0]
-            t_pf = time_call(torch, lambda: p.pareto(True), flush=flush)[0]
-            t_km = time_call(torch, lambda: p.topk(False), flush=flush)[0]
-            t_pm = time_call(torch, lambda: p.pareto(False), flush=flush)[0]
-            res["C5"] = {"configs": n, "front": int(p.fcnt.item()), "found": int(p.cnt.item()),
-                         "fused_ms": {"topk": t_kf, "pareto": t_pf}, "fused_configs_per_s": n / (t_kf + t_pf) * 1e3,
-                         "materialised_ms": {"simulate": t_sim, "topk": t_km, "pareto": t_pm},
-                         "materialised_configs_per_s": n / (t_sim + t_km + t_pm) * 1e3,
-                         "simulate_write_gbs": BYTES_SIM * n / t_sim / 1e6,
-                         "simulate_frac_of_hbm": BYTES_SIM * n / t_sim / 1e6 / hbm_peak, "kernel_launches": 5}
+            fl = flush if k == 2 else None          # workload 2's outputs fit in L2: evict them
+            t_sim = time_call(torch, p.simulate, flush=fl)[0]
+            t_kf = time_call(torch, lambda: p.topk(True), flush=fl)[0]
+            t_pf = time_call(torch, lambda: p.pareto(True), flush=fl)[0]
+            t_km = time_call(torch, lambda: p.topk(False), flush=fl)[0]
+            t_pm = time_call(torch, lambda: p.pareto(False), flush=fl)[0]
+            res[f"C{k}"] = {"configs": n, "front": int(p.fcnt.item()), "found": int(p.cnt.item()),
+                            "fused_ms": {"topk": t_kf, "pareto": t_pf}, "fused_configs_per_s": n / (t_kf + t_pf) * 1e3,
+                            "materialised_ms": {"simulate": t_sim, "topk": t_km, "pareto": t_pm},
+                            "materialised_configs_per_s": n / (t_sim + t_km + t_pm) * 1e3,
+                            "simulate_write_gbs": BYTES_SIM * n / t_sim / 1e6,
+                            "simulate_frac_of_hbm": BYTES_SIM * n / t_sim / 1e6 / hbm_peak,
+                            "kernel_launches": 3 + 2 * 2 + 1}
             del p
         torch.cuda.empty_cache()
     return res
@@ -253,14 +254,14 @@ def run_ours(args):
     guide.lib()
 
     hbm_peak, peak_kind = measured_peaks()
-    # workload 2; with N ranks the hardware axis is N times longer and each rank takes one slice
-    w = inputs.workload(2, scale=float(world))
+    # workload 5; with N ranks the hardware axis is N times longer and each rank takes one slice
+    w = inputs.workload(5, scale=float(world) * (args.trace_fraction if args.main_fraction else 1.0))
     global_space = w["space"]
     local_space, hw_off = sharding.shard_space(global_space, rank, world) if world > 1 else (global_space, 0)
     k, key, cons = w["topk"]["k"], w["topk"]["key"], w["constraints"]
     path = ClosedFormPath(guide, torch, local_space, cons, key, k)
     n_local = path.n
-    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")   # used for workload 2 only
 
     def exchange():
         """all-gather of the k local candidates, then the same kernel merges them"""
@@ -270,7 +271,7 @@ def run_ours(args):
         order = sharding.order_for_merge(all_idx)
         all_idx, all_val = all_idx[order], all_val[order]
         m = all_idx.numel()
-        gathered = {"status": (all_idx < 0).to(torch.uint8), "cost_per_token": all_val.contiguous()}
+        gathered = {"status": (all_idx < 0).to(torch.uint8), key: all_val.contiguous()}
         guide.guide_select_topk(path.sp, None, gathered, {}, key, k, path.idx, path.val, path.cnt, path.ws_k, count=m)
         return all_idx
 
@@ -300,8 +301,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     wall0 = time.perf_counter()
     for i in range(args.steps):
-        flush.zero_()                     # outputs (52 MB) fit in L2: evict them between steps
-        step(evs[i])
+        step(evs[i])                      # 0.89 GB written and re-read per step: nothing survives in L2
     torch.cuda.synchronize()
     wall = time.perf_counter() - wall0
     sampler.stop_flag = True
@@ -323,7 +323,7 @@ def run_ours(args):
     host = {f: torch.empty_like(t, device="cpu").pin_memory() for f, t in path.out.items()}
     host_idx, host_val = torch.empty(k, dtype=torch.int64).pin_memory(), torch.empty(k, dtype=torch.float64).pin_memory()
     host_front = torch.empty(guide.PARETO_MAX, dtype=torch.int64).pin_memory()
-    e2e_steps = min(args.steps, 20)
+    e2e_steps = min(args.steps, 5)
 
     def e2e_step():
         sp = guide.Space(local_space)                      # host tables -> validated -> uploaded on first use
@@ -338,7 +338,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         sp.close()
 
-    for _ in range(3):
+    for _ in range(2):
         e2e_step()
     torch.cuda.synchronize()
     if world > 1:
@@ -360,9 +360,15 @@ def run_ours(args):
         return
 
     # ---- roofline of the dominant kernel of the step ----
+    # bytes a scan must read per config: status, each distinct metric array, each bounded array
+    bounded = {"max_latency": "latency", "max_cost_per_hr": "cost_per_hr", "min_throughput": "thr_decode",
+               "max_ttft": "ttft"}
+    cons_arrays = {arr for name, arr in bounded.items() if name in cons}
+    bytes_topk = 1 + 8 * len(cons_arrays | {key})
+    bytes_pareto = 1 + 8 * len(cons_arrays | {"latency", "cost_per_hr"})
     per = {"guide_simulate (k_closed_form_tiled)": (t_sim / args.steps, BYTES_SIM),
-           "guide_select_topk (k_topk)": (t_topk / args.steps, BYTES_TOPK),
-           "guide_pareto (k_pareto)": (t_par / args.steps, BYTES_PARETO)}
+           "guide_select_topk (k_topk_scan + k_topk_merge)": (t_topk / args.steps, bytes_topk),
+           "guide_pareto (k_pareto_scan)": (t_par / args.steps, bytes_pareto)}
     dom = max(per, key=lambda name: per[name][0])
     dom_ms, dom_bytes = per[dom]
     achieved = dom_bytes * n_local / (dom_ms * 1e-3) / 1e9
@@ -378,25 +384,27 @@ def run_ours(args):
         import oracle
         oracle_step(oracle, w)
         reps, t0 = 0, time.perf_counter()
-        while reps < 5 or time.perf_counter() - t0 < 2.0:
+        while reps < 3 or time.perf_counter() - t0 < 10.0:
             oracle_step(oracle, w)
             reps += 1
         dt = time.perf_counter() - t0
         cpu = {"value": n_local * reps / dt, "unit": "configs/s", "cores": oracle.threads(), "kind": "oracle",
-               "sample": f"the whole 983040-config workload (simulate + top-{k} + Pareto), {reps} passes"}
+               "sample": f"the whole {n_local}-config workload (simulate + top-{k} + Pareto), {reps} passes"}
 
     extras = {}
     if world == 1 and args.extras:
         which = [int(x) for x in args.extras.split(",") if x]
         extras = extra_workloads(guide, torch, inputs, which, flush, hbm_peak, args.full, args.trace_fraction)
 
-    launches_per_step = 3 + (1 if world > 1 else 0)
+    launches_per_step = 4 + (2 if world > 1 else 0)      # simulate, top-k scan + merge, Pareto (+ merge of gathered lists)
     line = {"metric": "configs/sec", "value": value, "unit": "configs/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "C2 closed-form grid: 8 models x 16 hw x 3 fw x 10 batch x 4 TP x 64 length pairs "
-                                   f"= {n_local} configs per GPU; simulate + top-{k} by cost/token + Pareto(latency, $/h)",
-                       "l2": "256 MB buffer written between timed steps", "timing": "CUDA events per step, summed"},
+            "config": {"workload": "C5 closed-form sweep: 16 models x 64 hw x 4 fw x 16 batch x 4 TP x 64 length pairs "
+                                   f"= {n_local} configs per GPU; simulate (materialised) + top-{k} by cost/token under the "
+                                   "latency bound + Pareto(latency, $/h)",
+                       "l2": "no flush: each step writes and re-reads 0.89 GB, several times the 126 MB L2",
+                       "timing": "CUDA events per step, summed"},
             "clocks": sampler.summary(),
             "e2e": {"value": e2e_value, "unit": "configs/s", "h2d_bytes_per_step": table_bytes(local_space),
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps},
@@ -414,11 +422,13 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--extras", default="1,3,4,5", help="other workloads to time after the main loop ('' = none)")
+    ap.add_argument("--extras", default="1,2,3,4,5", help="other workloads to time after the main loop ('' = none)")
+    ap.add_argument("--main-fraction", action="store_true",
+                    help="apply --trace-fraction to the main workload's hardware axis too (small cases for profiler captures)")
     ap.add_argument("--full", action="store_true", help="(kept for compatibility: workloads 3 and 4 now always run whole)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
     ap.add_argument("--trace-fraction", type=float, default=None,
-                    help="fraction of the hardware axis of workloads 3 and 4 (small cases for profiler captures)")
+                    help="fraction of the hardware axis of workloads 3, 4 and 5 in the extras (small cases for profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
