@@ -405,14 +405,15 @@ struct ParetoAcc {
     u32 *cnt;
     u32 *scratch;     // shared, 2 * 32 words
     u32 nf, c;
+    u32 cap;          // entries of buf this accumulator may use
     u32 budget, ramp;
     u64 kx[4], ky[4];  // a few front points kept in registers: most configs are beaten by one of them
     bool overflow;
     bool lazy;        // folding fronts: incoming points are mostly keepers, merge only when the buffer fills
 
-    __device__ void init(P3 *b, u32 *cn, u32 *sc, bool lazy_ = false) {
-        buf = b; cnt = cn; scratch = sc; nf = 0; c = 0; overflow = false; lazy = lazy_;
-        budget = lazy_ ? (PARETO_CAP / 2) / blockDim.x : 1; ramp = lazy_ ? MAX_BUDGET : 1;
+    __device__ void init(P3 *b, u32 *cn, u32 *sc, bool lazy_ = false, u32 cap_ = PARETO_CAP) {
+        buf = b; cnt = cn; scratch = sc; nf = 0; c = 0; overflow = false; lazy = lazy_; cap = cap_;
+        budget = lazy_ ? max(1u, (cap_ / 2) / blockDim.x) : 1; ramp = lazy_ ? min(budget, MAX_BUDGET) : 1;
 #pragma unroll
         for (int i = 0; i < 4; i++) { kx[i] = KEY_MAX; ky[i] = KEY_MAX; }
         if (threadIdx.x == 0) *cnt = 0;
@@ -482,6 +483,7 @@ struct ParetoAcc {
             __syncthreads();
         }
         if (out > GUIDE_PARETO_MAX) { overflow = true; out = GUIDE_PARETO_MAX; }
+        if (out + blockDim.x > cap) { overflow = true; out = cap - blockDim.x; }
         nf = out; c = out;
         if (threadIdx.x == 0) *cnt = out;
         __syncthreads();
@@ -504,23 +506,130 @@ struct ParetoAcc {
     // filtered) and whenever a block's worth of points has slipped past the stale front.
     __device__ void checkpoint() {
         __syncthreads();
-        c = *cnt;
+        c = min(*cnt, cap);
         __syncthreads();
-        if (ramp < MAX_BUDGET) ramp *= 2;
+        if (ramp < MAX_BUDGET && 4 * ramp * blockDim.x <= cap) ramp *= 2;
         const bool early = !lazy && ((nf == 0 && c > 0) || c >= nf + blockDim.x);
-        if (early || c + ramp * blockDim.x > PARETO_CAP) merge();
-        budget = min(ramp, (PARETO_CAP - c) / blockDim.x);
+        if (early || c + ramp * blockDim.x > cap) merge();
+        // a front that leaves no room for one more round of appends cannot be handled in this buffer
+        if (c + blockDim.x > cap) { overflow = true; nf = c = cap - blockDim.x; if (threadIdx.x == 0) *cnt = c; __syncthreads(); }
+        budget = max(1u, min(ramp, (cap - c) / blockDim.x));
     }
     // every thread of the block calls it the same number of times; a barrier only when the budget runs out
     __device__ __forceinline__ void push(bool ok, const P3 &it) {
-        if (ok && !killed(it) && !beaten(it)) buf[atomicAdd(cnt, 1)] = it;
+        if (ok && !killed(it) && !beaten(it)) {
+            const u32 pos = atomicAdd(cnt, 1);
+            if (pos < cap) buf[pos] = it;      // always true by the checkpoint rule; kept as a guard
+        }
         if (--budget == 0) checkpoint();
     }
     __device__ void finish() {
         __syncthreads();
-        c = *cnt;
+        c = min(*cnt, cap);
         __syncthreads();
         merge();
+    }
+};
+
+// ---- per-warp Pareto accumulator ---------------------------------------------------------------
+//
+// The barrier-free counterpart of ParetoAcc for the common case of small fronts.  Each warp keeps
+// its own front, sorted by x, in a small segment of shared memory; survivors of a round are placed
+// behind it by ballot, and when a warp-load of them has gathered the warp sorts and sweeps its
+// segment alone.  A front that outgrows the segment raises a flag and the caller's general
+// (block-level) kernel redoes the work.
+
+static constexpr u32 WSEG = 128;                 // entries per warp segment
+
+struct WarpPareto {
+    P3 *seg;
+    u32 nf, fill;
+    u64 kx[4], ky[4];
+    bool overflow;
+
+    __device__ void init(P3 *smem) {
+        seg = smem + (size_t)(threadIdx.x >> 5) * WSEG;
+        nf = 0; fill = 0; overflow = false;
+#pragma unroll
+        for (int i = 0; i < 4; i++) { kx[i] = KEY_MAX; ky[i] = KEY_MAX; }
+    }
+    __device__ __forceinline__ bool killed(const P3 &it) const {
+        bool k = false;
+#pragma unroll
+        for (int i = 0; i < 4; i++) k |= (kx[i] <= it.x && ky[i] <= it.y) && (kx[i] < it.x || ky[i] < it.y);
+        return k;
+    }
+    __device__ __forceinline__ bool beaten(const P3 &it) const {
+        u32 lo = 0, hi = nf;                   // first front point with x > it.x
+        while (lo < hi) {
+            const u32 mid = (lo + hi) >> 1;
+            if (seg[mid].x <= it.x) lo = mid + 1; else hi = mid;
+        }
+        if (lo == 0) return false;
+        const P3 p = seg[lo - 1];
+        if (p.y < it.y) return true;
+        if (p.y > it.y) return false;
+        return p.x < it.x || p.idx < it.idx;
+    }
+    // sort the segment by (x, y, idx); a point stays iff its y is below every earlier y
+    __device__ void merge() {
+        const u32 lane = threadIdx.x & 31;
+        const u32 P = next_pow2(fill);
+        for (u32 i = fill + lane; i < P; i += 32) { seg[i].x = KEY_MAX; seg[i].y = KEY_MAX; seg[i].idx = KEY_MAX; }
+        __syncwarp();
+        for (u32 size = 2; size <= P; size <<= 1) {
+            for (u32 stride = size >> 1; stride > 0; stride >>= 1) {
+                for (u32 i = lane; i < (P >> 1); i += 32) {
+                    const u32 lo = ((i & ~(stride - 1)) << 1) | (i & (stride - 1));
+                    const u32 hi = lo + stride;
+                    const bool up = (lo & size) == 0;
+                    const P3 a = seg[lo], b = seg[hi];
+                    if (p3_less(b, a) == up) { seg[lo] = b; seg[hi] = a; }
+                }
+                __syncwarp();
+            }
+        }
+        u64 carry = KEY_MAX;
+        u32 out = 0;
+        for (u32 base = 0; base < fill; base += 32) {
+            const u32 pos = base + lane;
+            const bool valid = pos < fill;
+            P3 it;
+            if (valid) it = seg[pos]; else { it.x = KEY_MAX; it.y = KEY_MAX; it.idx = KEY_MAX; }
+            u64 incl = it.y;
+            for (u32 d = 1; d < 32; d <<= 1) {
+                const u64 o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                if (lane >= d && o < incl) incl = o;
+            }
+            const u64 prev = __shfl_up_sync(0xFFFFFFFFu, incl, 1);
+            const u64 before = lane == 0 ? carry : (prev < carry ? prev : carry);   // smallest y before this point
+            const bool keep = valid && it.y < before;
+            const u32 ballot = __ballot_sync(0xFFFFFFFFu, keep);      // also orders this round's reads before its writes
+            if (keep) seg[out + __popc(ballot & ((1u << lane) - 1))] = it;
+            out += __popc(ballot);
+            const u64 last = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            if (last < carry) carry = last;
+            __syncwarp();
+        }
+        if (out + 32 > WSEG) { overflow = true; out = WSEG - 32; }     // no room for another round: flag it
+        nf = out; fill = out;
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            if (nf > 0) { const P3 p = seg[(nf * (2 * i + 1)) / 8]; kx[i] = p.x; ky[i] = p.y; }
+            else { kx[i] = KEY_MAX; ky[i] = KEY_MAX; }
+        }
+        __syncwarp();
+    }
+    // all 32 lanes of the warp call it together
+    __device__ __forceinline__ void push(bool ok, const P3 &it) {
+        const bool take = ok && !killed(it) && !beaten(it);
+        const u32 ballot = __ballot_sync(0xFFFFFFFFu, take);
+        if (ballot) {
+            if (take) seg[fill + __popc(ballot & ((1u << (threadIdx.x & 31)) - 1))] = it;
+            fill += __popc(ballot);
+            __syncwarp();
+            if (nf == 0 || fill >= nf + 32 || fill + 32 > WSEG) merge();
+        }
     }
 };
 
@@ -692,7 +801,7 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_merge(u32 nblk, u32 k, con
 // sum over the front sizes turns them into one flat list, so the number of collective steps
 // depends on the number of points, not on the number of blocks.
 __device__ void pareto_store_and_fold(ParetoAcc &acc, u32 block, u32 nblk, u32 *ticket, u32 *sizes, P3 *partial,
-                                      u64 *idx_out, u32 out_cap, u32 *count_out) {
+                                      u64 *idx_out, u32 out_cap, u32 *count_out, u32 *redo_flag = nullptr) {
     __shared__ u32 last_flag;
     __shared__ u32 pre[SEL_MAX_BLOCKS + 1];
     __shared__ u32 wsum[SEL_THREADS / 32];
@@ -732,7 +841,7 @@ __device__ void pareto_store_and_fold(ParetoAcc &acc, u32 block, u32 nblk, u32 *
         run += bi < nblk ? (__ldcg(sizes + bi) & 0x7FFFFFFFu) : 0u;
     }
     if (threadIdx.x == blockDim.x - 1) pre[SEL_MAX_BLOCKS] = run;
-    acc.init(acc.buf, acc.cnt, acc.scratch, true);      // includes a barrier: pre[] is complete
+    acc.init(acc.buf, acc.cnt, acc.scratch, true, acc.cap);   // includes a barrier: pre[] is complete
     const u32 total = pre[SEL_MAX_BLOCKS];
     for (u32 base = 0; base < total; base += blockDim.x) {
         const u32 i = base + threadIdx.x;
@@ -752,17 +861,55 @@ __device__ void pareto_store_and_fold(ParetoAcc &acc, u32 block, u32 nblk, u32 *
     acc.finish();
     overflow |= acc.overflow;
     for (u32 i = threadIdx.x; i < acc.nf && i < out_cap; i += blockDim.x) idx_out[i] = acc.buf[i].idx;
-    if (threadIdx.x == 0) *count_out = overflow ? 0xFFFFFFFFu : acc.nf;
+    if (threadIdx.x == 0) {
+        *count_out = overflow ? 0xFFFFFFFFu : acc.nf;
+        if (overflow && redo_flag) *redo_flag = 1;       // the general kernel, queued behind, redoes the work
+    }
 }
 
-template <class Src>
-__global__ void __launch_bounds__(SEL_THREADS) k_pareto_scan(Src src, Range r, u32 *ticket, u32 *sizes, P3 *partial,
-                                                             u64 *idx_out, u32 out_cap, u32 *count_out) {
+// Block end of the per-warp mode: the warps' fronts are pooled into one block accumulator (its
+// buffer is the segments' own shared memory), which then goes the usual way.
+__device__ void warp_pareto_pool(WarpPareto &w, ParetoAcc &acc, P3 *smem, u32 *cnt, u32 *scratch) {
+    __shared__ u32 wfill[SEL_THREADS / 32];
+    const u32 lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    if (w.fill > w.nf) w.merge();
+    P3 mine[WSEG / 32];
+#pragma unroll
+    for (u32 q = 0; q < WSEG / 32; q++) {
+        const u32 i = q * 32 + lane;
+        if (i < w.nf) mine[q] = w.seg[i];
+    }
+    if (lane == 0) wfill[warp] = w.nf;
+    const bool any_overflow = __syncthreads_or(w.overflow) != 0;     // also: every segment is in registers
+    u32 off = 0, total = 0;
+    for (u32 x = 0; x < n_warps; x++) {
+        if (x < warp) off += wfill[x];
+        total += wfill[x];
+    }
+#pragma unroll
+    for (u32 q = 0; q < WSEG / 32; q++) {
+        const u32 i = q * 32 + lane;
+        if (i < w.nf) smem[off + i] = mine[q];
+    }
+    acc.init(smem, cnt, scratch, false, n_warps * WSEG);            // barrier inside: the pool is complete
+    if (threadIdx.x == 0) *cnt = total;
+    acc.overflow = any_overflow;
+}
+
+// Workspace header of a Pareto call: word 0 = ticket of the per-warp (fast) kernel, word 1 = redo
+// flag it raises when a front outgrew a warp segment, word 2 = ticket of the general kernel.
+// The general kernel with `gate` set does nothing unless the redo flag is up.
+
+template <class Src, bool WARP>
+__global__ void __launch_bounds__(SEL_THREADS) k_pareto_scan(Src src, Range r, u32 *header, const u32 *gate, u32 *sizes,
+                                                             P3 *partial, u64 *idx_out, u32 out_cap, u32 *count_out) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ u32 cnt;
     __shared__ __align__(8) u32 scratch[64];
+    if (gate && __ldcg(gate) == 0) return;
     ParetoAcc acc;
-    acc.init((P3 *)smem_raw, &cnt, scratch);
+    WarpPareto wacc;
+    if (WARP) wacc.init((P3 *)smem_raw); else acc.init((P3 *)smem_raw, &cnt, scratch);
     constexpr int ITEMS = Src::ITEMS;
     const u64 span = (u64)ITEMS * blockDim.x;
     const u64 tiles = (r.count + span - 1) / span;
@@ -775,30 +922,35 @@ __global__ void __launch_bounds__(SEL_THREADS) k_pareto_scan(Src src, Range r, u
         for (int u = 0; u < ITEMS; u++) {
             P3 it;
             it.x = enc(a[u]); it.y = enc(b[u]); it.idx = r.first + jj[u];
-            acc.push(ok[u], it);
+            if (WARP) wacc.push(ok[u], it); else acc.push(ok[u], it);
         }
     }
-    pareto_store_and_fold(acc, blockIdx.x, gridDim.x, ticket, sizes, partial, idx_out, out_cap, count_out);
+    if (WARP) warp_pareto_pool(wacc, acc, (P3 *)smem_raw, &cnt, scratch);
+    pareto_store_and_fold(acc, blockIdx.x, gridDim.x, header + (WARP ? 0 : 2), sizes, partial, idx_out, out_cap, count_out,
+                          WARP ? header + 1 : nullptr);
 }
 
-template <int TIME_SUM>
+template <int TIME_SUM, bool WARP>
 __global__ void __launch_bounds__(SEL_THREADS, 2)
-k_pareto_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, Cons c, int xm, int ym, u32 *ticket,
-               u32 *sizes, P3 *partial, u64 *idx_out, u32 out_cap, u32 *count_out) {
+k_pareto_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, Cons c, int xm, int ym, u32 *header,
+               const u32 *gate, u32 *sizes, P3 *partial, u64 *idx_out, u32 out_cap, u32 *count_out) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ u32 cnt;
     __shared__ __align__(8) u32 scratch[64];
+    if (gate && __ldcg(gate) == 0) return;
     ParetoAcc acc;
-    acc.init((P3 *)smem_raw, &cnt, scratch);
+    WarpPareto wacc;
+    if (WARP) wacc.init((P3 *)smem_raw); else acc.init((P3 *)smem_raw, &cnt, scratch);
     tiled_visit<TIME_SUM>(s, r, tp_model, hf_chunk, tiles_per_mb, [&](bool valid, u64 idx, const Metrics &m) {
         double a = 0.0, b = 0.0;
         const bool ok = valid && fused_pick(m, c, xm, ym, a, b);
         P3 it;
         it.x = enc(a); it.y = enc(b); it.idx = idx;
-        acc.push(ok, it);
+        if (WARP) wacc.push(ok, it); else acc.push(ok, it);
     });
-    pareto_store_and_fold(acc, blockIdx.y * gridDim.x + blockIdx.x, gridDim.x * gridDim.y, ticket, sizes, partial, idx_out,
-                          out_cap, count_out);
+    if (WARP) warp_pareto_pool(wacc, acc, (P3 *)smem_raw, &cnt, scratch);
+    pareto_store_and_fold(acc, blockIdx.y * gridDim.x + blockIdx.x, gridDim.x * gridDim.y, header + (WARP ? 0 : 2), sizes,
+                          partial, idx_out, out_cap, count_out, WARP ? header + 1 : nullptr);
 }
 
 // ---- host side -----------------------------------------------------------------------------------------
@@ -934,16 +1086,25 @@ int launch_topk(const DSpace &s, Range r, const guide_outputs *mat, int time_mod
     return run_topk_scan(src, r, k, negate, SEL_MAX_BLOCKS, w, idx_out, key_out, count_out, st);
 }
 
+// Per-warp kernel first; the general kernel is queued right behind it and returns at once unless
+// the first one raised the redo flag (a front too large for a warp segment).
 template <class Src>
 static int run_pareto_scan(const Src &src, Range r, u64 *idx_out, u32 cap, u32 *count_out, void *ws, cudaStream_t st) {
-    const size_t smem = (size_t)PARETO_CAP * sizeof(P3);
-    int rc = allow_smem(k_pareto_scan<Src>, smem);
+    const size_t smem_fast = (size_t)(SEL_THREADS / 32) * WSEG * sizeof(P3);
+    const size_t smem_gen = (size_t)PARETO_CAP * sizeof(P3);
+    int rc = allow_smem(k_pareto_scan<Src, false>, smem_gen);
     if (rc) return rc;
-    const u32 grid = grid_for(r.count, Src::ITEMS, 2, SEL_MAX_BLOCKS);
     GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
+    u32 *header = (u32 *)ws;
     u32 *sizes = (u32 *)((char *)ws + 256);
     P3 *partial = (P3 *)((char *)ws + 256 + (size_t)SEL_MAX_BLOCKS * sizeof(u32));
-    k_pareto_scan<Src><<<grid, SEL_THREADS, smem, st>>>(src, r, (u32 *)ws, sizes, partial, idx_out, cap, count_out);
+    const u32 grid_fast = grid_for(r.count, Src::ITEMS, 4, SEL_MAX_BLOCKS);
+    k_pareto_scan<Src, true><<<grid_fast, SEL_THREADS, smem_fast, st>>>(src, r, header, nullptr, sizes, partial, idx_out, cap,
+                                                                         count_out);
+    GUIDE_CUDA(cudaGetLastError());
+    const u32 grid_gen = grid_for(r.count, Src::ITEMS, 2, SEL_MAX_BLOCKS);
+    k_pareto_scan<Src, false><<<grid_gen, SEL_THREADS, smem_gen, st>>>(src, r, header, header + 1, sizes, partial, idx_out, cap,
+                                                                        count_out);
     GUIDE_CUDA(cudaGetLastError());
     return GUIDE_OK;
 }
@@ -951,15 +1112,21 @@ static int run_pareto_scan(const Src &src, Range r, u64 *idx_out, u32 cap, u32 *
 template <int TIME_SUM>
 static int run_pareto_tiled(const DSpace &s, Range r, const TileGeom &g, int tp_model, const Cons &c, int xm, int ym,
                             u64 *idx_out, u32 cap, u32 *count_out, void *ws, cudaStream_t st) {
-    const size_t smem = (size_t)PARETO_CAP * sizeof(P3);
-    int rc = allow_smem(k_pareto_tiled<TIME_SUM>, smem);
+    const size_t smem_fast = (size_t)(SEL_THREADS / 32) * WSEG * sizeof(P3);
+    const size_t smem_gen = (size_t)PARETO_CAP * sizeof(P3);
+    int rc = allow_smem(k_pareto_tiled<TIME_SUM, false>, smem_gen);
     if (rc) return rc;
     GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
+    u32 *header = (u32 *)ws;
     u32 *sizes = (u32 *)((char *)ws + 256);
     P3 *partial = (P3 *)((char *)ws + 256 + (size_t)SEL_MAX_BLOCKS * sizeof(u32));
     const dim3 grid(g.gx, g.splits);
-    k_pareto_tiled<TIME_SUM><<<grid, g.threads, smem, st>>>(s, r, tp_model, g.hf_chunk, g.tiles_per_mb, c, xm, ym,
-                                                           (u32 *)ws, sizes, partial, idx_out, cap, count_out);
+    k_pareto_tiled<TIME_SUM, true><<<grid, g.threads, smem_fast, st>>>(s, r, tp_model, g.hf_chunk, g.tiles_per_mb, c, xm, ym,
+                                                                      header, nullptr, sizes, partial, idx_out, cap, count_out);
+    GUIDE_CUDA(cudaGetLastError());
+    k_pareto_tiled<TIME_SUM, false><<<grid, g.threads, smem_gen, st>>>(s, r, tp_model, g.hf_chunk, g.tiles_per_mb, c, xm, ym,
+                                                                      header, header + 1, sizes, partial, idx_out, cap,
+                                                                      count_out);
     GUIDE_CUDA(cudaGetLastError());
     return GUIDE_OK;
 }
