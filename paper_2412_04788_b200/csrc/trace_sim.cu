@@ -89,7 +89,7 @@ __device__ __forceinline__ u64 work_to_index(const DSpace &s, u64 w, bool reorde
 }
 
 template <int TIME_SUM>
-__global__ void __launch_bounds__(SIM_THREADS, 2)
+__global__ void __launch_bounds__(SIM_THREADS, 3)
 k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide_outputs o, u32 *counter,
             unsigned char *scratch, size_t per_warp, u32 gen_bytes, u32 first_bytes, int reorder) {
     __shared__ SlotArrays sh[SIM_WARPS_PER_BLOCK];
