@@ -35,6 +35,9 @@ if ROOT not in sys.path:
 import numpy as np
 
 BYTES_SIM = 6 * 8 + 1 + 4          # six fp64 metrics + status + bmax written per config
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_closed_form_tiled launch on the full workload 5
+# (profiles/k_closed_form_tiled_c5.md); only meaningful for that size and that kernel version
+K1_TRAFFIC_C5 = 850_617_600 + 145_664
 SIM_FIELDS = ("latency", "ttft", "tpot", "thr_decode", "cost_per_hr", "cost_per_token", "status", "bmax")
 TRACE_FIELDS = ("latency", "ttft", "ttft_p50", "ttft_p99", "tpot", "thr_decode", "cost_per_hr", "cost_per_token",
                 "status", "bmax", "n_iters", "n_req_iters")
@@ -373,7 +376,9 @@ def run_ours(args):
     dom_ms, dom_bytes = per[dom]
     achieved = dom_bytes * n_local / (dom_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
-                "frac": achieved / hbm_peak, "traffic": None, "peak_kind": f"of {peak_kind}",
+                "frac": achieved / hbm_peak,
+                "traffic": K1_TRAFFIC_C5 if (dom.startswith("guide_simulate") and n_local == 16777216) else None,
+                "peak_kind": f"of {peak_kind}",
                 "bytes_per_config": dom_bytes,
                 "per_kernel_ms": {name: v[0] for name, v in per.items()},
                 "per_kernel_gbs": {name: v[1] * n_local / (v[0] * 1e-3) / 1e9 for name, v in per.items()}}
