@@ -59,6 +59,10 @@ def test_topk_large_k_and_ties(c2_small):
     check_topk(sp, out_dev, want, {}, "cost_per_hr", 1024)
     check_topk(sp, out_dev, want, {}, "cost_per_token", 1024)
     check_topk(sp, None, want, {}, "cost_per_hr", 300)
+    # 128 is the largest k of the per-warp accumulators, 129 the smallest of the per-block ones
+    for k in (128, 129):
+        check_topk(sp, out_dev, want, {}, "cost_per_token", k)
+        check_topk(sp, None, want, {}, "latency", k)
 
 
 def test_topk_fewer_than_k_and_none(c2_small):
