@@ -9,7 +9,6 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libguide.so")
 SOURCES = ["guide_api.cu", "closed_form.cu", "select.cu", "trace_sim.cu"]
-HEADERS = ["guide_internal.cuh", "model.cuh", os.path.join("..", "..", "include", "guide.h")]
 
 # -fmad=false: the model's arithmetic is defined without fused multiply-add (bit-exact with any
 # IEEE-754 binary64 implementation that evaluates the same expression order).
@@ -25,7 +24,8 @@ def stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = sources() + [os.path.join(CSRC, h) for h in HEADERS]
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh", ".h"))]
+    deps.append(os.path.join(HERE, "..", "include", "guide.h"))
     return any(os.path.getmtime(d) > t for d in deps if os.path.exists(d))
 
 

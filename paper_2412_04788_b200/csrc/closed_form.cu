@@ -34,8 +34,8 @@ __global__ void __launch_bounds__(256) k_closed_form_flat(DSpace s, Range r, int
 template <int TIME_SUM>
 __global__ void __launch_bounds__(256, 2) k_closed_form_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk,
                                                               u32 tiles_per_mb, guide_outputs o) {
-    tiled_visit<TIME_SUM>(s, r, tp_model, hf_chunk, tiles_per_mb, [&](bool valid, u64 idx, const Metrics &m) {
-        if (valid) store_metrics(o, idx - r.first, m);
+    tiled_visit<TIME_SUM>(s, r, tp_model, hf_chunk, tiles_per_mb, [&](bool valid, u64 j, const Metrics &m) {
+        if (valid) store_metrics(o, j, m);
     });
 }
 

@@ -1,4 +1,5 @@
 // Host side of the C ABI: validation, handles, table upload, argument checks, kernel dispatch.
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <new>
@@ -94,7 +95,7 @@ static int check_trace_overflow(const guide_space &s, const guide_trace &t) {
 // Derived per-model quantities and the reciprocal rates of every hardware x framework pair.
 __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *gh, u32 n_h, const guide_fw *gf,
                                u32 n_f, const u32 *tp, u32 n_t, DModel *dm, DRate *dr, double *cost_hr,
-                               double *cost_sec) {
+                               double *cost_sec, ulonglong2 *hfmem) {
     const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n_m) {
         const guide_model m = gm[i];
@@ -125,6 +126,7 @@ __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *g
         r.flash = f.flash;
         r.kv_block = f.kv_block;
         dr[i] = r;
+        hfmem[i] = make_ulonglong2(r.usable, (u64)r.kv_block);
         for (u32 k = 0; k < n_t; k++) {
             const double c = h.price_per_hr * (double)tp[k];
             cost_hr[i * n_t + k] = c;
@@ -149,7 +151,8 @@ int space_on_device(guide_space *s, DSpace *out) {
                  o_gf = take(n_f * sizeof(guide_fw)), o_dm = take(n_m * sizeof(DModel)),
                  o_dr = take(n_h * n_f * sizeof(DRate)), o_b = take(s->batch.size() * 4),
                  o_t = take(s->tp.size() * 4), o_p = take(s->pairs.size() * 8),
-                 o_ch = take(n_h * n_f * s->tp.size() * 8), o_cs = take(n_h * n_f * s->tp.size() * 8);
+                 o_ch = take(n_h * n_f * s->tp.size() * 8), o_cs = take(n_h * n_f * s->tp.size() * 8),
+                 o_lo = take(s->pairs.size() * 4), o_hm = take(n_h * n_f * 16);
     char *blob = nullptr;
     GUIDE_CUDA(cudaMalloc(&blob, off));
     cudaError_t e = cudaSuccess;
@@ -162,6 +165,15 @@ int space_on_device(guide_space *s, DSpace *out) {
     put(o_b, s->batch.data(), s->batch.size() * 4);
     put(o_t, s->tp.data(), s->tp.size() * 4);
     put(o_p, s->pairs.data(), s->pairs.size() * 8);
+    {
+        // walk order of the length pairs for the tiled kernels (an ordering only: no model arithmetic)
+        std::vector<uint32_t> order(s->pairs.size());
+        for (size_t i = 0; i < order.size(); i++) order[i] = (uint32_t)i;
+        std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) {
+            return (uint64_t)s->pairs[a].lin + s->pairs[a].lout < (uint64_t)s->pairs[b].lin + s->pairs[b].lout;
+        });
+        put(o_lo, order.data(), order.size() * 4);
+    }
     if (e == cudaSuccess) {
         const u32 n = (u32)std::max(n_m, n_h * n_f);
         k_build_tables<<<(n + 127) / 128, 128>>>((const guide_model *)(blob + o_gm), (u32)n_m,
@@ -169,7 +181,8 @@ int space_on_device(guide_space *s, DSpace *out) {
                                                  (const guide_fw *)(blob + o_gf), (u32)n_f,
                                                  (const u32 *)(blob + o_t), (u32)s->tp.size(),
                                                  (DModel *)(blob + o_dm), (DRate *)(blob + o_dr),
-                                                 (double *)(blob + o_ch), (double *)(blob + o_cs));
+                                                 (double *)(blob + o_ch), (double *)(blob + o_cs),
+                                                 (ulonglong2 *)(blob + o_hm));
         e = cudaGetLastError();
         if (e == cudaSuccess) e = cudaStreamSynchronize(0);
     }
@@ -184,6 +197,8 @@ int space_on_device(guide_space *s, DSpace *out) {
     d.view.pairs = (const uint2 *)(blob + o_p);
     d.view.cost_hr = (const double *)(blob + o_ch);
     d.view.cost_sec = (const double *)(blob + o_cs);
+    d.view.lorder = (const u32 *)(blob + o_lo);
+    d.view.hfmem = (const ulonglong2 *)(blob + o_hm);
     d.view.n_m = (u32)n_m; d.view.n_h = (u32)n_h; d.view.n_f = (u32)n_f;
     d.view.n_b = (u32)s->batch.size(); d.view.n_t = (u32)s->tp.size(); d.view.n_l = (u32)s->pairs.size();
     s->dev.push_back(d);

@@ -710,11 +710,11 @@ k_topk_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, Co
     __shared__ u32 cnt;
     typename TopKPick<WARP>::type acc;
     topk_begin(acc, (KI *)smem_raw, &cnt, k, gthr);
-    tiled_visit<TIME_SUM>(s, r, tp_model, hf_chunk, tiles_per_mb, [&](bool valid, u64 idx, const Metrics &m) {
+    tiled_visit<TIME_SUM>(s, r, tp_model, hf_chunk, tiles_per_mb, [&](bool valid, u64 j, const Metrics &m) {
         double a = 0.0, b;
         const bool ok = valid && fused_pick(m, c, key, -1, a, b);
         KI it;
-        it.key = enc(a); it.idx = idx;
+        it.key = enc(a); it.idx = r.first + j;
         acc.push(ok, it);
     });
     topk_end(acc, (KI *)smem_raw, blockIdx.y * gridDim.x + blockIdx.x, k, counts, lists);
@@ -941,11 +941,11 @@ k_pareto_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, 
     ParetoAcc acc;
     WarpPareto wacc;
     if (WARP) wacc.init((P3 *)smem_raw); else acc.init((P3 *)smem_raw, &cnt, scratch);
-    tiled_visit<TIME_SUM>(s, r, tp_model, hf_chunk, tiles_per_mb, [&](bool valid, u64 idx, const Metrics &m) {
+    tiled_visit<TIME_SUM>(s, r, tp_model, hf_chunk, tiles_per_mb, [&](bool valid, u64 j, const Metrics &m) {
         double a = 0.0, b = 0.0;
         const bool ok = valid && fused_pick(m, c, xm, ym, a, b);
         P3 it;
-        it.x = enc(a); it.y = enc(b); it.idx = idx;
+        it.x = enc(a); it.y = enc(b); it.idx = r.first + j;
         if (WARP) wacc.push(ok, it); else acc.push(ok, it);
     });
     if (WARP) warp_pareto_pool(wacc, acc, (P3 *)smem_raw, &cnt, scratch);

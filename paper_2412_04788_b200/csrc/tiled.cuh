@@ -22,8 +22,8 @@ struct TileGeom {
     u32 hf_chunk;       // pairs per chunk
 };
 
-// emit(valid, idx, metrics) is called by every thread of the block exactly hf_chunk times, valid or
-// not, so emit may contain block-wide barriers.
+// emit(valid, j, metrics), j = config index - r.first, is called by every thread of the block exactly
+// hf_chunk times, valid or not, so emit may contain block-wide barriers.
 template <int TIME_SUM, class Emit>
 __device__ __forceinline__ void tiled_visit(const DSpace &s, const Range &r, int tp_model, u32 hf_chunk,
                                             u32 tiles_per_mb, Emit &&emit) {
@@ -35,8 +35,12 @@ __device__ __forceinline__ void tiled_visit(const DSpace &s, const Range &r, int
     const u32 bpos = mb % s.n_b, mpos = mb / s.n_b;
     const u32 tl_raw = tile * blockDim.x + threadIdx.x;
     const bool active = tl_raw < n_tl;
-    const u32 tl = active ? tl_raw : n_tl - 1;
-    const u32 tpos = tl / s.n_l, lpos = tl % s.n_l;
+    // Threads walk the length pairs in order of lin + lout: whether a config fits in memory is
+    // monotone in that sum, so a warp's 32 configs are almost always all feasible or all not,
+    // instead of every warp paying for the evaluation of a few feasible lanes.
+    const u32 tl_t = active ? tl_raw : n_tl - 1;
+    const u32 tpos = tl_t / s.n_l, lpos = s.lorder[tl_t % s.n_l];
+    const u32 tl = tpos * s.n_l + lpos;
     const u32 hf0 = blockIdx.y * hf_chunk;
 
     const DModel m = s.models[mpos];
@@ -48,60 +52,79 @@ __device__ __forceinline__ void tiled_visit(const DSpace &s, const Range &r, int
     const double lf = log2_rule_factor(t, tp_model);
     const double Nd = (double)m.N;
 
+    // The stage tables are built when the first config of this thread turns out to fit: threads
+    // whose configs never do (head counts not divisible by the TP degree, lengths too long for
+    // every memory in the chunk) skip the integer work altogether.
     TaskTab kp, kd;
-    const u64 Tp = (u64)b * lin;
-    build_fixed_tasks(m, tt, Tp, b, 1, kp);
-    build_attn_tasks(m, tt, Tp, Tp * lin, Tp, kp);
-    {
+    bool built = false;
+    auto build_tables = [&]() {
+        const u64 Tp = (u64)b * lin;
+        build_fixed_tasks(m, tt, Tp, b, 1, kp);
+        build_attn_tasks(m, tt, Tp, Tp * lin, Tp, kp);
         const u32 nn = n > 0 ? n : 1;          // a table is built either way; unused when n == 0
         const u64 Td = (u64)b * nn;
         const u64 ctx = (u64)b * ((u64)nn * lin + ((u64)nn * (nn + 1)) / 2);
         build_fixed_tasks(m, tt, Td, Td, nn, kd);
         build_attn_tasks(m, tt, Td, ctx, ctx, kd);
-    }
-    // index of this thread's config for pair (h, f): ((((m n_h + h) n_f + f) n_b + b) n_t n_l) + tl
+        built = true;
+    };
+    // index of this thread's config for pair (h, f): ((((m n_h + h) n_f + f) n_b + b) n_t n_l) + tl.
+    // j is its offset in the caller's range, kept as a running value; as an unsigned number it is
+    // below r.count exactly when the index lies inside [first, first + count).
     const u64 stride_hf = (u64)s.n_b * n_tl;
-    const u64 base = ((u64)mpos * n_hf) * stride_hf + (u64)bpos * n_tl + tl;
+    u64 j = ((u64)mpos * n_hf + hf0) * stride_hf + (u64)bpos * n_tl + tl - r.first;
 
     ReqBytes rq;
     rq.block = 0; rq.bytes = 1; rq.inv = 1.0; rq.small = false;
     const u64 S = (u64)lin + lout;
     const double nd = (double)n;
     const double tok = cvt((u64)b * n);
+    const u32 heads_bad = ((m.nh & (t - 1)) != 0 || (m.nkv & (t - 1)) != 0) ? 4u : 0u;   // t is a power of two
+    const u32 hf_end = min(hf_chunk, n_hf > hf0 ? n_hf - hf0 : 0u);
 
-    for (u32 i = 0; i < hf_chunk; i++) {
+#pragma unroll 2
+    for (u32 i = 0; i < hf_chunk; i++, j += stride_hf) {
         const u32 hf = hf0 + i;
-        const u64 idx = base + (u64)hf * stride_hf;
-        const bool valid = active && hf < n_hf && idx >= r.first && idx - r.first < r.count;
+        const bool valid = active && i < hf_end && j < r.count;
         Metrics out;
+        out.status = 0xFF;
         if (valid) {
-            const DRate &rt = s.rates[hf];
-            const u32 block = rt.kv_block;
+            // memory check (Sec. 3.2 Step 1, Sec. 3.3.1): one 16-byte load per pair
+            const ulonglong2 hm = __ldg(s.hfmem + hf);
+            const u32 block = (u32)hm.y;
             if (block != rq.block) req_bytes_for(rq, block, S, mi.kv_tok);
-            out.status = feasibility_cached(m, rt.usable, mi, t, b, rq, out.bmax);
-            if (out.status) set_infeasible(out);
+            u64 bmax = 0;
+            u32 st = heads_bad;
+            if (hm.x > mi.w_gpu) {
+                const u64 avail = hm.x - mi.w_gpu;
+                bmax = (rq.small && (avail >> 52) == 0) ? floor_div_recip(avail, rq.bytes, rq.inv) : avail / rq.bytes;
+            } else st |= 1;
+            if ((u64)b > bmax) st |= 2;
+            out.status = st;
+            out.bmax = clamp_u32(bmax);
+            if (st) set_infeasible(out);
             else {
+                if (!built) build_tables();
+                const DRate &rt = s.rates[hf];
                 const double inf = __longlong_as_double(0x7FF0000000000000LL);
                 const double t_pre = eval_phase<TIME_SUM>(kp, rt, Nd, lf);
                 const double t_dec = n > 0 ? eval_phase<TIME_SUM>(kd, rt, Nd, lf) : 0.0;
                 const u32 ci = hf * s.n_t + tpos;
                 out.ttft = t_pre;
                 out.latency = t_pre + t_dec;
-                out.cost_hr = s.cost_hr[ci];
+                out.cost_hr = __ldg(s.cost_hr + ci);
                 if (n > 0) {
                     out.tpot = t_dec / nd;
                     out.thr = tok / t_dec;
-                    out.cost_tok = s.cost_sec[ci] / out.thr;
+                    out.cost_tok = __ldg(s.cost_sec + ci) / out.thr;
                 } else {
                     out.tpot = 0.0; out.thr = 0.0; out.cost_tok = inf;
                 }
                 out.n_iters = 1 + (u64)n;
                 out.n_req_iters = (u64)b * (1 + (u64)n);
             }
-        } else {
-            out.status = 0xFF;
         }
-        emit(valid, idx, out);
+        emit(valid, j, out);
     }
 }
 
