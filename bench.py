@@ -107,6 +107,9 @@ def oracle_step(oracle, w):
     return out
 
 
+REF_STRIDE = 8      # the reference arm evaluates every 8th config of the workload per step
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -115,20 +118,27 @@ def run_reference(args):
     from paper_2412_04788_b200 import inputs
     w = inputs.workload(5)
     n = inputs.space_size(w["space"])
+    count = (n + REF_STRIDE - 1) // REF_STRIDE
+
+    def step():
+        out = oracle.simulate(w["space"], first=0, count=count, stride=REF_STRIDE)
+        oracle.select_topk(out, w["constraints"], w["topk"]["key"], w["topk"]["k"])
+        oracle.pareto(out, w["constraints"], "latency", "cost_per_hr")
+
     for _ in range(args.warmup):
-        oracle_step(oracle, w)
+        step()
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle_step(oracle, w)
+        step()
     dt = time.perf_counter() - t0
-    value = n * args.steps / dt
+    value = count * args.steps / dt
     cores = oracle.threads()
+    sample = f"every {REF_STRIDE}th config of the 16777216-config sweep per step ({count} configs): simulate + top-64 + Pareto"
     line = {"impl": "reference", "metric": "configs/sec", "value": value, "unit": "configs/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "C5 closed-form sweep, 16777216 configs: simulate + top-64 + Pareto"},
-            "cpu_baseline": {"value": value, "unit": "configs/s", "cores": cores, "kind": "oracle",
-                             "sample": f"the whole workload, {args.steps} passes"},
+            "config": {"workload": "C5 closed-form sweep, 16777216 configs: simulate + top-64 + Pareto", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": "configs/s", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": "configs/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
