@@ -225,3 +225,20 @@ def test_iteration_cap_sets_status(golden):
     assert out["status"][0] == oracle.ST_ITER and np.isinf(out["latency"][0])
     out = oracle.simulate(sp, tr, max_iters=6)
     assert out["status"][0] == 0
+
+
+def test_percentile_ranks(golden):
+    """p50 / p99 are order statistics at the nearest rank; request counts where a floor-based rank
+    would pick a different element."""
+    hw, mem = I.seeded_hw(21, 1, mem_gb=[1])
+    fw_f, fw_i = I.seeded_fw(21, 1)
+    small = [4, 256, 8, 4, 512, 1000, 1, 2, 2, 2]
+    for case in golden["percentile_ranks"]["cases"]:
+        n = case["n"]
+        tr = I.make_trace(300 + n, n, 2.0e5, lengths=True, in_clip=48, out_clip=6)     # arrivals faster than service: queueing
+        sp = I._space(np.array([small]), hw, mem, fw_f, fw_i, [2], [1], [(1, 1)])
+        out = oracle.simulate(sp, tr, per_request=True)
+        srt = np.sort(out["req_ttft"][0])
+        assert len(np.unique(srt)) > n // 2          # distinct enough for the rank to matter
+        assert out["ttft_p50"][0] == srt[case["p50"]], n
+        assert out["ttft_p99"][0] == srt[case["p99"]], n
