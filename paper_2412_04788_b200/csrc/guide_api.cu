@@ -81,6 +81,11 @@ static int check_closed_form_overflow(const guide_space &s) {
 static int check_trace_overflow(const guide_space &s, const guide_trace &t) {
     const u128 q = std::max<uint64_t>(t.max_tokens, t.n_zero ? (uint64_t)s.max_lin + s.max_lout : 0);
     const u128 b = s.max_batch;
+    uint32_t max_block = 1;
+    for (const guide_fw &f : s.fw) max_block = std::max(max_block, f.kv_block);
+    for (const guide_model &m : s.models)
+        if ((q + max_block) * (2ull * m.n_layers * m.n_kv_heads * (m.hidden / m.n_heads) * m.kv_bytes) >= LIMIT)
+            return fail(GUIDE_ERR_OVERFLOW, "KV bytes of the longest request overflow");
     for (size_t mi = 0; mi < s.models.size(); mi++) {
         Maxima pre{b * q, b, b * q * q, b * q, 1};
         Maxima dec{b, b, b * q, b * q, 1};
@@ -368,8 +373,10 @@ int guide_space_create(const guide_space_desc *d, guide_space **out) {
         s->size = (uint64_t)n;
     }
     if (!rc) {
-        // capacity arithmetic: (lin+lout rounded to blocks) x KV bytes per token
-        u128 worst = ((u128)s->max_lin + s->max_lout + 0xFFFFFFFFull);
+        // capacity arithmetic: (lin+lout rounded up to whole blocks) x KV bytes per token
+        uint32_t max_block = 1;
+        for (const guide_fw &f : s->fw) max_block = std::max(max_block, f.kv_block);
+        u128 worst = (u128)s->max_lin + s->max_lout + max_block;
         for (const guide_model &m : s->models)
             if (worst * (2ull * m.n_layers * m.n_kv_heads * (m.hidden / m.n_heads) * m.kv_bytes) >= LIMIT)
                 rc = fail(GUIDE_ERR_OVERFLOW, "KV bytes of one request overflow");

@@ -153,3 +153,14 @@ def test_workload5_full_size_fused_selection():
     fidx, fcnt = run_pareto(sp, None, cons, w["pareto"]["x"], w["pareto"]["y"])
     w_f, w_n = oracle.pareto(want, cons, w["pareto"]["x"], w["pareto"]["y"])
     assert fcnt == w_n and np.array_equal(fidx, w_f) and fcnt >= 2
+
+
+def test_empty_range_selects_nothing(c2_small):
+    """A range of zero configs (first = size of the space): count 0, unused slots marked."""
+    w, want, out_dev, sp = c2_small
+    n = sp.size
+    empty = {k: v[n:n] for k, v in out_dev.items()}
+    idx, val, cnt = run_topk(sp, None, {}, "latency", 4, first=n, count=0)
+    assert cnt == 0 and np.all(idx == U64_MAX) and np.all(np.isinf(val))
+    fidx, fcnt = run_pareto(sp, None, {}, "latency", "cost_per_hr", first=n, count=0)
+    assert fcnt == 0

@@ -134,3 +134,57 @@ def test_full_size_trace_workloads_sampled(k, stride):
     assert bool(torch.isfinite(out["latency"][ok]).all()) and bool(torch.isinf(out["latency"][~ok]).all())
     if k == 4:
         assert want["n_preempt"].sum() > 0          # the sampled configs include evictions
+
+
+def test_block_sizes_outside_the_histogram_path():
+    """KV blocks of 100 and 65 tokens (above the 64-entry phase histogram: needs are counted by a
+    slot scan and iterations are not bursted), next to 1, 3, 64: all against the oracle."""
+    n = 80
+    tr = {"arrival": I.poisson_arrivals(9, n, 2500.0), "in_len": I.randint(9, 81, n, 1, 300).astype(np.uint32),
+          "out_len": I.randint(9, 82, n, 1, 150).astype(np.uint32)}
+    hw, _ = I.seeded_hw(9, 3, mem_gb=[1] * 3)
+    w_bytes, kv_tok = oracle.weight_bytes_per_gpu(SMALL, 1), oracle.kv_bytes_per_token(SMALL, 1)
+    mem = np.array([w_bytes + tok * kv_tok for tok in (1000, 3000, 200000)], dtype=np.uint64)
+    fw_f, fw_i = I.seeded_fw(9, 5, reserve_permille=0)
+    fw_i[:, 1] = [100, 65, 1, 3, 64]
+    sp = I._space(np.array([SMALL]), hw, mem, fw_f, fw_i, [1, 4, 33, 256], [1, 2], [(1, 1)])
+    want = oracle.simulate(sp, tr, per_request=True)
+    got, *_ = run_simulate(sp, tr, per_request=True)
+    fields = guide.F64_OUTPUTS + ("req_ttft", "req_tpot")
+    assert_parity(got, want, fields=fields)
+    assert sum(bit_mismatches(got, want, fields).values()) == 0
+    assert want["n_preempt"].sum() > 0 and (want["status"] == 0).sum() >= 40
+
+
+def test_counts_beyond_2_to_53_use_the_integer_path():
+    """64 KiB KV elements and 16k-token prompts: with a few hundred residents the per-iteration KV
+    read count exceeds 2^53, so it cannot be carried as an exact double; the kernel must fall back
+    to the integer form (the small-batch configs of the same space stay on the fast path) and
+    still agree with the oracle bit for bit."""
+    fat = [1, 2**15, 2**5, 2**5, 16, 64, 1, 2, 2, 2**16]
+    n = 300
+    tr = {"arrival": np.zeros(n), "in_len": (2**14 - np.arange(n)).astype(np.uint32),
+          "out_len": (2 + np.arange(n) % 3).astype(np.uint32)}
+    hw, _ = I.seeded_hw(4, 2, mem_gb=[1, 1])
+    mem = np.array([2**61, 2**62], dtype=np.uint64)
+    fw_f, fw_i = I.seeded_fw(4, 2)
+    fw_i[1, 0] = 0                      # one profile without FlashAttention: score-matrix terms too
+    sp = I._space(np.array([fat]), hw, mem, fw_f, fw_i, [2, 256], [1, 4], [(1, 1)])
+    assert 256 * (2**14 + 5) * 2**15 * 2**16 >= 2**53          # the premise, for max batch 256
+    want = oracle.simulate(sp, tr, per_request=True)
+    assert (want["status"] == 0).all()
+    got, *_ = run_simulate(sp, tr, per_request=True)
+    fields = guide.F64_OUTPUTS + ("req_ttft", "req_tpot")
+    assert_parity(got, want, fields=fields)
+    assert sum(bit_mismatches(got, want, fields).values()) == 0
+
+
+def test_single_request_and_single_config():
+    tr = {"arrival": np.array([0.25]), "in_len": np.array([17], np.uint32), "out_len": np.array([1], np.uint32)}
+    hw, mem = I.seeded_hw(2, 1, mem_gb=[8])
+    fw_f, fw_i = I.seeded_fw(2, 1)
+    sp = I._space(np.array([SMALL]), hw, mem, fw_f, fw_i, [1], [1], [(1, 1)])
+    want = oracle.simulate(sp, tr, per_request=True)
+    got, *_ = run_simulate(sp, tr, per_request=True)
+    assert_parity(got, want, fields=guide.F64_OUTPUTS + ("req_ttft", "req_tpot"))
+    assert got["n_iters"][0] == 1 and got["thr_decode"][0] == 0.0 and np.isinf(got["cost_per_token"][0])
