@@ -37,7 +37,7 @@ import numpy as np
 BYTES_SIM = 6 * 8 + 1 + 4          # six fp64 metrics + status + bmax written per config
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_closed_form_tiled launch on the full workload 5
 # (profiles/k_closed_form_tiled_c5.md); only meaningful for that size and that kernel version
-K1_TRAFFIC_C5 = 850_617_600 + 145_664
+K1_TRAFFIC_C5 = 857_484_032 + 393_472
 SIM_FIELDS = ("latency", "ttft", "tpot", "thr_decode", "cost_per_hr", "cost_per_token", "status", "bmax")
 TRACE_FIELDS = ("latency", "ttft", "ttft_p50", "ttft_p99", "tpot", "thr_decode", "cost_per_hr", "cost_per_token",
                 "status", "bmax", "n_iters", "n_req_iters")

@@ -157,7 +157,7 @@ int space_on_device(guide_space *s, DSpace *out) {
                  o_dr = take(n_h * n_f * sizeof(DRate)), o_b = take(s->batch.size() * 4),
                  o_t = take(s->tp.size() * 4), o_p = take(s->pairs.size() * 8),
                  o_ch = take(n_h * n_f * s->tp.size() * 8), o_cs = take(n_h * n_f * s->tp.size() * 8),
-                 o_lo = take(s->pairs.size() * 4), o_hm = take(n_h * n_f * 16);
+                 o_hm = take(n_h * n_f * 16);
     char *blob = nullptr;
     GUIDE_CUDA(cudaMalloc(&blob, off));
     cudaError_t e = cudaSuccess;
@@ -170,15 +170,6 @@ int space_on_device(guide_space *s, DSpace *out) {
     put(o_b, s->batch.data(), s->batch.size() * 4);
     put(o_t, s->tp.data(), s->tp.size() * 4);
     put(o_p, s->pairs.data(), s->pairs.size() * 8);
-    {
-        // walk order of the length pairs for the tiled kernels (an ordering only: no model arithmetic)
-        std::vector<uint32_t> order(s->pairs.size());
-        for (size_t i = 0; i < order.size(); i++) order[i] = (uint32_t)i;
-        std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) {
-            return (uint64_t)s->pairs[a].lin + s->pairs[a].lout < (uint64_t)s->pairs[b].lin + s->pairs[b].lout;
-        });
-        put(o_lo, order.data(), order.size() * 4);
-    }
     if (e == cudaSuccess) {
         const u32 n = (u32)std::max(n_m, n_h * n_f);
         k_build_tables<<<(n + 127) / 128, 128>>>((const guide_model *)(blob + o_gm), (u32)n_m,
@@ -202,7 +193,6 @@ int space_on_device(guide_space *s, DSpace *out) {
     d.view.pairs = (const uint2 *)(blob + o_p);
     d.view.cost_hr = (const double *)(blob + o_ch);
     d.view.cost_sec = (const double *)(blob + o_cs);
-    d.view.lorder = (const u32 *)(blob + o_lo);
     d.view.hfmem = (const ulonglong2 *)(blob + o_hm);
     d.view.n_m = (u32)n_m; d.view.n_h = (u32)n_h; d.view.n_f = (u32)n_f;
     d.view.n_b = (u32)s->batch.size(); d.view.n_t = (u32)s->tp.size(); d.view.n_l = (u32)s->pairs.size();

@@ -40,7 +40,6 @@ struct DSpace {
     const uint2 *pairs;          // (lin, lout)
     const double *cost_hr;       // [n_h * n_f][n_t]: price x TP degree
     const double *cost_sec;      // [n_h * n_f][n_t]: (price x TP degree) / 3600
-    const u32 *lorder;           // [n_l]: length-pair positions in ascending lin + lout (ties by position)
     const ulonglong2 *hfmem;     // [n_h * n_f]: x = usable bytes, y = KV block size (what the memory check reads)
     u32 n_m, n_h, n_f, n_b, n_t, n_l;
 };

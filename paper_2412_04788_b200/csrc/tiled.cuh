@@ -35,12 +35,8 @@ __device__ __forceinline__ void tiled_visit(const DSpace &s, const Range &r, int
     const u32 bpos = mb % s.n_b, mpos = mb / s.n_b;
     const u32 tl_raw = tile * blockDim.x + threadIdx.x;
     const bool active = tl_raw < n_tl;
-    // Threads walk the length pairs in order of lin + lout: whether a config fits in memory is
-    // monotone in that sum, so a warp's 32 configs are almost always all feasible or all not,
-    // instead of every warp paying for the evaluation of a few feasible lanes.
-    const u32 tl_t = active ? tl_raw : n_tl - 1;
-    const u32 tpos = tl_t / s.n_l, lpos = s.lorder[tl_t % s.n_l];
-    const u32 tl = tpos * s.n_l + lpos;
+    const u32 tl = active ? tl_raw : n_tl - 1;
+    const u32 tpos = tl / s.n_l, lpos = tl % s.n_l;
     const u32 hf0 = blockIdx.y * hf_chunk;
 
     const DModel m = s.models[mpos];
