@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libguide.so")
-SOURCES = ["guide_api.cu", "closed_form.cu", "select.cu", "trace_sim.cu"]
+SOURCES = ["guide_api.cu", "closed_form.cu", "select.cu", "select_stream.cu", "trace_sim.cu"]
 
 # -fmad=false: the model's arithmetic is defined without fused multiply-add (bit-exact with any
 # IEEE-754 binary64 implementation that evaluates the same expression order).

@@ -13,31 +13,13 @@
 // The metrics come either from materialised arrays or, fused, from the closed-form evaluation
 // itself, walked in the tiled order of tiled.cuh so the integer task tables are built once per
 // (model, batch, TP, length) point.
-#include "guide_internal.cuh"
+#include "select.cuh"
 
 namespace guide {
 
-static constexpr u32 SEL_THREADS = 256;
-static constexpr u32 SEL_MAX_BLOCKS = 1024;
 static constexpr u32 PARETO_CAP = 4096;          // shared-memory items per block
 static constexpr u32 TOPK_CAP = 4096;            // shared-memory candidates per block
 static constexpr u32 MAX_BUDGET = 16;            // most appends per thread between two checkpoints
-static constexpr u64 KEY_MAX = ~0ull;
-
-// order-preserving map double -> u64 (after -0.0 -> +0.0)
-__device__ __forceinline__ u64 enc(double v) {
-    const u64 b = (u64)__double_as_longlong(v + 0.0);
-    return (b >> 63) ? ~b : (b | 0x8000000000000000ull);
-}
-__device__ __forceinline__ double dec(u64 k) {
-    const u64 b = (k >> 63) ? (k ^ 0x8000000000000000ull) : ~k;
-    return __longlong_as_double((long long)b);
-}
-
-struct Cons {
-    double max_ttft, max_latency, max_cost_hr, min_thr;
-    int ttft_stat;
-};
 
 __device__ __forceinline__ double pick_metric(int key, double latency, double ttft, double ttft_p99, double tpot,
                                               double thr, double cost_hr, double cost_tok) {
@@ -199,38 +181,6 @@ __device__ __forceinline__ void fetch_round(const Src &src, const Range &r, u64 
     }
 }
 
-// ---- block-wide helpers ---------------------------------------------------------------------------
-
-struct KI { u64 key, idx; };
-__device__ __forceinline__ bool ki_less(const KI &a, const KI &b) {
-    return a.key < b.key || (a.key == b.key && a.idx < b.idx);
-}
-struct P3 { u64 x, y, idx; };
-__device__ __forceinline__ bool p3_less(const P3 &a, const P3 &b) {
-    if (a.x != b.x) return a.x < b.x;
-    if (a.y != b.y) return a.y < b.y;
-    return a.idx < b.idx;
-}
-
-__device__ __forceinline__ u32 next_pow2(u32 v) { return v <= 1 ? 1 : 1u << (32 - __clz(v - 1)); }
-
-// in-place ascending bitonic sort of buf[0..P), P a power of two; ends with a barrier
-template <class T, class Less>
-__device__ void block_bitonic_sort(T *buf, u32 P, Less less) {
-    for (u32 size = 2; size <= P; size <<= 1) {
-        for (u32 stride = size >> 1; stride > 0; stride >>= 1) {
-            for (u32 i = threadIdx.x; i < (P >> 1); i += blockDim.x) {
-                const u32 lo = ((i & ~(stride - 1)) << 1) | (i & (stride - 1));
-                const u32 hi = lo + stride;
-                const bool up = (lo & size) == 0;
-                const T a = buf[lo], b = buf[hi];
-                if (less(b, a) == up) { buf[lo] = b; buf[hi] = a; }
-            }
-            __syncthreads();
-        }
-    }
-}
-
 // ---- top-k accumulator -------------------------------------------------------------------------------
 
 struct TopKAcc {
@@ -293,7 +243,8 @@ struct TopKAcc {
 // No block barrier on the hot path.  Each warp owns a segment of shared memory with its own sorted
 // candidates and its own threshold; takers of a round are placed by ballot, and when the segment
 // fills (or about k entries have slipped under a stale threshold) the warp sorts it alone.  A warp
-// that holds k candidates publishes its k-th key to a grid-wide word (atomicMin); every warp drops
+// that holds k candidates publishes its k-th key to a grid-wide word (kept as the complement, so a
+// zeroed workspace header means "no bound"; atomicMax tightens it); every warp drops
 // anything above that word at once, so once a few warps have found good candidates the rest of
 // the grid hardly appends at all.  The word only bounds keys (strictly larger keys are dropped),
 // ties on the key are still decided by the index in the exact per-warp test.
@@ -308,7 +259,7 @@ __host__ __device__ inline u32 warp_seg_cap(u32 k) {
 
 struct WarpTopK {
     KI *seg;          // this warp's segment, cap entries
-    u64 *gptr;        // grid-wide upper bound on the k-th key
+    u64 *gptr;        // grid-wide upper bound on the k-th key, stored as its complement (0 = no bound yet)
     u64 gthr;         // cached copy
     u32 cap, k, fill, tick;
     bool has_thr;
@@ -317,7 +268,7 @@ struct WarpTopK {
     __device__ void init(KI *smem, u32 k_, u64 *gptr_) {
         k = k_; cap = warp_seg_cap(k_);
         seg = smem + (size_t)(threadIdx.x >> 5) * cap;
-        gptr = gptr_; gthr = __ldcg(gptr_);
+        gptr = gptr_; gthr = ~__ldcg(gptr_);
         fill = 0; tick = 0; has_thr = false; thr.key = KEY_MAX; thr.idx = KEY_MAX;
     }
     __device__ void compact() {
@@ -339,7 +290,7 @@ struct WarpTopK {
         }
         if (fill >= k) {
             fill = k; has_thr = true; thr = seg[k - 1];
-            if (lane == 0) atomicMin((unsigned long long *)gptr, (unsigned long long)thr.key);
+            if (lane == 0) atomicMax((unsigned long long *)gptr, (unsigned long long)~thr.key);
             if (thr.key < gthr) gthr = thr.key;
         }
         __syncwarp();
@@ -347,7 +298,7 @@ struct WarpTopK {
     // largest key that can still matter to this warp
     __device__ __forceinline__ u64 bound() const { return has_thr && thr.key < gthr ? thr.key : gthr; }
     __device__ __forceinline__ void refresh() {
-        if ((++tick & 15u) == 0) { const u64 g = __ldcg(gptr); if (g < gthr) gthr = g; }
+        if ((++tick & 15u) == 0) { const u64 g = ~__ldcg(gptr); if (g < gthr) gthr = g; }
     }
     // all 32 lanes of the warp call it together
     __device__ __forceinline__ void push(bool ok, const KI &it) {
@@ -673,9 +624,11 @@ __device__ __forceinline__ void topk_end(WarpTopK &acc, KI *smem, u32 block, u32
 }
 
 template <class Src, bool WARP>
-__global__ void __launch_bounds__(SEL_THREADS) k_topk_scan(Src src, Range r, u32 k, u32 *counts, KI *lists, u64 *gthr) {
+__global__ void __launch_bounds__(SEL_THREADS) k_topk_scan(Src src, Range r, u32 k, u32 *counts, KI *lists, u64 *gthr,
+                                                           const u32 *gate) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ u32 cnt;
+    if (gate && __ldcg(gate) == 0) return;
     typename TopKPick<WARP>::type acc;
     topk_begin(acc, (KI *)smem_raw, &cnt, k, gthr);
     constexpr int ITEMS = Src::ITEMS;
@@ -726,9 +679,11 @@ k_topk_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, Co
 // above the smallest k-th entry of any full list cannot be among the k smallest and are skipped.
 // Ranks below k are distinct, so every output slot has one writer.
 __global__ void __launch_bounds__(SEL_THREADS) k_topk_merge(u32 nblk, u32 k, const u32 *counts, const KI *lists,
-                                                            int negate_out, u64 *idx_out, double *key_out, u32 *count_out) {
+                                                            int negate_out, u64 *idx_out, double *key_out, u32 *count_out,
+                                                            const u32 *gate) {
     __shared__ KI s_best[SEL_THREADS / 32];
     __shared__ u32 s_tot[SEL_THREADS / 32];
+    if (gate && __ldcg(gate) == 0) return;
     KI best; best.key = KEY_MAX; best.idx = KEY_MAX;
     u32 tot = 0;
     for (u32 b = threadIdx.x; b < nblk; b += blockDim.x) {
@@ -958,27 +913,15 @@ k_pareto_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, 
 // top-k workspace: 256 B header | counts u32[max_blocks] | lists KI[max_blocks][k]
 static size_t topk_lists_offset(u32 max_blocks) { return 256 + ((size_t)max_blocks * 4 + 255) / 256 * 256; }
 
-size_t topk_workspace_bytes(u32 k) { return topk_lists_offset(SEL_MAX_BLOCKS) + (size_t)SEL_MAX_BLOCKS * k * sizeof(KI); }
-size_t pareto_workspace_bytes() {
-    return 256 + (size_t)SEL_MAX_BLOCKS * sizeof(u32) + (size_t)SEL_MAX_BLOCKS * GUIDE_PARETO_MAX * sizeof(P3);
+// ... followed by the streaming path's region (sample results and survivor list)
+static size_t topk_stream_offset(u32 k) {
+    return (topk_lists_offset(SEL_MAX_BLOCKS) + (size_t)SEL_MAX_BLOCKS * k * sizeof(KI) + 255) / 256 * 256;
 }
-
-// Are all arrays a scan over materialised metrics will touch aligned for 16-byte loads?
-static int mat_vec_ok(const guide_outputs &o, const guide_constraints &c, int m0, int m1) {
-    auto al = [](const void *p, uintptr_t a) { return ((uintptr_t)p % a) == 0; };
-    const double *arrs[] = {o.latency, o.ttft, o.ttft_p50, o.ttft_p99, o.tpot, o.thr_decode, o.cost_per_hr, o.cost_per_token};
-    (void)c; (void)m0; (void)m1;
-    for (const double *p : arrs)
-        if (p && !al(p, 16)) return 0;
-    return al(o.status, 4) ? 1 : 0;
+static size_t pareto_stream_offset() {
+    return (256 + (size_t)SEL_MAX_BLOCKS * sizeof(u32) + (size_t)SEL_MAX_BLOCKS * GUIDE_PARETO_MAX * sizeof(P3) + 255) / 256 * 256;
 }
-
-static Cons make_cons(const guide_constraints &c) {
-    Cons k;
-    k.max_ttft = c.max_ttft; k.max_latency = c.max_latency; k.max_cost_hr = c.max_cost_per_hr;
-    k.min_thr = c.min_throughput; k.ttft_stat = c.ttft_stat;
-    return k;
-}
+size_t topk_workspace_bytes(u32 k) { return topk_stream_offset(k) + topk_stream_bytes(); }
+size_t pareto_workspace_bytes() { return pareto_stream_offset() + pareto_stream_bytes(); }
 
 static u32 grid_for(u64 count, u32 items, u32 blocks_per_sm, u32 max_blocks) {
     // every block has fixed costs (first sorts, final sort, its list in the merge): give each at
@@ -1002,43 +945,43 @@ static int allow_smem(K kernel, size_t bytes) {
 }
 
 static int run_topk_merge(u32 nblk, u32 k, int negate, u32 *counts, KI *lists, u64 *idx_out, double *key_out,
-                          u32 *count_out, cudaStream_t st) {
+                          u32 *count_out, const u32 *gate, cudaStream_t st) {
     const u64 cand = (u64)nblk * k;                      // one warp per candidate, a few candidates per warp
     const u64 want = (cand + (SEL_THREADS / 32) * 4 - 1) / ((SEL_THREADS / 32) * 4);
     const u32 grid = (u32)std::min<u64>(std::max<u64>(want, 1), (u64)num_sms() * 8);
-    k_topk_merge<<<grid, SEL_THREADS, 0, st>>>(nblk, k, counts, lists, negate,
-                                                                                       idx_out, key_out, count_out);
+    k_topk_merge<<<grid, SEL_THREADS, 0, st>>>(nblk, k, counts, lists, negate, idx_out, key_out, count_out, gate);
     GUIDE_CUDA(cudaGetLastError());
     return GUIDE_OK;
 }
 
-// The first 256 bytes of a top-k workspace hold the grid-wide key bound of the per-warp mode; it
-// has to start at all-ones.
-static int topk_reset_bound(unsigned char *ws, cudaStream_t st) {
-    GUIDE_CUDA(cudaMemsetAsync(ws, 0xFF, 256, st));
+// The first 256 bytes of a top-k workspace are its header (select.cuh); every word starts at zero.
+static int topk_reset_header(unsigned char *ws, cudaStream_t st) {
+    GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
     return GUIDE_OK;
 }
 
 template <class Src, bool WARP>
 static int run_topk_scan_mode(const Src &src, Range r, u32 k, int negate, u32 max_blocks, unsigned char *ws, u64 *idx_out,
-                              double *key_out, u32 *count_out, cudaStream_t st) {
+                              double *key_out, u32 *count_out, const u32 *gate, cudaStream_t st) {
     u32 *counts = (u32 *)(ws + 256);
     KI *lists = (KI *)(ws + topk_lists_offset(max_blocks));
     const size_t smem = WARP ? (size_t)(SEL_THREADS / 32) * warp_seg_cap(k) * sizeof(KI) : (size_t)TOPK_CAP * sizeof(KI);
     int rc = allow_smem(k_topk_scan<Src, WARP>, smem);
     if (rc) return rc;
-    if ((rc = topk_reset_bound(ws, st))) return rc;
+    // a gated launch runs behind the streaming path, which has reset the header for the whole call
+    if (!gate && (rc = topk_reset_header(ws, st))) return rc;
     const u32 grid = grid_for(r.count, Src::ITEMS, WARP ? 4 : 3, max_blocks);
-    k_topk_scan<Src, WARP><<<grid, SEL_THREADS, smem, st>>>(src, r, k, counts, lists, (u64 *)ws);
+    k_topk_scan<Src, WARP><<<grid, SEL_THREADS, smem, st>>>(src, r, k, counts, lists, (u64 *)ws, gate);
     GUIDE_CUDA(cudaGetLastError());
-    return run_topk_merge(grid, k, negate, counts, lists, idx_out, key_out, count_out, st);
+    return run_topk_merge(grid, k, negate, counts, lists, idx_out, key_out, count_out, gate, st);
 }
 
 template <class Src>
 static int run_topk_scan(const Src &src, Range r, u32 k, int negate, u32 max_blocks, unsigned char *ws, u64 *idx_out,
-                         double *key_out, u32 *count_out, cudaStream_t st) {
-    return k <= TOPK_WARP_K ? run_topk_scan_mode<Src, true>(src, r, k, negate, max_blocks, ws, idx_out, key_out, count_out, st)
-                            : run_topk_scan_mode<Src, false>(src, r, k, negate, max_blocks, ws, idx_out, key_out, count_out, st);
+                         double *key_out, u32 *count_out, cudaStream_t st, const u32 *gate = nullptr) {
+    return k <= TOPK_WARP_K
+               ? run_topk_scan_mode<Src, true>(src, r, k, negate, max_blocks, ws, idx_out, key_out, count_out, gate, st)
+               : run_topk_scan_mode<Src, false>(src, r, k, negate, max_blocks, ws, idx_out, key_out, count_out, gate, st);
 }
 
 template <int TIME_SUM, bool WARP>
@@ -1049,12 +992,12 @@ static int run_topk_tiled_mode(const DSpace &s, Range r, const TileGeom &g, int 
     const size_t smem = WARP ? (size_t)(SEL_THREADS / 32) * warp_seg_cap(k) * sizeof(KI) : (size_t)TOPK_CAP * sizeof(KI);
     int rc = allow_smem(k_topk_tiled<TIME_SUM, WARP>, smem);
     if (rc) return rc;
-    if ((rc = topk_reset_bound(ws, st))) return rc;
+    if ((rc = topk_reset_header(ws, st))) return rc;
     const dim3 grid(g.gx, g.splits);
     k_topk_tiled<TIME_SUM, WARP><<<grid, g.threads, smem, st>>>(s, r, tp_model, g.hf_chunk, g.tiles_per_mb, c, key, k,
                                                                counts, lists, (u64 *)ws);
     GUIDE_CUDA(cudaGetLastError());
-    return run_topk_merge(g.gx * g.splits, k, key == GUIDE_THROUGHPUT, counts, lists, idx_out, key_out, count_out, st);
+    return run_topk_merge(g.gx * g.splits, k, key == GUIDE_THROUGHPUT, counts, lists, idx_out, key_out, count_out, nullptr, st);
 }
 
 template <int TIME_SUM>
@@ -1071,7 +1014,17 @@ int launch_topk(const DSpace &s, Range r, const guide_outputs *mat, int time_mod
     const int negate = key == GUIDE_THROUGHPUT;
     unsigned char *w = (unsigned char *)ws;
     if (mat) {
-        MatSource src{*mat, make_cons(c), key, -1, mat_vec_ok(*mat, c, key, -1)};
+        MatSource src{*mat, make_cons(c), key, -1, mat_vec_ok(*mat)};
+        if (k <= STREAM_TOPK_MAX_K && stream_eligible(*mat, r)) {
+            // streaming path first; the accumulator kernels are queued behind it and return at once
+            // unless it raised the redo flag
+            int rc = topk_reset_header(w, st);
+            if (rc) return rc;
+            u32 *header = (u32 *)w;
+            if ((rc = launch_topk_stream(r, *mat, c, key, k, header, w + topk_stream_offset(k), idx_out, key_out, count_out, st)))
+                return rc;
+            return run_topk_scan(src, r, k, negate, SEL_MAX_BLOCKS, w, idx_out, key_out, count_out, st, header + TK_REDO);
+        }
         return run_topk_scan(src, r, k, negate, SEL_MAX_BLOCKS, w, idx_out, key_out, count_out, st);
     }
     TileGeom g;
@@ -1109,6 +1062,22 @@ static int run_pareto_scan(const Src &src, Range r, u64 *idx_out, u32 cap, u32 *
     return GUIDE_OK;
 }
 
+// The general kernel alone, gated on the redo flag a preceding kernel of the same call may have raised.
+template <class Src>
+static int run_pareto_general(const Src &src, Range r, u64 *idx_out, u32 cap, u32 *count_out, void *ws, cudaStream_t st) {
+    const size_t smem_gen = (size_t)PARETO_CAP * sizeof(P3);
+    int rc = allow_smem(k_pareto_scan<Src, false>, smem_gen);
+    if (rc) return rc;
+    u32 *header = (u32 *)ws;
+    u32 *sizes = (u32 *)((char *)ws + 256);
+    P3 *partial = (P3 *)((char *)ws + 256 + (size_t)SEL_MAX_BLOCKS * sizeof(u32));
+    const u32 grid_gen = grid_for(r.count, Src::ITEMS, 2, SEL_MAX_BLOCKS);
+    k_pareto_scan<Src, false><<<grid_gen, SEL_THREADS, smem_gen, st>>>(src, r, header, header + 1, sizes, partial, idx_out, cap,
+                                                                        count_out);
+    GUIDE_CUDA(cudaGetLastError());
+    return GUIDE_OK;
+}
+
 template <int TIME_SUM>
 static int run_pareto_tiled(const DSpace &s, Range r, const TileGeom &g, int tp_model, const Cons &c, int xm, int ym,
                             u64 *idx_out, u32 cap, u32 *count_out, void *ws, cudaStream_t st) {
@@ -1135,7 +1104,16 @@ int launch_pareto(const DSpace &s, Range r, const guide_outputs *mat, int time_m
                   const guide_constraints &c, int xm, int ym, u64 *idx_out, u32 cap, u32 *count_out, void *ws,
                   cudaStream_t st) {
     if (mat) {
-        MatSource src{*mat, make_cons(c), xm, ym, mat_vec_ok(*mat, c, xm, ym)};
+        MatSource src{*mat, make_cons(c), xm, ym, mat_vec_ok(*mat)};
+        if (stream_eligible(*mat, r)) {
+            // streaming path, then the general kernel gated on the redo flag (header word 1)
+            GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
+            u32 *header = (u32 *)ws;
+            int rc = launch_pareto_stream(r, *mat, c, xm, ym, header, (unsigned char *)ws + pareto_stream_offset(), idx_out, cap,
+                                          count_out, st);
+            if (rc) return rc;
+            return run_pareto_general(src, r, idx_out, cap, count_out, ws, st);
+        }
         return run_pareto_scan(src, r, idx_out, cap, count_out, ws, st);
     }
     TileGeom g;
@@ -1186,7 +1164,7 @@ int launch_topk_noalloc(Range r, const guide_outputs &mat, const guide_constrain
     const int rc = noalloc_scratch_address(&scratch);
     if (rc) return rc;
     static_assert(256 + NOALLOC_BLOCKS * 4 == 1280, "list offset below assumes a 256-byte multiple");
-    MatSource src{mat, make_cons(c), key, -1, mat_vec_ok(mat, c, key, -1)};
+    MatSource src{mat, make_cons(c), key, -1, mat_vec_ok(mat)};
     // The array still holds the previous call's bound, counts and lists.  The bound word is reset
     // on this stream before the scan; counts and lists need no clearing: every block of this
     // launch writes its own before the merge kernel, which follows on the same stream and reads
