@@ -628,6 +628,8 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_scan(Src src, Range r, u32
                                                            const u32 *gate) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ u32 cnt;
+    grid_dep_launch();
+    grid_dep_wait();                            // a gated launch may have started before its predecessor finished
     if (gate && __ldcg(gate) == 0) return;
     typename TopKPick<WARP>::type acc;
     topk_begin(acc, (KI *)smem_raw, &cnt, k, gthr);
@@ -683,6 +685,7 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_merge(u32 nblk, u32 k, con
                                                             const u32 *gate) {
     __shared__ KI s_best[SEL_THREADS / 32];
     __shared__ u32 s_tot[SEL_THREADS / 32];
+    grid_dep_wait();
     if (gate && __ldcg(gate) == 0) return;
     KI best; best.key = KEY_MAX; best.idx = KEY_MAX;
     u32 tot = 0;
@@ -861,6 +864,7 @@ __global__ void __launch_bounds__(SEL_THREADS) k_pareto_scan(Src src, Range r, u
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ u32 cnt;
     __shared__ __align__(8) u32 scratch[64];
+    grid_dep_wait();                            // a gated launch may have started before its predecessor finished
     if (gate && __ldcg(gate) == 0) return;
     ParetoAcc acc;
     WarpPareto wacc;
@@ -949,8 +953,13 @@ static int run_topk_merge(u32 nblk, u32 k, int negate, u32 *counts, KI *lists, u
     const u64 cand = (u64)nblk * k;                      // one warp per candidate, a few candidates per warp
     const u64 want = (cand + (SEL_THREADS / 32) * 4 - 1) / ((SEL_THREADS / 32) * 4);
     const u32 grid = (u32)std::min<u64>(std::max<u64>(want, 1), (u64)num_sms() * 8);
-    k_topk_merge<<<grid, SEL_THREADS, 0, st>>>(nblk, k, counts, lists, negate, idx_out, key_out, count_out, gate);
-    GUIDE_CUDA(cudaGetLastError());
+    if (gate) {
+        GUIDE_CUDA(launch_dependent(k_topk_merge, grid, SEL_THREADS, 0, st, nblk, k, (const u32 *)counts, (const KI *)lists, negate,
+                                    idx_out, key_out, count_out, gate));
+    } else {
+        k_topk_merge<<<grid, SEL_THREADS, 0, st>>>(nblk, k, counts, lists, negate, idx_out, key_out, count_out, gate);
+        GUIDE_CUDA(cudaGetLastError());
+    }
     return GUIDE_OK;
 }
 
@@ -971,8 +980,12 @@ static int run_topk_scan_mode(const Src &src, Range r, u32 k, int negate, u32 ma
     // a gated launch runs behind the streaming path, which has reset the header for the whole call
     if (!gate && (rc = topk_reset_header(ws, st))) return rc;
     const u32 grid = grid_for(r.count, Src::ITEMS, WARP ? 4 : 3, max_blocks);
-    k_topk_scan<Src, WARP><<<grid, SEL_THREADS, smem, st>>>(src, r, k, counts, lists, (u64 *)ws, gate);
-    GUIDE_CUDA(cudaGetLastError());
+    if (gate) {
+        GUIDE_CUDA(launch_dependent(k_topk_scan<Src, WARP>, grid, SEL_THREADS, smem, st, src, r, k, counts, lists, (u64 *)ws, gate));
+    } else {
+        k_topk_scan<Src, WARP><<<grid, SEL_THREADS, smem, st>>>(src, r, k, counts, lists, (u64 *)ws, gate);
+        GUIDE_CUDA(cudaGetLastError());
+    }
     return run_topk_merge(grid, k, negate, counts, lists, idx_out, key_out, count_out, gate, st);
 }
 
@@ -1072,9 +1085,8 @@ static int run_pareto_general(const Src &src, Range r, u64 *idx_out, u32 cap, u3
     u32 *sizes = (u32 *)((char *)ws + 256);
     P3 *partial = (P3 *)((char *)ws + 256 + (size_t)SEL_MAX_BLOCKS * sizeof(u32));
     const u32 grid_gen = grid_for(r.count, Src::ITEMS, 2, SEL_MAX_BLOCKS);
-    k_pareto_scan<Src, false><<<grid_gen, SEL_THREADS, smem_gen, st>>>(src, r, header, header + 1, sizes, partial, idx_out, cap,
-                                                                        count_out);
-    GUIDE_CUDA(cudaGetLastError());
+    GUIDE_CUDA(launch_dependent(k_pareto_scan<Src, false>, grid_gen, SEL_THREADS, smem_gen, st, src, r, header,
+                                (const u32 *)(header + 1), sizes, partial, idx_out, cap, count_out));
     return GUIDE_OK;
 }
 

@@ -82,6 +82,28 @@ __device__ void block_bitonic_sort(T *buf, u32 P, Less less) {
     }
 }
 
+// ---- programmatic dependent launch ---------------------------------------------------------------
+// The kernels of one selection call form a chain of short launches.  A kernel launched with
+// launch_dependent() may start (and sit in grid_dep_wait()) while its predecessor in the stream is
+// still running, which hides its launch latency; it must call grid_dep_wait() before touching
+// anything the predecessor writes.  grid_dep_wait() returns only when the predecessor grid has
+// completed and its writes are visible, and is a no-op in a kernel launched the ordinary way.
+// grid_dep_launch() in the predecessor lets the dependent start early; without it the dependent
+// starts when the predecessor's blocks have exited.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <class... KArgs, class... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- workspace headers (first 256 bytes of a selection workspace, zeroed at the start of a call) ----
 // top-k:  u64 at word 0: complement of the grid-wide key bound of the per-warp accumulators (0 = none);
 //         words 2..: the streaming path's tickets, candidate and sample counts, redo flag and (two u64 at word 6) its bound pair.

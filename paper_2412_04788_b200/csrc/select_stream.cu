@@ -202,6 +202,7 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_sample(Src<NA> s, Sample s
     __shared__ ulonglong2 sl[TK_SAMPLE_BLOCKS];
     __shared__ u32 last;
     static_assert(TK_SAMPLE_BLOCKS == SEL_THREADS, "one block minimum per thread in the last block");
+    grid_dep_launch();
     const u32 lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = SEL_THREADS / 32;
     u64 bk = KEY_MAX, bi = KEY_MAX;
     const u64 stride = (u64)gridDim.x * n_warps;
@@ -251,6 +252,8 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_refine(Src<NA> s, Sample s
     constexpr u32 PER = TK_SKEYS_CAP / SEL_THREADS;
     __shared__ ulonglong2 sl[TK_SKEYS_CAP];
     __shared__ u32 last;
+    grid_dep_launch();
+    grid_dep_wait();
     const u64 *bp = reinterpret_cast<const u64 *>(header + TK_BOUND);
     const u64 bkey = __ldcg(bp), bidx = __ldcg(bp + 1);
     const u32 lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = SEL_THREADS / 32;
@@ -307,6 +310,8 @@ __device__ __forceinline__ void topk_keep(u64 key, u64 idx, u32 *header, KI *can
 // Filter pass: passing configs within the bound go to the candidate list.
 template <int NA>
 __global__ void __launch_bounds__(SEL_THREADS, 4) k_topk_filter(Src<NA> s, Range r, u32 *header, KI *cand) {
+    grid_dep_launch();
+    grid_dep_wait();
     const u64 *bp = reinterpret_cast<const u64 *>(header + TK_BOUND);
     const u64 bkey = __ldcg(bp), bidx = __ldcg(bp + 1);
     const u64 tiles = r.count / TILE;
@@ -346,6 +351,8 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_rank(u32 *header, const KI
                                                            double *key_out, u32 *count_out) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     ulonglong2 *sl = reinterpret_cast<ulonglong2 *>(smem_raw);
+    grid_dep_launch();
+    grid_dep_wait();
     const u32 n = __ldcg(header + TK_COUNT);
     if (n > TK_CAND_CAP) {                                   // the list overflowed: hand the call to the fallback
         if (blockIdx.x == 0 && threadIdx.x == 0) header[TK_REDO] = 1;
@@ -422,6 +429,7 @@ __global__ void __launch_bounds__(SEL_THREADS) k_pareto_sample(Src<NA> s, Sample
     static_assert(PA_ROWS_PER_WARP % SAMPLE_BATCH == 0, "whole batches");
     const u32 lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = SEL_THREADS / 32;
     if (threadIdx.x == 0) { n_list = 0; n_front = 0; }
+    grid_dep_launch();
     u64 px[N_PTS], py[N_PTS];
     const u64 stride = (u64)gridDim.x * n_warps;
 #pragma unroll
@@ -578,6 +586,8 @@ __device__ __forceinline__ void pareto_keep(u64 x, u64 y, u64 idx, u32 *header, 
 template <int NA>
 __global__ void __launch_bounds__(SEL_THREADS, 4) k_pareto_filter(Src<NA> s, Range r, u32 *header, const P2 *killers, P3 *surv) {
     __shared__ P2 ks[PA_KILLERS];
+    grid_dep_launch();
+    grid_dep_wait();
     KillerSet K;
     K.k = ks;
     K.n = min(__ldcg(header + PH_KILLERS), PA_KILLERS);
@@ -626,6 +636,8 @@ __global__ void __launch_bounds__(SEL_THREADS) k_pareto_rank(u32 *header, const 
                                                              u32 *count_out) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ u32 last;
+    grid_dep_launch();
+    grid_dep_wait();
     const u32 n = __ldcg(header + PH_COUNT);
     if (n > PA_SURV_CAP) {                                   // the list overflowed: the general kernel redoes the call
         if (blockIdx.x == 0 && threadIdx.x == 0) header[1] = 1;
@@ -728,14 +740,12 @@ static int topk_stream_na(const Arr *arr, Range r, const guide_outputs &mat, u32
     sm.n_slots = sm.n_groups;
     k_topk_sample<NA><<<TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st>>>(s, sm, r.first, k, header, minima);
     GUIDE_CUDA(cudaGetLastError());
-    k_topk_refine<NA><<<TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st>>>(s, sm, r.first, k, header, spairs);
-    GUIDE_CUDA(cudaGetLastError());
-    k_topk_filter<NA><<<filter_grid(r.count), SEL_THREADS, 0, st>>>(s, r, header, cand);
-    GUIDE_CUDA(cudaGetLastError());
+    GUIDE_CUDA(launch_dependent(k_topk_refine<NA>, TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st, s, sm, r.first, k, header, spairs));
+    GUIDE_CUDA(launch_dependent(k_topk_filter<NA>, filter_grid(r.count), SEL_THREADS, 0, st, s, r, header, cand));
     const size_t smem = (size_t)TK_CAND_CAP * sizeof(KI);
     GUIDE_CUDA(cudaFuncSetAttribute(k_topk_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_topk_rank<<<num_sms(), SEL_THREADS, smem, st>>>(header, cand, k, negate, idx_out, key_out, count_out);
-    GUIDE_CUDA(cudaGetLastError());
+    GUIDE_CUDA(launch_dependent(k_topk_rank, num_sms(), SEL_THREADS, smem, st, header, (const KI *)cand, k, negate, idx_out,
+                                key_out, count_out));
     return GUIDE_OK;
 }
 
@@ -768,12 +778,12 @@ static int pareto_stream_na(const Arr *arr, Range r, const guide_outputs &mat, u
     const Sample sm = make_sample(r.count / ROW, PA_SAMPLE_ROWS, 1u << 20);
     k_pareto_sample<NA><<<PA_SAMPLE_BLOCKS, SEL_THREADS, 0, st>>>(s, sm, header, local, local_n, killers);
     GUIDE_CUDA(cudaGetLastError());
-    k_pareto_filter<NA><<<filter_grid(r.count), SEL_THREADS, 0, st>>>(s, r, header, killers, surv);
-    GUIDE_CUDA(cudaGetLastError());
+    GUIDE_CUDA(launch_dependent(k_pareto_filter<NA>, filter_grid(r.count), SEL_THREADS, 0, st, s, r, header, (const P2 *)killers,
+                                surv));
     const size_t smem = (size_t)PA_SURV_CAP * sizeof(P3);
     GUIDE_CUDA(cudaFuncSetAttribute(k_pareto_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_pareto_rank<<<num_sms(), SEL_THREADS, smem, st>>>(header, surv, front, idx_out, cap, count_out);
-    GUIDE_CUDA(cudaGetLastError());
+    GUIDE_CUDA(launch_dependent(k_pareto_rank, num_sms(), SEL_THREADS, smem, st, header, (const P3 *)surv, front, idx_out, cap,
+                                count_out));
     return GUIDE_OK;
 }
 
