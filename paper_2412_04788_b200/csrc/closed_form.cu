@@ -1,5 +1,7 @@
 // Closed-form evaluation kernels: one prefill stage + one aggregated decode stage per config
 // (Sec. 3.2 Steps 1-2, roofline of Sec. 3.4.2, time decomposition of Sec. 3.5.1).
+#include <algorithm>
+
 #include "guide_internal.cuh"
 
 namespace guide {
@@ -39,11 +41,284 @@ __global__ void __launch_bounds__(256, 2) k_closed_form_tiled(DSpace s, Range r,
     });
 }
 
+// ---- split evaluation ----------------------------------------------------------------------------
+//
+// Most configs of a large sweep do not fit their memory (Sec. 3.2 Step 1) and need no performance
+// model at all: a status byte, B_max and constant metrics.  Whole-space calls are therefore served
+// by two kernels.  The unit they share out is the foursome: four consecutive length positions, 32
+// bytes of every metric array, one memory sector.  A sector is always written whole by one warp
+// instruction of one kernel; partly written sectors cost a read-modify-write in memory and were
+// measured to halve the write bandwidth.
+//
+//   memory kernel : every config's status and B_max, and the constant metrics of the foursomes in
+//     which no config fits.  A thread takes two neighbouring positions of one (model, pair) and
+//     walks the batch axis: B_max does not depend on the batch size, so its exact division is done
+//     once per position; a warp's stores are 512 contiguous bytes.  Needs few registers and few
+//     warps; bound by the write bandwidth.  A small persistent grid, so that the model kernel finds
+//     room beside it.
+//   model kernel  : the roofline model (Sec. 3.2 Step 2, Sec. 3.4.2, Sec. 3.5.1) for the configs
+//     that fit, and the metrics of every foursome in which at least one does (constants for the
+//     others).  A thread owns one (model, batch, TP, length) point, as in the tiled walk, and
+//     visits the pairs in the order of hf_sorted: per KV block size, falling usable memory, so the
+//     pairs the point fits are a prefix and the walk stops at the first pair no lane of the warp
+//     fits.  Whether a config fits is one comparison here:
+//     b <= floor(avail / bytes) <=> b x bytes <= avail.  Foursomes are dealt to lanes in
+//     plane_order, so the lanes of a warp stop at about the same place.  Small blocks (two warps)
+//     let the scheduler refill the slots of warps that had nothing to do.
+//
+// The model kernel is launched as a programmatic dependent of the memory kernel and waits for it
+// only at its very end: the two run side by side, one bound by bandwidth and one by arithmetic,
+// and write disjoint sectors.
+
+static constexpr u32 MEM_THREADS = 128;         // x 2 positions = 256 positions of the plane per work item
+static constexpr u32 MEM_BLOCKS_PER_SM = 2;
+static constexpr u32 MODEL_THREADS = 64;
+static constexpr int SPLIT_MAX_CONST = 10;
+
+// 8-byte arrays that receive a constant for a config that does not fit (+inf, or 0 for throughput and counters)
+struct ConstOut {
+    unsigned long long *p[SPLIT_MAX_CONST];
+    unsigned long long pat[SPLIT_MAX_CONST];
+    int n;
+};
+
+// programmatic dependent launch: a kernel launched with the attribute may start while its
+// predecessor runs; cf_dep_wait() returns when the predecessor has completed and flushed
+__device__ __forceinline__ void cf_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void cf_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Memory check of Sec. 3.2 Step 1 / Sec. 3.3.1 for every config.  Work items: (model, tile of 256
+// plane positions, pair), taken in turn by a persistent grid.
+__global__ void __launch_bounds__(MEM_THREADS) k_closed_form_memory(DSpace s, guide_outputs o, ConstOut co, u32 tiles) {
+    __shared__ unsigned long long *s_p[SPLIT_MAX_CONST];
+    __shared__ unsigned long long s_pat[SPLIT_MAX_CONST];
+    cf_dep_launch();
+    if (threadIdx.x < SPLIT_MAX_CONST) { s_p[threadIdx.x] = co.p[threadIdx.x]; s_pat[threadIdx.x] = co.pat[threadIdx.x]; }
+    __syncthreads();
+    const u32 n_tl = s.n_t * s.n_l, n_hf = s.n_h * s.n_f;
+    const u32 items = s.n_m * tiles * n_hf;
+    const int n_const = co.n;
+    for (u32 item = blockIdx.x; item < items; item += gridDim.x) {
+        const u32 hf = item % n_hf;
+        const u32 mt = item / n_hf;
+        const u32 tile = mt % tiles, mpos = mt / tiles;
+        const u32 tl_raw = tile * (2 * MEM_THREADS) + 2 * threadIdx.x;
+        const bool active = tl_raw < n_tl;                  // n_l is a multiple of 4: a foursome shares its TP degree
+        const u32 tl = active ? tl_raw : 0;                  // idle lanes still take part in the exchange below
+        const u32 tpos = tl / s.n_l, lpos = tl % s.n_l;
+        const DModel m = s.models[mpos];
+        const u32 t = s.tp[tpos];
+        const MemInfo mi = mem_info(m, t);
+        const u32 st_base = ((m.nh & (t - 1)) != 0 || (m.nkv & (t - 1)) != 0) ? 4u : 0u;
+        const ulonglong2 hm = __ldg(s.hfmem + hf);
+        u64 bmax[2] = {0, 0};
+        u32 st0 = st_base;
+        if (hm.x > mi.w_gpu) {
+            const u64 avail = hm.x - mi.w_gpu;
+#pragma unroll
+            for (int u = 0; u < 2; u++) {
+                const uint2 pr = s.pairs[lpos + u];
+                ReqBytes rq;
+                req_bytes_for(rq, (u32)hm.y, (u64)pr.x + pr.y, mi.kv_tok);
+                bmax[u] = (rq.small && (avail >> 52) == 0) ? floor_div_recip(avail, rq.bytes, rq.inv) : avail / rq.bytes;
+            }
+        } else st0 |= 1;
+        const uint2 bm = make_uint2(clamp_u32(bmax[0]), clamp_u32(bmax[1]));
+        // the largest batch size either of the two positions takes; the neighbouring lane holds the
+        // other half of the foursome
+        const u64 mine = st0 ? 0 : (bmax[0] > bmax[1] ? bmax[0] : bmax[1]);
+        const u64 other = __shfl_xor_sync(0xFFFFFFFFu, mine, 1);
+        const u64 four_max = mine > other ? mine : other;   // a config of the foursome fits <=> b <= four_max
+        u64 j = ((u64)mpos * n_hf + hf) * ((u64)s.n_b * n_tl) + tl;
+        if (active) {
+            for (u32 bi = 0; bi < s.n_b; bi++, j += n_tl) {
+                const u64 b = __ldg(s.batch + bi);
+                const u32 sa = st0 | (b > bmax[0] ? 2u : 0u), sb = st0 | (b > bmax[1] ? 2u : 0u);
+                if (o.status) __stcs(reinterpret_cast<unsigned short *>(o.status + j), (unsigned short)(sa | (sb << 8)));
+                if (o.bmax) __stcs(reinterpret_cast<uint2 *>(o.bmax + j), bm);
+                if (b > four_max) {                         // nothing in the foursome fits (batch sizes are >= 1)
+                    for (int a = 0; a < n_const; a++)
+                        __stcs(reinterpret_cast<ulonglong2 *>(s_p[a] + j), make_ulonglong2(s_pat[a], s_pat[a]));
+                }
+            }
+        }
+    }
+}
+
+// Performance model for the configs that fit.  Work items: (chunk of the sorted pair walk, group of
+// 16 foursomes in plane_order, model, batch), heaviest chunks and groups first, handed out through a
+// counter to a persistent grid: the items differ wildly in cost (most have nothing that fits).
+template <int TIME_SUM>
+__global__ void __launch_bounds__(MODEL_THREADS, 8)
+k_closed_form_model(DSpace s, int tp_model, guide_outputs o, u32 groups, u32 chunk, u32 n_chunks, unsigned *ticket) {
+    __shared__ u32 s_item;
+    const u32 n_tl = s.n_t * s.n_l, n_hf = s.n_h * s.n_f;
+    const u32 n_mb = s.n_m * s.n_b;
+    const u32 n_items = n_mb * groups * n_chunks;
+  for (;;) {
+    __syncthreads();                                  // everyone is done with the previous item
+    if (threadIdx.x == 0) s_item = atomicAdd(ticket, 1u);
+    __syncthreads();
+    const u32 item = s_item;
+    if (item >= n_items) break;
+    const u32 mb = item % n_mb;
+    const u32 grp = (item / n_mb) % groups, chunk_i = item / (n_mb * groups);
+    const u32 bpos = mb % s.n_b, mpos = mb / s.n_b;
+    const u32 lane = threadIdx.x & 31;
+    const u32 four = (grp * MODEL_THREADS + threadIdx.x) >> 2;          // rank of this lane's foursome in plane_order
+    const bool in_plane = four < (n_tl >> 2);
+    const u32 tl = __ldg(s.plane_order + (size_t)mpos * (n_tl >> 2) + (in_plane ? four : 0)) * 4 + (threadIdx.x & 3);
+    const u32 tpos = tl / s.n_l, lpos = tl % s.n_l;
+    const DModel m = s.models[mpos];
+    const u32 t = s.tp[tpos], b = s.batch[bpos];
+    // lanes without a point, or whose TP degree does not divide the heads, never fit; they stay for the warp votes
+    const bool alive = in_plane && (m.nh & (t - 1)) == 0 && (m.nkv & (t - 1)) == 0;
+    const uint2 pr = s.pairs[lpos];
+    const u32 lin = pr.x, lout = pr.y, n = lout - 1;
+    const MemInfo mi = mem_info(m, t);
+    const u64 S = (u64)lin + lout;
+    const double inf = __longlong_as_double(0x7FF0000000000000LL);
+    const u64 stride_hf = (u64)s.n_b * n_tl;
+    const u64 j0 = (u64)mpos * n_hf * stride_hf + (u64)bpos * n_tl + tl;
+    TaskTab kp, kd;
+    bool built = false;
+    u32 cur_block = 0;
+    u64 need = 0;
+    const u32 p_end = min(n_hf, (chunk_i + 1) * chunk);
+    u32 p = chunk_i * chunk;
+    while (p < p_end) {
+        const HfSorted e = s.hf_sorted[p];            // same address in every lane
+        if (e.block != cur_block) {
+            cur_block = e.block;
+            ReqBytes rq;
+            req_bytes_for(rq, e.block, S, mi.kv_tok);
+            need = __umul64hi((u64)b, rq.bytes) ? ~0ull : (u64)b * rq.bytes;
+        }
+        // fits <=> usable > weights and b <= floor((usable - weights) / bytes) <=> b x bytes <= usable - weights
+        const bool fits = alive && e.usable > mi.w_gpu && e.usable - mi.w_gpu >= need;
+        const u32 vote = __ballot_sync(0xFFFFFFFFu, fits);
+        if (vote == 0) {                              // nor will any later pair of this block size: skip to the next
+            p = e.seg_end;
+            continue;
+        }
+        Metrics out;
+        out.latency = inf; out.ttft = inf; out.tpot = inf; out.thr = 0.0; out.cost_hr = inf; out.cost_tok = inf;
+        out.n_iters = 0; out.n_req_iters = 0;
+        // The stage tables are built by the whole warp at the first pair any of its lanes fits: the
+        // lanes are ordered by need, so the others follow within a few pairs, and a build the warp
+        // does in step costs a fraction of builds scattered over the walk.
+        if (!built) {
+            if (alive) {
+                const u32 tt = tp_model ? 1u : t;
+                const u64 Tp = (u64)b * lin;
+                build_fixed_tasks(m, tt, Tp, b, 1, kp);
+                build_attn_tasks(m, tt, Tp, Tp * lin, Tp, kp);
+                const u32 nn = n > 0 ? n : 1;          // a table is built either way; unused when n == 0
+                const u64 Td = (u64)b * nn;
+                const u64 ctx = (u64)b * ((u64)nn * lin + ((u64)nn * (nn + 1)) / 2);
+                build_fixed_tasks(m, tt, Td, Td, nn, kd);
+                build_attn_tasks(m, tt, Td, ctx, ctx, kd);
+            }
+            built = true;
+        }
+        if (fits) {
+            const DRate &rt = s.rates[e.hf];
+            const double lf = log2_rule_factor(t, tp_model);
+            const double Nd = (double)m.N;
+            const double t_pre = eval_phase<TIME_SUM>(kp, rt, Nd, lf);
+            const double t_dec = n > 0 ? eval_phase<TIME_SUM>(kd, rt, Nd, lf) : 0.0;
+            const u32 ci = e.hf * s.n_t + tpos;
+            out.ttft = t_pre;
+            out.latency = t_pre + t_dec;
+            out.cost_hr = __ldg(s.cost_hr + ci);
+            if (n > 0) {
+                out.tpot = t_dec / (double)n;
+                out.thr = cvt((u64)b * n) / t_dec;
+                out.cost_tok = __ldg(s.cost_sec + ci) / out.thr;
+            } else {
+                out.tpot = 0.0; out.thr = 0.0; out.cost_tok = inf;
+            }
+            out.n_iters = 1 + (u64)n;
+            out.n_req_iters = (u64)b * (1 + (u64)n);
+        }
+        // the whole foursome is written here as soon as one of its configs fits
+        if ((vote >> (lane & ~3u)) & 0xFu) {
+            const u64 j = j0 + (u64)e.hf * stride_hf;
+            if (o.latency) __stcs(o.latency + j, out.latency);
+            if (o.ttft) __stcs(o.ttft + j, out.ttft);
+            if (o.ttft_p50) __stcs(o.ttft_p50 + j, out.ttft);
+            if (o.ttft_p99) __stcs(o.ttft_p99 + j, out.ttft);
+            if (o.tpot) __stcs(o.tpot + j, out.tpot);
+            if (o.thr_decode) __stcs(o.thr_decode + j, out.thr);
+            if (o.cost_per_hr) __stcs(o.cost_per_hr + j, out.cost_hr);
+            if (o.cost_per_token) __stcs(o.cost_per_token + j, out.cost_tok);
+            if (o.n_iters) __stcs(o.n_iters + j, out.n_iters);
+            if (o.n_req_iters) __stcs(o.n_req_iters + j, out.n_req_iters);
+        }
+        p++;
+    }
+  }
+    // the grid must not be complete before the memory kernel is: whatever follows in the stream
+    // waits for this one only
+    cf_dep_wait();
+}
+
+// Does the call suit the split kernels?  Fills the list of constant-filled arrays.
+static bool split_applies(const DSpace &s, Range r, const guide_outputs &o, ConstOut *co) {
+    const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
+    const u32 n_tl = s.n_t * s.n_l;
+    if (r.first != 0 || r.count != total || total < (1u << 16)) return false;       // whole spaces only
+    if (s.n_l % 4 != 0 || n_tl < 32) return false;
+    if ((u64)s.n_m * ((n_tl + 255) / 256) * s.n_h * s.n_f > 0x7FFFFFFFull) return false;
+    auto al = [](const void *p, uintptr_t a) { return ((uintptr_t)p % a) == 0; };
+    const void *wide[] = {o.latency, o.ttft, o.ttft_p50, o.ttft_p99, o.tpot, o.thr_decode, o.cost_per_hr, o.cost_per_token,
+                          o.n_iters, o.n_req_iters};
+    for (const void *p : wide)
+        if (p && !al(p, 32)) return false;                  // foursomes are sectors only if the arrays start on one
+    if ((o.bmax && !al(o.bmax, 8)) || (o.status && !al(o.status, 2))) return false;
+    const unsigned long long inf = 0x7FF0000000000000ull;
+    co->n = 0;
+    for (int i = 0; i < SPLIT_MAX_CONST; i++) { co->p[i] = nullptr; co->pat[i] = 0; }
+    auto add = [&](void *p, unsigned long long pat) { if (p) { co->p[co->n] = (unsigned long long *)p; co->pat[co->n] = pat; co->n++; } };
+    add(o.latency, inf); add(o.ttft, inf); add(o.ttft_p50, inf); add(o.ttft_p99, inf); add(o.tpot, inf);
+    add(o.thr_decode, 0); add(o.cost_per_hr, inf); add(o.cost_per_token, inf); add(o.n_iters, 0); add(o.n_req_iters, 0);
+    return true;
+}
+
+template <int TIME_SUM>
+static int launch_split(const DSpace &s, int tp_model, const guide_outputs &o, const ConstOut &co, unsigned *ticket,
+                        cudaStream_t st) {
+    const u32 n_tl = s.n_t * s.n_l, n_hf = s.n_h * s.n_f;
+    const u32 tiles = (n_tl + 2 * MEM_THREADS - 1) / (2 * MEM_THREADS);
+    const u32 items = s.n_m * tiles * n_hf;
+    const u32 mem_grid = std::min<u32>(items, (u32)num_sms() * MEM_BLOCKS_PER_SM);
+    GUIDE_CUDA(cudaMemsetAsync(ticket, 0, 4, st));           // the model kernel's work counter
+    k_closed_form_memory<<<mem_grid, MEM_THREADS, 0, st>>>(s, o, co, tiles);
+    GUIDE_CUDA(cudaGetLastError());
+    // chunks of the pair walk: 16 pairs, so that a point's stage tables serve many configs while
+    // the longest item stays short next to the whole launch
+    const u32 groups = (n_tl + MODEL_THREADS - 1) / MODEL_THREADS;
+    const u32 chunk = std::min<u32>(16, n_hf);
+    const u32 n_chunks = (n_hf + chunk - 1) / chunk;
+    if ((u64)s.n_m * s.n_b * groups * n_chunks > 0x7FFFFFFFull) return fail(GUIDE_ERR_UNSUPPORTED, "space too large for one launch");
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((u32)num_sms() * 8); cfg.blockDim = dim3(MODEL_THREADS); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_closed_form_model<TIME_SUM>, s, tp_model, o, groups, chunk, n_chunks, ticket));
+    return GUIDE_OK;
+}
+
 int launch_closed_form(const DSpace &s, Range r, int time_model, int tp_model, const guide_outputs &o,
-                       cudaStream_t st) {
+                       unsigned *ticket, cudaStream_t st) {
     const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
     // The tiled kernel pays off when a (TP, length) plane fills warps and the range is (most of)
     // the space; slivers of the space go through the flat kernel.
+    ConstOut co;
+    if (ticket && split_applies(s, r, o, &co))
+        return time_model ? launch_split<1>(s, tp_model, o, co, ticket, st) : launch_split<0>(s, tp_model, o, co, ticket, st);
     TileGeom g;
     const bool tiled = r.count * 2 >= total && tiled_geometry(s, (u64)num_sms() * 16, 1ull << 30, &g);
     if (!tiled) {

@@ -142,12 +142,73 @@ __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *g
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-int space_on_device(guide_space *s, DSpace *out) {
+// Work orders for the closed-form model kernel.  They decide which thread evaluates what, never a
+// value: any permutation gives the same outputs.
+//
+// The pairs, grouped by KV block size and, inside a group, by falling usable memory (the formula
+// of k_build_tables): the pairs a config fits are then a prefix of each group.
+static std::vector<HfSorted> sorted_pairs(const guide_space &s) {
+    const size_t n_f = s.fw.size(), n = s.hw.size() * n_f;
+    std::vector<HfSorted> v(n);
+    for (size_t i = 0; i < n; i++) {
+        const guide_hw &h = s.hw[i / n_f];
+        const guide_fw &f = s.fw[i % n_f];
+        v[i].usable = h.mem_bytes - (h.mem_bytes / 1000) * f.reserve_permille;
+        v[i].block = f.kv_block;
+        v[i].hf = (u32)i;
+        v[i].seg_end = 0; v[i].pad = 0;
+    }
+    std::stable_sort(v.begin(), v.end(), [](const HfSorted &a, const HfSorted &b) {
+        return a.block != b.block ? a.block < b.block : a.usable > b.usable;
+    });
+    for (size_t i = n; i-- > 0;) v[i].seg_end = (i + 1 < n && v[i + 1].block == v[i].block) ? v[i + 1].seg_end : (u32)(i + 1);
+    return v;
+}
+
+// Per model, the foursomes (four consecutive positions) of the (TP, length) plane by growing memory
+// need of their cheapest position (weights per GPU plus the KV cache of a middle batch size);
+// foursomes whose TP degree does not divide the heads last.  Lanes of a warp then fit about the
+// same number of pairs.  When the plane does not divide into foursomes the table is not used.
+static std::vector<u32> plane_orders(const guide_space &s) {
+    const size_t n_t = s.tp.size(), n_l = s.pairs.size(), n_tl = n_t * n_l, n_four = n_tl / 4;
+    std::vector<u32> out(s.models.size() * std::max<size_t>(n_four, 1), 0);
+    if (n_l % 4 != 0) return out;
+    const double b_ref = (double)s.batch[s.batch.size() / 2];
+    const double blk = (double)std::max<u32>(s.fw[0].kv_block, 1);
+    std::vector<double> key(n_four);
+    for (size_t mi = 0; mi < s.models.size(); mi++) {
+        const guide_model &m = s.models[mi];
+        const double H = m.hidden, Dkv = (double)m.n_kv_heads * (m.hidden / m.n_heads), I = m.ffn, V = m.vocab;
+        const double wbytes = (m.n_layers * (2 * H * H + 2 * H * Dkv + (2.0 + m.gated) * H * I) + 2 * V * H) * m.w_bytes;
+        const double kv2 = 2.0 * m.n_layers * Dkv * m.kv_bytes;
+        for (size_t q = 0; q < n_four; q++) {
+            const u32 t = s.tp[(4 * q) / n_l];
+            const bool bad = (m.n_heads % t) != 0 || (m.n_kv_heads % t) != 0;
+            double best = INFINITY;
+            for (size_t u = 0; u < 4 && !bad; u++) {
+                const guide_len_pair &pr = s.pairs[(4 * q + u) % n_l];
+                const double S = std::ceil(((double)pr.lin + pr.lout) / blk) * blk;
+                best = std::min(best, wbytes / t + b_ref * S * (kv2 / t));
+            }
+            key[q] = best;
+        }
+        u32 *o = out.data() + mi * n_four;
+        for (size_t q = 0; q < n_four; q++) o[q] = (u32)q;
+        std::stable_sort(o, o + n_four, [&](u32 a, u32 b) { return key[a] < key[b]; });
+    }
+    return out;
+}
+
+int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
     int dev = 0;
     GUIDE_CUDA(cudaGetDevice(&dev));
     std::lock_guard<std::mutex> lock(s->mu);
-    for (const DeviceTables &d : s->dev)
-        if (d.device == dev) { *out = d.view; return GUIDE_OK; }
+    for (DeviceTables &d : s->dev)
+        if (d.device == dev) {
+            *out = d.view;
+            if (ticket) *ticket = d.tickets + 32 * (d.next_ticket++ % TICKET_SLOTS);
+            return GUIDE_OK;
+        }
 
     const size_t n_m = s->models.size(), n_h = s->hw.size(), n_f = s->fw.size();
     size_t off = 0;
@@ -157,7 +218,9 @@ int space_on_device(guide_space *s, DSpace *out) {
                  o_dr = take(n_h * n_f * sizeof(DRate)), o_b = take(s->batch.size() * 4),
                  o_t = take(s->tp.size() * 4), o_p = take(s->pairs.size() * 8),
                  o_ch = take(n_h * n_f * s->tp.size() * 8), o_cs = take(n_h * n_f * s->tp.size() * 8),
-                 o_hm = take(n_h * n_f * 16);
+                 o_hm = take(n_h * n_f * 16), o_hs = take(n_h * n_f * sizeof(HfSorted)),
+                 o_po = take(std::max<size_t>(n_m * (s->tp.size() * s->pairs.size() / 4), 1) * 4),
+                 o_tk = take(TICKET_SLOTS * 128);
     char *blob = nullptr;
     GUIDE_CUDA(cudaMalloc(&blob, off));
     cudaError_t e = cudaSuccess;
@@ -170,6 +233,10 @@ int space_on_device(guide_space *s, DSpace *out) {
     put(o_b, s->batch.data(), s->batch.size() * 4);
     put(o_t, s->tp.data(), s->tp.size() * 4);
     put(o_p, s->pairs.data(), s->pairs.size() * 8);
+    const std::vector<HfSorted> hf_sorted = sorted_pairs(*s);
+    const std::vector<u32> plane_order = plane_orders(*s);
+    put(o_hs, hf_sorted.data(), hf_sorted.size() * sizeof(HfSorted));
+    put(o_po, plane_order.data(), plane_order.size() * 4);
     if (e == cudaSuccess) {
         const u32 n = (u32)std::max(n_m, n_h * n_f);
         k_build_tables<<<(n + 127) / 128, 128>>>((const guide_model *)(blob + o_gm), (u32)n_m,
@@ -194,8 +261,12 @@ int space_on_device(guide_space *s, DSpace *out) {
     d.view.cost_hr = (const double *)(blob + o_ch);
     d.view.cost_sec = (const double *)(blob + o_cs);
     d.view.hfmem = (const ulonglong2 *)(blob + o_hm);
+    d.view.hf_sorted = (const HfSorted *)(blob + o_hs);
+    d.view.plane_order = (const u32 *)(blob + o_po);
     d.view.n_m = (u32)n_m; d.view.n_h = (u32)n_h; d.view.n_f = (u32)n_f;
     d.view.n_b = (u32)s->batch.size(); d.view.n_t = (u32)s->tp.size(); d.view.n_l = (u32)s->pairs.size();
+    d.tickets = (unsigned *)(blob + o_tk);
+    if (ticket) *ticket = d.tickets + 32 * (d.next_ticket++ % TICKET_SLOTS);
     s->dev.push_back(d);
     *out = d.view;
     return GUIDE_OK;
@@ -472,8 +543,9 @@ int guide_simulate(const guide_space *space_c, const guide_trace *trace_c, const
     }
     if (r.count == 0) return GUIDE_OK;
     DSpace ds;
-    if ((rc = space_on_device(space, &ds))) return rc;
-    if (!trace) return launch_closed_form(ds, r, time_model, tp_model, *out, (cudaStream_t)stream);
+    unsigned *ticket = nullptr;
+    if ((rc = space_on_device(space, &ds, &ticket))) return rc;
+    if (!trace) return launch_closed_form(ds, r, time_model, tp_model, *out, ticket, (cudaStream_t)stream);
     DTrace dt;
     if ((rc = trace_on_device(trace, &dt))) return rc;
     return launch_trace_sim(ds, dt, r, time_model, tp_model, opts ? opts->max_iters : 0, *out, ws, ws_bytes,

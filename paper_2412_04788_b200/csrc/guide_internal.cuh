@@ -21,10 +21,16 @@ int cuda_fail(cudaError_t e, const char *what);
         if (e__ != cudaSuccess) return guide::cuda_fail(e__, #call); \
     } while (0)
 
+// Work counters of the persistent closed-form model kernel: one 128-byte slot per call in flight,
+// handed out in turn, so that calls on different streams do not share one.
+static constexpr unsigned TICKET_SLOTS = 64;
+
 struct DeviceTables {
     int device = -1;
     void *blob = nullptr;
     DSpace view{};
+    unsigned *tickets = nullptr;     // TICKET_SLOTS slots, 32 words apart
+    unsigned next_ticket = 0;
 };
 
 struct DeviceTrace {
@@ -59,12 +65,12 @@ struct guide_trace {
 namespace guide {
 
 // device views for the current device (uploads on first use)
-int space_on_device(guide_space *s, DSpace *out);
+int space_on_device(guide_space *s, DSpace *out, unsigned **ticket = nullptr);
 int trace_on_device(guide_trace *t, DTrace *out);
 
 // closed_form.cu
 int launch_closed_form(const DSpace &s, Range r, int time_model, int tp_model, const guide_outputs &o,
-                       cudaStream_t st);
+                       unsigned *ticket, cudaStream_t st);
 // trace_sim.cu
 size_t trace_workspace_bytes(u32 n_req);
 int launch_trace_sim(const DSpace &s, const DTrace &t, Range r, int time_model, int tp_model, u64 max_iters,

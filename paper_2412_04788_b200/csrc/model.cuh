@@ -33,6 +33,15 @@ struct DRate {
     u32 flash, kv_block;
 };
 
+// one hardware x framework pair in the sorted walk of the model kernel
+struct HfSorted {
+    u64 usable;
+    u32 block;        // KV block size
+    u32 hf;           // pair index h * n_f + f
+    u32 seg_end;      // sorted position one past the last pair with this block size
+    u32 pad;
+};
+
 struct DSpace {
     const DModel *models;
     const DRate *rates;          // [n_h * n_f]
@@ -41,6 +50,9 @@ struct DSpace {
     const double *cost_hr;       // [n_h * n_f][n_t]: price x TP degree
     const double *cost_sec;      // [n_h * n_f][n_t]: (price x TP degree) / 3600
     const ulonglong2 *hfmem;     // [n_h * n_f]: x = usable bytes, y = KV block size (what the memory check reads)
+    // Orders that only steer which thread does what (any permutation gives the same results):
+    const HfSorted *hf_sorted;   // [n_h * n_f]: the pairs grouped by KV block size, largest usable memory first
+    const u32 *plane_order;      // [n_m][n_t * n_l / 4]: foursomes of the (TP, length) plane by growing memory need
     u32 n_m, n_h, n_f, n_b, n_t, n_l;
 };
 
