@@ -72,7 +72,9 @@ __global__ void __launch_bounds__(256, 2) k_closed_form_tiled(DSpace s, Range r,
 
 static constexpr u32 MEM_THREADS = 128;         // x 2 positions = 256 positions of the plane per work item
 static constexpr u32 MEM_BLOCKS_PER_SM = 2;
-static constexpr u32 MODEL_THREADS = 64;
+static constexpr u32 MODEL_THREADS = 128;
+static constexpr u32 MODEL_BLOCKS_PER_SM = 8;
+static constexpr u32 MODEL_CHUNK = 64;          // sorted pairs per work item
 static constexpr int SPLIT_MAX_CONST = 10;
 
 // 8-byte arrays that receive a constant for a config that does not fit (+inf, or 0 for throughput and counters)
@@ -145,119 +147,180 @@ __global__ void __launch_bounds__(MEM_THREADS) k_closed_form_memory(DSpace s, gu
     }
 }
 
-// Performance model for the configs that fit.  Work items: (chunk of the sorted pair walk, group of
-// 16 foursomes in plane_order, model, batch), heaviest chunks and groups first, handed out through a
-// counter to a persistent grid: the items differ wildly in cost (most have nothing that fits).
+// Stage table of one point in shared memory: twelve (x, y) entries per stage, interleaved over
+// the four points of a foursome so that the lanes of a warp read neighbouring words.
+//   0 (F1,B1) 1 (F2,B2) 2 (F3,B3) 3 (F5,B5) 4 (F6,B6) 5 (F7,B7) 6 (F8,B8) 7 (F9,B9) 8 (B9x,F10)
+//   9 (B10x,F13) 10 (B13,hops) 11 (cbytes,Rd)
+typedef double2 StageTab[12][4];
+
+__device__ __forceinline__ void put_stage(StageTab &tb, u32 u, const TaskTab &k) {
+    tb[0][u] = make_double2(k.F1, k.B1); tb[1][u] = make_double2(k.F2, k.B2); tb[2][u] = make_double2(k.F3, k.B3);
+    tb[3][u] = make_double2(k.F5, k.B5); tb[4][u] = make_double2(k.F6, k.B6); tb[5][u] = make_double2(k.F7, k.B7);
+    tb[6][u] = make_double2(k.F8, k.B8); tb[7][u] = make_double2(k.F9, k.B9); tb[8][u] = make_double2(k.B9x, k.F10);
+    tb[9][u] = make_double2(k.B10x, k.F13); tb[10][u] = make_double2(k.B13, k.hops); tb[11][u] = make_double2(k.cbytes, k.Rd);
+}
+
+// Both stage tables of one point, written to shared memory.  Kept out of line: it runs once per
+// work item and needs far more registers than the walk around it.
+__device__ __noinline__ void build_point_tables(const DModel *mp, u32 tt, u32 b, u32 lin, u32 n, StageTab *tb_pre, StageTab *tb_dec,
+                                                u32 u) {
+    const DModel m = *mp;
+    TaskTab k;
+    const u64 Tp = (u64)b * lin;
+    build_fixed_tasks(m, tt, Tp, b, 1, k);
+    build_attn_tasks(m, tt, Tp, Tp * lin, Tp, k);
+    put_stage(*tb_pre, u, k);
+    const u32 nn = n > 0 ? n : 1;          // a table is built either way; unused when n == 0
+    const u64 Td = (u64)b * nn;
+    const u64 ctx = (u64)b * ((u64)nn * lin + ((u64)nn * (nn + 1)) / 2);
+    build_fixed_tasks(m, tt, Td, Td, nn, k);
+    build_attn_tasks(m, tt, Td, ctx, ctx, k);
+    put_stage(*tb_dec, u, k);
+}
+
+// rates of one pair in registers (a row of rate10)
+struct RateRegs { double icL, icA, icE, imL, imA, imE, inv_comm, clat, tovh, flash; };
+
+// eval_phase of model.cuh, operation for operation, with the task entries read from a StageTab
 template <int TIME_SUM>
-__global__ void __launch_bounds__(MODEL_THREADS, 8)
-k_closed_form_model(DSpace s, int tp_model, guide_outputs o, u32 groups, u32 chunk, u32 n_chunks, unsigned *ticket) {
-    __shared__ u32 s_item;
-    const u32 n_tl = s.n_t * s.n_l, n_hf = s.n_h * s.n_f;
+__device__ __forceinline__ double eval_stage(const StageTab &tb, u32 u, const RateRegs &r, double Nd, double log2_factor) {
+    const double2 e1 = tb[0][u], e2 = tb[1][u], e3 = tb[2][u], e5 = tb[3][u];
+    const double t2 = task_time<TIME_SUM>(e2.x, e2.y, r.icL, r.imL);
+    double sfix = task_time<TIME_SUM>(e1.x, e1.y, r.icE, r.imE);
+    sfix = sfix + t2;
+    sfix = sfix + task_time<TIME_SUM>(e3.x, e3.y, r.icL, r.imL);
+    sfix = sfix + t2;
+    sfix = sfix + task_time<TIME_SUM>(e5.x, e5.y, r.icE, r.imE);
+    const double2 e6 = tb[4][u], e7 = tb[5][u], e8 = tb[6][u];
+    sfix = sfix + task_time<TIME_SUM>(e6.x, e6.y, r.icL, r.imL);
+    sfix = sfix + task_time<TIME_SUM>(e7.x, e7.y, r.icE, r.imE);
+    sfix = sfix + task_time<TIME_SUM>(e8.x, e8.y, r.icL, r.imL);
+    const double2 e9 = tb[7][u], e9x = tb[8][u], e10x = tb[9][u];
+    const bool flash = r.flash != 0.0;
+    const double t9 = task_time<TIME_SUM>(e9.x, flash ? e9.y : e9x.x, r.icA, r.imA);
+    const double t10 = task_time<TIME_SUM>(e9x.y, flash ? 0.0 : e10x.x, r.icA, r.imA);
+    const double satt = (t9 + t10) + t9;
+    const double2 e13 = tb[10][u], ec = tb[11][u];
+    const double scomm = 2.0 * (e13.y * r.clat + ec.x * r.inv_comm);
+    const double thead = task_time<TIME_SUM>(e10x.y, e13.x, r.icL, r.imL);
+    return combine_phase(sfix, satt, scomm, thead, ec.y, Nd, r.tovh, log2_factor);
+}
+
+// Performance model for the configs that fit.  A warp takes one foursome of the plane for one
+// (model, batch) and a chunk of the sorted pair walk; its lanes are four points x eight pairs, so
+// the four lanes that share a pair write one whole sector.  The stage tables of the four points
+// sit in shared memory (built once per item by four lanes), the rates of a lane's pair in
+// registers: that is half the registers of a table per thread, hence twice the warps.  Work items
+// differ wildly in cost (most have nothing that fits): they are handed out through a counter to a
+// persistent grid, heaviest chunks and foursomes first.
+template <int TIME_SUM>
+__global__ void __launch_bounds__(MODEL_THREADS, MODEL_BLOCKS_PER_SM)
+k_closed_form_model(DSpace s, int tp_model, guide_outputs o, u32 n_chunks, unsigned *ticket) {
+    __shared__ StageTab s_tab[MODEL_THREADS / 32][2];
+    const u32 lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const u32 u = lane & 3, h = lane >> 2;
+    StageTab &tb_pre = s_tab[warp][0], &tb_dec = s_tab[warp][1];
+    const u32 n_tl = s.n_t * s.n_l, n_hf = s.n_h * s.n_f, n_four = n_tl >> 2;
     const u32 n_mb = s.n_m * s.n_b;
-    const u32 n_items = n_mb * groups * n_chunks;
-  for (;;) {
-    __syncthreads();                                  // everyone is done with the previous item
-    if (threadIdx.x == 0) s_item = atomicAdd(ticket, 1u);
-    __syncthreads();
-    const u32 item = s_item;
-    if (item >= n_items) break;
-    const u32 mb = item % n_mb;
-    const u32 grp = (item / n_mb) % groups, chunk_i = item / (n_mb * groups);
-    const u32 bpos = mb % s.n_b, mpos = mb / s.n_b;
-    const u32 lane = threadIdx.x & 31;
-    const u32 four = (grp * MODEL_THREADS + threadIdx.x) >> 2;          // rank of this lane's foursome in plane_order
-    const bool in_plane = four < (n_tl >> 2);
-    const u32 tl = __ldg(s.plane_order + (size_t)mpos * (n_tl >> 2) + (in_plane ? four : 0)) * 4 + (threadIdx.x & 3);
-    const u32 tpos = tl / s.n_l, lpos = tl % s.n_l;
-    const DModel m = s.models[mpos];
-    const u32 t = s.tp[tpos], b = s.batch[bpos];
-    // lanes without a point, or whose TP degree does not divide the heads, never fit; they stay for the warp votes
-    const bool alive = in_plane && (m.nh & (t - 1)) == 0 && (m.nkv & (t - 1)) == 0;
-    const uint2 pr = s.pairs[lpos];
-    const u32 lin = pr.x, lout = pr.y, n = lout - 1;
-    const MemInfo mi = mem_info(m, t);
-    const u64 S = (u64)lin + lout;
+    const u32 n_items = n_mb * n_four * n_chunks;
     const double inf = __longlong_as_double(0x7FF0000000000000LL);
     const u64 stride_hf = (u64)s.n_b * n_tl;
-    const u64 j0 = (u64)mpos * n_hf * stride_hf + (u64)bpos * n_tl + tl;
-    TaskTab kp, kd;
-    bool built = false;
-    u32 cur_block = 0;
-    u64 need = 0;
-    const u32 p_end = min(n_hf, (chunk_i + 1) * chunk);
-    u32 p = chunk_i * chunk;
-    while (p < p_end) {
-        const HfSorted e = s.hf_sorted[p];            // same address in every lane
-        if (e.block != cur_block) {
-            cur_block = e.block;
-            ReqBytes rq;
-            req_bytes_for(rq, e.block, S, mi.kv_tok);
-            need = __umul64hi((u64)b, rq.bytes) ? ~0ull : (u64)b * rq.bytes;
+    for (;;) {
+        u32 item = 0;
+        if (lane == 0) item = atomicAdd(ticket, 1u);
+        item = __shfl_sync(0xFFFFFFFFu, item, 0);
+        if (item >= n_items) break;
+        const u32 mb = item % n_mb, rest = item / n_mb;
+        const u32 rank = rest % n_four, chunk_i = rest / n_four;
+        const u32 bpos = mb % s.n_b, mpos = mb / s.n_b;
+        const u32 tl = __ldg(s.plane_order + (size_t)mpos * n_four + rank) * 4 + u;
+        const u32 tpos = tl / s.n_l, lpos = tl % s.n_l;
+        const DModel *mp = s.models + mpos;
+        const u32 t = s.tp[tpos], b = s.batch[bpos];
+        const u32 nh = mp->nh, nkv = mp->nkv;
+        if ((nh & (t - 1)) != 0 || (nkv & (t - 1)) != 0) continue;          // the foursome shares its TP degree: nothing fits
+        const uint2 pr = s.pairs[lpos];
+        const u32 lin = pr.x, lout = pr.y, n = lout - 1;
+        const u32 log2t = 31 - __clz(t);
+        const u64 w_gpu = (mp->wbytes + (u64)(t - 1)) >> log2t;            // as mem_info
+        const u64 kv_tok = mp->kv2 >> log2t;
+        const u64 S = (u64)lin + lout;
+        const u32 p_lo = chunk_i * MODEL_CHUNK, p_hi = min(n_hf, p_lo + MODEL_CHUNK);
+        // Does anything fit?  Per KV block size the first pair of the chunk has the most memory.
+        bool any = false;
+        for (u32 p0 = p_lo; p0 < p_hi;) {
+            const HfSorted e0 = s.hf_sorted[p0];
+            const u64 s_blk = e0.block == 1 ? S : ((S + e0.block - 1) / e0.block) * e0.block;
+            const u64 bytes = s_blk * kv_tok;
+            const u64 need = __umul64hi((u64)b, bytes) ? ~0ull : (u64)b * bytes;
+            any |= e0.usable > w_gpu && e0.usable - w_gpu >= need;
+            p0 = e0.seg_end;
         }
-        // fits <=> usable > weights and b <= floor((usable - weights) / bytes) <=> b x bytes <= usable - weights
-        const bool fits = alive && e.usable > mi.w_gpu && e.usable - mi.w_gpu >= need;
-        const u32 vote = __ballot_sync(0xFFFFFFFFu, fits);
-        if (vote == 0) {                              // nor will any later pair of this block size: skip to the next
-            p = e.seg_end;
-            continue;
-        }
-        Metrics out;
-        out.latency = inf; out.ttft = inf; out.tpot = inf; out.thr = 0.0; out.cost_hr = inf; out.cost_tok = inf;
-        out.n_iters = 0; out.n_req_iters = 0;
-        // The stage tables are built by the whole warp at the first pair any of its lanes fits: the
-        // lanes are ordered by need, so the others follow within a few pairs, and a build the warp
-        // does in step costs a fraction of builds scattered over the walk.
-        if (!built) {
-            if (alive) {
-                const u32 tt = tp_model ? 1u : t;
-                const u64 Tp = (u64)b * lin;
-                build_fixed_tasks(m, tt, Tp, b, 1, kp);
-                build_attn_tasks(m, tt, Tp, Tp * lin, Tp, kp);
-                const u32 nn = n > 0 ? n : 1;          // a table is built either way; unused when n == 0
-                const u64 Td = (u64)b * nn;
-                const u64 ctx = (u64)b * ((u64)nn * lin + ((u64)nn * (nn + 1)) / 2);
-                build_fixed_tasks(m, tt, Td, Td, nn, kd);
-                build_attn_tasks(m, tt, Td, ctx, ctx, kd);
+        if (!__any_sync(0xFFFFFFFFu, any)) continue;
+        __syncwarp();                                 // the previous item's reads of the tables are over
+        if (h == 0) build_point_tables(mp, tp_model ? 1u : t, b, lin, n, &tb_pre, &tb_dec, u);      // lane u: point u
+        __syncwarp();
+        const u64 j0 = (u64)mpos * n_hf * stride_hf + (u64)bpos * n_tl + tl;
+        const double lf = log2_rule_factor(t, tp_model);
+        const double Nd = (double)mp->N;
+        u32 p0 = p_lo;
+        while (p0 < p_hi) {
+            // one KV block size at a time: within it the pairs are sorted by falling usable memory
+            const HfSorted e0 = s.hf_sorted[p0];
+            const u32 seg_end = min(e0.seg_end, p_hi);
+            const u64 s_blk = e0.block == 1 ? S : ((S + e0.block - 1) / e0.block) * e0.block;
+            const u64 bytes = s_blk * kv_tok;
+            const u64 need = __umul64hi((u64)b, bytes) ? ~0ull : (u64)b * bytes;
+            for (u32 pp = p0; pp < seg_end; pp += 8) {
+                const u32 p = pp + h;
+                const bool in = p < seg_end;
+                const HfSorted e = s.hf_sorted[in ? p : seg_end - 1];
+                // fits <=> usable > weights and b <= floor((usable - weights) / bytes) <=> b x bytes <= usable - weights
+                const bool fits = in && e.usable > w_gpu && e.usable - w_gpu >= need;
+                const u32 vote = __ballot_sync(0xFFFFFFFFu, fits);
+                if (vote == 0) break;                 // nor does any later pair of this block size
+                double latency = inf, ttft = inf, tpot = inf, thr = 0.0, cost_hr = inf, cost_tok = inf;
+                u64 n_iters = 0, n_req_iters = 0;
+                if (fits) {
+                    const double2 *q = reinterpret_cast<const double2 *>(s.rate10 + (size_t)e.hf * 10);
+                    const double2 q0 = __ldg(q), q1 = __ldg(q + 1), q2 = __ldg(q + 2), q3 = __ldg(q + 3), q4 = __ldg(q + 4);
+                    RateRegs r;      // rate10 row: inv_c[LINEAR, ATTN, ELEM], inv_m[LINEAR, ATTN, ELEM], inv_comm, clat, tovh, flash
+                    r.icL = q0.x; r.icA = q0.y; r.icE = q1.x; r.imL = q1.y; r.imA = q2.x; r.imE = q2.y;
+                    r.inv_comm = q3.x; r.clat = q3.y; r.tovh = q4.x; r.flash = q4.y;
+                    const double t_pre = eval_stage<TIME_SUM>(tb_pre, u, r, Nd, lf);
+                    const double t_dec = n > 0 ? eval_stage<TIME_SUM>(tb_dec, u, r, Nd, lf) : 0.0;
+                    const u32 ci = e.hf * s.n_t + tpos;
+                    ttft = t_pre;
+                    latency = t_pre + t_dec;
+                    cost_hr = __ldg(s.cost_hr + ci);
+                    if (n > 0) {
+                        tpot = t_dec / (double)n;
+                        thr = cvt((u64)b * n) / t_dec;
+                        cost_tok = __ldg(s.cost_sec + ci) / thr;
+                    } else {
+                        tpot = 0.0; thr = 0.0; cost_tok = inf;
+                    }
+                    n_iters = 1 + (u64)n;
+                    n_req_iters = (u64)b * (1 + (u64)n);
+                }
+                // the four lanes of a pair write the whole foursome as soon as one of its configs fits
+                if ((vote >> (lane & ~3u)) & 0xFu) {
+                    const u64 j = j0 + (u64)e.hf * stride_hf;
+                    if (o.latency) __stcs(o.latency + j, latency);
+                    if (o.ttft) __stcs(o.ttft + j, ttft);
+                    if (o.ttft_p50) __stcs(o.ttft_p50 + j, ttft);
+                    if (o.ttft_p99) __stcs(o.ttft_p99 + j, ttft);
+                    if (o.tpot) __stcs(o.tpot + j, tpot);
+                    if (o.thr_decode) __stcs(o.thr_decode + j, thr);
+                    if (o.cost_per_hr) __stcs(o.cost_per_hr + j, cost_hr);
+                    if (o.cost_per_token) __stcs(o.cost_per_token + j, cost_tok);
+                    if (o.n_iters) __stcs(o.n_iters + j, n_iters);
+                    if (o.n_req_iters) __stcs(o.n_req_iters + j, n_req_iters);
+                }
             }
-            built = true;
+            p0 = e0.seg_end;
         }
-        if (fits) {
-            const DRate &rt = s.rates[e.hf];
-            const double lf = log2_rule_factor(t, tp_model);
-            const double Nd = (double)m.N;
-            const double t_pre = eval_phase<TIME_SUM>(kp, rt, Nd, lf);
-            const double t_dec = n > 0 ? eval_phase<TIME_SUM>(kd, rt, Nd, lf) : 0.0;
-            const u32 ci = e.hf * s.n_t + tpos;
-            out.ttft = t_pre;
-            out.latency = t_pre + t_dec;
-            out.cost_hr = __ldg(s.cost_hr + ci);
-            if (n > 0) {
-                out.tpot = t_dec / (double)n;
-                out.thr = cvt((u64)b * n) / t_dec;
-                out.cost_tok = __ldg(s.cost_sec + ci) / out.thr;
-            } else {
-                out.tpot = 0.0; out.thr = 0.0; out.cost_tok = inf;
-            }
-            out.n_iters = 1 + (u64)n;
-            out.n_req_iters = (u64)b * (1 + (u64)n);
-        }
-        // the whole foursome is written here as soon as one of its configs fits
-        if ((vote >> (lane & ~3u)) & 0xFu) {
-            const u64 j = j0 + (u64)e.hf * stride_hf;
-            if (o.latency) __stcs(o.latency + j, out.latency);
-            if (o.ttft) __stcs(o.ttft + j, out.ttft);
-            if (o.ttft_p50) __stcs(o.ttft_p50 + j, out.ttft);
-            if (o.ttft_p99) __stcs(o.ttft_p99 + j, out.ttft);
-            if (o.tpot) __stcs(o.tpot + j, out.tpot);
-            if (o.thr_decode) __stcs(o.thr_decode + j, out.thr);
-            if (o.cost_per_hr) __stcs(o.cost_per_hr + j, out.cost_hr);
-            if (o.cost_per_token) __stcs(o.cost_per_token + j, out.cost_tok);
-            if (o.n_iters) __stcs(o.n_iters + j, out.n_iters);
-            if (o.n_req_iters) __stcs(o.n_req_iters + j, out.n_req_iters);
-        }
-        p++;
     }
-  }
     // the grid must not be complete before the memory kernel is: whatever follows in the stream
     // waits for this one only
     cf_dep_wait();
@@ -295,19 +358,15 @@ static int launch_split(const DSpace &s, int tp_model, const guide_outputs &o, c
     GUIDE_CUDA(cudaMemsetAsync(ticket, 0, 4, st));           // the model kernel's work counter
     k_closed_form_memory<<<mem_grid, MEM_THREADS, 0, st>>>(s, o, co, tiles);
     GUIDE_CUDA(cudaGetLastError());
-    // chunks of the pair walk: 16 pairs, so that a point's stage tables serve many configs while
-    // the longest item stays short next to the whole launch
-    const u32 groups = (n_tl + MODEL_THREADS - 1) / MODEL_THREADS;
-    const u32 chunk = std::min<u32>(16, n_hf);
-    const u32 n_chunks = (n_hf + chunk - 1) / chunk;
-    if ((u64)s.n_m * s.n_b * groups * n_chunks > 0x7FFFFFFFull) return fail(GUIDE_ERR_UNSUPPORTED, "space too large for one launch");
+    const u32 n_chunks = (n_hf + MODEL_CHUNK - 1) / MODEL_CHUNK;
+    if ((u64)s.n_m * s.n_b * (n_tl / 4) * n_chunks > 0x7FFFFFFFull) return fail(GUIDE_ERR_UNSUPPORTED, "space too large for one launch");
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((u32)num_sms() * 8); cfg.blockDim = dim3(MODEL_THREADS); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cfg.gridDim = dim3((u32)num_sms() * MODEL_BLOCKS_PER_SM); cfg.blockDim = dim3(MODEL_THREADS); cfg.dynamicSmemBytes = 0; cfg.stream = st;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
-    GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_closed_form_model<TIME_SUM>, s, tp_model, o, groups, chunk, n_chunks, ticket));
+    GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_closed_form_model<TIME_SUM>, s, tp_model, o, n_chunks, ticket));
     return GUIDE_OK;
 }
 

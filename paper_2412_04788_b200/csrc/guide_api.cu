@@ -100,7 +100,7 @@ static int check_trace_overflow(const guide_space &s, const guide_trace &t) {
 // Derived per-model quantities and the reciprocal rates of every hardware x framework pair.
 __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *gh, u32 n_h, const guide_fw *gf,
                                u32 n_f, const u32 *tp, u32 n_t, DModel *dm, DRate *dr, double *cost_hr,
-                               double *cost_sec, ulonglong2 *hfmem) {
+                               double *cost_sec, ulonglong2 *hfmem, double *rate10) {
     const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n_m) {
         const guide_model m = gm[i];
@@ -132,6 +132,9 @@ __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *g
         r.kv_block = f.kv_block;
         dr[i] = r;
         hfmem[i] = make_ulonglong2(r.usable, (u64)r.kv_block);
+        double *q = rate10 + (size_t)i * 10;
+        for (int k = 0; k < 3; k++) { q[k] = r.inv_c[k]; q[3 + k] = r.inv_m[k]; }
+        q[6] = r.inv_comm; q[7] = r.clat; q[8] = r.tovh; q[9] = r.flash ? 1.0 : 0.0;
         for (u32 k = 0; k < n_t; k++) {
             const double c = h.price_per_hr * (double)tp[k];
             cost_hr[i * n_t + k] = c;
@@ -220,7 +223,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
                  o_ch = take(n_h * n_f * s->tp.size() * 8), o_cs = take(n_h * n_f * s->tp.size() * 8),
                  o_hm = take(n_h * n_f * 16), o_hs = take(n_h * n_f * sizeof(HfSorted)),
                  o_po = take(std::max<size_t>(n_m * (s->tp.size() * s->pairs.size() / 4), 1) * 4),
-                 o_tk = take(TICKET_SLOTS * 128);
+                 o_tk = take(TICKET_SLOTS * 128), o_r10 = take(n_h * n_f * 80);
     char *blob = nullptr;
     GUIDE_CUDA(cudaMalloc(&blob, off));
     cudaError_t e = cudaSuccess;
@@ -245,7 +248,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
                                                  (const u32 *)(blob + o_t), (u32)s->tp.size(),
                                                  (DModel *)(blob + o_dm), (DRate *)(blob + o_dr),
                                                  (double *)(blob + o_ch), (double *)(blob + o_cs),
-                                                 (ulonglong2 *)(blob + o_hm));
+                                                 (ulonglong2 *)(blob + o_hm), (double *)(blob + o_r10));
         e = cudaGetLastError();
         if (e == cudaSuccess) e = cudaStreamSynchronize(0);
     }
@@ -261,6 +264,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
     d.view.cost_hr = (const double *)(blob + o_ch);
     d.view.cost_sec = (const double *)(blob + o_cs);
     d.view.hfmem = (const ulonglong2 *)(blob + o_hm);
+    d.view.rate10 = (const double *)(blob + o_r10);
     d.view.hf_sorted = (const HfSorted *)(blob + o_hs);
     d.view.plane_order = (const u32 *)(blob + o_po);
     d.view.n_m = (u32)n_m; d.view.n_h = (u32)n_h; d.view.n_f = (u32)n_f;

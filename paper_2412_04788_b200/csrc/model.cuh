@@ -50,6 +50,7 @@ struct DSpace {
     const double *cost_hr;       // [n_h * n_f][n_t]: price x TP degree
     const double *cost_sec;      // [n_h * n_f][n_t]: (price x TP degree) / 3600
     const ulonglong2 *hfmem;     // [n_h * n_f]: x = usable bytes, y = KV block size (what the memory check reads)
+    const double *rate10;        // [n_h * n_f][10]: inv_c[3], inv_m[3], inv_comm, clat, tovh, flash (0.0 or 1.0); 16-byte aligned rows
     // Orders that only steer which thread does what (any permutation gives the same results):
     const HfSorted *hf_sorted;   // [n_h * n_f]: the pairs grouped by KV block size, largest usable memory first
     const u32 *plane_order;      // [n_m][n_t * n_l / 4]: foursomes of the (TP, length) plane by growing memory need
