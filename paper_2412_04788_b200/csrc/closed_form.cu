@@ -147,17 +147,19 @@ __global__ void __launch_bounds__(MEM_THREADS) k_closed_form_memory(DSpace s, gu
     }
 }
 
-// Stage table of one point in shared memory: twelve (x, y) entries per stage, interleaved over
-// the four points of a foursome so that the lanes of a warp read neighbouring words.
-//   0 (F1,B1) 1 (F2,B2) 2 (F3,B3) 3 (F5,B5) 4 (F6,B6) 5 (F7,B7) 6 (F8,B8) 7 (F9,B9) 8 (B9x,F10)
-//   9 (B10x,F13) 10 (B13,hops) 11 (cbytes,Rd)
-typedef double2 StageTab[12][4];
+// Stage table of one point in shared memory: the 24 entries of a TaskTab, interleaved over the
+// four points of a foursome so that the lanes of a warp read neighbouring 8-byte words (a 64-bit
+// shared load of a warp costs two wavefronts, a 128-bit one four, whatever the lanes share).
+typedef double StageTab[24][4];
+enum { E_F1, E_B1, E_F2, E_B2, E_F3, E_B3, E_F5, E_B5, E_F6, E_B6, E_F7, E_B7, E_F8, E_B8, E_F9, E_B9, E_B9X, E_F10, E_B10X,
+       E_F13, E_B13, E_HOPS, E_CBYTES, E_RD };
 
 __device__ __forceinline__ void put_stage(StageTab &tb, u32 u, const TaskTab &k) {
-    tb[0][u] = make_double2(k.F1, k.B1); tb[1][u] = make_double2(k.F2, k.B2); tb[2][u] = make_double2(k.F3, k.B3);
-    tb[3][u] = make_double2(k.F5, k.B5); tb[4][u] = make_double2(k.F6, k.B6); tb[5][u] = make_double2(k.F7, k.B7);
-    tb[6][u] = make_double2(k.F8, k.B8); tb[7][u] = make_double2(k.F9, k.B9); tb[8][u] = make_double2(k.B9x, k.F10);
-    tb[9][u] = make_double2(k.B10x, k.F13); tb[10][u] = make_double2(k.B13, k.hops); tb[11][u] = make_double2(k.cbytes, k.Rd);
+    tb[E_F1][u] = k.F1; tb[E_B1][u] = k.B1; tb[E_F2][u] = k.F2; tb[E_B2][u] = k.B2; tb[E_F3][u] = k.F3; tb[E_B3][u] = k.B3;
+    tb[E_F5][u] = k.F5; tb[E_B5][u] = k.B5; tb[E_F6][u] = k.F6; tb[E_B6][u] = k.B6; tb[E_F7][u] = k.F7; tb[E_B7][u] = k.B7;
+    tb[E_F8][u] = k.F8; tb[E_B8][u] = k.B8; tb[E_F9][u] = k.F9; tb[E_B9][u] = k.B9; tb[E_B9X][u] = k.B9x; tb[E_F10][u] = k.F10;
+    tb[E_B10X][u] = k.B10x; tb[E_F13][u] = k.F13; tb[E_B13][u] = k.B13; tb[E_HOPS][u] = k.hops; tb[E_CBYTES][u] = k.cbytes;
+    tb[E_RD][u] = k.Rd;
 }
 
 // Both stage tables of one point, written to shared memory.  Kept out of line: it runs once per
@@ -184,26 +186,24 @@ struct RateRegs { double icL, icA, icE, imL, imA, imE, inv_comm, clat, tovh, fla
 // eval_phase of model.cuh, operation for operation, with the task entries read from a StageTab
 template <int TIME_SUM>
 __device__ __forceinline__ double eval_stage(const StageTab &tb, u32 u, const RateRegs &r, double Nd, double log2_factor) {
-    const double2 e1 = tb[0][u], e2 = tb[1][u], e3 = tb[2][u], e5 = tb[3][u];
-    const double t2 = task_time<TIME_SUM>(e2.x, e2.y, r.icL, r.imL);
-    double sfix = task_time<TIME_SUM>(e1.x, e1.y, r.icE, r.imE);
+    const double t2 = task_time<TIME_SUM>(tb[E_F2][u], tb[E_B2][u], r.icL, r.imL);
+    double sfix = task_time<TIME_SUM>(tb[E_F1][u], tb[E_B1][u], r.icE, r.imE);
     sfix = sfix + t2;
-    sfix = sfix + task_time<TIME_SUM>(e3.x, e3.y, r.icL, r.imL);
+    sfix = sfix + task_time<TIME_SUM>(tb[E_F3][u], tb[E_B3][u], r.icL, r.imL);
     sfix = sfix + t2;
-    sfix = sfix + task_time<TIME_SUM>(e5.x, e5.y, r.icE, r.imE);
-    const double2 e6 = tb[4][u], e7 = tb[5][u], e8 = tb[6][u];
-    sfix = sfix + task_time<TIME_SUM>(e6.x, e6.y, r.icL, r.imL);
-    sfix = sfix + task_time<TIME_SUM>(e7.x, e7.y, r.icE, r.imE);
-    sfix = sfix + task_time<TIME_SUM>(e8.x, e8.y, r.icL, r.imL);
-    const double2 e9 = tb[7][u], e9x = tb[8][u], e10x = tb[9][u];
-    const bool flash = r.flash != 0.0;
-    const double t9 = task_time<TIME_SUM>(e9.x, flash ? e9.y : e9x.x, r.icA, r.imA);
-    const double t10 = task_time<TIME_SUM>(e9x.y, flash ? 0.0 : e10x.x, r.icA, r.imA);
+    sfix = sfix + task_time<TIME_SUM>(tb[E_F5][u], tb[E_B5][u], r.icE, r.imE);
+    sfix = sfix + task_time<TIME_SUM>(tb[E_F6][u], tb[E_B6][u], r.icL, r.imL);
+    sfix = sfix + task_time<TIME_SUM>(tb[E_F7][u], tb[E_B7][u], r.icE, r.imE);
+    sfix = sfix + task_time<TIME_SUM>(tb[E_F8][u], tb[E_B8][u], r.icL, r.imL);
+    // without FlashAttention the score matrix adds to the bytes of qk / sv and gives softmax its own
+    const double b9 = r.flash != 0.0 ? tb[E_B9][u] : tb[E_B9X][u];
+    const double b10 = r.flash != 0.0 ? 0.0 : tb[E_B10X][u];
+    const double t9 = task_time<TIME_SUM>(tb[E_F9][u], b9, r.icA, r.imA);
+    const double t10 = task_time<TIME_SUM>(tb[E_F10][u], b10, r.icA, r.imA);
     const double satt = (t9 + t10) + t9;
-    const double2 e13 = tb[10][u], ec = tb[11][u];
-    const double scomm = 2.0 * (e13.y * r.clat + ec.x * r.inv_comm);
-    const double thead = task_time<TIME_SUM>(e10x.y, e13.x, r.icL, r.imL);
-    return combine_phase(sfix, satt, scomm, thead, ec.y, Nd, r.tovh, log2_factor);
+    const double scomm = 2.0 * (tb[E_HOPS][u] * r.clat + tb[E_CBYTES][u] * r.inv_comm);
+    const double thead = task_time<TIME_SUM>(tb[E_F13][u], tb[E_B13][u], r.icL, r.imL);
+    return combine_phase(sfix, satt, scomm, thead, tb[E_RD][u], Nd, r.tovh, log2_factor);
 }
 
 // Performance model for the configs that fit.  A warp takes one foursome of the plane for one

@@ -79,6 +79,47 @@ def test_null_outputs_are_skipped():
     assert np.array_equal(out["latency"].cpu().numpy(), want["latency"])
 
 
+def test_split_kernels_mixed_block_sizes_and_ragged_plane():
+    """A whole space of 216,000 configs goes through the memory kernel + model kernel pair: three KV
+    block sizes (unpaged, 16, 24) so the sorted pair walk has three segments, a (TP, length) plane
+    of 60 positions that fills neither a 64-wide group nor a 256-wide tile, small memories so that
+    most foursomes are mixed."""
+    hw, mem = I.seeded_hw(11, 40, mem_choices=[16, 24, 48, 80])
+    fw_f, fw_i = I.seeded_fw(12, 3, kv_block=16)
+    fw_i[0, 1] = 1
+    fw_i[2, 1] = 24
+    sp = I._space(I.models_from_shapes(I.SHAPES_8[0:6]), hw, mem, fw_f, fw_i, [1, 3, 17, 64, 200], [1, 2, 4, 8, 16],
+                  I.pairs_grid([64, 700, 3000], [1, 2, 130, 4000]))
+    want = oracle.simulate(sp)
+    assert len(want["status"]) == 216000
+    for tm, tpm in ((0, 0), (1, 1)):
+        want = oracle.simulate(sp, time_model=tm, tp_model=tpm)
+        got, *_ = run_simulate(sp, time_model=tm, tp_model=tpm)
+        assert_parity(got, want)
+        assert sum(bit_mismatches(got, want).values()) == 0
+    assert (want["status"] == 0).any() and (want["status"] != 0).any()
+
+
+def test_split_kernels_output_subsets():
+    """Whole-space calls with only some output arrays: each kernel of the pair must skip the rest."""
+    import torch
+    w = I.workload(2, scale=0.125)
+    want = oracle.simulate(w["space"])
+    sp = guide.Space(w["space"])
+    n = sp.size
+    assert n >= 65536
+    for fields in (("latency",), ("status", "bmax"), ("thr_decode", "cost_per_token", "n_iters"), ("ttft_p99", "status", "n_req_iters")):
+        out = guide.alloc_outputs(n, fields=fields)
+        for t in out.values():
+            t.fill_(7)
+        guide.guide_simulate(sp, None, out)
+        torch.cuda.synchronize()
+        for f in fields:
+            g = out[f].cpu().numpy()
+            x = want["ttft"] if f == "ttft_p99" else want[f]
+            assert np.array_equal(g.view(np.uint8), x.view(np.uint8)), (fields, f)
+
+
 def test_full_size_grid_983040():
     """Workload 2 at full size in the launch shape the benchmark times; compared in full."""
     w = I.workload(2)

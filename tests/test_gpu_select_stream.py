@@ -168,6 +168,8 @@ def test_workload5_full_size_materialised_selection():
     w = I.workload(5)
     want = oracle.simulate(w["space"])
     got, out_dev, sp5, _ = run_simulate(w["space"])
+    for f in ("status", "bmax", "n_iters", "n_req_iters") + tuple(guide.F64_OUTPUTS):     # the whole sweep, bit for bit
+        assert np.array_equal(got[f].view(np.uint8), want[f].view(np.uint8)), f
     cons, k, key = w["constraints"], w["topk"]["k"], w["topk"]["key"]
     idx, val, cnt = run_topk(sp5, out_dev, cons, key, k)
     w_idx, w_val, w_cnt = oracle.select_topk(want, cons, key, k)
