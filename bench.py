@@ -4,8 +4,10 @@
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--extras LIST]
 
 A step is one pass of the whole closed-form path over the 16,777,216-config sweep (workload 5):
-guide_simulate (memory check, task list, roofline, metrics -> 6 fp64 arrays + mask + B_max),
-guide_select_topk (constraint filter + top-64 by cost per token) and guide_pareto (latency vs $/h),
+guide_simulate (memory check, task list, roofline, metrics -> 6 fp64 arrays + mask + B_max; a
+bandwidth-bound memory kernel and a model kernel for the configs that fit, side by side),
+guide_select_topk (constraint filter + top-64 by cost per token) and guide_pareto (latency vs $/h;
+both: a sampled bound, one filter pass at memory speed, an exact finish),
 with the space tables already resident on the device.  `value` is configs per second over the K
 timed steps; the 0.89 GB of outputs a step writes and reads back exceed L2 several times over, so
 no flush is needed between steps.  The trace-driven workloads (1, 3, 4), the 983,040-config grid
@@ -35,9 +37,10 @@ if ROOT not in sys.path:
 import numpy as np
 
 BYTES_SIM = 6 * 8 + 1 + 4          # six fp64 metrics + status + bmax written per config
-# dram__bytes_read.sum + dram__bytes_write.sum of one k_closed_form_tiled launch on the full workload 5
-# (profiles/k_closed_form_tiled_c5.md); only meaningful for that size and that kernel version
-K1_TRAFFIC_C5 = 857_484_032 + 393_472
+# dram__bytes_read.sum + dram__bytes_write.sum of one guide_simulate call on the full workload 5: the
+# k_closed_form_memory and k_closed_form_model launches together (profiles/k_closed_form_split_c5.md);
+# only meaningful for that size and those kernel versions
+K1_TRAFFIC_C5 = 644_200_000 + 151_100_000 + 1_000_000
 SIM_FIELDS = ("latency", "ttft", "tpot", "thr_decode", "cost_per_hr", "cost_per_token", "status", "bmax")
 TRACE_FIELDS = ("latency", "ttft", "ttft_p50", "ttft_p99", "tpot", "thr_decode", "cost_per_hr", "cost_per_token",
                 "status", "bmax", "n_iters", "n_req_iters")
@@ -243,7 +246,7 @@ def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full, fraction
                             "materialised_configs_per_s": n / (t_sim + t_km + t_pm) * 1e3,
                             "simulate_write_gbs": BYTES_SIM * n / t_sim / 1e6,
                             "simulate_frac_of_hbm": BYTES_SIM * n / t_sim / 1e6 / hbm_peak,
-                            "kernel_launches": 1 + 2 * 2 + 2 * 2}
+                            "kernel_launches": 2 + 2 + 2 + 6 + 4}
             del p
         torch.cuda.empty_cache()
     return res
@@ -379,9 +382,9 @@ def run_ours(args):
     cons_arrays = {arr for name, arr in bounded.items() if name in cons}
     bytes_topk = 1 + 8 * len(cons_arrays | {key})
     bytes_pareto = 1 + 8 * len(cons_arrays | {"latency", "cost_per_hr"})
-    per = {"guide_simulate (k_closed_form_tiled)": (t_sim / args.steps, BYTES_SIM),
-           "guide_select_topk (k_topk_scan + k_topk_merge)": (t_topk / args.steps, bytes_topk),
-           "guide_pareto (k_pareto_scan)": (t_par / args.steps, bytes_pareto)}
+    per = {"guide_simulate (k_closed_form_memory + k_closed_form_model)": (t_sim / args.steps, BYTES_SIM),
+           "guide_select_topk (k_topk_sample + k_topk_refine + k_topk_filter + k_topk_rank)": (t_topk / args.steps, bytes_topk),
+           "guide_pareto (k_pareto_sample + k_pareto_filter + k_pareto_rank)": (t_par / args.steps, bytes_pareto)}
     dom = max(per, key=lambda name: per[name][0])
     dom_ms, dom_bytes = per[dom]
     achieved = dom_bytes * n_local / (dom_ms * 1e-3) / 1e9
@@ -390,6 +393,7 @@ def run_ours(args):
                 "traffic": K1_TRAFFIC_C5 if (dom.startswith("guide_simulate") and n_local == 16777216) else None,
                 "peak_kind": f"of {peak_kind}",
                 "bytes_per_config": dom_bytes,
+                "per_call_frac_of_hbm": {name: v[1] * n_local / (v[0] * 1e-3) / 1e9 / hbm_peak for name, v in per.items()},
                 "per_kernel_ms": {name: v[0] for name, v in per.items()},
                 "per_kernel_gbs": {name: v[1] * n_local / (v[0] * 1e-3) / 1e9 for name, v in per.items()}}
 
@@ -411,8 +415,11 @@ def run_ours(args):
         which = [int(x) for x in args.extras.split(",") if x]
         extras = extra_workloads(guide, torch, inputs, which, flush, hbm_peak, args.full, args.trace_fraction)
 
-    # simulate, top-k scan + merge, Pareto per-warp kernel + its gated general kernel (+ merge of gathered lists)
-    launches_per_step = 5 + (2 if world > 1 else 0)
+    # simulate: memory + model kernel; top-k: sample, refine, filter, rank and the two gated fallback
+    # kernels (scan, merge: they return at once); Pareto: sample, filter, rank and the gated general
+    # kernel; with several ranks the merge of the gathered lists (scan + merge, too short for the
+    # streaming path)
+    launches_per_step = 2 + 6 + 4 + (2 if world > 1 else 0)
     line = {"metric": "configs/sec", "value": value, "unit": "configs/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
