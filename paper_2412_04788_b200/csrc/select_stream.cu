@@ -43,8 +43,10 @@ static constexpr u32 SAMPLE_BATCH = 4;          // rows a warp has in flight at 
 static constexpr u32 TK_SAMPLE_BLOCKS = 256;    // block minima of the coarse bound (must stay >= 2 x STREAM_TOPK_MAX_K)
 static constexpr u32 TK_SAMPLE_ROWS = 8192;     // rows the sample aims at
 static constexpr u32 TK_SAMPLE_MAX_R = 32;
-static constexpr u32 TK_SKEYS_CAP = 2048;       // sample pairs within the coarse bound
-static constexpr u32 TK_CAND_CAP = 8192;        // survivors the workspace can hold
+static constexpr u32 TK_SKEYS_CAP = 8192;       // sample pairs within the coarse bound the workspace holds
+static constexpr u32 TK_SKEYS_SMEM = 2048;      // ... and how many the last block of the refinement sorts at once
+static constexpr u32 TK_CAND_CAP = 16384;       // survivors the workspace can hold
+static constexpr u32 TK_CAND_SMEM = 8192;       // ... of which the rank kernel stages this many in shared memory
 
 static constexpr u32 PA_SAMPLE_BLOCKS = 64;
 static constexpr u32 PA_ROWS_PER_WARP = 8;
@@ -52,7 +54,7 @@ static constexpr u32 PA_SAMPLE_ROWS = PA_SAMPLE_BLOCKS * (SEL_THREADS / 32) * PA
 static constexpr u32 PA_LOCAL_CAP = 1024;       // per-block list of sample points that survive the two seeds
 static constexpr u32 PA_PER_BLOCK = 4;          // front points a sample block hands on
 static constexpr u32 PA_KILLERS = PA_SAMPLE_BLOCKS * PA_PER_BLOCK;   // 256
-static constexpr u32 PA_SURV_CAP = 4096;        // survivors the workspace can hold
+static constexpr u32 PA_SURV_CAP = 8192;        // survivors the workspace can hold
 
 struct P2 { u64 x, y; };
 
@@ -245,12 +247,13 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_sample(Src<NA> s, Sample s
 
 // Refinement: the sample's pairs within the coarse bound are gathered (few: the coarse bound is at
 // worst the k-th best row of the sample) and the last block replaces the bound by their k-th
-// smallest, the exact k-th pair of the sample.  If they do not fit, the coarse bound stays.
+// smallest, the exact k-th pair of the sample (of the stored part of it, if they do not all fit).
 template <int NA>
 __global__ void __launch_bounds__(SEL_THREADS) k_topk_refine(Src<NA> s, Sample sm, u64 first, u32 k, u32 *header,
                                                              ulonglong2 *spairs) {
-    constexpr u32 PER = TK_SKEYS_CAP / SEL_THREADS;
-    __shared__ ulonglong2 sl[TK_SKEYS_CAP];
+    constexpr u32 PER = TK_SKEYS_SMEM / SEL_THREADS;
+    __shared__ ulonglong2 sl[TK_SKEYS_SMEM];
+    __shared__ u32 s_n;
     __shared__ u32 last;
     grid_dep_launch();
     grid_dep_wait();
@@ -283,23 +286,64 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_refine(Src<NA> s, Sample s
     __syncthreads();
     if (!last) return;
     __threadfence();
-    const u32 n = __ldcg(header + TK_SAMPLED);
-    if (n < k || n > TK_SKEYS_CAP) return;       // below k only when the coarse bound is all-ones; too many: it stays
-    const u32 P = n <= 2 * SEL_THREADS ? n : next_pow2(n);
+    // More pairs than the workspace holds: the ones that were stored are still real configs within
+    // the coarse bound, so their k-th smallest is a valid (if looser) bound.  Fewer than k happens
+    // only when the coarse bound is all-ones: it stays.
+    const u32 n = min(__ldcg(header + TK_SAMPLED), TK_SKEYS_CAP);
+    if (n < k) return;
+    auto pair_before = [](const ulonglong2 &a, const ulonglong2 &b) { return a.x < b.x || (a.x == b.x && a.y < b.y); };
+    u64 *bound = reinterpret_cast<u64 *>(header + TK_BOUND);
+    if (n <= 2 * SEL_THREADS) {                      // a short list: counting is quicker than sorting
+#pragma unroll
+        for (u32 u = 0; u < 2; u++) {
+            const u32 i = threadIdx.x + u * blockDim.x;
+            if (i < n) sl[i] = __ldcg(spairs + i);
+        }
+        __syncthreads();
+        write_kth_pair<2>(sl, n, k, header);
+        return;
+    }
+    // Longer lists are sorted in shared memory, at most TK_SKEYS_SMEM pairs at a time.  A list above
+    // that goes in two steps: every step-th pair first, whose k-th smallest bounds the k-th of the
+    // whole list from above; then all pairs within that bound (about k x step of them).
+    const u32 step = (n + TK_SKEYS_SMEM - 1) / TK_SKEYS_SMEM;
+    const u32 m = (n + step - 1) / step;
+    u32 P = next_pow2(m);
 #pragma unroll
     for (u32 u = 0; u < PER; u++) {
         const u32 i = threadIdx.x + u * blockDim.x;
         ulonglong2 e; e.x = KEY_MAX; e.y = KEY_MAX;
-        if (i < n) e = __ldcg(spairs + i);
+        if (i < m) e = __ldcg(spairs + (size_t)i * step);
         if (i < P) sl[i] = e;
     }
     __syncthreads();
-    if (n <= 2 * SEL_THREADS) { write_kth_pair<2>(sl, n, k, header); return; }     // a short list: counting is quicker
-    block_bitonic_sort(sl, P, [](const ulonglong2 &a, const ulonglong2 &b) { return a.x < b.x || (a.x == b.x && a.y < b.y); });
-    if (threadIdx.x == 0) {
-        u64 *b = reinterpret_cast<u64 *>(header + TK_BOUND);
-        b[0] = sl[k - 1].x; b[1] = sl[k - 1].y;
+    block_bitonic_sort(sl, P, pair_before);
+    const ulonglong2 b1 = sl[k - 1];                 // m >= k: n > 512 >= 2k and step <= 4
+    __syncthreads();
+    if (step == 1) {
+        if (threadIdx.x == 0) { bound[0] = b1.x; bound[1] = b1.y; }
+        return;
     }
+    if (threadIdx.x == 0) s_n = 0;
+    __syncthreads();
+    for (u32 i = threadIdx.x; i < n; i += blockDim.x) {
+        const ulonglong2 e = __ldcg(spairs + i);
+        if (!pair_before(b1, e)) {                   // e <= b1
+            const u32 pos = atomicAdd(&s_n, 1u);
+            if (pos < TK_SKEYS_SMEM) sl[pos] = e;
+        }
+    }
+    __syncthreads();
+    const u32 c = s_n;                               // >= k: the k pairs that put b1 at rank k-1 of its subset are among them
+    if (c > TK_SKEYS_SMEM) {                         // does not fit (heavy ties): the first bound stands
+        if (threadIdx.x == 0) { bound[0] = b1.x; bound[1] = b1.y; }
+        return;
+    }
+    P = next_pow2(c);
+    for (u32 i = c + threadIdx.x; i < P; i += blockDim.x) { sl[i].x = KEY_MAX; sl[i].y = KEY_MAX; }
+    __syncthreads();
+    block_bitonic_sort(sl, P, pair_before);
+    if (threadIdx.x == 0) { bound[0] = sl[k - 1].x; bound[1] = sl[k - 1].y; }
 }
 
 __device__ __forceinline__ void topk_keep(u64 key, u64 idx, u32 *header, KI *cand) {
@@ -369,14 +413,19 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_rank(u32 *header, const KI
     const u32 n_warps = gridDim.x * (blockDim.x >> 5);
     if (blockIdx.x * (blockDim.x >> 5) >= n) return;         // no candidate for this block
     const ulonglong2 *list = reinterpret_cast<const ulonglong2 *>(cand);
-    for (u32 i = threadIdx.x; i < n; i += blockDim.x) sl[i] = __ldcg(list + i);
+    const u32 ns = min(n, TK_CAND_SMEM);             // a longer list is read past this point straight from memory
+    for (u32 i = threadIdx.x; i < ns; i += blockDim.x) sl[i] = __ldcg(list + i);
     __syncthreads();
     const u32 lane = threadIdx.x & 31;
     for (u32 g = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); g < n; g += n_warps) {
-        const ulonglong2 me = sl[g];
+        const ulonglong2 me = g < ns ? sl[g] : __ldcg(list + g);
         u32 ahead = 0;
-        for (u32 i = lane; i < n; i += 32) {
+        for (u32 i = lane; i < ns; i += 32) {
             const ulonglong2 o = sl[i];
+            ahead += (o.x < me.x || (o.x == me.x && o.y < me.y)) ? 1u : 0u;
+        }
+        for (u32 i = ns + lane; i < n; i += 32) {
+            const ulonglong2 o = __ldcg(list + i);
             ahead += (o.x < me.x || (o.x == me.x && o.y < me.y)) ? 1u : 0u;
         }
         for (int d = 16; d > 0; d >>= 1) ahead += __shfl_xor_sync(0xFFFFFFFFu, ahead, d);
@@ -643,23 +692,22 @@ __global__ void __launch_bounds__(SEL_THREADS) k_pareto_rank(u32 *header, const 
         if (blockIdx.x == 0 && threadIdx.x == 0) header[1] = 1;
         return;
     }
-    u64 *sx = reinterpret_cast<u64 *>(smem_raw), *sy = sx + n, *si = sy + n;
+    u64 *sx = reinterpret_cast<u64 *>(smem_raw), *sy = sx + n;      // x and y staged; the index is read only for equal points
     const u32 lane = threadIdx.x & 31;
     const u32 n_warps = gridDim.x * (blockDim.x >> 5);
+    const u64 *w = reinterpret_cast<const u64 *>(surv);
     if (blockIdx.x * (blockDim.x >> 5) < n) {               // this block has survivors to judge
-        const u64 *w = reinterpret_cast<const u64 *>(surv);
         for (u32 i = threadIdx.x; i < 3 * n; i += blockDim.x) {
-            const u64 val = __ldcg(w + i);
             const u32 e = i / 3, f = i % 3;
-            (f == 0 ? sx : f == 1 ? sy : si)[e] = val;
+            if (f < 2) (f == 0 ? sx : sy)[e] = __ldcg(w + i);
         }
         __syncthreads();
         for (u32 g = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); g < n; g += n_warps) {
-            const u64 mx = sx[g], my = sy[g], mi = si[g];
+            const u64 mx = sx[g], my = sy[g], mi = __ldcg(w + 3 * (size_t)g + 2);
             bool out = false;
             for (u32 i = lane; i < n; i += 32) {
                 const u64 ox = sx[i], oy = sy[i];
-                out |= dominates(ox, oy, mx, my) || (ox == mx && oy == my && si[i] < mi);
+                out |= dominates(ox, oy, mx, my) || (ox == mx && oy == my && __ldcg(w + 3 * (size_t)i + 2) < mi);
             }
             if (!__any_sync(0xFFFFFFFFu, out) && lane == 0) {
                 const u32 pos = atomicAdd(header + PH_FRONT, 1);   // pos < n <= PA_SURV_CAP
@@ -742,7 +790,7 @@ static int topk_stream_na(const Arr *arr, Range r, const guide_outputs &mat, u32
     GUIDE_CUDA(cudaGetLastError());
     GUIDE_CUDA(launch_dependent(k_topk_refine<NA>, TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st, s, sm, r.first, k, header, spairs));
     GUIDE_CUDA(launch_dependent(k_topk_filter<NA>, filter_grid(r.count), SEL_THREADS, 0, st, s, r, header, cand));
-    const size_t smem = (size_t)TK_CAND_CAP * sizeof(KI);
+    const size_t smem = (size_t)TK_CAND_SMEM * sizeof(KI);
     GUIDE_CUDA(cudaFuncSetAttribute(k_topk_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     GUIDE_CUDA(launch_dependent(k_topk_rank, num_sms(), SEL_THREADS, smem, st, header, (const KI *)cand, k, negate, idx_out,
                                 key_out, count_out));
@@ -780,7 +828,7 @@ static int pareto_stream_na(const Arr *arr, Range r, const guide_outputs &mat, u
     GUIDE_CUDA(cudaGetLastError());
     GUIDE_CUDA(launch_dependent(k_pareto_filter<NA>, filter_grid(r.count), SEL_THREADS, 0, st, s, r, header, (const P2 *)killers,
                                 surv));
-    const size_t smem = (size_t)PA_SURV_CAP * sizeof(P3);
+    const size_t smem = (size_t)PA_SURV_CAP * 16;
     GUIDE_CUDA(cudaFuncSetAttribute(k_pareto_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     GUIDE_CUDA(launch_dependent(k_pareto_rank, num_sms(), SEL_THREADS, smem, st, header, (const P3 *)surv, front, idx_out, cap,
                                 count_out));

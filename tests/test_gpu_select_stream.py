@@ -73,8 +73,8 @@ def test_topk_random_keys_bounds_and_ragged_lengths(sp):
 
 
 def test_topk_ties_on_the_key(sp):
-    """Every key equal: the bound excludes nothing, the survivor list overflows and the call is
-    redone by the accumulator kernels; the answer is the k lowest passing indices."""
+    """Every key equal: the key alone excludes nothing, the index half of the (key, index) bound
+    does; the answer is the k lowest passing indices."""
     n = 2 * N_MIN + 77
     host = synth(n, 5)
     host["cost_per_token"][:] = 0.25
