@@ -30,6 +30,8 @@
 #include <algorithm>
 #include <cmath>
 
+#include <cooperative_groups.h>
+
 #include "select.cuh"
 
 namespace guide {
@@ -344,6 +346,96 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_refine(Src<NA> s, Sample s
     __syncthreads();
     block_bitonic_sort(sl, P, pair_before);
     if (threadIdx.x == 0) { bound[0] = sl[k - 1].x; bound[1] = sl[k - 1].y; }
+}
+
+// The two kernels above as one cooperative launch: the same steps, with grid-wide barriers in place
+// of the kernel boundary and of the "last block" selections, which here are spread over the whole
+// grid (one warp ranks one pair).  A dependent chain of short latencies, so every hand-over it
+// saves counts.  Used when the device supports cooperative launches.
+template <int NA>
+__global__ void __launch_bounds__(SEL_THREADS) k_topk_bound(Src<NA> s, Sample sm, u64 first, u32 k, u32 *header,
+                                                            ulonglong2 *minima, ulonglong2 *spairs) {
+    namespace cg = cooperative_groups;
+    cg::grid_group grid = cg::this_grid();
+    __shared__ ulonglong2 sl[SEL_THREADS / 32];
+    grid_dep_launch();
+    const u32 lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = SEL_THREADS / 32;
+    const u32 gwarp = blockIdx.x * n_warps + warp, total_warps = gridDim.x * n_warps;
+    const u64 stride = (u64)gridDim.x * n_warps;
+    u64 *bound = reinterpret_cast<u64 *>(header + TK_BOUND);
+    // 1: block minima of the passing sample pairs
+    u64 bk = KEY_MAX, bi = KEY_MAX;
+    for (u64 c0 = (u64)warp * gridDim.x + blockIdx.x; c0 < sm.n_slots; c0 += SAMPLE_BATCH * stride) {
+        u32 st[SAMPLE_BATCH];
+        double2 v[SAMPLE_BATCH][NA];
+        u64 j[SAMPLE_BATCH];
+        load_batch(s, sm, c0, stride, lane, st, v, j);
+#pragma unroll
+        for (u32 u = 0; u < SAMPLE_BATCH; u++) {
+            bool ok0, ok1;
+            eval_pair(s, st[u], v[u], ok0, ok1);
+            if (j[u] != KEY_MAX && ok0) pair_min(bk, bi, metric_key(s.a[0], v[u][0].x), first + j[u]);
+            if (j[u] != KEY_MAX && ok1) pair_min(bk, bi, metric_key(s.a[0], v[u][0].y), first + j[u] + 1);
+        }
+    }
+    for (int d = 16; d > 0; d >>= 1)
+        pair_min(bk, bi, __shfl_xor_sync(0xFFFFFFFFu, bk, d), __shfl_xor_sync(0xFFFFFFFFu, bi, d));
+    if (lane == 0) { sl[warp].x = bk; sl[warp].y = bi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (u32 w = 1; w < n_warps; w++) pair_min(bk, bi, sl[w].x, sl[w].y);
+        ulonglong2 m; m.x = bk; m.y = bi;
+        minima[blockIdx.x] = m;
+    }
+    grid.sync();
+    // 2: coarse bound = k-th smallest block minimum (equal all-ones entries ordered by position)
+    if (gwarp < gridDim.x) {
+        const ulonglong2 me = __ldcg(minima + gwarp);
+        u32 ahead = 0;
+        for (u32 q = lane; q < gridDim.x; q += 32) {
+            const ulonglong2 o = __ldcg(minima + q);
+            ahead += (o.x < me.x || (o.x == me.x && (o.y < me.y || (o.y == me.y && q < gwarp)))) ? 1u : 0u;
+        }
+        for (int d = 16; d > 0; d >>= 1) ahead += __shfl_xor_sync(0xFFFFFFFFu, ahead, d);
+        if (lane == 0 && ahead == k - 1) { bound[0] = me.x; bound[1] = me.y; }
+    }
+    grid.sync();
+    // 3: the sample pairs within the coarse bound (the rows come from L2 this time)
+    const u64 bkey = __ldcg(bound), bidx = __ldcg(bound + 1);
+    for (u64 c0 = (u64)warp * gridDim.x + blockIdx.x; c0 < sm.n_slots; c0 += SAMPLE_BATCH * stride) {
+        u32 st[SAMPLE_BATCH];
+        double2 v[SAMPLE_BATCH][NA];
+        u64 j[SAMPLE_BATCH];
+        load_batch(s, sm, c0, stride, lane, st, v, j);
+#pragma unroll
+        for (u32 u = 0; u < SAMPLE_BATCH; u++) {
+            bool ok[2];
+            eval_pair(s, st[u], v[u], ok[0], ok[1]);
+            const u64 key[2] = {metric_key(s.a[0], v[u][0].x), metric_key(s.a[0], v[u][0].y)};
+#pragma unroll
+            for (u32 h = 0; h < 2; h++) {
+                if (j[u] != KEY_MAX && ok[h] && pair_le(key[h], first + j[u] + h, bkey, bidx)) {
+                    const u32 p = atomicAdd(header + TK_SAMPLED, 1);
+                    if (p < TK_SKEYS_CAP) { ulonglong2 e; e.x = key[h]; e.y = first + j[u] + h; spairs[p] = e; }
+                }
+            }
+        }
+    }
+    grid.sync();
+    // 4: their k-th smallest (of the stored ones, if they did not all fit: still a valid bound);
+    // fewer than k only when the coarse bound is all-ones, which then stays
+    const u32 n = min(__ldcg(header + TK_SAMPLED), TK_SKEYS_CAP);
+    if (n < k) return;
+    for (u32 g = gwarp; g < n; g += total_warps) {
+        const ulonglong2 me = __ldcg(spairs + g);
+        u32 ahead = 0;
+        for (u32 q = lane; q < n; q += 32) {
+            const ulonglong2 o = __ldcg(spairs + q);
+            ahead += (o.x < me.x || (o.x == me.x && o.y < me.y)) ? 1u : 0u;
+        }
+        for (int d = 16; d > 0; d >>= 1) ahead += __shfl_xor_sync(0xFFFFFFFFu, ahead, d);
+        if (lane == 0 && ahead == k - 1) { bound[0] = me.x; bound[1] = me.y; }
+    }
 }
 
 __device__ __forceinline__ void topk_keep(u64 key, u64 idx, u32 *header, KI *cand) {
@@ -774,6 +866,22 @@ static Sample make_sample(u64 n_rows, u32 want_rows, u32 max_r) {
     return sm;
 }
 
+// Can the bound kernel's grid (TK_SAMPLE_BLOCKS blocks of SEL_THREADS threads) be resident at once on
+// the current device, and does the device launch cooperatively?  Asked once per device.
+template <int NA>
+static bool cooperative_ok() {
+    static int cached[64] = {};                      // 0 unknown, 1 yes, 2 no
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (!cached[dev]) {
+        int coop = 0, per_sm = 0;
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_topk_bound<NA>, SEL_THREADS, 0);
+        cached[dev] = (coop && (u64)per_sm * num_sms() >= TK_SAMPLE_BLOCKS) ? 1 : 2;
+    }
+    return cached[dev] == 1;
+}
+
 template <int NA>
 static int topk_stream_na(const Arr *arr, Range r, const guide_outputs &mat, u32 k, int negate, u32 *header,
                           unsigned char *region, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st) {
@@ -786,9 +894,19 @@ static int topk_stream_na(const Arr *arr, Range r, const guide_outputs &mat, u32
     // the coarse bound needs every block to see rows: the walk covers the whole sample (all groups)
     Sample sm = make_sample(r.count / ROW, TK_SAMPLE_ROWS, TK_SAMPLE_MAX_R);
     sm.n_slots = sm.n_groups;
-    k_topk_sample<NA><<<TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st>>>(s, sm, r.first, k, header, minima);
-    GUIDE_CUDA(cudaGetLastError());
-    GUIDE_CUDA(launch_dependent(k_topk_refine<NA>, TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st, s, sm, r.first, k, header, spairs));
+    if (cooperative_ok<NA>()) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(TK_SAMPLE_BLOCKS); cfg.blockDim = dim3(SEL_THREADS); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeCooperative;
+        at[0].val.cooperative = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_topk_bound<NA>, s, sm, r.first, k, header, minima, spairs));
+    } else {
+        k_topk_sample<NA><<<TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st>>>(s, sm, r.first, k, header, minima);
+        GUIDE_CUDA(cudaGetLastError());
+        GUIDE_CUDA(launch_dependent(k_topk_refine<NA>, TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st, s, sm, r.first, k, header, spairs));
+    }
     GUIDE_CUDA(launch_dependent(k_topk_filter<NA>, filter_grid(r.count), SEL_THREADS, 0, st, s, r, header, cand));
     const size_t smem = (size_t)TK_CAND_SMEM * sizeof(KI);
     GUIDE_CUDA(cudaFuncSetAttribute(k_topk_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
