@@ -50,11 +50,11 @@ static constexpr u32 TK_SKEYS_SMEM = 2048;      // ... and how many the last blo
 static constexpr u32 TK_CAND_CAP = 16384;       // survivors the workspace can hold
 static constexpr u32 TK_CAND_SMEM = 8192;       // ... of which the rank kernel stages this many in shared memory
 
-static constexpr u32 PA_SAMPLE_BLOCKS = 64;
-static constexpr u32 PA_ROWS_PER_WARP = 8;
+static constexpr u32 PA_SAMPLE_BLOCKS = 128;
+static constexpr u32 PA_ROWS_PER_WARP = 4;
 static constexpr u32 PA_SAMPLE_ROWS = PA_SAMPLE_BLOCKS * (SEL_THREADS / 32) * PA_ROWS_PER_WARP;   // 4096
 static constexpr u32 PA_LOCAL_CAP = 1024;       // per-block list of sample points that survive the two seeds
-static constexpr u32 PA_PER_BLOCK = 4;          // front points a sample block hands on
+static constexpr u32 PA_PER_BLOCK = 2;          // front points a sample block hands on
 static constexpr u32 PA_KILLERS = PA_SAMPLE_BLOCKS * PA_PER_BLOCK;   // 256
 static constexpr u32 PA_SURV_CAP = 8192;        // survivors the workspace can hold
 
@@ -82,9 +82,9 @@ size_t topk_stream_bytes() { return TK_OFF_CAND + (size_t)TK_CAND_CAP * sizeof(K
 //                        | P3 surv[PA_SURV_CAP] | KI front[PA_SURV_CAP]
 static constexpr size_t PA_OFF_KILLERS = (size_t)PA_KILLERS * sizeof(P2);
 static constexpr size_t PA_OFF_LOCAL_N = 2 * PA_OFF_KILLERS;
-static constexpr size_t PA_OFF_SURV = PA_OFF_LOCAL_N + 256;
+static constexpr size_t PA_OFF_SURV = PA_OFF_LOCAL_N + 512;
 static constexpr size_t PA_OFF_FRONT = PA_OFF_SURV + (size_t)PA_SURV_CAP * sizeof(P3);
-static_assert(PA_SAMPLE_BLOCKS * 4 <= 256, "local_n fits its slot");
+static_assert(PA_SAMPLE_BLOCKS * 4 <= 512, "local_n fits its slot");
 size_t pareto_stream_bytes() { return PA_OFF_FRONT + (size_t)PA_SURV_CAP * sizeof(KI); }
 
 bool stream_eligible(const guide_outputs &mat, Range r) { return r.count >= STREAM_MIN_COUNT && mat_vec_ok(mat) != 0; }
