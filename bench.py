@@ -40,7 +40,7 @@ BYTES_SIM = 6 * 8 + 1 + 4          # six fp64 metrics + status + bmax written pe
 # dram__bytes_read.sum + dram__bytes_write.sum of one guide_simulate call on the full workload 5: the
 # k_closed_form_memory and k_closed_form_model launches together (profiles/k_closed_form_split_c5.md);
 # only meaningful for that size and those kernel versions
-K1_TRAFFIC_C5 = 644_200_000 + 151_100_000 + 1_000_000
+K1_TRAFFIC_C5 = 644_400_000 + 151_100_000 + 1_000_000
 SIM_FIELDS = ("latency", "ttft", "tpot", "thr_decode", "cost_per_hr", "cost_per_token", "status", "bmax")
 TRACE_FIELDS = ("latency", "ttft", "ttft_p50", "ttft_p99", "tpot", "thr_decode", "cost_per_hr", "cost_per_token",
                 "status", "bmax", "n_iters", "n_req_iters")
@@ -246,7 +246,7 @@ def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full, fraction
                             "materialised_configs_per_s": n / (t_sim + t_km + t_pm) * 1e3,
                             "simulate_write_gbs": BYTES_SIM * n / t_sim / 1e6,
                             "simulate_frac_of_hbm": BYTES_SIM * n / t_sim / 1e6 / hbm_peak,
-                            "kernel_launches": 2 + 2 + 2 + 6 + 4}
+                            "kernel_launches": 2 + 2 + 2 + 5 + 4}
             del p
         torch.cuda.empty_cache()
     return res
@@ -383,7 +383,7 @@ def run_ours(args):
     bytes_topk = 1 + 8 * len(cons_arrays | {key})
     bytes_pareto = 1 + 8 * len(cons_arrays | {"latency", "cost_per_hr"})
     per = {"guide_simulate (k_closed_form_memory + k_closed_form_model)": (t_sim / args.steps, BYTES_SIM),
-           "guide_select_topk (k_topk_sample + k_topk_refine + k_topk_filter + k_topk_rank)": (t_topk / args.steps, bytes_topk),
+           "guide_select_topk (k_topk_bound + k_topk_filter + k_topk_rank)": (t_topk / args.steps, bytes_topk),
            "guide_pareto (k_pareto_sample + k_pareto_filter + k_pareto_rank)": (t_par / args.steps, bytes_pareto)}
     dom = max(per, key=lambda name: per[name][0])
     dom_ms, dom_bytes = per[dom]
@@ -415,11 +415,10 @@ def run_ours(args):
         which = [int(x) for x in args.extras.split(",") if x]
         extras = extra_workloads(guide, torch, inputs, which, flush, hbm_peak, args.full, args.trace_fraction)
 
-    # simulate: memory + model kernel; top-k: sample, refine, filter, rank and the two gated fallback
-    # kernels (scan, merge: they return at once); Pareto: sample, filter, rank and the gated general
-    # kernel; with several ranks the merge of the gathered lists (scan + merge, too short for the
-    # streaming path)
-    launches_per_step = 2 + 6 + 4 + (2 if world > 1 else 0)
+    # simulate: memory + model kernel; top-k: bound, filter, rank and the two gated fallback kernels
+    # (scan, merge: they return at once); Pareto: sample, filter, rank and the gated general kernel;
+    # with several ranks the merge of the gathered lists (scan + merge, too short for the streaming path)
+    launches_per_step = 2 + 5 + 4 + (2 if world > 1 else 0)
     line = {"metric": "configs/sec", "value": value, "unit": "configs/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
