@@ -29,6 +29,7 @@
 // thread takes two consecutive configs, 16 bytes), two such rows per thread and round.
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 
 #include <cooperative_groups.h>
 
@@ -867,7 +868,8 @@ static Sample make_sample(u64 n_rows, u32 want_rows, u32 max_r) {
 }
 
 // Can the bound kernel's grid (TK_SAMPLE_BLOCKS blocks of SEL_THREADS threads) be resident at once on
-// the current device, and does the device launch cooperatively?  Asked once per device.
+// the current device, and does the device launch cooperatively?  Asked once per device.  Setting
+// GUIDE_NO_COOPERATIVE in the environment forces the two-kernel form (the tests use it to cover both).
 template <int NA>
 static bool cooperative_ok() {
     static int cached[64] = {};                      // 0 unknown, 1 yes, 2 no
@@ -877,6 +879,7 @@ static bool cooperative_ok() {
         int coop = 0, per_sm = 0;
         cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_topk_bound<NA>, SEL_THREADS, 0);
+        if (getenv("GUIDE_NO_COOPERATIVE")) coop = 0;
         cached[dev] = (coop && (u64)per_sm * num_sms() >= TK_SAMPLE_BLOCKS) ? 1 : 2;
     }
     return cached[dev] == 1;

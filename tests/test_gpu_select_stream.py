@@ -119,6 +119,29 @@ def test_topk_sorted_inputs_and_winners_in_one_corner(sp):
     check_topk(sp, host, dev, {}, "cost_per_token", 128)
 
 
+def test_topk_bound_in_two_kernels():
+    """The top-k bound is one cooperative kernel where the device launches cooperatively, two
+    kernels otherwise; GUIDE_NO_COOPERATIVE forces the second form.  The library reads the variable
+    once per process, so the check runs in a child process: same cases, same oracle."""
+    import os
+    import subprocess
+    import sys
+    code = (
+        "import sys; sys.path.insert(0, 'tests')\n"
+        "import test_gpu_select_stream as t\n"
+        "from paper_2412_04788_b200 import guide, inputs as I\n"
+        "sp = guide.Space(I.workload(5, scale=0.125)['space'])\n"
+        "for n, seed in ((t.N_MIN + 1, 21), (5 * t.N_MIN + 65, 22)):\n"
+        "    host = t.synth(n, seed); dev = t.to_dev(host)\n"
+        "    for key, k in (('cost_per_token', 64), ('cost_per_hr', 128), ('throughput', 1)):\n"
+        "        assert t.check_topk(sp, host, dev, {'max_latency': 6.0}, key, k) == k\n"
+        "print('two-kernel bound ok')\n")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, "-c", code], cwd=root, env=dict(os.environ, GUIDE_NO_COOPERATIVE="1"),
+                         capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0 and "two-kernel bound ok" in res.stdout, res.stdout[-2000:] + res.stderr[-2000:]
+
+
 def test_pareto_random_pairs(sp):
     for n, seed in ((N_MIN, 11), (2 * N_MIN + 513, 12), (6 * N_MIN + 1, 13)):
         host = synth(n, seed)
