@@ -246,7 +246,7 @@ def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full, fraction
                             "materialised_configs_per_s": n / (t_sim + t_km + t_pm) * 1e3,
                             "simulate_write_gbs": BYTES_SIM * n / t_sim / 1e6,
                             "simulate_frac_of_hbm": BYTES_SIM * n / t_sim / 1e6 / hbm_peak,
-                            "kernel_launches": 2 + 2 + 2 + 5 + 4}
+                            "kernel_launches": 2 + 6 + 5 + 5 + 4}
             del p
         torch.cuda.empty_cache()
     return res

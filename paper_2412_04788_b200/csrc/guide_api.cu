@@ -574,9 +574,10 @@ int guide_select_topk(const guide_space *space_c, const guide_trace *trace, cons
     if ((rc = resolve_range(space, opts, &r))) return rc;
     if ((rc = check_workspace(ws, ws_bytes, topk_workspace_bytes(k)))) return rc;
     DSpace ds;
-    if ((rc = space_on_device(space, &ds))) return rc;
+    unsigned *ticket = nullptr;                  // the fused path's model walk takes its work items through it
+    if ((rc = space_on_device(space, &ds, outputs ? nullptr : &ticket))) return rc;
     return launch_topk(ds, r, outputs, opts ? opts->time_model : 0, opts ? opts->tp_model : 0, *cons, key, k,
-                       (u64 *)idx_out, key_out, count_out, ws, (cudaStream_t)stream);
+                       (u64 *)idx_out, key_out, count_out, ws, ticket, (cudaStream_t)stream);
 }
 
 int guide_pareto(const guide_space *space_c, const guide_trace *trace, const guide_outputs *outputs,
@@ -591,9 +592,10 @@ int guide_pareto(const guide_space *space_c, const guide_trace *trace, const gui
     if ((rc = resolve_range(space, opts, &r))) return rc;
     if ((rc = check_workspace(ws, ws_bytes, pareto_workspace_bytes()))) return rc;
     DSpace ds;
-    if ((rc = space_on_device(space, &ds))) return rc;
+    unsigned *ticket = nullptr;
+    if ((rc = space_on_device(space, &ds, outputs ? nullptr : &ticket))) return rc;
     return launch_pareto(ds, r, outputs, opts ? opts->time_model : 0, opts ? opts->tp_model : 0, *cons, xm, ym,
-                         (u64 *)idx_out, cap, count_out, ws, (cudaStream_t)stream);
+                         (u64 *)idx_out, cap, count_out, ws, ticket, (cudaStream_t)stream);
 }
 
 int guide_select_topk_noalloc(const guide_outputs *outputs, uint64_t first, uint64_t count,

@@ -80,10 +80,10 @@ size_t topk_workspace_bytes(u32 k);
 size_t pareto_workspace_bytes();
 int launch_topk(const DSpace &s, Range r, const guide_outputs *mat, int time_model, int tp_model,
                 const guide_constraints &c, int key, u32 k, u64 *idx_out, double *key_out, u32 *count_out,
-                void *ws, cudaStream_t st);
+                void *ws, unsigned *ticket, cudaStream_t st);
 int launch_pareto(const DSpace &s, Range r, const guide_outputs *mat, int time_model, int tp_model,
                   const guide_constraints &c, int xm, int ym, u64 *idx_out, u32 cap, u32 *count_out,
-                  void *ws, cudaStream_t st);
+                  void *ws, unsigned *ticket, cudaStream_t st);
 int launch_topk_noalloc(Range r, const guide_outputs &mat, const guide_constraints &c, int key, u32 k,
                         u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st);
 

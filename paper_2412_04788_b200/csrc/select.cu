@@ -21,19 +21,6 @@ static constexpr u32 PARETO_CAP = 4096;          // shared-memory items per bloc
 static constexpr u32 TOPK_CAP = 4096;            // shared-memory candidates per block
 static constexpr u32 MAX_BUDGET = 16;            // most appends per thread between two checkpoints
 
-__device__ __forceinline__ double pick_metric(int key, double latency, double ttft, double ttft_p99, double tpot,
-                                              double thr, double cost_hr, double cost_tok) {
-    switch (key) {
-    case GUIDE_LATENCY: return latency;
-    case GUIDE_TTFT: return ttft;
-    case GUIDE_TTFT_P99: return ttft_p99;
-    case GUIDE_TPOT: return tpot;
-    case GUIDE_THROUGHPUT: return 0.0 - thr;      // larger is better
-    case GUIDE_COST_PER_HR: return cost_hr;
-    default: return cost_tok;
-    }
-}
-
 // ---- where the metrics come from --------------------------------------------------------------
 
 // materialised arrays written by guide_simulate
@@ -584,16 +571,6 @@ struct WarpPareto {
     }
 };
 
-// constraint filter and metric choice on freshly evaluated closed-form metrics
-__device__ __forceinline__ bool fused_pick(const Metrics &m, const Cons &c, int m0, int m1, double &a, double &b) {
-    if (m.status) return false;
-    if (!(m.ttft <= c.max_ttft) || !(m.latency <= c.max_latency) || !(m.cost_hr <= c.max_cost_hr) || !(m.thr >= c.min_thr))
-        return false;
-    a = pick_metric(m0, m.latency, m.ttft, m.ttft, m.tpot, m.thr, m.cost_hr, m.cost_tok);
-    b = m1 >= 0 ? pick_metric(m1, m.latency, m.ttft, m.ttft, m.tpot, m.thr, m.cost_hr, m.cost_tok) : 0.0;
-    return true;
-}
-
 // ---- top-k kernels -----------------------------------------------------------------------------------
 
 // a block's sorted candidates and their number go to the workspace
@@ -660,9 +637,12 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_scan(Src src, Range r, u32
 template <int TIME_SUM, bool WARP>
 __global__ void __launch_bounds__(SEL_THREADS, 2)
 k_topk_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, Cons c, int key, u32 k, u32 *counts, KI *lists,
-             u64 *gthr) {
+             u64 *gthr, const u32 *gate) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ u32 cnt;
+    grid_dep_launch();
+    grid_dep_wait();                            // a gated launch may have started before its predecessor finished
+    if (gate && __ldcg(gate) == 0) return;
     typename TopKPick<WARP>::type acc;
     topk_begin(acc, (KI *)smem_raw, &cnt, k, gthr);
     tiled_visit<TIME_SUM>(s, r, tp_model, hf_chunk, tiles_per_mb, [&](bool valid, u64 j, const Metrics &m) {
@@ -896,6 +876,7 @@ k_pareto_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk, u32 tiles_per_mb, 
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ u32 cnt;
     __shared__ __align__(8) u32 scratch[64];
+    grid_dep_wait();                            // a gated launch may have started before its predecessor finished
     if (gate && __ldcg(gate) == 0) return;
     ParetoAcc acc;
     WarpPareto wacc;
@@ -999,31 +980,39 @@ static int run_topk_scan(const Src &src, Range r, u32 k, int negate, u32 max_blo
 
 template <int TIME_SUM, bool WARP>
 static int run_topk_tiled_mode(const DSpace &s, Range r, const TileGeom &g, int tp_model, const Cons &c, int key, u32 k,
-                               unsigned char *ws, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st) {
+                               unsigned char *ws, u64 *idx_out, double *key_out, u32 *count_out, const u32 *gate,
+                               cudaStream_t st) {
     u32 *counts = (u32 *)(ws + 256);
     KI *lists = (KI *)(ws + topk_lists_offset(SEL_MAX_BLOCKS));
     const size_t smem = WARP ? (size_t)(SEL_THREADS / 32) * warp_seg_cap(k) * sizeof(KI) : (size_t)TOPK_CAP * sizeof(KI);
     int rc = allow_smem(k_topk_tiled<TIME_SUM, WARP>, smem);
     if (rc) return rc;
-    if ((rc = topk_reset_header(ws, st))) return rc;
+    // a gated launch runs behind the fused streaming path, which has reset the header for the whole call
+    if (!gate && (rc = topk_reset_header(ws, st))) return rc;
     const dim3 grid(g.gx, g.splits);
-    k_topk_tiled<TIME_SUM, WARP><<<grid, g.threads, smem, st>>>(s, r, tp_model, g.hf_chunk, g.tiles_per_mb, c, key, k,
-                                                               counts, lists, (u64 *)ws);
-    GUIDE_CUDA(cudaGetLastError());
-    return run_topk_merge(g.gx * g.splits, k, key == GUIDE_THROUGHPUT, counts, lists, idx_out, key_out, count_out, nullptr, st);
+    if (gate) {
+        GUIDE_CUDA(launch_dependent(k_topk_tiled<TIME_SUM, WARP>, grid, g.threads, smem, st, s, r, tp_model, g.hf_chunk,
+                                    g.tiles_per_mb, c, key, k, counts, lists, (u64 *)ws, gate));
+    } else {
+        k_topk_tiled<TIME_SUM, WARP><<<grid, g.threads, smem, st>>>(s, r, tp_model, g.hf_chunk, g.tiles_per_mb, c, key, k,
+                                                                   counts, lists, (u64 *)ws, gate);
+        GUIDE_CUDA(cudaGetLastError());
+    }
+    return run_topk_merge(g.gx * g.splits, k, key == GUIDE_THROUGHPUT, counts, lists, idx_out, key_out, count_out, gate, st);
 }
 
 template <int TIME_SUM>
 static int run_topk_tiled(const DSpace &s, Range r, const TileGeom &g, int tp_model, const Cons &c, int key, u32 k,
-                          unsigned char *ws, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st) {
+                          unsigned char *ws, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st,
+                          const u32 *gate = nullptr) {
     return k <= TOPK_WARP_K
-               ? run_topk_tiled_mode<TIME_SUM, true>(s, r, g, tp_model, c, key, k, ws, idx_out, key_out, count_out, st)
-               : run_topk_tiled_mode<TIME_SUM, false>(s, r, g, tp_model, c, key, k, ws, idx_out, key_out, count_out, st);
+               ? run_topk_tiled_mode<TIME_SUM, true>(s, r, g, tp_model, c, key, k, ws, idx_out, key_out, count_out, gate, st)
+               : run_topk_tiled_mode<TIME_SUM, false>(s, r, g, tp_model, c, key, k, ws, idx_out, key_out, count_out, gate, st);
 }
 
 int launch_topk(const DSpace &s, Range r, const guide_outputs *mat, int time_model, int tp_model,
                 const guide_constraints &c, int key, u32 k, u64 *idx_out, double *key_out, u32 *count_out,
-                void *ws, cudaStream_t st) {
+                void *ws, unsigned *ticket, cudaStream_t st) {
     const int negate = key == GUIDE_THROUGHPUT;
     unsigned char *w = (unsigned char *)ws;
     if (mat) {
@@ -1041,9 +1030,22 @@ int launch_topk(const DSpace &s, Range r, const guide_outputs *mat, int time_mod
         return run_topk_scan(src, r, k, negate, SEL_MAX_BLOCKS, w, idx_out, key_out, count_out, st);
     }
     TileGeom g;
-    if (fused_tiled(s, r, &g))
-        return time_model ? run_topk_tiled<1>(s, r, g, tp_model, make_cons(c), key, k, w, idx_out, key_out, count_out, st)
-                          : run_topk_tiled<0>(s, r, g, tp_model, make_cons(c), key, k, w, idx_out, key_out, count_out, st);
+    if (fused_tiled(s, r, &g)) {
+        const u32 *gate = nullptr;
+        if (!mat && ticket && k <= STREAM_TOPK_MAX_K && fused_stream_eligible(s, r)) {
+            // fused streaming path first (sampled bound, model walk as the filter); the tiled kernels
+            // are queued behind it and return at once unless it raised the redo flag
+            int rc = topk_reset_header(w, st);
+            if (rc) return rc;
+            u32 *header = (u32 *)w;
+            if ((rc = launch_topk_fused(s, time_model, tp_model, c, key, k, header, w + topk_stream_offset(k), ticket, idx_out,
+                                        key_out, count_out, st)))
+                return rc;
+            gate = header + TK_REDO;
+        }
+        return time_model ? run_topk_tiled<1>(s, r, g, tp_model, make_cons(c), key, k, w, idx_out, key_out, count_out, st, gate)
+                          : run_topk_tiled<0>(s, r, g, tp_model, make_cons(c), key, k, w, idx_out, key_out, count_out, st, gate);
+    }
     if (time_model) {
         FusedSource<1> src{s, make_cons(c), key, -1, tp_model};
         return run_topk_scan(src, r, k, negate, SEL_MAX_BLOCKS, w, idx_out, key_out, count_out, st);
@@ -1092,16 +1094,23 @@ static int run_pareto_general(const Src &src, Range r, u64 *idx_out, u32 cap, u3
 
 template <int TIME_SUM>
 static int run_pareto_tiled(const DSpace &s, Range r, const TileGeom &g, int tp_model, const Cons &c, int xm, int ym,
-                            u64 *idx_out, u32 cap, u32 *count_out, void *ws, cudaStream_t st) {
+                            u64 *idx_out, u32 cap, u32 *count_out, void *ws, cudaStream_t st, bool general_only = false) {
     const size_t smem_fast = (size_t)(SEL_THREADS / 32) * WSEG * sizeof(P3);
     const size_t smem_gen = (size_t)PARETO_CAP * sizeof(P3);
     int rc = allow_smem(k_pareto_tiled<TIME_SUM, false>, smem_gen);
     if (rc) return rc;
-    GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
     u32 *header = (u32 *)ws;
     u32 *sizes = (u32 *)((char *)ws + 256);
     P3 *partial = (P3 *)((char *)ws + 256 + (size_t)SEL_MAX_BLOCKS * sizeof(u32));
     const dim3 grid(g.gx, g.splits);
+    if (general_only) {
+        // behind the fused streaming path, which has reset the header: the general kernel alone, gated on the redo flag
+        GUIDE_CUDA(launch_dependent(k_pareto_tiled<TIME_SUM, false>, grid, g.threads, smem_gen, st, s, r, tp_model, g.hf_chunk,
+                                    g.tiles_per_mb, c, xm, ym, header, (const u32 *)(header + 1), sizes, partial, idx_out, cap,
+                                    count_out));
+        return GUIDE_OK;
+    }
+    GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
     k_pareto_tiled<TIME_SUM, true><<<grid, g.threads, smem_fast, st>>>(s, r, tp_model, g.hf_chunk, g.tiles_per_mb, c, xm, ym,
                                                                       header, nullptr, sizes, partial, idx_out, cap, count_out);
     GUIDE_CUDA(cudaGetLastError());
@@ -1114,7 +1123,7 @@ static int run_pareto_tiled(const DSpace &s, Range r, const TileGeom &g, int tp_
 
 int launch_pareto(const DSpace &s, Range r, const guide_outputs *mat, int time_model, int tp_model,
                   const guide_constraints &c, int xm, int ym, u64 *idx_out, u32 cap, u32 *count_out, void *ws,
-                  cudaStream_t st) {
+                  unsigned *ticket, cudaStream_t st) {
     if (mat) {
         MatSource src{*mat, make_cons(c), xm, ym, mat_vec_ok(*mat)};
         if (stream_eligible(*mat, r)) {
@@ -1129,9 +1138,18 @@ int launch_pareto(const DSpace &s, Range r, const guide_outputs *mat, int time_m
         return run_pareto_scan(src, r, idx_out, cap, count_out, ws, st);
     }
     TileGeom g;
-    if (fused_tiled(s, r, &g))
-        return time_model ? run_pareto_tiled<1>(s, r, g, tp_model, make_cons(c), xm, ym, idx_out, cap, count_out, ws, st)
-                          : run_pareto_tiled<0>(s, r, g, tp_model, make_cons(c), xm, ym, idx_out, cap, count_out, ws, st);
+    if (fused_tiled(s, r, &g)) {
+        bool behind = false;
+        if (!mat && ticket && fused_stream_eligible(s, r)) {
+            GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
+            int rc = launch_pareto_fused(s, time_model, tp_model, c, xm, ym, (u32 *)ws, (unsigned char *)ws + pareto_stream_offset(),
+                                         ticket, idx_out, cap, count_out, st);
+            if (rc) return rc;
+            behind = true;
+        }
+        return time_model ? run_pareto_tiled<1>(s, r, g, tp_model, make_cons(c), xm, ym, idx_out, cap, count_out, ws, st, behind)
+                          : run_pareto_tiled<0>(s, r, g, tp_model, make_cons(c), xm, ym, idx_out, cap, count_out, ws, st, behind);
+    }
     if (time_model) {
         FusedSource<1> src{s, make_cons(c), xm, ym, tp_model};
         return run_pareto_scan(src, r, idx_out, cap, count_out, ws, st);

@@ -24,6 +24,29 @@ struct Cons {
     int ttft_stat;
 };
 
+__device__ __forceinline__ double pick_metric(int key, double latency, double ttft, double ttft_p99, double tpot,
+                                              double thr, double cost_hr, double cost_tok) {
+    switch (key) {
+    case GUIDE_LATENCY: return latency;
+    case GUIDE_TTFT: return ttft;
+    case GUIDE_TTFT_P99: return ttft_p99;
+    case GUIDE_TPOT: return tpot;
+    case GUIDE_THROUGHPUT: return 0.0 - thr;      // larger is better
+    case GUIDE_COST_PER_HR: return cost_hr;
+    default: return cost_tok;
+    }
+}
+
+// constraint filter and metric choice on freshly evaluated closed-form metrics
+__device__ __forceinline__ bool fused_pick(const Metrics &m, const Cons &c, int m0, int m1, double &a, double &b) {
+    if (m.status) return false;
+    if (!(m.ttft <= c.max_ttft) || !(m.latency <= c.max_latency) || !(m.cost_hr <= c.max_cost_hr) || !(m.thr >= c.min_thr))
+        return false;
+    a = pick_metric(m0, m.latency, m.ttft, m.ttft, m.tpot, m.thr, m.cost_hr, m.cost_tok);
+    b = m1 >= 0 ? pick_metric(m1, m.latency, m.ttft, m.ttft, m.tpot, m.thr, m.cost_hr, m.cost_tok) : 0.0;
+    return true;
+}
+
 inline Cons make_cons(const guide_constraints &c) {
     Cons k;
     k.max_ttft = c.max_ttft; k.max_latency = c.max_latency; k.max_cost_hr = c.max_cost_per_hr;
@@ -127,5 +150,15 @@ int launch_topk_stream(Range r, const guide_outputs &mat, const guide_constraint
                        unsigned char *region, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st);
 int launch_pareto_stream(Range r, const guide_outputs &mat, const guide_constraints &c, int xm, int ym, u32 *header,
                          unsigned char *region, u64 *idx_out, u32 cap, u32 *count_out, cudaStream_t st);
+
+
+// Fused form (nothing materialised, whole closed-form spaces): the sample rows are evaluated into a
+// compact scratch in the workspace, the same bound / killer kernels run on that, and the filter pass
+// is the model walk of model_walk.cuh with a sink that keeps candidates instead of storing metrics.
+bool fused_stream_eligible(const DSpace &s, Range r);
+int launch_topk_fused(const DSpace &s, int time_model, int tp_model, const guide_constraints &c, int key, u32 k, u32 *header,
+                      unsigned char *region, unsigned *ticket, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st);
+int launch_pareto_fused(const DSpace &s, int time_model, int tp_model, const guide_constraints &c, int xm, int ym, u32 *header,
+                        unsigned char *region, unsigned *ticket, u64 *idx_out, u32 cap, u32 *count_out, cudaStream_t st);
 
 }  // namespace guide

@@ -33,6 +33,7 @@
 
 #include <cooperative_groups.h>
 
+#include "model_walk.cuh"
 #include "select.cuh"
 
 namespace guide {
@@ -73,12 +74,26 @@ template <int NA>
 struct Src {
     Arr a[NA];
     const uint8_t *status;
+    const u64 *row_base;   // null: entry j is config first + j.  Else the arrays hold sampled rows of 64 configs
+                           // back to back and row_base[j / 64] is the index of the row's first config.
 };
+
+template <int NA>
+__device__ __forceinline__ u64 cfg_index(const Src<NA> &s, u64 first, u64 j) {
+    return s.row_base ? __ldg(s.row_base + (j >> 6)) + (j & 63) : first + j;
+}
 
 // region layout, top-k: pairs minima[TK_SAMPLE_BLOCKS] | pairs spairs[TK_SKEYS_CAP] | KI cand[TK_CAND_CAP]
 static constexpr size_t TK_OFF_SKEYS = (size_t)TK_SAMPLE_BLOCKS * 16;
 static constexpr size_t TK_OFF_CAND = TK_OFF_SKEYS + (size_t)TK_SKEYS_CAP * 16;
-size_t topk_stream_bytes() { return TK_OFF_CAND + (size_t)TK_CAND_CAP * sizeof(KI); }
+// ... | fused form only: u64 row_base[FUSED_ROWS] | u8 pass[FUSED_ROWS][64] | f64 a0[FUSED_ROWS][64] | f64 a1[FUSED_ROWS][64]
+static constexpr u32 FUSED_ROWS = 8192;         // sample rows the compact scratch holds
+static constexpr size_t FU_OFF_PASS = (size_t)FUSED_ROWS * 8;
+static constexpr size_t FU_OFF_A0 = FU_OFF_PASS + (size_t)FUSED_ROWS * 64;
+static constexpr size_t FU_OFF_A1 = FU_OFF_A0 + (size_t)FUSED_ROWS * 64 * 8;
+static constexpr size_t FU_BYTES = FU_OFF_A1 + (size_t)FUSED_ROWS * 64 * 8;
+static constexpr size_t TK_OFF_FUSED = (TK_OFF_CAND + (size_t)TK_CAND_CAP * sizeof(KI) + 255) / 256 * 256;
+size_t topk_stream_bytes() { return TK_OFF_FUSED + FU_BYTES; }
 // region layout, Pareto: P2 local[PA_KILLERS] | P2 killers[PA_KILLERS] | u32 local_n[PA_SAMPLE_BLOCKS] (padded to 256 B)
 //                        | P3 surv[PA_SURV_CAP] | KI front[PA_SURV_CAP]
 static constexpr size_t PA_OFF_KILLERS = (size_t)PA_KILLERS * sizeof(P2);
@@ -86,7 +101,8 @@ static constexpr size_t PA_OFF_LOCAL_N = 2 * PA_OFF_KILLERS;
 static constexpr size_t PA_OFF_SURV = PA_OFF_LOCAL_N + 512;
 static constexpr size_t PA_OFF_FRONT = PA_OFF_SURV + (size_t)PA_SURV_CAP * sizeof(P3);
 static_assert(PA_SAMPLE_BLOCKS * 4 <= 512, "local_n fits its slot");
-size_t pareto_stream_bytes() { return PA_OFF_FRONT + (size_t)PA_SURV_CAP * sizeof(KI); }
+static constexpr size_t PA_OFF_FUSED = (PA_OFF_FRONT + (size_t)PA_SURV_CAP * sizeof(KI) + 255) / 256 * 256;
+size_t pareto_stream_bytes() { return PA_OFF_FUSED + FU_BYTES; }
 
 bool stream_eligible(const guide_outputs &mat, Range r) { return r.count >= STREAM_MIN_COUNT && mat_vec_ok(mat) != 0; }
 
@@ -220,8 +236,8 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_sample(Src<NA> s, Sample s
         for (u32 u = 0; u < SAMPLE_BATCH; u++) {
             bool ok0, ok1;
             eval_pair(s, st[u], v[u], ok0, ok1);
-            if (j[u] != KEY_MAX && ok0) pair_min(bk, bi, metric_key(s.a[0], v[u][0].x), first + j[u]);
-            if (j[u] != KEY_MAX && ok1) pair_min(bk, bi, metric_key(s.a[0], v[u][0].y), first + j[u] + 1);
+            if (j[u] != KEY_MAX && ok0) pair_min(bk, bi, metric_key(s.a[0], v[u][0].x), cfg_index(s, first, j[u]));
+            if (j[u] != KEY_MAX && ok1) pair_min(bk, bi, metric_key(s.a[0], v[u][0].y), cfg_index(s, first, j[u]) + 1);
         }
     }
     for (int d = 16; d > 0; d >>= 1)
@@ -276,9 +292,9 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_refine(Src<NA> s, Sample s
             const u64 key[2] = {metric_key(s.a[0], v[u][0].x), metric_key(s.a[0], v[u][0].y)};
 #pragma unroll
             for (u32 h = 0; h < 2; h++) {
-                if (j[u] != KEY_MAX && ok[h] && pair_le(key[h], first + j[u] + h, bkey, bidx)) {
+                if (j[u] != KEY_MAX && ok[h] && pair_le(key[h], cfg_index(s, first, j[u]) + h, bkey, bidx)) {
                     const u32 p = atomicAdd(header + TK_SAMPLED, 1);
-                    if (p < TK_SKEYS_CAP) { ulonglong2 e; e.x = key[h]; e.y = first + j[u] + h; spairs[p] = e; }
+                    if (p < TK_SKEYS_CAP) { ulonglong2 e; e.x = key[h]; e.y = cfg_index(s, first, j[u]) + h; spairs[p] = e; }
                 }
             }
         }
@@ -375,8 +391,8 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_bound(Src<NA> s, Sample sm
         for (u32 u = 0; u < SAMPLE_BATCH; u++) {
             bool ok0, ok1;
             eval_pair(s, st[u], v[u], ok0, ok1);
-            if (j[u] != KEY_MAX && ok0) pair_min(bk, bi, metric_key(s.a[0], v[u][0].x), first + j[u]);
-            if (j[u] != KEY_MAX && ok1) pair_min(bk, bi, metric_key(s.a[0], v[u][0].y), first + j[u] + 1);
+            if (j[u] != KEY_MAX && ok0) pair_min(bk, bi, metric_key(s.a[0], v[u][0].x), cfg_index(s, first, j[u]));
+            if (j[u] != KEY_MAX && ok1) pair_min(bk, bi, metric_key(s.a[0], v[u][0].y), cfg_index(s, first, j[u]) + 1);
         }
     }
     for (int d = 16; d > 0; d >>= 1)
@@ -415,9 +431,9 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_bound(Src<NA> s, Sample sm
             const u64 key[2] = {metric_key(s.a[0], v[u][0].x), metric_key(s.a[0], v[u][0].y)};
 #pragma unroll
             for (u32 h = 0; h < 2; h++) {
-                if (j[u] != KEY_MAX && ok[h] && pair_le(key[h], first + j[u] + h, bkey, bidx)) {
+                if (j[u] != KEY_MAX && ok[h] && pair_le(key[h], cfg_index(s, first, j[u]) + h, bkey, bidx)) {
                     const u32 p = atomicAdd(header + TK_SAMPLED, 1);
-                    if (p < TK_SKEYS_CAP) { ulonglong2 e; e.x = key[h]; e.y = first + j[u] + h; spairs[p] = e; }
+                    if (p < TK_SKEYS_CAP) { ulonglong2 e; e.x = key[h]; e.y = cfg_index(s, first, j[u]) + h; spairs[p] = e; }
                 }
             }
         }
@@ -891,6 +907,7 @@ static int topk_stream_na(const Arr *arr, Range r, const guide_outputs &mat, u32
     Src<NA> s;
     for (int i = 0; i < NA; i++) s.a[i] = arr[i];
     s.status = mat.status;
+    s.row_base = nullptr;
     ulonglong2 *minima = reinterpret_cast<ulonglong2 *>(region);
     ulonglong2 *spairs = reinterpret_cast<ulonglong2 *>(region + TK_OFF_SKEYS);
     KI *cand = reinterpret_cast<KI *>(region + TK_OFF_CAND);
@@ -939,6 +956,7 @@ static int pareto_stream_na(const Arr *arr, Range r, const guide_outputs &mat, u
     Src<NA> s;
     for (int i = 0; i < NA; i++) s.a[i] = arr[i];
     s.status = mat.status;
+    s.row_base = nullptr;
     P2 *local = reinterpret_cast<P2 *>(region);
     P2 *killers = reinterpret_cast<P2 *>(region + PA_OFF_KILLERS);
     u32 *local_n = reinterpret_cast<u32 *>(region + PA_OFF_LOCAL_N);
@@ -968,6 +986,217 @@ int launch_pareto_stream(Range r, const guide_outputs &mat, const guide_constrai
     case 6: return pareto_stream_na<6>(arr, r, mat, header, region, idx_out, cap, count_out, st);
     default: return fail(GUIDE_ERR_UNSUPPORTED, "a Pareto call touches two to six arrays");
     }
+}
+
+// ---- fused form: nothing materialised ---------------------------------------------------------------
+
+// The sample rows of a whole closed-form space, evaluated config by config into the compact
+// scratch: pass flag (0 = fits and meets the constraints), the metric(s) of the call, and where
+// each row starts.  One thread per config; 64 consecutive configs of a row share everything but
+// the length pair.
+template <int TIME_SUM>
+__global__ void __launch_bounds__(SEL_THREADS) k_fused_sample(DSpace s, int tp_model, Sample sm, Cons c, int m0, int m1,
+                                                              u64 *row_base, uint8_t *pass, double *a0, double *a1) {
+    grid_dep_launch();
+    const u64 slot = (u64)blockIdx.x * (SEL_THREADS / ROW) + threadIdx.x / ROW;
+    if (slot >= sm.n_slots) return;
+    const u32 l = threadIdx.x % ROW;
+    const u64 first = sm.row(slot) * ROW;
+    Metrics m;
+    closed_form_eval<TIME_SUM>(s, decode_index(s, first + l), tp_model, m);
+    double a = 0.0, b = 0.0;
+    const bool ok = fused_pick(m, c, m0, m1, a, b);
+    const u64 q = slot * ROW + l;
+    pass[q] = ok ? 0 : 1;
+    a0[q] = a;
+    if (m1 >= 0) a1[q] = b;
+    if (l == 0) row_base[slot] = first;
+}
+
+__device__ __forceinline__ bool meets(const Cons &c, double latency, double ttft, double thr, double cost_hr) {
+    return ttft <= c.max_ttft && latency <= c.max_latency && cost_hr <= c.max_cost_hr && thr >= c.min_thr;
+}
+
+// Filter pass of the fused top-k: the model walk, with the configs that fit, meet the constraints
+// and are within the bound going to the candidate list.
+template <int TIME_SUM>
+__global__ void __launch_bounds__(MODEL_THREADS, MODEL_BLOCKS_PER_SM)
+k_topk_model(DSpace s, int tp_model, u32 n_chunks, unsigned *ticket, Cons c, int key, u32 *header, KI *cand) {
+    grid_dep_launch();
+    grid_dep_wait();
+    const u64 *bp = reinterpret_cast<const u64 *>(header + TK_BOUND);
+    const u64 bkey = __ldcg(bp), bidx = __ldcg(bp + 1);
+    model_walk<TIME_SUM>(s, tp_model, n_chunks, ticket,
+                         [&](bool fits, u32, u32, u64 j, double latency, double ttft, double tpot, double thr, double cost_hr,
+                             double cost_tok, u64, u64) {
+        if (!fits || !meets(c, latency, ttft, thr, cost_hr)) return;
+        const u64 k64 = enc(pick_metric(key, latency, ttft, ttft, tpot, thr, cost_hr, cost_tok));
+        if (pair_le(k64, j, bkey, bidx)) topk_keep(k64, j, header, cand);
+    });
+}
+
+// Filter pass of the fused Pareto front: configs no killer strictly dominates go to the survivor list.
+template <int TIME_SUM>
+__global__ void __launch_bounds__(MODEL_THREADS, MODEL_BLOCKS_PER_SM)
+k_pareto_model(DSpace s, int tp_model, u32 n_chunks, unsigned *ticket, Cons c, int xm, int ym, u32 *header, const P2 *killers,
+               P3 *surv) {
+    __shared__ P2 ks[PA_KILLERS];
+    grid_dep_launch();
+    grid_dep_wait();
+    KillerSet K;
+    K.k = ks;
+    K.n = min(__ldcg(header + PH_KILLERS), PA_KILLERS);
+    for (u32 i = threadIdx.x; i < K.n; i += blockDim.x) {
+        const ulonglong2 w = __ldcg(reinterpret_cast<const ulonglong2 *>(killers + i));
+        ks[i].x = w.x; ks[i].y = w.y;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        if (K.n > 0) { const P2 p = ks[(K.n * (2 * i + 1)) / 8]; K.rx[i] = p.x; K.ry[i] = p.y; }
+        else { K.rx[i] = KEY_MAX; K.ry[i] = KEY_MAX; }
+    }
+    model_walk<TIME_SUM>(s, tp_model, n_chunks, ticket,
+                         [&](bool fits, u32, u32, u64 j, double latency, double ttft, double tpot, double thr, double cost_hr,
+                             double cost_tok, u64, u64) {
+        if (!fits || !meets(c, latency, ttft, thr, cost_hr)) return;
+        const u64 x = enc(pick_metric(xm, latency, ttft, ttft, tpot, thr, cost_hr, cost_tok));
+        const u64 y = enc(pick_metric(ym, latency, ttft, ttft, tpot, thr, cost_hr, cost_tok));
+        if (!K.kills(x, y)) pareto_keep(x, y, j, header, surv);
+    });
+}
+
+// Whole closed-form spaces whose (TP, length) plane divides into foursomes (what model_walk needs),
+// large enough for the sampled bound to pay.
+bool fused_stream_eligible(const DSpace &s, Range r) {
+    const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
+    const u32 n_tl = s.n_t * s.n_l;
+    if (r.first != 0 || r.count != total || total < STREAM_MIN_COUNT) return false;
+    if (s.n_l % 4 != 0 || n_tl < 32) return false;
+    const u64 n_hf = (u64)s.n_h * s.n_f;
+    return (u64)s.n_m * s.n_b * (n_tl / 4) * ((n_hf + MODEL_CHUNK - 1) / MODEL_CHUNK) <= 0x7FFFFFFFull;
+}
+
+// the compact scratch as the arrays of a selection source
+struct FusedScratch {
+    u64 *row_base;
+    uint8_t *pass;
+    double *a0, *a1;
+};
+static FusedScratch fused_scratch(unsigned char *base) {
+    return FusedScratch{reinterpret_cast<u64 *>(base), base + FU_OFF_PASS, reinterpret_cast<double *>(base + FU_OFF_A0),
+                        reinterpret_cast<double *>(base + FU_OFF_A1)};
+}
+
+// sample rows of the space -> compact scratch; returns the walk over the scratch (row c of it is slot c)
+template <int TIME_SUM>
+static int fused_sample(const DSpace &s, int tp_model, const Cons &c, int m0, int m1, u32 want_rows, u32 max_r, const FusedScratch &f,
+                        Sample *compact, cudaStream_t st) {
+    const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
+    Sample sm = make_sample(total / ROW, want_rows, max_r);
+    sm.n_slots = std::min<u64>(sm.n_groups, FUSED_ROWS);
+    const u32 grid = (u32)((sm.n_slots + SEL_THREADS / ROW - 1) / (SEL_THREADS / ROW));
+    k_fused_sample<TIME_SUM><<<grid, SEL_THREADS, 0, st>>>(s, tp_model, sm, c, m0, m1, f.row_base, f.pass, f.a0, f.a1);
+    GUIDE_CUDA(cudaGetLastError());
+    compact->n_groups = sm.n_slots; compact->n_slots = sm.n_slots; compact->mul = 1; compact->r = 1;
+    return GUIDE_OK;
+}
+
+static cudaError_t launch_model_dependent_cfg(cudaLaunchConfig_t *cfg, cudaLaunchAttribute *at, cudaStream_t st) {
+    *cfg = cudaLaunchConfig_t{};
+    cfg->gridDim = dim3((u32)num_sms() * MODEL_BLOCKS_PER_SM); cfg->blockDim = dim3(MODEL_THREADS); cfg->dynamicSmemBytes = 0;
+    cfg->stream = st;
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg->attrs = at; cfg->numAttrs = 1;
+    return cudaSuccess;
+}
+
+template <int TIME_SUM>
+static int topk_fused_t(const DSpace &s, int tp_model, const guide_constraints &gc, int key, u32 k, u32 *header,
+                        unsigned char *region, unsigned *ticket, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st) {
+    const Cons c = make_cons(gc);
+    const FusedScratch f = fused_scratch(region + TK_OFF_FUSED);
+    ulonglong2 *minima = reinterpret_cast<ulonglong2 *>(region);
+    ulonglong2 *spairs = reinterpret_cast<ulonglong2 *>(region + TK_OFF_SKEYS);
+    KI *cand = reinterpret_cast<KI *>(region + TK_OFF_CAND);
+    GUIDE_CUDA(cudaMemsetAsync(ticket, 0, 4, st));           // the model walk's work counter
+    Sample sm;
+    int rc = fused_sample<TIME_SUM>(s, tp_model, c, key, -1, TK_SAMPLE_ROWS, TK_SAMPLE_MAX_R, f, &sm, st);
+    if (rc) return rc;
+    Src<1> src;
+    src.a[0] = Arr{f.a0, 0.0, 0, 0};                         // pick_metric has negated the throughput already
+    src.status = f.pass;
+    src.row_base = f.row_base;
+    if (cooperative_ok<1>()) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(TK_SAMPLE_BLOCKS); cfg.blockDim = dim3(SEL_THREADS); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeCooperative;
+        at[0].val.cooperative = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_topk_bound<1>, src, sm, (u64)0, k, header, minima, spairs));
+    } else {
+        k_topk_sample<1><<<TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st>>>(src, sm, (u64)0, k, header, minima);
+        GUIDE_CUDA(cudaGetLastError());
+        GUIDE_CUDA(launch_dependent(k_topk_refine<1>, TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st, src, sm, (u64)0, k, header, spairs));
+    }
+    const u32 n_chunks = (s.n_h * s.n_f + MODEL_CHUNK - 1) / MODEL_CHUNK;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute at[1];
+    launch_model_dependent_cfg(&cfg, at, st);
+    GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_topk_model<TIME_SUM>, s, tp_model, n_chunks, ticket, c, key, header, cand));
+    const size_t smem = (size_t)TK_CAND_SMEM * sizeof(KI);
+    GUIDE_CUDA(cudaFuncSetAttribute(k_topk_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    GUIDE_CUDA(launch_dependent(k_topk_rank, num_sms(), SEL_THREADS, smem, st, header, (const KI *)cand, k,
+                                key == GUIDE_THROUGHPUT ? 1 : 0, idx_out, key_out, count_out));
+    return GUIDE_OK;
+}
+
+int launch_topk_fused(const DSpace &s, int time_model, int tp_model, const guide_constraints &c, int key, u32 k, u32 *header,
+                      unsigned char *region, unsigned *ticket, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st) {
+    return time_model ? topk_fused_t<1>(s, tp_model, c, key, k, header, region, ticket, idx_out, key_out, count_out, st)
+                      : topk_fused_t<0>(s, tp_model, c, key, k, header, region, ticket, idx_out, key_out, count_out, st);
+}
+
+template <int TIME_SUM>
+static int pareto_fused_t(const DSpace &s, int tp_model, const guide_constraints &gc, int xm, int ym, u32 *header,
+                          unsigned char *region, unsigned *ticket, u64 *idx_out, u32 cap, u32 *count_out, cudaStream_t st) {
+    const Cons c = make_cons(gc);
+    const FusedScratch f = fused_scratch(region + PA_OFF_FUSED);
+    P2 *local = reinterpret_cast<P2 *>(region);
+    P2 *killers = reinterpret_cast<P2 *>(region + PA_OFF_KILLERS);
+    u32 *local_n = reinterpret_cast<u32 *>(region + PA_OFF_LOCAL_N);
+    P3 *surv = reinterpret_cast<P3 *>(region + PA_OFF_SURV);
+    KI *front = reinterpret_cast<KI *>(region + PA_OFF_FRONT);
+    GUIDE_CUDA(cudaMemsetAsync(ticket, 0, 4, st));
+    Sample sm;
+    int rc = fused_sample<TIME_SUM>(s, tp_model, c, xm, ym, PA_SAMPLE_ROWS, 1u << 20, f, &sm, st);
+    if (rc) return rc;
+    Src<2> src;
+    src.a[0] = Arr{f.a0, 0.0, 0, 0};
+    src.a[1] = Arr{f.a1, 0.0, 0, 0};
+    src.status = f.pass;
+    src.row_base = f.row_base;
+    k_pareto_sample<2><<<PA_SAMPLE_BLOCKS, SEL_THREADS, 0, st>>>(src, sm, header, local, local_n, killers);
+    GUIDE_CUDA(cudaGetLastError());
+    const u32 n_chunks = (s.n_h * s.n_f + MODEL_CHUNK - 1) / MODEL_CHUNK;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute at[1];
+    launch_model_dependent_cfg(&cfg, at, st);
+    GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_pareto_model<TIME_SUM>, s, tp_model, n_chunks, ticket, c, xm, ym, header,
+                                  (const P2 *)killers, surv));
+    const size_t smem = (size_t)PA_SURV_CAP * 16;
+    GUIDE_CUDA(cudaFuncSetAttribute(k_pareto_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    GUIDE_CUDA(launch_dependent(k_pareto_rank, num_sms(), SEL_THREADS, smem, st, header, (const P3 *)surv, front, idx_out, cap,
+                                count_out));
+    return GUIDE_OK;
+}
+
+int launch_pareto_fused(const DSpace &s, int time_model, int tp_model, const guide_constraints &c, int xm, int ym, u32 *header,
+                        unsigned char *region, unsigned *ticket, u64 *idx_out, u32 cap, u32 *count_out, cudaStream_t st) {
+    return time_model ? pareto_fused_t<1>(s, tp_model, c, xm, ym, header, region, ticket, idx_out, cap, count_out, st)
+                      : pareto_fused_t<0>(s, tp_model, c, xm, ym, header, region, ticket, idx_out, cap, count_out, st);
 }
 
 }  // namespace guide

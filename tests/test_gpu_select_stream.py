@@ -142,6 +142,34 @@ def test_topk_bound_in_two_kernels():
     assert res.returncode == 0 and "two-kernel bound ok" in res.stdout, res.stdout[-2000:] + res.stderr[-2000:]
 
 
+def test_fused_streaming_selection_half_of_workload_2():
+    """Nothing materialised, 491,520 configs: the sample rows are evaluated into the workspace, the
+    bound / killers come from them and the model walk is the filter pass.  All keys, with and
+    without constraints, both time models."""
+    w = I.workload(2, scale=0.5)
+    sp2 = guide.Space(w["space"])
+    assert sp2.size >= N_MIN
+    for tm, tpm in ((0, 0), (1, 1)):
+        want = oracle.simulate(w["space"], time_model=tm, tp_model=tpm)
+        med = float(np.median(want["latency"][want["status"] == 0]))
+        for cons in ({}, {"max_latency": med, "max_cost_per_hr": 60.0, "min_throughput": 50.0, "max_ttft": 5.0, "ttft_stat": "mean"}):
+            for key in guide.METRICS:
+                for k in ((1, 64, 128) if key == "cost_per_token" else (8,)):
+                    idx, val, cnt = run_topk(sp2, None, cons, key, k, time_model=tm, tp_model=tpm)
+                    w_idx, w_val, w_cnt = oracle.select_topk(want, cons, key, k)
+                    assert cnt == w_cnt and np.array_equal(idx, w_idx), (tm, key, k)
+                    assert np.array_equal(val.view(np.uint64), w_val.view(np.uint64)), (tm, key, k)
+            for x, y in (("latency", "cost_per_hr"), ("latency", "cost_per_token"), ("ttft", "throughput"), ("tpot", "cost_per_hr")):
+                fidx, fcnt = run_pareto(sp2, None, cons, x, y, time_model=tm, tp_model=tpm)
+                w_f, w_n = oracle.pareto(want, cons, x, y, cap=guide.PARETO_MAX)
+                assert fcnt == w_n and np.array_equal(fidx, w_f), (tm, x, y)
+    # nothing passes
+    idx, val, cnt = run_topk(sp2, None, {"max_latency": 0.0}, "latency", 8)
+    assert cnt == 0 and np.all(idx == U64_MAX)
+    fidx, fcnt = run_pareto(sp2, None, {"max_latency": 0.0}, "latency", "cost_per_hr")
+    assert fcnt == 0
+
+
 def test_pareto_random_pairs(sp):
     for n, seed in ((N_MIN, 11), (2 * N_MIN + 513, 12), (6 * N_MIN + 1, 13)):
         host = synth(n, seed)
