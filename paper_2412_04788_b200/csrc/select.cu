@@ -960,7 +960,7 @@ static int run_topk_scan_mode(const Src &src, Range r, u32 k, int negate, u32 ma
     if (rc) return rc;
     // a gated launch runs behind the streaming path, which has reset the header for the whole call
     if (!gate && (rc = topk_reset_header(ws, st))) return rc;
-    const u32 grid = grid_for(r.count, Src::ITEMS, WARP ? 4 : 3, max_blocks);
+    const u32 grid = grid_for(r.count, Src::ITEMS, gate ? 1 : (WARP ? 4 : 3), max_blocks);   // gated: rarely runs, keep the launch small
     if (gate) {
         GUIDE_CUDA(launch_dependent(k_topk_scan<Src, WARP>, grid, SEL_THREADS, smem, st, src, r, k, counts, lists, (u64 *)ws, gate));
     } else {
@@ -1020,9 +1020,8 @@ int launch_topk(const DSpace &s, Range r, const guide_outputs *mat, int time_mod
         if (k <= STREAM_TOPK_MAX_K && stream_eligible(*mat, r)) {
             // streaming path first; the accumulator kernels are queued behind it and return at once
             // unless it raised the redo flag
-            int rc = topk_reset_header(w, st);
-            if (rc) return rc;
-            u32 *header = (u32 *)w;
+            int rc;
+            u32 *header = (u32 *)w;                         // reset by the streaming path itself
             if ((rc = launch_topk_stream(r, *mat, c, key, k, header, w + topk_stream_offset(k), idx_out, key_out, count_out, st)))
                 return rc;
             return run_topk_scan(src, r, k, negate, SEL_MAX_BLOCKS, w, idx_out, key_out, count_out, st, header + TK_REDO);
@@ -1035,9 +1034,8 @@ int launch_topk(const DSpace &s, Range r, const guide_outputs *mat, int time_mod
         if (!mat && ticket && k <= STREAM_TOPK_MAX_K && fused_stream_eligible(s, r)) {
             // fused streaming path first (sampled bound, model walk as the filter); the tiled kernels
             // are queued behind it and return at once unless it raised the redo flag
-            int rc = topk_reset_header(w, st);
-            if (rc) return rc;
-            u32 *header = (u32 *)w;
+            int rc;
+            u32 *header = (u32 *)w;                         // reset by the streaming path itself
             if ((rc = launch_topk_fused(s, time_model, tp_model, c, key, k, header, w + topk_stream_offset(k), ticket, idx_out,
                                         key_out, count_out, st)))
                 return rc;
@@ -1086,7 +1084,7 @@ static int run_pareto_general(const Src &src, Range r, u64 *idx_out, u32 cap, u3
     u32 *header = (u32 *)ws;
     u32 *sizes = (u32 *)((char *)ws + 256);
     P3 *partial = (P3 *)((char *)ws + 256 + (size_t)SEL_MAX_BLOCKS * sizeof(u32));
-    const u32 grid_gen = grid_for(r.count, Src::ITEMS, 2, SEL_MAX_BLOCKS);
+    const u32 grid_gen = grid_for(r.count, Src::ITEMS, 1, SEL_MAX_BLOCKS);      // rarely runs: keep the launch small
     GUIDE_CUDA(launch_dependent(k_pareto_scan<Src, false>, grid_gen, SEL_THREADS, smem_gen, st, src, r, header,
                                 (const u32 *)(header + 1), sizes, partial, idx_out, cap, count_out));
     return GUIDE_OK;

@@ -376,6 +376,9 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_bound(Src<NA> s, Sample sm
     cg::grid_group grid = cg::this_grid();
     __shared__ ulonglong2 sl[SEL_THREADS / 32];
     grid_dep_launch();
+    // the call's header is reset here rather than by a memset in front: nothing reads it before the
+    // first grid barrier, and the kernels queued behind wait for this grid to complete
+    if (blockIdx.x == 0 && threadIdx.x < 64) header[threadIdx.x] = 0;
     const u32 lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = SEL_THREADS / 32;
     const u32 gwarp = blockIdx.x * n_warps + warp, total_warps = gridDim.x * n_warps;
     const u64 stride = (u64)gridDim.x * n_warps;
@@ -923,6 +926,7 @@ static int topk_stream_na(const Arr *arr, Range r, const guide_outputs &mat, u32
         cfg.attrs = at; cfg.numAttrs = 1;
         GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_topk_bound<NA>, s, sm, r.first, k, header, minima, spairs));
     } else {
+        GUIDE_CUDA(cudaMemsetAsync(header, 0, 256, st));
         k_topk_sample<NA><<<TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st>>>(s, sm, r.first, k, header, minima);
         GUIDE_CUDA(cudaGetLastError());
         GUIDE_CUDA(launch_dependent(k_topk_refine<NA>, TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st, s, sm, r.first, k, header, spairs));
@@ -1137,6 +1141,7 @@ static int topk_fused_t(const DSpace &s, int tp_model, const guide_constraints &
         cfg.attrs = at; cfg.numAttrs = 1;
         GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_topk_bound<1>, src, sm, (u64)0, k, header, minima, spairs));
     } else {
+        GUIDE_CUDA(cudaMemsetAsync(header, 0, 256, st));
         k_topk_sample<1><<<TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st>>>(src, sm, (u64)0, k, header, minima);
         GUIDE_CUDA(cudaGetLastError());
         GUIDE_CUDA(launch_dependent(k_topk_refine<1>, TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st, src, sm, (u64)0, k, header, spairs));
