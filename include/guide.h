@@ -90,11 +90,20 @@ typedef struct guide_space_desc {
     const uint32_t *batch;       uint32_t n_batch;    /* batch size (closed form) / max batch (trace) */
     const uint32_t *tp;          uint32_t n_tp;       /* modelled tensor-parallel degree, powers of two */
     const guide_len_pair *pairs; uint32_t n_pairs;    /* (input length, output length) */
+    /* Hybrid parallelism (Sec. 3.5.2, Sec. 3.5.3): dp[i] is the data-parallel degree that goes with
+     * tp[i], so entry i of the parallelism axis is the pair (dp[i], tp[i]) on dp[i] * tp[i] GPUs;
+     * enumerating the pairs under a GPU budget is the caller's get_configurations step.  The batch is
+     * split over the dp replicas and a stage lasts as long as the replica with ceil(batch / dp)
+     * requests; B_max and the memory check are per replica (Sec. 3.2 Step 1), throughput counts all
+     * replicas, the hourly cost all dp * tp GPUs.  NULL = every dp is 1.  Closed form only: with any
+     * dp > 1, guide_simulate on a trace returns GUIDE_ERR_UNSUPPORTED. */
+    const uint32_t *dp;
 } guide_space_desc;
 
 typedef struct guide_config {
     uint32_t model, hw, fw, batch_pos, tp_pos, pair_pos;   /* axis positions */
     uint32_t batch, tp, lin, lout;                         /* axis values */
+    uint32_t dp;                                           /* data-parallel degree of the tp_pos entry */
 } guide_config;
 
 typedef struct guide_space guide_space;

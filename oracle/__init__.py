@@ -39,7 +39,8 @@ class _Space(C.Structure):
                 ("fw_f", C.c_void_p), ("fw_i", C.c_void_p), ("n_f", C.c_uint32),
                 ("batch", C.c_void_p), ("n_b", C.c_uint32),
                 ("tp", C.c_void_p), ("n_t", C.c_uint32),
-                ("pairs", C.c_void_p), ("n_l", C.c_uint32)]
+                ("pairs", C.c_void_p), ("n_l", C.c_uint32),
+                ("dp", C.c_void_p)]
 
 
 class _Trace(C.Structure):
@@ -102,7 +103,8 @@ def _p(a):
 def _space_struct(space):
     return _Space(_p(space["models"]), len(space["models"]), _p(space["hw"]), _p(space["hw_mem"]), len(space["hw"]),
                   _p(space["fw_f"]), _p(space["fw_i"]), len(space["fw_f"]), _p(space["batch"]), len(space["batch"]),
-                  _p(space["tp"]), len(space["tp"]), _p(space["pairs"]), len(space["pairs"]))
+                  _p(space["tp"]), len(space["tp"]), _p(space["pairs"]), len(space["pairs"]),
+                  _p(space["dp"]) if space.get("dp") is not None else None)
 
 
 def simulate(space, trace=None, first=0, count=None, stride=1, time_model=TIME_MAX, tp_model=TP_EXPLICIT,
@@ -135,7 +137,8 @@ def simulate(space, trace=None, first=0, count=None, stride=1, time_model=TIME_M
     rc = lib().oracle_simulate(C.byref(sp), C.byref(ts) if ts is not None else None, first, count, stride,
                                time_model, tp_model, max_iters, C.byref(o), n_threads)
     if rc != 0:
-        raise ValueError(f"oracle_simulate failed: {rc} ({'invalid input' if rc == -1 else '64-bit overflow'})")
+        why = {-1: "invalid input", -2: "64-bit overflow", -3: "data parallelism with a trace is not modelled"}.get(rc, "?")
+        raise ValueError(f"oracle_simulate failed: {rc} ({why})")
     return out
 
 

@@ -57,6 +57,7 @@ typedef struct {
     const u32 *batch; u32 n_b;
     const u32 *tp; u32 n_t;
     const u32 *pairs; u32 n_l;             /* [n_l][2]: Lin Lout */
+    const u32 *dp;                         /* [n_t] data-parallel degree of each entry of the parallelism axis; NULL = all 1 */
 } ospace;
 
 typedef struct {
@@ -231,8 +232,13 @@ static void closed_form_one(const ospace *s, u64 idx, u64 j, int time_model, int
     pos_t p = decode(s, idx);
     model_t m = load_model(s->models + 10 * p.m);
     rates_t r = load_rates(s->hw + 5 * p.h, s->fw_f + 8 * p.f, s->fw_i + 4 * p.f);
-    u64 t = s->tp[p.t], b = s->batch[p.b], Lin = s->pairs[2 * p.l], Lout = s->pairs[2 * p.l + 1];
+    u64 t = s->tp[p.t], b_all = s->batch[p.b], Lin = s->pairs[2 * p.l], Lout = s->pairs[2 * p.l + 1];
     u64 kv_block = s->fw_i[4 * p.f + 1], reserve = s->fw_i[4 * p.f + 2];
+    /* Hybrid parallelism (Sec. 3.5.2, Sec. 3.5.3): the batch is split over dp replicas of t GPUs each;
+     * a stage lasts as long as its slowest replica, the one with ceil(b / dp) requests.  The memory
+     * bound is per replica: "Max Batch Size = Maximum Parallelism / Data Parallelism" (Sec. 3.2 Step 1). */
+    u64 dp = s->dp ? s->dp[p.t] : 1;
+    u64 b = ceil_div(b_all, dp);
 
     /* Step 1: what fits */
     u64 usable = usable_bytes(s->hw_mem[p.h], reserve);
@@ -259,16 +265,16 @@ static void closed_form_one(const ospace *s, u64 idx, u64 j, int time_model, int
     }
     o->ttft[j] = T_pre; o->ttft_p50[j] = T_pre; o->ttft_p99[j] = T_pre;
     o->latency[j] = T_pre + T_dec;
-    o->cost_per_hr[j] = r.price * (double)t;
+    o->cost_per_hr[j] = r.price * (double)mul(t, dp);        /* every GPU of every replica is paid for */
     if (n > 0) {
         o->tpot[j] = T_dec / (double)n;
-        o->thr_decode[j] = (double)mul(b, n) / T_dec;
+        o->thr_decode[j] = (double)mul(b_all, n) / T_dec;     /* all replicas decode at once (Sec. 3.2: N x T_single) */
         o->cost_per_token[j] = (o->cost_per_hr[j] / 3600.0) / o->thr_decode[j];
     } else {
         o->tpot[j] = 0.0; o->thr_decode[j] = 0.0; o->cost_per_token[j] = INFINITY;
     }
     o->n_iters[j] = 1 + n;
-    o->n_req_iters[j] = mul(b, 1 + n);
+    o->n_req_iters[j] = mul(b_all, 1 + n);
 }
 
 /* ---- trace-driven continuous batching with paged KV and preempt-and-recompute --------------- */
@@ -469,6 +475,10 @@ int oracle_simulate(const ospace *s, const otrace *tr, u64 first, u64 count, u64
     }
     for (u32 i = 0; i < s->n_f; i++) if (s->fw_i[4 * i + 1] == 0 || s->fw_i[4 * i + 2] > 1000) return -1;
     for (u32 i = 0; i < s->n_b; i++) if (s->batch[i] == 0) return -1;
+    if (s->dp) for (u32 i = 0; i < s->n_t; i++) {
+        if (s->dp[i] == 0) return -1;
+        if (tr && s->dp[i] != 1) return -3;      /* the trace simulation models one replica */
+    }
     for (u32 i = 0; i < s->n_l; i++) if (s->pairs[2 * i] == 0 || s->pairs[2 * i + 1] == 0) return -1;
     if (tr) for (u64 i = 0; i < tr->n; i++) {
         if (i && tr->arrival[i] < tr->arrival[i - 1]) return -1;

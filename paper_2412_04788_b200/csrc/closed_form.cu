@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(MEM_THREADS) k_closed_form_memory(DSpace s, gu
         const u32 tl = active ? tl_raw : 0;                  // idle lanes still take part in the exchange below
         const u32 tpos = tl / s.n_l, lpos = tl % s.n_l;
         const DModel m = s.models[mpos];
-        const u32 t = s.tp[tpos];
+        const u32 t = s.tp[tpos], dp = s.dp[tpos];
         const MemInfo mi = mem_info(m, t);
         const u32 st_base = ((m.nh & (t - 1)) != 0 || (m.nkv & (t - 1)) != 0) ? 4u : 0u;
         const ulonglong2 hm = __ldg(s.hfmem + hf);
@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(MEM_THREADS) k_closed_form_memory(DSpace s, gu
         u64 j = ((u64)mpos * n_hf + hf) * ((u64)s.n_b * n_tl) + tl;
         if (active) {
             for (u32 bi = 0; bi < s.n_b; bi++, j += n_tl) {
-                const u64 b = __ldg(s.batch + bi);
+                const u64 b = replica_batch(__ldg(s.batch + bi), dp);
                 const u32 sa = st0 | (b > bmax[0] ? 2u : 0u), sb = st0 | (b > bmax[1] ? 2u : 0u);
                 if (o.status) __stcs(reinterpret_cast<unsigned short *>(o.status + j), (unsigned short)(sa | (sb << 8)));
                 if (o.bmax) __stcs(reinterpret_cast<uint2 *>(o.bmax + j), bm);

@@ -99,7 +99,7 @@ static int check_trace_overflow(const guide_space &s, const guide_trace &t) {
 
 // Derived per-model quantities and the reciprocal rates of every hardware x framework pair.
 __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *gh, u32 n_h, const guide_fw *gf,
-                               u32 n_f, const u32 *tp, u32 n_t, DModel *dm, DRate *dr, double *cost_hr,
+                               u32 n_f, const u32 *tp, const u32 *dp, u32 n_t, DModel *dm, DRate *dr, double *cost_hr,
                                double *cost_sec, ulonglong2 *hfmem, double *rate10) {
     const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n_m) {
@@ -136,7 +136,7 @@ __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *g
         for (int k = 0; k < 3; k++) { q[k] = r.inv_c[k]; q[3 + k] = r.inv_m[k]; }
         q[6] = r.inv_comm; q[7] = r.clat; q[8] = r.tovh; q[9] = r.flash ? 1.0 : 0.0;
         for (u32 k = 0; k < n_t; k++) {
-            const double c = h.price_per_hr * (double)tp[k];
+            const double c = h.price_per_hr * (double)((u64)tp[k] * dp[k]);      // every GPU of every replica
             cost_hr[i * n_t + k] = c;
             cost_sec[i * n_t + k] = c / 3600.0;
         }
@@ -186,12 +186,13 @@ static std::vector<u32> plane_orders(const guide_space &s) {
         const double kv2 = 2.0 * m.n_layers * Dkv * m.kv_bytes;
         for (size_t q = 0; q < n_four; q++) {
             const u32 t = s.tp[(4 * q) / n_l];
+            const double b_rep = std::ceil(b_ref / (double)s.dp[(4 * q) / n_l]);   // one replica's share
             const bool bad = (m.n_heads % t) != 0 || (m.n_kv_heads % t) != 0;
             double best = INFINITY;
             for (size_t u = 0; u < 4 && !bad; u++) {
                 const guide_len_pair &pr = s.pairs[(4 * q + u) % n_l];
                 const double S = std::ceil(((double)pr.lin + pr.lout) / blk) * blk;
-                best = std::min(best, wbytes / t + b_ref * S * (kv2 / t));
+                best = std::min(best, wbytes / t + b_rep * S * (kv2 / t));
             }
             key[q] = best;
         }
@@ -219,7 +220,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
     const size_t o_gm = take(n_m * sizeof(guide_model)), o_gh = take(n_h * sizeof(guide_hw)),
                  o_gf = take(n_f * sizeof(guide_fw)), o_dm = take(n_m * sizeof(DModel)),
                  o_dr = take(n_h * n_f * sizeof(DRate)), o_b = take(s->batch.size() * 4),
-                 o_t = take(s->tp.size() * 4), o_p = take(s->pairs.size() * 8),
+                 o_t = take(s->tp.size() * 4), o_d = take(s->tp.size() * 4), o_p = take(s->pairs.size() * 8),
                  o_ch = take(n_h * n_f * s->tp.size() * 8), o_cs = take(n_h * n_f * s->tp.size() * 8),
                  o_hm = take(n_h * n_f * 16), o_hs = take(n_h * n_f * sizeof(HfSorted)),
                  o_po = take(std::max<size_t>(n_m * (s->tp.size() * s->pairs.size() / 4), 1) * 4),
@@ -235,6 +236,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
     put(o_gf, s->fw.data(), n_f * sizeof(guide_fw));
     put(o_b, s->batch.data(), s->batch.size() * 4);
     put(o_t, s->tp.data(), s->tp.size() * 4);
+    put(o_d, s->dp.data(), s->dp.size() * 4);
     put(o_p, s->pairs.data(), s->pairs.size() * 8);
     const std::vector<HfSorted> hf_sorted = sorted_pairs(*s);
     const std::vector<u32> plane_order = plane_orders(*s);
@@ -245,7 +247,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
         k_build_tables<<<(n + 127) / 128, 128>>>((const guide_model *)(blob + o_gm), (u32)n_m,
                                                  (const guide_hw *)(blob + o_gh), (u32)n_h,
                                                  (const guide_fw *)(blob + o_gf), (u32)n_f,
-                                                 (const u32 *)(blob + o_t), (u32)s->tp.size(),
+                                                 (const u32 *)(blob + o_t), (const u32 *)(blob + o_d), (u32)s->tp.size(),
                                                  (DModel *)(blob + o_dm), (DRate *)(blob + o_dr),
                                                  (double *)(blob + o_ch), (double *)(blob + o_cs),
                                                  (ulonglong2 *)(blob + o_hm), (double *)(blob + o_r10));
@@ -260,6 +262,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
     d.view.rates = (const DRate *)(blob + o_dr);
     d.view.batch = (const u32 *)(blob + o_b);
     d.view.tp = (const u32 *)(blob + o_t);
+    d.view.dp = (const u32 *)(blob + o_d);
     d.view.pairs = (const uint2 *)(blob + o_p);
     d.view.cost_hr = (const double *)(blob + o_ch);
     d.view.cost_sec = (const double *)(blob + o_cs);
@@ -389,8 +392,13 @@ int guide_space_create(const guide_space_desc *d, guide_space **out) {
     s->fw.assign(d->fw, d->fw + d->n_fw);
     s->batch.assign(d->batch, d->batch + d->n_batch);
     s->tp.assign(d->tp, d->tp + d->n_tp);
+    if (d->dp) s->dp.assign(d->dp, d->dp + d->n_tp); else s->dp.assign(d->n_tp, 1u);
     s->pairs.assign(d->pairs, d->pairs + d->n_pairs);
     int rc = GUIDE_OK;
+    for (uint32_t v : s->dp) {
+        if (!v || v > 65536) { rc = fail(GUIDE_ERR_INVALID, "data-parallel degree %u is outside 1..65536", v); break; }
+        s->max_dp = std::max(s->max_dp, v);
+    }
     for (uint32_t v : s->tp) {
         if (!pow2(v) || v > 1024) { rc = fail(GUIDE_ERR_UNSUPPORTED, "TP degree %u is not a power of two in 1..1024", v); break; }
         s->max_tp = std::max(s->max_tp, v);
@@ -475,6 +483,7 @@ int guide_space_decode(const guide_space *s, uint64_t idx, guide_config *o) {
     o->hw = (uint32_t)(idx % s->hw.size()); idx /= s->hw.size();
     o->model = (uint32_t)idx;
     o->batch = s->batch[o->batch_pos];
+    o->dp = s->dp[o->tp_pos];
     o->tp = s->tp[o->tp_pos];
     o->lin = s->pairs[o->pair_pos].lin;
     o->lout = s->pairs[o->pair_pos].lout;
@@ -539,6 +548,9 @@ int guide_simulate(const guide_space *space_c, const guide_trace *trace_c, const
     if (!trace && (out->req_ttft || out->req_tpot))
         return fail(GUIDE_ERR_INVALID, "per-request outputs need a trace");
     if (trace) {
+        if (space->max_dp > 1)
+            return fail(GUIDE_ERR_UNSUPPORTED, "the trace simulation models one replica: the space has a data-parallel degree of %u",
+                        space->max_dp);
         if (space->max_batch > GUIDE_TRACE_MAX_BATCH)
             return fail(GUIDE_ERR_UNSUPPORTED, "the trace kernel keeps at most %u requests resident; the batch axis goes to %u",
                         GUIDE_TRACE_MAX_BATCH, space->max_batch);

@@ -46,6 +46,7 @@ struct DSpace {
     const DModel *models;
     const DRate *rates;          // [n_h * n_f]
     const u32 *batch, *tp;
+    const u32 *dp;               // [n_t]: data-parallel degree that goes with tp[i] (Sec. 3.5.2)
     const uint2 *pairs;          // (lin, lout)
     const double *cost_hr;       // [n_h * n_f][n_t]: price x TP degree
     const double *cost_sec;      // [n_h * n_f][n_t]: (price x TP degree) / 3600
@@ -296,6 +297,10 @@ __device__ __forceinline__ void set_infeasible(Metrics &o) {
 }
 
 // status and B_max of a closed-form config
+// Sec. 3.2 Step 1: with data parallelism the batch is shared out over dp replicas; the slowest one
+// (the one with the rounded-up share) sets the time and the memory need.
+__device__ __forceinline__ u32 replica_batch(u32 b, u32 dp) { return dp == 1 ? b : (b + dp - 1) / dp; }
+
 __device__ __forceinline__ u32 closed_form_feasibility(const DModel &m, const DRate &r, const MemInfo &mi, u32 t,
                                                        u32 b, u32 lin, u32 lout, u32 &bmax_out) {
     const u64 S = (u64)lin + lout;
@@ -315,7 +320,7 @@ __device__ __forceinline__ void closed_form_metrics(double t_pre, double t_dec, 
     const double inf = __longlong_as_double(0x7FF0000000000000LL);
     o.ttft = t_pre;
     o.latency = t_pre + t_dec;
-    o.cost_hr = cost_hr;                 // price x TP degree
+    o.cost_hr = cost_hr;                 // price x TP degree x DP degree
     if (n > 0) {
         o.tpot = t_dec / (double)n;
         o.thr = cvt((u64)b * n) / t_dec;
@@ -333,7 +338,8 @@ template <int TIME_SUM>
 __device__ __forceinline__ void closed_form_eval(const DSpace &s, const Cfg &c, int tp_model, Metrics &o) {
     const DModel m = s.models[c.m];
     const DRate &r = s.rates[c.h * s.n_f + c.f];
-    const u32 t = s.tp[c.t], b = s.batch[c.b];
+    const u32 t = s.tp[c.t], b_all = s.batch[c.b];
+    const u32 b = replica_batch(b_all, s.dp[c.t]);   // each of the dp replicas serves its share of the batch
     const uint2 pr = s.pairs[c.l];
     const u32 lin = pr.x, lout = pr.y;
     const MemInfo mi = mem_info(m, t);
@@ -357,7 +363,7 @@ __device__ __forceinline__ void closed_form_eval(const DSpace &s, const Cfg &c, 
         t_dec = eval_phase<TIME_SUM>(k, r, Nd, lf);
     }
     const u32 ci = (c.h * s.n_f + c.f) * s.n_t + c.t;
-    closed_form_metrics(t_pre, t_dec, b, n, s.cost_hr[ci], s.cost_sec[ci], o);
+    closed_form_metrics(t_pre, t_dec, b_all, n, s.cost_hr[ci], s.cost_sec[ci], o);
 }
 
 }  // namespace guide

@@ -102,7 +102,8 @@ __device__ __forceinline__ void model_walk(const DSpace &s, int tp_model, u32 n_
         const u32 tl = __ldg(s.plane_order + (size_t)mpos * n_four + rank) * 4 + u;
         const u32 tpos = tl / s.n_l, lpos = tl % s.n_l;
         const DModel *mp = s.models + mpos;
-        const u32 t = s.tp[tpos], b = s.batch[bpos];
+        const u32 t = s.tp[tpos], b_all = s.batch[bpos];
+        const u32 b = replica_batch(b_all, s.dp[tpos]);
         const u32 nh = mp->nh, nkv = mp->nkv;
         if ((nh & (t - 1)) != 0 || (nkv & (t - 1)) != 0) continue;          // the foursome shares its TP degree: nothing fits
         const uint2 pr = s.pairs[lpos];
@@ -161,13 +162,13 @@ __device__ __forceinline__ void model_walk(const DSpace &s, int tp_model, u32 n_
                     cost_hr = __ldg(s.cost_hr + ci);
                     if (n > 0) {
                         tpot = t_dec / (double)n;
-                        thr = cvt((u64)b * n) / t_dec;
+                        thr = cvt((u64)b_all * n) / t_dec;
                         cost_tok = __ldg(s.cost_sec + ci) / thr;
                     } else {
                         tpot = 0.0; thr = 0.0; cost_tok = inf;
                     }
                     n_iters = 1 + (u64)n;
-                    n_req_iters = (u64)b * (1 + (u64)n);
+                    n_req_iters = (u64)b_all * (1 + (u64)n);
                 }
                 emit(fits, vote, lane, j0 + (u64)e.hf * stride_hf, latency, ttft, tpot, thr, cost_hr, cost_tok, n_iters, n_req_iters);
             }

@@ -40,7 +40,8 @@ __device__ __forceinline__ void tiled_visit(const DSpace &s, const Range &r, int
     const u32 hf0 = blockIdx.y * hf_chunk;
 
     const DModel m = s.models[mpos];
-    const u32 t = s.tp[tpos], b = s.batch[bpos];
+    const u32 t = s.tp[tpos], b_all = s.batch[bpos];
+    const u32 b = replica_batch(b_all, s.dp[tpos]);
     const uint2 pr = s.pairs[lpos];
     const u32 lin = pr.x, lout = pr.y, n = lout - 1;
     const MemInfo mi = mem_info(m, t);
@@ -74,7 +75,7 @@ __device__ __forceinline__ void tiled_visit(const DSpace &s, const Range &r, int
     rq.block = 0; rq.bytes = 1; rq.inv = 1.0; rq.small = false;
     const u64 S = (u64)lin + lout;
     const double nd = (double)n;
-    const double tok = cvt((u64)b * n);
+    const double tok = cvt((u64)b_all * n);
     const u32 heads_bad = ((m.nh & (t - 1)) != 0 || (m.nkv & (t - 1)) != 0) ? 4u : 0u;   // t is a power of two
     const u32 hf_end = min(hf_chunk, n_hf > hf0 ? n_hf - hf0 : 0u);
 
@@ -117,7 +118,7 @@ __device__ __forceinline__ void tiled_visit(const DSpace &s, const Range &r, int
                     out.tpot = 0.0; out.thr = 0.0; out.cost_tok = inf;
                 }
                 out.n_iters = 1 + (u64)n;
-                out.n_req_iters = (u64)b * (1 + (u64)n);
+                out.n_req_iters = (u64)b_all * (1 + (u64)n);
             }
         }
         emit(valid, j, out);

@@ -62,11 +62,12 @@ class LenPair(C.Structure):
 class SpaceDesc(C.Structure):
     _fields_ = [("models", C.POINTER(Model)), ("n_models", C.c_uint32), ("hw", C.POINTER(Hw)), ("n_hw", C.c_uint32),
                 ("fw", C.POINTER(Fw)), ("n_fw", C.c_uint32), ("batch", C.POINTER(C.c_uint32)), ("n_batch", C.c_uint32),
-                ("tp", C.POINTER(C.c_uint32)), ("n_tp", C.c_uint32), ("pairs", C.POINTER(LenPair)), ("n_pairs", C.c_uint32)]
+                ("tp", C.POINTER(C.c_uint32)), ("n_tp", C.c_uint32), ("pairs", C.POINTER(LenPair)), ("n_pairs", C.c_uint32),
+                ("dp", C.POINTER(C.c_uint32))]
 
 
 class Config(C.Structure):
-    _fields_ = [(k, C.c_uint32) for k in ("model", "hw", "fw", "batch_pos", "tp_pos", "pair_pos", "batch", "tp", "lin", "lout")]
+    _fields_ = [(k, C.c_uint32) for k in ("model", "hw", "fw", "batch_pos", "tp_pos", "pair_pos", "batch", "tp", "lin", "lout", "dp")]
 
 
 class SimOpts(C.Structure):
@@ -150,7 +151,12 @@ class Space:
         batch = (C.c_uint32 * len(space["batch"]))(*[int(v) for v in space["batch"]])
         tp = (C.c_uint32 * len(space["tp"]))(*[int(v) for v in space["tp"]])
         pairs = (LenPair * len(space["pairs"]))(*[LenPair(int(a), int(b)) for a, b in space["pairs"]])
-        desc = SpaceDesc(models, len(models), hws, len(hws), fws, len(fws), batch, len(batch), tp, len(tp), pairs, len(pairs))
+        dp = None                                   # NULL: every data-parallel degree is 1
+        if space.get("dp") is not None:
+            if len(space["dp"]) != len(space["tp"]):
+                raise ValueError("dp and tp describe the same axis: one data-parallel degree per TP degree")
+            dp = (C.c_uint32 * len(space["dp"]))(*[int(v) for v in space["dp"]])
+        desc = SpaceDesc(models, len(models), hws, len(hws), fws, len(fws), batch, len(batch), tp, len(tp), pairs, len(pairs), dp)
         self.handle = C.c_void_p()
         _check(lib().guide_space_create(C.byref(desc), C.byref(self.handle)))
 

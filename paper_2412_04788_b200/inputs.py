@@ -183,8 +183,23 @@ def decode_index(space, idx: int):
     return tuple(reversed(pos))
 
 
-def _space(models, hw, hw_mem, fw_f, fw_i, batch, tp, pairs):
-    return {
+def hybrid_axis(n_gpus: int):
+    """Every (dp, tp) with tp a power of two and dp * tp <= n_gpus, dp slowest: the candidate
+    parallel configurations of the hybrid enumeration.  Returns (dp list, tp list)."""
+    dps, tps = [], []
+    for dp in range(1, n_gpus + 1):
+        tp = 1
+        while dp * tp <= n_gpus:
+            dps.append(dp)
+            tps.append(tp)
+            tp *= 2
+    return dps, tps
+
+
+def _space(models, hw, hw_mem, fw_f, fw_i, batch, tp, pairs, dp=None):
+    extra = {} if dp is None else {"dp": np.ascontiguousarray(dp, dtype=np.uint32)}
+    assert dp is None or len(dp) == len(tp)
+    return {**extra,
         "models": np.ascontiguousarray(models, dtype=np.uint32),
         "hw": np.ascontiguousarray(hw, dtype=np.float64),
         "hw_mem": np.ascontiguousarray(hw_mem, dtype=np.uint64),
@@ -298,3 +313,19 @@ def workload(k: int, scale: float = 1.0, trace_scale: float | None = None):
                 "topk": {"key": "cost_per_token", "k": 64},
                 "pareto": {"x": "latency", "y": "cost_per_hr"}}
     raise ValueError("workload must be 1..5")
+
+
+def hybrid_workload(n_gpus: int = 8, n_hw: int = 8, n_fw: int = 3, seed_offset: int = 20):
+    """Closed-form sweep whose parallelism axis is every (dp, tp) pair under a budget of n_gpus:
+    the eight model shapes, seeded hardware and frameworks, batch sizes that are and are not
+    multiples of the replica counts, the 8 x 8 length grid."""
+    seed = SEED_BASE + seed_offset
+    models = models_from_shapes(SHAPES_8)
+    hw, mem = seeded_hw(seed, n_hw, mem_choices=[24, 48, 80, 192])
+    fw_f, fw_i = seeded_fw(seed, n_fw)
+    dp, tp = hybrid_axis(n_gpus)
+    space = _space(models, hw, mem, fw_f, fw_i, [1, 2, 3, 5, 8, 16, 31, 64, 100, 256, 509, 1024], tp,
+                   pairs_grid(LEN_GRID_8, LEN_GRID_8), dp=dp)
+    return {"name": f"hybrid-{n_gpus}", "space": space, "trace": None, "constraints": {},
+            "topk": {"key": "cost_per_token", "k": 64},
+            "pareto": {"x": "latency", "y": "cost_per_hr"}}

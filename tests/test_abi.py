@@ -51,6 +51,17 @@ def test_space_size_and_decode_follow_the_mixed_radix_order():
     for k in range(2, 6):
         w = I.workload(k)
         assert guide.Space(w["space"]).size == I.space_size(w["space"])
+    # the data-parallel degree rides on the TP axis: 1 everywhere when none is given
+    assert {sp.decode(i)["dp"] for i in range(504)} == {1}
+    w = I.hybrid_workload(8)["space"]
+    hy = guide.Space(w)
+    assert hy.size == I.space_size(w) == 8 * 8 * 3 * 12 * 15 * 64
+    for idx in (0, 63, 64, 15 * 64 - 1, 1234567):
+        got = hy.decode(idx)
+        assert (got["dp"], got["tp"]) == (int(w["dp"][got["tp_pos"]]), int(w["tp"][got["tp_pos"]]))
+        assert got["dp"] * got["tp"] <= 8
+    with pytest.raises(ValueError):
+        guide.Space(dict(w, dp=w["dp"][:3]))
 
 
 def test_space_validation():
@@ -59,6 +70,8 @@ def test_space_validation():
         (dict(batch=np.array([0, 1], np.uint32)), guide.GUIDE_ERR_INVALID),
         (dict(pairs=np.array([[0, 4]], np.uint32)), guide.GUIDE_ERR_INVALID),
         (dict(batch=np.zeros(0, np.uint32)), guide.GUIDE_ERR_INVALID),                 # empty axis
+        (dict(dp=np.array([1, 0, 1], np.uint32)), guide.GUIDE_ERR_INVALID),            # no replicas
+        (dict(dp=np.array([1, 1, 65537], np.uint32)), guide.GUIDE_ERR_INVALID),
     ]
     for over, code in bad:
         with pytest.raises(guide.GuideError) as e:

@@ -56,3 +56,15 @@ def test_decode_index_order():
     w5 = I.workload(5)
     assert len(set(w5["space"]["batch"].tolist())) == 16
     assert list(w5["space"]["batch"]) == sorted(w5["space"]["batch"])
+
+
+def test_hybrid_axis_enumerates_the_gpu_budget():
+    dp, tp = I.hybrid_axis(8)
+    pairs = set(zip(dp, tp))
+    assert len(pairs) == len(dp) == 15
+    want = {(d, t) for d in range(1, 9) for t in (1, 2, 4, 8) if d * t <= 8}
+    assert pairs == want
+    assert I.hybrid_axis(1) == ([1], [1])
+    w = I.hybrid_workload(8)["space"]
+    assert w["dp"].dtype == np.uint32 and len(w["dp"]) == len(w["tp"])
+    assert (len(w["tp"]) * len(w["pairs"])) % 4 == 0

@@ -11,14 +11,14 @@ from paper_2412_04788_b200 import inputs as I
 
 
 def toy_space(golden, mem, kv_block, batch, pairs=((4, 3),), tp=(1,), e=None, t_ovh=0.0, flash=1, reserve=0,
-              layers=None):
+              layers=None, dp=None):
     model = list(golden["model"])
     if layers:
         model[0] = layers
     fw_f = list(e) if e is not None else [1.0] * 7
     return I._space(np.array([model]), np.array([golden["hw"]]), np.array([mem]),
                     np.array([fw_f + [t_ovh]]), np.array([[flash, kv_block, reserve, 0]]),
-                    list(batch), list(tp), [list(p) for p in pairs])
+                    list(batch), list(tp), [list(p) for p in pairs], dp=None if dp is None else list(dp))
 
 
 def test_weight_count_and_kv_bytes(golden):
@@ -101,6 +101,68 @@ def test_closed_form_toy(golden):
     assert out["cost_per_hr"][0] == 1.0 and np.isinf(out["cost_per_hr"][1])
     assert out["cost_per_token"][0] == (1.0 / 3600.0) / out["thr_decode"][0]
     assert out["n_iters"].tolist() == [3, 0] and out["n_req_iters"].tolist() == [6, 0]
+
+
+def test_data_parallel_replicas(golden):
+    """Sec. 3.2 Step 1 (the batch a replica sees is the whole batch over the DP degree) and the
+    hybrid rule of Sec. 3.5.2 - 3.5.3: dp replicas of the hand-worked batch-2 case."""
+    want = golden["closed_form_b2_Lin4_Lout3"]["t1"]
+    sp = toy_space(golden, 10**6, 1, [4, 3], tp=(1, 1), dp=(2, 1))
+    out = oracle.simulate(sp)
+    assert out["status"].tolist() == [0, 0, 0, 0]
+    num, den = want["thr_decode_num"], want["thr_decode_den"]        # 2 requests x 2 steps over the decode time
+    for c, b in ((0, 4), (2, 3)):                                     # dp = 2: each replica runs at most 2 requests
+        assert out["ttft"][c] == want["ttft"] and out["latency"][c] == want["latency"] and out["tpot"][c] == want["tpot"]
+        assert out["thr_decode"][c] == (num * b / 2) / den            # every replica's tokens count
+        assert out["cost_per_hr"][c] == 2.0                           # price 1.0 x 1 GPU x 2 replicas
+        assert out["cost_per_token"][c] == (2.0 / 3600.0) / out["thr_decode"][c]
+        assert out["n_iters"][c] == 3 and out["n_req_iters"][c] == 3 * b
+    # dp = 1 next to it: four (three) requests on one replica take longer than two
+    assert out["latency"][1] > out["latency"][3] > want["latency"] and out["cost_per_hr"][1] == 1.0
+    # an explicit axis of ones is the same as none
+    ones = oracle.simulate(toy_space(golden, 10**6, 1, [4, 3], tp=(1, 1), dp=(1, 1)))
+    none = oracle.simulate(toy_space(golden, 10**6, 1, [4, 3], tp=(1, 1)))
+    for k in ones:
+        assert np.array_equal(ones[k], none[k]), k
+    # memory is per replica: room for exactly two requests of 4 + 3 tokens
+    mem = oracle.weight_bytes_per_gpu(golden["model"], 1) + 2 * 7 * oracle.kv_bytes_per_token(golden["model"], 1)
+    out = oracle.simulate(toy_space(golden, mem, 1, [4, 5], tp=(1, 1), dp=(1, 2)))
+    assert out["bmax"].tolist() == [2, 2, 2, 2]
+    assert out["status"].tolist() == [oracle.ST_KV, 0, oracle.ST_KV, oracle.ST_KV]     # ceil(5 / 2) = 3 > 2
+    # general degrees against the single-replica run of the share: times bit for bit
+    hw, mem = I.seeded_hw(9, 2, mem_gb=[80, 192])
+    fw_f, fw_i = I.seeded_fw(9, 2)
+    models = I.models_from_shapes(I.SHAPES_8[:3])
+    pairs = [(128, 64), (500, 1), (33, 17)]
+    batch, degrees = [1, 7, 24, 100], [1, 2, 3, 5, 8]
+    shares = sorted({-(-b // d) for b in batch for d in degrees})
+    for t in (1, 2):
+        hyb = oracle.simulate(I._space(models, hw, mem, fw_f, fw_i, batch, [t] * len(degrees), pairs, dp=degrees))
+        one = oracle.simulate(I._space(models, hw, mem, fw_f, fw_i, shares, [t], pairs))
+        H = {k: v.reshape(3, 2, 2, len(batch), len(degrees), 3) for k, v in hyb.items()}
+        O = {k: v.reshape(3, 2, 2, len(shares), 1, 3) for k, v in one.items()}
+        for bi, b in enumerate(batch):
+            for di, d in enumerate(degrees):
+                si = shares.index(-(-b // d))
+                for k in ("status", "bmax", "latency", "ttft", "tpot", "n_iters"):
+                    assert np.array_equal(H[k][:, :, :, bi, di], O[k][:, :, :, si, 0]), (k, b, d)
+                ok = H["status"][:, :, :, bi, di] == 0
+                n = np.array([p[1] - 1 for p in pairs])
+                t_dec = (O["latency"] - O["ttft"])[:, :, :, si, 0]
+                thr = H["thr_decode"][:, :, :, bi, di]
+                dec = ok & (n > 0)                                    # a single output token has no decode stage
+                with np.errstate(invalid="ignore"):
+                    assert np.allclose(thr[dec], ((b * n) / t_dec)[dec], rtol=1e-12, atol=0)
+                assert np.all(thr[ok & (n == 0)] == 0.0)
+                assert np.array_equal(H["cost_per_hr"][:, :, :, bi, di][ok], (O["cost_per_hr"][:, :, :, si, 0] * d)[ok]) \
+                    or np.allclose(H["cost_per_hr"][:, :, :, bi, di][ok], (O["cost_per_hr"][:, :, :, si, 0] * d)[ok], rtol=1e-15)
+                assert np.array_equal(H["n_req_iters"][:, :, :, bi, di][ok], np.broadcast_to(b * (1 + n), ok.shape)[ok])
+    # no replica split of a trace, no zero degree
+    tr = {"arrival": np.array([0.0, 1.0]), "in_len": np.zeros(2, np.uint32), "out_len": np.zeros(2, np.uint32)}
+    with pytest.raises(ValueError, match="data parallelism"):
+        oracle.simulate(toy_space(golden, 10**6, 1, [2], dp=(2,)), tr)
+    with pytest.raises(ValueError):
+        oracle.simulate(toy_space(golden, 10**6, 1, [2], dp=(0,)))
 
 
 def test_closed_form_aggregates_match_token_loops(golden):
