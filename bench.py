@@ -248,6 +248,19 @@ def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full, fraction
                             "simulate_frac_of_hbm": BYTES_SIM * n / t_sim / 1e6 / hbm_peak,
                             "kernel_launches": 2 + 6 + 5 + 5 + 4}
             del p
+        elif k in (6, 7):
+            # the (dp, tp) sweep under a budget of 8 GPUs (whole-space kernels) and workload 2 with
+            # frameworks that process prompts in sub-batches / segments (one thread per config)
+            w = inputs.hybrid_workload(8) if k == 6 else inputs.chunked_workload(scale=1.0)
+            p = ClosedFormPath(guide, torch, w["space"], w["constraints"], w["topk"]["key"], w["topk"]["k"])
+            n = p.n
+            t_sim = time_call(torch, p.simulate, flush=flush)[0]
+            t_kf = time_call(torch, lambda: p.topk(True), flush=flush)[0]
+            res[w["name"]] = {"configs": n, "simulate_ms": t_sim, "simulate_configs_per_s": n / t_sim * 1e3,
+                              "simulate_write_gbs": BYTES_SIM * n / t_sim / 1e6,
+                              "simulate_frac_of_hbm": BYTES_SIM * n / t_sim / 1e6 / hbm_peak,
+                              "fused_topk_ms": t_kf, "found": int(p.cnt.item())}
+            del p
         torch.cuda.empty_cache()
     return res
 
@@ -444,7 +457,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--extras", default="1,2,3,4,5", help="other workloads to time after the main loop ('' = none)")
+    ap.add_argument("--extras", default="1,2,3,4,5,6,7", help="other workloads to time after the main loop ('' = none)")
     ap.add_argument("--main-fraction", action="store_true",
                     help="apply --trace-fraction to the main workload's hardware axis too (small cases for profiler captures)")
     ap.add_argument("--full", action="store_true", help="(kept for compatibility: workloads 3 and 4 now always run whole)")

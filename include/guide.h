@@ -76,6 +76,16 @@ typedef struct guide_fw {
     uint32_t kv_block;      /* tokens per KV block (fixed-granularity paging, Sec. 2.4.1); 1 = unpaged */
     uint32_t reserve_permille; /* thousandths of device memory kept back */
     uint32_t policy;        /* GUIDE_POLICY_PREFILL_FIRST */
+    /* Prompt processing in pieces (closed form only; a trace with either set is GUIDE_ERR_UNSUPPORTED):
+     * split_size: requests per prompt sub-batch (Sec. 3.3.1: the batch is divided into sub-batches of
+     *   split_size, the remainder forming one more); 0 or >= the batch = the whole batch at once.
+     * seg_tokens: tokens per prompt segment (Sec. 3.3.2: ceil(Lin / segment) splits, base value times
+     *   tuning factor supplied as one number); 0 or >= Lin = the whole prompt at once.
+     * Every (sub-batch, segment) pass reads the weights and pays t_ovh; a segment's tokens attend
+     * their prompt up to the end of that segment; only the last segment runs the LM head.  TTFT is
+     * the time of all passes, n_iters counts them, n_req_iters = batch x (segments + Lout - 1). */
+    uint32_t split_size;
+    uint32_t seg_tokens;
 } guide_fw;
 
 typedef struct guide_len_pair { uint32_t lin, lout; } guide_len_pair;

@@ -40,7 +40,7 @@ class _Space(C.Structure):
                 ("batch", C.c_void_p), ("n_b", C.c_uint32),
                 ("tp", C.c_void_p), ("n_t", C.c_uint32),
                 ("pairs", C.c_void_p), ("n_l", C.c_uint32),
-                ("dp", C.c_void_p)]
+                ("dp", C.c_void_p), ("fw_chunk", C.c_void_p)]
 
 
 class _Trace(C.Structure):
@@ -104,7 +104,8 @@ def _space_struct(space):
     return _Space(_p(space["models"]), len(space["models"]), _p(space["hw"]), _p(space["hw_mem"]), len(space["hw"]),
                   _p(space["fw_f"]), _p(space["fw_i"]), len(space["fw_f"]), _p(space["batch"]), len(space["batch"]),
                   _p(space["tp"]), len(space["tp"]), _p(space["pairs"]), len(space["pairs"]),
-                  _p(space["dp"]) if space.get("dp") is not None else None)
+                  _p(space["dp"]) if space.get("dp") is not None else None,
+                  _p(space["fw_chunk"]) if space.get("fw_chunk") is not None else None)
 
 
 def simulate(space, trace=None, first=0, count=None, stride=1, time_model=TIME_MAX, tp_model=TP_EXPLICIT,
@@ -137,7 +138,7 @@ def simulate(space, trace=None, first=0, count=None, stride=1, time_model=TIME_M
     rc = lib().oracle_simulate(C.byref(sp), C.byref(ts) if ts is not None else None, first, count, stride,
                                time_model, tp_model, max_iters, C.byref(o), n_threads)
     if rc != 0:
-        why = {-1: "invalid input", -2: "64-bit overflow", -3: "data parallelism with a trace is not modelled"}.get(rc, "?")
+        why = {-1: "invalid input", -2: "64-bit overflow", -3: "data parallelism or prompt splitting with a trace is not modelled"}.get(rc, "?")
         raise ValueError(f"oracle_simulate failed: {rc} ({why})")
     return out
 

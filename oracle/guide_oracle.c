@@ -58,6 +58,8 @@ typedef struct {
     const u32 *tp; u32 n_t;
     const u32 *pairs; u32 n_l;             /* [n_l][2]: Lin Lout */
     const u32 *dp;                         /* [n_t] data-parallel degree of each entry of the parallelism axis; NULL = all 1 */
+    const u32 *fw_chunk;                   /* [n_f][2]: split_size (requests per prompt sub-batch), seg_tokens (prompt
+                                              segment length); 0 = no splitting; NULL = none anywhere */
 } ospace;
 
 typedef struct {
@@ -176,8 +178,10 @@ static double phase_time(const model_t *m, const rates_t *r, u64 tp, u64 T, u64 
     tk[9] = task_time(mul(2, mul(H, A)), 0, add(add(THa, kv_read), X), 0, t, ic[CLS_ATTN], im[CLS_ATTN], time_model);
     tk[10] = task_time(mul(5, mul(m->nh, A)), 0, mul(2, X), 0, t, ic[CLS_ATTN], im[CLS_ATTN], time_model);
     tk[11] = task_time(mul(2, mul(H, A)), 0, add(add(kv_read, THa), X), 0, t, ic[CLS_ATTN], im[CLS_ATTN], time_model);
-    tk[13] = task_time(mul(2, mul(mul(E, H), V)), 0, add(mul(R, mul(mul(H, V), wb)), mul(mul(E, V), ab)),
-                       mul(mul(E, H), ab), t, ic[CLS_LINEAR], im[CLS_LINEAR], time_model);
+    /* no sequence emits a token (a prompt segment that is not the last one): no LM head at all */
+    tk[13] = E == 0 ? 0.0
+                    : task_time(mul(2, mul(mul(E, H), V)), 0, add(mul(R, mul(mul(H, V), wb)), mul(mul(E, V), ab)),
+                                mul(mul(E, H), ab), t, ic[CLS_LINEAR], im[CLS_LINEAR], time_model);
 
     double S_fix = tk[1];
     for (int k = 2; k <= 8; k++) S_fix = S_fix + tk[k];
@@ -228,6 +232,24 @@ static void write_infeasible(const oout *o, u64 j) {
 
 /* ---- closed form: one prefill pass + an aggregated decode stage ----------------------------- */
 
+/*
+ * Prompt processing of one sub-batch of sb requests whose prompts are cut into segments of seg
+ * tokens (Sec. 3.3.2: number of splits = ceil(Lin / split size), the last one short): one pass per
+ * segment; its q tokens attend the done + q tokens of their own prompt seen so far, and only the
+ * last segment emits a token.  Every pass reads the weights and pays the iteration overhead.
+ */
+static double segmented_prefill(const model_t *m, const rates_t *r, u64 t, u64 sb, u64 Lin, u64 seg,
+                                int time_model, int tp_model) {
+    double sum = 0.0;
+    for (u64 done = 0; done < Lin; done += seg) {
+        u64 q = Lin - done < seg ? Lin - done : seg;
+        u64 T = mul(sb, q);
+        u64 E = done + q == Lin ? sb : 0;
+        sum = sum + phase_time(m, r, t, T, E, mul(T, done + q), mul(sb, done + q), 1, time_model, tp_model, NULL);
+    }
+    return sum;
+}
+
 static void closed_form_one(const ospace *s, u64 idx, u64 j, int time_model, int tp_model, const oout *o) {
     pos_t p = decode(s, idx);
     model_t m = load_model(s->models + 10 * p.m);
@@ -254,9 +276,15 @@ static void closed_form_one(const ospace *s, u64 idx, u64 j, int time_model, int
     o->bmax[j] = bmax > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)bmax;
     if (st) { write_infeasible(o, j); return; }
 
-    /* Step 2: the two stages */
-    double T_pre = phase_time(&m, &r, t, mul(b, Lin), b, mul(b, mul(Lin, Lin)), mul(b, Lin), 1,
-                              time_model, tp_model, NULL);
+    /* Step 2: the two stages.  Prompt processing (Sec. 3.3.1): the batch goes through in sub-batches
+     * of split_size requests, "any remaining portion of the batch forming an additional sub-batch";
+     * equal sub-batches take equal time.  Without splitting this is one pass over b x Lin tokens. */
+    u64 split = s->fw_chunk ? s->fw_chunk[2 * p.f] : 0, seg = s->fw_chunk ? s->fw_chunk[2 * p.f + 1] : 0;
+    if (split == 0 || split > b) split = b;
+    if (seg == 0 || seg > Lin) seg = Lin;
+    u64 n_full = b / split, rest = b % split, n_seg = ceil_div(Lin, seg);
+    double T_pre = (double)n_full * segmented_prefill(&m, &r, t, split, Lin, seg, time_model, tp_model);
+    if (rest) T_pre = T_pre + segmented_prefill(&m, &r, t, rest, Lin, seg, time_model, tp_model);
     u64 n = Lout - 1;                 /* the prefill pass emits token 1 */
     double T_dec = 0.0;
     if (n > 0) {
@@ -273,8 +301,8 @@ static void closed_form_one(const ospace *s, u64 idx, u64 j, int time_model, int
     } else {
         o->tpot[j] = 0.0; o->thr_decode[j] = 0.0; o->cost_per_token[j] = INFINITY;
     }
-    o->n_iters[j] = 1 + n;
-    o->n_req_iters[j] = mul(b_all, 1 + n);
+    o->n_iters[j] = add(mul(n_full + (rest != 0), n_seg), n);   /* passes of one replica */
+    o->n_req_iters[j] = mul(b_all, add(n_seg, n));
 }
 
 /* ---- trace-driven continuous batching with paged KV and preempt-and-recompute --------------- */
@@ -478,6 +506,9 @@ int oracle_simulate(const ospace *s, const otrace *tr, u64 first, u64 count, u64
     if (s->dp) for (u32 i = 0; i < s->n_t; i++) {
         if (s->dp[i] == 0) return -1;
         if (tr && s->dp[i] != 1) return -3;      /* the trace simulation models one replica */
+    }
+    if (s->fw_chunk && tr) for (u32 i = 0; i < 2 * s->n_f; i++) {
+        if (s->fw_chunk[i] != 0) return -3;      /* the trace simulation has the prompt-first policy only */
     }
     for (u32 i = 0; i < s->n_l; i++) if (s->pairs[2 * i] == 0 || s->pairs[2 * i + 1] == 0) return -1;
     if (tr) for (u64 i = 0; i < tr->n; i++) {

@@ -24,6 +24,34 @@ def prefill_aggregates(b: int, lin: int):
     return T, E, A, Cc
 
 
+def segment_passes(sb: int, lin: int, seg: int):
+    """One (T, E, A, C) per prompt segment of a sub-batch of sb requests (Sec. 3.3.2): the tokens of
+    a segment attend their prompt up to the end of that segment; the last segment emits a token."""
+    passes = []
+    done = 0
+    while done < lin:
+        q = min(seg, lin - done)
+        T = E = A = Cc = 0
+        for _seq in range(sb):
+            if done + q == lin:
+                E += 1
+            Cc += done + q
+            for _tok in range(q):
+                T += 1
+                A += done + q
+        passes.append((T, E, A, Cc))
+        done += q
+    return passes
+
+
+def sub_batches(b: int, split: int):
+    """Sec. 3.3.1: sub-batches of split requests, the remainder as one more."""
+    out = [split] * (b // split)
+    if b % split:
+        out.append(b % split)
+    return out
+
+
 def decode_aggregates(b: int, lin: int, lout: int):
     """(T, E, A, C, R) of the whole decode stage: steps 1..Lout-1, step j attends Lin + j tokens."""
     T = E = A = Cc = R = 0

@@ -177,7 +177,7 @@ static bool split_applies(const DSpace &s, Range r, const guide_outputs &o, Cons
     const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
     const u32 n_tl = s.n_t * s.n_l;
     if (r.first != 0 || r.count != total || total < (1u << 16)) return false;       // whole spaces only
-    if (s.n_l % 4 != 0 || n_tl < 32) return false;
+    if (s.n_l % 4 != 0 || n_tl < 32 || s.chunked) return false;
     if ((u64)s.n_m * ((n_tl + 255) / 256) * s.n_h * s.n_f > 0x7FFFFFFFull) return false;
     auto al = [](const void *p, uintptr_t a) { return ((uintptr_t)p % a) == 0; };
     const void *wide[] = {o.latency, o.ttft, o.ttft_p50, o.ttft_p99, o.tpot, o.thr_decode, o.cost_per_hr, o.cost_per_token,

@@ -130,6 +130,8 @@ __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *g
         r.usable = h.mem_bytes - (h.mem_bytes / 1000) * f.reserve_permille;
         r.flash = f.flash;
         r.kv_block = f.kv_block;
+        r.split = f.split_size;
+        r.seg = f.seg_tokens;
         dr[i] = r;
         hfmem[i] = make_ulonglong2(r.usable, (u64)r.kv_block);
         double *q = rate10 + (size_t)i * 10;
@@ -263,6 +265,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
     d.view.batch = (const u32 *)(blob + o_b);
     d.view.tp = (const u32 *)(blob + o_t);
     d.view.dp = (const u32 *)(blob + o_d);
+    d.view.chunked = s->chunked ? 1u : 0u;
     d.view.pairs = (const uint2 *)(blob + o_p);
     d.view.cost_hr = (const double *)(blob + o_ch);
     d.view.cost_sec = (const double *)(blob + o_cs);
@@ -439,6 +442,7 @@ int guide_space_create(const guide_space_desc *d, guide_space **out) {
         for (int k = 0; k < 3; k++) ok = ok && f.e_c[k] > 0 && f.e_m[k] > 0 && std::isfinite(f.e_c[k] + f.e_m[k]);
         if (!ok) rc = fail(GUIDE_ERR_INVALID, "framework profile %zu has a bad efficiency, kv_block or reserve", i);
         else if (f.policy != GUIDE_POLICY_PREFILL_FIRST) rc = fail(GUIDE_ERR_UNSUPPORTED, "framework profile %zu: unknown policy", i);
+        s->chunked = s->chunked || f.split_size || f.seg_tokens;
     }
     if (!rc) {
         u128 n = (u128)d->n_models * d->n_hw * d->n_fw * d->n_batch * d->n_tp * d->n_pairs;
@@ -551,6 +555,9 @@ int guide_simulate(const guide_space *space_c, const guide_trace *trace_c, const
         if (space->max_dp > 1)
             return fail(GUIDE_ERR_UNSUPPORTED, "the trace simulation models one replica: the space has a data-parallel degree of %u",
                         space->max_dp);
+        if (space->chunked)
+            return fail(GUIDE_ERR_UNSUPPORTED, "the trace simulation has the prompt-first policy only: a framework profile "
+                                               "sets split_size or seg_tokens");
         if (space->max_batch > GUIDE_TRACE_MAX_BATCH)
             return fail(GUIDE_ERR_UNSUPPORTED, "the trace kernel keeps at most %u requests resident; the batch axis goes to %u",
                         GUIDE_TRACE_MAX_BATCH, space->max_batch);

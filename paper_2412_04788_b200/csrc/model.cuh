@@ -31,6 +31,7 @@ struct DRate {
     double inv_c[3], inv_m[3], inv_comm, clat, tovh, price;
     u64 usable;   // MEM - (MEM/1000) * reserve_permille
     u32 flash, kv_block;
+    u32 split, seg;   // requests per prompt sub-batch, tokens per prompt segment (0: whole batch / prompt)
 };
 
 // one hardware x framework pair in the sorted walk of the model kernel
@@ -56,6 +57,7 @@ struct DSpace {
     const HfSorted *hf_sorted;   // [n_h * n_f]: the pairs grouped by KV block size, largest usable memory first
     const u32 *plane_order;      // [n_m][n_t * n_l / 4]: foursomes of the (TP, length) plane by growing memory need
     u32 n_m, n_h, n_f, n_b, n_t, n_l;
+    u32 chunked;                 // some framework splits prompt processing: only the flat evaluation handles that
 };
 
 struct DTrace {
@@ -316,7 +318,7 @@ __device__ __forceinline__ u32 closed_form_feasibility(const DModel &m, const DR
 
 // final metrics from the two stage times (Sec. 3.2: TTFT = prefill time, throughput; Sec. 5.1)
 __device__ __forceinline__ void closed_form_metrics(double t_pre, double t_dec, u32 b, u32 n, double cost_hr,
-                                                    double cost_sec, Metrics &o) {
+                                                    double cost_sec, Metrics &o, u64 n_pass = 1, u64 n_seg = 1) {
     const double inf = __longlong_as_double(0x7FF0000000000000LL);
     o.ttft = t_pre;
     o.latency = t_pre + t_dec;
@@ -328,8 +330,29 @@ __device__ __forceinline__ void closed_form_metrics(double t_pre, double t_dec, 
     } else {
         o.tpot = 0.0; o.thr = 0.0; o.cost_tok = inf;
     }
-    o.n_iters = 1 + (u64)n;
-    o.n_req_iters = (u64)b * (1 + (u64)n);
+    o.n_iters = n_pass + (u64)n;                    // prompt passes of one replica + decode steps
+    o.n_req_iters = (u64)b * (n_seg + (u64)n);
+}
+
+// Prompt processing of one sub-batch of sb requests in segments of seg tokens (Sec. 3.3.2): one pass
+// per segment, its tokens attending the prompt up to the end of the segment; the LM head runs with
+// the last segment only.  Passes are summed in order from 0.0.
+template <int TIME_SUM>
+__device__ __noinline__ double segmented_prefill(const DModel &m, const DRate &r, u32 tt, u32 sb, u32 lin, u32 seg,
+                                                 double Nd, double lf) {
+    TaskTab k;
+    double sum = 0.0;
+    for (u32 done = 0; done < lin; done += seg) {
+        const u32 q = min(seg, lin - done);
+        const bool last = done + q == lin;
+        const u64 T = (u64)sb * q;
+        build_fixed_tasks(m, tt, T, last ? sb : 0, 1, k);
+        build_attn_tasks(m, tt, T, T * (done + q), (u64)sb * (done + q), k);
+        const double head = last ? eval_head<TIME_SUM>(k, r) : 0.0;
+        sum = sum + combine_phase(eval_fixed<TIME_SUM>(k, r), eval_attn<TIME_SUM>(k, r), eval_comm(k, r), head, k.Rd, Nd,
+                                  r.tovh, lf);
+    }
+    return sum;
 }
 
 // Whole closed-form evaluation of one config, nothing cached (used where configs arrive in
@@ -349,10 +372,23 @@ __device__ __forceinline__ void closed_form_eval(const DSpace &s, const Cfg &c, 
     const double lf = log2_rule_factor(t, tp_model);
     const double Nd = (double)m.N;
     TaskTab k;
-    const u64 Tp = (u64)b * lin;
-    build_fixed_tasks(m, tt, Tp, b, 1, k);
-    build_attn_tasks(m, tt, Tp, Tp * lin, Tp, k);
-    const double t_pre = eval_phase<TIME_SUM>(k, r, Nd, lf);
+    double t_pre;
+    u64 n_pass = 1, n_seg = 1;
+    if (r.split | r.seg) {
+        // Sec. 3.3.1: sub-batches of split requests, the remainder as one more; equal ones take equal time
+        const u32 split = (r.split == 0 || r.split > b) ? b : r.split;
+        const u32 seg = (r.seg == 0 || r.seg > lin) ? lin : r.seg;
+        const u32 n_full = b / split, rest = b % split;
+        t_pre = (double)n_full * segmented_prefill<TIME_SUM>(m, r, tt, split, lin, seg, Nd, lf);
+        if (rest) t_pre = t_pre + segmented_prefill<TIME_SUM>(m, r, tt, rest, lin, seg, Nd, lf);
+        n_seg = (lin + seg - 1) / seg;
+        n_pass = (u64)(n_full + (rest != 0)) * n_seg;
+    } else {
+        const u64 Tp = (u64)b * lin;
+        build_fixed_tasks(m, tt, Tp, b, 1, k);
+        build_attn_tasks(m, tt, Tp, Tp * lin, Tp, k);
+        t_pre = eval_phase<TIME_SUM>(k, r, Nd, lf);
+    }
     const u32 n = lout - 1;
     double t_dec = 0.0;
     if (n > 0) {
@@ -363,7 +399,7 @@ __device__ __forceinline__ void closed_form_eval(const DSpace &s, const Cfg &c, 
         t_dec = eval_phase<TIME_SUM>(k, r, Nd, lf);
     }
     const u32 ci = (c.h * s.n_f + c.f) * s.n_t + c.t;
-    closed_form_metrics(t_pre, t_dec, b_all, n, s.cost_hr[ci], s.cost_sec[ci], o);
+    closed_form_metrics(t_pre, t_dec, b_all, n, s.cost_hr[ci], s.cost_sec[ci], o, n_pass, n_seg);
 }
 
 }  // namespace guide

@@ -1076,7 +1076,7 @@ bool fused_stream_eligible(const DSpace &s, Range r) {
     const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
     const u32 n_tl = s.n_t * s.n_l;
     if (r.first != 0 || r.count != total || total < STREAM_MIN_COUNT) return false;
-    if (s.n_l % 4 != 0 || n_tl < 32) return false;
+    if (s.n_l % 4 != 0 || n_tl < 32 || s.chunked) return false;
     const u64 n_hf = (u64)s.n_h * s.n_f;
     return (u64)s.n_m * s.n_b * (n_tl / 4) * ((n_hf + MODEL_CHUNK - 1) / MODEL_CHUNK) <= 0x7FFFFFFFull;
 }

@@ -130,7 +130,7 @@ __device__ __forceinline__ void tiled_visit(const DSpace &s, const Range &r, int
 // Returns false when the space does not suit the tiled walk.
 inline bool tiled_geometry(const DSpace &s, u64 want_blocks, u64 max_blocks, TileGeom *g) {
     const u32 n_tl = s.n_t * s.n_l, n_hf = s.n_h * s.n_f;
-    if (n_tl < 32) return false;
+    if (n_tl < 32 || s.chunked) return false;     // split prompt processing differs per framework: no shared tables
     g->threads = n_tl >= 256 ? 256 : ((n_tl + 31) / 32) * 32;
     g->tiles_per_mb = (n_tl + g->threads - 1) / g->threads;
     const u64 gx = (u64)s.n_m * s.n_b * g->tiles_per_mb;

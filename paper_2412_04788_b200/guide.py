@@ -52,7 +52,8 @@ class Hw(C.Structure):
 
 class Fw(C.Structure):
     _fields_ = [("e_c", C.c_double * 3), ("e_m", C.c_double * 3), ("e_comm", C.c_double), ("t_ovh", C.c_double),
-                ("flash", C.c_uint32), ("kv_block", C.c_uint32), ("reserve_permille", C.c_uint32), ("policy", C.c_uint32)]
+                ("flash", C.c_uint32), ("kv_block", C.c_uint32), ("reserve_permille", C.c_uint32), ("policy", C.c_uint32),
+                ("split_size", C.c_uint32), ("seg_tokens", C.c_uint32)]
 
 
 class LenPair(C.Structure):
@@ -148,6 +149,8 @@ class Space:
             fws[i].e_m[:] = [float(x) for x in ff[3:6]]
             fws[i].e_comm, fws[i].t_ovh = float(ff[6]), float(ff[7])
             fws[i].flash, fws[i].kv_block, fws[i].reserve_permille, fws[i].policy = (int(x) for x in fi)
+            if space.get("fw_chunk") is not None:
+                fws[i].split_size, fws[i].seg_tokens = (int(x) for x in space["fw_chunk"][i])
         batch = (C.c_uint32 * len(space["batch"]))(*[int(v) for v in space["batch"]])
         tp = (C.c_uint32 * len(space["tp"]))(*[int(v) for v in space["tp"]])
         pairs = (LenPair * len(space["pairs"]))(*[LenPair(int(a), int(b)) for a, b in space["pairs"]])

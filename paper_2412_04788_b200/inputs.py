@@ -196,9 +196,14 @@ def hybrid_axis(n_gpus: int):
     return dps, tps
 
 
-def _space(models, hw, hw_mem, fw_f, fw_i, batch, tp, pairs, dp=None):
+def _space(models, hw, hw_mem, fw_f, fw_i, batch, tp, pairs, dp=None, fw_chunk=None):
+    """dp (optional): data-parallel degree per entry of the TP axis.  fw_chunk (optional): per
+    framework (split_size, seg_tokens) = requests per prompt sub-batch, tokens per prompt segment;
+    0 = whole batch / whole prompt."""
     extra = {} if dp is None else {"dp": np.ascontiguousarray(dp, dtype=np.uint32)}
     assert dp is None or len(dp) == len(tp)
+    if fw_chunk is not None:
+        extra["fw_chunk"] = np.ascontiguousarray(fw_chunk, dtype=np.uint32).reshape(len(fw_f), 2)
     return {**extra,
         "models": np.ascontiguousarray(models, dtype=np.uint32),
         "hw": np.ascontiguousarray(hw, dtype=np.float64),
@@ -329,3 +334,18 @@ def hybrid_workload(n_gpus: int = 8, n_hw: int = 8, n_fw: int = 3, seed_offset: 
     return {"name": f"hybrid-{n_gpus}", "space": space, "trace": None, "constraints": {},
             "topk": {"key": "cost_per_token", "k": 64},
             "pareto": {"x": "latency", "y": "cost_per_hr"}}
+
+
+def chunked_workload(scale: float = 0.5, n_gpus: int = 1):
+    """Workload 2's sweep with frameworks that process prompts in pieces: profile 0 whole batches and
+    prompts, profile 1 sub-batches of 4 requests and 512-token segments, profile 2 sub-batches of
+    16 requests.  n_gpus > 1 replaces the TP axis by the (dp, tp) pairs under that budget."""
+    w = workload(2, scale=scale)
+    sp = dict(w["space"])
+    sp["fw_chunk"] = np.array([[0, 0], [4, 512], [16, 0]], dtype=np.uint32)
+    if n_gpus > 1:
+        dp, tp = hybrid_axis(n_gpus)
+        sp["dp"] = np.array(dp, dtype=np.uint32)
+        sp["tp"] = np.array(tp, dtype=np.uint32)
+    return {"name": "C2-chunked", "space": sp, "trace": None, "constraints": {},
+            "topk": {"key": "cost_per_token", "k": 8}, "pareto": {"x": "latency", "y": "cost_per_hr"}}

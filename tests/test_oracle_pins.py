@@ -11,14 +11,15 @@ from paper_2412_04788_b200 import inputs as I
 
 
 def toy_space(golden, mem, kv_block, batch, pairs=((4, 3),), tp=(1,), e=None, t_ovh=0.0, flash=1, reserve=0,
-              layers=None, dp=None):
+              layers=None, dp=None, chunk=None):
     model = list(golden["model"])
     if layers:
         model[0] = layers
     fw_f = list(e) if e is not None else [1.0] * 7
     return I._space(np.array([model]), np.array([golden["hw"]]), np.array([mem]),
                     np.array([fw_f + [t_ovh]]), np.array([[flash, kv_block, reserve, 0]]),
-                    list(batch), list(tp), [list(p) for p in pairs], dp=None if dp is None else list(dp))
+                    list(batch), list(tp), [list(p) for p in pairs], dp=None if dp is None else list(dp),
+                    fw_chunk=None if chunk is None else [list(chunk)])
 
 
 def test_weight_count_and_kv_bytes(golden):
@@ -163,6 +164,71 @@ def test_data_parallel_replicas(golden):
         oracle.simulate(toy_space(golden, 10**6, 1, [2], dp=(2,)), tr)
     with pytest.raises(ValueError):
         oracle.simulate(toy_space(golden, 10**6, 1, [2], dp=(0,)))
+
+
+def test_prompt_sub_batches_and_segments(golden):
+    """Sec. 3.3.1 (sub-batches of split_size requests plus a remainder) and Sec. 3.3.2 (prompts cut
+    into ceil(Lin / segment) segments): hand-worked batch-2 case, explicit token walks."""
+    want = golden["closed_form_b2_Lin4_Lout3"]["t1"]
+    hw, ff, fi = golden["hw"], [1.0] * 7 + [0.0], [1, 1, 0, 0]
+    one = oracle.simulate(toy_space(golden, 10**6, 1, [1, 2, 4, 5]))
+    # sub-batches of two: 2 = one pass, 4 = two equal passes, 5 = two passes and a single request
+    out = oracle.simulate(toy_space(golden, 10**6, 1, [1, 2, 4, 5], chunk=(2, 0)))
+    assert out["ttft"][1] == want["ttft"] and out["latency"][1] == want["latency"]
+    assert out["ttft"][2] == 2.0 * want["ttft"] and out["ttft"][3] == 2.0 * want["ttft"] + one["ttft"][0]
+    assert out["ttft"][0] == one["ttft"][0]
+    assert out["n_iters"].tolist() == [1 + 2, 1 + 2, 2 + 2, 3 + 2]
+    assert out["n_req_iters"].tolist() == [3, 6, 12, 15]
+    # the decode stage is that of the whole batch
+    assert np.array_equal(out["latency"] - out["ttft"] > 0, [True] * 4)
+    for c in range(4):
+        assert out["tpot"][c] == one["tpot"][c] and out["thr_decode"][c] == one["thr_decode"][c]
+    # segments of two tokens of the 4-token prompt, two requests: (T, E, A, C) by hand
+    out = oracle.simulate(toy_space(golden, 10**6, 1, [2], chunk=(0, 2)))
+    p1, d1 = oracle.phase_time(golden["model"], hw, ff, fi, 1, 4, 0, 8, 4, 1)     # 2 x 2 tokens attend 2; no token out
+    p2, d2 = oracle.phase_time(golden["model"], hw, ff, fi, 1, 4, 2, 16, 8, 1)    # 2 x 2 tokens attend 4; 2 tokens out
+    assert out["ttft"][0] == (0.0 + p1) + p2
+    assert d1[12] == 0.0 and d2[12] > 0.0                                         # no LM head without an emitted token
+    assert p1 == golden["model"][0] * ((d1[13] + d1[14]) + d1[11])                # layers x per-layer time, nothing else
+    assert out["n_iters"][0] == 2 + 2 and out["n_req_iters"][0] == 2 * (2 + 2)
+    assert out["ttft"][0] > want["ttft"]                                          # the weights are read twice
+    # sizes that split nothing change nothing, bit for bit
+    base = oracle.simulate(toy_space(golden, 10**6, 1, [1, 2, 3], pairs=[(4, 3), (7, 1)]))
+    for chunk in ((0, 0), (3, 7), (100, 100), (0, 8)):
+        same = oracle.simulate(toy_space(golden, 10**6, 1, [1, 2, 3], pairs=[(4, 3), (7, 1)], chunk=chunk))
+        for k in base:
+            assert np.array_equal(base[k], same[k]), (chunk, k)
+    # general sizes against explicit walks over sub-batches, segments, sequences and tokens
+    hw2 = [3.0e3, 5.0e2, 1.0e2, 1e-3, 2.0]
+    ff2, fi2 = [0.5, 0.25, 0.75, 0.5, 0.5, 0.25, 0.5, 1e-2], [0, 1, 0, 0]
+    for b, lin, lout, split, seg in [(5, 7, 3, 2, 3), (7, 16, 2, 3, 16), (4, 9, 1, 4, 2), (6, 5, 4, 1, 1), (3, 33, 2, 5, 8)]:
+        for tm in (oracle.TIME_MAX, oracle.TIME_SUM):
+            sp = I._space(np.array([golden["model"]]), np.array([hw2]), np.array([10**9]), np.array([ff2]),
+                          np.array([fi2]), [b], [1], [(lin, lout)], fw_chunk=[[split, seg]])
+            out = oracle.simulate(sp, time_model=tm)
+            subs = naive.sub_batches(b, split)
+            per_size = {}
+            for sb in set(subs):
+                t = 0.0
+                for T, E, A, Cc in naive.segment_passes(sb, lin, seg):
+                    t = t + oracle.phase_time(golden["model"], hw2, ff2, fi2, 1, T, E, A, Cc, 1, time_model=tm)[0]
+                per_size[sb] = t
+            t_pre = subs.count(split) * per_size[split] if split in per_size else 0.0
+            if b % split:
+                t_pre = t_pre + per_size[b % split]
+            assert out["ttft"][0] == t_pre, (b, lin, split, seg)
+            n_seg = len(naive.segment_passes(1, lin, seg))
+            assert out["n_iters"][0] == len(subs) * n_seg + (lout - 1)
+            assert out["n_req_iters"][0] == b * (n_seg + lout - 1)
+            # all prompt tokens are processed exactly once
+            assert sum(T for sb in subs for T, *_ in naive.segment_passes(sb, lin, seg)) == b * lin
+    # a replica's share is what gets split (Sec. 3.2 Step 1)
+    out = oracle.simulate(toy_space(golden, 10**6, 1, [8, 7], tp=(1,), dp=(2,), chunk=(2, 0)))
+    assert out["ttft"].tolist() == [2.0 * want["ttft"]] * 2 and out["n_iters"].tolist() == [4, 4]
+    # traces keep the prompt-first policy: splitting is refused there
+    tr = {"arrival": np.array([0.0, 1.0]), "in_len": np.zeros(2, np.uint32), "out_len": np.zeros(2, np.uint32)}
+    with pytest.raises(ValueError, match="splitting"):
+        oracle.simulate(toy_space(golden, 10**6, 1, [2], chunk=(0, 2)), tr)
 
 
 def test_closed_form_aggregates_match_token_loops(golden):
