@@ -7,7 +7,7 @@ namespace guide {
 
 static constexpr u32 MODEL_THREADS = 128;
 static constexpr u32 MODEL_BLOCKS_PER_SM = 8;
-static constexpr u32 MODEL_CHUNK = 64;          // sorted pairs per work item
+static constexpr u32 MODEL_CHUNK = 64;  // sorted pairs per work item
 
 // Stage table of one point in shared memory: the 24 entries of a TaskTab, interleaved over the
 // four points of a foursome so that the lanes of a warp read neighbouring 8-byte words (a 64-bit
@@ -24,22 +24,20 @@ __device__ __forceinline__ void put_stage(StageTab &tb, u32 u, const TaskTab &k)
     tb[E_RD][u] = k.Rd;
 }
 
-// Both stage tables of one point, written to shared memory.  Kept out of line: it runs once per
-// work item and needs far more registers than the walk around it.
-static __device__ __noinline__ void build_point_tables(const DModel *mp, u32 tt, u32 b, u32 lin, u32 n, StageTab *tb_pre, StageTab *tb_dec,
-                                                u32 u) {
+// One stage table of one point, written to shared memory: stage 0 is the prompt pass, stage 1 the
+// aggregated decode steps.  Eight lanes of a warp call it together (four points x two stages): the
+// instruction stream is the same for both stages, only the token counts differ.  Kept out of line:
+// it runs once per work item and needs far more registers than the walk around it.
+static __device__ __noinline__ void build_stage_table(const DModel *mp, u32 tt, u32 b, u32 lin, u32 n, u32 stage, StageTab *tb, u32 u) {
     const DModel m = *mp;
     TaskTab k;
-    const u64 Tp = (u64)b * lin;
-    build_fixed_tasks(m, tt, Tp, b, 1, k);
-    build_attn_tasks(m, tt, Tp, Tp * lin, Tp, k);
-    put_stage(*tb_pre, u, k);
-    const u32 nn = n > 0 ? n : 1;          // a table is built either way; unused when n == 0
-    const u64 Td = (u64)b * nn;
+    const u32 nn = n > 0 ? n : 1;          // a decode table is built either way; unused when n == 0
+    const u64 Tp = (u64)b * lin, Td = (u64)b * nn;
     const u64 ctx = (u64)b * ((u64)nn * lin + ((u64)nn * (nn + 1)) / 2);
-    build_fixed_tasks(m, tt, Td, Td, nn, k);
-    build_attn_tasks(m, tt, Td, ctx, ctx, k);
-    put_stage(*tb_dec, u, k);
+    const u64 T = stage ? Td : Tp;
+    build_fixed_tasks(m, tt, T, stage ? Td : (u64)b, stage ? (u64)nn : 1ull, k);
+    build_attn_tasks(m, tt, T, stage ? ctx : Tp * lin, stage ? ctx : Tp, k);
+    put_stage(*tb, u, k);
 }
 
 // rates of one pair in registers (a row of rate10)
@@ -71,7 +69,7 @@ __device__ __forceinline__ double eval_stage(const StageTab &tb, u32 u, const Ra
 // Performance model for the configs that fit (Sec. 3.2 Step 2, Sec. 3.4.2, Sec. 3.5.1).  A warp takes one foursome of the plane for one
 // (model, batch) and a chunk of the sorted pair walk; its lanes are four points x eight pairs, so
 // the four lanes that share a pair write one whole sector.  The stage tables of the four points
-// sit in shared memory (built once per item by four lanes), the rates of a lane's pair in
+// sit in shared memory (built once per item by eight lanes), the rates of a lane's pair in
 // registers: that is half the registers of a table per thread, hence twice the warps.  Work items
 // differ wildly in cost (most have nothing that fits): they are handed out through a counter to a
 // persistent grid, heaviest chunks and foursomes first.
@@ -125,7 +123,7 @@ __device__ __forceinline__ void model_walk(const DSpace &s, int tp_model, u32 n_
         }
         if (!__any_sync(0xFFFFFFFFu, any)) continue;
         __syncwarp();                                 // the previous item's reads of the tables are over
-        if (h == 0) build_point_tables(mp, tp_model ? 1u : t, b, lin, n, &tb_pre, &tb_dec, u);      // lane u: point u
+        if (h < 2) build_stage_table(mp, tp_model ? 1u : t, b, lin, n, h, h ? &tb_dec : &tb_pre, u);   // lanes 0-3: prompt stage of point u; 4-7: decode stage
         __syncwarp();
         const u64 j0 = (u64)mpos * n_hf * stride_hf + (u64)bpos * n_tl + tl;
         const double lf = log2_rule_factor(t, tp_model);
