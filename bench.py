@@ -304,20 +304,41 @@ def run_ours(args):
         guide.guide_select_topk(path.sp, None, gathered, {}, key, k, path.idx, path.val, path.cnt, path.ws_k, count=m)
         return all_idx
 
+    # The two selections of a step read the same metrics and share nothing else: top-k runs on the
+    # step's stream, the Pareto front beside it on a second one (both after guide_simulate; the next
+    # step's guide_simulate after both).
+    main = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
+    ev_sim = torch.cuda.Event()
+    ev_side = torch.cuda.Event()
+
     def step(events=None):
         if events:
             events[0].record()
         path.simulate()
         if events:
             events[1].record()
+        ev_sim.record()
+        side.wait_event(ev_sim)
+        with torch.cuda.stream(side):
+            path.pareto()
+            ev_side.record()
         path.topk()
-        if events:
-            events[2].record()
-        path.pareto()
+        main.wait_event(ev_side)
         if world > 1:
             exchange()
         if events:
-            events[3].record()
+            events[2].record()
+
+    def step_in_turn(events):
+        """the same calls one after the other on one stream: the time of each call by itself"""
+        events[0].record()
+        path.simulate()
+        events[1].record()
+        path.topk()
+        events[2].record()
+        path.pareto()
+        events[3].record()
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -326,7 +347,7 @@ def run_ours(args):
         dist.barrier()
     sampler = ClockSampler(local_rank)
     sampler.start()
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     torch.cuda.synchronize()
     wall0 = time.perf_counter()
     for i in range(args.steps):
@@ -336,9 +357,16 @@ def run_ours(args):
     sampler.stop_flag = True
     sampler.join()
     t_sim = sum(e[0].elapsed_time(e[1]) for e in evs)
-    t_topk = sum(e[1].elapsed_time(e[2]) for e in evs)
-    t_par = sum(e[2].elapsed_time(e[3]) for e in evs)
-    total_ms = t_sim + t_topk + t_par
+    total_ms = sum(e[0].elapsed_time(e[2]) for e in evs)
+    # each selection call by itself, for the per-call figures (not part of `value`)
+    n_turn = min(args.steps, 50)
+    evt = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_turn)]
+    for i in range(n_turn):
+        step_in_turn(evt[i])
+    torch.cuda.synchronize()
+    t_topk = sum(e[1].elapsed_time(e[2]) for e in evt) * args.steps / n_turn
+    t_par = sum(e[2].elapsed_time(e[3]) for e in evt) * args.steps / n_turn
+    t_turn = sum(e[0].elapsed_time(e[3]) for e in evt) / n_turn
     if world > 1:
         tt = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
@@ -439,7 +467,10 @@ def run_ours(args):
                                    f"= {n_local} configs per GPU; simulate (materialised) + top-{k} by cost/token under the "
                                    "latency bound + Pareto(latency, $/h)",
                        "l2": "no flush: each step writes and re-reads 0.89 GB, several times the 126 MB L2",
-                       "timing": "CUDA events per step, summed"},
+                       "timing": "CUDA events around each step on its stream, summed",
+                       "streams": "guide_select_topk on the step's stream, guide_pareto beside it on a second stream, both "
+                                  "after guide_simulate; per-call figures from the same calls issued one after the other"},
+            "ms_per_step_calls_in_turn": t_turn,
             "clocks": sampler.summary(),
             "e2e": {"value": e2e_value, "unit": "configs/s", "h2d_bytes_per_step": table_bytes(local_space),
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps},
