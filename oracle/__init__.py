@@ -16,6 +16,7 @@ _SRC = os.path.join(_HERE, "guide_oracle.c")
 _LIB = os.path.join(_HERE, "libguide_oracle.so")
 
 TIME_MAX, TIME_SUM = 0, 1
+POLICY_PREFILL_FIRST, POLICY_SPLIT_FUSE = 0, 1
 TP_EXPLICIT, TP_PAPER_LOG2 = 0, 1
 ST_WEIGHTS, ST_KV, ST_HEADS, ST_ITER = 1, 2, 4, 8
 KEYS = {"latency": 0, "ttft": 1, "ttft_p99": 2, "tpot": 3, "throughput": 4, "cost_per_hr": 5,

@@ -73,6 +73,7 @@ typedef struct {
     u64 *n_preempt;                        /* optional: preemptions per config (diagnostic) */
 } oout;
 
+enum { POLICY_PREFILL_FIRST = 0, POLICY_SPLIT_FUSE = 1 };
 typedef struct { u64 N, H, nh, nkv, I, V, g, wb, ab, kvb, d, Dkv; } model_t;
 
 typedef struct {
@@ -313,19 +314,19 @@ static int cmp_double(const void *a, const void *b) {
 }
 
 typedef struct {
-    u32 *gen, *cache, *held, *running;
+    u32 *gen, *cache, *held, *running, *todo, *pdone;
     uint8_t *done, *needs_prefill, *has_first;
     double *first, *finish, *sorted;
 } simbuf;
 
 static void simbuf_alloc(simbuf *w, u64 n) {
     w->gen = malloc(n * sizeof(u32)); w->cache = malloc(n * sizeof(u32)); w->held = malloc(n * sizeof(u32));
-    w->running = malloc(n * sizeof(u32));
+    w->running = malloc(n * sizeof(u32)); w->todo = malloc(n * sizeof(u32)); w->pdone = malloc(n * sizeof(u32));
     w->done = malloc(n); w->needs_prefill = malloc(n); w->has_first = malloc(n);
     w->first = malloc(n * sizeof(double)); w->finish = malloc(n * sizeof(double)); w->sorted = malloc(n * sizeof(double));
 }
 static void simbuf_free(simbuf *w) {
-    free(w->gen); free(w->cache); free(w->held); free(w->running); free(w->done); free(w->needs_prefill);
+    free(w->gen); free(w->cache); free(w->held); free(w->running); free(w->todo); free(w->pdone); free(w->done); free(w->needs_prefill);
     free(w->has_first); free(w->first); free(w->finish); free(w->sorted);
 }
 
@@ -336,6 +337,8 @@ static void trace_sim_one(const ospace *s, const otrace *tr, u64 idx, u64 j, int
     rates_t r = load_rates(s->hw + 5 * p.h, s->fw_f + 8 * p.f, s->fw_i + 4 * p.f);
     u64 t = s->tp[p.t], b = s->batch[p.b], Lin = s->pairs[2 * p.l], Lout = s->pairs[2 * p.l + 1];
     u64 blk = s->fw_i[4 * p.f + 1], reserve = s->fw_i[4 * p.f + 2];
+    int fuse = s->fw_i[4 * p.f + 3] == POLICY_SPLIT_FUSE;
+    u64 budget_tokens = fuse ? s->fw_chunk[2 * p.f + 1] : 0;   /* tokens per iteration (checked > 0 by the caller) */
     u64 n = tr->n;
 #define IN(i)  ((u64)(tr->in_len[i] ? tr->in_len[i] : Lin))
 #define OUT(i) ((u64)(tr->in_len[i] ? tr->out_len[i] : Lout))
@@ -349,6 +352,7 @@ static void trace_sim_one(const ospace *s, const otrace *tr, u64 idx, u64 j, int
         u64 need = ceil_div(IN(i) + OUT(i), blk);
         if (need > worst) worst = need;
         sum_out += OUT(i);
+        if (fuse) sum_out += IN(i);      /* prompt chunks take iterations too: the backstop counts them */
     }
     u64 fit = worst ? blocks_total / worst : 0;      /* worst-case requests resident at once */
     uint8_t st = 0;
@@ -379,6 +383,8 @@ static void trace_sim_one(const ospace *s, const otrace *tr, u64 idx, u64 j, int
             free_blocks -= need;
             w->held[next] = (u32)need;
             w->needs_prefill[next] = 1;
+            w->todo[next] = (u32)(IN(next) + w->gen[next]);      /* split-fuse: prompt tokens still to process */
+            w->pdone[next] = 0;
             run[nrun++] = (u32)next;
             next++;
         }
@@ -390,10 +396,71 @@ static void trace_sim_one(const ospace *s, const otrace *tr, u64 idx, u64 j, int
         }
         /* 3. build the iteration: prompts first, everything else stalls */
         if (n_iters >= max_iters) { st |= ST_ITER; break; }   /* backstop against a runaway schedule */
-        u64 n_pre = 0;
-        for (u64 k = 0; k < nrun; k++) n_pre += w->needs_prefill[run[k]];
         double T_iter;
         u64 participants;
+        if (fuse) {
+            /*
+             * Dynamic split and fuse (the FastGen-like framework model, Sec. 2.3.2 / Sec. 3.1): every
+             * iteration carries about budget_tokens tokens.  Each resident past its prompt decodes one
+             * token; what is left of the budget goes to prompts in arrival order, a long prompt
+             * spread over several iterations, short ones sharing one.  A prompt chunk of q tokens
+             * attends the pdone + q tokens of its request seen so far; the request emits its first
+             * token in the iteration that finishes its prompt.
+             */
+            u64 needed = 0;
+            for (u64 k = 0; k < nrun; k++) needed += (!w->needs_prefill[run[k]] && w->cache[run[k]] % blk == 0);
+            while (needed > free_blocks) {            /* preempt the youngest, recompute later */
+                u32 v = run[nrun - 1];
+                free_blocks += w->held[v];
+                if (!w->needs_prefill[v] && w->cache[v] % blk == 0) needed--;
+                w->cache[v] = 0; w->held[v] = 0; w->needs_prefill[v] = 0;
+                nrun--; next = v; n_preempt++;
+            }
+            free_blocks -= needed;
+            u64 n_dec = 0, n_chunk = 0, T = 0, E = 0, A = 0, C = 0;
+            for (u64 k = 0; k < nrun; k++) {
+                u32 i = run[k];
+                if (w->needs_prefill[i]) continue;
+                if (w->cache[i] % blk == 0) w->held[i] += 1;
+                u64 c = IN(i) + w->gen[i];
+                n_dec++; A = add(A, c); C = add(C, c);
+            }
+            T = n_dec; E = n_dec;
+            u64 left = budget_tokens > n_dec ? budget_tokens - n_dec : 0;
+            double after;
+            for (u64 k = 0; k < nrun && left > 0; k++) {          /* plan the chunks */
+                u32 i = run[k];
+                if (!w->needs_prefill[i]) continue;
+                u64 q = w->todo[i] < left ? w->todo[i] : left;
+                T = add(T, q); A = add(A, mul(q, w->pdone[i] + q)); C = add(C, w->pdone[i] + q);
+                if (q == w->todo[i]) E++;
+                left -= q; n_chunk++;
+            }
+            T_iter = phase_time(&m, &r, t, T, E, A, C, 1, time_model, tp_model, NULL);
+            after = clock + T_iter;
+            for (u64 k = 0; k < nrun; k++) {                      /* decodes advance */
+                u32 i = run[k];
+                if (!w->needs_prefill[i]) { w->cache[i] += 1; w->gen[i] += 1; }
+            }
+            left = budget_tokens > n_dec ? budget_tokens - n_dec : 0;
+            for (u64 k = 0; k < nrun && left > 0; k++) {          /* the planned chunks are processed */
+                u32 i = run[k];
+                if (!w->needs_prefill[i] || w->todo[i] == 0) continue;
+                u64 q = w->todo[i] < left ? w->todo[i] : left;
+                w->pdone[i] += (u32)q; w->todo[i] -= (u32)q; left -= q;
+                if (w->todo[i] == 0) {                            /* prompt finished: first token */
+                    w->cache[i] = (u32)(IN(i) + w->gen[i]);
+                    w->gen[i] += 1;
+                    w->needs_prefill[i] = 0;
+                    if (!w->has_first[i]) { w->has_first[i] = 1; w->first[i] = after; }
+                }
+            }
+            if (n_dec > 0) { dec_time = dec_time + T_iter; dec_tok += n_dec; }
+            participants = n_dec + n_chunk;
+            goto advance;
+        }
+        u64 n_pre = 0;
+        for (u64 k = 0; k < nrun; k++) n_pre += w->needs_prefill[run[k]];
         if (n_pre > 0) {
             u64 T = 0, A = 0;
             for (u64 k = 0; k < nrun; k++) {
@@ -438,6 +505,7 @@ static void trace_sim_one(const ospace *s, const otrace *tr, u64 idx, u64 j, int
             participants = nrun;
         }
         /* 4. advance the clock */
+advance:
         clock = clock + T_iter;
         n_iters++; n_req_iters += participants;
         /* 5. retire finished sequences, keep the rest in order */
@@ -507,8 +575,13 @@ int oracle_simulate(const ospace *s, const otrace *tr, u64 first, u64 count, u64
         if (s->dp[i] == 0) return -1;
         if (tr && s->dp[i] != 1) return -3;      /* the trace simulation models one replica */
     }
-    if (s->fw_chunk && tr) for (u32 i = 0; i < 2 * s->n_f; i++) {
-        if (s->fw_chunk[i] != 0) return -3;      /* the trace simulation has the prompt-first policy only */
+    for (u32 i = 0; i < s->n_f; i++) {
+        u32 policy = s->fw_i[4 * i + 3];
+        u32 split = s->fw_chunk ? s->fw_chunk[2 * i] : 0, seg = s->fw_chunk ? s->fw_chunk[2 * i + 1] : 0;
+        if (policy > POLICY_SPLIT_FUSE) return -1;
+        if (!tr) continue;
+        if (policy == POLICY_PREFILL_FIRST && (split || seg)) return -3;   /* prompt-first passes take whole prompts */
+        if (policy == POLICY_SPLIT_FUSE && (seg == 0 || split != 0)) return -1;   /* needs its token budget, and only that */
     }
     for (u32 i = 0; i < s->n_l; i++) if (s->pairs[2 * i] == 0 || s->pairs[2 * i + 1] == 0) return -1;
     if (tr) for (u64 i = 0; i < tr->n; i++) {

@@ -68,7 +68,7 @@ def decode_aggregates(b: int, lin: int, lout: int):
 # ---- continuous batching with explicit objects ----------------------------------------------------
 
 class _Req:
-    __slots__ = ("idx", "arrival", "lin", "lout", "gen", "cache", "blocks", "needs_prefill", "first", "finish")
+    __slots__ = ("idx", "arrival", "lin", "lout", "gen", "cache", "blocks", "needs_prefill", "first", "finish", "todo", "seen")
 
     def __init__(self, idx, arrival, lin, lout):
         self.idx, self.arrival, self.lin, self.lout = idx, arrival, lin, lout
@@ -185,6 +185,115 @@ def trace_sim(arrival, in_len, out_len, max_batch, n_blocks, kv_block, iter_time
     return {"first": [r.first for r in reqs], "finish": [r.finish for r in reqs], "makespan": clock,
             "dec_time": dec_time, "dec_tok": dec_tok, "n_iters": n_iters, "n_req_iters": n_req_iters,
             "n_preempt": n_preempt, "max_running": max_running}
+
+
+def trace_sim_fuse(arrival, in_len, out_len, max_batch, n_blocks, kv_block, budget, iter_time, max_iters=10**6):
+    """Dynamic split-and-fuse continuous batching: every iteration carries `budget` tokens, one per
+    decoding request first, the rest filled with prompt tokens in arrival order (long prompts are
+    spread over iterations, short ones share one).  Blocks for the whole prompt are taken at
+    admission; evict-youngest + recompute as in trace_sim.  Also returns the composition of every
+    iteration: (clock before, decoding request ids, [(request id, first token, q)])."""
+    reqs = [_Req(i, arrival[i], in_len[i], out_len[i]) for i in range(len(arrival))]
+    for r in reqs:
+        r.todo = 0          # prompt tokens (and tokens to recompute) not yet processed
+        r.seen = 0          # ... already processed
+    waiting = list(reqs)
+    running = []
+    free = list(range(n_blocks))
+    clock = 0.0
+    dec_time = 0.0
+    dec_tok = n_iters = n_req_iters = n_preempt = 0
+    log = []
+    while True:
+        while waiting and waiting[0].arrival <= clock and len(running) < max_batch:
+            r = waiting[0]
+            need = math.ceil((r.lin + r.gen) / kv_block)
+            if need > len(free):
+                break
+            r.blocks = [free.pop() for _ in range(need)]
+            r.todo, r.seen = r.lin + r.gen, 0
+            running.append(waiting.pop(0))
+        if not running:
+            if not waiting:
+                break
+            assert waiting[0].arrival > clock, "stuck with an empty machine"
+            clock = waiting[0].arrival
+            continue
+        assert n_iters < max_iters
+        assert [r.idx for r in running] == sorted(r.idx for r in running)
+
+        def needers():
+            return [r for r in running if r.todo == 0 and r.cache % kv_block == 0]
+        while len(needers()) > len(free):
+            victim = max(running, key=lambda r: r.idx)
+            running.remove(victim)
+            free.extend(victim.blocks)
+            victim.blocks, victim.cache, victim.todo, victim.seen = [], 0, 0, 0
+            waiting.insert(0, victim)
+            n_preempt += 1
+        assert running
+        for r in needers():
+            r.blocks.append(free.pop())
+        decoders = [r for r in running if r.todo == 0]
+        # decoders come before requests still in their prompt (arrival order, oldest served first)
+        assert [r.idx for r in running] == [r.idx for r in decoders] + [r.idx for r in running if r.todo > 0]
+        T = E = A = Cc = 0
+        for r in decoders:
+            T += 1
+            E += 1
+            A += r.cache + 1
+            Cc += r.cache + 1
+        left = max(0, budget - len(decoders))
+        chunks = []
+        for r in running:
+            if r.todo == 0 or left == 0:
+                continue
+            q = min(r.todo, left)
+            for _ in range(q):
+                T += 1
+                A += r.seen + q             # every token of the chunk attends the prompt up to the chunk's end
+            Cc += r.seen + q
+            if q == r.todo:
+                E += 1
+            chunks.append((r, q))
+            left -= q
+        assert T > 0 and T <= max(budget, len(decoders))
+        dt = iter_time(T, E, A, Cc)
+        log.append((clock, [r.idx for r in decoders], [(r.idx, r.seen, q) for r, q in chunks]))
+        after = clock + dt
+        for r in decoders:
+            r.cache += 1
+            r.gen += 1
+        for r, q in chunks:
+            r.seen += q
+            r.todo -= q
+            if r.todo == 0:
+                r.cache = r.lin + r.gen
+                r.gen += 1
+                if r.first is None:
+                    r.first = after
+        if decoders:
+            dec_time = dec_time + dt
+            dec_tok += len(decoders)
+        clock = after
+        n_iters += 1
+        n_req_iters += len(decoders) + len(chunks)
+        for r in list(running):
+            if r.todo == 0 and r.gen == r.lout:
+                r.finish = clock
+                free.extend(r.blocks)
+                r.blocks = []
+                running.remove(r)
+        owned = [blk for r in running for blk in r.blocks]
+        assert len(owned) == len(set(owned)) and len(owned) + len(free) == n_blocks
+        for r in running:
+            if r.todo == 0:
+                assert len(r.blocks) == math.ceil(r.cache / kv_block)
+    assert all(r.finish is not None and r.first is not None for r in reqs), "a request never finished"
+    assert len(free) == n_blocks
+    return {"first": [r.first for r in reqs], "finish": [r.finish for r in reqs], "makespan": clock,
+            "dec_time": dec_time, "dec_tok": dec_tok, "n_iters": n_iters, "n_req_iters": n_req_iters,
+            "n_preempt": n_preempt, "log": log}
 
 
 # ---- selection by brute force ----------------------------------------------------------------------

@@ -198,3 +198,89 @@ def test_strided_and_ranged_evaluation_agree():
     part = oracle.simulate(sp, first=5, count=40, stride=7)
     for k in oracle.F64_FIELDS + ("status", "bmax"):
         assert np.array_equal(part[k], full[k][5:5 + 40 * 7:7])
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3, 4])
+def test_split_fuse_against_naive_scheduler(seed):
+    """The split-and-fuse policy (token budget per iteration, prompts chunked in arrival order,
+    decodes fused in) against an explicit scheduler with request objects and per-token loops."""
+    n = 24
+    arrival = I.poisson_arrivals(seed, n, 2000.0)
+    in_len = I.randint(seed, 81, n, 1, 40).astype(np.uint32)
+    out_len = I.randint(seed, 82, n, 1, 24).astype(np.uint32)
+    tr = {"arrival": arrival, "in_len": in_len, "out_len": out_len}
+    hw, _ = I.seeded_hw(seed, 1, mem_gb=[1])
+    fw_f, fw_i = I.seeded_fw(seed, 1, kv_block=4, reserve_permille=0)
+    fw_i[0, 3] = oracle.POLICY_SPLIT_FUSE
+    w_bytes = oracle.weight_bytes_per_gpu(SMALL, 1)
+    kv_tok = oracle.kv_bytes_per_token(SMALL, 1)
+    total_preempt = chunked = fused = 0
+    for n_blocks in (16, 23, 40, 400):
+        mem = w_bytes + n_blocks * 4 * kv_tok + 5
+        for b, budget in ((1, 7), (3, 16), (8, 5), (8, 64), (4, 1)):
+            sp = I._space(np.array([SMALL]), hw, np.array([mem]), fw_f, fw_i, [b], [1], [(1, 1)], fw_chunk=[[0, budget]])
+            got = oracle.simulate(sp, tr, per_request=True)
+            assert got["status"][0] == 0
+            ref = naive.trace_sim_fuse(arrival.tolist(), in_len.tolist(), out_len.tolist(), b, n_blocks, 4, budget,
+                                       _iter_time(SMALL, sp, 0, 0, 1))
+            assert got["latency"][0] == ref["makespan"]
+            ttft = np.array(ref["first"]) - arrival
+            assert np.array_equal(got["req_ttft"][0], ttft)
+            tpot = [(fi - fr) / (o - 1) if o > 1 else 0.0 for fi, fr, o in zip(ref["finish"], ref["first"], out_len)]
+            assert np.array_equal(got["req_tpot"][0], np.array(tpot))
+            assert got["n_iters"][0] == ref["n_iters"] and got["n_req_iters"][0] == ref["n_req_iters"]
+            assert got["n_preempt"][0] == ref["n_preempt"]
+            assert got["thr_decode"][0] == (ref["dec_tok"] / ref["dec_time"] if ref["dec_time"] else 0.0)
+            total_preempt += ref["n_preempt"]
+            # what the policy is for: prompts longer than the budget take several iterations, and
+            # iterations mix decoding requests with prompt chunks
+            per_req = {}
+            for _, dec, chunks in ref["log"]:
+                for i, _seen, _q in chunks:
+                    per_req[i] = per_req.get(i, 0) + 1
+                fused += bool(dec and chunks)
+                assert len(dec) + sum(q for *_, q in chunks) <= max(budget, len(dec))
+            chunked += sum(1 for i, c in per_req.items() if c > 1)
+            # every prompt token (and every token recomputed after an eviction) is processed once per residency
+            if ref["n_preempt"] == 0:
+                assert sum(q for _, _, chunks in ref["log"] for *_, q in chunks) == int(in_len.sum())
+    assert total_preempt > 0 and chunked > 0 and fused > 0
+
+
+def test_split_fuse_timeline_worked_by_hand():
+    """Two requests, budget 4, block size 4, ample memory.  Request 0: prompt 6, 3 tokens out, at t = 0;
+    request 1: prompt 3, 2 tokens out, also at t = 0.
+      iteration 1: chunk (0: 4 of 6)                         T=4 E=0 A=4*4=16      C=4
+      iteration 2: chunk (0: last 2, attends 6) + (1: 2 of 3) T=4 E=1 A=2*6+2*2=16  C=6+2=8
+      iteration 3: decode 0 (ctx 7) + chunk (1: last 1, attends 3)  T=2 E=2 A=7+3=10 C=10
+      iteration 4: decode 0 (ctx 8), decode 1 (ctx 4)         T=2 E=2 A=12 C=12   -> both finish"""
+    tr = {"arrival": np.array([0.0, 0.0]), "in_len": np.array([6, 3], np.uint32), "out_len": np.array([3, 2], np.uint32)}
+    hw, _ = I.seeded_hw(7, 1, mem_gb=[1])
+    fw_f, fw_i = I.seeded_fw(7, 1, kv_block=4, reserve_permille=0)
+    fw_i[0, 3] = oracle.POLICY_SPLIT_FUSE
+    sp = I._space(np.array([SMALL]), hw, np.array([10**9]), fw_f, fw_i, [4], [1], [(1, 1)], fw_chunk=[[0, 4]])
+    got = oracle.simulate(sp, tr, per_request=True)
+    it = _iter_time(SMALL, sp, 0, 0, 1)
+    t1 = it(4, 0, 16, 4)
+    t2 = t1 + it(4, 1, 16, 8)
+    t3 = t2 + it(2, 2, 10, 10)
+    t4 = t3 + it(2, 2, 12, 12)
+    assert got["latency"][0] == t4
+    assert got["req_ttft"][0].tolist() == [t2, t3]
+    assert got["req_tpot"][0].tolist() == [(t4 - t2) / 2, (t4 - t3) / 1]
+    assert got["n_iters"][0] == 4 and got["n_req_iters"][0] == 1 + 2 + 2 + 2
+    assert got["thr_decode"][0] == 3 / ((t3 - t2) + (t4 - t3))
+    # a budget that covers everything waiting is prompt-first scheduling when nothing decodes yet
+    both = oracle.simulate(I._space(np.array([SMALL]), hw, np.array([10**9]), fw_f, fw_i, [4], [1], [(1, 1)],
+                                    fw_chunk=[[0, 9]]), tr, per_request=True)
+    fw_p = fw_i.copy()
+    fw_p[0, 3] = 0
+    first = oracle.simulate(I._space(np.array([SMALL]), hw, np.array([10**9]), fw_f, fw_p, [4], [1], [(1, 1)]), tr,
+                            per_request=True)
+    assert both["req_ttft"][0].tolist() == first["req_ttft"][0].tolist()       # one pass over 6 + 3 tokens either way
+    # the policy needs its budget and is a trace policy only
+    with pytest.raises(ValueError):
+        oracle.simulate(I._space(np.array([SMALL]), hw, np.array([10**9]), fw_f, fw_i, [4], [1], [(1, 1)]), tr)
+    with pytest.raises(ValueError):
+        oracle.simulate(I._space(np.array([SMALL]), hw, np.array([10**9]), fw_f, fw_i, [4], [1], [(1, 1)],
+                                 fw_chunk=[[2, 4]]), tr)
