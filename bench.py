@@ -248,6 +248,28 @@ def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full, fraction
                             "simulate_frac_of_hbm": BYTES_SIM * n / t_sim / 1e6 / hbm_peak,
                             "kernel_launches": 2 + 6 + 5 + 5 + 4}
             del p
+        elif k == 8:
+            # workload 3 on an eighth of its hardware axis with every framework on the split-and-fuse
+            # policy (token budgets 256 .. 8192 per iteration)
+            import numpy as np
+            w = inputs.workload(3, scale=0.125, trace_scale=1.0)
+            space = dict(w["space"])
+            fw_i = np.array(space["fw_i"], dtype=np.uint32).copy()
+            fw_i[:, 3] = guide.GUIDE_POLICY_SPLIT_FUSE
+            space["fw_i"] = fw_i
+            space["fw_chunk"] = np.array([[0, 256], [0, 512], [0, 2048], [0, 8192]], dtype=np.uint32)
+            sp, tr = guide.Space(space), guide.Trace(w["trace"])
+            n = sp.size
+            out = guide.alloc_outputs(n, tr.n, fields=TRACE_FIELDS, per_request=False)
+            ws = torch.empty(guide.guide_workspace_bytes(sp, tr), dtype=torch.uint8, device="cuda")
+            best, med = time_call(torch, lambda: guide.guide_simulate(sp, tr, out, workspace=ws), reps=2, warm=1)
+            iters = int(out["n_iters"].sum().item())
+            req_iters = int(out["n_req_iters"].sum().item())
+            res["C3-split-fuse"] = {"configs": n, "requests": tr.n, "feasible": int((out["status"] == 0).sum().item()),
+                                    "ms": best, "configs_per_s": n / best * 1e3, "iters_per_s": iters / best * 1e3,
+                                    "request_iters_per_s": req_iters / best * 1e3, "hardware_axis_fraction": 0.125,
+                                    "kernel_launches": 1}
+            del out, ws
         elif k in (6, 7):
             # the (dp, tp) sweep under a budget of 8 GPUs (whole-space kernels) and workload 2 with
             # frameworks that process prompts in sub-batches / segments (one thread per config)
@@ -488,7 +510,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--extras", default="1,2,3,4,5,6,7", help="other workloads to time after the main loop ('' = none)")
+    ap.add_argument("--extras", default="1,2,3,4,5,6,7,8", help="other workloads to time after the main loop ('' = none)")
     ap.add_argument("--main-fraction", action="store_true",
                     help="apply --trace-fraction to the main workload's hardware axis too (small cases for profiler captures)")
     ap.add_argument("--full", action="store_true", help="(kept for compatibility: workloads 3 and 4 now always run whole)")

@@ -75,8 +75,9 @@ typedef struct guide_fw {
     uint32_t flash;         /* 1: FlashAttention (no score-matrix traffic), Sec. 3.2 Step 1 */
     uint32_t kv_block;      /* tokens per KV block (fixed-granularity paging, Sec. 2.4.1); 1 = unpaged */
     uint32_t reserve_permille; /* thousandths of device memory kept back */
-    uint32_t policy;        /* GUIDE_POLICY_PREFILL_FIRST */
-    /* Prompt processing in pieces (closed form only; a trace with either set is GUIDE_ERR_UNSUPPORTED):
+    uint32_t policy;        /* GUIDE_POLICY_*: how the trace simulation composes an iteration */
+    /* Prompt processing in pieces (closed form; with a trace: GUIDE_ERR_UNSUPPORTED under the prompt-first
+     * policy, and seg_tokens is the per-iteration token budget under GUIDE_POLICY_SPLIT_FUSE):
      * split_size: requests per prompt sub-batch (Sec. 3.3.1: the batch is divided into sub-batches of
      *   split_size, the remainder forming one more); 0 or >= the batch = the whole batch at once.
      * seg_tokens: tokens per prompt segment (Sec. 3.3.2: ceil(Lin / segment) splits, base value times
@@ -90,7 +91,12 @@ typedef struct guide_fw {
 
 typedef struct guide_len_pair { uint32_t lin, lout; } guide_len_pair;
 
-enum { GUIDE_POLICY_PREFILL_FIRST = 0 };
+enum { GUIDE_POLICY_PREFILL_FIRST = 0,  /* an iteration is either all waiting prompts, whole, or one decode step (Sec. 2.4.2) */
+       /* Dynamic split and fuse (the FastGen-like framework model, Sec. 2.3.2 / Sec. 3.1): every iteration
+        * carries seg_tokens tokens, one per request past its prompt, the rest prompt tokens in arrival
+        * order (long prompts spread over iterations, short ones sharing one).  Trace simulation only;
+        * needs seg_tokens >= 1 and split_size == 0 there.  The closed form ignores the policy. */
+       GUIDE_POLICY_SPLIT_FUSE = 1 };
 
 /* The candidate space of Sec. 3.1.  All pointers: host; copied by guide_space_create. */
 typedef struct guide_space_desc {

@@ -132,6 +132,8 @@ __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *g
         r.kv_block = f.kv_block;
         r.split = f.split_size;
         r.seg = f.seg_tokens;
+        r.policy = f.policy;
+        r.pad = 0;
         dr[i] = r;
         hfmem[i] = make_ulonglong2(r.usable, (u64)r.kv_block);
         double *q = rate10 + (size_t)i * 10;
@@ -306,6 +308,7 @@ int trace_on_device(guide_trace *t, DTrace *out) {
     d.view.max_tokens = t->max_tokens;
     d.view.any_zero = t->n_zero ? 1 : 0;
     d.view.sum_out = t->sum_out;
+    d.view.sum_in = t->sum_in;
     d.view.n_zero = t->n_zero;
     t->dev.push_back(d);
     *out = d.view;
@@ -441,7 +444,8 @@ int guide_space_create(const guide_space_desc *d, guide_space **out) {
                   std::isfinite(f.e_comm + f.t_ovh);
         for (int k = 0; k < 3; k++) ok = ok && f.e_c[k] > 0 && f.e_m[k] > 0 && std::isfinite(f.e_c[k] + f.e_m[k]);
         if (!ok) rc = fail(GUIDE_ERR_INVALID, "framework profile %zu has a bad efficiency, kv_block or reserve", i);
-        else if (f.policy != GUIDE_POLICY_PREFILL_FIRST) rc = fail(GUIDE_ERR_UNSUPPORTED, "framework profile %zu: unknown policy", i);
+        else if (f.policy != GUIDE_POLICY_PREFILL_FIRST && f.policy != GUIDE_POLICY_SPLIT_FUSE)
+            rc = fail(GUIDE_ERR_UNSUPPORTED, "framework profile %zu: unknown policy", i);
         s->chunked = s->chunked || f.split_size || f.seg_tokens;
     }
     if (!rc) {
@@ -516,6 +520,7 @@ int guide_trace_load(const double *arrival, const uint32_t *in_len, const uint32
             t->max_out = std::max(t->max_out, out_len[i]);
             t->max_tokens = std::max(t->max_tokens, in_len[i] + out_len[i]);
             t->sum_out += out_len[i];
+            t->sum_in += in_len[i];
         } else t->n_zero++;
     }
     if (rc) { delete t; return rc; }
@@ -555,9 +560,16 @@ int guide_simulate(const guide_space *space_c, const guide_trace *trace_c, const
         if (space->max_dp > 1)
             return fail(GUIDE_ERR_UNSUPPORTED, "the trace simulation models one replica: the space has a data-parallel degree of %u",
                         space->max_dp);
-        if (space->chunked)
-            return fail(GUIDE_ERR_UNSUPPORTED, "the trace simulation has the prompt-first policy only: a framework profile "
-                                               "sets split_size or seg_tokens");
+        for (size_t i = 0; i < space->fw.size(); i++) {
+            const guide_fw &f = space->fw[i];
+            if (f.policy == GUIDE_POLICY_PREFILL_FIRST && (f.split_size || f.seg_tokens))
+                return fail(GUIDE_ERR_UNSUPPORTED, "framework profile %zu: prompt-first iterations take whole prompts and whole "
+                                                   "batches; split_size and seg_tokens apply to the closed form or to the "
+                                                   "split-and-fuse policy", i);
+            if (f.policy == GUIDE_POLICY_SPLIT_FUSE && (f.seg_tokens == 0 || f.split_size != 0))
+                return fail(GUIDE_ERR_INVALID, "framework profile %zu: the split-and-fuse policy needs seg_tokens >= 1 (its token "
+                                               "budget per iteration) and split_size 0", i);
+        }
         if (space->max_batch > GUIDE_TRACE_MAX_BATCH)
             return fail(GUIDE_ERR_UNSUPPORTED, "the trace kernel keeps at most %u requests resident; the batch axis goes to %u",
                         GUIDE_TRACE_MAX_BATCH, space->max_batch);
@@ -571,8 +583,10 @@ int guide_simulate(const guide_space *space_c, const guide_trace *trace_c, const
     if (!trace) return launch_closed_form(ds, r, time_model, tp_model, *out, ticket, (cudaStream_t)stream);
     DTrace dt;
     if ((rc = trace_on_device(trace, &dt))) return rc;
+    u32 policies = 0;
+    for (const guide_fw &f : space->fw) policies |= f.policy == GUIDE_POLICY_SPLIT_FUSE ? 2u : 1u;
     return launch_trace_sim(ds, dt, r, time_model, tp_model, opts ? opts->max_iters : 0, *out, ws, ws_bytes,
-                            (cudaStream_t)stream);
+                            (cudaStream_t)stream, policies);
 }
 
 size_t guide_select_workspace_bytes(const guide_space *, uint32_t k) {

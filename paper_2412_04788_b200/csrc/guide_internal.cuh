@@ -57,7 +57,7 @@ struct guide_trace {
     std::vector<double> arrival;
     std::vector<uint32_t> in_len, out_len;
     uint32_t max_in = 0, max_out = 0, max_tokens = 0, n_zero = 0;
-    uint64_t sum_out = 0;
+    uint64_t sum_out = 0, sum_in = 0;
     std::mutex mu;
     std::vector<guide::DeviceTrace> dev;
 };
@@ -74,7 +74,7 @@ int launch_closed_form(const DSpace &s, Range r, int time_model, int tp_model, c
 // trace_sim.cu
 size_t trace_workspace_bytes(u32 n_req);
 int launch_trace_sim(const DSpace &s, const DTrace &t, Range r, int time_model, int tp_model, u64 max_iters,
-                     const guide_outputs &o, void *ws, size_t ws_bytes, cudaStream_t st);
+                     const guide_outputs &o, void *ws, size_t ws_bytes, cudaStream_t st, u32 policies);
 // select.cu
 size_t topk_workspace_bytes(u32 k);
 size_t pareto_workspace_bytes();

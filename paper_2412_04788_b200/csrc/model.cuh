@@ -32,6 +32,7 @@ struct DRate {
     u64 usable;   // MEM - (MEM/1000) * reserve_permille
     u32 flash, kv_block;
     u32 split, seg;   // requests per prompt sub-batch, tokens per prompt segment (0: whole batch / prompt)
+    u32 policy, pad;  // trace scheduling: GUIDE_POLICY_*; with SPLIT_FUSE seg is the token budget of an iteration
 };
 
 // one hardware x framework pair in the sorted walk of the model kernel
@@ -67,6 +68,7 @@ struct DTrace {
     u32 max_tokens;              // max over requests of in+out (0-length requests excluded)
     u32 any_zero;                // some request takes the config's lengths
     u64 sum_out;                 // sum of out_len over requests with explicit lengths
+    u64 sum_in;                  // sum of in_len over the same requests
     u32 n_zero;                  // number of requests taking the config's lengths
 };
 

@@ -1,0 +1,266 @@
+// Split-and-fuse scheduling for the trace simulation (the FastGen-like framework model: dynamic
+// splitting of prompts and fusion with decoding, Sec. 2.3.2 / Sec. 3.1 / Sec. 3.3), one warp per
+// config, called by k_trace_sim for configs whose framework has this policy.
+//
+// Every iteration carries about `budget` tokens: one per resident request past its prompt, the
+// rest prompt tokens in arrival order, so a long prompt is spread over several iterations and short
+// ones share one.  A chunk of q tokens attends the pdone + q tokens of its request seen so far; a
+// request emits its first token in the iteration that finishes its prompt.  Blocks for the whole
+// prompt are taken at admission; a decoding request whose last block is full takes one more, and
+// when none is free the youngest resident is evicted and recomputed later.
+//
+// Unlike the prompt-first path nothing is carried between iterations but the slots themselves:
+// every iteration scans them with all 32 lanes (plan, evaluate one stage time, apply, retire).
+#pragma once
+#include "guide_internal.cuh"
+
+namespace guide {
+
+struct FuseResult {
+    double clock, dec_time;
+    u64 dec_tok, n_iters, n_req_iters;
+};
+
+struct FuseSlots {
+    FuseResult res;                     // what the schedule hands back to the kernel around it
+    u32 req[GUIDE_TRACE_MAX_BATCH];     // request index, ascending
+    u32 seen[GUIDE_TRACE_MAX_BATCH];    // prompt phase: tokens processed so far; decoding: tokens cached
+    u32 todo[GUIDE_TRACE_MAX_BATCH];    // prompt (and recompute) tokens still to process; 0 = decoding
+    u32 rem[GUIDE_TRACE_MAX_BATCH];     // tokens still to emit
+    unsigned char fresh[GUIDE_TRACE_MAX_BATCH];   // no token emitted yet: the first one sets the TTFT
+};
+
+
+__device__ __forceinline__ u64 fuse_warp_sum(u64 v) {
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
+    return v;
+}
+__device__ __forceinline__ u32 fuse_warp_sum32(u32 v) {
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
+    return v;
+}
+// inclusive prefix sum over the lanes
+__device__ __forceinline__ u64 fuse_warp_scan(u64 v, u32 lane) {
+    for (int d = 1; d < 32; d <<= 1) {
+        const u64 o = __shfl_up_sync(0xFFFFFFFFu, v, d);
+        if (lane >= (u32)d) v += o;
+    }
+    return v;
+}
+
+// Runs the whole schedule of one config.  gen / first / tpot: the warp's per-request slices of the
+// workspace (tokens generated so far with the done flag in the top bit, first-token time, time per
+// output token).  Returns the status bits (0, or the iteration limit) and leaves the totals in
+// sl.res.  The model, the rates and the trace come as pointers to device memory so that the kernel
+// around this call keeps its own copies in registers.
+struct FuseTrace { const double *arrival; const u32 *in_len, *out_len; };
+
+template <int TIME_SUM>
+__device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, const double *arrival, const u32 *in_len,
+                                          const u32 *out_len, u32 n, u32 tt, u32 b, u32 Lin, u32 Lout, u64 blocks_total,
+                                          double lf, u64 max_iters, FuseSlots &sl, u32 *gen, double *first, double *tpot) {
+    const DModel m = *mp;
+    const DRate rt = *rp;
+    const FuseTrace tr = {arrival, in_len, out_len};
+    const double Nd = (double)m.N;
+    const u32 lane = threadIdx.x & 31;
+    const u32 lt_mask = (1u << lane) - 1;
+    const u32 blk = rt.kv_block, budget = rt.seg;
+    const u32 done_flag = 0x80000000u;
+    const double inf = __longlong_as_double(0x7FF0000000000000LL);
+    auto blocks_of = [&](u32 tokens) { return (tokens + blk - 1) / blk; };
+
+    double clock = 0.0, dec_time = 0.0;
+    u64 dec_tok = 0, n_iters = 0, n_req_iters = 0, free_blocks = blocks_total;
+    u32 next = 0, high_water = 0, nrun = 0, st = 0;
+    double arr_next = 0.0;
+    u32 need_next = 0;
+    auto refresh_head = [&]() {
+        while (next < high_water && (gen[next] & done_flag)) next++;
+        if (next < n) {
+            arr_next = __ldg(tr.arrival + next);
+            const u32 g = next < high_water ? gen[next] : 0u;
+            const u32 in = __ldg(tr.in_len + next);
+            need_next = blocks_of((in ? in : Lin) + g);
+        } else {
+            arr_next = inf; need_next = 0;
+        }
+    };
+    refresh_head();
+
+    for (;;) {
+        // ---- admit in arrival order, no overtaking ----
+        if (nrun < b && arr_next <= clock && need_next <= free_blocks) {
+            do {
+                const u32 g = next < high_water ? gen[next] : 0u;
+                u32 in = __ldg(tr.in_len + next), out = __ldg(tr.out_len + next);
+                if (in == 0) { in = Lin; out = Lout; }
+                free_blocks -= need_next;
+                if (lane == 0) {
+                    sl.req[nrun] = next;
+                    sl.seen[nrun] = 0;
+                    sl.todo[nrun] = in + g;                   // prompt + tokens to recompute
+                    sl.rem[nrun] = out - g;
+                    sl.fresh[nrun] = g == 0;
+                }
+                nrun++; next++;
+                if (next > high_water) high_water = next;
+                refresh_head();
+            } while (nrun < b && arr_next <= clock && need_next <= free_blocks);
+            __syncwarp();
+        }
+        if (nrun == 0) {
+            if (next >= n) break;
+            if (arr_next > clock) { clock = arr_next; continue; }
+            st |= GUIDE_ST_ITER;                                   // cannot happen when each request fits alone
+            break;
+        }
+        if (n_iters >= max_iters) { st |= GUIDE_ST_ITER; break; }
+
+        // ---- decoding requests whose last block is full need one more; evict the youngest if short ----
+        u32 needed = 0;
+        for (u32 base = 0; base < nrun; base += 32) {
+            const u32 k = base + lane;
+            needed += (k < nrun && sl.todo[k] == 0 && sl.seen[k] % blk == 0) ? 1u : 0u;
+        }
+        needed = fuse_warp_sum32(needed);
+        if (needed > free_blocks) {
+            while (needed > free_blocks) {
+                const u32 v = nrun - 1;
+                const u32 td = sl.todo[v], sn = sl.seen[v], rq = sl.req[v], rm = sl.rem[v];
+                free_blocks += blocks_of(sn + td);                 // what it took at admission, plus its decode blocks
+                if (td == 0 && sn % blk == 0) needed--;
+                const u32 out = __ldg(tr.in_len + rq) ? __ldg(tr.out_len + rq) : Lout;
+                __syncwarp();
+                if (lane == 0) gen[rq] = out - rm;
+                nrun--;
+                next = rq;
+            }
+            __syncwarp();
+            refresh_head();
+        }
+        free_blocks -= needed;
+
+        // ---- plan: one token per decoding request, the rest of the budget to prompts in order ----
+        u32 n_dec = 0;
+        u64 ctx = 0;
+        for (u32 base = 0; base < nrun; base += 32) {
+            const u32 k = base + lane;
+            if (k < nrun && sl.todo[k] == 0) { n_dec++; ctx += (u64)sl.seen[k] + 1; }   // cached tokens + the new one
+        }
+        n_dec = fuse_warp_sum32(n_dec);
+        ctx = fuse_warp_sum(ctx);
+        const u64 left0 = budget > n_dec ? budget - n_dec : 0;
+        u64 T = n_dec, A = ctx, C = ctx;
+        u32 E = n_dec, n_chunk = 0;
+        {
+            u64 carry = 0, pT = 0, pA = 0, pC = 0;
+            u32 pE = 0, pN = 0;
+            for (u32 base = 0; base < nrun && carry < left0; base += 32) {
+                const u32 k = base + lane;
+                const u64 td = k < nrun ? sl.todo[k] : 0;
+                const u64 incl = fuse_warp_scan(td, lane);
+                const u64 start = carry + incl - td;               // prompt tokens asked for by older requests
+                u64 q = 0;
+                if (td > 0 && start < left0) q = min(td, left0 - start);
+                if (q > 0) {
+                    const u64 upto = (u64)sl.seen[k] + q;
+                    pT += q; pA += q * upto; pC += upto; pN++;
+                    if (q == td) pE++;
+                }
+                carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+            }
+            T += fuse_warp_sum(pT); A += fuse_warp_sum(pA); C += fuse_warp_sum(pC);
+            E += fuse_warp_sum32(pE); n_chunk = fuse_warp_sum32(pN);
+        }
+        double t_iter;
+        {
+            TaskTab kt;
+            build_fixed_tasks(m, tt, T, E, 1, kt);
+            build_attn_tasks(m, tt, T, A, C, kt);
+            const double head = E ? eval_head<TIME_SUM>(kt, rt) : 0.0;   // nobody emits a token: no LM head
+            t_iter = combine_phase(eval_fixed<TIME_SUM>(kt, rt), eval_attn<TIME_SUM>(kt, rt), eval_comm(kt, rt), head, kt.Rd, Nd,
+                                   rt.tovh, lf);
+        }
+        const double after = clock + t_iter;
+
+        // ---- apply ----
+        bool any_done = false;
+        {
+            u64 carry = 0;
+            for (u32 base = 0; base < nrun; base += 32) {
+                const u32 k = base + lane;
+                const bool valid = k < nrun;
+                const u64 td = valid ? sl.todo[k] : 0;
+                const u64 incl = fuse_warp_scan(td, lane);
+                const u64 start = carry + incl - td;
+                if (valid) {
+                    if (td == 0) {                                  // decoded one token
+                        sl.seen[k] += 1;
+                        const u32 rm = sl.rem[k] - 1;
+                        sl.rem[k] = rm;
+                        any_done |= rm == 0;
+                    } else if (start < left0) {
+                        const u64 q = min(td, left0 - start);
+                        sl.seen[k] += (u32)q;
+                        sl.todo[k] = (u32)(td - q);
+                        if (q == td) {                              // prompt finished: first token
+                            const u32 rm = sl.rem[k] - 1;
+                            sl.rem[k] = rm;
+                            any_done |= rm == 0;
+                            if (sl.fresh[k]) { first[sl.req[k]] = after; sl.fresh[k] = 0; }
+                        }
+                    }
+                }
+                carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+            }
+        }
+        any_done = __any_sync(0xFFFFFFFFu, any_done);
+        if (n_dec > 0) { dec_time = dec_time + t_iter; dec_tok += n_dec; }
+        clock = after;
+        n_iters++;
+        n_req_iters += (u64)n_dec + n_chunk;
+        __syncwarp();
+
+        // ---- retire finished requests, keep the rest in order ----
+        if (any_done) {
+            u32 kept = 0;
+            u64 freed = 0;
+            const u32 n_before = nrun;
+            for (u32 base = 0; base < n_before; base += 32) {
+                const u32 k = base + lane;
+                const bool valid = k < n_before;
+                u32 rq = 0, sn = 0, td = 0, rm = 0, fr = 0;
+                if (valid) { rq = sl.req[k]; sn = sl.seen[k]; td = sl.todo[k]; rm = sl.rem[k]; fr = sl.fresh[k]; }
+                const bool done = valid && td == 0 && rm == 0;
+                if (done) {
+                    gen[rq] = done_flag;
+                    const u32 out = __ldg(tr.in_len + rq) ? __ldg(tr.out_len + rq) : Lout;
+                    tpot[rq] = out > 1 ? (clock - first[rq]) / (double)(out - 1) : 0.0;
+                    freed += blocks_of(sn);
+                }
+                const bool keep = valid && !done;
+                const u32 ballot = __ballot_sync(0xFFFFFFFFu, keep);
+                __syncwarp();
+                if (keep) {
+                    const u32 d = kept + __popc(ballot & lt_mask);
+                    sl.req[d] = rq; sl.seen[d] = sn; sl.todo[d] = td; sl.rem[d] = rm; sl.fresh[d] = (unsigned char)fr;
+                }
+                kept += __popc(ballot);
+                __syncwarp();
+            }
+            free_blocks += fuse_warp_sum(freed);
+            nrun = kept;
+            refresh_head();
+        }
+    }
+    __syncwarp();
+    if (lane == 0) {
+        sl.res.clock = clock; sl.res.dec_time = dec_time; sl.res.dec_tok = dec_tok; sl.res.n_iters = n_iters;
+        sl.res.n_req_iters = n_req_iters;
+    }
+    __syncwarp();
+    return st;
+}
+
+}  // namespace guide

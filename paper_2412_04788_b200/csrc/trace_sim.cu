@@ -23,6 +23,7 @@
 // output token) sit in a per-warp slice of the workspace.  The request trace is the same for every
 // config and is read through the read-only path, so it stays cache resident.
 #include "guide_internal.cuh"
+#include "trace_fuse.cuh"
 
 namespace guide {
 
@@ -88,6 +89,90 @@ __device__ __forceinline__ u64 work_to_index(const DSpace &s, u64 w, bool reorde
     return (mhf * s.n_b + b) * tl + x;
 }
 
+// Results of one simulated config: per-request values, means in request order, nearest-rank
+// percentiles (sorted in the tpot slice, which is free by then).  Called by the whole warp.
+__device__ __forceinline__ void write_trace_results(const guide_outputs &o, u64 j, u32 n, u32 st, u32 fit, double clock,
+                                                    double dec_time, u64 dec_tok, u64 n_iters, u64 n_req_iters, double cost_hr,
+                                                    const double *arrival, double *first, double *tpot, u32 lane) {
+    const double inf = __longlong_as_double(0x7FF0000000000000LL);
+    double *rq_ttft = o.req_ttft ? o.req_ttft + j * n : nullptr;
+    double *rq_tpot = o.req_tpot ? o.req_tpot + j * n : nullptr;
+    __syncwarp();
+    if (st) {
+        if (lane == 0) {
+            if (o.latency) o.latency[j] = inf;
+            if (o.ttft) o.ttft[j] = inf;
+            if (o.ttft_p50) o.ttft_p50[j] = inf;
+            if (o.ttft_p99) o.ttft_p99[j] = inf;
+            if (o.tpot) o.tpot[j] = inf;
+            if (o.thr_decode) o.thr_decode[j] = 0.0;
+            if (o.cost_per_hr) o.cost_per_hr[j] = inf;
+            if (o.cost_per_token) o.cost_per_token[j] = inf;
+            if (o.status) o.status[j] = (uint8_t)st;
+            if (o.bmax) o.bmax[j] = fit;
+            if (o.n_iters) o.n_iters[j] = 0;
+            if (o.n_req_iters) o.n_req_iters[j] = 0;
+        }
+        for (u32 i = lane; i < n; i += 32) {
+            if (rq_ttft) __stcs(rq_ttft + i, inf);
+            if (rq_tpot) __stcs(rq_tpot + i, inf);
+        }
+        return;
+    }
+    // means in request order: 32 values at a time, added one after the other
+    double s_ttft = 0.0, s_tpot = 0.0;
+    for (u32 base = 0; base < n; base += 32) {
+        const u32 i = base + lane;
+        double vt = 0.0, vp = 0.0;
+        if (i < n) {
+            vt = first[i] - __ldg(arrival + i);
+            vp = tpot[i];
+            if (rq_ttft) __stcs(rq_ttft + i, vt);
+            if (rq_tpot) __stcs(rq_tpot + i, vp);
+        }
+        const u32 lim = min(32u, n - base);
+        for (u32 l = 0; l < lim; l++) {
+            s_ttft = s_ttft + __shfl_sync(0xFFFFFFFFu, vt, l);
+            s_tpot = s_tpot + __shfl_sync(0xFFFFFFFFu, vp, l);
+        }
+        if (i < n) first[i] = vt;             // keep TTFT for the percentile sort
+    }
+    // nearest-rank percentiles: sort the TTFTs in the (now free) tpot slice
+    u32 P = 1;
+    while (P < n) P <<= 1;
+    __syncwarp();
+    for (u32 i = lane; i < P; i += 32) tpot[i] = i < n ? first[i] : inf;
+    __syncwarp();
+    for (u32 size = 2; size <= P; size <<= 1) {
+        for (u32 stride = size >> 1; stride > 0; stride >>= 1) {
+            for (u32 i = lane; i < (P >> 1); i += 32) {
+                const u32 lo = ((i & ~(stride - 1)) << 1) | (i & (stride - 1));
+                const u32 hi = lo + stride;
+                const bool up = (lo & size) == 0;
+                const double a = tpot[lo], bb = tpot[hi];
+                if ((bb < a) == up) { tpot[lo] = bb; tpot[hi] = a; }
+            }
+            __syncwarp();
+        }
+    }
+    if (lane == 0) {
+        const double nd = (double)n;
+        const double thr = dec_time > 0.0 ? cvt(dec_tok) / dec_time : 0.0;
+                    if (o.latency) o.latency[j] = clock;
+        if (o.ttft) o.ttft[j] = s_ttft / nd;
+        if (o.ttft_p50) o.ttft_p50[j] = tpot[(50ull * n + 99) / 100 - 1];
+        if (o.ttft_p99) o.ttft_p99[j] = tpot[(99ull * n + 99) / 100 - 1];
+        if (o.tpot) o.tpot[j] = s_tpot / nd;
+        if (o.thr_decode) o.thr_decode[j] = thr;
+        if (o.cost_per_hr) o.cost_per_hr[j] = cost_hr;
+        if (o.cost_per_token) o.cost_per_token[j] = thr > 0.0 ? (cost_hr / 3600.0) / thr : inf;
+        if (o.status) o.status[j] = 0;
+        if (o.bmax) o.bmax[j] = fit;
+        if (o.n_iters) o.n_iters[j] = n_iters;
+        if (o.n_req_iters) o.n_req_iters[j] = n_req_iters;
+    }
+}
+
 template <int TIME_SUM>
 __global__ void __launch_bounds__(SIM_THREADS, 3)
 k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide_outputs o, u32 *counter,
@@ -114,6 +199,7 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         const Cfg c = decode_index(s, idx);
         const DModel m = s.models[c.m];
         const DRate rt = s.rates[c.h * s.n_f + c.f];
+        if (rt.policy != GUIDE_POLICY_PREFILL_FIRST) continue;       // k_trace_fuse simulates those
         const u32 t = s.tp[c.t], b = s.batch[c.b];
         const uint2 pr = s.pairs[c.l];
         const u32 Lin = pr.x, Lout = pr.y, blk = rt.kv_block;
@@ -402,90 +488,71 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         }
 
         // ---- results ----
-        double *rq_ttft = o.req_ttft ? o.req_ttft + j * n : nullptr;
-        double *rq_tpot = o.req_tpot ? o.req_tpot + j * n : nullptr;
+        write_trace_results(o, j, n, st, fit, clock, dec_time, dec_tok, n_iters, n_req_iters, rt.price * (double)t, tr.arrival,
+                            first, tpot, lane);
         __syncwarp();
-        if (st) {
-            if (lane == 0) {
-                if (o.latency) o.latency[j] = inf;
-                if (o.ttft) o.ttft[j] = inf;
-                if (o.ttft_p50) o.ttft_p50[j] = inf;
-                if (o.ttft_p99) o.ttft_p99[j] = inf;
-                if (o.tpot) o.tpot[j] = inf;
-                if (o.thr_decode) o.thr_decode[j] = 0.0;
-                if (o.cost_per_hr) o.cost_per_hr[j] = inf;
-                if (o.cost_per_token) o.cost_per_token[j] = inf;
-                if (o.status) o.status[j] = (uint8_t)st;
-                if (o.bmax) o.bmax[j] = fit;
-                if (o.n_iters) o.n_iters[j] = 0;
-                if (o.n_req_iters) o.n_req_iters[j] = 0;
-            }
-            for (u32 i = lane; i < n; i += 32) {
-                if (rq_ttft) __stcs(rq_ttft + i, inf);
-                if (rq_tpot) __stcs(rq_tpot + i, inf);
-            }
-            continue;
+    }
+}
+
+// Configs whose framework schedules by split and fuse (trace_fuse.cuh): the same work loop, memory
+// check and results as k_trace_sim around fuse_schedule.  Configs of the other policy are skipped
+// here and simulated there.
+template <int TIME_SUM>
+__global__ void __launch_bounds__(SIM_THREADS, 3)
+k_trace_fuse(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide_outputs o, u32 *counter,
+             unsigned char *scratch, size_t per_warp, u32 gen_bytes, u32 first_bytes, int reorder) {
+    __shared__ FuseSlots sh[SIM_WARPS_PER_BLOCK];
+    const u32 lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const u32 warp_global = blockIdx.x * SIM_WARPS_PER_BLOCK + wib;
+    unsigned char *mine = scratch + (size_t)warp_global * per_warp;
+    u32 *gen = (u32 *)mine;
+    double *first = (double *)(mine + gen_bytes);
+    double *tpot = (double *)(mine + gen_bytes + first_bytes);
+    const u32 n = tr.n;
+    for (;;) {
+        u64 w = 0;
+        if (lane == 0) w = atomicAdd(counter, 1u);
+        w = __shfl_sync(0xFFFFFFFFu, w, 0);
+        if (w >= r.count) break;
+        const u64 idx = reorder ? work_to_index(s, w, true) : r.first + w;
+        const u64 j = idx - r.first;
+        const Cfg c = decode_index(s, idx);
+        const DRate *rp = s.rates + (c.h * s.n_f + c.f);
+        if (rp->policy != GUIDE_POLICY_SPLIT_FUSE) continue;
+        const DModel *mp = s.models + c.m;
+        const u32 t = s.tp[c.t], b = s.batch[c.b];
+        const uint2 pr = s.pairs[c.l];
+        const u32 Lin = pr.x, Lout = pr.y, blk = rp->kv_block;
+        const MemInfo mi = mem_info(*mp, t);
+        // ---- what fits (Sec. 3.2 Step 1) ----
+        const u64 usable = rp->usable;
+        const u64 blocks_total = usable > mi.w_gpu ? floor_div(usable - mi.w_gpu, (u64)blk * mi.kv_tok) : 0;
+        const u32 longest = max(tr.max_tokens, tr.any_zero ? Lin + Lout : 0u);
+        const u64 worst = ceil_div32(longest, blk);
+        u32 st = 0;
+        if (usable <= mi.w_gpu) st |= GUIDE_ST_WEIGHTS;
+        if (worst > blocks_total) st |= GUIDE_ST_KV;
+        if ((mp->nh & (t - 1)) != 0 || (mp->nkv & (t - 1)) != 0) st |= GUIDE_ST_HEADS;
+        const u32 fit = clamp_u32(blocks_total / worst);
+        // prompt chunks take iterations too: the default backstop counts prompt tokens as well
+        const u64 sched_tokens = tr.sum_out + tr.sum_in + (u64)tr.n_zero * ((u64)Lin + Lout);
+        const u64 max_iters = max_iters_opt ? max_iters_opt : 64 * sched_tokens + 4 * (u64)n;
+        FuseResult fr = {0.0, 0.0, 0, 0, 0};
+        if (!st) {
+            __syncwarp();
+            st |= fuse_schedule<TIME_SUM>(mp, rp, tr.arrival, tr.in_len, tr.out_len, n, tp_model ? 1u : t, b, Lin, Lout, blocks_total,
+                                          log2_rule_factor(t, tp_model), max_iters, sh[wib], gen, first, tpot);
+            fr = sh[wib].res;
         }
-        // means in request order: 32 values at a time, added one after the other
-        double s_ttft = 0.0, s_tpot = 0.0;
-        for (u32 base = 0; base < n; base += 32) {
-            const u32 i = base + lane;
-            double vt = 0.0, vp = 0.0;
-            if (i < n) {
-                vt = first[i] - __ldg(tr.arrival + i);
-                vp = tpot[i];
-                if (rq_ttft) __stcs(rq_ttft + i, vt);
-                if (rq_tpot) __stcs(rq_tpot + i, vp);
-            }
-            const u32 lim = min(32u, n - base);
-            for (u32 l = 0; l < lim; l++) {
-                s_ttft = s_ttft + __shfl_sync(0xFFFFFFFFu, vt, l);
-                s_tpot = s_tpot + __shfl_sync(0xFFFFFFFFu, vp, l);
-            }
-            if (i < n) first[i] = vt;             // keep TTFT for the percentile sort
-        }
-        // nearest-rank percentiles: sort the TTFTs in the (now free) tpot slice
-        u32 P = 1;
-        while (P < n) P <<= 1;
-        __syncwarp();
-        for (u32 i = lane; i < P; i += 32) tpot[i] = i < n ? first[i] : inf;
-        __syncwarp();
-        for (u32 size = 2; size <= P; size <<= 1) {
-            for (u32 stride = size >> 1; stride > 0; stride >>= 1) {
-                for (u32 i = lane; i < (P >> 1); i += 32) {
-                    const u32 lo = ((i & ~(stride - 1)) << 1) | (i & (stride - 1));
-                    const u32 hi = lo + stride;
-                    const bool up = (lo & size) == 0;
-                    const double a = tpot[lo], bb = tpot[hi];
-                    if ((bb < a) == up) { tpot[lo] = bb; tpot[hi] = a; }
-                }
-                __syncwarp();
-            }
-        }
-        if (lane == 0) {
-            const double nd = (double)n;
-            const double thr = dec_time > 0.0 ? cvt(dec_tok) / dec_time : 0.0;
-            const double cost_hr = rt.price * (double)t;
-            if (o.latency) o.latency[j] = clock;
-            if (o.ttft) o.ttft[j] = s_ttft / nd;
-            if (o.ttft_p50) o.ttft_p50[j] = tpot[(50ull * n + 99) / 100 - 1];
-            if (o.ttft_p99) o.ttft_p99[j] = tpot[(99ull * n + 99) / 100 - 1];
-            if (o.tpot) o.tpot[j] = s_tpot / nd;
-            if (o.thr_decode) o.thr_decode[j] = thr;
-            if (o.cost_per_hr) o.cost_per_hr[j] = cost_hr;
-            if (o.cost_per_token) o.cost_per_token[j] = thr > 0.0 ? (cost_hr / 3600.0) / thr : inf;
-            if (o.status) o.status[j] = 0;
-            if (o.bmax) o.bmax[j] = fit;
-            if (o.n_iters) o.n_iters[j] = n_iters;
-            if (o.n_req_iters) o.n_req_iters[j] = n_req_iters;
-        }
+        write_trace_results(o, j, n, st, fit, fr.clock, fr.dec_time, fr.dec_tok, fr.n_iters, fr.n_req_iters,
+                            rp->price * (double)t, tr.arrival, first, tpot, lane);
         __syncwarp();
     }
 }
 
 template <int TIME_SUM>
 static int launch_one(const DSpace &s, const DTrace &t, Range r, int tp_model, u64 max_iters, const guide_outputs &o,
-                      void *ws, cudaStream_t st) {
+                      void *ws, cudaStream_t st, u32 policies) {
     const size_t pw = per_warp_bytes(t.n);
     const u32 gen_bytes = (u32)(((size_t)t.n * 4 + 255) / 256 * 256);
     const u32 first_bytes = (u32)(((size_t)t.n * 8 + 255) / 256 * 256);
@@ -498,19 +565,29 @@ static int launch_one(const DSpace &s, const DTrace &t, Range r, int tp_model, u
     blocks = (u32)std::min<u64>(blocks, (r.count + SIM_WARPS_PER_BLOCK - 1) / SIM_WARPS_PER_BLOCK);
     const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
     const int reorder = r.first == 0 && r.count == total;
-    GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
     unsigned char *scratch = (unsigned char *)ws + 256;
-    k_trace_sim<TIME_SUM><<<blocks, SIM_THREADS, 0, st>>>(s, t, r, tp_model, max_iters, o, (u32 *)ws, scratch, pw,
-                                                         gen_bytes, first_bytes, reorder);
-    GUIDE_CUDA(cudaGetLastError());
+    // one kernel per scheduling policy present in the space; each skips the other's configs
+    if (policies & 1) {
+        GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
+        k_trace_sim<TIME_SUM><<<blocks, SIM_THREADS, 0, st>>>(s, t, r, tp_model, max_iters, o, (u32 *)ws, scratch, pw,
+                                                             gen_bytes, first_bytes, reorder);
+        GUIDE_CUDA(cudaGetLastError());
+    }
+    if (policies & 2) {
+        GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
+        k_trace_fuse<TIME_SUM><<<blocks, SIM_THREADS, 0, st>>>(s, t, r, tp_model, max_iters, o, (u32 *)ws, scratch, pw,
+                                                              gen_bytes, first_bytes, reorder);
+        GUIDE_CUDA(cudaGetLastError());
+    }
     return GUIDE_OK;
 }
 
+// policies: bit 0 = some framework schedules prompt-first, bit 1 = some by split and fuse
 int launch_trace_sim(const DSpace &s, const DTrace &t, Range r, int time_model, int tp_model, u64 max_iters,
-                     const guide_outputs &o, void *ws, size_t, cudaStream_t st) {
+                     const guide_outputs &o, void *ws, size_t, cudaStream_t st, u32 policies) {
     if (r.count > 0xFFFFFFF0ull) return fail(GUIDE_ERR_UNSUPPORTED, "at most 2^32 - 16 configs per trace launch");
-    return time_model ? launch_one<1>(s, t, r, tp_model, max_iters, o, ws, st)
-                      : launch_one<0>(s, t, r, tp_model, max_iters, o, ws, st);
+    return time_model ? launch_one<1>(s, t, r, tp_model, max_iters, o, ws, st, policies)
+                      : launch_one<0>(s, t, r, tp_model, max_iters, o, ws, st, policies);
 }
 
 }  // namespace guide

@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libguide.so")
 GUIDE_OK, GUIDE_ERR_INVALID, GUIDE_ERR_OVERFLOW, GUIDE_ERR_UNSUPPORTED = 0, -1, -2, -3
 GUIDE_ERR_CUDA, GUIDE_ERR_WORKSPACE, GUIDE_ERR_ITER_LIMIT = -4, -5, -6
 TIME_MAX, TIME_SUM = 0, 1
+GUIDE_POLICY_PREFILL_FIRST, GUIDE_POLICY_SPLIT_FUSE = 0, 1
 TP_EXPLICIT, TP_PAPER_LOG2 = 0, 1
 ST_WEIGHTS, ST_KV, ST_HEADS, ST_ITER = 1, 2, 4, 8
 METRICS = {"latency": 0, "ttft": 1, "ttft_p99": 2, "tpot": 3, "throughput": 4, "cost_per_hr": 5,
