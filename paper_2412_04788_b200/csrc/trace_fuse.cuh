@@ -9,8 +9,10 @@
 // prompt are taken at admission; a decoding request whose last block is full takes one more, and
 // when none is free the youngest resident is evicted and recomputed later.
 //
-// Unlike the prompt-first path nothing is carried between iterations but the slots themselves:
-// every iteration scans them with all 32 lanes (plan, evaluate one stage time, apply, retire).
+// Unlike the prompt-first path little is carried between iterations besides the slots themselves:
+// every iteration scans them with all 32 lanes (count the decoders, plan the prompt chunks while
+// some request is in its prompt, evaluate one stage time, apply, retire); the non-attention terms
+// of the stage time are kept while the iteration's token counts repeat.
 #pragma once
 #include "guide_internal.cuh"
 
@@ -73,6 +75,9 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
     double clock = 0.0, dec_time = 0.0;
     u64 dec_tok = 0, n_iters = 0, n_req_iters = 0, free_blocks = blocks_total;
     u32 next = 0, high_water = 0, nrun = 0, st = 0;
+    u32 n_pre = 0;                                   // residents still in their prompt
+    u64 dc_T = ~0ull, dc_E = ~0ull;                  // stage terms kept while the token counts repeat
+    double dc_fix = 0.0, dc_comm = 0.0, dc_head = 0.0;
     double arr_next = 0.0;
     u32 need_next = 0;
     auto refresh_head = [&]() {
@@ -103,7 +108,7 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
                     sl.rem[nrun] = out - g;
                     sl.fresh[nrun] = g == 0;
                 }
-                nrun++; next++;
+                nrun++; next++; n_pre++;
                 if (next > high_water) high_water = next;
                 refresh_head();
             } while (nrun < b && arr_next <= clock && need_next <= free_blocks);
@@ -117,19 +122,33 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
         }
         if (n_iters >= max_iters) { st |= GUIDE_ST_ITER; break; }
 
-        // ---- decoding requests whose last block is full need one more; evict the youngest if short ----
-        u32 needed = 0;
-        for (u32 base = 0; base < nrun; base += 32) {
-            const u32 k = base + lane;
-            needed += (k < nrun && sl.todo[k] == 0 && sl.seen[k] % blk == 0) ? 1u : 0u;
-        }
-        needed = fuse_warp_sum32(needed);
-        if (needed > free_blocks) {
+        // ---- one pass over the slots: decoding requests (one token each, context = cached + 1) and
+        // how many of them need one more block because their last one is full ----
+        u32 n_dec, needed;
+        u64 ctx;
+        auto count_decoders = [&]() {
+            u32 packed = 0;                                        // needed << 16 | decoders: both <= 256 per lane sum
+            u64 c = 0;
+            for (u32 base = 0; base < nrun; base += 32) {
+                const u32 k = base + lane;
+                if (k < nrun && sl.todo[k] == 0) {
+                    const u32 sn = sl.seen[k];
+                    packed += 1u + ((sn % blk == 0) ? 0x10000u : 0u);
+                    c += (u64)sn + 1;
+                }
+            }
+            packed = fuse_warp_sum32(packed);
+            n_dec = packed & 0xFFFFu; needed = packed >> 16;
+            ctx = fuse_warp_sum(c);
+        };
+        count_decoders();
+        if (needed > free_blocks) {                                // evict the youngest, recompute later
             while (needed > free_blocks) {
                 const u32 v = nrun - 1;
                 const u32 td = sl.todo[v], sn = sl.seen[v], rq = sl.req[v], rm = sl.rem[v];
                 free_blocks += blocks_of(sn + td);                 // what it took at admission, plus its decode blocks
                 if (td == 0 && sn % blk == 0) needed--;
+                if (td > 0) n_pre--;
                 const u32 out = __ldg(tr.in_len + rq) ? __ldg(tr.out_len + rq) : Lout;
                 __syncwarp();
                 if (lane == 0) gen[rq] = out - rm;
@@ -138,55 +157,66 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
             }
             __syncwarp();
             refresh_head();
+            count_decoders();
         }
         free_blocks -= needed;
 
-        // ---- plan: one token per decoding request, the rest of the budget to prompts in order ----
-        u32 n_dec = 0;
-        u64 ctx = 0;
-        for (u32 base = 0; base < nrun; base += 32) {
-            const u32 k = base + lane;
-            if (k < nrun && sl.todo[k] == 0) { n_dec++; ctx += (u64)sl.seen[k] + 1; }   // cached tokens + the new one
-        }
-        n_dec = fuse_warp_sum32(n_dec);
-        ctx = fuse_warp_sum(ctx);
+        // ---- plan: the rest of the budget goes to prompts in arrival order ----
         const u64 left0 = budget > n_dec ? budget - n_dec : 0;
         u64 T = n_dec, A = ctx, C = ctx;
-        u32 E = n_dec, n_chunk = 0;
-        {
+        u32 E = n_dec, n_chunk = 0, n_finish = 0;
+        const bool chunks = n_pre > 0 && left0 > 0;
+        if (chunks) {
             u64 carry = 0, pT = 0, pA = 0, pC = 0;
-            u32 pE = 0, pN = 0;
+            u32 pEN = 0;                                           // finishing << 16 | chunks
             for (u32 base = 0; base < nrun && carry < left0; base += 32) {
                 const u32 k = base + lane;
                 const u64 td = k < nrun ? sl.todo[k] : 0;
                 const u64 incl = fuse_warp_scan(td, lane);
                 const u64 start = carry + incl - td;               // prompt tokens asked for by older requests
-                u64 q = 0;
-                if (td > 0 && start < left0) q = min(td, left0 - start);
-                if (q > 0) {
+                if (td > 0 && start < left0) {
+                    const u64 q = min(td, left0 - start);
                     const u64 upto = (u64)sl.seen[k] + q;
-                    pT += q; pA += q * upto; pC += upto; pN++;
-                    if (q == td) pE++;
+                    pT += q; pA += q * upto; pC += upto;
+                    pEN += 1u + (q == td ? 0x10000u : 0u);
                 }
                 carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
             }
             T += fuse_warp_sum(pT); A += fuse_warp_sum(pA); C += fuse_warp_sum(pC);
-            E += fuse_warp_sum32(pE); n_chunk = fuse_warp_sum32(pN);
+            pEN = fuse_warp_sum32(pEN);
+            n_chunk = pEN & 0xFFFFu; n_finish = pEN >> 16;
+            E += n_finish;
+        }
+        // ---- one stage time from (T, E, A, C); everything but attention is kept while T and E repeat ----
+        if (T != dc_T || E != dc_E) {
+            TaskTab kf;
+            build_fixed_tasks(m, tt, T, E, 1, kf);
+            dc_T = T; dc_E = E;
+            dc_fix = eval_fixed<TIME_SUM>(kf, rt);
+            dc_comm = eval_comm(kf, rt);
+            dc_head = E ? eval_head<TIME_SUM>(kf, rt) : 0.0;       // nobody emits a token: no LM head
         }
         double t_iter;
         {
-            TaskTab kt;
-            build_fixed_tasks(m, tt, T, E, 1, kt);
-            build_attn_tasks(m, tt, T, A, C, kt);
-            const double head = E ? eval_head<TIME_SUM>(kt, rt) : 0.0;   // nobody emits a token: no LM head
-            t_iter = combine_phase(eval_fixed<TIME_SUM>(kt, rt), eval_attn<TIME_SUM>(kt, rt), eval_comm(kt, rt), head, kt.Rd, Nd,
-                                   rt.tovh, lf);
+            TaskTab ka;
+            build_attn_tasks(m, tt, T, A, C, ka);
+            t_iter = combine_phase(dc_fix, eval_attn<TIME_SUM>(ka, rt), dc_comm, dc_head, 1.0, Nd, rt.tovh, lf);
         }
         const double after = clock + t_iter;
 
         // ---- apply ----
         bool any_done = false;
-        {
+        if (!chunks) {
+            for (u32 base = 0; base < nrun; base += 32) {
+                const u32 k = base + lane;
+                if (k < nrun && sl.todo[k] == 0) {                  // decoded one token
+                    sl.seen[k] += 1;
+                    const u32 rm = sl.rem[k] - 1;
+                    sl.rem[k] = rm;
+                    any_done |= rm == 0;
+                }
+            }
+        } else {
             u64 carry = 0;
             for (u32 base = 0; base < nrun; base += 32) {
                 const u32 k = base + lane;
@@ -214,6 +244,7 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
                 }
                 carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
             }
+            n_pre -= n_finish;
         }
         any_done = __any_sync(0xFFFFFFFFu, any_done);
         if (n_dec > 0) { dec_time = dec_time + t_iter; dec_tok += n_dec; }
