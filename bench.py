@@ -8,7 +8,8 @@ guide_simulate (memory check, task list, roofline, metrics -> 6 fp64 arrays + ma
 bandwidth-bound memory kernel and a model kernel for the configs that fit, side by side),
 guide_select_topk (constraint filter + top-64 by cost per token) and guide_pareto (latency vs $/h;
 both: a sampled bound, one filter pass at memory speed, an exact finish),
-with the space tables already resident on the device.  `value` is configs per second over the K
+with the space tables already resident on the device; the two selections read the same metrics and
+run side by side on two streams.  `value` is configs per second over the K
 timed steps; the 0.89 GB of outputs a step writes and reads back exceed L2 several times over, so
 no flush is needed between steps.  The trace-driven workloads (1, 3, 4), the 983,040-config grid
 (2) and the fused (nothing materialised) selection on workload 5 are timed once each afterwards
@@ -40,7 +41,7 @@ BYTES_SIM = 6 * 8 + 1 + 4          # six fp64 metrics + status + bmax written pe
 # dram__bytes_read.sum + dram__bytes_write.sum of one guide_simulate call on the full workload 5: the
 # k_closed_form_memory and k_closed_form_model launches together (profiles/k_closed_form_split_c5.md);
 # only meaningful for that size and those kernel versions
-K1_TRAFFIC_C5 = 644_400_000 + 151_100_000 + 1_000_000
+K1_TRAFFIC_C5 = 644_500_000 + 150_700_000 + 100_000
 SIM_FIELDS = ("latency", "ttft", "tpot", "thr_decode", "cost_per_hr", "cost_per_token", "status", "bmax")
 TRACE_FIELDS = ("latency", "ttft", "ttft_p50", "ttft_p99", "tpot", "thr_decode", "cost_per_hr", "cost_per_token",
                 "status", "bmax", "n_iters", "n_req_iters")
