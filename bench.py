@@ -250,10 +250,10 @@ def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full, fraction
                             "kernel_launches": 2 + 6 + 5 + 5 + 4}
             del p
         elif k == 8:
-            # workload 3 on an eighth of its hardware axis with every framework on the split-and-fuse
+            # workload 3 on half of its hardware axis with every framework on the split-and-fuse
             # policy (token budgets 256 .. 8192 per iteration)
             import numpy as np
-            w = inputs.workload(3, scale=0.125, trace_scale=1.0)
+            w = inputs.workload(3, scale=fraction or 0.5, trace_scale=1.0)
             space = dict(w["space"])
             fw_i = np.array(space["fw_i"], dtype=np.uint32).copy()
             fw_i[:, 3] = guide.GUIDE_POLICY_SPLIT_FUSE
@@ -268,8 +268,8 @@ def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full, fraction
             req_iters = int(out["n_req_iters"].sum().item())
             res["C3-split-fuse"] = {"configs": n, "requests": tr.n, "feasible": int((out["status"] == 0).sum().item()),
                                     "ms": best, "configs_per_s": n / best * 1e3, "iters_per_s": iters / best * 1e3,
-                                    "request_iters_per_s": req_iters / best * 1e3, "hardware_axis_fraction": 0.125,
-                                    "kernel_launches": 1}
+                                    "request_iters_per_s": req_iters / best * 1e3,
+                                    "hardware_axis_fraction": fraction or 0.5, "kernel_launches": 1}
             del out, ws
         elif k in (6, 7):
             # the (dp, tp) sweep under a budget of 8 GPUs (whole-space kernels) and workload 2 with

@@ -18,6 +18,8 @@
 
 namespace guide {
 
+static constexpr u32 FUSE_HIST = 64;      // block sizes up to this take the decode-only runs
+
 struct FuseResult {
     double clock, dec_time;
     u64 dec_tok, n_iters, n_req_iters;
@@ -30,6 +32,7 @@ struct FuseSlots {
     u32 todo[GUIDE_TRACE_MAX_BATCH];    // prompt (and recompute) tokens still to process; 0 = decoding
     u32 rem[GUIDE_TRACE_MAX_BATCH];     // tokens still to emit
     unsigned char fresh[GUIDE_TRACE_MAX_BATCH];   // no token emitted yet: the first one sets the TTFT
+    u32 hist[FUSE_HIST];                // decode-only runs: residents per (cached tokens mod block size)
 };
 
 
@@ -93,6 +96,52 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
     };
     refresh_head();
 
+    // one stage time from (T, E, A, C); everything but attention is kept while T and E repeat
+    auto stage_time = [&](u64 T, u64 E, u64 A, u64 C) {
+        if (T != dc_T || E != dc_E) {
+            TaskTab kf;
+            build_fixed_tasks(m, tt, T, E, 1, kf);
+            dc_T = T; dc_E = E;
+            dc_fix = eval_fixed<TIME_SUM>(kf, rt);
+            dc_comm = eval_comm(kf, rt);
+            dc_head = E ? eval_head<TIME_SUM>(kf, rt) : 0.0;       // nobody emits a token: no LM head
+        }
+        TaskTab ka;
+        build_attn_tasks(m, tt, T, A, C, ka);
+        return combine_phase(dc_fix, eval_attn<TIME_SUM>(ka, rt), dc_comm, dc_head, 1.0, Nd, rt.tovh, lf);
+    };
+    // retire finished requests, keep the rest in order
+    auto retire = [&]() {
+        u32 kept = 0;
+        u64 freed = 0;
+        const u32 n_before = nrun;
+        for (u32 base = 0; base < n_before; base += 32) {
+            const u32 k = base + lane;
+            const bool valid = k < n_before;
+            u32 rq = 0, sn = 0, td = 0, rm = 0, fr = 0;
+            if (valid) { rq = sl.req[k]; sn = sl.seen[k]; td = sl.todo[k]; rm = sl.rem[k]; fr = sl.fresh[k]; }
+            const bool done = valid && td == 0 && rm == 0;
+            if (done) {
+                gen[rq] = done_flag;
+                const u32 out = __ldg(tr.in_len + rq) ? __ldg(tr.out_len + rq) : Lout;
+                tpot[rq] = out > 1 ? (clock - first[rq]) / (double)(out - 1) : 0.0;
+                freed += blocks_of(sn);
+            }
+            const bool keep = valid && !done;
+            const u32 ballot = __ballot_sync(0xFFFFFFFFu, keep);
+            __syncwarp();
+            if (keep) {
+                const u32 d = kept + __popc(ballot & lt_mask);
+                sl.req[d] = rq; sl.seen[d] = sn; sl.todo[d] = td; sl.rem[d] = rm; sl.fresh[d] = (unsigned char)fr;
+            }
+            kept += __popc(ballot);
+            __syncwarp();
+        }
+        free_blocks += fuse_warp_sum(freed);
+        nrun = kept;
+        refresh_head();
+    };
+
     for (;;) {
         // ---- admit in arrival order, no overtaking ----
         if (nrun < b && arr_next <= clock && need_next <= free_blocks) {
@@ -121,6 +170,57 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
             break;
         }
         if (n_iters >= max_iters) { st |= GUIDE_ST_ITER; break; }
+
+        // ---- nobody is in its prompt: a run of decode iterations up to the next event (a completion,
+        // a block shortage, room for the head of the queue, the iteration limit).  One pass finds the
+        // summed context, the first completion and how many residents sit at each offset within a
+        // block; the iterations of the run then touch no slot, and one pass settles them. ----
+        if (n_pre == 0 && blk <= FUSE_HIST) {
+            for (u32 i = lane; i < blk; i += 32) sl.hist[i] = 0;
+            __syncwarp();
+            u64 c = 0;
+            u32 local_min = 0xFFFFFFFFu;
+            for (u32 base = 0; base < nrun; base += 32) {
+                const u32 k = base + lane;
+                if (k < nrun) {
+                    const u32 sn = sl.seen[k];
+                    c += (u64)sn + 1;
+                    local_min = min(local_min, sl.rem[k]);
+                    atomicAdd(&sl.hist[sn % blk], 1u);
+                }
+            }
+            u64 ctx_i = fuse_warp_sum(c);
+            for (int d = 16; d > 0; d >>= 1) local_min = min(local_min, __shfl_xor_sync(0xFFFFFFFFu, local_min, d));
+            const u32 min_rem = local_min;
+            __syncwarp();
+            const u64 cap_left = max_iters - n_iters;
+            const bool room = nrun < b;
+            u32 it = 0, off = 0;                                   // off = it mod block size
+            for (;;) {
+                const u32 need_i = sl.hist[off == 0 ? 0 : blk - off];    // residents whose last block is full now
+                if (need_i > free_blocks) break;                   // eviction: the general path below
+                free_blocks -= need_i;
+                const double t_i = stage_time(nrun, nrun, ctx_i, ctx_i);
+                clock = clock + t_i;
+                dec_time = dec_time + t_i;
+                it++;
+                off = off + 1 == blk ? 0 : off + 1;
+                ctx_i += nrun;
+                if (it == min_rem || it == cap_left) break;
+                if (room && arr_next <= clock && need_next <= free_blocks) break;
+            }
+            if (it > 0) {
+                for (u32 base = 0; base < nrun; base += 32) {
+                    const u32 k = base + lane;
+                    if (k < nrun) { sl.seen[k] += it; sl.rem[k] -= it; }
+                }
+                const u64 tok = (u64)it * nrun;
+                dec_tok += tok; n_req_iters += tok; n_iters += it;
+                __syncwarp();
+                if (it == min_rem) retire();
+                continue;
+            }
+        }
 
         // ---- one pass over the slots: decoding requests (one token each, context = cached + 1) and
         // how many of them need one more block because their last one is full ----
@@ -187,21 +287,7 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
             n_chunk = pEN & 0xFFFFu; n_finish = pEN >> 16;
             E += n_finish;
         }
-        // ---- one stage time from (T, E, A, C); everything but attention is kept while T and E repeat ----
-        if (T != dc_T || E != dc_E) {
-            TaskTab kf;
-            build_fixed_tasks(m, tt, T, E, 1, kf);
-            dc_T = T; dc_E = E;
-            dc_fix = eval_fixed<TIME_SUM>(kf, rt);
-            dc_comm = eval_comm(kf, rt);
-            dc_head = E ? eval_head<TIME_SUM>(kf, rt) : 0.0;       // nobody emits a token: no LM head
-        }
-        double t_iter;
-        {
-            TaskTab ka;
-            build_attn_tasks(m, tt, T, A, C, ka);
-            t_iter = combine_phase(dc_fix, eval_attn<TIME_SUM>(ka, rt), dc_comm, dc_head, 1.0, Nd, rt.tovh, lf);
-        }
+        const double t_iter = stage_time(T, E, A, C);
         const double after = clock + t_iter;
 
         // ---- apply ----
@@ -253,37 +339,7 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
         n_req_iters += (u64)n_dec + n_chunk;
         __syncwarp();
 
-        // ---- retire finished requests, keep the rest in order ----
-        if (any_done) {
-            u32 kept = 0;
-            u64 freed = 0;
-            const u32 n_before = nrun;
-            for (u32 base = 0; base < n_before; base += 32) {
-                const u32 k = base + lane;
-                const bool valid = k < n_before;
-                u32 rq = 0, sn = 0, td = 0, rm = 0, fr = 0;
-                if (valid) { rq = sl.req[k]; sn = sl.seen[k]; td = sl.todo[k]; rm = sl.rem[k]; fr = sl.fresh[k]; }
-                const bool done = valid && td == 0 && rm == 0;
-                if (done) {
-                    gen[rq] = done_flag;
-                    const u32 out = __ldg(tr.in_len + rq) ? __ldg(tr.out_len + rq) : Lout;
-                    tpot[rq] = out > 1 ? (clock - first[rq]) / (double)(out - 1) : 0.0;
-                    freed += blocks_of(sn);
-                }
-                const bool keep = valid && !done;
-                const u32 ballot = __ballot_sync(0xFFFFFFFFu, keep);
-                __syncwarp();
-                if (keep) {
-                    const u32 d = kept + __popc(ballot & lt_mask);
-                    sl.req[d] = rq; sl.seen[d] = sn; sl.todo[d] = td; sl.rem[d] = rm; sl.fresh[d] = (unsigned char)fr;
-                }
-                kept += __popc(ballot);
-                __syncwarp();
-            }
-            free_blocks += fuse_warp_sum(freed);
-            nrun = kept;
-            refresh_head();
-        }
+        if (any_done) retire();
     }
     __syncwarp();
     if (lane == 0) {
