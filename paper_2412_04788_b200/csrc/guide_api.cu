@@ -172,14 +172,16 @@ static std::vector<HfSorted> sorted_pairs(const guide_space &s) {
     return v;
 }
 
-// Per model, the foursomes (four consecutive positions) of the (TP, length) plane by growing memory
-// need of their cheapest position (weights per GPU plus the KV cache of a middle batch size);
-// foursomes whose TP degree does not divide the heads last.  Lanes of a warp then fit about the
-// same number of pairs.  When the plane does not divide into foursomes the table is not used.
-static std::vector<u32> plane_orders(const guide_space &s) {
-    const size_t n_t = s.tp.size(), n_l = s.pairs.size(), n_tl = n_t * n_l, n_four = n_tl / 4;
+// Per model, the groups of `group` consecutive positions of the (TP, length) plane (foursomes: one
+// memory sector of every metric array; lines of sixteen: 128 bytes) by growing memory need of
+// their cheapest position (weights per GPU plus the KV cache of a middle batch size); groups whose
+// TP degree does not divide the heads last.  Heavy work items then come first and lanes of a warp
+// fit about the same number of pairs.  When the plane does not divide into such groups the table
+// is not used.
+static std::vector<u32> plane_orders(const guide_space &s, size_t group) {
+    const size_t n_t = s.tp.size(), n_l = s.pairs.size(), n_tl = n_t * n_l, n_four = n_tl / group;
     std::vector<u32> out(s.models.size() * std::max<size_t>(n_four, 1), 0);
-    if (n_l % 4 != 0) return out;
+    if (n_l % group != 0) return out;
     const double b_ref = (double)s.batch[s.batch.size() / 2];
     const double blk = (double)std::max<u32>(s.fw[0].kv_block, 1);
     std::vector<double> key(n_four);
@@ -189,12 +191,12 @@ static std::vector<u32> plane_orders(const guide_space &s) {
         const double wbytes = (m.n_layers * (2 * H * H + 2 * H * Dkv + (2.0 + m.gated) * H * I) + 2 * V * H) * m.w_bytes;
         const double kv2 = 2.0 * m.n_layers * Dkv * m.kv_bytes;
         for (size_t q = 0; q < n_four; q++) {
-            const u32 t = s.tp[(4 * q) / n_l];
-            const double b_rep = std::ceil(b_ref / (double)s.dp[(4 * q) / n_l]);   // one replica's share
+            const u32 t = s.tp[(group * q) / n_l];
+            const double b_rep = std::ceil(b_ref / (double)s.dp[(group * q) / n_l]);   // one replica's share
             const bool bad = (m.n_heads % t) != 0 || (m.n_kv_heads % t) != 0;
             double best = INFINITY;
-            for (size_t u = 0; u < 4 && !bad; u++) {
-                const guide_len_pair &pr = s.pairs[(4 * q + u) % n_l];
+            for (size_t u = 0; u < group && !bad; u++) {
+                const guide_len_pair &pr = s.pairs[(group * q + u) % n_l];
                 const double S = std::ceil(((double)pr.lin + pr.lout) / blk) * blk;
                 best = std::min(best, wbytes / t + b_rep * S * (kv2 / t));
             }
@@ -228,6 +230,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
                  o_ch = take(n_h * n_f * s->tp.size() * 8), o_cs = take(n_h * n_f * s->tp.size() * 8),
                  o_hm = take(n_h * n_f * 16), o_hs = take(n_h * n_f * sizeof(HfSorted)),
                  o_po = take(std::max<size_t>(n_m * (s->tp.size() * s->pairs.size() / 4), 1) * 4),
+                 o_lo = take(std::max<size_t>(n_m * (s->tp.size() * s->pairs.size() / 16), 1) * 4),
                  o_tk = take(TICKET_SLOTS * 128), o_r10 = take(n_h * n_f * 80);
     char *blob = nullptr;
     GUIDE_CUDA(cudaMalloc(&blob, off));
@@ -243,9 +246,10 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
     put(o_d, s->dp.data(), s->dp.size() * 4);
     put(o_p, s->pairs.data(), s->pairs.size() * 8);
     const std::vector<HfSorted> hf_sorted = sorted_pairs(*s);
-    const std::vector<u32> plane_order = plane_orders(*s);
+    const std::vector<u32> plane_order = plane_orders(*s, 4), line_order = plane_orders(*s, 16);
     put(o_hs, hf_sorted.data(), hf_sorted.size() * sizeof(HfSorted));
     put(o_po, plane_order.data(), plane_order.size() * 4);
+    put(o_lo, line_order.data(), line_order.size() * 4);
     if (e == cudaSuccess) {
         const u32 n = (u32)std::max(n_m, n_h * n_f);
         k_build_tables<<<(n + 127) / 128, 128>>>((const guide_model *)(blob + o_gm), (u32)n_m,
@@ -275,6 +279,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
     d.view.rate10 = (const double *)(blob + o_r10);
     d.view.hf_sorted = (const HfSorted *)(blob + o_hs);
     d.view.plane_order = (const u32 *)(blob + o_po);
+    d.view.line_order = (const u32 *)(blob + o_lo);
     d.view.n_m = (u32)n_m; d.view.n_h = (u32)n_h; d.view.n_f = (u32)n_f;
     d.view.n_b = (u32)s->batch.size(); d.view.n_t = (u32)s->tp.size(); d.view.n_l = (u32)s->pairs.size();
     d.tickets = (unsigned *)(blob + o_tk);

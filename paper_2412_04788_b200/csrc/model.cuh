@@ -57,6 +57,7 @@ struct DSpace {
     // Orders that only steer which thread does what (any permutation gives the same results):
     const HfSorted *hf_sorted;   // [n_h * n_f]: the pairs grouped by KV block size, largest usable memory first
     const u32 *plane_order;      // [n_m][n_t * n_l / 4]: foursomes of the (TP, length) plane by growing memory need
+    const u32 *line_order;       // [n_m][n_t * n_l / 16]: the same for lines of sixteen positions
     u32 n_m, n_h, n_f, n_b, n_t, n_l;
     u32 chunked;                 // some framework splits prompt processing: only the flat evaluation handles that
 };

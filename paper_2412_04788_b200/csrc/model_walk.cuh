@@ -16,7 +16,11 @@ typedef double StageTab[24][4];
 enum { E_F1, E_B1, E_F2, E_B2, E_F3, E_B3, E_F5, E_B5, E_F6, E_B6, E_F7, E_B7, E_F8, E_B8, E_F9, E_B9, E_B9X, E_F10, E_B10X,
        E_F13, E_B13, E_HOPS, E_CBYTES, E_RD };
 
-__device__ __forceinline__ void put_stage(StageTab &tb, u32 u, const TaskTab &k) {
+// A line of the plane (sixteen points, 128 bytes of every metric array) keeps its tables the same way.
+typedef double LineTab[24][16];
+
+template <class Tab>
+__device__ __forceinline__ void put_stage(Tab &tb, u32 u, const TaskTab &k) {
     tb[E_F1][u] = k.F1; tb[E_B1][u] = k.B1; tb[E_F2][u] = k.F2; tb[E_B2][u] = k.B2; tb[E_F3][u] = k.F3; tb[E_B3][u] = k.B3;
     tb[E_F5][u] = k.F5; tb[E_B5][u] = k.B5; tb[E_F6][u] = k.F6; tb[E_B6][u] = k.B6; tb[E_F7][u] = k.F7; tb[E_B7][u] = k.B7;
     tb[E_F8][u] = k.F8; tb[E_B8][u] = k.B8; tb[E_F9][u] = k.F9; tb[E_B9][u] = k.B9; tb[E_B9X][u] = k.B9x; tb[E_F10][u] = k.F10;
@@ -28,7 +32,8 @@ __device__ __forceinline__ void put_stage(StageTab &tb, u32 u, const TaskTab &k)
 // aggregated decode steps.  Eight lanes of a warp call it together (four points x two stages): the
 // instruction stream is the same for both stages, only the token counts differ.  Kept out of line:
 // it runs once per work item and needs far more registers than the walk around it.
-static __device__ __noinline__ void build_stage_table(const DModel *mp, u32 tt, u32 b, u32 lin, u32 n, u32 stage, StageTab *tb, u32 u) {
+template <class Tab>
+static __device__ __noinline__ void build_stage_table(const DModel *mp, u32 tt, u32 b, u32 lin, u32 n, u32 stage, Tab *tb, u32 u) {
     const DModel m = *mp;
     TaskTab k;
     const u32 nn = n > 0 ? n : 1;          // a decode table is built either way; unused when n == 0
@@ -44,8 +49,8 @@ static __device__ __noinline__ void build_stage_table(const DModel *mp, u32 tt, 
 struct RateRegs { double icL, icA, icE, imL, imA, imE, inv_comm, clat, tovh, flash; };
 
 // eval_phase of model.cuh, operation for operation, with the task entries read from a StageTab
-template <int TIME_SUM>
-__device__ __forceinline__ double eval_stage(const StageTab &tb, u32 u, const RateRegs &r, double Nd, double log2_factor) {
+template <int TIME_SUM, class Tab>
+__device__ __forceinline__ double eval_stage(const Tab &tb, u32 u, const RateRegs &r, double Nd, double log2_factor) {
     const double t2 = task_time<TIME_SUM>(tb[E_F2][u], tb[E_B2][u], r.icL, r.imL);
     double sfix = task_time<TIME_SUM>(tb[E_F1][u], tb[E_B1][u], r.icE, r.imE);
     sfix = sfix + t2;
