@@ -39,9 +39,9 @@ import numpy as np
 
 BYTES_SIM = 6 * 8 + 1 + 4          # six fp64 metrics + status + bmax written per config
 # dram__bytes_read.sum + dram__bytes_write.sum of one guide_simulate call on the full workload 5: the
-# k_closed_form_memory and k_closed_form_model launches together (profiles/k_closed_form_split_c5.md);
+# k_closed_form_memory and k_closed_form_lines launches together (profiles/launch_list_bench_c5_step.md);
 # only meaningful for that size and those kernel versions
-K1_TRAFFIC_C5 = 644_500_000 + 150_700_000 + 100_000
+K1_TRAFFIC_C5 = 592_300_000 + 171_600_000 + 100_000
 SIM_FIELDS = ("latency", "ttft", "tpot", "thr_decode", "cost_per_hr", "cost_per_token", "status", "bmax")
 TRACE_FIELDS = ("latency", "ttft", "ttft_p50", "ttft_p99", "tpot", "thr_decode", "cost_per_hr", "cost_per_token",
                 "status", "bmax", "n_iters", "n_req_iters")
@@ -470,7 +470,7 @@ def run_ours(args):
     cons_arrays = {arr for name, arr in bounded.items() if name in cons}
     bytes_topk = 1 + 8 * len(cons_arrays | {key})
     bytes_pareto = 1 + 8 * len(cons_arrays | {"latency", "cost_per_hr"})
-    per = {"guide_simulate (k_closed_form_memory + k_closed_form_model)": (t_sim / args.steps, BYTES_SIM),
+    per = {"guide_simulate (k_closed_form_memory + k_closed_form_lines)": (t_sim / args.steps, BYTES_SIM),
            "guide_select_topk (k_topk_bound + k_topk_filter + k_topk_rank)": (t_topk / args.steps, bytes_topk),
            "guide_pareto (k_pareto_sample + k_pareto_filter + k_pareto_rank)": (t_par / args.steps, bytes_pareto)}
     dom = max(per, key=lambda name: per[name][0])

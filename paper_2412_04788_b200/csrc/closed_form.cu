@@ -197,6 +197,7 @@ k_closed_form_model(DSpace s, int tp_model, guide_outputs o, u32 n_chunks, unsig
 // leave it as whole lines: eight lanes x 16 bytes per (pair, array), for every pair with a config
 // that fits anywhere in the line.
 static constexpr u32 LINE_BLOCKS_PER_SM = 4;
+static constexpr u32 LINE_CHUNK = 64;           // sorted pairs per work item
 static constexpr u32 LINE_STAGE_ARRAYS = 6;     // latency, ttft, tpot, throughput, cost per hour, cost per token
 static constexpr u32 LINE_STAGE_ROW = 20;       // doubles per (array, pair) row: 16 + 4 of padding against bank conflicts
 static constexpr u32 LINE_WARP_DOUBLES = 2 * 24 * 16 + LINE_STAGE_ARRAYS * 8 * LINE_STAGE_ROW;
@@ -235,7 +236,7 @@ k_closed_form_lines(DSpace s, int tp_model, guide_outputs o, u32 n_chunks, unsig
         const u32 log2t = 31 - __clz(t);
         const u64 w_gpu = (mp->wbytes + (u64)(t - 1)) >> log2t;  // as mem_info
         const u64 kv_tok = mp->kv2 >> log2t;
-        const u32 p_lo = chunk_i * MODEL_CHUNK, p_hi = min(n_hf, p_lo + MODEL_CHUNK);
+        const u32 p_lo = chunk_i * LINE_CHUNK, p_hi = min(n_hf, p_lo + LINE_CHUNK);
         auto need_of = [&](u64 S, u32 block) {
             const u64 s_blk = block == 1 ? S : ((S + block - 1) / block) * block;
             const u64 bytes = s_blk * kv_tok;
@@ -401,6 +402,11 @@ static bool split_applies(const DSpace &s, Range r, const guide_outputs &o, Cons
 // 8-byte array start on a 128-byte boundary.
 static bool lines_apply(const DSpace &s, const guide_outputs &o) {
     if (s.n_l % 16 != 0) return false;
+    // a line is four times the work of a foursome: with fewer than two work items per resident warp
+    // the foursome kernel's finer grain fills the machine better
+    const u64 n_hf = (u64)s.n_h * s.n_f;
+    const u64 items = (u64)s.n_m * s.n_b * (s.n_t * s.n_l / 16) * ((n_hf + LINE_CHUNK - 1) / LINE_CHUNK);
+    if (items < 2ull * (u64)num_sms() * LINE_BLOCKS_PER_SM * (MODEL_THREADS / 32)) return false;
     const void *wide[] = {o.latency, o.ttft, o.ttft_p50, o.ttft_p99, o.tpot, o.thr_decode, o.cost_per_hr, o.cost_per_token,
                           o.n_iters, o.n_req_iters};
     for (const void *p : wide)
@@ -420,7 +426,7 @@ static int launch_split(const DSpace &s, int tp_model, const guide_outputs &o, c
     if (lines) k_closed_form_memory<1><<<mem_grid, MEM_THREADS, 0, st>>>(s, o, co, tiles);
     else k_closed_form_memory<0><<<mem_grid, MEM_THREADS, 0, st>>>(s, o, co, tiles);
     GUIDE_CUDA(cudaGetLastError());
-    const u32 n_chunks = (n_hf + MODEL_CHUNK - 1) / MODEL_CHUNK;
+    const u32 n_chunks = lines ? (n_hf + LINE_CHUNK - 1) / LINE_CHUNK : (n_hf + MODEL_CHUNK - 1) / MODEL_CHUNK;
     if ((u64)s.n_m * s.n_b * (n_tl / 4) * n_chunks > 0x7FFFFFFFull) return fail(GUIDE_ERR_UNSUPPORTED, "space too large for one launch");
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(MODEL_THREADS); cfg.stream = st;
