@@ -70,6 +70,9 @@ __global__ void __launch_bounds__(256, 2) k_closed_form_tiled(DSpace s, Range r,
 // The model kernel is launched as a programmatic dependent of the memory kernel and waits for it
 // only at its very end: the two run side by side, one bound by bandwidth and one by arithmetic,
 // and write disjoint sectors.
+//
+// On large spaces whose length axis divides into sixteens the unit becomes the line (sixteen
+// positions, 128 bytes) and k_closed_form_lines takes the model kernel's place: see below.
 
 static constexpr u32 MEM_THREADS = 128;         // x 2 positions = 256 positions of the plane per work item
 static constexpr u32 MEM_BLOCKS_PER_SM = 2;

@@ -100,6 +100,52 @@ def test_split_kernels_mixed_block_sizes_and_ragged_plane():
     assert (want["status"] == 0).any() and (want["status"] != 0).any()
 
 
+def test_line_kernels_mixed_block_sizes_and_output_subsets():
+    """4,915,200 configs, enough lines per resident warp for the pair of kernels that shares out
+    128-byte lines: three KV block sizes (three segments in the sorted pair walk, four chunks of
+    pairs), a TP degree that does not divide every model's heads, memories small enough that most
+    lines are mixed; then calls with only some output arrays."""
+    import torch
+    hw, mem = I.seeded_hw(21, 80, mem_choices=[16, 24, 48, 80, 192])
+    fw_f, fw_i = I.seeded_fw(22, 3, kv_block=16)
+    fw_i[0, 1] = 1
+    fw_i[2, 1] = 24
+    sp_np = I._space(I.models_from_shapes(I.SHAPES_8), hw, mem, fw_f, fw_i,
+                     [1, 2, 3, 5, 8, 13, 17, 32, 50, 64, 100, 128, 200, 256, 400, 512], [1, 2, 4, 8, 16],
+                     I.pairs_grid([64, 700, 3000, 8000], [1, 2, 64, 130, 500, 1000, 2000, 4000]))
+    assert len(sp_np["pairs"]) % 16 == 0
+    for tm, tpm in ((0, 0), (1, 1)):
+        want = oracle.simulate(sp_np, time_model=tm, tp_model=tpm)
+        assert len(want["status"]) == 4915200
+        got, *_ = run_simulate(sp_np, time_model=tm, tp_model=tpm)
+        assert_parity(got, want)
+        assert sum(bit_mismatches(got, want).values()) == 0
+    ok = want["status"] == 0
+    assert 0.05 < ok.mean() < 0.95 and (want["status"] & guide.ST_HEADS).any()
+    lines = ok.reshape(-1, 16)
+    assert (lines.any(axis=1) & ~lines.all(axis=1)).mean() > 0.05          # mixed lines: constants next to metrics
+    want = oracle.simulate(sp_np)
+    sp = guide.Space(sp_np)
+    n = sp.size
+    for fields in (("latency",), ("status", "bmax"), ("thr_decode", "cost_per_token", "n_iters"),
+                   ("ttft_p50", "ttft_p99", "status", "n_req_iters"), ("cost_per_hr", "tpot")):
+        out = guide.alloc_outputs(n, fields=fields)
+        for t in out.values():
+            t.fill_(7)
+        guide.guide_simulate(sp, None, out)
+        torch.cuda.synchronize()
+        for f in fields:
+            g = out[f].cpu().numpy()
+            x = want["ttft"] if f in ("ttft_p50", "ttft_p99") else want[f]
+            assert np.array_equal(g.view(np.uint8), x.view(np.uint8)), (fields, f)
+    # arrays that do not start on a 128-byte boundary go through the kernels that share out sectors
+    base = torch.empty(n + 4, dtype=torch.float64, device="cuda")
+    out = {"latency": base[4:], "status": torch.empty(n, dtype=torch.uint8, device="cuda")}
+    guide.guide_simulate(sp, None, out)
+    torch.cuda.synchronize()
+    assert np.array_equal(out["latency"].cpu().numpy().view(np.uint64), want["latency"].view(np.uint64))
+
+
 def test_split_kernels_output_subsets():
     """Whole-space calls with only some output arrays: each kernel of the pair must skip the rest."""
     import torch
