@@ -4,6 +4,7 @@
 
 #include "guide_internal.cuh"
 #include "model_walk.cuh"
+#include "line_walk.cuh"
 
 namespace guide {
 
@@ -200,10 +201,9 @@ k_closed_form_model(DSpace s, int tp_model, guide_outputs o, u32 n_chunks, unsig
 // leave it as whole lines: eight lanes x 16 bytes per (pair, array), for every pair with a config
 // that fits anywhere in the line.
 static constexpr u32 LINE_BLOCKS_PER_SM = 4;
-static constexpr u32 LINE_CHUNK = 64;           // sorted pairs per work item
 static constexpr u32 LINE_STAGE_ARRAYS = 6;     // latency, ttft, tpot, throughput, cost per hour, cost per token
 static constexpr u32 LINE_STAGE_ROW = 20;       // doubles per (array, pair) row: 16 + 4 of padding against bank conflicts
-static constexpr u32 LINE_WARP_DOUBLES = 2 * 24 * 16 + LINE_STAGE_ARRAYS * 8 * LINE_STAGE_ROW;
+static constexpr u32 LINE_WARP_DOUBLES = LINE_TABLE_DOUBLES + LINE_STAGE_ARRAYS * 8 * LINE_STAGE_ROW;
 static constexpr u32 LINE_SMEM_BYTES = (MODEL_THREADS / 32) * LINE_WARP_DOUBLES * 8;
 
 template <int TIME_SUM>
@@ -215,165 +215,63 @@ k_closed_form_lines(DSpace s, int tp_model, guide_outputs o, u32 n_chunks, unsig
     double *mine = line_smem + (size_t)warp * LINE_WARP_DOUBLES;
     LineTab &tb_pre = *reinterpret_cast<LineTab *>(mine);
     LineTab &tb_dec = *reinterpret_cast<LineTab *>(mine + 24 * 16);
-    double *stage = mine + 2 * 24 * 16;                           // [array][pair of the group][LINE_STAGE_ROW]
-    const u32 n_tl = s.n_t * s.n_l, n_hf = s.n_h * s.n_f, n_lines = n_tl >> 4;
-    const u32 n_mb = s.n_m * s.n_b;
-    const u32 n_items = n_mb * n_lines * n_chunks;
-    const double inf = __longlong_as_double(0x7FF0000000000000LL);
-    const u64 stride_hf = (u64)s.n_b * n_tl;
+    double *stage = mine + LINE_TABLE_DOUBLES;                    // [array][pair of the group][LINE_STAGE_ROW]
+    const u64 stride_hf = (u64)s.n_b * s.n_t * s.n_l;
     double *const arr[LINE_STAGE_ARRAYS] = {o.latency, o.ttft, o.tpot, o.thr_decode, o.cost_per_hr, o.cost_per_token};
-    for (;;) {
-        u32 item = 0;
-        if (lane == 0) item = atomicAdd(ticket, 1u);
-        item = __shfl_sync(0xFFFFFFFFu, item, 0);
-        if (item >= n_items) break;
-        const u32 mb = item % n_mb, rest = item / n_mb;
-        const u32 rank = rest % n_lines, chunk_i = rest / n_lines;
-        const u32 bpos = mb % s.n_b, mpos = mb / s.n_b;
-        const u32 tl0 = __ldg(s.line_order + (size_t)mpos * n_lines + rank) * 16;
-        const u32 tpos = tl0 / s.n_l, lpos0 = tl0 % s.n_l;        // sixteen divides the length axis: one TP degree per line
-        const DModel *mp = s.models + mpos;
-        const u32 t = s.tp[tpos], b_all = s.batch[bpos];
-        const u32 b = replica_batch(b_all, s.dp[tpos]);
-        if ((mp->nh & (t - 1)) != 0 || (mp->nkv & (t - 1)) != 0) continue;      // nothing of the line fits
-        const u32 log2t = 31 - __clz(t);
-        const u64 w_gpu = (mp->wbytes + (u64)(t - 1)) >> log2t;  // as mem_info
-        const u64 kv_tok = mp->kv2 >> log2t;
-        const u32 p_lo = chunk_i * LINE_CHUNK, p_hi = min(n_hf, p_lo + LINE_CHUNK);
-        auto need_of = [&](u64 S, u32 block) {
-            const u64 s_blk = block == 1 ? S : ((S + block - 1) / block) * block;
-            const u64 bytes = s_blk * kv_tok;
-            return __umul64hi((u64)b, bytes) ? ~0ull : (u64)b * bytes;
-        };
-        // Does anything fit?  Per KV block size the first pair of the chunk has the most memory.
-        const uint2 pr16 = s.pairs[lpos0 + (lane & 15)];          // the point this lane builds a table for
-        {
-            bool any = false;
-            const u64 S = (u64)pr16.x + pr16.y;
-            for (u32 p0 = p_lo; p0 < p_hi;) {
-                const HfSorted e0 = s.hf_sorted[p0];
-                any |= e0.usable > w_gpu && e0.usable - w_gpu >= need_of(S, e0.block);
-                p0 = e0.seg_end;
-            }
-            if (!__any_sync(0xFFFFFFFFu, any)) continue;
+    line_walk<TIME_SUM>(s, tp_model, n_chunks, ticket, tb_pre, tb_dec,
+        [&](int q, bool, bool pair_live, u64, double latency, double ttft, double tpot, double thr, double cost_hr, double cost_tok) {
+        if (pair_live) {
+            double *w = stage + (size_t)h * LINE_STAGE_ROW + u + 4 * q;
+            w[0 * 8 * LINE_STAGE_ROW] = latency; w[1 * 8 * LINE_STAGE_ROW] = ttft; w[2 * 8 * LINE_STAGE_ROW] = tpot;
+            w[3 * 8 * LINE_STAGE_ROW] = thr; w[4 * 8 * LINE_STAGE_ROW] = cost_hr; w[5 * 8 * LINE_STAGE_ROW] = cost_tok;
+
         }
-        __syncwarp();                                 // the previous item's reads of the tables are over
-        build_stage_table(mp, tp_model ? 1u : t, b, pr16.x, pr16.y - 1, lane >> 4, (lane >> 4) ? &tb_dec : &tb_pre, lane & 15);
+        },
+        [&](u32 live, u32 fit4, u32 hf, u64 j_line, u32 b_all, u32 lpos0) {
         __syncwarp();
-        // the four points this lane evaluates: 4q + u
-        u64 S4[4];
-        u32 n4[4];
+        // whole lines out: eight lanes x 16 bytes per (pair, array), four pairs per store instruction
 #pragma unroll
-        for (int q = 0; q < 4; q++) {
-            const uint2 pr = s.pairs[lpos0 + 4 * q + u];
-            S4[q] = (u64)pr.x + pr.y; n4[q] = pr.y - 1;
-        }
-        const u64 j_line = (u64)mpos * n_hf * stride_hf + (u64)bpos * n_tl + tl0;
-        const double lf = log2_rule_factor(t, tp_model);
-        const double Nd = (double)mp->N;
-        u32 p0 = p_lo;
-        while (p0 < p_hi) {
-            // one KV block size at a time: within it the pairs are sorted by falling usable memory
-            const HfSorted e0 = s.hf_sorted[p0];
-            const u32 seg_end = min(e0.seg_end, p_hi);
-            u64 need4[4];
+        for (int half = 0; half < 2; half++) {
+            const u32 hh = 4 * half + (lane >> 3), piece = lane & 7;
+            const u32 src = 4 * hh;                                  // the lane with point 0 of pair hh
+            const u32 hf_hh = __shfl_sync(0xFFFFFFFFu, hf, src);
+            const u32 fits_hh = (__shfl_sync(0xFFFFFFFFu, fit4, src) & 0xFu) | ((__shfl_sync(0xFFFFFFFFu, fit4, src + 1) & 0xFu) << 4) |
+                                ((__shfl_sync(0xFFFFFFFFu, fit4, src + 2) & 0xFu) << 8) | ((__shfl_sync(0xFFFFFFFFu, fit4, src + 3) & 0xFu) << 12);
+            // fits_hh: bit 4 * u' + q' = point 4 q' + u' of pair hh fits
+            if ((live >> src) & 0xFu) {
+                const u64 j = j_line + (u64)hf_hh * stride_hf + 2 * piece;
+                const double *rd = stage + (size_t)hh * LINE_STAGE_ROW + 2 * piece;
 #pragma unroll
-            for (int q = 0; q < 4; q++) need4[q] = need_of(S4[q], e0.block);
-            for (u32 pp = p0; pp < seg_end; pp += 8) {
-                const u32 p = pp + h;
-                const bool in = p < seg_end;
-                const HfSorted e = s.hf_sorted[in ? p : seg_end - 1];
-                const bool room = in && e.usable > w_gpu;
-                const u64 avail = room ? e.usable - w_gpu : 0;
-                u32 fit4 = 0;
-#pragma unroll
-                for (int q = 0; q < 4; q++) fit4 |= (room && avail >= need4[q]) ? 1u << q : 0u;
-                const u32 live = __ballot_sync(0xFFFFFFFFu, fit4 != 0);      // lanes with a config that fits
-                if (live == 0) break;                 // nor does any later pair of this block size
-                const bool pair_live = ((live >> (lane & ~3u)) & 0xFu) != 0;   // this lane's pair has one in the line
-                RateRegs r;
-                double c_hr = inf, c_sec = 0.0;
-                if (fit4) {
-                    const double2 *q = reinterpret_cast<const double2 *>(s.rate10 + (size_t)e.hf * 10);
-                    const double2 q0 = __ldg(q), q1 = __ldg(q + 1), q2 = __ldg(q + 2), q3 = __ldg(q + 3), q4 = __ldg(q + 4);
-                    r.icL = q0.x; r.icA = q0.y; r.icE = q1.x; r.imL = q1.y; r.imA = q2.x; r.imE = q2.y;
-                    r.inv_comm = q3.x; r.clat = q3.y; r.tovh = q4.x; r.flash = q4.y;
-                    const u32 ci = e.hf * s.n_t + tpos;
-                    c_hr = __ldg(s.cost_hr + ci);
-                    c_sec = __ldg(s.cost_sec + ci);
-                }
-                double *row = stage + (size_t)h * LINE_STAGE_ROW + u;
-#pragma unroll
-                for (int q = 0; q < 4; q++) {
-                    double latency = inf, ttft = inf, tpot = inf, thr = 0.0, cost_hr = inf, cost_tok = inf;
-                    if (fit4 & (1u << q)) {
-                        const u32 n = n4[q];
-                        const double t_pre = eval_stage<TIME_SUM>(tb_pre, 4 * q + u, r, Nd, lf);
-                        const double t_dec = n > 0 ? eval_stage<TIME_SUM>(tb_dec, 4 * q + u, r, Nd, lf) : 0.0;
-                        ttft = t_pre;
-                        latency = t_pre + t_dec;
-                        cost_hr = c_hr;
-                        if (n > 0) {
-                            tpot = t_dec / (double)n;
-                            thr = cvt((u64)b_all * n) / t_dec;
-                            cost_tok = c_sec / thr;
-                        } else {
-                            tpot = 0.0; thr = 0.0; cost_tok = inf;
-                        }
-                    }
-                    if (pair_live) {
-                        double *w = row + 4 * q;
-                        w[0 * 8 * LINE_STAGE_ROW] = latency; w[1 * 8 * LINE_STAGE_ROW] = ttft; w[2 * 8 * LINE_STAGE_ROW] = tpot;
-                        w[3 * 8 * LINE_STAGE_ROW] = thr; w[4 * 8 * LINE_STAGE_ROW] = cost_hr; w[5 * 8 * LINE_STAGE_ROW] = cost_tok;
+                for (u32 a = 0; a < LINE_STAGE_ARRAYS; a++) {
+                    if (arr[a]) {
+                        const double2 v = *reinterpret_cast<const double2 *>(rd + (size_t)a * 8 * LINE_STAGE_ROW);
+                        __stcs(reinterpret_cast<double2 *>(arr[a] + j), v);
                     }
                 }
-                __syncwarp();
-                // whole lines out: eight lanes x 16 bytes per (pair, array), four pairs per store instruction
-#pragma unroll
-                for (int half = 0; half < 2; half++) {
-                    const u32 hh = 4 * half + (lane >> 3), piece = lane & 7;
-                    const u32 src = 4 * hh;                                  // the lane with point 0 of pair hh
-                    const u32 hf_hh = __shfl_sync(0xFFFFFFFFu, e.hf, src);
-                    const u32 fits_hh = (__shfl_sync(0xFFFFFFFFu, fit4, src) & 0xFu) | ((__shfl_sync(0xFFFFFFFFu, fit4, src + 1) & 0xFu) << 4) |
-                                        ((__shfl_sync(0xFFFFFFFFu, fit4, src + 2) & 0xFu) << 8) | ((__shfl_sync(0xFFFFFFFFu, fit4, src + 3) & 0xFu) << 12);
-                    // fits_hh: bit 4 * u' + q' = point 4 q' + u' of pair hh fits
-                    if ((live >> src) & 0xFu) {
-                        const u64 j = j_line + (u64)hf_hh * stride_hf + 2 * piece;
-                        const double *rd = stage + (size_t)hh * LINE_STAGE_ROW + 2 * piece;
-#pragma unroll
-                        for (u32 a = 0; a < LINE_STAGE_ARRAYS; a++) {
-                            if (arr[a]) {
-                                const double2 v = *reinterpret_cast<const double2 *>(rd + (size_t)a * 8 * LINE_STAGE_ROW);
-                                __stcs(reinterpret_cast<double2 *>(arr[a] + j), v);
-                            }
-                        }
-                        if (o.ttft_p50 || o.ttft_p99) {
-                            const double2 v = *reinterpret_cast<const double2 *>(rd + (size_t)1 * 8 * LINE_STAGE_ROW);
-                            if (o.ttft_p50) __stcs(reinterpret_cast<double2 *>(o.ttft_p50 + j), v);
-                            if (o.ttft_p99) __stcs(reinterpret_cast<double2 *>(o.ttft_p99 + j), v);
-                        }
-                        if (o.n_iters || o.n_req_iters) {
-                            // iteration counts of the two points this lane writes: 1 + n and b (1 + n), 0 when the config does not fit
-                            ulonglong2 it, rq;
-                            u64 *itp = &it.x, *rqp = &rq.x;
-#pragma unroll
-                            for (u32 k = 0; k < 2; k++) {
-                                const u32 pt = 2 * piece + k;                 // point 4 q' + u'
-                                const bool f = (fits_hh >> (4 * (pt & 3) + (pt >> 2))) & 1u;
-                                const u64 n1 = 1 + (u64)(s.pairs[lpos0 + pt].y - 1);
-                                itp[k] = f ? n1 : 0;
-                                rqp[k] = f ? (u64)b_all * n1 : 0;
-                            }
-                            if (o.n_iters) __stcs(reinterpret_cast<ulonglong2 *>(o.n_iters + j), it);
-                            if (o.n_req_iters) __stcs(reinterpret_cast<ulonglong2 *>(o.n_req_iters + j), rq);
-                        }
-                    }
+                if (o.ttft_p50 || o.ttft_p99) {
+                    const double2 v = *reinterpret_cast<const double2 *>(rd + (size_t)1 * 8 * LINE_STAGE_ROW);
+                    if (o.ttft_p50) __stcs(reinterpret_cast<double2 *>(o.ttft_p50 + j), v);
+                    if (o.ttft_p99) __stcs(reinterpret_cast<double2 *>(o.ttft_p99 + j), v);
                 }
-                __syncwarp();                         // the staging area is free for the next eight pairs
+                if (o.n_iters || o.n_req_iters) {
+                    // iteration counts of the two points this lane writes: 1 + n and b (1 + n), 0 when the config does not fit
+                    ulonglong2 it, rq;
+                    u64 *itp = &it.x, *rqp = &rq.x;
+#pragma unroll
+                    for (u32 k = 0; k < 2; k++) {
+                        const u32 pt = 2 * piece + k;                 // point 4 q' + u'
+                        const bool f = (fits_hh >> (4 * (pt & 3) + (pt >> 2))) & 1u;
+                        const u64 n1 = 1 + (u64)(s.pairs[lpos0 + pt].y - 1);
+                        itp[k] = f ? n1 : 0;
+                        rqp[k] = f ? (u64)b_all * n1 : 0;
+                    }
+                    if (o.n_iters) __stcs(reinterpret_cast<ulonglong2 *>(o.n_iters + j), it);
+                    if (o.n_req_iters) __stcs(reinterpret_cast<ulonglong2 *>(o.n_req_iters + j), rq);
+                }
             }
-            p0 = e0.seg_end;
         }
-    }
+        __syncwarp();                         // the staging area is free for the next eight pairs
+        });
     // the grid must not be complete before the memory kernel is: whatever follows in the stream
     // waits for this one only
     cf_dep_wait();
@@ -438,8 +336,12 @@ static int launch_split(const DSpace &s, int tp_model, const guide_outputs &o, c
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
     if (lines) {
-        static bool opted_in[2] = {false, false};             // more dynamic shared memory than the default limit
-        if (!opted_in[TIME_SUM]) {
+        // function attributes belong to the device: set them once per device and kernel variant
+        static bool opted_in[64][2] = {};
+        int dev = 0;
+        GUIDE_CUDA(cudaGetDevice(&dev));
+        if (dev < 0 || dev >= 64 || !opted_in[dev][TIME_SUM]) {
+            // more dynamic shared memory than the default limit
             GUIDE_CUDA(cudaFuncSetAttribute(k_closed_form_lines<TIME_SUM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             (int)LINE_SMEM_BYTES));
             // An SM changes its split between L1 and shared memory only when it is empty.  The memory
@@ -449,7 +351,7 @@ static int launch_split(const DSpace &s, int tp_model, const guide_outputs &o, c
                                             (int)cudaSharedmemCarveoutMaxShared));
             GUIDE_CUDA(cudaFuncSetAttribute(k_closed_form_lines<TIME_SUM>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                             (int)cudaSharedmemCarveoutMaxShared));
-            opted_in[TIME_SUM] = true;
+            if (dev >= 0 && dev < 64) opted_in[dev][TIME_SUM] = true;
         }
         cfg.gridDim = dim3((u32)num_sms() * LINE_BLOCKS_PER_SM); cfg.dynamicSmemBytes = LINE_SMEM_BYTES;
         GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_closed_form_lines<TIME_SUM>, s, tp_model, o, n_chunks, ticket));
