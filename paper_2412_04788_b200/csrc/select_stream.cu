@@ -471,7 +471,10 @@ __global__ void __launch_bounds__(SEL_THREADS, 4) k_topk_filter(Src<NA> s, Range
     const u64 *bp = reinterpret_cast<const u64 *>(header + TK_BOUND);
     const u64 bkey = __ldcg(bp), bidx = __ldcg(bp + 1);
     const u64 tiles = r.count / TILE;
-    for (u64 tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    // from the end of the range backwards: when the metrics were written just before this call the
+    // end of the arrays is what the L2 still holds
+    for (u64 back = blockIdx.x; back < tiles; back += gridDim.x) {
+        const u64 tile = tiles - 1 - back;
         const u64 j0 = tile * TILE + 2 * threadIdx.x, j1 = j0 + TILE / 2;
         u32 st0, st1;
         double2 v0[NA], v1[NA];
@@ -763,7 +766,10 @@ __global__ void __launch_bounds__(SEL_THREADS, 4) k_pareto_filter(Src<NA> s, Ran
         else { K.rx[i] = KEY_MAX; K.ry[i] = KEY_MAX; }
     }
     const u64 tiles = r.count / TILE;
-    for (u64 tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    // from the end of the range backwards: when the metrics were written just before this call the
+    // end of the arrays is what the L2 still holds
+    for (u64 back = blockIdx.x; back < tiles; back += gridDim.x) {
+        const u64 tile = tiles - 1 - back;
         const u64 j0 = tile * TILE + 2 * threadIdx.x, j1 = j0 + TILE / 2;
         u32 st0, st1;
         double2 v0[NA], v1[NA];
