@@ -375,7 +375,6 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_bound(Src<NA> s, Sample sm
     namespace cg = cooperative_groups;
     cg::grid_group grid = cg::this_grid();
     __shared__ ulonglong2 sl[SEL_THREADS / 32];
-    grid_dep_launch();
     // the call's header is reset here rather than by a memset in front: nothing reads it before the
     // first grid barrier, and the kernels queued behind wait for this grid to complete
     if (blockIdx.x == 0 && threadIdx.x < 64) header[threadIdx.x] = 0;
@@ -442,6 +441,7 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_bound(Src<NA> s, Sample sm
         }
     }
     grid.sync();
+    grid_dep_launch();              // late: a dependent that starts early only sits on registers other streams could use
     // 4: their k-th smallest (of the stored ones, if they did not all fit: still a valid bound);
     // fewer than k only when the coarse bound is all-ones, which then stays
     const u32 n = min(__ldcg(header + TK_SAMPLED), TK_SKEYS_CAP);
@@ -466,7 +466,6 @@ __device__ __forceinline__ void topk_keep(u64 key, u64 idx, u32 *header, KI *can
 // Filter pass: passing configs within the bound go to the candidate list.
 template <int NA>
 __global__ void __launch_bounds__(SEL_THREADS, 4) k_topk_filter(Src<NA> s, Range r, u32 *header, KI *cand) {
-    grid_dep_launch();
     grid_dep_wait();
     const u64 *bp = reinterpret_cast<const u64 *>(header + TK_BOUND);
     const u64 bkey = __ldcg(bp), bidx = __ldcg(bp + 1);
@@ -495,6 +494,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 4) k_topk_filter(Src<NA> s, Range
             if (ok[u] && pair_le(key[u], idx, bkey, bidx)) topk_keep(key[u], idx, header, cand);
         }
     }
+    grid_dep_launch();              // late: the rank kernel needs this block's registers only now
     if (blockIdx.x == gridDim.x - 1) {                      // ragged tail, scalar loads
         for (u64 j = tiles * TILE + threadIdx.x; j < r.count; j += blockDim.x) {
             u64 k0, k1;
@@ -593,7 +593,6 @@ __global__ void __launch_bounds__(SEL_THREADS) k_pareto_sample(Src<NA> s, Sample
     static_assert(PA_ROWS_PER_WARP % SAMPLE_BATCH == 0, "whole batches");
     const u32 lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = SEL_THREADS / 32;
     if (threadIdx.x == 0) { n_list = 0; n_front = 0; }
-    grid_dep_launch();
     u64 px[N_PTS], py[N_PTS];
     const u64 stride = (u64)gridDim.x * n_warps;
 #pragma unroll
@@ -661,6 +660,7 @@ __global__ void __launch_bounds__(SEL_THREADS) k_pareto_sample(Src<NA> s, Sample
             if (pos < 32) front[pos] = me;
         }
     }
+    grid_dep_launch();              // late, as in k_topk_bound
     __syncthreads();
     const u32 nf = min(n_front, 32u);
     // hand on up to PA_PER_BLOCK of them, evenly spaced by rank in x
@@ -750,7 +750,6 @@ __device__ __forceinline__ void pareto_keep(u64 x, u64 y, u64 idx, u32 *header, 
 template <int NA>
 __global__ void __launch_bounds__(SEL_THREADS, 4) k_pareto_filter(Src<NA> s, Range r, u32 *header, const P2 *killers, P3 *surv) {
     __shared__ P2 ks[PA_KILLERS];
-    grid_dep_launch();
     grid_dep_wait();
     KillerSet K;
     K.k = ks;
@@ -787,6 +786,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 4) k_pareto_filter(Src<NA> s, Ran
         for (int u = 0; u < 4; u++)
             if (ok[u] && !K.kills(x[u], y[u])) pareto_keep(x[u], y[u], r.first + (u < 2 ? j0 : j1) + (u & 1), header, surv);
     }
+    grid_dep_launch();              // late: the rank kernel needs this block's registers only now
     if (blockIdx.x == gridDim.x - 1) {                      // ragged tail, scalar loads
         for (u64 j = tiles * TILE + threadIdx.x; j < r.count; j += blockDim.x) {
             u64 x, y;
