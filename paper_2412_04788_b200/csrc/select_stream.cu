@@ -121,6 +121,27 @@ __device__ __forceinline__ bool within(const Arr &a, double v) {
     return a.cmp == 0 || (a.cmp == 1 ? v <= a.bound : v >= a.bound);
 }
 
+// The two pairs of a thread in a filter tile (a warp: 64 consecutive configs at j0, 64 at j1).  The
+// status bytes come first; the metric values of a 64-config group are loaded only when some config of
+// the group passed its memory check, which most groups of a large sweep do not: whole runs of the
+// length axis do not fit, and their 512 bytes per array are never read.  Returns false when both
+// groups are dead.
+template <int NA>
+__device__ __forceinline__ bool load_live_pairs(const Src<NA> &s, u64 j0, u64 j1, u32 &st0, u32 &st1, double2 (&v0)[NA],
+                                                double2 (&v1)[NA]) {
+    st0 = __ldcs(reinterpret_cast<const unsigned short *>(s.status + j0));
+    st1 = __ldcs(reinterpret_cast<const unsigned short *>(s.status + j1));
+    const bool g0 = __any_sync(0xFFFFFFFFu, (st0 & 0xFFu) == 0 || (st0 >> 8) == 0);
+    const bool g1 = __any_sync(0xFFFFFFFFu, (st1 & 0xFFu) == 0 || (st1 >> 8) == 0);
+    if (!g0 && !g1) return false;
+#pragma unroll
+    for (int a = 0; a < NA; a++) {
+        v0[a] = g0 ? __ldcs(reinterpret_cast<const double2 *>(s.a[a].p + j0)) : make_double2(0.0, 0.0);
+        v1[a] = g1 ? __ldcs(reinterpret_cast<const double2 *>(s.a[a].p + j1)) : make_double2(0.0, 0.0);
+    }
+    return true;
+}
+
 template <int NA>
 __device__ __forceinline__ void eval_pair(const Src<NA> &s, u32 st, const double2 (&v)[NA], bool &ok0, bool &ok1) {
     ok0 = (st & 0xFFu) == 0;
@@ -477,8 +498,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 4) k_topk_filter(Src<NA> s, Range
         const u64 j0 = tile * TILE + 2 * threadIdx.x, j1 = j0 + TILE / 2;
         u32 st0, st1;
         double2 v0[NA], v1[NA];
-        load_pair(s, j0, st0, v0);
-        load_pair(s, j1, st1, v1);
+        if (!load_live_pairs(s, j0, j1, st0, st1, v0, v1)) continue;
         bool ok[4];
         eval_pair(s, st0, v0, ok[0], ok[1]);
         eval_pair(s, st1, v1, ok[2], ok[3]);
@@ -772,8 +792,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 4) k_pareto_filter(Src<NA> s, Ran
         const u64 j0 = tile * TILE + 2 * threadIdx.x, j1 = j0 + TILE / 2;
         u32 st0, st1;
         double2 v0[NA], v1[NA];
-        load_pair(s, j0, st0, v0);
-        load_pair(s, j1, st1, v1);
+        if (!load_live_pairs(s, j0, j1, st0, st1, v0, v1)) continue;
         bool ok[4];
         eval_pair(s, st0, v0, ok[0], ok[1]);
         eval_pair(s, st1, v1, ok[2], ok[3]);
