@@ -41,7 +41,7 @@ BYTES_SIM = 6 * 8 + 1 + 4          # six fp64 metrics + status + bmax written pe
 # dram__bytes_read.sum + dram__bytes_write.sum of one guide_simulate call on the full workload 5: the
 # k_closed_form_memory and k_closed_form_lines launches together (profiles/launch_list_bench_c5_step.md);
 # only meaningful for that size and those kernel versions
-K1_TRAFFIC_C5 = 592_300_000 + 171_600_000 + 100_000
+K1_TRAFFIC_C5 = 591_900_000 + 171_500_000 + 100_000
 SIM_FIELDS = ("latency", "ttft", "tpot", "thr_decode", "cost_per_hr", "cost_per_token", "status", "bmax")
 TRACE_FIELDS = ("latency", "ttft", "ttft_p50", "ttft_p99", "tpot", "thr_decode", "cost_per_hr", "cost_per_token",
                 "status", "bmax", "n_iters", "n_req_iters")
