@@ -249,6 +249,61 @@ def test_closed_form_aggregates_match_token_loops(golden):
             assert out["tpot"][0] == 0.0 and out["thr_decode"][0] == 0.0 and np.isinf(out["cost_per_token"][0])
 
 
+def _cost_space(golden, batch, tp, dp=None, pairs=((4, 3),)):
+    """The toy decoder with 8 heads (every degree up to 8 divides them) at the price of the cost pins."""
+    c = golden["costs"]
+    model = list(golden["model"])
+    model[2], model[3] = c["heads"], c["heads"]
+    hw = list(golden["hw"])
+    hw[4] = c["price_per_gpu_hr"]
+    return model, hw, I._space(np.array([model]), np.array([hw]), np.array([10**6]), np.array([[1.0] * 7 + [0.0]]),
+                               np.array([[1, 1, 0, 0]]), list(batch), list(tp), [list(p) for p in pairs],
+                               dp=None if dp is None else list(dp))
+
+
+def test_closed_form_cost_is_price_times_all_gpus(golden):
+    """Sec. 4.1 (selection under a budget) with Sec. 3.5.2: a deployment pays for t GPUs per replica
+    and dp replicas, so cost per hour = price x t x dp; cost per token = (cost per hour / 3600) /
+    decode throughput.  Values worked by hand in tests/golden (price 3 $/h per GPU)."""
+    rows = golden["costs"]["closed_form"]
+    model, hw, sp = _cost_space(golden, [6], [r["t"] for r in rows], dp=[r["dp"] for r in rows])
+    out = oracle.simulate(sp)
+    assert out["status"].tolist() == [0] * len(rows)
+    assert out["cost_per_hr"].tolist() == [r["cost_per_hr"] for r in rows]
+    ff, fi = [1.0] * 7 + [0.0], [1, 1, 0, 0]
+    for i, r in enumerate(rows):
+        b = -(-6 // r["dp"])                                       # the replica's share of the batch of 6
+        ctx = b * (2 * 4 + 3)                                      # two decode steps attending 5 and 6 tokens
+        t_dec = oracle.phase_time(model, hw, ff, fi, r["t"], 2 * b, 2 * b, ctx, ctx, 2)[0]
+        assert out["thr_decode"][i] == (6 * 2) / t_dec             # all replicas' tokens over one replica's time
+        assert out["cost_per_token"][i] == (r["cost_per_hr"] / 3600.0) / out["thr_decode"][i]
+    # twice the GPUs at the same throughput would cost twice as much per token: the factor is not folded away
+    assert out["cost_per_hr"][2] == 4.0 * out["cost_per_hr"][0]
+
+
+def test_trace_cost_is_price_times_tp_degree(golden):
+    """The trace simulation models one replica of t GPUs: cost per hour = price x t (Sec. 4.1), cost
+    per token = (cost per hour / 3600) / decode throughput, the throughput being decode tokens over
+    the time of the decode iterations (Sec. 5.1), which the hand-worked timelines pin."""
+    rows = golden["costs"]["trace"]
+    model, hw, sp = _cost_space(golden, [2], [r["t"] for r in rows])
+    tr = {"arrival": np.array([0.0, 1.0, 1.5]), "in_len": np.zeros(3, np.uint32), "out_len": np.zeros(3, np.uint32)}
+    out = oracle.simulate(sp, tr)
+    assert out["status"].tolist() == [0] * len(rows)
+    assert out["cost_per_hr"].tolist() == [r["cost_per_hr"] for r in rows]
+    for i, r in enumerate(rows):
+        assert out["thr_decode"][i] > 0.0
+        assert out["cost_per_token"][i] == (r["cost_per_hr"] / 3600.0) / out["thr_decode"][i]
+    # the same trace on the unsharded toy at price 1: the first timeline's decode tokens and time
+    tl = golden["timelines"][0]
+    sp1 = toy_space(golden, tl["mem"], tl["kv_block"], [tl["max_batch"]])
+    n = len(tl["arrival"])
+    tr1 = {"arrival": np.array(tl["arrival"]), "in_len": np.zeros(n, np.uint32), "out_len": np.zeros(n, np.uint32)}
+    out1 = oracle.simulate(sp1, tr1)
+    assert out1["cost_per_hr"][0] == 1.0
+    assert out1["cost_per_token"][0] == (1.0 / 3600.0) / (tl["dec_tok"] / tl["dec_time"])
+
+
 def test_paper_log2_rule(golden):
     """Sec. 3.2: multi-GPU throughput = N T_single / (1 + log2 P_TP)."""
     model = list(golden["model"])
