@@ -100,7 +100,7 @@ static int check_trace_overflow(const guide_space &s, const guide_trace &t) {
 // Derived per-model quantities and the reciprocal rates of every hardware x framework pair.
 __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *gh, u32 n_h, const guide_fw *gf,
                                u32 n_f, const u32 *tp, const u32 *dp, u32 n_t, DModel *dm, DRate *dr, double *cost_hr,
-                               double *cost_sec, ulonglong2 *hfmem, double *rate10) {
+                               double *cost_sec, ulonglong2 *hfmem, double *rate10, StageConst *stage_consts) {
     const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n_m) {
         const guide_model m = gm[i];
@@ -114,6 +114,7 @@ __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *g
         d.wbytes = ((u64)d.N * per_layer + 2 * V * H) * d.wb;
         d.kv2 = 2 * (u64)d.N * Dkv * d.kvb;
         dm[i] = d;
+        for (u32 k = 0; k <= n_t; k++) stage_consts[(size_t)k * n_m + i] = stage_const(d, k < n_t ? tp[k] : 1u);
     }
     if (i < n_h * n_f) {
         const guide_hw h = gh[i / n_f];
@@ -231,7 +232,8 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
                  o_hm = take(n_h * n_f * 16), o_hs = take(n_h * n_f * sizeof(HfSorted)),
                  o_po = take(std::max<size_t>(n_m * (s->tp.size() * s->pairs.size() / 4), 1) * 4),
                  o_lo = take(std::max<size_t>(n_m * (s->tp.size() * s->pairs.size() / 16), 1) * 4),
-                 o_tk = take(TICKET_SLOTS * 128), o_r10 = take(n_h * n_f * 80);
+                 o_tk = take(TICKET_SLOTS * 128), o_r10 = take(n_h * n_f * 80),
+                 o_sc = take((s->tp.size() + 1) * n_m * sizeof(StageConst));
     char *blob = nullptr;
     GUIDE_CUDA(cudaMalloc(&blob, off));
     cudaError_t e = cudaSuccess;
@@ -258,7 +260,8 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
                                                  (const u32 *)(blob + o_t), (const u32 *)(blob + o_d), (u32)s->tp.size(),
                                                  (DModel *)(blob + o_dm), (DRate *)(blob + o_dr),
                                                  (double *)(blob + o_ch), (double *)(blob + o_cs),
-                                                 (ulonglong2 *)(blob + o_hm), (double *)(blob + o_r10));
+                                                 (ulonglong2 *)(blob + o_hm), (double *)(blob + o_r10),
+                                                 (StageConst *)(blob + o_sc));
         e = cudaGetLastError();
         if (e == cudaSuccess) e = cudaStreamSynchronize(0);
     }
@@ -277,6 +280,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
     d.view.cost_sec = (const double *)(blob + o_cs);
     d.view.hfmem = (const ulonglong2 *)(blob + o_hm);
     d.view.rate10 = (const double *)(blob + o_r10);
+    d.view.stage_consts = (const StageConst *)(blob + o_sc);
     d.view.hf_sorted = (const HfSorted *)(blob + o_hs);
     d.view.plane_order = (const u32 *)(blob + o_po);
     d.view.line_order = (const u32 *)(blob + o_lo);
@@ -547,7 +551,7 @@ uint64_t guide_trace_size(const guide_trace *t) { return t ? t->arrival.size() :
 
 size_t guide_workspace_bytes(const guide_space *space, const guide_trace *trace, const guide_sim_opts *) {
     if (!space || !trace) return 0;
-    return trace_workspace_bytes((u32)trace->arrival.size());
+    return trace_workspace_bytes((u32)trace->arrival.size(), lane_hints(*space));
 }
 
 int guide_simulate(const guide_space *space_c, const guide_trace *trace_c, const guide_sim_opts *opts,
@@ -579,7 +583,7 @@ int guide_simulate(const guide_space *space_c, const guide_trace *trace_c, const
             return fail(GUIDE_ERR_UNSUPPORTED, "the trace kernel keeps at most %u requests resident; the batch axis goes to %u",
                         GUIDE_TRACE_MAX_BATCH, space->max_batch);
         if ((rc = check_trace_overflow(*space, *trace))) return rc;
-        if ((rc = check_workspace(ws, ws_bytes, trace_workspace_bytes((u32)trace->arrival.size())))) return rc;
+        if ((rc = check_workspace(ws, ws_bytes, trace_workspace_bytes((u32)trace->arrival.size(), lane_hints(*space))))) return rc;
     }
     if (r.count == 0) return GUIDE_OK;
     DSpace ds;
@@ -591,7 +595,7 @@ int guide_simulate(const guide_space *space_c, const guide_trace *trace_c, const
     u32 policies = 0;
     for (const guide_fw &f : space->fw) policies |= f.policy == GUIDE_POLICY_SPLIT_FUSE ? 2u : 1u;
     return launch_trace_sim(ds, dt, r, time_model, tp_model, opts ? opts->max_iters : 0, *out, ws, ws_bytes,
-                            (cudaStream_t)stream, policies);
+                            (cudaStream_t)stream, policies, lane_hints(*space));
 }
 
 size_t guide_select_workspace_bytes(const guide_space *, uint32_t k) {

@@ -72,9 +72,17 @@ int trace_on_device(guide_trace *t, DTrace *out);
 int launch_closed_form(const DSpace &s, Range r, int time_model, int tp_model, const guide_outputs &o,
                        unsigned *ticket, cudaStream_t st);
 // trace_sim.cu
-size_t trace_workspace_bytes(u32 n_req);
+// What the host knows about the configs the one-lane-per-config kernel would take: per class of max
+// batch, how many configs of the whole space have a prompt-first framework with a block size the
+// phase histogram covers (an upper bound: the kernel itself also checks that the config's integer
+// counts stay below 2^53), and the largest such block size.
+static constexpr unsigned LANE_N_CLASSES = 3;
+struct LaneHints { u64 class_configs[LANE_N_CLASSES]; u32 hist_n; };
+LaneHints lane_hints(const guide_space &s);
+size_t trace_workspace_bytes(u32 n_req, const LaneHints &hints);
 int launch_trace_sim(const DSpace &s, const DTrace &t, Range r, int time_model, int tp_model, u64 max_iters,
-                     const guide_outputs &o, void *ws, size_t ws_bytes, cudaStream_t st, u32 policies);
+                     const guide_outputs &o, void *ws, size_t ws_bytes, cudaStream_t st, u32 policies,
+                     const LaneHints &hints);
 // select.cu
 size_t topk_workspace_bytes(u32 k);
 size_t pareto_workspace_bytes();

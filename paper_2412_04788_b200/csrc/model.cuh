@@ -44,6 +44,8 @@ struct HfSorted {
     u32 pad;
 };
 
+struct StageConst;
+
 struct DSpace {
     const DModel *models;
     const DRate *rates;          // [n_h * n_f]
@@ -53,6 +55,7 @@ struct DSpace {
     const double *cost_hr;       // [n_h * n_f][n_t]: price x TP degree
     const double *cost_sec;      // [n_h * n_f][n_t]: (price x TP degree) / 3600
     const ulonglong2 *hfmem;     // [n_h * n_f]: x = usable bytes, y = KV block size (what the memory check reads)
+    const StageConst *stage_consts;   // [n_t + 1][n_m]: the task-table factors per (TP degree, model); the last group is t = 1
     const double *rate10;        // [n_h * n_f][10]: inv_c[3], inv_m[3], inv_comm, clat, tovh, flash (0.0 or 1.0); 16-byte aligned rows
     // Orders that only steer which thread does what (any permutation gives the same results):
     const HfSorted *hf_sorted;   // [n_h * n_f]: the pairs grouped by KV block size, largest usable memory first
@@ -163,6 +166,99 @@ __device__ __forceinline__ double task_time(double F, double B, double ic, doubl
     return TIME_SUM ? tc + tm : (tc > tm ? tc : tm);   // Sec. 3.5.1 literal sum, or the roofline of Sec. 3.4.2
 }
 
+// ---- the same table in doubles ---------------------------------------------------------------------
+// Per (model, tensor-parallel degree): the factors that turn the token counts of a stage into the
+// entries of its task table.  Products and sums of integers stay exact in binary64 below 2^53, and
+// scaling by 1/t (a power of two) and by the multiplicities commutes with rounding, so
+//   T x factor  ==  (double)(T * integer factor) x 1/t
+// bit for bit whenever the integer count is below 2^53.  A kernel that has checked that bound for a
+// config can build its tables without integer products and conversions.
+struct StageConst {
+    double f1, b1;        // norm x2:        8 H, 4 H a_b                   (per new token)
+    double f2, w2;        // q_proj, o_proj: 2 H H / t;  H H w_b
+    double ha;            // activations of one token: H a_b
+    double f3, w3, dk;    // k/v_proj x2:    4 H Dkv / t;  H Dkv w_b;  Dkv kv_b
+    double f5, b5;        // residual x2:    2 H, 6 H a_b
+    double f6, w6, ia;    // up (+ gate):    (1+g) 2 H I / t;  H I w_b;  I a_b
+    double mult6;         // 1 + g
+    double f7, b7;        // activation:     4 I / t, (2+g) I a_b / t
+    double f8;            // down:           2 I H / t  (weights and activations as up)
+    double f13, w13, va;  // lm_head:        2 H V / t;  H V w_b;  V a_b      (per emitting sequence)
+    double hops, cb;      // all-reduce:     2 (t-1);  2 (t-1) H a_b / t
+    double inv_t;
+    double f9, kv, f10, xb;   // attention:  2 H / t;  Dkv kv_b;  5 n_h / t;  n_h a_b (score bytes per unit of A)
+    double pad[5];        // 256 bytes
+};
+
+__device__ __forceinline__ StageConst stage_const(const DModel &m, u32 t) {
+    StageConst c;
+    const double inv_t = 1.0 / (double)t;
+    const u64 H = m.H, I = m.I, Dkv = m.Dkv, V = m.V, ab = m.ab, wb = m.wb, kvb = m.kvb;
+    c.f1 = cvt(8 * H); c.b1 = cvt(4 * H * ab);
+    c.f2 = cvt(2 * H * H) * inv_t; c.w2 = cvt(H * H * wb);
+    c.ha = cvt(H * ab);
+    c.f3 = cvt(4 * H * Dkv) * inv_t; c.w3 = cvt(H * Dkv * wb); c.dk = cvt(Dkv * kvb);
+    c.f5 = cvt(2 * H); c.b5 = cvt(6 * H * ab);
+    c.mult6 = (double)(1 + m.g);
+    c.f6 = c.mult6 * (cvt(2 * H * I) * inv_t); c.w6 = cvt(H * I * wb); c.ia = cvt(I * ab);
+    c.f7 = cvt(4 * I) * inv_t; c.b7 = cvt((2 + m.g) * I * ab) * inv_t;
+    c.f8 = cvt(2 * I * H) * inv_t;
+    c.f13 = cvt(2 * H * V) * inv_t; c.w13 = cvt(H * V * wb); c.va = cvt(V * ab);
+    c.hops = cvt((u64)(2 * (t - 1))); c.cb = cvt((u64)(2 * (t - 1)) * H * ab) * inv_t;
+    c.inv_t = inv_t;
+    c.f9 = cvt(2 * H) * inv_t; c.kv = cvt(Dkv * kvb); c.f10 = cvt(5 * (u64)m.nh) * inv_t; c.xb = cvt((u64)m.nh * ab);
+    for (int i = 0; i < 5; i++) c.pad[i] = 0.0;
+    return c;
+}
+
+// Upper bound (as a double: no wrap-around, rounding far below the margin) of the largest integer
+// count a stage of at most T new tokens, E emitting sequences, attention work A and context C
+// produces for this model (R = 1).  While it is below 2^52 the doubles above reproduce the integer
+// table exactly (the limit is 2^53; the factor of two covers this bound's own rounding).
+__device__ __forceinline__ double stage_count_bound(const DModel &m, u32 t, double T, double E, double A, double C) {
+    const double H = m.H, I = m.I, Dkv = m.Dkv, V = m.V, ab = m.ab, wb = m.wb, kvb = m.kvb, nh = m.nh, g = m.g;
+    const double big = fmax(fmax(H, I), Dkv), bytes = fmax(ab, kvb);
+    double v = 8.0 * T * H;
+    v = fmax(v, 6.0 * T * H * ab);
+    v = fmax(v, 4.0 * T * big * big);                    // 2 T H H, 4 T H Dkv, (1+g) 2 T H I, 2 T I H
+    v = fmax(v, big * big * wb + T * big * bytes);       // weights of one matrix + its activations / KV written
+    v = fmax(v, (2.0 + g) * T * I * ab);
+    v = fmax(v, 2.0 * E * H * V);
+    v = fmax(v, H * V * wb + E * V * ab + E * H * ab);
+    v = fmax(v, 2.0 * (double)t * T * H * ab);
+    v = fmax(v, 2.0 * H * A);
+    v = fmax(v, 5.0 * nh * A);
+    v = fmax(v, T * H * ab + C * Dkv * kvb + 2.0 * nh * A * ab);
+    return v;
+}
+
+// One stage time (R = 1) from the doubles: the same operations in the same order as
+// build_fixed_tasks / build_attn_tasks followed by eval_phase.  rate: a row of rate10
+// (inv_c[LINEAR, ATTN, ELEM], inv_m[LINEAR, ATTN, ELEM], inv_comm, clat, tovh, flash).
+struct StageFixed { double fix, comm, head, tha; };
+
+template <int TIME_SUM>
+__device__ __forceinline__ StageFixed stage_fixed(const StageConst &c, const double *rate, double Td, double Ed) {
+    const double icL = rate[0], icE = rate[2], imL = rate[3], imE = rate[5];
+    const double tha = Td * c.ha;
+    const double t2 = task_time<TIME_SUM>(Td * c.f2, (c.w2 + tha) * c.inv_t + tha, icL, imL);
+    double s = task_time<TIME_SUM>(Td * c.f1, Td * c.b1, icE, imE);
+    s = s + t2;
+    s = s + task_time<TIME_SUM>(Td * c.f3, 2.0 * ((c.w3 + Td * c.dk) * c.inv_t + tha), icL, imL);
+    s = s + t2;
+    s = s + task_time<TIME_SUM>(Td * c.f5, Td * c.b5, icE, imE);
+    const double up = (c.w6 + Td * c.ia) * c.inv_t + tha;        // bytes of one FFN matrix pass
+    s = s + task_time<TIME_SUM>(Td * c.f6, c.mult6 * up, icL, imL);
+    s = s + task_time<TIME_SUM>(Td * c.f7, Td * c.b7, icE, imE);
+    s = s + task_time<TIME_SUM>(Td * c.f8, up, icL, imL);
+    StageFixed o;
+    o.fix = s;
+    o.comm = 2.0 * (c.hops * rate[7] + (Td * c.cb) * rate[6]);
+    o.head = task_time<TIME_SUM>(Ed * c.f13, (c.w13 + Ed * c.va) * c.inv_t + Ed * c.ha, icL, imL);
+    o.tha = tha * c.inv_t;
+    return o;
+}
+
 // Sum of the eight non-attention layer tasks in their fixed order.
 template <int TIME_SUM>
 __device__ __forceinline__ double eval_fixed(const TaskTab &k, const DRate &r) {
@@ -205,6 +301,26 @@ __device__ __forceinline__ double combine_phase(double s_fix, double s_att, doub
     double tp = Rd * tovh + (Nd * layer + t_head);
     if (log2_factor != 1.0) tp = tp * log2_factor;   // x1.0 would be exact anyway
     return tp;
+}
+
+// Time of a prompt pass over T new tokens of E requests with attention work A = sum of squared
+// lengths (the context is the new tokens themselves), from the doubles; out of line: events are
+// rare next to decode iterations and the call keeps their registers apart.
+struct AttnRates { double c_f9, c_f10, c_b10, icA, imA, Nd, tovh, lf; };
+template <int TIME_SUM>
+__device__ __noinline__ double stage_prompt_pass(const StageConst *scp, const double *rate, double Td, double Ed, double Ad,
+                                                 const AttnRates *ar) {
+    const StageConst c = *scp;
+    const StageFixed sf = stage_fixed<TIME_SUM>(c, rate, Td, Ed);
+    const double xw = rate[9] != 0.0 ? 0.0 : c.xb;           // FlashAttention: no score-matrix traffic
+    const double t9 = task_time<TIME_SUM>(Ad * ar->c_f9, ((Td * c.ha + Td * c.kv) + Ad * xw) * c.inv_t, ar->icA, ar->imA);
+    const double t10 = task_time<TIME_SUM>(Ad * ar->c_f10, Ad * ar->c_b10, ar->icA, ar->imA);
+    return combine_phase(sf.fix, (t9 + t10) + t9, sf.comm, sf.head, 1.0, ar->Nd, ar->tovh, ar->lf);
+}
+// The terms of a decode iteration that depend on the number of residents only.
+template <int TIME_SUM>
+__device__ __noinline__ StageFixed stage_decode_terms(const StageConst *scp, const double *rate, double nd) {
+    return stage_fixed<TIME_SUM>(*scp, rate, nd, nd);
 }
 
 template <int TIME_SUM>

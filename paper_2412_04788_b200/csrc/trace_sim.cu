@@ -24,12 +24,14 @@
 // config and is read through the read-only path, so it stays cache resident.
 #include "guide_internal.cuh"
 #include "trace_fuse.cuh"
+#include "trace_lanes.cuh"
 
 namespace guide {
 
 static constexpr u32 SIM_WARPS_PER_BLOCK = 8;
 static constexpr u32 SIM_THREADS = SIM_WARPS_PER_BLOCK * 32;
 static constexpr u32 SIM_MAX_WARPS = 6144;        // workspace is sized for this many resident warps
+static constexpr u32 LANE_MAX_WARPS = 148 * 16;   // ... and for this many warps of the lane kernel
 static constexpr u32 SLOTS = GUIDE_TRACE_MAX_BATCH;
 static constexpr u32 HIST = 64;                   // block sizes up to this use the phase histogram
 static constexpr u32 M_PHASE = 0x3F, M_FIRST = 0x40, M_NEEDS_PREFILL = 0x80;
@@ -44,7 +46,6 @@ static size_t per_warp_bytes(u32 n_req) {
     return ((n * 4 + 255) / 256 * 256) + ((n * 8 + 255) / 256 * 256) + ((p * 8 + 255) / 256 * 256);
 }
 
-size_t trace_workspace_bytes(u32 n_req) { return 256 + (size_t)SIM_MAX_WARPS * per_warp_bytes(n_req); }
 
 __device__ __forceinline__ u64 warp_sum(u64 v) {
     for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
@@ -77,17 +78,6 @@ struct SlotArrays {
     u32 hist[HIST];     // residents per (cache - D) mod block
     unsigned char meta[SLOTS];   // phase (6 bits) | first-ever prompt pass | waiting for its prompt pass
 };
-
-// The work order visits the batch axis slowest when the whole space is simulated, so configs with
-// a small max batch (the long schedules) are started first.
-__device__ __forceinline__ u64 work_to_index(const DSpace &s, u64 w, bool reorder) {
-    if (!reorder) return w;
-    const u64 tl = (u64)s.n_t * s.n_l;
-    const u64 per_b = (u64)s.n_m * s.n_h * s.n_f * tl;
-    const u64 b = w / per_b, rest = w % per_b;
-    const u64 mhf = rest / tl, x = rest % tl;
-    return (mhf * s.n_b + b) * tl + x;
-}
 
 // Results of one simulated config: per-request values, means in request order, nearest-rank
 // percentiles (sorted in the tpot slice, which is free by then).  Called by the whole warp.
@@ -176,7 +166,7 @@ __device__ __forceinline__ void write_trace_results(const guide_outputs &o, u64 
 template <int TIME_SUM>
 __global__ void __launch_bounds__(SIM_THREADS, 3)
 k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide_outputs o, u32 *counter,
-            unsigned char *scratch, size_t per_warp, u32 gen_bytes, u32 first_bytes, int reorder) {
+            unsigned char *scratch, size_t per_warp, u32 gen_bytes, u32 first_bytes, int reorder, u32 lane_maxb, u32 lane_hist) {
     __shared__ SlotArrays sh[SIM_WARPS_PER_BLOCK];
     const u32 lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const u32 warp_global = blockIdx.x * SIM_WARPS_PER_BLOCK + wib;
@@ -208,6 +198,9 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         const double lf = log2_rule_factor(t, tp_model), Nd = (double)m.N;
         const double inv_tt = 1.0 / (double)tt;
         const double icA = rt.inv_c[CLS_ATTN], imA = rt.inv_m[CLS_ATTN];
+        // configs the lane kernel was launched for are simulated there
+        if (lanes_take(lane_maxb, lane_hist, b, blk,
+                       lanes_exact(m, tt, b, max(tr.max_tokens, tr.any_zero ? Lin + Lout : 0u)))) continue;
 
         // ---- what fits (Sec. 3.2 Step 1) ----
         const u64 blocks_total = rt.usable > mi.w_gpu ? floor_div(rt.usable - mi.w_gpu, (u64)blk * mi.kv_tok) : 0;
@@ -550,9 +543,224 @@ k_trace_fuse(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guid
     }
 }
 
+// Results of one config simulated by the lane kernel: per-request values, means in request order, nearest-rank
+// percentiles.  first[i]: time of request i's first token; finish[i]: time of its last one (the
+// slice has room for the next power of two of doubles and serves as the sort buffer afterwards).
+// Called by the whole warp; out of line, so that its registers (the sort keeps a batch of pairs in
+// flight) do not weigh on the simulation loops of its callers.
+__device__ __noinline__ void write_lane_results(const guide_outputs &o, u64 j, u32 n, u32 st, u32 fit, double clock,
+                                                 double dec_time, u64 dec_tok, u64 n_iters, u64 n_req_iters, double cost_hr,
+                                                 const DTrace &tr, u32 Lout, double *first, double *finish, u32 lane) {
+    const double inf = __longlong_as_double(0x7FF0000000000000LL);
+    double *rq_ttft = o.req_ttft ? o.req_ttft + j * n : nullptr;
+    double *rq_tpot = o.req_tpot ? o.req_tpot + j * n : nullptr;
+    __syncwarp();
+    if (st) {
+        if (lane == 0) {
+            if (o.latency) o.latency[j] = inf;
+            if (o.ttft) o.ttft[j] = inf;
+            if (o.ttft_p50) o.ttft_p50[j] = inf;
+            if (o.ttft_p99) o.ttft_p99[j] = inf;
+            if (o.tpot) o.tpot[j] = inf;
+            if (o.thr_decode) o.thr_decode[j] = 0.0;
+            if (o.cost_per_hr) o.cost_per_hr[j] = inf;
+            if (o.cost_per_token) o.cost_per_token[j] = inf;
+            if (o.status) o.status[j] = (uint8_t)st;
+            if (o.bmax) o.bmax[j] = fit;
+            if (o.n_iters) o.n_iters[j] = 0;
+            if (o.n_req_iters) o.n_req_iters[j] = 0;
+        }
+        for (u32 i = lane; i < n; i += 32) {
+            if (rq_ttft) __stcs(rq_ttft + i, inf);
+            if (rq_tpot) __stcs(rq_tpot + i, inf);
+        }
+        return;
+    }
+    // means in request order: 32 values at a time, added one after the other
+    double s_ttft = 0.0, s_tpot = 0.0;
+    for (u32 base = 0; base < n; base += 32) {
+        const u32 i = base + lane;
+        double vt = 0.0, vp = 0.0;
+        if (i < n) {
+            const double f = first[i];
+            const u32 out = __ldg(tr.in_len + i) ? __ldg(tr.out_len + i) : Lout;
+            vt = f - __ldg(tr.arrival + i);
+            vp = out > 1 ? (finish[i] - f) / (double)(out - 1) : 0.0;     // time per output token after the first
+            if (rq_ttft) __stcs(rq_ttft + i, vt);
+            if (rq_tpot) __stcs(rq_tpot + i, vp);
+        }
+        const u32 lim = min(32u, n - base);
+        for (u32 l = 0; l < lim; l++) {
+            s_ttft = s_ttft + __shfl_sync(0xFFFFFFFFu, vt, l);
+            s_tpot = s_tpot + __shfl_sync(0xFFFFFFFFu, vp, l);
+        }
+        if (i < n) first[i] = vt;             // keep TTFT for the percentile sort
+    }
+    // nearest-rank percentiles: bitonic sort of the TTFTs in the (now free) finish slice.  The pairs of
+    // a stage are disjoint, so a lane loads a batch of them before it stores any: the loads overlap.
+    double *buf = finish;
+    if (o.ttft_p50 || o.ttft_p99) {
+        u32 P = 1;
+        while (P < n) P <<= 1;
+        __syncwarp();
+        for (u32 i = lane; i < P; i += 32) buf[i] = i < n ? first[i] : inf;
+        __syncwarp();
+        constexpr u32 BATCH = 8;
+        for (u32 size = 2; size <= P; size <<= 1) {
+            for (u32 stride = size >> 1; stride > 0; stride >>= 1) {
+                for (u32 i0 = lane; i0 < (P >> 1); i0 += 32 * BATCH) {
+                    double a[BATCH], bb[BATCH];
+                    u32 lo[BATCH];
+#pragma unroll
+                    for (u32 u = 0; u < BATCH; u++) {
+                        const u32 i = i0 + 32 * u;
+                        lo[u] = ((i & ~(stride - 1)) << 1) | (i & (stride - 1));
+                        if (i < (P >> 1)) { a[u] = buf[lo[u]]; bb[u] = buf[lo[u] + stride]; }
+                    }
+#pragma unroll
+                    for (u32 u = 0; u < BATCH; u++) {
+                        const u32 i = i0 + 32 * u;
+                        const bool up = (lo[u] & size) == 0;
+                        if (i < (P >> 1) && (bb[u] < a[u]) == up) { buf[lo[u]] = bb[u]; buf[lo[u] + stride] = a[u]; }
+                    }
+                }
+                __syncwarp();
+            }
+        }
+    }
+    if (lane == 0) {
+        const double nd = (double)n;
+        const double thr = dec_time > 0.0 ? cvt(dec_tok) / dec_time : 0.0;
+        if (o.latency) o.latency[j] = clock;
+        if (o.ttft) o.ttft[j] = s_ttft / nd;
+        if (o.ttft_p50) o.ttft_p50[j] = buf[(50ull * n + 99) / 100 - 1];
+        if (o.ttft_p99) o.ttft_p99[j] = buf[(99ull * n + 99) / 100 - 1];
+        if (o.tpot) o.tpot[j] = s_tpot / nd;
+        if (o.thr_decode) o.thr_decode[j] = thr;
+        if (o.cost_per_hr) o.cost_per_hr[j] = cost_hr;
+        if (o.cost_per_token) o.cost_per_token[j] = thr > 0.0 ? (cost_hr / 3600.0) / thr : inf;
+        if (o.status) o.status[j] = 0;
+        if (o.bmax) o.bmax[j] = fit;
+        if (o.n_iters) o.n_iters[j] = n_iters;
+        if (o.n_req_iters) o.n_req_iters[j] = n_req_iters;
+    }
+}
+
+// Prompt-first configs, one per lane (trace_lanes.cuh), max batch in [minb, maxb]; everything else is
+// skipped here and simulated by another launch of this kernel or by k_trace_sim.
+template <int TIME_SUM, int UNROLL>
+__global__ void __launch_bounds__(LANE_MAX_THREADS, 4)
+k_trace_lanes(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide_outputs o, unsigned long long *counter,
+              unsigned char *scratch, size_t per_lane, u32 gen_bytes, u32 first_bytes, int reorder, u32 minb, u32 maxb,
+              u32 hist_n, u32 lanes_used, u32 round_len) {
+    extern __shared__ __align__(16) unsigned char lane_smem[];
+    const u32 lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    unsigned char *wsm = lane_smem + (size_t)wib * lanes_used * (12 * maxb + 4 * hist_n);
+    const u32 n = tr.n;
+    lanes_simulate<TIME_SUM, UNROLL>(s, tr, r, tp_model, max_iters_opt, counter, scratch, per_lane, gen_bytes, first_bytes, reorder, minb,
+                             maxb, hist_n, lanes_used, round_len, wsm,
+                             [&](u64 j, u32 st, u32 fit, double clock, double dec_time, u64 dec_tok, u64 n_iters, u64 n_req_iters,
+                                 double cost_hr, u32 Lout, double *first, double *tpot) {
+                                 write_lane_results(o, j, n, st, fit, clock, dec_time, dec_tok, n_iters, n_req_iters, cost_hr,
+                                                    tr, Lout, first, tpot, lane);
+                                 __syncwarp();
+                             });
+}
+
+// The lane kernel is launched once per class of max batch: the slots of a lane take 12 bytes per
+// resident request, so a launch for large batches gives a warp fewer lanes.
+// round: decode iterations a lane may run between two event phases (events come more often with larger batches)
+// unroll: iterations per trip of the run loop (4: long runs, where a lane's own chain latency is the limit)
+struct LaneClass { u32 minb, maxb, lanes, round, unroll; };
+static const LaneClass LANE_CLASSES[LANE_N_CLASSES] = {{1, 16, 32, 64, 4}, {17, 64, 32, 16, 1}, {65, GUIDE_TRACE_MAX_BATCH, 8, 8, 1}};
+#ifndef LANE_CLASSES_ENABLED
+#define LANE_CLASSES_ENABLED 1      // classes above this go to the warp-per-config kernel
+#endif
+
+typedef void (*LaneKernel)(DSpace, DTrace, Range, int, u64, guide_outputs, unsigned long long *, unsigned char *, size_t, u32, u32,
+                           int, u32, u32, u32, u32, u32);
+template <int TIME_SUM>
+static LaneKernel lane_kernel(u32 unroll) {
+    return unroll == 4 ? (LaneKernel)k_trace_lanes<TIME_SUM, 4> : (LaneKernel)k_trace_lanes<TIME_SUM, 1>;
+}
+static constexpr u32 LANE_BLOCK_WARPS = 4;
+static constexpr size_t LANE_SMEM_LIMIT = 112 * 1024;
+
+static size_t lane_block_smem(const LaneClass &c, u32 lanes, u32 hist_n) {
+    return (size_t)LANE_BLOCK_WARPS * lanes * (12 * c.maxb + 4 * hist_n);
+}
+
+LaneHints lane_hints(const guide_space &s) {
+    LaneHints h{};
+    h.hist_n = 1;
+    const u32 n_classes = std::min<u32>(LANE_CLASSES_ENABLED, LANE_N_CLASSES);
+    u64 n_fw = 0;
+    for (const guide_fw &f : s.fw)
+        if (f.policy == GUIDE_POLICY_PREFILL_FIRST && f.kv_block <= LANE_HIST_MAX) {
+            n_fw++;
+            h.hist_n = std::max(h.hist_n, f.kv_block);
+        }
+    const u64 per_b = (u64)s.models.size() * s.hw.size() * n_fw * s.tp.size() * s.pairs.size();
+    for (uint32_t b : s.batch)
+        for (u32 c = 0; c < n_classes; c++)
+            if (b >= LANE_CLASSES[c].minb && b <= LANE_CLASSES[c].maxb) h.class_configs[c] += per_b;
+    return h;
+}
+
+// The kernels of a call run one after the other and share the region: a slice per resident warp of
+// the warp-per-config kernels, a slice per lane that can get a config in a launch of the lane kernel
+// (a launch rounds its warps up to whole blocks: one block of slack covers that).
+size_t trace_workspace_bytes(u32 n_req, const LaneHints &hints) {
+    size_t slices = SIM_MAX_WARPS;
+    for (u32 c = 0; c < LANE_N_CLASSES; c++) {
+        const u64 lanes = LANE_CLASSES[c].lanes;
+        slices = std::max<size_t>(slices, std::min<u64>((u64)LANE_MAX_WARPS * lanes,
+                                                        hints.class_configs[c] + LANE_BLOCK_WARPS * lanes));
+    }
+    return 256 + slices * per_warp_bytes(n_req);
+}
+
+struct LanePlan { u32 blocks, lanes_used; size_t smem; };
+
+template <int TIME_SUM>
+static int plan_lanes(const DSpace &s, const LaneHints &h, Range r, u32 cls, LanePlan *p) {
+    const LaneClass &c = LANE_CLASSES[cls];
+    p->blocks = 0; p->lanes_used = c.lanes; p->smem = 0;
+    if (h.class_configs[cls] == 0) return GUIDE_OK;
+    static std::mutex mu;
+    static bool opted[64] = {};
+    int dev = 0;
+    GUIDE_CUDA(cudaGetDevice(&dev));
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (dev < 64 && !opted[dev]) {
+            for (u32 u : {1u, 4u})
+                GUIDE_CUDA(cudaFuncSetAttribute(lane_kernel<TIME_SUM>(u), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (int)LANE_SMEM_LIMIT));
+            opted[dev] = true;
+        }
+    }
+    // configs of this launch among the range: all of the class for a whole space, else at most the range
+    const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
+    const u64 mine = r.count == total ? h.class_configs[cls] : std::min<u64>(r.count, h.class_configs[cls]);
+    // Few configs: spread them over more warps, fewer lanes each (a lane's pace does not depend on its
+    // neighbours, a warp's issue slots are shared by them).  Aim at eight warps per SM.
+    const u64 lanes = (mine + (u64)num_sms() * 8 - 1) / ((u64)num_sms() * 8);
+    const u64 fit = LANE_SMEM_LIMIT / lane_block_smem(c, 1, h.hist_n);      // lanes whose slots fit a block's shared memory (>= 8)
+    p->lanes_used = (u32)std::max<u64>(1, std::min<u64>(std::min<u64>(c.lanes, fit), lanes));
+    p->smem = lane_block_smem(c, p->lanes_used, h.hist_n);
+    int per_sm = 0;
+    GUIDE_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, lane_kernel<TIME_SUM>(c.unroll), LANE_BLOCK_WARPS * 32, p->smem));
+    if (per_sm < 1) per_sm = 1;
+    const u64 resident_warps = std::min<u64>((u64)num_sms() * per_sm * LANE_BLOCK_WARPS, LANE_MAX_WARPS);
+    const u64 warps = std::min<u64>(resident_warps, (mine + p->lanes_used - 1) / p->lanes_used);
+    p->blocks = (u32)((warps + LANE_BLOCK_WARPS - 1) / LANE_BLOCK_WARPS);
+    return GUIDE_OK;
+}
+
 template <int TIME_SUM>
 static int launch_one(const DSpace &s, const DTrace &t, Range r, int tp_model, u64 max_iters, const guide_outputs &o,
-                      void *ws, cudaStream_t st, u32 policies) {
+                      void *ws, size_t ws_bytes, cudaStream_t st, u32 policies, const LaneHints &hints) {
     const size_t pw = per_warp_bytes(t.n);
     const u32 gen_bytes = (u32)(((size_t)t.n * 4 + 255) / 256 * 256);
     const u32 first_bytes = (u32)(((size_t)t.n * 8 + 255) / 256 * 256);
@@ -563,20 +771,47 @@ static int launch_one(const DSpace &s, const DTrace &t, Range r, int tp_model, u
     u32 blocks = (u32)num_sms() * (u32)per_sm;
     blocks = std::min<u32>(blocks, SIM_MAX_WARPS / SIM_WARPS_PER_BLOCK);
     blocks = (u32)std::min<u64>(blocks, (r.count + SIM_WARPS_PER_BLOCK - 1) / SIM_WARPS_PER_BLOCK);
+    int per_sm_f = 0;
+    GUIDE_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm_f, k_trace_fuse<TIME_SUM>, SIM_THREADS, 0));
+    if (per_sm_f < 1) per_sm_f = 1;
+    u32 blocks_f = (u32)num_sms() * (u32)per_sm_f;
+    blocks_f = std::min<u32>(blocks_f, SIM_MAX_WARPS / SIM_WARPS_PER_BLOCK);
+    blocks_f = (u32)std::min<u64>(blocks_f, (r.count + SIM_WARPS_PER_BLOCK - 1) / SIM_WARPS_PER_BLOCK);
     const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
     const int reorder = r.first == 0 && r.count == total;
     unsigned char *scratch = (unsigned char *)ws + 256;
-    // one kernel per scheduling policy present in the space; each skips the other's configs
+    // one kernel per scheduling policy present in the space; each skips the other's configs.  The
+    // prompt-first configs with a small max batch go to the lane kernel first (the long schedules).
+    if ((policies & 3) && 256 + (size_t)std::max(blocks, blocks_f) * SIM_WARPS_PER_BLOCK * pw > ws_bytes)
+        return fail(GUIDE_ERR_WORKSPACE, "workspace too small for the resident warps");
     if (policies & 1) {
+        u32 lane_maxb = 0;
+        for (u32 cls = 0; cls < LANE_N_CLASSES; cls++) {
+            LanePlan lp;
+            int rc = plan_lanes<TIME_SUM>(s, hints, r, cls, &lp);
+            if (rc) return rc;
+            if (lp.blocks == 0) continue;
+            // every lane that can get a config has its slice inside the workspace
+            if (256 + (size_t)lp.blocks * LANE_BLOCK_WARPS * lp.lanes_used * pw > ws_bytes)
+                return fail(GUIDE_ERR_WORKSPACE, "workspace too small for the lane kernel's %u blocks", lp.blocks);
+            GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
+            lane_kernel<TIME_SUM>(LANE_CLASSES[cls].unroll)<<<lp.blocks, LANE_BLOCK_WARPS * 32, lp.smem, st>>>(
+                s, t, r, tp_model, max_iters, o, (unsigned long long *)ws, scratch, pw, gen_bytes, first_bytes, reorder,
+                LANE_CLASSES[cls].minb, LANE_CLASSES[cls].maxb, hints.hist_n, lp.lanes_used, LANE_CLASSES[cls].round);
+            GUIDE_CUDA(cudaGetLastError());
+            lane_maxb = std::max(lane_maxb, LANE_CLASSES[cls].maxb);
+        }
+        // always launched: the lane kernel leaves it the configs whose counts do not stay below 2^53
+        // or whose block size the phase histogram does not cover
         GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
         k_trace_sim<TIME_SUM><<<blocks, SIM_THREADS, 0, st>>>(s, t, r, tp_model, max_iters, o, (u32 *)ws, scratch, pw,
-                                                             gen_bytes, first_bytes, reorder);
+                                                             gen_bytes, first_bytes, reorder, lane_maxb, hints.hist_n);
         GUIDE_CUDA(cudaGetLastError());
     }
     if (policies & 2) {
         GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
-        k_trace_fuse<TIME_SUM><<<blocks, SIM_THREADS, 0, st>>>(s, t, r, tp_model, max_iters, o, (u32 *)ws, scratch, pw,
-                                                              gen_bytes, first_bytes, reorder);
+        k_trace_fuse<TIME_SUM><<<blocks_f, SIM_THREADS, 0, st>>>(s, t, r, tp_model, max_iters, o, (u32 *)ws, scratch, pw,
+                                                                gen_bytes, first_bytes, reorder);
         GUIDE_CUDA(cudaGetLastError());
     }
     return GUIDE_OK;
@@ -584,10 +819,10 @@ static int launch_one(const DSpace &s, const DTrace &t, Range r, int tp_model, u
 
 // policies: bit 0 = some framework schedules prompt-first, bit 1 = some by split and fuse
 int launch_trace_sim(const DSpace &s, const DTrace &t, Range r, int time_model, int tp_model, u64 max_iters,
-                     const guide_outputs &o, void *ws, size_t, cudaStream_t st, u32 policies) {
+                     const guide_outputs &o, void *ws, size_t ws_bytes, cudaStream_t st, u32 policies, const LaneHints &hints) {
     if (r.count > 0xFFFFFFF0ull) return fail(GUIDE_ERR_UNSUPPORTED, "at most 2^32 - 16 configs per trace launch");
-    return time_model ? launch_one<1>(s, t, r, tp_model, max_iters, o, ws, st, policies)
-                      : launch_one<0>(s, t, r, tp_model, max_iters, o, ws, st, policies);
+    return time_model ? launch_one<1>(s, t, r, tp_model, max_iters, o, ws, ws_bytes, st, policies, hints)
+                      : launch_one<0>(s, t, r, tp_model, max_iters, o, ws, ws_bytes, st, policies, hints);
 }
 
 }  // namespace guide
