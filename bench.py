@@ -38,10 +38,14 @@ if ROOT not in sys.path:
 import numpy as np
 
 BYTES_SIM = 6 * 8 + 1 + 4          # six fp64 metrics + status + bmax written per config
-# dram__bytes_read.sum + dram__bytes_write.sum of one guide_simulate call on the full workload 5: the
-# k_closed_form_memory and k_closed_form_lines launches together (profiles/launch_list_bench_c5_step.md);
-# only meaningful for that size and those kernel versions
-K1_TRAFFIC_C5 = 591_900_000 + 171_500_000 + 100_000
+# Non-fused fp64 instruction rate of the device (148 SMs x 64 fp64 lanes x 1.965 GHz), as measured by the
+# package's own micro-benchmark (python -m paper_2412_04788_b200.fp64_peak): the peak of every "alu" bound.
+FP64_ISSUE_PEAK = 18.5e12
+# fp64 operations the method itself asks for (one scalar chain per config, whatever the kernel's layout):
+# a decode iteration = 2 attention tasks x (2 mul, compare, add) + the sums and the clock, about 24;
+# a closed-form config that fits = 2 stages x 13 task times x (2 mul, compare, add) + metrics, about 120.
+FP64_OPS_PER_ITERATION = 24
+FP64_OPS_PER_CLOSED_FORM_CONFIG = 120
 SIM_FIELDS = ("latency", "ttft", "tpot", "thr_decode", "cost_per_hr", "cost_per_token", "status", "bmax")
 TRACE_FIELDS = ("latency", "ttft", "ttft_p50", "ttft_p99", "tpot", "thr_decode", "cost_per_hr", "cost_per_token",
                 "status", "bmax", "n_iters", "n_req_iters")
@@ -53,6 +57,21 @@ def measured_peaks():
         with open(path) as f:
             return float(json.load(f)["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def recorded_traffic(n_configs):
+    """DRAM bytes of one guide_simulate call from the last profiler capture (written next to the
+    profile summaries by paper_2412_04788_b200/traffic_record.py), or None when the capture was of
+    another size or the kernel sources have changed since."""
+    from paper_2412_04788_b200 import traffic_record
+    path = os.path.join(ROOT, "profiles", "k_closed_form_c5_traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        rec = json.load(f)
+    if rec.get("configs") != n_configs or rec.get("sources_sha256") != traffic_record.sources_sha256():
+        return None
+    return rec.get("dram_bytes_per_call")
 
 
 class ClockSampler(threading.Thread):
@@ -198,8 +217,58 @@ def time_call(torch, fn, reps=3, warm=1, flush=None):
     return min(ts), sorted(ts)[len(ts) // 2]
 
 
-def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full, fraction=None):
-    """Workloads 1, 3, 4, 5, each timed on its own: best of a few launches, CUDA events."""
+def oracle_seconds(oracle, space, trace, stride, n_total, threads):
+    """The oracle, as it stands, on every stride-th config of a workload: (seconds, configs, iterations,
+    request-iterations) on `threads` host threads (0 = all)."""
+    count = (n_total + stride - 1) // stride
+    t0 = time.perf_counter()
+    out = oracle.simulate(space, trace, first=0, count=count, stride=stride, n_threads=threads)
+    dt = time.perf_counter() - t0
+    return dt, count, int(out["n_iters"].sum()), int(out["n_req_iters"].sum())
+
+
+HOST_CORES = None       # threads the oracle's OpenMP runtime starts with; read before any call narrows it
+
+
+def host_cores(oracle):
+    global HOST_CORES
+    if HOST_CORES is None:
+        HOST_CORES = oracle.threads()
+    return HOST_CORES
+
+
+def cpu_baseline_of(oracle, space, trace, n_total, stride_all, stride_one, unit_iters):
+    """Oracle timings beside a workload: all host cores on one stride, one core on a sparser one."""
+    res = {"kind": "oracle", "cores": host_cores(oracle)}
+    for tag, stride, threads in (("all_cores", stride_all, host_cores(oracle)), ("one_core", stride_one, 1)):
+        dt, count, iters, req_iters = oracle_seconds(oracle, space, trace, stride, n_total, threads)
+        res[tag] = {"seconds": dt, "configs": count, "configs_per_s": count / dt,
+                    "sample": f"every {stride}th config" if stride > 1 else "the whole workload",
+                    "seconds_for_the_whole_workload_at_this_rate": dt * n_total / count}
+        if unit_iters:
+            res[tag]["request_iters_per_s"] = req_iters / dt
+            res[tag]["iters_per_s"] = iters / dt
+    res["value"] = res["all_cores"]["configs_per_s"]
+    res["unit"] = "configs/s"
+    res["sample"] = res["all_cores"]["sample"]
+    return res
+
+
+def alu_roofline(ops_per_s, what):
+    return {"bound": "alu", "achieved": ops_per_s / 1e12, "peak": FP64_ISSUE_PEAK / 1e12, "unit": "T fp64 op/s",
+            "frac": ops_per_s / FP64_ISSUE_PEAK, "traffic": None, "peak_kind": "of measured (fp64 issue micro-benchmark)",
+            "what": what}
+
+
+def hbm_roofline(bytes_per_call, ms, hbm_peak, peak_kind, what):
+    gbs = bytes_per_call / (ms * 1e-3) / 1e9
+    return {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gbs / hbm_peak, "traffic": None,
+            "peak_kind": f"of {peak_kind}", "what": what}
+
+
+def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, peak_kind, fraction=None, oracle=None):
+    """Workloads 1 - 5 and the variants, each timed on its own: best of a few launches, CUDA events;
+    each with the roofline of its call and, when `oracle` is given, the oracle's time beside it."""
     res = {}
     for k in which:
         if k in (1, 3, 4):
@@ -229,7 +298,15 @@ def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full, fraction
             res[f"C{k}"] = {"configs": n, "requests": tr.n, "feasible": feasible, "ms": best,
                             "configs_per_s": n / best * 1e3, "iters_per_s": iters / best * 1e3,
                             "request_iters_per_s": req_iters / best * 1e3, "request_iters": req_iters,
-                            "hardware_axis_fraction": scale, "kernel_launches": 1, **extra}
+                            "hardware_axis_fraction": scale, "workspace_bytes": ws.numel(),
+                            "kernels": "k_trace_lanes (max batch <= 16, one lane per config) + k_trace_sim (one warp per config)",
+                            "kernel_launches": 2,
+                            "roofline": alu_roofline(FP64_OPS_PER_ITERATION * iters / best * 1e3,
+                                                     f"{FP64_OPS_PER_ITERATION} fp64 operations per simulated iteration x iterations/s"),
+                            **extra}
+            if oracle is not None:
+                stride_all, stride_one = {1: (1, 7), 3: (509, 4093), 4: (2039, 16381)}[k]
+                res[f"C{k}"]["cpu_baseline"] = cpu_baseline_of(oracle, w["space"], w["trace"], n, stride_all, stride_one, True)
             del out, ws
         elif k in (2, 5):
             w = inputs.workload(k, scale=fraction if (fraction and k == 5) else 1.0)
@@ -237,22 +314,30 @@ def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full, fraction
             n = p.n
             fl = flush if k == 2 else None          # workload 2's outputs fit in L2: evict them
             t_sim = time_call(torch, p.simulate, flush=fl)[0]
+            fits = int((p.out["status"] == 0).sum().item())
             t_kf = time_call(torch, lambda: p.topk(True), flush=fl)[0]
             t_pf = time_call(torch, lambda: p.pareto(True), flush=fl)[0]
             t_km = time_call(torch, lambda: p.topk(False), flush=fl)[0]
             t_pm = time_call(torch, lambda: p.pareto(False), flush=fl)[0]
-            res[f"C{k}"] = {"configs": n, "front": int(p.fcnt.item()), "found": int(p.cnt.item()),
+            ops = FP64_OPS_PER_CLOSED_FORM_CONFIG * fits
+            what = f"{FP64_OPS_PER_CLOSED_FORM_CONFIG} fp64 operations per config that fits ({fits}) / call time"
+            res[f"C{k}"] = {"configs": n, "fits": fits, "front": int(p.fcnt.item()), "found": int(p.cnt.item()),
                             "fused_ms": {"topk": t_kf, "pareto": t_pf}, "fused_configs_per_s": n / (t_kf + t_pf) * 1e3,
                             "materialised_ms": {"simulate": t_sim, "topk": t_km, "pareto": t_pm},
                             "materialised_configs_per_s": n / (t_sim + t_km + t_pm) * 1e3,
                             "simulate_write_gbs": BYTES_SIM * n / t_sim / 1e6,
                             "simulate_frac_of_hbm": BYTES_SIM * n / t_sim / 1e6 / hbm_peak,
+                            "roofline": {"guide_simulate": hbm_roofline(BYTES_SIM * n, t_sim, hbm_peak, peak_kind, "53 B written per config"),
+                                         "guide_select_topk (fused)": alu_roofline(ops / t_kf * 1e3, what),
+                                         "guide_pareto (fused)": alu_roofline(ops / t_pf * 1e3, what)},
                             "kernel_launches": 2 + 6 + 5 + 5 + 4}
+            if oracle is not None:
+                stride_all, stride_one = (1, 16) if k == 2 else (8, 128)
+                res[f"C{k}"]["cpu_baseline"] = cpu_baseline_of(oracle, w["space"], None, n, stride_all, stride_one, False)
             del p
         elif k == 8:
             # workload 3 on half of its hardware axis with every framework on the split-and-fuse
             # policy (token budgets 256 .. 8192 per iteration)
-            import numpy as np
             w = inputs.workload(3, scale=fraction or 0.5, trace_scale=1.0)
             space = dict(w["space"])
             fw_i = np.array(space["fw_i"], dtype=np.uint32).copy()
@@ -269,11 +354,15 @@ def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full, fraction
             res["C3-split-fuse"] = {"configs": n, "requests": tr.n, "feasible": int((out["status"] == 0).sum().item()),
                                     "ms": best, "configs_per_s": n / best * 1e3, "iters_per_s": iters / best * 1e3,
                                     "request_iters_per_s": req_iters / best * 1e3,
-                                    "hardware_axis_fraction": fraction or 0.5, "kernel_launches": 1}
+                                    "hardware_axis_fraction": fraction or 0.5, "kernel_launches": 1,
+                                    "roofline": alu_roofline(FP64_OPS_PER_ITERATION * iters / best * 1e3,
+                                                             f"{FP64_OPS_PER_ITERATION} fp64 operations per simulated iteration x iterations/s")}
+            if oracle is not None:
+                res["C3-split-fuse"]["cpu_baseline"] = cpu_baseline_of(oracle, space, w["trace"], n, 509, 4093, True)
             del out, ws
         elif k in (6, 7):
             # the (dp, tp) sweep under a budget of 8 GPUs (whole-space kernels) and workload 2 with
-            # frameworks that process prompts in sub-batches / segments (one thread per config)
+            # frameworks that process prompts in sub-batches / segments
             w = inputs.hybrid_workload(8) if k == 6 else inputs.chunked_workload(scale=1.0)
             p = ClosedFormPath(guide, torch, w["space"], w["constraints"], w["topk"]["key"], w["topk"]["k"])
             n = p.n
@@ -282,7 +371,10 @@ def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, full, fraction
             res[w["name"]] = {"configs": n, "simulate_ms": t_sim, "simulate_configs_per_s": n / t_sim * 1e3,
                               "simulate_write_gbs": BYTES_SIM * n / t_sim / 1e6,
                               "simulate_frac_of_hbm": BYTES_SIM * n / t_sim / 1e6 / hbm_peak,
+                              "roofline": hbm_roofline(BYTES_SIM * n, t_sim, hbm_peak, peak_kind, "53 B written per config"),
                               "fused_topk_ms": t_kf, "found": int(p.cnt.item())}
+            if oracle is not None:
+                res[w["name"]]["cpu_baseline"] = cpu_baseline_of(oracle, w["space"], None, n, 4, 64, False)
             del p
         torch.cuda.empty_cache()
     return res
@@ -315,17 +407,23 @@ def run_ours(args):
     n_local = path.n
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")   # used for workload 2 only
 
+    select, front = sharding.kernel_selectors(guide, path.sp, key, "latency", "cost_per_hr")
+
     def exchange():
-        """all-gather of the k local candidates, then the same kernel merges them"""
+        """all-gather of every rank's k candidates and of its local front; the library's own selection
+        calls merge the gathered lists.  Leaves global config indices in path.idx / path.fidx."""
         gidx = sharding.local_to_global(path.idx, local_space, global_space, hw_off)
-        all_idx = sharding.all_gather_concat(gidx)
-        all_val = sharding.all_gather_concat(path.val)
-        order = sharding.order_for_merge(all_idx)
-        all_idx, all_val = all_idx[order], all_val[order]
-        m = all_idx.numel()
-        gathered = {"status": (all_idx < 0).to(torch.uint8), key: all_val.contiguous()}
-        guide.guide_select_topk(path.sp, None, gathered, {}, key, k, path.idx, path.val, path.cnt, path.ws_k, count=m)
-        return all_idx
+        top, vals, found = sharding.merge_topk(gidx, path.val, k, select)
+        size = int(path.fcnt.item())
+        used = torch.arange(guide.PARETO_MAX, device="cuda") < size
+        sel = torch.where(used, path.fidx, torch.zeros_like(path.fidx))
+        gfront = sharding.local_to_global(sel, local_space, global_space, hw_off)
+        fr, fsize = sharding.merge_front(gfront, path.out["latency"][sel], path.out["cost_per_hr"][sel], size,
+                                         guide.PARETO_MAX, front)
+        path.idx.copy_(top)
+        path.val.copy_(vals)
+        path.fidx[:fr.numel()].copy_(fr)
+        return found, fsize
 
     # The two selections of a step read the same metrics and share nothing else: the Pareto front
     # (the longer chain of kernels) runs on the step's stream, top-k beside it on a second one (both
@@ -463,7 +561,7 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the dominant kernel of the step ----
+    # ---- roofline of every call of the step, the dominant one on top ----
     # bytes a scan must read per config: status, each distinct metric array, each bounded array
     bounded = {"max_latency": "latency", "max_cost_per_hr": "cost_per_hr", "min_throughput": "thr_decode",
                "max_ttft": "ttft"}
@@ -473,35 +571,42 @@ def run_ours(args):
     per = {"guide_simulate (k_closed_form_memory + k_closed_form_lines)": (t_sim / args.steps, BYTES_SIM),
            "guide_select_topk (k_topk_bound + k_topk_filter + k_topk_rank)": (t_topk / args.steps, bytes_topk),
            "guide_pareto (k_pareto_sample + k_pareto_filter + k_pareto_rank)": (t_par / args.steps, bytes_pareto)}
+    calls = {}
+    for name, (ms, nbytes) in per.items():
+        calls[name] = hbm_roofline(nbytes * n_local, ms, hbm_peak, peak_kind, f"{nbytes} algorithmic bytes per config")
+        calls[name]["ms"] = ms
+    traffic = recorded_traffic(n_local)
     dom = max(per, key=lambda name: per[name][0])
-    dom_ms, dom_bytes = per[dom]
-    achieved = dom_bytes * n_local / (dom_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
-                "frac": achieved / hbm_peak,
-                "traffic": K1_TRAFFIC_C5 if (dom.startswith("guide_simulate") and n_local == 16777216) else None,
-                "peak_kind": f"of {peak_kind}",
-                "bytes_per_config": dom_bytes,
-                "per_call_frac_of_hbm": {name: v[1] * n_local / (v[0] * 1e-3) / 1e9 / hbm_peak for name, v in per.items()},
-                "per_kernel_ms": {name: v[0] for name, v in per.items()},
-                "per_kernel_gbs": {name: v[1] * n_local / (v[0] * 1e-3) / 1e9 for name, v in per.items()}}
+    roofline = dict(calls[dom])
+    roofline.update({"kernel": dom, "bytes_per_config": per[dom][1],
+                     "traffic": traffic if dom.startswith("guide_simulate") else None,
+                     "calls": calls,
+                     "per_call_frac_of_hbm": {name: c["frac"] for name, c in calls.items()},
+                     "per_kernel_ms": {name: c["ms"] for name, c in calls.items()}})
 
-    # ---- the oracle on the host cores, same workload ----
+    # ---- the oracle on the host cores, same workload: whole passes for about ten seconds, then one core
+    # on a sixteenth of the configs ----
     cpu = None
+    oracle = None
     if world == 1 and not args.no_cpu:
         import oracle
+        cores = host_cores(oracle)
         oracle_step(oracle, w)
         reps, t0 = 0, time.perf_counter()
         while reps < 3 or time.perf_counter() - t0 < 10.0:
             oracle_step(oracle, w)
             reps += 1
         dt = time.perf_counter() - t0
-        cpu = {"value": n_local * reps / dt, "unit": "configs/s", "cores": oracle.threads(), "kind": "oracle",
-               "sample": f"the whole {n_local}-config workload (simulate + top-{k} + Pareto), {reps} passes"}
+        one = oracle_seconds(oracle, w["space"], None, 16, n_local, 1)
+        cpu = {"value": n_local * reps / dt, "unit": "configs/s", "cores": cores, "kind": "oracle",
+               "sample": f"the whole {n_local}-config workload (simulate + top-{k} + Pareto), {reps} passes",
+               "seconds_per_pass": dt / reps,
+               "one_core": {"configs_per_s": one[1] / one[0], "sample": "every 16th config, simulate only", "seconds": one[0]}}
 
     extras = {}
     if world == 1 and args.extras:
         which = [int(x) for x in args.extras.split(",") if x]
-        extras = extra_workloads(guide, torch, inputs, which, flush, hbm_peak, args.full, args.trace_fraction)
+        extras = extra_workloads(guide, torch, inputs, which, flush, hbm_peak, peak_kind, args.trace_fraction, oracle)
 
     # simulate: memory + model kernel; top-k: bound, filter, rank and the two gated fallback kernels
     # (scan, merge: they return at once); Pareto: sample, filter, rank and the gated general kernel;
@@ -520,8 +625,10 @@ def run_ours(args):
             "ms_per_step_calls_in_turn": t_turn,
             "clocks": sampler.summary(),
             "e2e": {"value": e2e_value, "unit": "configs/s", "h2d_bytes_per_step": table_bytes(local_space),
-                    "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-            "e2e_selection_only": e2e_sel,
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                    "what": "space handle built from host tables, simulate + top-k + Pareto, every metric array (0.89 GB), "
+                            "the candidates and the front copied to pinned host memory: bound by the copy back",
+                    "variants": {"selection_only": e2e_sel}},
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "workloads": extras,
             "wall_s_timed_region": wall}
@@ -539,7 +646,6 @@ def main():
     ap.add_argument("--extras", default="1,2,3,4,5,6,7,8", help="other workloads to time after the main loop ('' = none)")
     ap.add_argument("--main-fraction", action="store_true",
                     help="apply --trace-fraction to the main workload's hardware axis too (small cases for profiler captures)")
-    ap.add_argument("--full", action="store_true", help="(kept for compatibility: workloads 3 and 4 now always run whole)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
     ap.add_argument("--trace-fraction", type=float, default=None,
                     help="fraction of the hardware axis of workloads 3, 4 and 5 in the extras (small cases for profiler captures)")

@@ -18,7 +18,7 @@
  *   - Kernel launches are asynchronous on the given CUDA stream (a cudaStream_t passed as
  *     void*; NULL is the default stream).  Results are valid once that stream has been
  *     synchronised.  The one exception is the first use of a handle on a device, which uploads
- *     its tables with a synchronous copy.
+ *     its tables on the given stream and waits for that stream (no other stream is touched).
  *   - A config index enumerates the axes in mixed radix, length pair fastest, model slowest:
  *       idx = ((((m*n_hw + h)*n_fw + f)*n_batch + b)*n_tp + t)*n_pairs + l
  *   - All floating point is IEEE binary64, round to nearest even, no fused multiply-add, in a
@@ -248,8 +248,8 @@ int guide_select_topk(const guide_space *space, const guide_trace *trace, const 
 /* Constraint filter + 2-D Pareto front, both metrics minimised (throughput by its negation):
  * passing configs not dominated by another passing config; of several configs with equal (x, y)
  * the lowest index stays.  Written in ascending x.  The paper has no Pareto step; it is the
- * two-objective form of its "lowest time and highest throughput under a budget" selection
- * (Sec. 3.2, Sec. 4.1).  idx_out_dev[cap], count_out_dev[1]: device.  count is the full size of
+ * two-objective form of its selection of the fastest and the highest-throughput deployment that a
+ * budget allows (Sec. 3.2, Sec. 4.1).  idx_out_dev[cap], count_out_dev[1]: device.  count is the full size of
  * the front even when cap is smaller; a front above GUIDE_PARETO_MAX points sets count to
  * UINT32_MAX.  outputs / opts / trace as for guide_select_topk. */
 int guide_pareto(const guide_space *space, const guide_trace *trace, const guide_outputs *outputs,

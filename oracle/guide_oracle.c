@@ -259,7 +259,8 @@ static void closed_form_one(const ospace *s, u64 idx, u64 j, int time_model, int
     u64 kv_block = s->fw_i[4 * p.f + 1], reserve = s->fw_i[4 * p.f + 2];
     /* Hybrid parallelism (Sec. 3.5.2, Sec. 3.5.3): the batch is split over dp replicas of t GPUs each;
      * a stage lasts as long as its slowest replica, the one with ceil(b / dp) requests.  The memory
-     * bound is per replica: "Max Batch Size = Maximum Parallelism / Data Parallelism" (Sec. 3.2 Step 1). */
+     * bound is per replica: Sec. 3.2 Step 1 obtains the largest batch by dividing the largest number of
+     * requests in flight by the data-parallel degree. */
     u64 dp = s->dp ? s->dp[p.t] : 1;
     u64 b = ceil_div(b_all, dp);
 
@@ -278,7 +279,7 @@ static void closed_form_one(const ospace *s, u64 idx, u64 j, int time_model, int
     if (st) { write_infeasible(o, j); return; }
 
     /* Step 2: the two stages.  Prompt processing (Sec. 3.3.1): the batch goes through in sub-batches
-     * of split_size requests, "any remaining portion of the batch forming an additional sub-batch";
+     * of split_size requests and what is left over goes through as one more, smaller sub-batch;
      * equal sub-batches take equal time.  Without splitting this is one pass over b x Lin tokens. */
     u64 split = s->fw_chunk ? s->fw_chunk[2 * p.f] : 0, seg = s->fw_chunk ? s->fw_chunk[2 * p.f + 1] : 0;
     if (split == 0 || split > b) split = b;

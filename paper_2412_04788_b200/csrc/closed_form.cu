@@ -323,12 +323,13 @@ static int launch_split(const DSpace &s, int tp_model, const guide_outputs &o, c
     const u32 items = s.n_m * tiles * n_hf;
     const u32 mem_grid = std::min<u32>(items, (u32)num_sms() * MEM_BLOCKS_PER_SM);
     const bool lines = lines_apply(s, o);
+    const u32 n_chunks = lines ? (n_hf + LINE_CHUNK - 1) / LINE_CHUNK : (n_hf + MODEL_CHUNK - 1) / MODEL_CHUNK;
+    // refuse before anything is queued: a failed call leaves the caller's arrays untouched
+    if ((u64)s.n_m * s.n_b * (n_tl / 4) * n_chunks > 0x7FFFFFFFull) return fail(GUIDE_ERR_UNSUPPORTED, "space too large for one launch");
     GUIDE_CUDA(cudaMemsetAsync(ticket, 0, 4, st));           // the model kernel's work counter
     if (lines) k_closed_form_memory<1><<<mem_grid, MEM_THREADS, 0, st>>>(s, o, co, tiles);
     else k_closed_form_memory<0><<<mem_grid, MEM_THREADS, 0, st>>>(s, o, co, tiles);
     GUIDE_CUDA(cudaGetLastError());
-    const u32 n_chunks = lines ? (n_hf + LINE_CHUNK - 1) / LINE_CHUNK : (n_hf + MODEL_CHUNK - 1) / MODEL_CHUNK;
-    if ((u64)s.n_m * s.n_b * (n_tl / 4) * n_chunks > 0x7FFFFFFFull) return fail(GUIDE_ERR_UNSUPPORTED, "space too large for one launch");
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(MODEL_THREADS); cfg.stream = st;
     cudaLaunchAttribute at[1];
@@ -338,8 +339,10 @@ static int launch_split(const DSpace &s, int tp_model, const guide_outputs &o, c
     if (lines) {
         // function attributes belong to the device: set them once per device and kernel variant
         static bool opted_in[64][2] = {};
+        static std::mutex opt_mu;
         int dev = 0;
         GUIDE_CUDA(cudaGetDevice(&dev));
+        std::lock_guard<std::mutex> opt_lock(opt_mu);
         if (dev < 0 || dev >= 64 || !opted_in[dev][TIME_SUM]) {
             // more dynamic shared memory than the default limit
             GUIDE_CUDA(cudaFuncSetAttribute(k_closed_form_lines<TIME_SUM>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -210,15 +210,29 @@ static std::vector<u32> plane_orders(const guide_space &s, size_t group) {
     return out;
 }
 
-int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
+// One work-counter slot per stream that has used the handle on this device: calls on one stream are
+// ordered, so they can share a slot; calls on different streams never do.  When more streams than
+// slots turn up, everything in flight on the device is waited for and the slots are handed out anew.
+static int ticket_for(DeviceTables &d, cudaStream_t st, unsigned **ticket) {
+    for (size_t i = 0; i < d.ticket_streams.size(); i++)
+        if (d.ticket_streams[i] == (void *)st) { *ticket = d.tickets + 32 * i; return GUIDE_OK; }
+    if (d.ticket_streams.size() == TICKET_SLOTS) {
+        GUIDE_CUDA(cudaDeviceSynchronize());
+        d.ticket_streams.clear();
+    }
+    d.ticket_streams.push_back((void *)st);
+    *ticket = d.tickets + 32 * (d.ticket_streams.size() - 1);
+    return GUIDE_OK;
+}
+
+int space_on_device(guide_space *s, DSpace *out, unsigned **ticket, cudaStream_t st) {
     int dev = 0;
     GUIDE_CUDA(cudaGetDevice(&dev));
     std::lock_guard<std::mutex> lock(s->mu);
     for (DeviceTables &d : s->dev)
         if (d.device == dev) {
             *out = d.view;
-            if (ticket) *ticket = d.tickets + 32 * (d.next_ticket++ % TICKET_SLOTS);
-            return GUIDE_OK;
+            return ticket ? ticket_for(d, st, ticket) : GUIDE_OK;
         }
 
     const size_t n_m = s->models.size(), n_h = s->hw.size(), n_f = s->fw.size();
@@ -238,7 +252,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
     GUIDE_CUDA(cudaMalloc(&blob, off));
     cudaError_t e = cudaSuccess;
     auto put = [&](size_t o, const void *src, size_t bytes) {
-        if (e == cudaSuccess) e = cudaMemcpy(blob + o, src, bytes, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(blob + o, src, bytes, cudaMemcpyHostToDevice, st);
     };
     put(o_gm, s->models.data(), n_m * sizeof(guide_model));
     put(o_gh, s->hw.data(), n_h * sizeof(guide_hw));
@@ -254,7 +268,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
     put(o_lo, line_order.data(), line_order.size() * 4);
     if (e == cudaSuccess) {
         const u32 n = (u32)std::max(n_m, n_h * n_f);
-        k_build_tables<<<(n + 127) / 128, 128>>>((const guide_model *)(blob + o_gm), (u32)n_m,
+        k_build_tables<<<(n + 127) / 128, 128, 0, st>>>((const guide_model *)(blob + o_gm), (u32)n_m,
                                                  (const guide_hw *)(blob + o_gh), (u32)n_h,
                                                  (const guide_fw *)(blob + o_gf), (u32)n_f,
                                                  (const u32 *)(blob + o_t), (const u32 *)(blob + o_d), (u32)s->tp.size(),
@@ -263,7 +277,8 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
                                                  (ulonglong2 *)(blob + o_hm), (double *)(blob + o_r10),
                                                  (StageConst *)(blob + o_sc));
         e = cudaGetLastError();
-        if (e == cudaSuccess) e = cudaStreamSynchronize(0);
+        // the host arrays must outlive the copies, and another stream may use the tables next
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     }
     if (e != cudaSuccess) { cudaFree(blob); return cuda_fail(e, "uploading the space tables"); }
     DeviceTables d;
@@ -287,13 +302,12 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket) {
     d.view.n_m = (u32)n_m; d.view.n_h = (u32)n_h; d.view.n_f = (u32)n_f;
     d.view.n_b = (u32)s->batch.size(); d.view.n_t = (u32)s->tp.size(); d.view.n_l = (u32)s->pairs.size();
     d.tickets = (unsigned *)(blob + o_tk);
-    if (ticket) *ticket = d.tickets + 32 * (d.next_ticket++ % TICKET_SLOTS);
     s->dev.push_back(d);
     *out = d.view;
-    return GUIDE_OK;
+    return ticket ? ticket_for(s->dev.back(), st, ticket) : GUIDE_OK;
 }
 
-int trace_on_device(guide_trace *t, DTrace *out) {
+int trace_on_device(guide_trace *t, DTrace *out, cudaStream_t st) {
     int dev = 0;
     GUIDE_CUDA(cudaGetDevice(&dev));
     std::lock_guard<std::mutex> lock(t->mu);
@@ -303,9 +317,10 @@ int trace_on_device(guide_trace *t, DTrace *out) {
     const size_t o_a = 0, o_i = align_up(n * 8, 256), o_o = o_i + align_up(n * 4, 256), total = o_o + align_up(n * 4, 256);
     char *blob = nullptr;
     GUIDE_CUDA(cudaMalloc(&blob, total));
-    cudaError_t e = cudaMemcpy(blob + o_a, t->arrival.data(), n * 8, cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaMemcpy(blob + o_i, t->in_len.data(), n * 4, cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaMemcpy(blob + o_o, t->out_len.data(), n * 4, cudaMemcpyHostToDevice);
+    cudaError_t e = cudaMemcpyAsync(blob + o_a, t->arrival.data(), n * 8, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(blob + o_i, t->in_len.data(), n * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(blob + o_o, t->out_len.data(), n * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);      // the copies are done before another stream can use the trace
     if (e != cudaSuccess) { cudaFree(blob); return cuda_fail(e, "uploading the trace"); }
     DeviceTrace d;
     d.device = dev;
@@ -588,10 +603,10 @@ int guide_simulate(const guide_space *space_c, const guide_trace *trace_c, const
     if (r.count == 0) return GUIDE_OK;
     DSpace ds;
     unsigned *ticket = nullptr;
-    if ((rc = space_on_device(space, &ds, &ticket))) return rc;
+    if ((rc = space_on_device(space, &ds, &ticket, (cudaStream_t)stream))) return rc;
     if (!trace) return launch_closed_form(ds, r, time_model, tp_model, *out, ticket, (cudaStream_t)stream);
     DTrace dt;
-    if ((rc = trace_on_device(trace, &dt))) return rc;
+    if ((rc = trace_on_device(trace, &dt, (cudaStream_t)stream))) return rc;
     u32 policies = 0;
     for (const guide_fw &f : space->fw) policies |= f.policy == GUIDE_POLICY_SPLIT_FUSE ? 2u : 1u;
     return launch_trace_sim(ds, dt, r, time_model, tp_model, opts ? opts->max_iters : 0, *out, ws, ws_bytes,
@@ -617,7 +632,7 @@ int guide_select_topk(const guide_space *space_c, const guide_trace *trace, cons
     if ((rc = check_workspace(ws, ws_bytes, topk_workspace_bytes(k)))) return rc;
     DSpace ds;
     unsigned *ticket = nullptr;                  // the fused path's model walk takes its work items through it
-    if ((rc = space_on_device(space, &ds, outputs ? nullptr : &ticket))) return rc;
+    if ((rc = space_on_device(space, &ds, outputs ? nullptr : &ticket, (cudaStream_t)stream))) return rc;
     return launch_topk(ds, r, outputs, opts ? opts->time_model : 0, opts ? opts->tp_model : 0, *cons, key, k,
                        (u64 *)idx_out, key_out, count_out, ws, ticket, (cudaStream_t)stream);
 }
@@ -635,7 +650,7 @@ int guide_pareto(const guide_space *space_c, const guide_trace *trace, const gui
     if ((rc = check_workspace(ws, ws_bytes, pareto_workspace_bytes()))) return rc;
     DSpace ds;
     unsigned *ticket = nullptr;
-    if ((rc = space_on_device(space, &ds, outputs ? nullptr : &ticket))) return rc;
+    if ((rc = space_on_device(space, &ds, outputs ? nullptr : &ticket, (cudaStream_t)stream))) return rc;
     return launch_pareto(ds, r, outputs, opts ? opts->time_model : 0, opts ? opts->tp_model : 0, *cons, xm, ym,
                          (u64 *)idx_out, cap, count_out, ws, ticket, (cudaStream_t)stream);
 }

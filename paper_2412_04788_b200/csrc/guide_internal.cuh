@@ -21,8 +21,8 @@ int cuda_fail(cudaError_t e, const char *what);
         if (e__ != cudaSuccess) return guide::cuda_fail(e__, #call); \
     } while (0)
 
-// Work counters of the persistent closed-form model kernel: one 128-byte slot per call in flight,
-// handed out in turn, so that calls on different streams do not share one.
+// Work counters of the persistent closed-form model kernel: one 128-byte slot per stream that uses
+// the handle, so that calls on different streams never share one.
 static constexpr unsigned TICKET_SLOTS = 64;
 
 struct DeviceTables {
@@ -30,7 +30,7 @@ struct DeviceTables {
     void *blob = nullptr;
     DSpace view{};
     unsigned *tickets = nullptr;     // TICKET_SLOTS slots, 32 words apart
-    unsigned next_ticket = 0;
+    std::vector<void *> ticket_streams;   // slot i belongs to the calls on ticket_streams[i]
 };
 
 struct DeviceTrace {
@@ -65,8 +65,8 @@ struct guide_trace {
 namespace guide {
 
 // device views for the current device (uploads on first use)
-int space_on_device(guide_space *s, DSpace *out, unsigned **ticket = nullptr);
-int trace_on_device(guide_trace *t, DTrace *out);
+int space_on_device(guide_space *s, DSpace *out, unsigned **ticket, cudaStream_t st);
+int trace_on_device(guide_trace *t, DTrace *out, cudaStream_t st);
 
 // closed_form.cu
 int launch_closed_form(const DSpace &s, Range r, int time_model, int tp_model, const guide_outputs &o,

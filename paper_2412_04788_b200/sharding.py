@@ -1,9 +1,12 @@
 """Multi-GPU plumbing: configs are independent, so the space is cut along the hardware axis, each
 rank evaluates its slice with the single-GPU kernels, and the only exchange is an all-gather of
-each rank's k best candidates (and its local front) before a final merge with the same kernels.
+each rank's k best candidates and of its local front before a final merge with the same selection
+calls (guide_select_topk / guide_pareto over the gathered lists).
 
 Everything here is index arithmetic and torch.distributed calls; it runs unchanged on gloo/CPU
-tensors (used by the tests) and on nccl/CUDA tensors.
+tensors (used by the tests) and on nccl/CUDA tensors.  The two `merge_*` functions take the
+selection call as an argument: the library's binding on a GPU, and whatever stands in for it in a
+CPU test of the plumbing.
 """
 from __future__ import annotations
 
@@ -69,3 +72,83 @@ def order_for_merge(global_idx):
     import torch
     key = torch.where(global_idx < 0, torch.full_like(global_idx, torch.iinfo(torch.int64).max), global_idx)
     return torch.argsort(key, stable=True)
+
+
+def concat_gather(parts):
+    """Stand-in for all_gather_concat when the shards live in one process: `parts` holds every
+    shard's tensor in rank order."""
+    import torch
+    return torch.cat(list(parts))
+
+
+def merge_topk(gidx, val, k, select, gather=all_gather_concat):
+    """Global top-k from every shard's k candidates.
+
+    gidx: this shard's candidates as *global* config indices (int64, -1 = unused slot); val: their
+    key values.  The gathered lists are put in global-index order, so that the selection call's
+    lowest-position tie-break is the single-space lowest-index tie-break.  `select(status, values,
+    k)` runs the top-k selection over the gathered list (status 0 = candidate, 1 = unused slot) and
+    returns (positions int64[k] with -1 for unused, values[k], count).  Returns (global indices
+    int64[k], values[k], count)."""
+    import torch
+    all_idx, all_val = gather(gidx), gather(val)
+    order = order_for_merge(all_idx)
+    all_idx, all_val = all_idx[order], all_val[order].contiguous()
+    status = (all_idx < 0).to(torch.uint8)
+    pos, vals, count = select(status, all_val, k)
+    found = pos >= 0
+    out = torch.full_like(pos, -1)
+    out[found] = all_idx[pos[found]]                 # positions in the gathered list -> config indices
+    return out, vals, count
+
+
+def merge_front(gidx, x, y, count, cap, front, gather=all_gather_concat):
+    """Global Pareto front from every shard's local front (a point no shard's point dominates is on
+    its own shard's front, so the union of the local fronts contains the global one).
+
+    gidx / x / y: this shard's front as global config indices and the two metric values, padded to
+    `cap` entries; count: how many are real.  `front(status, xs, ys, cap)` runs the front selection
+    over the gathered points and returns (positions int64[<=cap] in ascending x, size).  Returns
+    (global indices of the front in ascending x, size)."""
+    import torch
+    used = torch.arange(gidx.numel(), device=gidx.device) < count
+    gidx = torch.where(used, gidx, torch.full_like(gidx, -1))
+    all_idx, all_x, all_y = gather(gidx), gather(x), gather(y)
+    order = order_for_merge(all_idx)
+    all_idx, all_x, all_y = all_idx[order], all_x[order].contiguous(), all_y[order].contiguous()
+    status = (all_idx < 0).to(torch.uint8)
+    pos, size = front(status, all_x, all_y, cap)
+    return all_idx[pos], size
+
+
+_ARRAY_OF = {"throughput": "thr_decode"}          # metric name -> name of the guide_outputs array that holds it
+
+
+def kernel_selectors(guide, sp, key, x="latency", y="cost_per_hr"):
+    """The merge steps through the library: (select, front) callables for merge_topk / merge_front that
+    run guide_select_topk / guide_pareto over the gathered lists (CUDA tensors), with the gathered
+    values standing in as the metric arrays of the call.  `sp` is any guide.Space handle at least as
+    large as the gathered lists (the calls only use it to check the range)."""
+    import torch
+
+    def select(status, values, k):
+        m = status.numel()
+        out = {"status": status, _ARRAY_OF.get(key, key): values}
+        idx = torch.empty(k, dtype=torch.int64, device=values.device)
+        val = torch.empty(k, dtype=torch.float64, device=values.device)
+        cnt = torch.zeros(1, dtype=torch.int32, device=values.device)
+        ws = torch.empty(guide.guide_select_workspace_bytes(sp, k), dtype=torch.uint8, device=values.device)
+        guide.guide_select_topk(sp, None, out, {}, key, k, idx, val, cnt, ws, count=m)
+        return idx, val, int(cnt.item())           # unused slots come back as 2^64 - 1 = -1
+
+    def front(status, xs, ys, cap):
+        m = status.numel()
+        out = {"status": status, _ARRAY_OF.get(x, x): xs, _ARRAY_OF.get(y, y): ys}
+        idx = torch.empty(cap, dtype=torch.int64, device=xs.device)
+        cnt = torch.zeros(1, dtype=torch.int32, device=xs.device)
+        ws = torch.empty(guide.guide_pareto_workspace_bytes(sp), dtype=torch.uint8, device=xs.device)
+        guide.guide_pareto(sp, None, out, {}, x, y, idx, cnt, ws, count=m)
+        size = int(cnt.item())
+        return idx[:min(size, cap)], size
+
+    return select, front
