@@ -41,7 +41,7 @@ class _Space(C.Structure):
                 ("batch", C.c_void_p), ("n_b", C.c_uint32),
                 ("tp", C.c_void_p), ("n_t", C.c_uint32),
                 ("pairs", C.c_void_p), ("n_l", C.c_uint32),
-                ("dp", C.c_void_p), ("fw_chunk", C.c_void_p)]
+                ("dp", C.c_void_p), ("fw_chunk", C.c_void_p), ("fw_keep", C.c_void_p)]
 
 
 class _Trace(C.Structure):
@@ -51,7 +51,7 @@ class _Trace(C.Structure):
 class _Out(C.Structure):
     _fields_ = [(k, C.c_void_p) for k in F64_FIELDS] + [
         ("status", C.c_void_p), ("bmax", C.c_void_p), ("n_iters", C.c_void_p), ("n_req_iters", C.c_void_p),
-        ("req_ttft", C.c_void_p), ("req_tpot", C.c_void_p), ("n_preempt", C.c_void_p)]
+        ("req_ttft", C.c_void_p), ("req_tpot", C.c_void_p), ("n_preempt", C.c_void_p), ("seq_used", C.c_void_p)]
 
 
 class _Cons(C.Structure):
@@ -72,7 +72,7 @@ def lib():
         _lib = C.CDLL(build())
         _lib.oracle_simulate.restype = C.c_int
         _lib.oracle_simulate.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint64,
-                                         C.c_int, C.c_int, C.c_uint64, C.c_void_p, C.c_int]
+                                         C.c_int, C.c_int, C.c_uint64, C.c_void_p, C.c_int, C.c_int]
         _lib.oracle_threads.restype = C.c_int
         for name in ("oracle_weight_params",):
             getattr(_lib, name).restype = C.c_uint64
@@ -106,11 +106,12 @@ def _space_struct(space):
                   _p(space["fw_f"]), _p(space["fw_i"]), len(space["fw_f"]), _p(space["batch"]), len(space["batch"]),
                   _p(space["tp"]), len(space["tp"]), _p(space["pairs"]), len(space["pairs"]),
                   _p(space["dp"]) if space.get("dp") is not None else None,
-                  _p(space["fw_chunk"]) if space.get("fw_chunk") is not None else None)
+                  _p(space["fw_chunk"]) if space.get("fw_chunk") is not None else None,
+                  _p(space["fw_keep"]) if space.get("fw_keep") is not None else None)
 
 
 def simulate(space, trace=None, first=0, count=None, stride=1, time_model=TIME_MAX, tp_model=TP_EXPLICIT,
-             max_iters=0, per_request=False, n_threads=0):
+             max_iters=0, per_request=False, n_threads=0, clamp_seq=False):
     """Evaluate configs first, first+stride, ...; returns a dict of numpy arrays (one slot per config)."""
     n_total = 1
     for k in ("models", "hw", "fw_f", "batch", "tp", "pairs"):
@@ -124,6 +125,7 @@ def simulate(space, trace=None, first=0, count=None, stride=1, time_model=TIME_M
     out["n_iters"] = np.empty(count, dtype=np.uint64)
     out["n_req_iters"] = np.empty(count, dtype=np.uint64)
     out["n_preempt"] = np.zeros(count, dtype=np.uint64)
+    out["seq_used"] = np.zeros(count, dtype=np.uint32)
     ts = None
     if trace is not None:
         n_req = len(trace["arrival"])
@@ -134,12 +136,12 @@ def simulate(space, trace=None, first=0, count=None, stride=1, time_model=TIME_M
     o = _Out(*[_p(out[k]) for k in F64_FIELDS], _p(out["status"]), _p(out["bmax"]), _p(out["n_iters"]),
              _p(out["n_req_iters"]),
              _p(out["req_ttft"]) if "req_ttft" in out else None,
-             _p(out["req_tpot"]) if "req_tpot" in out else None, _p(out["n_preempt"]))
+             _p(out["req_tpot"]) if "req_tpot" in out else None, _p(out["n_preempt"]), _p(out["seq_used"]))
     sp = _space_struct(space)
     rc = lib().oracle_simulate(C.byref(sp), C.byref(ts) if ts is not None else None, first, count, stride,
-                               time_model, tp_model, max_iters, C.byref(o), n_threads)
+                               time_model, tp_model, max_iters, C.byref(o), n_threads, int(bool(clamp_seq)))
     if rc != 0:
-        why = {-1: "invalid input", -2: "64-bit overflow", -3: "data parallelism or prompt splitting with a trace is not modelled"}.get(rc, "?")
+        why = {-1: "invalid input", -2: "64-bit overflow", -3: "data parallelism, prompt splitting, cache eviction or sequence clamping with a trace is not modelled"}.get(rc, "?")
         raise ValueError(f"oracle_simulate failed: {rc} ({why})")
     return out
 

@@ -60,6 +60,8 @@ typedef struct {
     const u32 *dp;                         /* [n_t] data-parallel degree of each entry of the parallelism axis; NULL = all 1 */
     const u32 *fw_chunk;                   /* [n_f][2]: split_size (requests per prompt sub-batch), seg_tokens (prompt
                                               segment length); 0 = no splitting; NULL = none anywhere */
+    const u32 *fw_keep;                    /* [n_f]: thousandths of the KV cache that the framework's cache-eviction policy
+                                              keeps (H2O, Sec. 3.2 Step 1 / Sec. 3.3); 0 or 1000 = everything; NULL = all 1000 */
 } ospace;
 
 typedef struct {
@@ -71,6 +73,8 @@ typedef struct {
     uint8_t *status; u32 *bmax; u64 *n_iters, *n_req_iters;
     double *req_ttft, *req_tpot;           /* optional [count][n_req] */
     u64 *n_preempt;                        /* optional: preemptions per config (diagnostic) */
+    u32 *seq_used;                         /* optional: tokens per request the metrics were computed for (Lin + Lout, less
+                                              when the sequence was cut to fit, Sec. 3.3.2); 0 for configs that do not fit */
 } oout;
 
 enum { POLICY_PREFILL_FIRST = 0, POLICY_SPLIT_FUSE = 1 };
@@ -251,12 +255,18 @@ static double segmented_prefill(const model_t *m, const rates_t *r, u64 t, u64 s
     return sum;
 }
 
-static void closed_form_one(const ospace *s, u64 idx, u64 j, int time_model, int tp_model, const oout *o) {
+/* Tokens of a cache of c tokens that stay when the eviction policy keeps p thousandths of it (H2O, named
+ * in Sec. 3.2 Step 1 and Sec. 3.3 among the optimisations that shrink the KV cache; the paper gives
+ * no rule, so: the kept share of the length, rounded up to a whole token). */
+static u64 kept_tokens(u64 c, u64 p) { return p >= 1000 ? c : ceil_div(mul(p, c), 1000); }
+
+static void closed_form_one(const ospace *s, u64 idx, u64 j, int time_model, int tp_model, int clamp_seq, const oout *o) {
     pos_t p = decode(s, idx);
     model_t m = load_model(s->models + 10 * p.m);
     rates_t r = load_rates(s->hw + 5 * p.h, s->fw_f + 8 * p.f, s->fw_i + 4 * p.f);
     u64 t = s->tp[p.t], b_all = s->batch[p.b], Lin = s->pairs[2 * p.l], Lout = s->pairs[2 * p.l + 1];
     u64 kv_block = s->fw_i[4 * p.f + 1], reserve = s->fw_i[4 * p.f + 2];
+    u64 keep = s->fw_keep && s->fw_keep[p.f] ? s->fw_keep[p.f] : 1000;
     /* Hybrid parallelism (Sec. 3.5.2, Sec. 3.5.3): the batch is split over dp replicas of t GPUs each;
      * a stage lasts as long as its slowest replica, the one with ceil(b / dp) requests.  The memory
      * bound is per replica: Sec. 3.2 Step 1 obtains the largest batch by dividing the largest number of
@@ -268,7 +278,18 @@ static void closed_form_one(const ospace *s, u64 idx, u64 j, int time_model, int
     u64 usable = usable_bytes(s->hw_mem[p.h], reserve);
     u64 W_gpu = weight_bytes_per_gpu(&m, t);
     u64 kv_tok = kv_bytes_per_token(&m, t);
-    u64 S_blk = mul(ceil_div(Lin + Lout, kv_block), kv_block);   /* fixed-granularity allocation */
+    u64 S = Lin + Lout;
+    if (clamp_seq && usable > W_gpu) {
+        /* Dynamic sequence length adjustment (Sec. 3.3.2): S_max = floor(C_available / KV bytes of one
+         * token of all B requests); a longer sequence is cut to it.  Whole blocks only; with a cache that
+         * keeps p thousandths, the longest sequence whose kept part fits.  The prompt is what gets cut:
+         * every output token is still generated. */
+        u64 cap_tok = (usable - W_gpu) / mul(kv_tok, b);
+        u64 cap_blk = (cap_tok / kv_block) * kv_block;
+        u64 S_max = keep >= 1000 ? cap_blk : mul(1000, cap_blk) / keep;
+        if (S > S_max && S_max > Lout) { Lin = S_max - Lout; S = S_max; }
+    }
+    u64 S_blk = mul(ceil_div(kept_tokens(S, keep), kv_block), kv_block);   /* fixed-granularity allocation of what is kept */
     u64 bmax = usable > W_gpu ? (usable - W_gpu) / mul(S_blk, kv_tok) : 0;
     uint8_t st = 0;
     if (usable <= W_gpu) st |= ST_WEIGHTS;
@@ -276,6 +297,7 @@ static void closed_form_one(const ospace *s, u64 idx, u64 j, int time_model, int
     if (m.nh % t != 0 || m.nkv % t != 0) st |= ST_HEADS;
     o->status[j] = st;
     o->bmax[j] = bmax > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)bmax;
+    if (o->seq_used) o->seq_used[j] = st ? 0 : (u32)S;
     if (st) { write_infeasible(o, j); return; }
 
     /* Step 2: the two stages.  Prompt processing (Sec. 3.3.1): the batch goes through in sub-batches
@@ -291,6 +313,7 @@ static void closed_form_one(const ospace *s, u64 idx, u64 j, int time_model, int
     double T_dec = 0.0;
     if (n > 0) {
         u64 ctx = mul(b, add(mul(n, Lin), mul(n, n + 1) / 2));   /* step j attends Lin + j */
+        ctx = kept_tokens(ctx, keep);                            /* ... of which the cache still holds this many: less work, less KV read */
         T_dec = phase_time(&m, &r, t, mul(b, n), mul(b, n), ctx, ctx, n, time_model, tp_model, NULL);
     }
     o->ttft[j] = T_pre; o->ttft_p50[j] = T_pre; o->ttft_p99[j] = T_pre;
@@ -542,11 +565,13 @@ advance:
     o->cost_per_token[j] = o->thr_decode[j] > 0.0 ? (o->cost_per_hr[j] / 3600.0) / o->thr_decode[j] : INFINITY;
     o->n_iters[j] = n_iters; o->n_req_iters[j] = n_req_iters;
     if (o->n_preempt) o->n_preempt[j] = n_preempt;
+    if (o->seq_used) o->seq_used[j] = 0;                 /* closed form only */
     return;
 
 infeasible:
     o->status[j] = st;
     write_infeasible(o, j);
+    if (o->seq_used) o->seq_used[j] = 0;
     if (rq_ttft) for (u64 i = 0; i < n; i++) rq_ttft[i] = INFINITY;
     if (rq_tpot) for (u64 i = 0; i < n; i++) rq_tpot[i] = INFINITY;
 #undef IN
@@ -558,7 +583,7 @@ infeasible:
 /* Evaluate configs first, first+stride, ... (count of them); output slot j for the j-th.
  * trace == NULL: closed form.  Returns 0, or -2 when a 64-bit product overflowed. */
 int oracle_simulate(const ospace *s, const otrace *tr, u64 first, u64 count, u64 stride,
-                    int time_model, int tp_model, u64 max_iters, const oout *o, int threads) {
+                    int time_model, int tp_model, u64 max_iters, const oout *o, int threads, int clamp_seq) {
     int bad = 0;
     /* reject shapes the model is not defined for: zero sizes, KV bytes per token rounding to 0 */
     u64 t_max = 0;
@@ -585,6 +610,11 @@ int oracle_simulate(const ospace *s, const otrace *tr, u64 first, u64 count, u64
         if (policy == POLICY_SPLIT_FUSE && (seg == 0 || split != 0)) return -1;   /* needs its token budget, and only that */
     }
     for (u32 i = 0; i < s->n_l; i++) if (s->pairs[2 * i] == 0 || s->pairs[2 * i + 1] == 0) return -1;
+    if (s->fw_keep) for (u32 i = 0; i < s->n_f; i++) {
+        if (s->fw_keep[i] > 1000) return -1;
+        if (tr && s->fw_keep[i] != 0 && s->fw_keep[i] != 1000) return -3;   /* cache eviction is modelled in the closed form only */
+    }
+    if (tr && clamp_seq) return -3;                                         /* a trace fixes the lengths of its requests */
     if (tr) for (u64 i = 0; i < tr->n; i++) {
         if (i && tr->arrival[i] < tr->arrival[i - 1]) return -1;
         if (tr->in_len[i] && !tr->out_len[i]) return -1;
@@ -601,7 +631,7 @@ int oracle_simulate(const ospace *s, const otrace *tr, u64 first, u64 count, u64
         for (long long j = 0; j < (long long)count; j++) {
             u64 idx = first + (u64)j * stride;
             if (tr) trace_sim_one(s, tr, idx, (u64)j, time_model, tp_model, max_iters, o, &w);
-            else closed_form_one(s, idx, (u64)j, time_model, tp_model, o);
+            else closed_form_one(s, idx, (u64)j, time_model, tp_model, clamp_seq, o);
         }
         if (tr) simbuf_free(&w);
         bad |= g_overflow;

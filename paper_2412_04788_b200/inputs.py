@@ -196,11 +196,14 @@ def hybrid_axis(n_gpus: int):
     return dps, tps
 
 
-def _space(models, hw, hw_mem, fw_f, fw_i, batch, tp, pairs, dp=None, fw_chunk=None):
+def _space(models, hw, hw_mem, fw_f, fw_i, batch, tp, pairs, dp=None, fw_chunk=None, fw_keep=None):
     """dp (optional): data-parallel degree per entry of the TP axis.  fw_chunk (optional): per
     framework (split_size, seg_tokens) = requests per prompt sub-batch, tokens per prompt segment;
-    0 = whole batch / whole prompt."""
+    0 = whole batch / whole prompt.  fw_keep (optional): per framework, thousandths of the KV cache
+    its eviction policy keeps (0 or 1000 = all of it)."""
     extra = {} if dp is None else {"dp": np.ascontiguousarray(dp, dtype=np.uint32)}
+    if fw_keep is not None:
+        extra["fw_keep"] = np.ascontiguousarray(fw_keep, dtype=np.uint32).reshape(len(fw_f))
     assert dp is None or len(dp) == len(tp)
     if fw_chunk is not None:
         extra["fw_chunk"] = np.ascontiguousarray(fw_chunk, dtype=np.uint32).reshape(len(fw_f), 2)

@@ -11,7 +11,7 @@ from paper_2412_04788_b200 import inputs as I
 
 
 def toy_space(golden, mem, kv_block, batch, pairs=((4, 3),), tp=(1,), e=None, t_ovh=0.0, flash=1, reserve=0,
-              layers=None, dp=None, chunk=None):
+              layers=None, dp=None, chunk=None, keep=None):
     model = list(golden["model"])
     if layers:
         model[0] = layers
@@ -19,7 +19,7 @@ def toy_space(golden, mem, kv_block, batch, pairs=((4, 3),), tp=(1,), e=None, t_
     return I._space(np.array([model]), np.array([golden["hw"]]), np.array([mem]),
                     np.array([fw_f + [t_ovh]]), np.array([[flash, kv_block, reserve, 0]]),
                     list(batch), list(tp), [list(p) for p in pairs], dp=None if dp is None else list(dp),
-                    fw_chunk=None if chunk is None else [list(chunk)])
+                    fw_chunk=None if chunk is None else [list(chunk)], fw_keep=None if keep is None else [keep])
 
 
 def test_weight_count_and_kv_bytes(golden):
@@ -302,6 +302,93 @@ def test_trace_cost_is_price_times_tp_degree(golden):
     out1 = oracle.simulate(sp1, tr1)
     assert out1["cost_per_hr"][0] == 1.0
     assert out1["cost_per_token"][0] == (1.0 / 3600.0) / (tl["dec_tok"] / tl["dec_time"])
+
+
+def test_cache_eviction_keeps_a_share_of_the_kv(golden):
+    """H2O (Sec. 3.2 Step 1, Sec. 3.3): a request's cache holds ceil(p c / 1000) of its c tokens - in the
+    memory check (per request, then whole blocks) and in the decode stage's attention work and KV
+    read (on the stage total).  The prompt pass is not touched.  Values worked by hand."""
+    g = golden["kv_reduction_and_clamp"]
+    weights = 2 * golden["weights"]["params"]
+    for row in g["bmax"]["rows"]:
+        out = oracle.simulate(toy_space(golden, weights + g["bmax"]["avail_bytes"], row["block"], [1, row["bmax"], row["bmax"] + 1],
+                                        keep=row["p"]))
+        assert out["bmax"].tolist() == [row["bmax"]] * 3, row
+        assert out["status"].tolist() == [0, 0, oracle.ST_KV], row
+    base = golden["closed_form_b2_Lin4_Lout3"]["t1"]
+    for row in g["decode"]["rows"]:
+        out = oracle.simulate(toy_space(golden, 10**6, 1, [2], keep=row["p"]))
+        assert out["ttft"][0] == base["ttft"]                                  # the prompt is attended in full
+        assert out["latency"][0] == row["latency"] and out["latency"][0] - out["ttft"][0] == row["T_dec"]
+        assert out["tpot"][0] == row["tpot"] and out["thr_decode"][0] == 4 / row["T_dec"]
+        kept = next(k["kept"] for k in g["kept"] if k["p"] == row["p"] and k["c"] == 22)
+        _, d = oracle.phase_time(golden["model"], golden["hw"], [1.0] * 7 + [0.0], [1, 1, 0, 0], 1, 4, 4, kept, kept, 2)
+        assert d[14] == row["S_att"]
+    # 0 and 1000 both mean that nothing is evicted; more than everything is refused
+    full = oracle.simulate(toy_space(golden, 10**6, 1, [1, 2, 3]))
+    for p in (0, 1000):
+        same = oracle.simulate(toy_space(golden, 10**6, 1, [1, 2, 3], keep=p))
+        for k in full:
+            assert np.array_equal(full[k], same[k]), (p, k)
+    with pytest.raises(ValueError):
+        oracle.simulate(toy_space(golden, 10**6, 1, [2], keep=1001))
+    # a smaller share never costs time or room (rounding is monotone)
+    hw, mem = I.seeded_hw(31, 3, mem_gb=[24, 48, 80])
+    fw_f, fw_i = I.seeded_fw(31, 1)
+    sp = lambda p: I._space(I.models_from_shapes(I.SHAPES_8[:4]), hw, mem, fw_f, fw_i, [1, 8, 64], [1, 2], I.pairs_grid([64, 1000], [1, 33, 512]),
+                            fw_keep=[p])
+    prev = oracle.simulate(sp(1000))
+    for p in (900, 501, 500, 37, 1):
+        cur = oracle.simulate(sp(p))
+        both = (prev["status"] == 0) & (cur["status"] == 0)
+        assert np.all(cur["bmax"] >= prev["bmax"]) and np.all(cur["status"][prev["status"] == 0] == 0)
+        assert np.all(cur["latency"][both] <= prev["latency"][both]) and np.array_equal(cur["ttft"][both], prev["ttft"][both])
+        prev = cur
+    # the trace simulation does not model it
+    tr = {"arrival": np.array([0.0, 1.0]), "in_len": np.zeros(2, np.uint32), "out_len": np.zeros(2, np.uint32)}
+    with pytest.raises(ValueError, match="cache eviction"):
+        oracle.simulate(toy_space(golden, 10**6, 1, [2], keep=500), tr)
+
+
+def test_sequence_cut_to_what_fits(golden):
+    """Sec. 3.3.2: S_max = floor(C_available / (KV bytes per token x B)); a longer sequence is cut to it
+    (whole blocks; the prompt is cut, the output tokens stay), and the length used is reported."""
+    g = golden["kv_reduction_and_clamp"]
+    weights = 2 * golden["weights"]["params"]
+    for row in g["clamp"]:
+        sp = toy_space(golden, weights + row["avail"], row["block"], [2], keep=row["p"])
+        out = oracle.simulate(sp, clamp_seq=True)
+        assert out["status"][0] == row["status"] and out["seq_used"][0] == row["seq_used"] and out["bmax"][0] == row["bmax"], row
+        if row["status"] == 0:
+            # the same numbers as the shorter prompt evaluated where memory is ample
+            ref = oracle.simulate(toy_space(golden, 10**6, row["block"], [2], pairs=[(row["lin_used"], 3)], keep=row["p"]))
+            for k in oracle.F64_FIELDS + ("n_iters", "n_req_iters"):
+                assert out[k][0] == ref[k][0], (row, k)
+        else:
+            assert np.isinf(out["latency"][0])
+        # without the option the long sequence is judged as it is
+        plain = oracle.simulate(sp)
+        assert plain["seq_used"][0] == (7 if plain["status"][0] == 0 else 0)
+        assert (plain["status"][0] == 0) == (row["seq_used"] == 7)
+    # a sweep: cut configs are exactly those that did not fit by their KV need alone and have room for
+    # one prompt token; nothing else changes; a cut config fills its memory to within one block per request
+    hw, mem = I.seeded_hw(32, 4, mem_gb=[16, 24, 48, 80])
+    fw_f, fw_i = I.seeded_fw(32, 2)
+    sp = I._space(I.models_from_shapes(I.SHAPES_8[:5]), hw, mem, fw_f, fw_i, [1, 16, 256], [1, 4], I.pairs_grid([128, 4096, 8192], [64, 2048]),
+                  fw_keep=[1000, 400])
+    a, c = oracle.simulate(sp), oracle.simulate(sp, clamp_seq=True)
+    cut = (c["status"] == 0) & (a["status"] != 0)
+    assert cut.sum() > 20 and np.all(a["status"][cut] == oracle.ST_KV)
+    same = ~cut
+    for k in a:
+        assert np.array_equal(a[k][same], c[k][same]), k
+    n_l = len(sp["pairs"])
+    S = (sp["pairs"][:, 0] + sp["pairs"][:, 1])[np.arange(len(cut)) % n_l]
+    lout = sp["pairs"][:, 1][np.arange(len(cut)) % n_l]
+    assert np.all(c["seq_used"][cut] < S[cut]) and np.all(c["seq_used"][cut] > lout[cut])
+    tr = {"arrival": np.array([0.0, 1.0]), "in_len": np.zeros(2, np.uint32), "out_len": np.zeros(2, np.uint32)}
+    with pytest.raises(ValueError, match="clamping"):
+        oracle.simulate(toy_space(golden, 10**6, 1, [2]), tr, clamp_seq=True)
 
 
 def test_paper_log2_rule(golden):
