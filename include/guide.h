@@ -87,6 +87,14 @@ typedef struct guide_fw {
      * the time of all passes, n_iters counts them, n_req_iters = batch x (segments + Lout - 1). */
     uint32_t split_size;
     uint32_t seg_tokens;
+    /* KV-cache eviction (H2O; Sec. 3.2 Step 1 and Sec. 3.3 name it among the optimisations that shrink
+     * the cache, without a rule): thousandths of a request's cache that the policy keeps; a cache of c
+     * tokens holds ceil(kv_keep_permille * c / 1000).  Used by the memory check (per request, then whole
+     * blocks) and by the decode stage (attention work and KV read of the stage total); the prompt pass
+     * attends its prompt in full.  0 or 1000 = nothing is evicted.  Closed form only: with a trace,
+     * any other value gives GUIDE_ERR_UNSUPPORTED. */
+    uint32_t kv_keep_permille;
+    uint32_t reserved;
 } guide_fw;
 
 typedef struct guide_len_pair { uint32_t lin, lout; } guide_len_pair;
@@ -138,6 +146,15 @@ typedef struct guide_sim_opts {
     int32_t time_model;   /* GUIDE_TIME_* */
     int32_t tp_model;     /* GUIDE_TP_* */
     uint64_t max_iters;   /* trace simulation: iteration cap per config; 0 = 64*sum(out_len) + 4*n_req */
+    /* Dynamic sequence length adjustment (Sec. 3.3.2), closed form only (with a trace:
+     * GUIDE_ERR_UNSUPPORTED).  1: a config whose sequence Lin + Lout is longer than
+     * S_max = floor(C_available / (KV bytes per token x B)) - in whole KV blocks, and with cache
+     * eviction the longest sequence whose kept part fits - is evaluated with its prompt cut so that
+     * Lin + Lout = S_max, provided at least one prompt token remains; bmax is then that of the length
+     * used.  outputs->seq_used tells which configs were cut.  0 (default): every config is judged
+     * with its own lengths. */
+    int32_t clamp_seq;
+    int32_t reserved;
 } guide_sim_opts;
 
 /* status bits */
@@ -165,6 +182,9 @@ typedef struct guide_outputs {
     uint64_t *n_req_iters;   /* sum over iterations of participating requests */
     double *req_ttft;        /* trace only, [count][n_req]: per-request TTFT */
     double *req_tpot;        /* trace only, [count][n_req]: per-request mean time per output token */
+    uint32_t *seq_used;      /* closed form: tokens per request the metrics were computed for: Lin + Lout, less when
+                                clamp_seq cut the prompt, 0 for configs that do not fit; trace: 0.  Asking for it
+                                sends a closed-form call through the one-thread-per-config kernel. */
 } guide_outputs;
 
 enum { GUIDE_STAT_MEAN = 0, GUIDE_STAT_P50 = 1, GUIDE_STAT_P99 = 2 };

@@ -21,6 +21,7 @@ __device__ __forceinline__ void store_metrics(const guide_outputs &o, u64 j, con
     if (o.bmax) __stcs(o.bmax + j, m.bmax);
     if (o.n_iters) __stcs(o.n_iters + j, m.n_iters);
     if (o.n_req_iters) __stcs(o.n_req_iters + j, m.n_req_iters);
+    if (o.seq_used) __stcs(o.seq_used + j, m.seq_used);
 }
 
 // One thread per config, nothing shared between configs.

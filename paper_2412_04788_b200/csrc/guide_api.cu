@@ -73,6 +73,7 @@ static int check_closed_form_overflow(const guide_space &s) {
                             "model %zu with batch %u and lengths (%u, %u) overflows a 64-bit FLOP/byte count",
                             mi, s.max_batch, p.lin, p.lout);
             if (b * (1 + n) >= LIMIT) return fail(GUIDE_ERR_OVERFLOW, "request-iteration count overflows");
+            if (dec.A * 1000 >= LIMIT) return fail(GUIDE_ERR_OVERFLOW, "decode context x 1000 (kept share of the KV cache) overflows");
         }
     }
     return GUIDE_OK;
@@ -134,7 +135,7 @@ __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *g
         r.split = f.split_size;
         r.seg = f.seg_tokens;
         r.policy = f.policy;
-        r.pad = 0;
+        r.keep = (f.kv_keep_permille == 0 || f.kv_keep_permille >= 1000) ? 1000u : f.kv_keep_permille;
         dr[i] = r;
         hfmem[i] = make_ulonglong2(r.usable, (u64)r.kv_block);
         double *q = rate10 + (size_t)i * 10;
@@ -290,6 +291,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket, cudaStream_t
     d.view.tp = (const u32 *)(blob + o_t);
     d.view.dp = (const u32 *)(blob + o_d);
     d.view.chunked = s->chunked ? 1u : 0u;
+    d.view.clamp_seq = 0;
     d.view.pairs = (const uint2 *)(blob + o_p);
     d.view.cost_hr = (const double *)(blob + o_ch);
     d.view.cost_sec = (const double *)(blob + o_cs);
@@ -349,6 +351,7 @@ static int resolve_range(const guide_space *s, const guide_sim_opts *o, Range *r
     if (r->count > s->size - r->first) return fail(GUIDE_ERR_INVALID, "range runs past the end of the space");
     if (o && (o->time_model < 0 || o->time_model > 1 || o->tp_model < 0 || o->tp_model > 1))
         return fail(GUIDE_ERR_INVALID, "unknown time_model or tp_model");
+    if (o && (o->clamp_seq < 0 || o->clamp_seq > 1)) return fail(GUIDE_ERR_INVALID, "clamp_seq must be 0 or 1");
     return GUIDE_OK;
 }
 
@@ -470,7 +473,10 @@ int guide_space_create(const guide_space_desc *d, guide_space **out) {
         if (!ok) rc = fail(GUIDE_ERR_INVALID, "framework profile %zu has a bad efficiency, kv_block or reserve", i);
         else if (f.policy != GUIDE_POLICY_PREFILL_FIRST && f.policy != GUIDE_POLICY_SPLIT_FUSE)
             rc = fail(GUIDE_ERR_UNSUPPORTED, "framework profile %zu: unknown policy", i);
-        s->chunked = s->chunked || f.split_size || f.seg_tokens;
+        else if (f.kv_keep_permille > 1000)
+            rc = fail(GUIDE_ERR_INVALID, "framework profile %zu: kv_keep_permille above 1000", i);
+        s->evicting = s->evicting || (f.kv_keep_permille != 0 && f.kv_keep_permille != 1000);
+        s->chunked = s->chunked || f.split_size || f.seg_tokens || (f.kv_keep_permille != 0 && f.kv_keep_permille != 1000);
     }
     if (!rc) {
         u128 n = (u128)d->n_models * d->n_hw * d->n_fw * d->n_batch * d->n_tp * d->n_pairs;
@@ -581,6 +587,10 @@ int guide_simulate(const guide_space *space_c, const guide_trace *trace_c, const
     if (!trace && (out->req_ttft || out->req_tpot))
         return fail(GUIDE_ERR_INVALID, "per-request outputs need a trace");
     if (trace) {
+        if (opts && opts->clamp_seq)
+            return fail(GUIDE_ERR_UNSUPPORTED, "clamp_seq cuts the lengths of a closed-form config; a trace fixes the lengths of its requests");
+        if (space->evicting)
+            return fail(GUIDE_ERR_UNSUPPORTED, "a framework profile evicts part of the KV cache (kv_keep_permille): modelled in the closed form only");
         if (space->max_dp > 1)
             return fail(GUIDE_ERR_UNSUPPORTED, "the trace simulation models one replica: the space has a data-parallel degree of %u",
                         space->max_dp);
@@ -604,7 +614,12 @@ int guide_simulate(const guide_space *space_c, const guide_trace *trace_c, const
     DSpace ds;
     unsigned *ticket = nullptr;
     if ((rc = space_on_device(space, &ds, &ticket, (cudaStream_t)stream))) return rc;
-    if (!trace) return launch_closed_form(ds, r, time_model, tp_model, *out, ticket, (cudaStream_t)stream);
+    if (!trace) {
+        // options and outputs only the one-thread-per-config evaluation knows: keep the whole-space kernels out
+        if ((opts && opts->clamp_seq) || out->seq_used) ds.chunked = 1;
+        ds.clamp_seq = opts ? (u32)opts->clamp_seq : 0u;
+        return launch_closed_form(ds, r, time_model, tp_model, *out, ticket, (cudaStream_t)stream);
+    }
     DTrace dt;
     if ((rc = trace_on_device(trace, &dt, (cudaStream_t)stream))) return rc;
     u32 policies = 0;
@@ -633,6 +648,7 @@ int guide_select_topk(const guide_space *space_c, const guide_trace *trace, cons
     DSpace ds;
     unsigned *ticket = nullptr;                  // the fused path's model walk takes its work items through it
     if ((rc = space_on_device(space, &ds, outputs ? nullptr : &ticket, (cudaStream_t)stream))) return rc;
+    if (!outputs && opts && opts->clamp_seq) { ds.chunked = 1; ds.clamp_seq = 1; }     // fused: evaluated with the option
     return launch_topk(ds, r, outputs, opts ? opts->time_model : 0, opts ? opts->tp_model : 0, *cons, key, k,
                        (u64 *)idx_out, key_out, count_out, ws, ticket, (cudaStream_t)stream);
 }
@@ -651,6 +667,7 @@ int guide_pareto(const guide_space *space_c, const guide_trace *trace, const gui
     DSpace ds;
     unsigned *ticket = nullptr;
     if ((rc = space_on_device(space, &ds, outputs ? nullptr : &ticket, (cudaStream_t)stream))) return rc;
+    if (!outputs && opts && opts->clamp_seq) { ds.chunked = 1; ds.clamp_seq = 1; }
     return launch_pareto(ds, r, outputs, opts ? opts->time_model : 0, opts ? opts->tp_model : 0, *cons, xm, ym,
                          (u64 *)idx_out, cap, count_out, ws, ticket, (cudaStream_t)stream);
 }

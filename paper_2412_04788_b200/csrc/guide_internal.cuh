@@ -48,7 +48,7 @@ struct guide_space {
     std::vector<uint32_t> batch, tp, dp;          // dp[i] goes with tp[i]; all 1 when the caller gave none
     std::vector<guide_len_pair> pairs;
     uint64_t size = 0;
-    uint32_t max_batch = 0, max_tp = 0, max_lin = 0, max_lout = 0, max_dp = 1, chunked = 0;
+    uint32_t max_batch = 0, max_tp = 0, max_lin = 0, max_lout = 0, max_dp = 1, chunked = 0, evicting = 0;
     std::mutex mu;
     std::vector<guide::DeviceTables> dev;
 };

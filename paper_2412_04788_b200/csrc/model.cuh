@@ -32,7 +32,8 @@ struct DRate {
     u64 usable;   // MEM - (MEM/1000) * reserve_permille
     u32 flash, kv_block;
     u32 split, seg;   // requests per prompt sub-batch, tokens per prompt segment (0: whole batch / prompt)
-    u32 policy, pad;  // trace scheduling: GUIDE_POLICY_*; with SPLIT_FUSE seg is the token budget of an iteration
+    u32 policy;       // trace scheduling: GUIDE_POLICY_*; with SPLIT_FUSE seg is the token budget of an iteration
+    u32 keep;         // thousandths of a request's KV cache the eviction policy keeps (1000: all of it)
 };
 
 // one hardware x framework pair in the sorted walk of the model kernel
@@ -62,7 +63,9 @@ struct DSpace {
     const u32 *plane_order;      // [n_m][n_t * n_l / 4]: foursomes of the (TP, length) plane by growing memory need
     const u32 *line_order;       // [n_m][n_t * n_l / 16]: the same for lines of sixteen positions
     u32 n_m, n_h, n_f, n_b, n_t, n_l;
-    u32 chunked;                 // some framework splits prompt processing: only the flat evaluation handles that
+    u32 chunked;                 // per-framework prompt splitting or cache eviction, or a per-call option below: only the
+                                 // one-thread-per-config evaluation handles those (no tables shared between frameworks)
+    u32 clamp_seq;               // cut sequences that do not fit to S_max (Sec. 3.3.2); set per call
 };
 
 struct DTrace {
@@ -409,6 +412,7 @@ struct Metrics {
     u64 n_iters, n_req_iters;
     u32 bmax;
     u32 status;
+    u32 seq_used;      // tokens per request the metrics were computed for; 0 when the config does not fit
 };
 
 __device__ __forceinline__ void set_infeasible(Metrics &o) {
@@ -422,9 +426,12 @@ __device__ __forceinline__ void set_infeasible(Metrics &o) {
 // (the one with the rounded-up share) sets the time and the memory need.
 __device__ __forceinline__ u32 replica_batch(u32 b, u32 dp) { return dp == 1 ? b : (b + dp - 1) / dp; }
 
+// Tokens of a cache of c tokens that stay when the eviction policy keeps p thousandths of it.
+__device__ __forceinline__ u64 kept_tokens(u64 c, u32 p) { return p >= 1000 ? c : (c * p + 999) / 1000; }
+
 __device__ __forceinline__ u32 closed_form_feasibility(const DModel &m, const DRate &r, const MemInfo &mi, u32 t,
                                                        u32 b, u32 lin, u32 lout, u32 &bmax_out) {
-    const u64 S = (u64)lin + lout;
+    const u64 S = kept_tokens((u64)lin + lout, r.keep);
     const u64 s_blk = r.kv_block == 1 ? S : ((S + r.kv_block - 1) / r.kv_block) * r.kv_block;
     const u64 bmax = r.usable > mi.w_gpu ? floor_div(r.usable - mi.w_gpu, s_blk * mi.kv_tok) : 0;
     u32 st = 0;
@@ -483,9 +490,20 @@ __device__ __forceinline__ void closed_form_eval(const DSpace &s, const Cfg &c, 
     const u32 t = s.tp[c.t], b_all = s.batch[c.b];
     const u32 b = replica_batch(b_all, s.dp[c.t]);   // each of the dp replicas serves its share of the batch
     const uint2 pr = s.pairs[c.l];
-    const u32 lin = pr.x, lout = pr.y;
+    u32 lin = pr.x;
+    const u32 lout = pr.y;
     const MemInfo mi = mem_info(m, t);
+    if (s.clamp_seq && r.usable > mi.w_gpu) {
+        // Sec. 3.3.2: S_max = floor(C_available / (KV bytes per token x B)), in whole blocks; with cache
+        // eviction the longest sequence whose kept part fits.  The prompt is what gets cut.
+        const u64 cap_tok = floor_div(r.usable - mi.w_gpu, mi.kv_tok * b);
+        const u64 cap_blk = (cap_tok / r.kv_block) * r.kv_block;
+        // room for 2^40 tokens or more is room for any sequence (lengths are 32-bit): no product that could wrap
+        const u64 s_max = (r.keep >= 1000 || cap_blk >= (1ull << 40)) ? cap_blk : (1000 * cap_blk) / r.keep;
+        if ((u64)lin + lout > s_max && s_max > lout) lin = (u32)(s_max - lout);
+    }
     o.status = closed_form_feasibility(m, r, mi, t, b, lin, lout, o.bmax);
+    o.seq_used = o.status ? 0u : lin + lout;
     if (o.status) { set_infeasible(o); return; }
     const u32 tt = tp_model ? 1u : t;
     const double lf = log2_rule_factor(t, tp_model);
@@ -512,7 +530,8 @@ __device__ __forceinline__ void closed_form_eval(const DSpace &s, const Cfg &c, 
     double t_dec = 0.0;
     if (n > 0) {
         const u64 Td = (u64)b * n;
-        const u64 ctx = (u64)b * ((u64)n * lin + ((u64)n * (n + 1)) / 2);
+        // step j attends lin + j tokens, of which the cache still holds the kept share
+        const u64 ctx = kept_tokens((u64)b * ((u64)n * lin + ((u64)n * (n + 1)) / 2), r.keep);
         build_fixed_tasks(m, tt, Td, Td, n, k);
         build_attn_tasks(m, tt, Td, ctx, ctx, k);
         t_dec = eval_phase<TIME_SUM>(k, r, Nd, lf);

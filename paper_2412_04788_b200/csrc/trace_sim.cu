@@ -102,6 +102,7 @@ __device__ __forceinline__ void write_trace_results(const guide_outputs &o, u64 
             if (o.bmax) o.bmax[j] = fit;
             if (o.n_iters) o.n_iters[j] = 0;
             if (o.n_req_iters) o.n_req_iters[j] = 0;
+            if (o.seq_used) o.seq_used[j] = 0;
         }
         for (u32 i = lane; i < n; i += 32) {
             if (rq_ttft) __stcs(rq_ttft + i, inf);
@@ -160,6 +161,7 @@ __device__ __forceinline__ void write_trace_results(const guide_outputs &o, u64 
         if (o.bmax) o.bmax[j] = fit;
         if (o.n_iters) o.n_iters[j] = n_iters;
         if (o.n_req_iters) o.n_req_iters[j] = n_req_iters;
+        if (o.seq_used) o.seq_used[j] = 0;          // closed form only
     }
 }
 
@@ -569,6 +571,7 @@ __device__ __noinline__ void write_lane_results(const guide_outputs &o, u64 j, u
             if (o.bmax) o.bmax[j] = fit;
             if (o.n_iters) o.n_iters[j] = 0;
             if (o.n_req_iters) o.n_req_iters[j] = 0;
+            if (o.seq_used) o.seq_used[j] = 0;
         }
         for (u32 i = lane; i < n; i += 32) {
             if (rq_ttft) __stcs(rq_ttft + i, inf);
@@ -643,6 +646,7 @@ __device__ __noinline__ void write_lane_results(const guide_outputs &o, u64 j, u
         if (o.bmax) o.bmax[j] = fit;
         if (o.n_iters) o.n_iters[j] = n_iters;
         if (o.n_req_iters) o.n_req_iters[j] = n_req_iters;
+        if (o.seq_used) o.seq_used[j] = 0;          // closed form only
     }
 }
 

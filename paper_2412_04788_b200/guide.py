@@ -54,7 +54,7 @@ class Hw(C.Structure):
 class Fw(C.Structure):
     _fields_ = [("e_c", C.c_double * 3), ("e_m", C.c_double * 3), ("e_comm", C.c_double), ("t_ovh", C.c_double),
                 ("flash", C.c_uint32), ("kv_block", C.c_uint32), ("reserve_permille", C.c_uint32), ("policy", C.c_uint32),
-                ("split_size", C.c_uint32), ("seg_tokens", C.c_uint32)]
+                ("split_size", C.c_uint32), ("seg_tokens", C.c_uint32), ("kv_keep_permille", C.c_uint32), ("reserved", C.c_uint32)]
 
 
 class LenPair(C.Structure):
@@ -74,11 +74,11 @@ class Config(C.Structure):
 
 class SimOpts(C.Structure):
     _fields_ = [("first", C.c_uint64), ("count", C.c_uint64), ("time_model", C.c_int32), ("tp_model", C.c_int32),
-                ("max_iters", C.c_uint64)]
+                ("max_iters", C.c_uint64), ("clamp_seq", C.c_int32), ("reserved", C.c_int32)]
 
 
 class Outputs(C.Structure):
-    _fields_ = [(k, C.c_void_p) for k in ALL_OUTPUTS + ("req_ttft", "req_tpot")]
+    _fields_ = [(k, C.c_void_p) for k in ALL_OUTPUTS + ("req_ttft", "req_tpot", "seq_used")]
 
 
 class Constraints(C.Structure):
@@ -152,6 +152,8 @@ class Space:
             fws[i].flash, fws[i].kv_block, fws[i].reserve_permille, fws[i].policy = (int(x) for x in fi)
             if space.get("fw_chunk") is not None:
                 fws[i].split_size, fws[i].seg_tokens = (int(x) for x in space["fw_chunk"][i])
+            if space.get("fw_keep") is not None:
+                fws[i].kv_keep_permille = int(space["fw_keep"][i])
         batch = (C.c_uint32 * len(space["batch"]))(*[int(v) for v in space["batch"]])
         tp = (C.c_uint32 * len(space["tp"]))(*[int(v) for v in space["tp"]])
         pairs = (LenPair * len(space["pairs"]))(*[LenPair(int(a), int(b)) for a, b in space["pairs"]])
@@ -206,8 +208,8 @@ class Trace:
             pass
 
 
-def _opts(first=0, count=0, time_model=TIME_MAX, tp_model=TP_EXPLICIT, max_iters=0):
-    return SimOpts(first, count, time_model, tp_model, max_iters)
+def _opts(first=0, count=0, time_model=TIME_MAX, tp_model=TP_EXPLICIT, max_iters=0, clamp_seq=False):
+    return SimOpts(first, count, time_model, tp_model, max_iters, int(bool(clamp_seq)), 0)
 
 
 def _cons(cons):
@@ -233,7 +235,7 @@ _TORCH_DTYPES = None
 def alloc_outputs(count, n_req=0, fields=ALL_OUTPUTS, per_request=False, device="cuda"):
     """Caller-owned device arrays for guide_outputs, as a dict of torch tensors."""
     import torch
-    dt = {"status": torch.uint8, "bmax": torch.int32, "n_iters": torch.int64, "n_req_iters": torch.int64}
+    dt = {"status": torch.uint8, "bmax": torch.int32, "n_iters": torch.int64, "n_req_iters": torch.int64, "seq_used": torch.int32}
     out = {k: torch.empty(count, dtype=dt.get(k, torch.float64), device=device) for k in fields}
     if per_request:
         out["req_ttft"] = torch.empty((count, n_req), dtype=torch.float64, device=device)
@@ -242,7 +244,7 @@ def alloc_outputs(count, n_req=0, fields=ALL_OUTPUTS, per_request=False, device=
 
 
 def _outputs_struct(out):
-    return Outputs(*[_ptr(out.get(k)) for k in ALL_OUTPUTS + ("req_ttft", "req_tpot")])
+    return Outputs(*[_ptr(out.get(k)) for k in ALL_OUTPUTS + ("req_ttft", "req_tpot", "seq_used")])
 
 
 def guide_workspace_bytes(space: Space, trace: Trace | None) -> int:
@@ -250,10 +252,10 @@ def guide_workspace_bytes(space: Space, trace: Trace | None) -> int:
 
 
 def guide_simulate(space: Space, trace: Trace | None, out: dict, first=0, count=0, time_model=TIME_MAX,
-                   tp_model=TP_EXPLICIT, max_iters=0, workspace=None, stream=None):
+                   tp_model=TP_EXPLICIT, max_iters=0, workspace=None, stream=None, clamp_seq=False):
     """out: dict of torch CUDA tensors (see alloc_outputs); workspace: torch uint8 CUDA tensor or None."""
     o = _outputs_struct(out)
-    opts = _opts(first, count, time_model, tp_model, max_iters)
+    opts = _opts(first, count, time_model, tp_model, max_iters, clamp_seq)
     ws_ptr = _ptr(workspace)
     ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
     _check(lib().guide_simulate(space.handle, trace.handle if trace else None, C.byref(opts), C.byref(o), ws_ptr,
@@ -270,10 +272,10 @@ def guide_pareto_workspace_bytes(space: Space) -> int:
 
 def guide_select_topk(space: Space, trace: Trace | None, out: dict | None, cons: dict | None, key: str, k: int,
                       idx_out, key_out, count_out, workspace, first=0, count=0, time_model=TIME_MAX,
-                      tp_model=TP_EXPLICIT, stream=None):
+                      tp_model=TP_EXPLICIT, stream=None, clamp_seq=False):
     """idx_out int64[k], key_out float64[k], count_out int32[1], workspace uint8: torch CUDA tensors."""
     o = _outputs_struct(out) if out is not None else None
-    opts = _opts(first, count, time_model, tp_model)
+    opts = _opts(first, count, time_model, tp_model, 0, clamp_seq)
     cs = _cons(cons)
     _check(lib().guide_select_topk(space.handle, trace.handle if trace else None, C.byref(o) if o is not None else None,
                                    C.byref(opts), C.byref(cs), METRICS[key], k, _ptr(idx_out), _ptr(key_out),
@@ -282,9 +284,10 @@ def guide_select_topk(space: Space, trace: Trace | None, out: dict | None, cons:
 
 
 def guide_pareto(space: Space, trace: Trace | None, out: dict | None, cons: dict | None, x: str, y: str, idx_out,
-                 count_out, workspace, first=0, count=0, time_model=TIME_MAX, tp_model=TP_EXPLICIT, stream=None):
+                 count_out, workspace, first=0, count=0, time_model=TIME_MAX, tp_model=TP_EXPLICIT, stream=None,
+                 clamp_seq=False):
     o = _outputs_struct(out) if out is not None else None
-    opts = _opts(first, count, time_model, tp_model)
+    opts = _opts(first, count, time_model, tp_model, 0, clamp_seq)
     cs = _cons(cons)
     _check(lib().guide_pareto(space.handle, trace.handle if trace else None, C.byref(o) if o is not None else None,
                               C.byref(opts), C.byref(cs), METRICS[x], METRICS[y], _ptr(idx_out), idx_out.numel(),
