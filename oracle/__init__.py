@@ -25,13 +25,19 @@ TTFT_STATS = {"mean": 0, "p50": 1, "p99": 2}
 F64_FIELDS = ("latency", "ttft", "ttft_p50", "ttft_p99", "tpot", "thr_decode", "cost_per_hr", "cost_per_token")
 
 
-def build(force: bool = False) -> str:
-    """gcc -O2, contraction off (GCC fuses multiply-add by default otherwise)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        cmd = ["gcc", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fopenmp", "-shared", "-fPIC",
-               _SRC, "-o", _LIB, "-lm"]
-        subprocess.run(cmd, check=True)
-    return _LIB
+_LIB_F32 = os.path.join(_HERE, "libguide_oracle_f32.so")
+
+
+def build(force: bool = False, precision: str = "f64") -> str:
+    """gcc -O2, contraction off (GCC fuses multiply-add by default otherwise).  precision "f32" builds
+    the same source with the model's arithmetic type set to binary32 (-DREAL=float)."""
+    out = _LIB if precision == "f64" else _LIB_F32
+    if force or not os.path.exists(out) or os.path.getmtime(out) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fopenmp", "-shared", "-fPIC"]
+        if precision != "f64":
+            cmd.append("-DREAL=float")
+        subprocess.run(cmd + [_SRC, "-o", out, "-lm"], check=True)
+    return out
 
 
 class _Space(C.Structure):
@@ -64,10 +70,19 @@ class _Metrics(C.Structure):
 
 
 _lib = None
+_libs = {}
 
 
-def lib():
+def lib(precision: str = "f64"):
     global _lib
+    if precision != "f64":
+        if precision not in _libs:
+            L = C.CDLL(build(precision=precision))
+            L.oracle_simulate.restype = C.c_int
+            L.oracle_simulate.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint64,
+                                          C.c_int, C.c_int, C.c_uint64, C.c_void_p, C.c_int, C.c_int]
+            _libs[precision] = L
+        return _libs[precision]
     if _lib is None:
         _lib = C.CDLL(build())
         _lib.oracle_simulate.restype = C.c_int
@@ -111,8 +126,11 @@ def _space_struct(space):
 
 
 def simulate(space, trace=None, first=0, count=None, stride=1, time_model=TIME_MAX, tp_model=TP_EXPLICIT,
-             max_iters=0, per_request=False, n_threads=0, clamp_seq=False):
-    """Evaluate configs first, first+stride, ...; returns a dict of numpy arrays (one slot per config)."""
+             max_iters=0, per_request=False, n_threads=0, clamp_seq=False, precision="f64"):
+    """Evaluate configs first, first+stride, ...; returns a dict of numpy arrays (one slot per config).
+    precision "f32": the closed form with every operation of the model in binary32 (values come back
+    widened to float64)."""
+    assert precision == "f64" or trace is None, "the reduced-precision variant covers the closed form only"
     n_total = 1
     for k in ("models", "hw", "fw_f", "batch", "tp", "pairs"):
         n_total *= len(space[k])
@@ -138,7 +156,7 @@ def simulate(space, trace=None, first=0, count=None, stride=1, time_model=TIME_M
              _p(out["req_ttft"]) if "req_ttft" in out else None,
              _p(out["req_tpot"]) if "req_tpot" in out else None, _p(out["n_preempt"]), _p(out["seq_used"]))
     sp = _space_struct(space)
-    rc = lib().oracle_simulate(C.byref(sp), C.byref(ts) if ts is not None else None, first, count, stride,
+    rc = lib(precision).oracle_simulate(C.byref(sp), C.byref(ts) if ts is not None else None, first, count, stride,
                                time_model, tp_model, max_iters, C.byref(o), n_threads, int(bool(clamp_seq)))
     if rc != 0:
         why = {-1: "invalid input", -2: "64-bit overflow", -3: "data parallelism, prompt splitting, cache eviction or sequence clamping with a trace is not modelled"}.get(rc, "?")

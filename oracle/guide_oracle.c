@@ -44,6 +44,14 @@
 typedef uint64_t u64;
 typedef uint32_t u32;
 
+/* The arithmetic type of the performance model: binary64, or binary32 when built with -DREAL=float
+ * (the reduced-precision variant the library offers for the closed form; same operations, same
+ * order, every value rounded to binary32; results are handed back widened to double). */
+#ifndef REAL
+#define REAL double
+#endif
+typedef REAL real;
+
 enum { CLS_LINEAR = 0, CLS_ATTN = 1, CLS_ELEM = 2 };
 enum { TIME_MAX = 0, TIME_SUM = 1 };
 enum { TP_EXPLICIT = 0, TP_PAPER_LOG2 = 1 };
@@ -81,7 +89,7 @@ enum { POLICY_PREFILL_FIRST = 0, POLICY_SPLIT_FUSE = 1 };
 typedef struct { u64 N, H, nh, nkv, I, V, g, wb, ab, kvb, d, Dkv; } model_t;
 
 typedef struct {
-    double inv_c[3], inv_m[3], inv_comm, clat, tovh, price;
+    real inv_c[3], inv_m[3], inv_comm, clat, tovh, price;
     int flash;
 } rates_t;
 
@@ -113,13 +121,13 @@ static model_t load_model(const u32 *r) {
 static rates_t load_rates(const double *hw, const double *ff, const u32 *fi) {
     rates_t r;
     for (int k = 0; k < 3; k++) {
-        r.inv_c[k] = 1.0 / (hw[0] * ff[k]);
-        r.inv_m[k] = 1.0 / (hw[1] * ff[3 + k]);
+        r.inv_c[k] = (real)1 / ((real)hw[0] * (real)ff[k]);
+        r.inv_m[k] = (real)1 / ((real)hw[1] * (real)ff[3 + k]);
     }
-    r.inv_comm = 1.0 / (hw[2] * ff[6]);
-    r.clat = hw[3];
-    r.price = hw[4];
-    r.tovh = ff[7];
+    r.inv_comm = (real)1 / ((real)hw[2] * (real)ff[6]);
+    r.clat = (real)hw[3];
+    r.price = (real)hw[4];
+    r.tovh = (real)ff[7];
     r.flash = (int)fi[0];
     return r;
 }
@@ -139,12 +147,12 @@ static u64 usable_bytes(u64 mem, u64 reserve_permille) { return mem - (mem / 100
 
 /* ---- one task: compute load, data size -> time (Sec. 3.4.1, 3.4.2, 3.5.1) ------------------ */
 
-static double task_time(u64 F_sh, u64 F_rp, u64 B_sh, u64 B_rp, double t, double inv_c, double inv_m,
-                        int time_model) {
-    double F = (double)F_sh / t + (double)F_rp;   /* sharded part splits over t GPUs */
-    double B = (double)B_sh / t + (double)B_rp;
-    double tc = F * inv_c;                        /* compute time = load / compute power */
-    double tm = B * inv_m;                        /* read/write time = data / memory bandwidth */
+static real task_time(u64 F_sh, u64 F_rp, u64 B_sh, u64 B_rp, real t, real inv_c, real inv_m,
+                      int time_model) {
+    real F = (real)F_sh / t + (real)F_rp;         /* sharded part splits over t GPUs */
+    real B = (real)B_sh / t + (real)B_rp;
+    real tc = F * inv_c;                          /* compute time = load / compute power */
+    real tm = B * inv_m;                          /* read/write time = data / memory bandwidth */
     if (time_model == TIME_SUM) return tc + tm;   /* literal sum of Sec. 3.5.1 */
     return tc > tm ? tc : tm;                     /* roofline: the slower resource binds */
 }
@@ -155,26 +163,26 @@ static double task_time(u64 F_sh, u64 F_rp, u64 B_sh, u64 B_rp, double t, double
  * detail (optional, 16 doubles): t1..t8 with multiplicity, t9, t10, t11, S_comm, t13, S_fix,
  * S_att, T_phase.
  */
-static double phase_time(const model_t *m, const rates_t *r, u64 tp, u64 T, u64 E, u64 A, u64 C, u64 R,
-                         int time_model, int tp_model, double *detail) {
+static real phase_time(const model_t *m, const rates_t *r, u64 tp, u64 T, u64 E, u64 A, u64 C, u64 R,
+                       int time_model, int tp_model, double *detail) {
     u64 tt = (tp_model == TP_PAPER_LOG2) ? 1 : tp;   /* log2 rule: single-GPU formulas, scaled below */
-    double t = (double)tt;
-    const double *ic = r->inv_c, *im = r->inv_m;
+    real t = (real)tt;
+    const real *ic = r->inv_c, *im = r->inv_m;
     u64 H = m->H, I = m->I, Dkv = m->Dkv, V = m->V, ab = m->ab, wb = m->wb, kvb = m->kvb;
     u64 TH = mul(T, H), THa = mul(TH, ab), TI = mul(T, I), TIa = mul(TI, ab);
     u64 X = r->flash ? 0 : mul(mul(m->nh, A), ab);  /* score-matrix traffic, gone with FlashAttention */
-    double tk[14];
+    real tk[14];
 
-    tk[1] = 2.0 * task_time(0, mul(4, TH), 0, mul(2, THa), t, ic[CLS_ELEM], im[CLS_ELEM], time_model);
+    tk[1] = (real)2 * task_time(0, mul(4, TH), 0, mul(2, THa), t, ic[CLS_ELEM], im[CLS_ELEM], time_model);
     tk[2] = task_time(mul(2, mul(TH, H)), 0, add(mul(R, mul(mul(H, H), wb)), THa), THa, t,
                       ic[CLS_LINEAR], im[CLS_LINEAR], time_model);
-    tk[3] = 2.0 * task_time(mul(2, mul(TH, Dkv)), 0,
+    tk[3] = (real)2 * task_time(mul(2, mul(TH, Dkv)), 0,
                             add(mul(R, mul(mul(H, Dkv), wb)), mul(mul(T, Dkv), kvb)), THa, t,
                             ic[CLS_LINEAR], im[CLS_LINEAR], time_model);
     tk[4] = task_time(mul(2, mul(TH, H)), 0, add(mul(R, mul(mul(H, H), wb)), THa), THa, t,
                       ic[CLS_LINEAR], im[CLS_LINEAR], time_model);
-    tk[5] = 2.0 * task_time(0, TH, 0, mul(3, THa), t, ic[CLS_ELEM], im[CLS_ELEM], time_model);
-    tk[6] = (double)(1 + m->g) * task_time(mul(2, mul(TH, I)), 0, add(mul(R, mul(mul(H, I), wb)), TIa), THa, t,
+    tk[5] = (real)2 * task_time(0, TH, 0, mul(3, THa), t, ic[CLS_ELEM], im[CLS_ELEM], time_model);
+    tk[6] = (real)(1 + m->g) * task_time(mul(2, mul(TH, I)), 0, add(mul(R, mul(mul(H, I), wb)), TIa), THa, t,
                                            ic[CLS_LINEAR], im[CLS_LINEAR], time_model);
     tk[7] = task_time(mul(4, TI), 0, mul(2 + m->g, TIa), 0, t, ic[CLS_ELEM], im[CLS_ELEM], time_model);
     tk[8] = task_time(mul(2, mul(TI, H)), 0, add(mul(R, mul(mul(I, H), wb)), TIa), THa, t,
@@ -184,29 +192,29 @@ static double phase_time(const model_t *m, const rates_t *r, u64 tp, u64 T, u64 
     tk[10] = task_time(mul(5, mul(m->nh, A)), 0, mul(2, X), 0, t, ic[CLS_ATTN], im[CLS_ATTN], time_model);
     tk[11] = task_time(mul(2, mul(H, A)), 0, add(add(kv_read, THa), X), 0, t, ic[CLS_ATTN], im[CLS_ATTN], time_model);
     /* no sequence emits a token (a prompt segment that is not the last one): no LM head at all */
-    tk[13] = E == 0 ? 0.0
+    tk[13] = E == 0 ? (real)0
                     : task_time(mul(2, mul(mul(E, H), V)), 0, add(mul(R, mul(mul(H, V), wb)), mul(mul(E, V), ab)),
                                 mul(mul(E, H), ab), t, ic[CLS_LINEAR], im[CLS_LINEAR], time_model);
 
-    double S_fix = tk[1];
+    real S_fix = tk[1];
     for (int k = 2; k <= 8; k++) S_fix = S_fix + tk[k];
-    double S_att = tk[9] + tk[10];
+    real S_att = tk[9] + tk[10];
     S_att = S_att + tk[11];
 
     /* ring all-reduce of the T x H activations, twice per layer; only when really sharded */
-    double S_comm = 0.0;
+    real S_comm = 0;
     if (tt > 1) {
         u64 M = THa;
-        double t12 = (double)mul(R, 2 * (tt - 1)) * r->clat + ((double)mul(2 * (tt - 1), M) / t) * r->inv_comm;
-        S_comm = 2.0 * t12;
+        real t12 = (real)mul(R, 2 * (tt - 1)) * r->clat + ((real)mul(2 * (tt - 1), M) / t) * r->inv_comm;
+        S_comm = (real)2 * t12;
     }
-    double T_layer = (S_fix + S_att) + S_comm;
-    double T_phase = (double)R * r->tovh + ((double)m->N * T_layer + tk[13]);
+    real T_layer = (S_fix + S_att) + S_comm;
+    real T_phase = (real)R * r->tovh + ((real)m->N * T_layer + tk[13]);
     if (tp_model == TP_PAPER_LOG2) {
         /* throughput N T_single / (1 + log2 P_TP) with N = P_TP GPUs: time scales by (1+log2 t)/t */
         u64 lg = 0;
         while (((u64)1 << (lg + 1)) <= tp) lg++;
-        T_phase = T_phase * ((double)(1 + lg) / (double)tp);
+        T_phase = T_phase * ((real)(1 + lg) / (real)tp);
     }
     if (detail) {
         for (int k = 1; k <= 11; k++) detail[k - 1] = tk[k];
@@ -243,9 +251,9 @@ static void write_infeasible(const oout *o, u64 j) {
  * segment; its q tokens attend the done + q tokens of their own prompt seen so far, and only the
  * last segment emits a token.  Every pass reads the weights and pays the iteration overhead.
  */
-static double segmented_prefill(const model_t *m, const rates_t *r, u64 t, u64 sb, u64 Lin, u64 seg,
-                                int time_model, int tp_model) {
-    double sum = 0.0;
+static real segmented_prefill(const model_t *m, const rates_t *r, u64 t, u64 sb, u64 Lin, u64 seg,
+                              int time_model, int tp_model) {
+    real sum = 0;
     for (u64 done = 0; done < Lin; done += seg) {
         u64 q = Lin - done < seg ? Lin - done : seg;
         u64 T = mul(sb, q);
@@ -307,22 +315,25 @@ static void closed_form_one(const ospace *s, u64 idx, u64 j, int time_model, int
     if (split == 0 || split > b) split = b;
     if (seg == 0 || seg > Lin) seg = Lin;
     u64 n_full = b / split, rest = b % split, n_seg = ceil_div(Lin, seg);
-    double T_pre = (double)n_full * segmented_prefill(&m, &r, t, split, Lin, seg, time_model, tp_model);
+    real T_pre = (real)n_full * segmented_prefill(&m, &r, t, split, Lin, seg, time_model, tp_model);
     if (rest) T_pre = T_pre + segmented_prefill(&m, &r, t, rest, Lin, seg, time_model, tp_model);
     u64 n = Lout - 1;                 /* the prefill pass emits token 1 */
-    double T_dec = 0.0;
+    real T_dec = 0;
     if (n > 0) {
         u64 ctx = mul(b, add(mul(n, Lin), mul(n, n + 1) / 2));   /* step j attends Lin + j */
         ctx = kept_tokens(ctx, keep);                            /* ... of which the cache still holds this many: less work, less KV read */
         T_dec = phase_time(&m, &r, t, mul(b, n), mul(b, n), ctx, ctx, n, time_model, tp_model, NULL);
     }
     o->ttft[j] = T_pre; o->ttft_p50[j] = T_pre; o->ttft_p99[j] = T_pre;
-    o->latency[j] = T_pre + T_dec;
-    o->cost_per_hr[j] = r.price * (double)mul(t, dp);        /* every GPU of every replica is paid for */
+    real lat = T_pre + T_dec;
+    o->latency[j] = lat;
+    real cost_hr = r.price * (real)mul(t, dp);               /* every GPU of every replica is paid for */
+    o->cost_per_hr[j] = cost_hr;
     if (n > 0) {
-        o->tpot[j] = T_dec / (double)n;
-        o->thr_decode[j] = (double)mul(b_all, n) / T_dec;     /* all replicas decode at once (Sec. 3.2: N x T_single) */
-        o->cost_per_token[j] = (o->cost_per_hr[j] / 3600.0) / o->thr_decode[j];
+        real tpot = T_dec / (real)n;
+        real thr = (real)mul(b_all, n) / T_dec;               /* all replicas decode at once (Sec. 3.2: N x T_single) */
+        real cost_tok = (cost_hr / (real)3600) / thr;
+        o->tpot[j] = tpot; o->thr_decode[j] = thr; o->cost_per_token[j] = cost_tok;
     } else {
         o->tpot[j] = 0.0; o->thr_decode[j] = 0.0; o->cost_per_token[j] = INFINITY;
     }

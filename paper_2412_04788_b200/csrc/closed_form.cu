@@ -35,6 +35,17 @@ __global__ void __launch_bounds__(256) k_closed_form_flat(DSpace s, Range r, int
     store_metrics(o, j, m);
 }
 
+// The same in binary32 (model_f32.cuh): the reduced-precision variant, values stored widened.
+template <int TIME_SUM>
+__global__ void __launch_bounds__(256) k_closed_form_flat_f32(DSpace s, Range r, int tp_model, guide_outputs o) {
+    const u64 j = (u64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= r.count) return;
+    const Cfg c = decode_index(s, r.first + j);
+    Metrics m;
+    closed_form_eval_f32<TIME_SUM>(s, s.ratef, c, tp_model, m);
+    store_metrics(o, j, m);
+}
+
 // Tiled evaluation (see tiled.cuh): every valid config's metrics are stored.
 template <int TIME_SUM>
 __global__ void __launch_bounds__(256, 2) k_closed_form_tiled(DSpace s, Range r, int tp_model, u32 hf_chunk,
@@ -363,6 +374,15 @@ static int launch_split(const DSpace &s, int tp_model, const guide_outputs &o, c
         cfg.gridDim = dim3((u32)num_sms() * MODEL_BLOCKS_PER_SM); cfg.dynamicSmemBytes = 0;
         GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_closed_form_model<TIME_SUM>, s, tp_model, o, n_chunks, ticket));
     }
+    return GUIDE_OK;
+}
+
+int launch_closed_form_f32(const DSpace &s, Range r, int time_model, int tp_model, const guide_outputs &o, cudaStream_t st) {
+    const u64 blocks = (r.count + 255) / 256;
+    if (blocks > 0x7FFFFFFFull) return fail(GUIDE_ERR_UNSUPPORTED, "range too large for one launch");
+    if (time_model) k_closed_form_flat_f32<1><<<(u32)blocks, 256, 0, st>>>(s, r, tp_model, o);
+    else k_closed_form_flat_f32<0><<<(u32)blocks, 256, 0, st>>>(s, r, tp_model, o);
+    GUIDE_CUDA(cudaGetLastError());
     return GUIDE_OK;
 }
 

@@ -101,7 +101,7 @@ static int check_trace_overflow(const guide_space &s, const guide_trace &t) {
 // Derived per-model quantities and the reciprocal rates of every hardware x framework pair.
 __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *gh, u32 n_h, const guide_fw *gf,
                                u32 n_f, const u32 *tp, const u32 *dp, u32 n_t, DModel *dm, DRate *dr, double *cost_hr,
-                               double *cost_sec, ulonglong2 *hfmem, double *rate10, StageConst *stage_consts) {
+                               double *cost_sec, ulonglong2 *hfmem, double *rate10, StageConst *stage_consts, RateF *ratef) {
     const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n_m) {
         const guide_model m = gm[i];
@@ -138,6 +138,15 @@ __global__ void k_build_tables(const guide_model *gm, u32 n_m, const guide_hw *g
         r.keep = (f.kv_keep_permille == 0 || f.kv_keep_permille >= 1000) ? 1000u : f.kv_keep_permille;
         dr[i] = r;
         hfmem[i] = make_ulonglong2(r.usable, (u64)r.kv_block);
+        RateF rf;
+        for (int k = 0; k < 3; k++) {
+            rf.inv_c[k] = 1.0f / ((float)h.peak_flops * (float)f.e_c[k]);
+            rf.inv_m[k] = 1.0f / ((float)h.mem_bw * (float)f.e_m[k]);
+        }
+        rf.inv_comm = 1.0f / ((float)h.comm_bw * (float)f.e_comm);
+        rf.clat = (float)h.comm_lat; rf.tovh = (float)f.t_ovh; rf.price = (float)h.price_per_hr;
+        rf.flash = f.flash; rf.pad = 0;
+        ratef[i] = rf;
         double *q = rate10 + (size_t)i * 10;
         for (int k = 0; k < 3; k++) { q[k] = r.inv_c[k]; q[3 + k] = r.inv_m[k]; }
         q[6] = r.inv_comm; q[7] = r.clat; q[8] = r.tovh; q[9] = r.flash ? 1.0 : 0.0;
@@ -248,7 +257,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket, cudaStream_t
                  o_po = take(std::max<size_t>(n_m * (s->tp.size() * s->pairs.size() / 4), 1) * 4),
                  o_lo = take(std::max<size_t>(n_m * (s->tp.size() * s->pairs.size() / 16), 1) * 4),
                  o_tk = take(TICKET_SLOTS * 128), o_r10 = take(n_h * n_f * 80),
-                 o_sc = take((s->tp.size() + 1) * n_m * sizeof(StageConst));
+                 o_sc = take((s->tp.size() + 1) * n_m * sizeof(StageConst)), o_rf = take(n_h * n_f * sizeof(RateF));
     char *blob = nullptr;
     GUIDE_CUDA(cudaMalloc(&blob, off));
     cudaError_t e = cudaSuccess;
@@ -276,7 +285,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket, cudaStream_t
                                                  (DModel *)(blob + o_dm), (DRate *)(blob + o_dr),
                                                  (double *)(blob + o_ch), (double *)(blob + o_cs),
                                                  (ulonglong2 *)(blob + o_hm), (double *)(blob + o_r10),
-                                                 (StageConst *)(blob + o_sc));
+                                                 (StageConst *)(blob + o_sc), (RateF *)(blob + o_rf));
         e = cudaGetLastError();
         // the host arrays must outlive the copies, and another stream may use the tables next
         if (e == cudaSuccess) e = cudaStreamSynchronize(st);
@@ -298,6 +307,7 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket, cudaStream_t
     d.view.hfmem = (const ulonglong2 *)(blob + o_hm);
     d.view.rate10 = (const double *)(blob + o_r10);
     d.view.stage_consts = (const StageConst *)(blob + o_sc);
+    d.view.ratef = (const RateF *)(blob + o_rf);
     d.view.hf_sorted = (const HfSorted *)(blob + o_hs);
     d.view.plane_order = (const u32 *)(blob + o_po);
     d.view.line_order = (const u32 *)(blob + o_lo);
@@ -352,6 +362,7 @@ static int resolve_range(const guide_space *s, const guide_sim_opts *o, Range *r
     if (o && (o->time_model < 0 || o->time_model > 1 || o->tp_model < 0 || o->tp_model > 1))
         return fail(GUIDE_ERR_INVALID, "unknown time_model or tp_model");
     if (o && (o->clamp_seq < 0 || o->clamp_seq > 1)) return fail(GUIDE_ERR_INVALID, "clamp_seq must be 0 or 1");
+    if (o && o->precision != GUIDE_PREC_F64 && o->precision != GUIDE_PREC_F32) return fail(GUIDE_ERR_INVALID, "unknown precision");
     return GUIDE_OK;
 }
 
@@ -587,6 +598,9 @@ int guide_simulate(const guide_space *space_c, const guide_trace *trace_c, const
     if (!trace && (out->req_ttft || out->req_tpot))
         return fail(GUIDE_ERR_INVALID, "per-request outputs need a trace");
     if (trace) {
+        if (opts && opts->precision == GUIDE_PREC_F32)
+            return fail(GUIDE_ERR_UNSUPPORTED, "the binary32 variant covers the closed form only: a trace simulation sums its clock over "
+                                               "too many iterations for admission decisions to survive the rounding");
         if (opts && opts->clamp_seq)
             return fail(GUIDE_ERR_UNSUPPORTED, "clamp_seq cuts the lengths of a closed-form config; a trace fixes the lengths of its requests");
         if (space->evicting)
@@ -618,6 +632,8 @@ int guide_simulate(const guide_space *space_c, const guide_trace *trace_c, const
         // options and outputs only the one-thread-per-config evaluation knows: keep the whole-space kernels out
         if ((opts && opts->clamp_seq) || out->seq_used) ds.chunked = 1;
         ds.clamp_seq = opts ? (u32)opts->clamp_seq : 0u;
+        if (opts && opts->precision == GUIDE_PREC_F32)
+            return launch_closed_form_f32(ds, r, time_model, tp_model, *out, (cudaStream_t)stream);
         return launch_closed_form(ds, r, time_model, tp_model, *out, ticket, (cudaStream_t)stream);
     }
     DTrace dt;
@@ -648,6 +664,8 @@ int guide_select_topk(const guide_space *space_c, const guide_trace *trace, cons
     DSpace ds;
     unsigned *ticket = nullptr;                  // the fused path's model walk takes its work items through it
     if ((rc = space_on_device(space, &ds, outputs ? nullptr : &ticket, (cudaStream_t)stream))) return rc;
+    if (!outputs && opts && opts->precision == GUIDE_PREC_F32)
+        return fail(GUIDE_ERR_UNSUPPORTED, "the fused selection evaluates in binary64: run guide_simulate with the binary32 option and select on its outputs");
     if (!outputs && opts && opts->clamp_seq) { ds.chunked = 1; ds.clamp_seq = 1; }     // fused: evaluated with the option
     return launch_topk(ds, r, outputs, opts ? opts->time_model : 0, opts ? opts->tp_model : 0, *cons, key, k,
                        (u64 *)idx_out, key_out, count_out, ws, ticket, (cudaStream_t)stream);
@@ -667,6 +685,8 @@ int guide_pareto(const guide_space *space_c, const guide_trace *trace, const gui
     DSpace ds;
     unsigned *ticket = nullptr;
     if ((rc = space_on_device(space, &ds, outputs ? nullptr : &ticket, (cudaStream_t)stream))) return rc;
+    if (!outputs && opts && opts->precision == GUIDE_PREC_F32)
+        return fail(GUIDE_ERR_UNSUPPORTED, "the fused selection evaluates in binary64: run guide_simulate with the binary32 option and select on its outputs");
     if (!outputs && opts && opts->clamp_seq) { ds.chunked = 1; ds.clamp_seq = 1; }
     return launch_pareto(ds, r, outputs, opts ? opts->time_model : 0, opts ? opts->tp_model : 0, *cons, xm, ym,
                          (u64 *)idx_out, cap, count_out, ws, ticket, (cudaStream_t)stream);

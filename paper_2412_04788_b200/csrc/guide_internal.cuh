@@ -8,6 +8,7 @@
 
 #include "../../include/guide.h"
 #include "model.cuh"
+#include "model_f32.cuh"
 #include "tiled.cuh"
 
 namespace guide {
@@ -71,6 +72,7 @@ int trace_on_device(guide_trace *t, DTrace *out, cudaStream_t st);
 // closed_form.cu
 int launch_closed_form(const DSpace &s, Range r, int time_model, int tp_model, const guide_outputs &o,
                        unsigned *ticket, cudaStream_t st);
+int launch_closed_form_f32(const DSpace &s, Range r, int time_model, int tp_model, const guide_outputs &o, cudaStream_t st);
 // trace_sim.cu
 // What the host knows about the configs the one-lane-per-config kernel would take: per class of max
 // batch, how many configs of the whole space have a prompt-first framework with a block size the

@@ -46,6 +46,7 @@ struct HfSorted {
 };
 
 struct StageConst;
+struct RateF;
 
 struct DSpace {
     const DModel *models;
@@ -57,6 +58,7 @@ struct DSpace {
     const double *cost_sec;      // [n_h * n_f][n_t]: (price x TP degree) / 3600
     const ulonglong2 *hfmem;     // [n_h * n_f]: x = usable bytes, y = KV block size (what the memory check reads)
     const StageConst *stage_consts;   // [n_t + 1][n_m]: the task-table factors per (TP degree, model); the last group is t = 1
+    const RateF *ratef;          // [n_h * n_f]: the rates in binary32 (reduced-precision variant of the closed form)
     const double *rate10;        // [n_h * n_f][10]: inv_c[3], inv_m[3], inv_comm, clat, tovh, flash (0.0 or 1.0); 16-byte aligned rows
     // Orders that only steer which thread does what (any permutation gives the same results):
     const HfSorted *hf_sorted;   // [n_h * n_f]: the pairs grouped by KV block size, largest usable memory first

@@ -74,7 +74,7 @@ class Config(C.Structure):
 
 class SimOpts(C.Structure):
     _fields_ = [("first", C.c_uint64), ("count", C.c_uint64), ("time_model", C.c_int32), ("tp_model", C.c_int32),
-                ("max_iters", C.c_uint64), ("clamp_seq", C.c_int32), ("reserved", C.c_int32)]
+                ("max_iters", C.c_uint64), ("clamp_seq", C.c_int32), ("precision", C.c_int32)]
 
 
 class Outputs(C.Structure):
@@ -208,8 +208,11 @@ class Trace:
             pass
 
 
-def _opts(first=0, count=0, time_model=TIME_MAX, tp_model=TP_EXPLICIT, max_iters=0, clamp_seq=False):
-    return SimOpts(first, count, time_model, tp_model, max_iters, int(bool(clamp_seq)), 0)
+PREC_F64, PREC_F32 = 0, 1
+
+
+def _opts(first=0, count=0, time_model=TIME_MAX, tp_model=TP_EXPLICIT, max_iters=0, clamp_seq=False, precision=PREC_F64):
+    return SimOpts(first, count, time_model, tp_model, max_iters, int(bool(clamp_seq)), precision)
 
 
 def _cons(cons):
@@ -252,10 +255,10 @@ def guide_workspace_bytes(space: Space, trace: Trace | None) -> int:
 
 
 def guide_simulate(space: Space, trace: Trace | None, out: dict, first=0, count=0, time_model=TIME_MAX,
-                   tp_model=TP_EXPLICIT, max_iters=0, workspace=None, stream=None, clamp_seq=False):
+                   tp_model=TP_EXPLICIT, max_iters=0, workspace=None, stream=None, clamp_seq=False, precision=PREC_F64):
     """out: dict of torch CUDA tensors (see alloc_outputs); workspace: torch uint8 CUDA tensor or None."""
     o = _outputs_struct(out)
-    opts = _opts(first, count, time_model, tp_model, max_iters, clamp_seq)
+    opts = _opts(first, count, time_model, tp_model, max_iters, clamp_seq, precision)
     ws_ptr = _ptr(workspace)
     ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
     _check(lib().guide_simulate(space.handle, trace.handle if trace else None, C.byref(opts), C.byref(o), ws_ptr,
@@ -272,10 +275,10 @@ def guide_pareto_workspace_bytes(space: Space) -> int:
 
 def guide_select_topk(space: Space, trace: Trace | None, out: dict | None, cons: dict | None, key: str, k: int,
                       idx_out, key_out, count_out, workspace, first=0, count=0, time_model=TIME_MAX,
-                      tp_model=TP_EXPLICIT, stream=None, clamp_seq=False):
+                      tp_model=TP_EXPLICIT, stream=None, clamp_seq=False, precision=PREC_F64):
     """idx_out int64[k], key_out float64[k], count_out int32[1], workspace uint8: torch CUDA tensors."""
     o = _outputs_struct(out) if out is not None else None
-    opts = _opts(first, count, time_model, tp_model, 0, clamp_seq)
+    opts = _opts(first, count, time_model, tp_model, 0, clamp_seq, precision)
     cs = _cons(cons)
     _check(lib().guide_select_topk(space.handle, trace.handle if trace else None, C.byref(o) if o is not None else None,
                                    C.byref(opts), C.byref(cs), METRICS[key], k, _ptr(idx_out), _ptr(key_out),

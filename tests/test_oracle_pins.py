@@ -391,6 +391,37 @@ def test_sequence_cut_to_what_fits(golden):
         oracle.simulate(toy_space(golden, 10**6, 1, [2]), tr, clamp_seq=True)
 
 
+def test_binary32_variant(golden):
+    """The reduced-precision variant of the closed form (every operation of the model in binary32): the
+    hand-worked toy values are dyadic with few bits, so they must come out bit for bit here too; on a
+    sweep it stays within 1e-5 of the binary64 result (about sixty rounded operations of 6e-8 each on
+    sums of positive terms); integer outputs do not depend on the precision."""
+    want = golden["closed_form_b2_Lin4_Lout3"]["t1"]
+    out = oracle.simulate(toy_space(golden, 10**6, 1, [2], tp=(1, 2)), precision="f32")
+    assert out["ttft"][0] == want["ttft"] and out["latency"][0] == want["latency"] and out["tpot"][0] == want["tpot"]
+    assert out["thr_decode"][0] == float(np.float32(want["thr_decode_num"]) / np.float32(want["thr_decode_den"]))
+    for row in golden["kv_reduction_and_clamp"]["decode"]["rows"]:
+        o = oracle.simulate(toy_space(golden, 10**6, 1, [2], keep=row["p"]), precision="f32")
+        assert o["latency"][0] == row["latency"] and o["tpot"][0] == row["tpot"]
+    w = I.workload(2, scale=0.25)
+    a = oracle.simulate(w["space"])
+    b = oracle.simulate(w["space"], precision="f32")
+    for k in ("status", "bmax", "n_iters", "n_req_iters", "seq_used"):
+        assert np.array_equal(a[k], b[k]), k
+    ok = a["status"] == 0
+    worst = 0.0
+    for k in oracle.F64_FIELDS:
+        assert np.array_equal(np.isinf(a[k]), np.isinf(b[k])), k
+        fin = ok & np.isfinite(a[k]) & (a[k] != 0)
+        assert np.array_equal(b[k][fin], b[k][fin].astype(np.float32).astype(np.float64)), k     # binary32 values
+        rel = np.abs(b[k][fin] - a[k][fin]) / np.abs(a[k][fin])
+        worst = max(worst, float(rel.max()))
+    assert 1e-9 < worst <= 1e-5, worst          # really rounded, and within the bar
+    with pytest.raises(AssertionError):
+        tr = {"arrival": np.array([0.0]), "in_len": np.zeros(1, np.uint32), "out_len": np.zeros(1, np.uint32)}
+        oracle.simulate(toy_space(golden, 10**6, 1, [2]), tr, precision="f32")
+
+
 def test_paper_log2_rule(golden):
     """Sec. 3.2: multi-GPU throughput = N T_single / (1 + log2 P_TP)."""
     model = list(golden["model"])
