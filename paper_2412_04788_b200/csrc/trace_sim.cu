@@ -747,16 +747,22 @@ static int plan_lanes(const DSpace &s, const LaneHints &h, Range r, u32 cls, Lan
     // configs of this launch among the range: all of the class for a whole space, else at most the range
     const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
     const u64 mine = r.count == total ? h.class_configs[cls] : std::min<u64>(r.count, h.class_configs[cls]);
-    // Few configs: spread them over more warps, fewer lanes each (a lane's pace does not depend on its
-    // neighbours, a warp's issue slots are shared by them).  Aim at eight warps per SM.
-    const u64 lanes = (mine + (u64)num_sms() * 8 - 1) / ((u64)num_sms() * 8);
+    // The kernel is bound by the latency of each lane's own chain, so warps are worth more than lanes:
+    // as few lanes per warp as still lets every config be resident at once (fewer lanes also need less
+    // shared memory per block, so more blocks fit; two rounds settle that).
+    const LaneKernel kern = lane_kernel<TIME_SUM>(c.unroll);
     const u64 fit = LANE_SMEM_LIMIT / lane_block_smem(c, 1, h.hist_n);      // lanes whose slots fit a block's shared memory (>= 8)
-    p->lanes_used = (u32)std::max<u64>(1, std::min<u64>(std::min<u64>(c.lanes, fit), lanes));
+    u64 lanes = std::min<u64>(c.lanes, fit), resident_warps = 1;
+    for (int round = 0; round < 3; round++) {
+        int per_sm = 0;
+        GUIDE_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, LANE_BLOCK_WARPS * 32,
+                                                                 lane_block_smem(c, (u32)lanes, h.hist_n)));
+        if (per_sm < 1) per_sm = 1;
+        resident_warps = std::min<u64>((u64)num_sms() * per_sm * LANE_BLOCK_WARPS, LANE_MAX_WARPS);
+        lanes = std::max<u64>(1, std::min<u64>(std::min<u64>(c.lanes, fit), (mine + resident_warps - 1) / resident_warps));
+    }
+    p->lanes_used = (u32)lanes;
     p->smem = lane_block_smem(c, p->lanes_used, h.hist_n);
-    int per_sm = 0;
-    GUIDE_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, lane_kernel<TIME_SUM>(c.unroll), LANE_BLOCK_WARPS * 32, p->smem));
-    if (per_sm < 1) per_sm = 1;
-    const u64 resident_warps = std::min<u64>((u64)num_sms() * per_sm * LANE_BLOCK_WARPS, LANE_MAX_WARPS);
     const u64 warps = std::min<u64>(resident_warps, (mine + p->lanes_used - 1) / p->lanes_used);
     p->blocks = (u32)((warps + LANE_BLOCK_WARPS - 1) / LANE_BLOCK_WARPS);
     return GUIDE_OK;
