@@ -678,8 +678,13 @@ k_trace_lanes(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, gui
 struct LaneClass { u32 minb, maxb, lanes, round, unroll; };
 static const LaneClass LANE_CLASSES[LANE_N_CLASSES] = {{1, 16, 32, 64, 4}, {17, 64, 32, 16, 1}, {65, GUIDE_TRACE_MAX_BATCH, 8, 8, 1}};
 #ifndef LANE_CLASSES_ENABLED
-#define LANE_CLASSES_ENABLED 1      // classes above this go to the warp-per-config kernel
+#define LANE_CLASSES_ENABLED 2      // classes from this one on always go to the warp-per-config kernel
 #endif
+// A class above the first is launched only when it has at least this many configs: the lane kernel is
+// bound by the latency of each lane's chain and needs several waves of configs to pay for the slot
+// scans it does one lane at a time (measured: max batch 24-64 on workload 4, 262,144 configs, 117 ms
+// against about 220 ms in the warp-per-config kernel; on workload 3, 16,384 configs, 259 against 170 ms).
+static constexpr u64 LANE_CLASS_MIN_CONFIGS = (u64)LANE_MAX_WARPS * 32;
 
 typedef void (*LaneKernel)(DSpace, DTrace, Range, int, u64, guide_outputs, unsigned long long *, unsigned char *, size_t, u32, u32,
                            int, u32, u32, u32, u32, u32);
@@ -708,6 +713,11 @@ LaneHints lane_hints(const guide_space &s) {
     for (uint32_t b : s.batch)
         for (u32 c = 0; c < n_classes; c++)
             if (b >= LANE_CLASSES[c].minb && b <= LANE_CLASSES[c].maxb) h.class_configs[c] += per_b;
+    // classes are taken from the first one up, without gaps: the warp-per-config kernel leaves out
+    // every max batch up to the last launched class's limit
+    for (u32 c = 1; c < LANE_N_CLASSES; c++)
+        if (h.class_configs[c] < LANE_CLASS_MIN_CONFIGS)
+            for (u32 d = c; d < LANE_N_CLASSES; d++) h.class_configs[d] = 0;
     return h;
 }
 
