@@ -690,7 +690,8 @@ typedef void (*LaneKernel)(DSpace, DTrace, Range, int, u64, guide_outputs, unsig
                            int, u32, u32, u32, u32, u32);
 template <int TIME_SUM>
 static LaneKernel lane_kernel(u32 unroll) {
-    return unroll == 4 ? (LaneKernel)k_trace_lanes<TIME_SUM, 4> : (LaneKernel)k_trace_lanes<TIME_SUM, 1>;
+    return unroll == 4 ? (LaneKernel)k_trace_lanes<TIME_SUM, 4>
+           : unroll == 1 ? (LaneKernel)k_trace_lanes<TIME_SUM, 1> : (LaneKernel)k_trace_lanes<TIME_SUM, 0>;
 }
 static constexpr u32 LANE_BLOCK_WARPS = 4;
 static constexpr size_t LANE_SMEM_LIMIT = 112 * 1024;
@@ -710,14 +711,24 @@ LaneHints lane_hints(const guide_space &s) {
             h.hist_n = std::max(h.hist_n, f.kv_block);
         }
     const u64 per_b = (u64)s.models.size() * s.hw.size() * n_fw * s.tp.size() * s.pairs.size();
+    u64 all[LANE_N_CLASSES] = {}, total = 0;
     for (uint32_t b : s.batch)
-        for (u32 c = 0; c < n_classes; c++)
-            if (b >= LANE_CLASSES[c].minb && b <= LANE_CLASSES[c].maxb) h.class_configs[c] += per_b;
-    // classes are taken from the first one up, without gaps: the warp-per-config kernel leaves out
-    // every max batch up to the last launched class's limit
-    for (u32 c = 1; c < LANE_N_CLASSES; c++)
-        if (h.class_configs[c] < LANE_CLASS_MIN_CONFIGS)
-            for (u32 d = c; d < LANE_N_CLASSES; d++) h.class_configs[d] = 0;
+        for (u32 c = 0; c < LANE_N_CLASSES; c++)
+            if (b >= LANE_CLASSES[c].minb && b <= LANE_CLASSES[c].maxb) { all[c] += per_b; total += per_b; }
+    if (total <= LANE_MAX_WARPS) {
+        // a space this small gives every config a warp of its own (one lane each): the launch lasts as
+        // long as its longest schedule whatever the max batch, and one kernel does it all
+        h.class_configs[0] = total;
+        h.single = 1;
+        return h;
+    }
+    // Otherwise classes are taken from the first one up, without gaps (the warp-per-config kernel leaves
+    // out every max batch up to the last launched class's limit), the later ones only when they are
+    // large enough to pay.
+    for (u32 c = 0; c < n_classes; c++) {
+        if (c > 0 && all[c] < LANE_CLASS_MIN_CONFIGS) break;
+        h.class_configs[c] = all[c];
+    }
     return h;
 }
 
@@ -727,7 +738,7 @@ LaneHints lane_hints(const guide_space &s) {
 size_t trace_workspace_bytes(u32 n_req, const LaneHints &hints) {
     size_t slices = SIM_MAX_WARPS;
     for (u32 c = 0; c < LANE_N_CLASSES; c++) {
-        const u64 lanes = LANE_CLASSES[c].lanes;
+        const u64 lanes = hints.single ? 1 : LANE_CLASSES[c].lanes;
         slices = std::max<size_t>(slices, std::min<u64>((u64)LANE_MAX_WARPS * lanes,
                                                         hints.class_configs[c] + LANE_BLOCK_WARPS * lanes));
     }
@@ -736,9 +747,11 @@ size_t trace_workspace_bytes(u32 n_req, const LaneHints &hints) {
 
 struct LanePlan { u32 blocks, lanes_used; size_t smem; };
 
+static const LaneClass LANE_SINGLE = {1, GUIDE_TRACE_MAX_BATCH, 1, 64, 0};     // small spaces: one lane per warp, every max batch
+
 template <int TIME_SUM>
 static int plan_lanes(const DSpace &s, const LaneHints &h, Range r, u32 cls, LanePlan *p) {
-    const LaneClass &c = LANE_CLASSES[cls];
+    const LaneClass &c = h.single ? LANE_SINGLE : LANE_CLASSES[cls];
     p->blocks = 0; p->lanes_used = c.lanes; p->smem = 0;
     if (h.class_configs[cls] == 0) return GUIDE_OK;
     static std::mutex mu;
@@ -748,7 +761,7 @@ static int plan_lanes(const DSpace &s, const LaneHints &h, Range r, u32 cls, Lan
     {
         std::lock_guard<std::mutex> lock(mu);
         if (dev < 64 && !opted[dev]) {
-            for (u32 u : {1u, 4u})
+            for (u32 u : {0u, 1u, 4u})
                 GUIDE_CUDA(cudaFuncSetAttribute(lane_kernel<TIME_SUM>(u), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                 (int)LANE_SMEM_LIMIT));
             opted[dev] = true;
@@ -806,7 +819,8 @@ static int launch_one(const DSpace &s, const DTrace &t, Range r, int tp_model, u
         return fail(GUIDE_ERR_WORKSPACE, "workspace too small for the resident warps");
     if (policies & 1) {
         u32 lane_maxb = 0;
-        for (u32 cls = 0; cls < LANE_N_CLASSES; cls++) {
+        for (u32 cls = 0; cls < (hints.single ? 1u : LANE_N_CLASSES); cls++) {
+            const LaneClass &lc = hints.single ? LANE_SINGLE : LANE_CLASSES[cls];
             LanePlan lp;
             int rc = plan_lanes<TIME_SUM>(s, hints, r, cls, &lp);
             if (rc) return rc;
@@ -815,11 +829,12 @@ static int launch_one(const DSpace &s, const DTrace &t, Range r, int tp_model, u
             if (256 + (size_t)lp.blocks * LANE_BLOCK_WARPS * lp.lanes_used * pw > ws_bytes)
                 return fail(GUIDE_ERR_WORKSPACE, "workspace too small for the lane kernel's %u blocks", lp.blocks);
             GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
-            lane_kernel<TIME_SUM>(LANE_CLASSES[cls].unroll)<<<lp.blocks, LANE_BLOCK_WARPS * 32, lp.smem, st>>>(
+            // one lane per warp: the run loop that skips from one block need to the next (unroll 0)
+            lane_kernel<TIME_SUM>(lp.lanes_used == 1 ? 0u : lc.unroll)<<<lp.blocks, LANE_BLOCK_WARPS * 32, lp.smem, st>>>(
                 s, t, r, tp_model, max_iters, o, (unsigned long long *)ws, scratch, pw, gen_bytes, first_bytes, reorder,
-                LANE_CLASSES[cls].minb, LANE_CLASSES[cls].maxb, hints.hist_n, lp.lanes_used, LANE_CLASSES[cls].round);
+                lc.minb, lc.maxb, hints.hist_n, lp.lanes_used, lc.round);
             GUIDE_CUDA(cudaGetLastError());
-            lane_maxb = std::max(lane_maxb, LANE_CLASSES[cls].maxb);
+            lane_maxb = std::max(lane_maxb, lc.maxb);
         }
         // always launched: the lane kernel leaves it the configs whose counts do not stay below 2^53
         // or whose block size the phase histogram does not cover
