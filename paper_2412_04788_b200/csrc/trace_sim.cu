@@ -684,7 +684,10 @@ static const LaneClass LANE_CLASSES[LANE_N_CLASSES] = {{1, 16, 32, 64, 4}, {17, 
 // bound by the latency of each lane's chain and needs several waves of configs to pay for the slot
 // scans it does one lane at a time (measured: max batch 24-64 on workload 4, 262,144 configs, 117 ms
 // against about 220 ms in the warp-per-config kernel; on workload 3, 16,384 configs, 259 against 170 ms).
-static constexpr u64 LANE_CLASS_MIN_CONFIGS = (u64)LANE_MAX_WARPS * 32;
+#ifndef LANE_CLASS_MIN_CONFIGS_DEF
+#define LANE_CLASS_MIN_CONFIGS_DEF ((u64)LANE_MAX_WARPS * 32)
+#endif
+static constexpr u64 LANE_CLASS_MIN_CONFIGS = LANE_CLASS_MIN_CONFIGS_DEF;
 
 typedef void (*LaneKernel)(DSpace, DTrace, Range, int, u64, guide_outputs, unsigned long long *, unsigned char *, size_t, u32, u32,
                            int, u32, u32, u32, u32, u32);
