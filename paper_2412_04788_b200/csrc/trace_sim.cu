@@ -28,6 +28,10 @@
 
 namespace guide {
 
+#ifndef SIM_MIN_BLOCKS
+#define SIM_MIN_BLOCKS 2          // resident blocks per SM k_trace_sim is compiled for (128 registers, no spills: it keeps the
+                                  // event-heavy large batches now; 3 blocks of 80 registers measured 3 % slower)
+#endif
 static constexpr u32 SIM_WARPS_PER_BLOCK = 8;
 static constexpr u32 SIM_THREADS = SIM_WARPS_PER_BLOCK * 32;
 static constexpr u32 SIM_MAX_WARPS = 6144;        // workspace is sized for this many resident warps
@@ -166,7 +170,7 @@ __device__ __forceinline__ void write_trace_results(const guide_outputs &o, u64 
 }
 
 template <int TIME_SUM>
-__global__ void __launch_bounds__(SIM_THREADS, 3)
+__global__ void __launch_bounds__(SIM_THREADS, SIM_MIN_BLOCKS)
 k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide_outputs o, u32 *counter,
             unsigned char *scratch, size_t per_warp, u32 gen_bytes, u32 first_bytes, int reorder, u32 lane_maxb, u32 lane_hist) {
     __shared__ SlotArrays sh[SIM_WARPS_PER_BLOCK];
