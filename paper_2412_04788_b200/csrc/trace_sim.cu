@@ -241,6 +241,7 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         u32 dc_n = 0;
         double dc_fix = 0.0, dc_comm = 0.0, dc_head = 0.0, dc_tha = 0.0, dc_nd = 0.0;
         u64 dc_tha_i = 0;
+        u64 pre_T = 0, pre_A = 0;        // prompt tokens (and their squares) admitted since the last prompt pass
         // the head of the waiting queue: its arrival time and the blocks it needs
         double arr_next = 0.0;
         u32 need_next = 0;
@@ -275,6 +276,7 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                         sl.fin[nrun] = out - g;
                         sl.meta[nrun] = (unsigned char)(M_NEEDS_PREFILL | (g == 0 ? M_FIRST : 0u));
                     }
+                    pre_T += (u64)(in + g); pre_A += (u64)(in + g) * (in + g);
                     nrun++; n_new++; next++;
                     if (next > high_water) high_water = next;
                     refresh_head();
@@ -292,15 +294,8 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
             // ---- 3./4. build the iteration (prompts first, everything else stalls) and advance the clock ----
             bool any_done;
             if (n_new > 0) {
-                u64 T = 0, A = 0;
-                for (u32 base = 0; base < nrun; base += 32) {
-                    const u32 k = base + lane;
-                    if (k < nrun && (sl.meta[k] & M_NEEDS_PREFILL)) {
-                        const u64 q = sl.base[k];
-                        T += q; A += q * q;
-                    }
-                }
-                T = warp_sum(T); A = warp_sum(A);
+                const u64 T = pre_T, A = pre_A;          // summed at admission: tokens and tokens squared of the new prompts
+                pre_T = 0; pre_A = 0;
                 double t_iter;
                 {
                     TaskTab kt;
@@ -310,7 +305,7 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                 }
                 const double after = clock + t_iter;
                 u32 local_min = NO_COMPLETION;
-                for (u32 base = 0; base < nrun; base += 32) {
+                for (u32 base = nrun - n_new; base < nrun; base += 32) {     // admissions append: the new ones are the last slots
                     const u32 k = base + lane;
                     if (k < nrun) {
                         const u32 mt = sl.meta[k];
