@@ -79,7 +79,7 @@ int launch_closed_form_f32(const DSpace &s, Range r, int time_model, int tp_mode
 // phase histogram covers (an upper bound: the kernel itself also checks that the config's integer
 // counts stay below 2^53), and the largest such block size.
 static constexpr unsigned LANE_N_CLASSES = 3;
-struct LaneHints { u64 class_configs[LANE_N_CLASSES]; u32 hist_n; u32 single; };   // single: one launch, one lane per warp, every max batch
+struct LaneHints { u64 class_configs[LANE_N_CLASSES]; u32 hist_n; };
 LaneHints lane_hints(const guide_space &s);
 size_t trace_workspace_bytes(u32 n_req, const LaneHints &hints);
 int launch_trace_sim(const DSpace &s, const DTrace &t, Range r, int time_model, int tp_model, u64 max_iters,

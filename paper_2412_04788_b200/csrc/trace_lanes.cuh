@@ -1,12 +1,13 @@
 // Trace-driven simulation with one LANE per config (prompt-first policy), for configs whose max batch
-// is small.  Those are the long schedules - with a max batch of 1 every output token of the trace is
-// its own iteration - and the iteration itself is one scalar chain of two dozen fp64 operations that
-// touches no request, so a warp that steps one config spends 31 of its lanes repeating the same
-// numbers.  Here every lane of a warp steps its own config.
+// is small, when a space has enough of them to fill most lanes of every resident warp.  Those are the
+// long schedules - with a max batch of 1 every output token of the trace is its own iteration - and
+// a scheduler event (admission, prompt pass, completion) handles one or two requests, so a warp that
+// steps one config has most of its lanes idle at events.  Here every lane of a warp steps its own config.
 //
 // A warp alternates between two phases so that its lanes stay on the same instructions:
 //   - run: every lane that is between events advances its config by up to round_len decode iterations
-//     (the same pipelined loop as in the warp-per-config kernel, same operations in the same order);
+//     (one scalar chain per lane; the clock is advanced by the same additions in the same order as in
+//     the warp-per-config kernel);
 //   - events: every lane whose run ended (a completion, a block shortage, room for the head of the
 //     queue) makes scheduler passes - settle the run, retire, admit, a prompt pass, evictions, refresh
 //     of the cached stage terms - until it is ready to run again or its trace is finished.
@@ -117,7 +118,6 @@ struct LaneState {
     u64 dec_tok, n_iters, n_req_iters, free_blocks, csum;
     u64 pre_T, pre_A;                         // prompt tokens (and their squares) admitted since the last prompt pass
     u32 next, high_water, nheap, n_new, D, Dmod;
-    u64 nzmask;                               // bit p set: some resident has (cache - D) mod block == p (histogram bin not empty)
     u32 need_next, dc_n;
     double arr_next;
     double dc_fix, dc_comm, dc_head, dc_tha, dc_nd;   // decode-stage terms that depend on the resident count only
@@ -196,7 +196,7 @@ __device__ __forceinline__ void lane_retire(LaneState &L, const LaneEnv &e) {
         L.csum -= cv;
         if (L.blk > 1) {
             const u32 ph = (rqm >> LS_PHASE_SHIFT) & LS_PHASE_MASK;
-            if ((SL(s_hist, ph) -= 1) == 0) L.nzmask &= ~(1ull << ph);
+            SL(s_hist, ph) -= 1;
         }
         L.nheap--;
         if (L.nheap > 0) lane_sift_down(e, L.nheap, L.D, 0, SL(s_fin, L.nheap), SL(s_base, L.nheap), SL(s_rqm, L.nheap));
@@ -265,7 +265,6 @@ __device__ __forceinline__ void lane_sched_body(LaneState &L, const LaneEnv &e) 
                 ph = q - div_small(q, L.blk, L.magic) * L.blk + L.blk - L.Dmod;     // (cache - D) mod block
                 if (ph >= L.blk) ph -= L.blk;
                 SL(s_hist, ph) += 1;
-                L.nzmask |= 1ull << ph;
             }
             lane_sift_up(e, L.D, L.nheap, L.D + left, q - L.D, rq | (ph << LS_PHASE_SHIFT));
             L.nheap++;
@@ -299,7 +298,7 @@ __device__ __forceinline__ void lane_sched_body(LaneState &L, const LaneEnv &e) 
             e.gen[vrq] = out - rem;
             if (L.blk > 1) {
                 const u32 ph = (rqm >> LS_PHASE_SHIFT) & LS_PHASE_MASK;
-                if ((SL(s_hist, ph) -= 1) == 0) L.nzmask &= ~(1ull << ph);
+                SL(s_hist, ph) -= 1;
             }
             L.nheap--;
             if (v < L.nheap) {                               // the last entry takes the hole, then finds its level
@@ -387,7 +386,7 @@ __device__ __noinline__ void lane_start_config(LaneState *Lp, const LaneEnv *ep,
     L.clock = 0.0; L.dec_time = 0.0; L.csum_d = 0.0;
     L.dec_tok = 0; L.n_iters = 0; L.n_req_iters = 0; L.free_blocks = blocks_total; L.csum = 0;
     L.next = 0; L.high_water = 0; L.nheap = 0; L.n_new = 0; L.D = 0; L.Dmod = 0;
-    L.dc_n = 0; L.in_run = 0; L.pre_T = 0; L.pre_A = 0; L.nzmask = 0;
+    L.dc_n = 0; L.in_run = 0; L.pre_T = 0; L.pre_A = 0;
     L.max_iters = lp->max_iters_opt ? lp->max_iters_opt : 64 * (tr.sum_out + (u64)tr.n_zero * pr.y) + 4 * (u64)tr.n;
     if (st) { L.mode = LM_FINISHED; return; }
     for (u32 i = 0; i < lp->hist_n; i++) SL(s_hist, i) = 0;
@@ -496,72 +495,6 @@ __device__ __forceinline__ void lanes_simulate(const DSpace &s, const DTrace &tr
                     LANE_APPLY(tcur, ctxd)
                     tcur = t1; ctxd = c1;
                     if (--left == 0) break;
-                }
-            } else {
-                // UNROLL == 0: a launch with one lane per warp (few configs: each warp's pace is its one
-                // lane's chain, and nothing has to stay in step).
-                // Between two iterations in which some resident needs a new block - the histogram is sparse when
-                // few requests are resident - an iteration can only end the run by completing a request (a
-                // count known in advance) or by letting the head of the queue in (only when there is room for
-                // it): such stretches advance the clock without looking at anything else, four iterations per
-                // trip as four independent chains when no arrival has to be watched.
-                const u64 nz = L.nzmask;
-                for (;;) {
-                    u32 dist = 0;                                // iterations before the next one with needers
-                    if (blk > 1) {
-                        const u64 low = hidx + 1 < 64 ? nz >> (hidx + 1) : 0ull;       // bins above hidx come last
-                        const u64 rot = ((nz << (blk - 1 - hidx)) | low) & ((blk == 64) ? ~0ull : ((1ull << blk) - 1));
-                        dist = rot ? (u32)__clzll((long long)rot) - (64 - blk) : 0xFFFFFFFFu;
-                    }
-                    u32 nf = min(min(dist, steps_max - it), left);
-                    if (nf == 0) {
-                        // an iteration with block needs: the general step
-                        const double c1 = ctxd + nd;
-                        const double t1 = LANE_TIME(c1);
-                        LANE_APPLY(tcur, ctxd)
-                        tcur = t1; ctxd = c1;
-                        if (--left == 0) break;
-                        continue;
-                    }
-                    left -= nf;
-                    { const u32 back = nf % blk; hidx = hidx >= back ? hidx - back : hidx + blk - back; }
-                    bool stop = false;
-                    const bool watch = room && need_next <= fb;  // the queue head could come in as soon as it has arrived
-                    if (watch) {
-                        for (; nf > 0; nf--) {
-                            const double c1 = ctxd + nd;
-                            const double t1 = LANE_TIME(c1);
-                            clock = clock + tcur; dec_time = dec_time + tcur; cd = ctxd; it++;
-                            tcur = t1; ctxd = c1;
-                            if (arr_next <= clock && it != steps_max) { stop = true; break; }
-                        }
-                        if (stop) {                              // the rest of the stretch is not run: put the bin index back
-                            const u32 fwd = (nf - 1) % blk;
-                            hidx = hidx + fwd >= blk ? hidx + fwd - blk : hidx + fwd;
-                            left += nf - 1;
-                            mode = LM_SCHED;
-                            break;
-                        }
-                    } else {
-                        {
-                            for (; nf >= 4; nf -= 4) {
-                                const double c1 = ctxd + nd, c2 = c1 + nd, c3 = c2 + nd, c4 = c3 + nd;
-                                const double t1 = LANE_TIME(c1), t2 = LANE_TIME(c2), t3 = LANE_TIME(c3), t4 = LANE_TIME(c4);
-                                clock = clock + tcur; clock = clock + t1; clock = clock + t2; clock = clock + t3;
-                                dec_time = dec_time + tcur; dec_time = dec_time + t1; dec_time = dec_time + t2; dec_time = dec_time + t3;
-                                cd = c3; it += 4;
-                                tcur = t4; ctxd = c4;
-                            }
-                        }
-                        for (; nf > 0; nf--) {
-                            const double c1 = ctxd + nd;
-                            const double t1 = LANE_TIME(c1);
-                            clock = clock + tcur; dec_time = dec_time + tcur; cd = ctxd; it++;
-                            tcur = t1; ctxd = c1;
-                        }
-                    }
-                    if (it == steps_max) { mode = LM_SCHED; break; }      // a completion (or the cap) follows
-                    if (left == 0) break;
                 }
             }
 #undef LANE_APPLY

@@ -51,14 +51,13 @@ static size_t per_warp_bytes(u32 n_req) {
 }
 
 
+// Sum over the warp of values below 2^51 (block and token counts), by the integer reduction unit:
+// the low 24 bits and the rest are summed apart so that neither sum leaves 32 bits.
 __device__ __forceinline__ u64 warp_sum(u64 v) {
-    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
-    return v;
+    const u32 lo = __reduce_add_sync(0xFFFFFFFFu, (u32)v & 0xFFFFFFu), hi = __reduce_add_sync(0xFFFFFFFFu, (u32)(v >> 24));
+    return ((u64)hi << 24) + lo;
 }
-__device__ __forceinline__ u32 warp_min(u32 v) {
-    for (int d = 16; d > 0; d >>= 1) v = min(v, __shfl_xor_sync(0xFFFFFFFFu, v, d));
-    return v;
-}
+__device__ __forceinline__ u32 warp_min(u32 v) { return __reduce_min_sync(0xFFFFFFFFu, v); }
 __device__ __forceinline__ u32 ceil_div32(u32 a, u32 b) { return (a + b - 1) / b; }
 
 // Time of one decode iteration from the summed context (as an exact double), when every integer
@@ -76,6 +75,8 @@ __device__ __forceinline__ double decode_time(double ctxd, double c_f9, double t
 }
 
 struct SlotArrays {
+    double tbuf[32];    // times of the 32 iterations a run computes at once
+    double dterm[32][4];   // decode terms (fixed tasks, all-reduce, head, activation bytes) of 32 neighbouring resident counts
     u32 req[SLOTS];     // request index
     u32 base[SLOTS];    // resident: cache - D (mod 2^32); waiting for its prompt pass: prompt + recompute tokens
     u32 fin[SLOTS];     // resident: D at which it completes; waiting for its prompt pass: tokens still to emit
@@ -236,11 +237,12 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         u32 D = 0, Dmod = 0, min_rem = NO_COMPLETION;
         const bool use_hist = blk > 1 && blk <= HIST;
         const bool burst_ok = exact53 && (blk == 1 || use_hist);
+        const u32 lmod = lane % blk, m32 = 32u % blk;     // lane and warp width modulo the block size
         const u64 max_iters = max_iters_opt ? max_iters_opt : 64 * (tr.sum_out + (u64)tr.n_zero * Lout) + 4 * (u64)n;
         // cached while the running count stays the same
         u32 dc_n = 0;
         double dc_fix = 0.0, dc_comm = 0.0, dc_head = 0.0, dc_tha = 0.0, dc_nd = 0.0;
-        u64 dc_tha_i = 0;
+        u32 dc_w0 = 0x80000000u;         // first resident count of the window of decode terms in shared memory (none yet)
         u64 pre_T = 0, pre_A = 0;        // prompt tokens (and their squares) admitted since the last prompt pass
         // the head of the waiting queue: its arrival time and the blocks it needs
         double arr_next = 0.0;
@@ -367,14 +369,24 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                 }
                 free_blocks -= needed;
                 if (dc_n != nrun) {
-                    TaskTab kt;
-                    build_fixed_tasks(m, tt, nrun, nrun, 1, kt);
+                    if (nrun - dc_w0 >= 32u) {
+                        // The terms of a decode iteration that depend on the resident count only, for 32
+                        // neighbouring counts at once (one per lane): the count moves by one or two per
+                        // event, so most events find theirs in the window.
+                        dc_w0 = nrun > 16 ? nrun - 16 : 1;
+                        const u32 nl = dc_w0 + lane;
+                        TaskTab kt;
+                        build_fixed_tasks(m, tt, nl, nl, 1, kt);
+                        __syncwarp();
+                        sl.dterm[lane][0] = eval_fixed<TIME_SUM>(kt, rt);
+                        sl.dterm[lane][1] = eval_comm(kt, rt);
+                        sl.dterm[lane][2] = eval_head<TIME_SUM>(kt, rt);
+                        sl.dterm[lane][3] = (double)((u64)nl * m.H * m.ab) * inv_tt;
+                        __syncwarp();
+                    }
                     dc_n = nrun;
-                    dc_fix = eval_fixed<TIME_SUM>(kt, rt);
-                    dc_comm = eval_comm(kt, rt);
-                    dc_head = eval_head<TIME_SUM>(kt, rt);
-                    dc_tha_i = (u64)nrun * m.H * m.ab;
-                    dc_tha = (double)dc_tha_i * inv_tt;
+                    const double2 d01 = *(const double2 *)&sl.dterm[nrun - dc_w0][0], d23 = *(const double2 *)&sl.dterm[nrun - dc_w0][2];
+                    dc_fix = d01.x; dc_comm = d01.y; dc_head = d23.x; dc_tha = d23.y;
                     dc_nd = (double)nrun;
                 }
                 if (burst_ok) {
@@ -388,27 +400,72 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                     u32 fb = fb0, it = 0;
                     u32 hidx = Dmod + 1 == blk ? 0 : blk - (Dmod + 1);     // histogram bin of the next iteration's needers
                     const bool room = nrun < b;
-                    const double nd = dc_nd, tha = dc_tha, fix = dc_fix, comm = dc_comm, head = dc_head, tovh = rt.tovh;
-                    double cd = csum_d;
-                    double ctxd = cd + nd;
-                    double tcur = decode_time<TIME_SUM>(ctxd, c_f9, tha, c_kvx, c_f10, c_b10, icA, imA, fix, comm, head, Nd,
-                                                        tovh, lf);
+                    const double nd = dc_nd, cd0 = csum_d;
+                    // The iterations of a run do not depend on one another except through the clock:
+                    // the summed context of the i-th is cd0 + i * nd (exact), so the 32 lanes compute
+                    // the times of 32 consecutive iterations at once; which of them ends the run on
+                    // block counts is a prefix sum over the histogram bins, and the clock is then
+                    // advanced one iteration after the other (same order of additions as a scalar
+                    // loop), watching for the arrival of the queue head where it could come in.
                     for (;;) {
-                        clock = clock + tcur;
-                        dec_time = dec_time + tcur;
-                        cd = ctxd;
-                        it++;
-                        ctxd = cd + nd;
-                        const double tnext = decode_time<TIME_SUM>(ctxd, c_f9, tha, c_kvx, c_f10, c_b10, icA, imA, fix, comm,
-                                                                   head, Nd, tovh, lf);
-                        if (it == steps_max) break;                               // a completion (or the cap) follows
-                        const u32 need2 = blk == 1 ? nrun : sl.hist[hidx];
-                        if (need2 > fb) break;                                    // eviction needed
-                        if (room && arr_next <= clock && need_next <= fb) break;  // the queue head can come in
-                        fb -= need2;
-                        hidx = hidx == 0 ? blk - 1 : hidx - 1;
-                        tcur = tnext;
+                        const u32 nb = min(32u, steps_max - it);
+                        const double t_k = decode_time<TIME_SUM>(cd0 + nd * (double)(it + lane + 1), c_f9, dc_tha, c_kvx, c_f10, c_b10,
+                                                                 icA, imA, dc_fix, dc_comm, dc_head, Nd, rt.tovh, lf);
+                        // blocks the residents need before the iteration after lane's, and what is free by then
+                        u32 need_k = 0;
+                        if (lane < nb) need_k = blk == 1 ? nrun : sl.hist[hidx >= lmod ? hidx - lmod : hidx + blk - lmod];
+                        u32 incl = need_k;
+                        #pragma unroll
+                        for (int d = 1; d < 32; d <<= 1) {
+                            const u32 up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                            if (lane >= (u32)d) incl += up;
+                        }
+                        const u32 fb_k = fb - (incl - need_k);            // wraps only behind a lane that already stops
+                        const u32 stops = __ballot_sync(0xFFFFFFFFu, lane < nb && (it + lane + 1 == steps_max || need_k > fb_k));
+                        const u32 last = stops ? (u32)__ffs(stops) - 1 : 31u;   // a completion, the cap or an eviction follows it
+                        const u32 watch = __ballot_sync(0xFFFFFFFFu, room && need_next <= fb_k) & (0xFFFFFFFFu >> (31 - last));
+                        sl.tbuf[lane] = t_k;
+                        __syncwarp();
+                        // the clock, one iteration after the other: four per trip, the arrival tests of a trip taken together
+                        u32 k = 0;
+                        bool arrived = false;
+                        const u32 cnt = last + 1;
+                        while (k + 4 <= cnt) {
+                            const double2 va = *(const double2 *)&sl.tbuf[k], vb = *(const double2 *)&sl.tbuf[k + 2];
+                            const double c1 = clock + va.x, c2 = c1 + va.y, c3 = c2 + vb.x, c4 = c3 + vb.y;
+                            const double d1 = dec_time + va.x, d2 = d1 + va.y, d3 = d2 + vb.x, d4 = d3 + vb.y;
+                            const u32 wbits = (watch >> k) & 15u;
+                            u32 hit = 0;
+                            if (wbits)
+                                hit = ((u32)(arr_next <= c1) | ((u32)(arr_next <= c2) << 1) | ((u32)(arr_next <= c3) << 2) |
+                                       ((u32)(arr_next <= c4) << 3)) & wbits;
+                            if (hit) {                                             // the queue head can come in after one of the four
+                                const u32 f = (u32)__ffs(hit) - 1;
+                                clock = f == 0 ? c1 : f == 1 ? c2 : f == 2 ? c3 : c4;
+                                dec_time = f == 0 ? d1 : f == 1 ? d2 : f == 2 ? d3 : d4;
+                                k += f;
+                                arrived = true;
+                                break;
+                            }
+                            clock = c4; dec_time = d4;
+                            k += 4;
+                        }
+                        if (!arrived) {
+                            for (; k < cnt; k++) {
+                                const double v = sl.tbuf[k];
+                                clock = clock + v;
+                                dec_time = dec_time + v;
+                                if (((watch >> k) & 1u) && arr_next <= clock) { arrived = true; break; }
+                            }
+                            if (!arrived) k = last;
+                        }
+                        it += k + 1;
+                        __syncwarp();
+                        if (stops || arrived) { fb = __shfl_sync(0xFFFFFFFFu, fb_k, k); break; }
+                        fb = __shfl_sync(0xFFFFFFFFu, fb_k - need_k, 31);
+                        hidx = hidx >= m32 ? hidx - m32 : hidx + blk - m32;
                     }
+                    const double cd = cd0 + nd * (double)it;
                     const u64 tok = (u64)it * nrun;
                     D += it;
                     Dmod = (Dmod + it) % blk;
@@ -421,7 +478,7 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                     const u64 ctx = csum + nrun;                       // cached tokens + the new one, summed
                     const u64 X = xw * ctx;
                     const double F9 = cvt(2 * (u64)m.H * ctx) * inv_tt;
-                    const double B9 = cvt(dc_tha_i + ctx * m.Dkv * m.kvb + X) * inv_tt;
+                    const double B9 = cvt((u64)nrun * m.H * m.ab + ctx * m.Dkv * m.kvb + X) * inv_tt;
                     const double F10 = cvt(5 * (u64)m.nh * ctx) * inv_tt;
                     const double B10 = cvt(2 * X) * inv_tt;
                     const double t9 = task_time<TIME_SUM>(F9, B9, icA, imA);
@@ -674,26 +731,25 @@ k_trace_lanes(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, gui
 // resident request, so a launch for large batches gives a warp fewer lanes.
 // round: decode iterations a lane may run between two event phases (events come more often with larger batches)
 // unroll: iterations per trip of the run loop (4: long runs, where a lane's own chain latency is the limit)
-struct LaneClass { u32 minb, maxb, lanes, round, unroll; };
-static const LaneClass LANE_CLASSES[LANE_N_CLASSES] = {{1, 16, 32, 64, 4}, {17, 64, 32, 16, 1}, {65, GUIDE_TRACE_MAX_BATCH, 8, 8, 1}};
-#ifndef LANE_CLASSES_ENABLED
-#define LANE_CLASSES_ENABLED 2      // classes from this one on always go to the warp-per-config kernel
+// min_configs: the class is launched only when the space has at least this many of its configs.  The
+// lane kernel handles events one lane at a time and its run loop is one dependent chain per lane, so it
+// needs most lanes of every resident warp busy to beat the warp-per-config kernel, whose run loop
+// spreads the iterations of one config over the lanes (measured on workload 3, max batch 6-16: 4,096
+// configs 110 ms in lanes against 42 ms in warps; 32,768 configs 215 against 283 ms; max batch 24-64
+// on workload 4, 262,144 configs: 117 against about 220 ms).
+struct LaneClass { u32 minb, maxb, lanes, round, unroll; u64 min_configs; };
+#ifndef LANE_CLASS0_MIN_WAVES
+#define LANE_CLASS0_MIN_WAVES 8
 #endif
-// A class above the first is launched only when it has at least this many configs: the lane kernel is
-// bound by the latency of each lane's chain and needs several waves of configs to pay for the slot
-// scans it does one lane at a time (measured: max batch 24-64 on workload 4, 262,144 configs, 117 ms
-// against about 220 ms in the warp-per-config kernel; on workload 3, 16,384 configs, 259 against 170 ms).
-#ifndef LANE_CLASS_MIN_CONFIGS_DEF
-#define LANE_CLASS_MIN_CONFIGS_DEF ((u64)LANE_MAX_WARPS * 32)
-#endif
-static constexpr u64 LANE_CLASS_MIN_CONFIGS = LANE_CLASS_MIN_CONFIGS_DEF;
+static const LaneClass LANE_CLASSES[LANE_N_CLASSES] = {{1, 16, 32, 64, 4, (u64)LANE_MAX_WARPS * LANE_CLASS0_MIN_WAVES},
+                                                       {17, 64, 32, 16, 1, (u64)LANE_MAX_WARPS * 32},
+                                                       {65, GUIDE_TRACE_MAX_BATCH, 8, 8, 1, ~0ull}};
 
 typedef void (*LaneKernel)(DSpace, DTrace, Range, int, u64, guide_outputs, unsigned long long *, unsigned char *, size_t, u32, u32,
                            int, u32, u32, u32, u32, u32);
 template <int TIME_SUM>
 static LaneKernel lane_kernel(u32 unroll) {
-    return unroll == 4 ? (LaneKernel)k_trace_lanes<TIME_SUM, 4>
-           : unroll == 1 ? (LaneKernel)k_trace_lanes<TIME_SUM, 1> : (LaneKernel)k_trace_lanes<TIME_SUM, 0>;
+    return unroll == 4 ? (LaneKernel)k_trace_lanes<TIME_SUM, 4> : (LaneKernel)k_trace_lanes<TIME_SUM, 1>;
 }
 static constexpr u32 LANE_BLOCK_WARPS = 4;
 static constexpr size_t LANE_SMEM_LIMIT = 112 * 1024;
@@ -705,7 +761,6 @@ static size_t lane_block_smem(const LaneClass &c, u32 lanes, u32 hist_n) {
 LaneHints lane_hints(const guide_space &s) {
     LaneHints h{};
     h.hist_n = 1;
-    const u32 n_classes = std::min<u32>(LANE_CLASSES_ENABLED, LANE_N_CLASSES);
     u64 n_fw = 0;
     for (const guide_fw &f : s.fw)
         if (f.policy == GUIDE_POLICY_PREFILL_FIRST && f.kv_block <= LANE_HIST_MAX) {
@@ -713,22 +768,14 @@ LaneHints lane_hints(const guide_space &s) {
             h.hist_n = std::max(h.hist_n, f.kv_block);
         }
     const u64 per_b = (u64)s.models.size() * s.hw.size() * n_fw * s.tp.size() * s.pairs.size();
-    u64 all[LANE_N_CLASSES] = {}, total = 0;
+    u64 all[LANE_N_CLASSES] = {};
     for (uint32_t b : s.batch)
         for (u32 c = 0; c < LANE_N_CLASSES; c++)
-            if (b >= LANE_CLASSES[c].minb && b <= LANE_CLASSES[c].maxb) { all[c] += per_b; total += per_b; }
-    if (total <= LANE_MAX_WARPS) {
-        // a space this small gives every config a warp of its own (one lane each): the launch lasts as
-        // long as its longest schedule whatever the max batch, and one kernel does it all
-        h.class_configs[0] = total;
-        h.single = 1;
-        return h;
-    }
-    // Otherwise classes are taken from the first one up, without gaps (the warp-per-config kernel leaves
-    // out every max batch up to the last launched class's limit), the later ones only when they are
-    // large enough to pay.
-    for (u32 c = 0; c < n_classes; c++) {
-        if (c > 0 && all[c] < LANE_CLASS_MIN_CONFIGS) break;
+            if (b >= LANE_CLASSES[c].minb && b <= LANE_CLASSES[c].maxb) all[c] += per_b;
+    // Classes are taken from the first one up, without gaps (the warp-per-config kernel leaves out every
+    // max batch up to the last launched class's limit), each only when it is large enough to pay.
+    for (u32 c = 0; c < LANE_N_CLASSES; c++) {
+        if (all[c] < LANE_CLASSES[c].min_configs) break;
         h.class_configs[c] = all[c];
     }
     return h;
@@ -740,7 +787,7 @@ LaneHints lane_hints(const guide_space &s) {
 size_t trace_workspace_bytes(u32 n_req, const LaneHints &hints) {
     size_t slices = SIM_MAX_WARPS;
     for (u32 c = 0; c < LANE_N_CLASSES; c++) {
-        const u64 lanes = hints.single ? 1 : LANE_CLASSES[c].lanes;
+        const u64 lanes = LANE_CLASSES[c].lanes;
         slices = std::max<size_t>(slices, std::min<u64>((u64)LANE_MAX_WARPS * lanes,
                                                         hints.class_configs[c] + LANE_BLOCK_WARPS * lanes));
     }
@@ -749,11 +796,9 @@ size_t trace_workspace_bytes(u32 n_req, const LaneHints &hints) {
 
 struct LanePlan { u32 blocks, lanes_used; size_t smem; };
 
-static const LaneClass LANE_SINGLE = {1, GUIDE_TRACE_MAX_BATCH, 1, 64, 0};     // small spaces: one lane per warp, every max batch
-
 template <int TIME_SUM>
 static int plan_lanes(const DSpace &s, const LaneHints &h, Range r, u32 cls, LanePlan *p) {
-    const LaneClass &c = h.single ? LANE_SINGLE : LANE_CLASSES[cls];
+    const LaneClass &c = LANE_CLASSES[cls];
     p->blocks = 0; p->lanes_used = c.lanes; p->smem = 0;
     if (h.class_configs[cls] == 0) return GUIDE_OK;
     static std::mutex mu;
@@ -763,7 +808,7 @@ static int plan_lanes(const DSpace &s, const LaneHints &h, Range r, u32 cls, Lan
     {
         std::lock_guard<std::mutex> lock(mu);
         if (dev < 64 && !opted[dev]) {
-            for (u32 u : {0u, 1u, 4u})
+            for (u32 u : {1u, 4u})
                 GUIDE_CUDA(cudaFuncSetAttribute(lane_kernel<TIME_SUM>(u), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                 (int)LANE_SMEM_LIMIT));
             opted[dev] = true;
@@ -821,8 +866,8 @@ static int launch_one(const DSpace &s, const DTrace &t, Range r, int tp_model, u
         return fail(GUIDE_ERR_WORKSPACE, "workspace too small for the resident warps");
     if (policies & 1) {
         u32 lane_maxb = 0;
-        for (u32 cls = 0; cls < (hints.single ? 1u : LANE_N_CLASSES); cls++) {
-            const LaneClass &lc = hints.single ? LANE_SINGLE : LANE_CLASSES[cls];
+        for (u32 cls = 0; cls < LANE_N_CLASSES; cls++) {
+            const LaneClass &lc = LANE_CLASSES[cls];
             LanePlan lp;
             int rc = plan_lanes<TIME_SUM>(s, hints, r, cls, &lp);
             if (rc) return rc;
@@ -831,8 +876,7 @@ static int launch_one(const DSpace &s, const DTrace &t, Range r, int tp_model, u
             if (256 + (size_t)lp.blocks * LANE_BLOCK_WARPS * lp.lanes_used * pw > ws_bytes)
                 return fail(GUIDE_ERR_WORKSPACE, "workspace too small for the lane kernel's %u blocks", lp.blocks);
             GUIDE_CUDA(cudaMemsetAsync(ws, 0, 256, st));
-            // one lane per warp: the run loop that skips from one block need to the next (unroll 0)
-            lane_kernel<TIME_SUM>(lp.lanes_used == 1 ? 0u : lc.unroll)<<<lp.blocks, LANE_BLOCK_WARPS * 32, lp.smem, st>>>(
+            lane_kernel<TIME_SUM>(lc.unroll)<<<lp.blocks, LANE_BLOCK_WARPS * 32, lp.smem, st>>>(
                 s, t, r, tp_model, max_iters, o, (unsigned long long *)ws, scratch, pw, gen_bytes, first_bytes, reorder,
                 lc.minb, lc.maxb, hints.hist_n, lp.lanes_used, lc.round);
             GUIDE_CUDA(cudaGetLastError());
