@@ -86,9 +86,13 @@ struct SlotArrays {
 
 // Results of one simulated config: per-request values, means in request order, nearest-rank
 // percentiles (sorted in the tpot slice, which is free by then).  Called by the whole warp.
+// FINISH: tpot[i] holds the time of request i's last token, and the time per output token is worked
+// out here, 32 requests at a time (Lout: output length of the requests that take the config's lengths).
+template <bool FINISH>
 __device__ __forceinline__ void write_trace_results(const guide_outputs &o, u64 j, u32 n, u32 st, u32 fit, double clock,
                                                     double dec_time, u64 dec_tok, u64 n_iters, u64 n_req_iters, double cost_hr,
-                                                    const double *arrival, double *first, double *tpot, u32 lane) {
+                                                    const DTrace &tr, u32 Lout, double *first, double *tpot, u32 lane) {
+    const double *arrival = tr.arrival;
     const double inf = __longlong_as_double(0x7FF0000000000000LL);
     double *rq_ttft = o.req_ttft ? o.req_ttft + j * n : nullptr;
     double *rq_tpot = o.req_tpot ? o.req_tpot + j * n : nullptr;
@@ -121,8 +125,13 @@ __device__ __forceinline__ void write_trace_results(const guide_outputs &o, u64 
         const u32 i = base + lane;
         double vt = 0.0, vp = 0.0;
         if (i < n) {
-            vt = first[i] - __ldg(arrival + i);
+            const double f = first[i];
+            vt = f - __ldg(arrival + i);
             vp = tpot[i];
+            if (FINISH) {
+                const u32 out = __ldg(tr.in_len + i) ? __ldg(tr.out_len + i) : Lout;
+                vp = out > 1 ? (vp - f) / (double)(out - 1) : 0.0;
+            }
             if (rq_ttft) __stcs(rq_ttft + i, vt);
             if (rq_tpot) __stcs(rq_tpot + i, vp);
         }
@@ -158,6 +167,111 @@ __device__ __forceinline__ void write_trace_results(const guide_outputs &o, u64 
         if (o.ttft) o.ttft[j] = s_ttft / nd;
         if (o.ttft_p50) o.ttft_p50[j] = tpot[(50ull * n + 99) / 100 - 1];
         if (o.ttft_p99) o.ttft_p99[j] = tpot[(99ull * n + 99) / 100 - 1];
+        if (o.tpot) o.tpot[j] = s_tpot / nd;
+        if (o.thr_decode) o.thr_decode[j] = thr;
+        if (o.cost_per_hr) o.cost_per_hr[j] = cost_hr;
+        if (o.cost_per_token) o.cost_per_token[j] = thr > 0.0 ? (cost_hr / 3600.0) / thr : inf;
+        if (o.status) o.status[j] = 0;
+        if (o.bmax) o.bmax[j] = fit;
+        if (o.n_iters) o.n_iters[j] = n_iters;
+        if (o.n_req_iters) o.n_req_iters[j] = n_req_iters;
+        if (o.seq_used) o.seq_used[j] = 0;          // closed form only
+    }
+}
+
+// Results of one config simulated by k_trace_sim or the lane kernel: per-request values, means in request order, nearest-rank
+// percentiles.  first[i]: time of request i's first token; finish[i]: time of its last one (the
+// slice has room for the next power of two of doubles and serves as the sort buffer afterwards).
+// Called by the whole warp; out of line, so that its registers (the sort keeps a batch of pairs in
+// flight) do not weigh on the simulation loops of its callers.
+__device__ __noinline__ void write_lane_results(const guide_outputs &o, u64 j, u32 n, u32 st, u32 fit, double clock,
+                                                 double dec_time, u64 dec_tok, u64 n_iters, u64 n_req_iters, double cost_hr,
+                                                 const DTrace &tr, u32 Lout, double *first, double *finish, u32 lane) {
+    const double inf = __longlong_as_double(0x7FF0000000000000LL);
+    double *rq_ttft = o.req_ttft ? o.req_ttft + j * n : nullptr;
+    double *rq_tpot = o.req_tpot ? o.req_tpot + j * n : nullptr;
+    __syncwarp();
+    if (st) {
+        if (lane == 0) {
+            if (o.latency) o.latency[j] = inf;
+            if (o.ttft) o.ttft[j] = inf;
+            if (o.ttft_p50) o.ttft_p50[j] = inf;
+            if (o.ttft_p99) o.ttft_p99[j] = inf;
+            if (o.tpot) o.tpot[j] = inf;
+            if (o.thr_decode) o.thr_decode[j] = 0.0;
+            if (o.cost_per_hr) o.cost_per_hr[j] = inf;
+            if (o.cost_per_token) o.cost_per_token[j] = inf;
+            if (o.status) o.status[j] = (uint8_t)st;
+            if (o.bmax) o.bmax[j] = fit;
+            if (o.n_iters) o.n_iters[j] = 0;
+            if (o.n_req_iters) o.n_req_iters[j] = 0;
+            if (o.seq_used) o.seq_used[j] = 0;
+        }
+        for (u32 i = lane; i < n; i += 32) {
+            if (rq_ttft) __stcs(rq_ttft + i, inf);
+            if (rq_tpot) __stcs(rq_tpot + i, inf);
+        }
+        return;
+    }
+    // means in request order: 32 values at a time, added one after the other
+    double s_ttft = 0.0, s_tpot = 0.0;
+    for (u32 base = 0; base < n; base += 32) {
+        const u32 i = base + lane;
+        double vt = 0.0, vp = 0.0;
+        if (i < n) {
+            const double f = first[i];
+            const u32 out = __ldg(tr.in_len + i) ? __ldg(tr.out_len + i) : Lout;
+            vt = f - __ldg(tr.arrival + i);
+            vp = out > 1 ? (finish[i] - f) / (double)(out - 1) : 0.0;     // time per output token after the first
+            if (rq_ttft) __stcs(rq_ttft + i, vt);
+            if (rq_tpot) __stcs(rq_tpot + i, vp);
+        }
+        const u32 lim = min(32u, n - base);
+        for (u32 l = 0; l < lim; l++) {
+            s_ttft = s_ttft + __shfl_sync(0xFFFFFFFFu, vt, l);
+            s_tpot = s_tpot + __shfl_sync(0xFFFFFFFFu, vp, l);
+        }
+        if (i < n) first[i] = vt;             // keep TTFT for the percentile sort
+    }
+    // nearest-rank percentiles: bitonic sort of the TTFTs in the (now free) finish slice.  The pairs of
+    // a stage are disjoint, so a lane loads a batch of them before it stores any: the loads overlap.
+    double *buf = finish;
+    if (o.ttft_p50 || o.ttft_p99) {
+        u32 P = 1;
+        while (P < n) P <<= 1;
+        __syncwarp();
+        for (u32 i = lane; i < P; i += 32) buf[i] = i < n ? first[i] : inf;
+        __syncwarp();
+        constexpr u32 BATCH = 8;
+        for (u32 size = 2; size <= P; size <<= 1) {
+            for (u32 stride = size >> 1; stride > 0; stride >>= 1) {
+                for (u32 i0 = lane; i0 < (P >> 1); i0 += 32 * BATCH) {
+                    double a[BATCH], bb[BATCH];
+                    u32 lo[BATCH];
+#pragma unroll
+                    for (u32 u = 0; u < BATCH; u++) {
+                        const u32 i = i0 + 32 * u;
+                        lo[u] = ((i & ~(stride - 1)) << 1) | (i & (stride - 1));
+                        if (i < (P >> 1)) { a[u] = buf[lo[u]]; bb[u] = buf[lo[u] + stride]; }
+                    }
+#pragma unroll
+                    for (u32 u = 0; u < BATCH; u++) {
+                        const u32 i = i0 + 32 * u;
+                        const bool up = (lo[u] & size) == 0;
+                        if (i < (P >> 1) && (bb[u] < a[u]) == up) { buf[lo[u]] = bb[u]; buf[lo[u] + stride] = a[u]; }
+                    }
+                }
+                __syncwarp();
+            }
+        }
+    }
+    if (lane == 0) {
+        const double nd = (double)n;
+        const double thr = dec_time > 0.0 ? cvt(dec_tok) / dec_time : 0.0;
+        if (o.latency) o.latency[j] = clock;
+        if (o.ttft) o.ttft[j] = s_ttft / nd;
+        if (o.ttft_p50) o.ttft_p50[j] = buf[(50ull * n + 99) / 100 - 1];
+        if (o.ttft_p99) o.ttft_p99[j] = buf[(99ull * n + 99) / 100 - 1];
         if (o.tpot) o.tpot[j] = s_tpot / nd;
         if (o.thr_decode) o.thr_decode[j] = thr;
         if (o.cost_per_hr) o.cost_per_hr[j] = cost_hr;
@@ -238,6 +352,11 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         const bool use_hist = blk > 1 && blk <= HIST;
         const bool burst_ok = exact53 && (blk == 1 || use_hist);
         const u32 lmod = lane % blk, m32 = 32u % blk;     // lane and warp width modulo the block size
+        // block sizes are powers of two as a rule: their divisions are shifts
+        const u32 blk_shift = (blk & (blk - 1)) == 0 ? (u32)__ffs(blk) - 1 : 0xFFFFFFFFu;
+        auto divb = [&](u32 x) { return blk_shift != 0xFFFFFFFFu ? x >> blk_shift : x / blk; };
+        auto modb = [&](u32 x) { return blk_shift != 0xFFFFFFFFu ? x & (blk - 1) : x % blk; };
+        auto blocks_of = [&](u32 tokens) { return divb(tokens + blk - 1); };
         const u64 max_iters = max_iters_opt ? max_iters_opt : 64 * (tr.sum_out + (u64)tr.n_zero * Lout) + 4 * (u64)n;
         // cached while the running count stays the same
         u32 dc_n = 0;
@@ -246,14 +365,14 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         u64 pre_T = 0, pre_A = 0;        // prompt tokens (and their squares) admitted since the last prompt pass
         // the head of the waiting queue: its arrival time and the blocks it needs
         double arr_next = 0.0;
-        u32 need_next = 0;
+        u32 need_next = 0, in_next = 0, g_next = 0;              // ... its prompt length (0: the config's) and the tokens kept from before an eviction
         auto refresh_head = [&]() {
             while (next < high_water && (gen[next] & GEN_DONE)) next++;
             if (next < n) {
                 arr_next = __ldg(tr.arrival + next);
-                const u32 g = next < high_water ? gen[next] : 0u;       // tokens kept from before an eviction
-                const u32 in = __ldg(tr.in_len + next);
-                need_next = ceil_div32((in ? in : Lin) + g, blk);
+                g_next = next < high_water ? gen[next] : 0u;
+                in_next = __ldg(tr.in_len + next);
+                need_next = blocks_of((in_next ? in_next : Lin) + g_next);
             } else {
                 arr_next = inf; need_next = 0;
             }
@@ -268,9 +387,10 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
             // ---- 1. admit in arrival order, no overtaking ----
             if (nrun < b && arr_next <= clock && need_next <= free_blocks) {
                 do {
-                    const u32 g = next < high_water ? gen[next] : 0u;
-                    u32 in = __ldg(tr.in_len + next), out = __ldg(tr.out_len + next);
-                    if (in == 0) { in = Lin; out = Lout; }
+                    const u32 g = g_next;
+                    u32 in = in_next, out = Lout;
+                    if (in == 0) in = Lin;
+                    else out = __ldg(tr.out_len + next);
                     free_blocks -= need_next;
                     if (lane == 0) {
                         sl.req[nrun] = next;
@@ -316,7 +436,8 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                             const u32 q = sl.base[k], left = sl.fin[k] - 1;
                             u32 ph = 0;
                             if (use_hist) {
-                                ph = (q % blk + blk - Dmod) % blk;          // (cache - D) mod block
+                                ph = modb(q) + blk - Dmod;                  // (cache - D) mod block
+                                if (ph >= blk) ph -= blk;
                                 atomicAdd(&sl.hist[ph], 1u);
                             }
                             sl.base[k] = q - D;
@@ -344,15 +465,15 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                     needed = 0;
                     for (u32 base = 0; base < nrun; base += 32) {
                         const u32 k = base + lane;
-                        needed += __popc(__ballot_sync(0xFFFFFFFFu, k < nrun && (sl.base[k] + D) % blk == 0));
+                        needed += __popc(__ballot_sync(0xFFFFFFFFu, k < nrun && modb(sl.base[k] + D) == 0));
                     }
                 }
                 if (needed > free_blocks) {
                     while (needed > free_blocks) {                     // evict the youngest, recompute later
                         const u32 v = nrun - 1;
                         const u32 cv = sl.base[v] + D, rq = sl.req[v], rem = sl.fin[v] - D, ph = sl.meta[v] & M_PHASE;
-                        free_blocks += ceil_div32(cv, blk);
-                        if (cv % blk == 0) needed--;
+                        free_blocks += blocks_of(cv);
+                        if (modb(cv) == 0) needed--;
                         csum -= cv;
                         const u32 out = __ldg(tr.in_len + rq) ? __ldg(tr.out_len + rq) : Lout;
                         __syncwarp();
@@ -468,7 +589,8 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                     const double cd = cd0 + nd * (double)it;
                     const u64 tok = (u64)it * nrun;
                     D += it;
-                    Dmod = (Dmod + it) % blk;
+                    Dmod += it < blk ? it : modb(it);           // short runs are the rule
+                    if (Dmod >= blk) Dmod -= blk;
                     csum += tok; csum_d = cd;
                     dec_tok += tok; n_req_iters += tok; n_iters += it;
                     min_rem -= it;
@@ -513,9 +635,8 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                     if (done) {
                         const u32 cv = bs + D;
                         gen[rq] = GEN_DONE;
-                        const u32 out = __ldg(tr.in_len + rq) ? __ldg(tr.out_len + rq) : Lout;
-                        tpot[rq] = out > 1 ? (clock - first[rq]) / (double)(out - 1) : 0.0;
-                        freed += ceil_div32(cv, blk);
+                        tpot[rq] = clock;              // time of its last token; the results turn it into time per output token
+                        freed += blocks_of(cv);
                         gone += cv;
                         if (use_hist) atomicSub(&sl.hist[mt & M_PHASE], 1u);
                     }
@@ -539,8 +660,8 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         }
 
         // ---- results ----
-        write_trace_results(o, j, n, st, fit, clock, dec_time, dec_tok, n_iters, n_req_iters, rt.price * (double)t, tr.arrival,
-                            first, tpot, lane);
+        write_trace_results<true>(o, j, n, st, fit, clock, dec_time, dec_tok, n_iters, n_req_iters, rt.price * (double)t, tr, Lout,
+                                  first, tpot, lane);
         __syncwarp();
     }
 }
@@ -595,114 +716,9 @@ k_trace_fuse(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guid
                                           log2_rule_factor(t, tp_model), max_iters, sh[wib], gen, first, tpot);
             fr = sh[wib].res;
         }
-        write_trace_results(o, j, n, st, fit, fr.clock, fr.dec_time, fr.dec_tok, fr.n_iters, fr.n_req_iters,
-                            rp->price * (double)t, tr.arrival, first, tpot, lane);
+        write_trace_results<false>(o, j, n, st, fit, fr.clock, fr.dec_time, fr.dec_tok, fr.n_iters, fr.n_req_iters,
+                                   rp->price * (double)t, tr, Lout, first, tpot, lane);
         __syncwarp();
-    }
-}
-
-// Results of one config simulated by the lane kernel: per-request values, means in request order, nearest-rank
-// percentiles.  first[i]: time of request i's first token; finish[i]: time of its last one (the
-// slice has room for the next power of two of doubles and serves as the sort buffer afterwards).
-// Called by the whole warp; out of line, so that its registers (the sort keeps a batch of pairs in
-// flight) do not weigh on the simulation loops of its callers.
-__device__ __noinline__ void write_lane_results(const guide_outputs &o, u64 j, u32 n, u32 st, u32 fit, double clock,
-                                                 double dec_time, u64 dec_tok, u64 n_iters, u64 n_req_iters, double cost_hr,
-                                                 const DTrace &tr, u32 Lout, double *first, double *finish, u32 lane) {
-    const double inf = __longlong_as_double(0x7FF0000000000000LL);
-    double *rq_ttft = o.req_ttft ? o.req_ttft + j * n : nullptr;
-    double *rq_tpot = o.req_tpot ? o.req_tpot + j * n : nullptr;
-    __syncwarp();
-    if (st) {
-        if (lane == 0) {
-            if (o.latency) o.latency[j] = inf;
-            if (o.ttft) o.ttft[j] = inf;
-            if (o.ttft_p50) o.ttft_p50[j] = inf;
-            if (o.ttft_p99) o.ttft_p99[j] = inf;
-            if (o.tpot) o.tpot[j] = inf;
-            if (o.thr_decode) o.thr_decode[j] = 0.0;
-            if (o.cost_per_hr) o.cost_per_hr[j] = inf;
-            if (o.cost_per_token) o.cost_per_token[j] = inf;
-            if (o.status) o.status[j] = (uint8_t)st;
-            if (o.bmax) o.bmax[j] = fit;
-            if (o.n_iters) o.n_iters[j] = 0;
-            if (o.n_req_iters) o.n_req_iters[j] = 0;
-            if (o.seq_used) o.seq_used[j] = 0;
-        }
-        for (u32 i = lane; i < n; i += 32) {
-            if (rq_ttft) __stcs(rq_ttft + i, inf);
-            if (rq_tpot) __stcs(rq_tpot + i, inf);
-        }
-        return;
-    }
-    // means in request order: 32 values at a time, added one after the other
-    double s_ttft = 0.0, s_tpot = 0.0;
-    for (u32 base = 0; base < n; base += 32) {
-        const u32 i = base + lane;
-        double vt = 0.0, vp = 0.0;
-        if (i < n) {
-            const double f = first[i];
-            const u32 out = __ldg(tr.in_len + i) ? __ldg(tr.out_len + i) : Lout;
-            vt = f - __ldg(tr.arrival + i);
-            vp = out > 1 ? (finish[i] - f) / (double)(out - 1) : 0.0;     // time per output token after the first
-            if (rq_ttft) __stcs(rq_ttft + i, vt);
-            if (rq_tpot) __stcs(rq_tpot + i, vp);
-        }
-        const u32 lim = min(32u, n - base);
-        for (u32 l = 0; l < lim; l++) {
-            s_ttft = s_ttft + __shfl_sync(0xFFFFFFFFu, vt, l);
-            s_tpot = s_tpot + __shfl_sync(0xFFFFFFFFu, vp, l);
-        }
-        if (i < n) first[i] = vt;             // keep TTFT for the percentile sort
-    }
-    // nearest-rank percentiles: bitonic sort of the TTFTs in the (now free) finish slice.  The pairs of
-    // a stage are disjoint, so a lane loads a batch of them before it stores any: the loads overlap.
-    double *buf = finish;
-    if (o.ttft_p50 || o.ttft_p99) {
-        u32 P = 1;
-        while (P < n) P <<= 1;
-        __syncwarp();
-        for (u32 i = lane; i < P; i += 32) buf[i] = i < n ? first[i] : inf;
-        __syncwarp();
-        constexpr u32 BATCH = 8;
-        for (u32 size = 2; size <= P; size <<= 1) {
-            for (u32 stride = size >> 1; stride > 0; stride >>= 1) {
-                for (u32 i0 = lane; i0 < (P >> 1); i0 += 32 * BATCH) {
-                    double a[BATCH], bb[BATCH];
-                    u32 lo[BATCH];
-#pragma unroll
-                    for (u32 u = 0; u < BATCH; u++) {
-                        const u32 i = i0 + 32 * u;
-                        lo[u] = ((i & ~(stride - 1)) << 1) | (i & (stride - 1));
-                        if (i < (P >> 1)) { a[u] = buf[lo[u]]; bb[u] = buf[lo[u] + stride]; }
-                    }
-#pragma unroll
-                    for (u32 u = 0; u < BATCH; u++) {
-                        const u32 i = i0 + 32 * u;
-                        const bool up = (lo[u] & size) == 0;
-                        if (i < (P >> 1) && (bb[u] < a[u]) == up) { buf[lo[u]] = bb[u]; buf[lo[u] + stride] = a[u]; }
-                    }
-                }
-                __syncwarp();
-            }
-        }
-    }
-    if (lane == 0) {
-        const double nd = (double)n;
-        const double thr = dec_time > 0.0 ? cvt(dec_tok) / dec_time : 0.0;
-        if (o.latency) o.latency[j] = clock;
-        if (o.ttft) o.ttft[j] = s_ttft / nd;
-        if (o.ttft_p50) o.ttft_p50[j] = buf[(50ull * n + 99) / 100 - 1];
-        if (o.ttft_p99) o.ttft_p99[j] = buf[(99ull * n + 99) / 100 - 1];
-        if (o.tpot) o.tpot[j] = s_tpot / nd;
-        if (o.thr_decode) o.thr_decode[j] = thr;
-        if (o.cost_per_hr) o.cost_per_hr[j] = cost_hr;
-        if (o.cost_per_token) o.cost_per_token[j] = thr > 0.0 ? (cost_hr / 3600.0) / thr : inf;
-        if (o.status) o.status[j] = 0;
-        if (o.bmax) o.bmax[j] = fit;
-        if (o.n_iters) o.n_iters[j] = n_iters;
-        if (o.n_req_iters) o.n_req_iters[j] = n_req_iters;
-        if (o.seq_used) o.seq_used[j] = 0;          // closed form only
     }
 }
 
