@@ -33,6 +33,7 @@ struct FuseSlots {
     u32 rem[GUIDE_TRACE_MAX_BATCH];     // tokens still to emit
     unsigned char fresh[GUIDE_TRACE_MAX_BATCH];   // no token emitted yet: the first one sets the TTFT
     u32 hist[FUSE_HIST];                // decode-only runs: residents per (cached tokens mod block size)
+    double tbuf[32];                    // decode-only runs: times of the 32 iterations worked out at once
 };
 
 
@@ -195,19 +196,53 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
             __syncwarp();
             const u64 cap_left = max_iters - n_iters;
             const bool room = nrun < b;
+            const u32 steps_max = (u32)min((u64)min_rem, cap_left);
+            const u32 lmod = lane % blk;
             u32 it = 0, off = 0;                                   // off = it mod block size
+            // The iterations of the run depend on one another through the clock only: the lanes work out
+            // the times of 32 consecutive ones at once (summed context ctx_i + k * nrun), a prefix sum
+            // over the histogram bins tells which of them finds its blocks, and the clock then advances
+            // one iteration after the other, in order, watching for the arrival of the queue head.
             for (;;) {
-                const u32 need_i = sl.hist[off == 0 ? 0 : blk - off];    // residents whose last block is full now
-                if (need_i > free_blocks) break;                   // eviction: the general path below
-                free_blocks -= need_i;
-                const double t_i = stage_time(nrun, nrun, ctx_i, ctx_i);
-                clock = clock + t_i;
-                dec_time = dec_time + t_i;
-                it++;
-                off = off + 1 == blk ? 0 : off + 1;
-                ctx_i += nrun;
-                if (it == min_rem || it == cap_left) break;
-                if (room && arr_next <= clock && need_next <= free_blocks) break;
+                const u32 nb = min(32u, steps_max - it);
+                const u64 ctx_k = ctx_i + (u64)lane * nrun;
+                const double t_k = stage_time(nrun, nrun, ctx_k, ctx_k);
+                u32 need_k = 0;                                    // residents whose last block is full before lane's iteration
+                if (lane < nb) {
+                    const u32 o = off + lmod >= blk ? off + lmod - blk : off + lmod;
+                    need_k = sl.hist[o == 0 ? 0 : blk - o];
+                }
+                u32 incl = need_k;
+                #pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const u32 up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                    if (lane >= (u32)d) incl += up;
+                }
+                // free blocks before lane's iteration takes its own (meaningful up to the first shortage)
+                const u64 free_k = free_blocks - (incl - need_k);
+                const u32 short_at = __ballot_sync(0xFFFFFFFFu, lane < nb && need_k > free_k);   // eviction: the general path below
+                const u32 can = short_at ? (u32)__ffs(short_at) - 1 : nb;     // iterations that find their blocks
+                if (can == 0) break;
+                const u32 last = can - 1;
+                const bool counted_out = it + can == steps_max;    // a completion or the cap follows the last one
+                const u32 watch = __ballot_sync(0xFFFFFFFFu, room && need_next <= free_k - need_k) & (0xFFFFFFFFu >> (31 - last));
+                sl.tbuf[lane] = t_k;
+                __syncwarp();
+                u32 k = 0;
+                bool arrived = false;
+                for (;; k++) {
+                    const double v = sl.tbuf[k];
+                    clock = clock + v;
+                    dec_time = dec_time + v;
+                    if (((watch >> k) & 1u) && arr_next <= clock) { arrived = true; break; }   // the queue head can come in
+                    if (k == last) break;
+                }
+                free_blocks -= __shfl_sync(0xFFFFFFFFu, incl, k);
+                it += k + 1;
+                ctx_i += (u64)(k + 1) * nrun;
+                { const u32 adv = (k + 1) % blk; off = off + adv >= blk ? off + adv - blk : off + adv; }
+                __syncwarp();
+                if (arrived || counted_out || short_at) break;
             }
             if (it > 0) {
                 for (u32 base = 0; base < nrun; base += 32) {
