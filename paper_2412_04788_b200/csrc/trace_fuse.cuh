@@ -34,17 +34,19 @@ struct FuseSlots {
     unsigned char fresh[GUIDE_TRACE_MAX_BATCH];   // no token emitted yet: the first one sets the TTFT
     u32 hist[FUSE_HIST];                // decode-only runs: residents per (cached tokens mod block size)
     double tbuf[32];                    // decode-only runs: times of the 32 iterations worked out at once
+    double dterm[32][3];                // decode-only runs: fixed-task, all-reduce and head terms of 32 neighbouring resident counts
 };
 
 
+// Sum over the warp of 64-bit counts by the integer reduction unit: three pieces of 22, 22 and 20
+// bits are summed apart (no piece's sum leaves 32 bits) and put together again modulo 2^64.
 __device__ __forceinline__ u64 fuse_warp_sum(u64 v) {
-    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
-    return v;
+    const u32 a = __reduce_add_sync(0xFFFFFFFFu, (u32)v & 0x3FFFFFu);
+    const u32 b = __reduce_add_sync(0xFFFFFFFFu, (u32)(v >> 22) & 0x3FFFFFu);
+    const u32 c = __reduce_add_sync(0xFFFFFFFFu, (u32)(v >> 44));
+    return ((u64)c << 44) + ((u64)b << 22) + a;
 }
-__device__ __forceinline__ u32 fuse_warp_sum32(u32 v) {
-    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
-    return v;
-}
+__device__ __forceinline__ u32 fuse_warp_sum32(u32 v) { return __reduce_add_sync(0xFFFFFFFFu, v); }
 // inclusive prefix sum over the lanes
 __device__ __forceinline__ u64 fuse_warp_scan(u64 v, u32 lane) {
     for (int d = 1; d < 32; d <<= 1) {
@@ -55,8 +57,8 @@ __device__ __forceinline__ u64 fuse_warp_scan(u64 v, u32 lane) {
 }
 
 // Runs the whole schedule of one config.  gen / first / tpot: the warp's per-request slices of the
-// workspace (tokens generated so far with the done flag in the top bit, first-token time, time per
-// output token).  Returns the status bits (0, or the iteration limit) and leaves the totals in
+// workspace (tokens generated so far with the done flag in the top bit, first-token time, time of the
+// last token).  Returns the status bits (0, or the iteration limit) and leaves the totals in
 // sl.res.  The model, the rates and the trace come as pointers to device memory so that the kernel
 // around this call keeps its own copies in registers.
 struct FuseTrace { const double *arrival; const u32 *in_len, *out_len; };
@@ -74,12 +76,17 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
     const u32 blk = rt.kv_block, budget = rt.seg;
     const u32 done_flag = 0x80000000u;
     const double inf = __longlong_as_double(0x7FF0000000000000LL);
-    auto blocks_of = [&](u32 tokens) { return (tokens + blk - 1) / blk; };
+    // block sizes are powers of two as a rule: their divisions are shifts
+    const u32 blk_shift = (blk & (blk - 1)) == 0 ? (u32)__ffs(blk) - 1 : 0xFFFFFFFFu;
+    auto divb = [&](u32 x) { return blk_shift != 0xFFFFFFFFu ? x >> blk_shift : x / blk; };
+    auto modb = [&](u32 x) { return blk_shift != 0xFFFFFFFFu ? x & (blk - 1) : x % blk; };
+    auto blocks_of = [&](u32 tokens) { return divb(tokens + blk - 1); };
 
     double clock = 0.0, dec_time = 0.0;
     u64 dec_tok = 0, n_iters = 0, n_req_iters = 0, free_blocks = blocks_total;
     u32 next = 0, high_water = 0, nrun = 0, st = 0;
     u32 n_pre = 0;                                   // residents still in their prompt
+    u32 dw0 = 0x80000000u;                           // first resident count of the window of decode terms (none yet)
     u64 dc_T = ~0ull, dc_E = ~0ull;                  // stage terms kept while the token counts repeat
     double dc_fix = 0.0, dc_comm = 0.0, dc_head = 0.0;
     double arr_next = 0.0;
@@ -124,8 +131,7 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
             const bool done = valid && td == 0 && rm == 0;
             if (done) {
                 gen[rq] = done_flag;
-                const u32 out = __ldg(tr.in_len + rq) ? __ldg(tr.out_len + rq) : Lout;
-                tpot[rq] = out > 1 ? (clock - first[rq]) / (double)(out - 1) : 0.0;
+                tpot[rq] = clock;          // time of its last token; the results turn it into time per output token
                 freed += blocks_of(sn);
             }
             const bool keep = valid && !done;
@@ -187,7 +193,7 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
                     const u32 sn = sl.seen[k];
                     c += (u64)sn + 1;
                     local_min = min(local_min, sl.rem[k]);
-                    atomicAdd(&sl.hist[sn % blk], 1u);
+                    atomicAdd(&sl.hist[modb(sn)], 1u);
                 }
             }
             u64 ctx_i = fuse_warp_sum(c);
@@ -197,7 +203,21 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
             const u64 cap_left = max_iters - n_iters;
             const bool room = nrun < b;
             const u32 steps_max = (u32)min((u64)min_rem, cap_left);
-            const u32 lmod = lane % blk;
+            const u32 lmod = modb(lane);
+            // The terms of a decode iteration that depend on the resident count only are kept for a window
+            // of 32 neighbouring counts (worked out one per lane): the count moves by one or two per event.
+            if (nrun - dw0 >= 32u) {
+                dw0 = nrun > 16 ? nrun - 16 : 1;
+                const u32 nl = dw0 + lane;
+                TaskTab kf;
+                build_fixed_tasks(m, tt, nl, nl, 1, kf);
+                __syncwarp();
+                sl.dterm[lane][0] = eval_fixed<TIME_SUM>(kf, rt);
+                sl.dterm[lane][1] = eval_comm(kf, rt);
+                sl.dterm[lane][2] = eval_head<TIME_SUM>(kf, rt);
+                __syncwarp();
+            }
+            const double d_fix = sl.dterm[nrun - dw0][0], d_comm = sl.dterm[nrun - dw0][1], d_head = sl.dterm[nrun - dw0][2];
             u32 it = 0, off = 0;                                   // off = it mod block size
             // The iterations of the run depend on one another through the clock only: the lanes work out
             // the times of 32 consecutive ones at once (summed context ctx_i + k * nrun), a prefix sum
@@ -206,7 +226,9 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
             for (;;) {
                 const u32 nb = min(32u, steps_max - it);
                 const u64 ctx_k = ctx_i + (u64)lane * nrun;
-                const double t_k = stage_time(nrun, nrun, ctx_k, ctx_k);
+                TaskTab ka;
+                build_attn_tasks(m, tt, nrun, ctx_k, ctx_k, ka);
+                const double t_k = combine_phase(d_fix, eval_attn<TIME_SUM>(ka, rt), d_comm, d_head, 1.0, Nd, rt.tovh, lf);
                 u32 need_k = 0;                                    // residents whose last block is full before lane's iteration
                 if (lane < nb) {
                     const u32 o = off + lmod >= blk ? off + lmod - blk : off + lmod;
@@ -240,7 +262,7 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
                 free_blocks -= __shfl_sync(0xFFFFFFFFu, incl, k);
                 it += k + 1;
                 ctx_i += (u64)(k + 1) * nrun;
-                { const u32 adv = (k + 1) % blk; off = off + adv >= blk ? off + adv - blk : off + adv; }
+                { const u32 adv = modb(k + 1); off = off + adv >= blk ? off + adv - blk : off + adv; }
                 __syncwarp();
                 if (arrived || counted_out || short_at) break;
             }
@@ -268,7 +290,7 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
                 const u32 k = base + lane;
                 if (k < nrun && sl.todo[k] == 0) {
                     const u32 sn = sl.seen[k];
-                    packed += 1u + ((sn % blk == 0) ? 0x10000u : 0u);
+                    packed += 1u + ((modb(sn) == 0) ? 0x10000u : 0u);
                     c += (u64)sn + 1;
                 }
             }
@@ -282,7 +304,7 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
                 const u32 v = nrun - 1;
                 const u32 td = sl.todo[v], sn = sl.seen[v], rq = sl.req[v], rm = sl.rem[v];
                 free_blocks += blocks_of(sn + td);                 // what it took at admission, plus its decode blocks
-                if (td == 0 && sn % blk == 0) needed--;
+                if (td == 0 && modb(sn) == 0) needed--;
                 if (td > 0) n_pre--;
                 const u32 out = __ldg(tr.in_len + rq) ? __ldg(tr.out_len + rq) : Lout;
                 __syncwarp();

@@ -32,6 +32,9 @@ namespace guide {
 #define SIM_MIN_BLOCKS 2          // resident blocks per SM k_trace_sim is compiled for (128 registers, no spills: it keeps the
                                   // event-heavy large batches now; 3 blocks of 80 registers measured 3 % slower)
 #endif
+#ifndef FUSE_MIN_BLOCKS
+#define FUSE_MIN_BLOCKS 2         // ... and k_trace_fuse (measured 2.5 % faster than 3 blocks of 80 registers)
+#endif
 static constexpr u32 SIM_WARPS_PER_BLOCK = 8;
 static constexpr u32 SIM_THREADS = SIM_WARPS_PER_BLOCK * 32;
 static constexpr u32 SIM_MAX_WARPS = 6144;        // workspace is sized for this many resident warps
@@ -86,9 +89,8 @@ struct SlotArrays {
 
 // Results of one simulated config: per-request values, means in request order, nearest-rank
 // percentiles (sorted in the tpot slice, which is free by then).  Called by the whole warp.
-// FINISH: tpot[i] holds the time of request i's last token, and the time per output token is worked
-// out here, 32 requests at a time (Lout: output length of the requests that take the config's lengths).
-template <bool FINISH>
+// tpot[i] holds the time of request i's last token on entry; the time per output token is worked out
+// here, 32 requests at a time (Lout: output length of the requests that take the config's lengths).
 __device__ __forceinline__ void write_trace_results(const guide_outputs &o, u64 j, u32 n, u32 st, u32 fit, double clock,
                                                     double dec_time, u64 dec_tok, u64 n_iters, u64 n_req_iters, double cost_hr,
                                                     const DTrace &tr, u32 Lout, double *first, double *tpot, u32 lane) {
@@ -128,10 +130,8 @@ __device__ __forceinline__ void write_trace_results(const guide_outputs &o, u64 
             const double f = first[i];
             vt = f - __ldg(arrival + i);
             vp = tpot[i];
-            if (FINISH) {
-                const u32 out = __ldg(tr.in_len + i) ? __ldg(tr.out_len + i) : Lout;
-                vp = out > 1 ? (vp - f) / (double)(out - 1) : 0.0;
-            }
+            const u32 out = __ldg(tr.in_len + i) ? __ldg(tr.out_len + i) : Lout;
+            vp = out > 1 ? (vp - f) / (double)(out - 1) : 0.0;
             if (rq_ttft) __stcs(rq_ttft + i, vt);
             if (rq_tpot) __stcs(rq_tpot + i, vp);
         }
@@ -660,7 +660,7 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         }
 
         // ---- results ----
-        write_trace_results<true>(o, j, n, st, fit, clock, dec_time, dec_tok, n_iters, n_req_iters, rt.price * (double)t, tr, Lout,
+        write_trace_results(o, j, n, st, fit, clock, dec_time, dec_tok, n_iters, n_req_iters, rt.price * (double)t, tr, Lout,
                                   first, tpot, lane);
         __syncwarp();
     }
@@ -670,7 +670,7 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
 // check and results as k_trace_sim around fuse_schedule.  Configs of the other policy are skipped
 // here and simulated there.
 template <int TIME_SUM>
-__global__ void __launch_bounds__(SIM_THREADS, 3)
+__global__ void __launch_bounds__(SIM_THREADS, FUSE_MIN_BLOCKS)
 k_trace_fuse(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide_outputs o, u32 *counter,
              unsigned char *scratch, size_t per_warp, u32 gen_bytes, u32 first_bytes, int reorder) {
     __shared__ FuseSlots sh[SIM_WARPS_PER_BLOCK];
@@ -716,7 +716,7 @@ k_trace_fuse(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guid
                                           log2_rule_factor(t, tp_model), max_iters, sh[wib], gen, first, tpot);
             fr = sh[wib].res;
         }
-        write_trace_results<false>(o, j, n, st, fit, fr.clock, fr.dec_time, fr.dec_tok, fr.n_iters, fr.n_req_iters,
+        write_trace_results(o, j, n, st, fit, fr.clock, fr.dec_time, fr.dec_tok, fr.n_iters, fr.n_req_iters,
                                    rp->price * (double)t, tr, Lout, first, tpot, lane);
         __syncwarp();
     }
