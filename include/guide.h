@@ -285,6 +285,43 @@ int guide_pareto(const guide_space *space, const guide_trace *trace, const guide
                  uint64_t *idx_out_dev, uint32_t cap, uint32_t *count_out_dev,
                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* guide_simulate (closed form), guide_select_topk and guide_pareto of the same space in one call:
+ * the steps of Sec. 3.2 (memory check, performance model, selection under the constraints of Sec. 4.1)
+ * as one pass.  out receives the metrics exactly as guide_simulate writes them; the two answers are
+ * exactly those of the separate calls on those arrays.  What the call saves is the read-back: for a
+ * whole space that goes through the line-wise kernels, a sample of configs evaluated first gives the
+ * top-k bound and a set of dominating points, every config is tested against them while its metrics
+ * are being stored, and only the few survivors are ranked.  Other spaces, sub-ranges and k above 128
+ * run the three steps one after the other on the stream, with the same results.
+ *   sel->topk_cons / pareto_cons, key, k, x_metric, y_metric: as for guide_select_topk / guide_pareto;
+ *   both selections are required.  The metric arrays that the keys and the active constraints need
+ *   must be present in out (as for a selection on materialised metrics).
+ *   sel->topk_idx_dev[k], topk_key_dev[k], topk_count_dev[1], front_idx_dev[front_cap],
+ *   front_count_dev[1]: device, written as by the separate calls.
+ *   topk_workspace: device, 256-byte aligned, at least guide_select_workspace_bytes(space, k);
+ *   pareto_workspace: likewise, guide_pareto_workspace_bytes(space).  The caller keeps ownership.
+ * opts: time_model and tp_model as for guide_simulate; a sub-range is allowed; clamp_seq and the
+ * binary32 variant give GUIDE_ERR_UNSUPPORTED (use the separate calls).  Errors as for the three
+ * calls; nothing is queued when an argument is refused. */
+typedef struct guide_selection {
+    const guide_constraints *topk_cons;
+    int32_t key;
+    uint32_t k;
+    uint64_t *topk_idx_dev;
+    double *topk_key_dev;
+    uint32_t *topk_count_dev;
+    const guide_constraints *pareto_cons;
+    int32_t x_metric, y_metric;
+    uint64_t *front_idx_dev;
+    uint32_t front_cap;
+    uint32_t *front_count_dev;
+    void *sweep_begin_event;      /* optional cudaEvent_t pair (NULL: none), recorded on the stream right before and   */
+    void *sweep_end_event;        /* right after the kernels that evaluate and store the metrics: for callers that time them */
+} guide_selection;
+int guide_simulate_select(const guide_space *space, const guide_sim_opts *opts, const guide_outputs *out,
+                          const guide_selection *sel, void *topk_workspace, size_t topk_workspace_bytes,
+                          void *pareto_workspace, size_t pareto_workspace_bytes, void *cuda_stream);
+
 /* Top-k over materialised metrics for callers that must not allocate device memory.  (The paper
  * has no counterpart: this is a packaging variant of guide_select_topk, not a step of the method.)
  *

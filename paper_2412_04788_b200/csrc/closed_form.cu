@@ -5,6 +5,7 @@
 #include "guide_internal.cuh"
 #include "model_walk.cuh"
 #include "line_walk.cuh"
+#include "select_sink.cuh"
 
 namespace guide {
 
@@ -217,11 +218,41 @@ static constexpr u32 LINE_STAGE_ARRAYS = 6;     // latency, ttft, tpot, throughp
 static constexpr u32 LINE_STAGE_ROW = 20;       // doubles per (array, pair) row: 16 + 4 of padding against bank conflicts
 static constexpr u32 LINE_WARP_DOUBLES = LINE_TABLE_DOUBLES + LINE_STAGE_ARRAYS * 8 * LINE_STAGE_ROW;
 static constexpr u32 LINE_SMEM_BYTES = (MODEL_THREADS / 32) * LINE_WARP_DOUBLES * 8;
+static constexpr u32 LINE_KILLERS = 64;          // killers the selecting variant keeps in shared memory (1 KB)
 
-template <int TIME_SUM>
+// SELECT: the kernel is also the filter pass of a top-k and a Pareto selection whose bound and killers
+// were worked out from a sample before the launch: every config that fits is tested while its metrics
+// are in registers, and the few that either selection may still want go to its survivor list, so the
+// arrays need not be read back.
+template <int TIME_SUM, bool SELECT>
 __global__ void __launch_bounds__(MODEL_THREADS, LINE_BLOCKS_PER_SM + 1)      // registers: four blocks beside the memory kernel's two
-k_closed_form_lines(DSpace s, int tp_model, guide_outputs o, u32 n_chunks, unsigned *ticket) {
+k_closed_form_lines(DSpace s, int tp_model, guide_outputs o, u32 n_chunks, unsigned *ticket, LineSelect sel) {
     extern __shared__ __align__(16) double line_smem[];
+    // Four blocks of this kernel fill an SM's shared memory but for a few KB: the filter keeps every
+    // fourth killer of the staircase (any subset of it is a valid set of killers; fewer only let more
+    // survivors through) and four pivots spread over it, which rule out most configs by themselves.
+    __shared__ P2 s_killers[SELECT ? LINE_KILLERS : 1];
+    __shared__ ulonglong2 s_pivot[4];
+    u64 bkey = 0, bidx = 0;
+    KillerSet K;
+    K.k = s_killers; K.n = 0;
+    if (SELECT) {
+        // the kernels that made the bound and the killers completed before the memory kernel started
+        const u64 *bp = reinterpret_cast<const u64 *>(sel.header_t + TK_BOUND);
+        bkey = __ldcg(bp); bidx = __ldcg(bp + 1);
+        const u32 n_all = min(__ldcg(sel.header_p + PH_KILLERS), PA_KILLERS);
+        K.n = min(n_all, LINE_KILLERS);
+        for (u32 i = threadIdx.x; i < K.n; i += blockDim.x) {
+            const ulonglong2 w = __ldcg(reinterpret_cast<const ulonglong2 *>(sel.killers + ((u64)i * n_all) / K.n));
+            s_killers[i].x = w.x; s_killers[i].y = w.y;
+        }
+        if (threadIdx.x < 4) {
+            ulonglong2 w = make_ulonglong2(KEY_MAX, KEY_MAX);
+            if (n_all > 0) w = __ldcg(reinterpret_cast<const ulonglong2 *>(sel.killers + (n_all * (2 * threadIdx.x + 1)) / 8));
+            s_pivot[threadIdx.x] = w;
+        }
+        __syncthreads();
+    }
     const u32 lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const u32 u = lane & 3, h = lane >> 2;
     double *mine = line_smem + (size_t)warp * LINE_WARP_DOUBLES;
@@ -231,7 +262,18 @@ k_closed_form_lines(DSpace s, int tp_model, guide_outputs o, u32 n_chunks, unsig
     const u64 stride_hf = (u64)s.n_b * s.n_t * s.n_l;
     double *const arr[LINE_STAGE_ARRAYS] = {o.latency, o.ttft, o.tpot, o.thr_decode, o.cost_per_hr, o.cost_per_token};
     line_walk<TIME_SUM>(s, tp_model, n_chunks, ticket, tb_pre, tb_dec,
-        [&](int q, bool, bool pair_live, u64, double latency, double ttft, double tpot, double thr, double cost_hr, double cost_tok) {
+        [&](int q, bool fits, bool pair_live, u64 j, double latency, double ttft, double tpot, double thr, double cost_hr, double cost_tok) {
+        if (SELECT && fits) {
+            // the cheap exclusions first: most configs are beyond the bound and under a pivot
+            const u64 k64 = enc(pick_metric(sel.key, latency, ttft, ttft, tpot, thr, cost_hr, cost_tok));
+            if (pair_le(k64, j, bkey, bidx) && meets(sel.ct, latency, ttft, thr, cost_hr)) topk_keep(k64, j, sel.header_t, sel.cand);
+            const u64 x = enc(pick_metric(sel.xm, latency, ttft, ttft, tpot, thr, cost_hr, cost_tok));
+            const u64 y = enc(pick_metric(sel.ym, latency, ttft, ttft, tpot, thr, cost_hr, cost_tok));
+            const ulonglong2 p0 = s_pivot[0], p1 = s_pivot[1], p2 = s_pivot[2], p3 = s_pivot[3];
+            const bool dead = dominates(p0.x, p0.y, x, y) || dominates(p1.x, p1.y, x, y) || dominates(p2.x, p2.y, x, y) ||
+                              dominates(p3.x, p3.y, x, y);
+            if (!dead && meets(sel.cp, latency, ttft, thr, cost_hr) && !K.kills_sorted(x, y)) pareto_keep(x, y, j, sel.header_p, sel.surv);
+        }
         if (pair_live) {
             double *w = stage + (size_t)h * LINE_STAGE_ROW + u + 4 * q;
             w[0 * 8 * LINE_STAGE_ROW] = latency; w[1 * 8 * LINE_STAGE_ROW] = ttft; w[2 * 8 * LINE_STAGE_ROW] = tpot;
@@ -329,7 +371,7 @@ static bool lines_apply(const DSpace &s, const guide_outputs &o) {
 
 template <int TIME_SUM>
 static int launch_split(const DSpace &s, int tp_model, const guide_outputs &o, const ConstOut &co, unsigned *ticket,
-                        cudaStream_t st) {
+                        cudaStream_t st, const LineSelect *sel) {
     const u32 n_tl = s.n_t * s.n_l, n_hf = s.n_h * s.n_f;
     const u32 tiles = (n_tl + 2 * MEM_THREADS - 1) / (2 * MEM_THREADS);
     const u32 items = s.n_m * tiles * n_hf;
@@ -351,25 +393,28 @@ static int launch_split(const DSpace &s, int tp_model, const guide_outputs &o, c
     if (lines) {
         // function attributes belong to the device: set them once per device and kernel variant
         static bool opted_in[64][2] = {};
+        const auto plain = k_closed_form_lines<TIME_SUM, false>;
+        const auto selecting = k_closed_form_lines<TIME_SUM, true>;
         static std::mutex opt_mu;
         int dev = 0;
         GUIDE_CUDA(cudaGetDevice(&dev));
         std::lock_guard<std::mutex> opt_lock(opt_mu);
         if (dev < 0 || dev >= 64 || !opted_in[dev][TIME_SUM]) {
             // more dynamic shared memory than the default limit
-            GUIDE_CUDA(cudaFuncSetAttribute(k_closed_form_lines<TIME_SUM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)LINE_SMEM_BYTES));
+            GUIDE_CUDA(cudaFuncSetAttribute(plain, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LINE_SMEM_BYTES));
+            GUIDE_CUDA(cudaFuncSetAttribute(selecting, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LINE_SMEM_BYTES));
             // An SM changes its split between L1 and shared memory only when it is empty.  The memory
             // kernel gets there first and needs neither: it asks for the split the line kernel needs,
             // so that the line kernel's blocks find room beside it instead of waiting for it to leave.
             GUIDE_CUDA(cudaFuncSetAttribute(k_closed_form_memory<1>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                             (int)cudaSharedmemCarveoutMaxShared));
-            GUIDE_CUDA(cudaFuncSetAttribute(k_closed_form_lines<TIME_SUM>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                            (int)cudaSharedmemCarveoutMaxShared));
+            GUIDE_CUDA(cudaFuncSetAttribute(plain, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared));
+            GUIDE_CUDA(cudaFuncSetAttribute(selecting, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared));
             if (dev >= 0 && dev < 64) opted_in[dev][TIME_SUM] = true;
         }
         cfg.gridDim = dim3((u32)num_sms() * LINE_BLOCKS_PER_SM); cfg.dynamicSmemBytes = LINE_SMEM_BYTES;
-        GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_closed_form_lines<TIME_SUM>, s, tp_model, o, n_chunks, ticket));
+        if (sel) GUIDE_CUDA(cudaLaunchKernelEx(&cfg, selecting, s, tp_model, o, n_chunks, ticket, *sel));
+        else GUIDE_CUDA(cudaLaunchKernelEx(&cfg, plain, s, tp_model, o, n_chunks, ticket, LineSelect{}));
     } else {
         cfg.gridDim = dim3((u32)num_sms() * MODEL_BLOCKS_PER_SM); cfg.dynamicSmemBytes = 0;
         GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_closed_form_model<TIME_SUM>, s, tp_model, o, n_chunks, ticket));
@@ -386,14 +431,23 @@ int launch_closed_form_f32(const DSpace &s, Range r, int time_model, int tp_mode
     return GUIDE_OK;
 }
 
+// Would launch_closed_form write this call through the memory and line kernels (the pair that can
+// also act as the filter pass of a combined simulate-and-select call)?
+bool closed_form_by_lines(const DSpace &s, Range r, const guide_outputs &o) {
+    ConstOut co;
+    return split_applies(s, r, o, &co) && lines_apply(s, o);
+}
+
+// sel: non-null only when closed_form_by_lines() holds for the call
 int launch_closed_form(const DSpace &s, Range r, int time_model, int tp_model, const guide_outputs &o,
-                       unsigned *ticket, cudaStream_t st) {
+                       unsigned *ticket, cudaStream_t st, const LineSelect *sel) {
     const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
+    if (sel && !(ticket && closed_form_by_lines(s, r, o))) return fail(GUIDE_ERR_UNSUPPORTED, "the call does not go through the line kernel");
     // The tiled kernel pays off when a (TP, length) plane fills warps and the range is (most of)
     // the space; slivers of the space go through the flat kernel.
     ConstOut co;
     if (ticket && split_applies(s, r, o, &co))
-        return time_model ? launch_split<1>(s, tp_model, o, co, ticket, st) : launch_split<0>(s, tp_model, o, co, ticket, st);
+        return time_model ? launch_split<1>(s, tp_model, o, co, ticket, st, sel) : launch_split<0>(s, tp_model, o, co, ticket, st, sel);
     TileGeom g;
     const bool tiled = r.count * 2 >= total && tiled_geometry(s, (u64)num_sms() * 16, 1ull << 30, &g);
     if (!tiled) {

@@ -692,6 +692,38 @@ int guide_pareto(const guide_space *space_c, const guide_trace *trace, const gui
                          (u64 *)idx_out, cap, count_out, ws, ticket, (cudaStream_t)stream);
 }
 
+int guide_simulate_select(const guide_space *space_c, const guide_sim_opts *opts, const guide_outputs *out,
+                          const guide_selection *sel, void *ws_t, size_t ws_t_bytes, void *ws_p, size_t ws_p_bytes,
+                          void *stream) {
+    guide_space *space = const_cast<guide_space *>(space_c);
+    if (!space || !out || !sel) return fail(GUIDE_ERR_INVALID, "space, out and sel are required");
+    if (out->req_ttft || out->req_tpot) return fail(GUIDE_ERR_INVALID, "per-request outputs need a trace");
+    if (opts && (opts->clamp_seq || opts->precision == GUIDE_PREC_F32))
+        return fail(GUIDE_ERR_UNSUPPORTED, "clamp_seq and the binary32 variant go through guide_simulate and the separate selection calls");
+    if (out->seq_used) return fail(GUIDE_ERR_UNSUPPORTED, "seq_used is written by guide_simulate with clamp_seq only");
+    int key = sel->key;
+    int rc = check_selection_args(space, nullptr, out, sel->topk_cons, &key, 1);
+    if (rc) return rc;
+    const int xy[2] = {sel->x_metric, sel->y_metric};
+    if ((rc = check_selection_args(space, nullptr, out, sel->pareto_cons, xy, 2))) return rc;
+    if (sel->k == 0 || sel->k > GUIDE_TOPK_MAX) return fail(GUIDE_ERR_INVALID, "k must be in 1..%u", GUIDE_TOPK_MAX);
+    if (!sel->topk_idx_dev || !sel->topk_key_dev || !sel->topk_count_dev || !sel->front_count_dev ||
+        (sel->front_cap && !sel->front_idx_dev))
+        return fail(GUIDE_ERR_INVALID, "an output pointer is NULL");
+    Range r;
+    if ((rc = resolve_range(space, opts, &r))) return rc;
+    if ((rc = check_workspace(ws_t, ws_t_bytes, topk_workspace_bytes(sel->k)))) return rc;
+    if ((rc = check_workspace(ws_p, ws_p_bytes, pareto_workspace_bytes()))) return rc;
+    DSpace ds;
+    unsigned *ticket = nullptr;
+    if ((rc = space_on_device(space, &ds, &ticket, (cudaStream_t)stream))) return rc;
+    return launch_simulate_select(ds, r, *out, opts ? opts->time_model : GUIDE_TIME_MAX, opts ? opts->tp_model : GUIDE_TP_EXPLICIT,
+                                  *sel->topk_cons, key, sel->k, (u64 *)sel->topk_idx_dev, sel->topk_key_dev, sel->topk_count_dev, ws_t,
+                                  *sel->pareto_cons, xy[0], xy[1], (u64 *)sel->front_idx_dev, sel->front_cap, sel->front_count_dev,
+                                  ws_p, ticket, (cudaStream_t)stream, (cudaEvent_t)sel->sweep_begin_event,
+                                  (cudaEvent_t)sel->sweep_end_event);
+}
+
 int guide_select_topk_noalloc(const guide_outputs *outputs, uint64_t first, uint64_t count,
                               const guide_constraints *cons, int key, uint32_t k, uint64_t *idx_out,
                               double *key_out, uint32_t *count_out, void *stream) {

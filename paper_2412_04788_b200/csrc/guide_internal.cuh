@@ -70,8 +70,10 @@ int space_on_device(guide_space *s, DSpace *out, unsigned **ticket, cudaStream_t
 int trace_on_device(guide_trace *t, DTrace *out, cudaStream_t st);
 
 // closed_form.cu
+struct LineSelect;           // select_sink.cuh: both selections of a combined simulate-and-select call
+bool closed_form_by_lines(const DSpace &s, Range r, const guide_outputs &o);
 int launch_closed_form(const DSpace &s, Range r, int time_model, int tp_model, const guide_outputs &o,
-                       unsigned *ticket, cudaStream_t st);
+                       unsigned *ticket, cudaStream_t st, const LineSelect *sel = nullptr);
 int launch_closed_form_f32(const DSpace &s, Range r, int time_model, int tp_model, const guide_outputs &o, cudaStream_t st);
 // trace_sim.cu
 // What the host knows about the configs the one-lane-per-config kernel would take: per class of max
@@ -94,6 +96,10 @@ int launch_topk(const DSpace &s, Range r, const guide_outputs *mat, int time_mod
 int launch_pareto(const DSpace &s, Range r, const guide_outputs *mat, int time_model, int tp_model,
                   const guide_constraints &c, int xm, int ym, u64 *idx_out, u32 cap, u32 *count_out,
                   void *ws, unsigned *ticket, cudaStream_t st);
+int launch_simulate_select(const DSpace &s, Range r, const guide_outputs &o, int time_model, int tp_model,
+                           const guide_constraints &ct, int key, u32 k, u64 *tk_idx, double *tk_key, u32 *tk_count, void *ws_t,
+                           const guide_constraints &cp, int xm, int ym, u64 *pf_idx, u32 cap, u32 *pf_count, void *ws_p,
+                           unsigned *ticket, cudaStream_t st, cudaEvent_t sweep_begin, cudaEvent_t sweep_end);
 int launch_topk_noalloc(Range r, const guide_outputs &mat, const guide_constraints &c, int key, u32 k,
                         u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st);
 

@@ -13,7 +13,7 @@
 // The metrics come either from materialised arrays or, fused, from the closed-form evaluation
 // itself, walked in the tiled order of tiled.cuh so the integer task tables are built once per
 // (model, batch, TP, length) point.
-#include "select.cuh"
+#include "select_sink.cuh"
 
 namespace guide {
 
@@ -1154,6 +1154,58 @@ int launch_pareto(const DSpace &s, Range r, const guide_outputs *mat, int time_m
     }
     FusedSource<0> src{s, make_cons(c), xm, ym, tp_model};
     return run_pareto_scan(src, r, idx_out, cap, count_out, ws, st);
+}
+
+// ---- simulate and select in one call ---------------------------------------------------------------
+//
+// A whole closed-form space, its metrics written out, and a top-k and a Pareto selection over it.
+// Where the space goes through the memory and line kernels, the selections cost no pass of their own:
+// their bound and killers come from a sample of configs evaluated first (the fused selection's first
+// half), the line kernel tests every config it evaluates against them while it stores the metrics, and
+// the rank kernels finish on the two short survivor lists.  The answers are those of the separate
+// calls (bound and killers only ever exclude configs that cannot be part of them); a survivor list
+// that overflows raises the redo flag, and the tiled fused kernels queued behind redo that selection.
+// Anything else runs the three calls one after the other on the stream.
+int launch_simulate_select(const DSpace &s, Range r, const guide_outputs &o, int time_model, int tp_model,
+                           const guide_constraints &ct, int key, u32 k, u64 *tk_idx, double *tk_key, u32 *tk_count, void *ws_t,
+                           const guide_constraints &cp, int xm, int ym, u64 *pf_idx, u32 cap, u32 *pf_count, void *ws_p,
+                           unsigned *ticket, cudaStream_t st, cudaEvent_t sweep_begin, cudaEvent_t sweep_end) {
+    int rc;
+    TileGeom g;
+    if (!(ticket && k <= STREAM_TOPK_MAX_K && fused_tiled(s, r, &g) && fused_stream_eligible(s, r) && closed_form_by_lines(s, r, o))) {
+        if (sweep_begin) GUIDE_CUDA(cudaEventRecord(sweep_begin, st));
+        if ((rc = launch_closed_form(s, r, time_model, tp_model, o, ticket, st))) return rc;
+        if (sweep_end) GUIDE_CUDA(cudaEventRecord(sweep_end, st));
+        if ((rc = launch_topk(s, r, &o, time_model, tp_model, ct, key, k, tk_idx, tk_key, tk_count, ws_t, nullptr, st))) return rc;
+        return launch_pareto(s, r, &o, time_model, tp_model, cp, xm, ym, pf_idx, cap, pf_count, ws_p, nullptr, st);
+    }
+    unsigned char *wt = (unsigned char *)ws_t, *wp = (unsigned char *)ws_p;
+    u32 *ht = (u32 *)wt, *hp = (u32 *)wp;                   // the top-k header is reset by its bound kernel
+    unsigned char *rt = wt + topk_stream_offset(k), *rp = wp + pareto_stream_offset();
+    // the two samples side by side, then the two bound kernels
+    GUIDE_CUDA(cudaMemsetAsync(wp, 0, 256, st));
+    if ((rc = launch_topk_fused(s, time_model, tp_model, ct, key, k, ht, rt, ticket, tk_idx, tk_key, tk_count, st, FUSED_SAMPLE))) return rc;
+    if ((rc = launch_pareto_fused(s, time_model, tp_model, cp, xm, ym, hp, rp, ticket, pf_idx, cap, pf_count, st, FUSED_SAMPLE_BESIDE)))
+        return rc;
+    if ((rc = launch_topk_fused(s, time_model, tp_model, ct, key, k, ht, rt, ticket, tk_idx, tk_key, tk_count, st, FUSED_BOUND_ONLY)))
+        return rc;
+    if ((rc = launch_pareto_fused(s, time_model, tp_model, cp, xm, ym, hp, rp, ticket, pf_idx, cap, pf_count, st, FUSED_BOUND_ONLY)))
+        return rc;
+    LineSelect sel;
+    sel.ct = make_cons(ct); sel.key = key; sel.header_t = ht;
+    sel.cp = make_cons(cp); sel.xm = xm; sel.ym = ym; sel.header_p = hp;
+    fused_lists(rt, rp, &sel);
+    if (sweep_begin) GUIDE_CUDA(cudaEventRecord(sweep_begin, st));
+    if ((rc = launch_closed_form(s, r, time_model, tp_model, o, ticket, st, &sel))) return rc;
+    if (sweep_end) GUIDE_CUDA(cudaEventRecord(sweep_end, st));
+    // both rank kernels, then the gated fallbacks (they return at once unless a survivor list overflowed)
+    if ((rc = launch_topk_fused(s, time_model, tp_model, ct, key, k, ht, rt, ticket, tk_idx, tk_key, tk_count, st, FUSED_RANK))) return rc;
+    if ((rc = launch_pareto_fused(s, time_model, tp_model, cp, xm, ym, hp, rp, ticket, pf_idx, cap, pf_count, st, FUSED_RANK))) return rc;
+    rc = time_model ? run_topk_tiled<1>(s, r, g, tp_model, sel.ct, key, k, wt, tk_idx, tk_key, tk_count, st, ht + TK_REDO)
+                    : run_topk_tiled<0>(s, r, g, tp_model, sel.ct, key, k, wt, tk_idx, tk_key, tk_count, st, ht + TK_REDO);
+    if (rc) return rc;
+    return time_model ? run_pareto_tiled<1>(s, r, g, tp_model, sel.cp, xm, ym, pf_idx, cap, pf_count, wp, st, true)
+                      : run_pareto_tiled<0>(s, r, g, tp_model, sel.cp, xm, ym, pf_idx, cap, pf_count, wp, st, true);
 }
 
 // ---- top-k over materialised metrics with library-owned scratch ----------------------------------

@@ -155,10 +155,20 @@ int launch_pareto_stream(Range r, const guide_outputs &mat, const guide_constrai
 // Fused form (nothing materialised, whole closed-form spaces): the sample rows are evaluated into a
 // compact scratch in the workspace, the same bound / killer kernels run on that, and the filter pass
 // is the model walk of model_walk.cuh with a sink that keeps candidates instead of storing metrics.
+// phase: the whole call, or a part of it around a filter pass that somebody else runs (the line
+// kernel of a combined simulate-and-select call): up to the bound / the killers (FUSED_BOUND; or in
+// two steps: the sample rows, possibly beside the stream's previous kernel when that is the other
+// selection's sample, then the bound kernels alone), or the ranking of what that pass left in the
+// lists (fused_lists() tells it where they are).
+enum { FUSED_ALL = 0, FUSED_BOUND = 1, FUSED_RANK = 2, FUSED_SAMPLE = 3, FUSED_SAMPLE_BESIDE = 4, FUSED_BOUND_ONLY = 5 };
 bool fused_stream_eligible(const DSpace &s, Range r);
 int launch_topk_fused(const DSpace &s, int time_model, int tp_model, const guide_constraints &c, int key, u32 k, u32 *header,
-                      unsigned char *region, unsigned *ticket, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st);
+                      unsigned char *region, unsigned *ticket, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st,
+                      int phase = FUSED_ALL);
 int launch_pareto_fused(const DSpace &s, int time_model, int tp_model, const guide_constraints &c, int xm, int ym, u32 *header,
-                        unsigned char *region, unsigned *ticket, u64 *idx_out, u32 cap, u32 *count_out, cudaStream_t st);
+                        unsigned char *region, unsigned *ticket, u64 *idx_out, u32 cap, u32 *count_out, cudaStream_t st,
+                        int phase = FUSED_ALL);
+struct LineSelect;
+void fused_lists(unsigned char *topk_region, unsigned char *pareto_region, LineSelect *sel);
 
 }  // namespace guide

@@ -34,7 +34,7 @@
 #include <cooperative_groups.h>
 
 #include "model_walk.cuh"
-#include "select.cuh"
+#include "select_sink.cuh"
 
 namespace guide {
 
@@ -49,7 +49,6 @@ static constexpr u32 TK_SAMPLE_ROWS = 8192;     // rows the sample aims at
 static constexpr u32 TK_SAMPLE_MAX_R = 32;
 static constexpr u32 TK_SKEYS_CAP = 8192;       // sample pairs within the coarse bound the workspace holds
 static constexpr u32 TK_SKEYS_SMEM = 2048;      // ... and how many the last block of the refinement sorts at once
-static constexpr u32 TK_CAND_CAP = 16384;       // survivors the workspace can hold
 static constexpr u32 TK_CAND_SMEM = 8192;       // ... of which the rank kernel stages this many in shared memory
 
 static constexpr u32 PA_SAMPLE_BLOCKS = 128;
@@ -57,10 +56,7 @@ static constexpr u32 PA_ROWS_PER_WARP = 4;
 static constexpr u32 PA_SAMPLE_ROWS = PA_SAMPLE_BLOCKS * (SEL_THREADS / 32) * PA_ROWS_PER_WARP;   // 4096
 static constexpr u32 PA_LOCAL_CAP = 1024;       // per-block list of sample points that survive the two seeds
 static constexpr u32 PA_PER_BLOCK = 2;          // front points a sample block hands on
-static constexpr u32 PA_KILLERS = PA_SAMPLE_BLOCKS * PA_PER_BLOCK;   // 256
-static constexpr u32 PA_SURV_CAP = 8192;        // survivors the workspace can hold
-
-struct P2 { u64 x, y; };
+static_assert(PA_KILLERS == PA_SAMPLE_BLOCKS * PA_PER_BLOCK, "every sample block hands on its share of the killers");
 
 // one metric array with the role it plays in this call
 struct Arr {
@@ -202,13 +198,6 @@ __device__ __forceinline__ void load_batch(const Src<NA> &s, const Sample &sm, u
 
 // ---- top-k ---------------------------------------------------------------------------------------
 //
-// Bounds are (key, index) pairs in the same total order as the answer, so that a key shared by
-// many configs (a metric with few distinct values) does not let them all through: of equal keys
-// only the indices up to the bound's survive.
-
-__device__ __forceinline__ bool pair_le(u64 key, u64 idx, u64 bkey, u64 bidx) {
-    return key < bkey || (key == bkey && idx <= bidx);
-}
 __device__ __forceinline__ void pair_min(u64 &key, u64 &idx, u64 okey, u64 oidx) {
     if (okey < key || (okey == key && oidx < idx)) { key = okey; idx = oidx; }
 }
@@ -479,11 +468,6 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_bound(Src<NA> s, Sample sm
     }
 }
 
-__device__ __forceinline__ void topk_keep(u64 key, u64 idx, u32 *header, KI *cand) {
-    const u32 pos = atomicAdd(header + TK_COUNT, 1);
-    if (pos < TK_CAND_CAP) { cand[pos].key = key; cand[pos].idx = idx; }
-}
-
 // Filter pass: passing configs within the bound go to the candidate list.
 template <int NA>
 __global__ void __launch_bounds__(SEL_THREADS, 4) k_topk_filter(Src<NA> s, Range r, u32 *header, KI *cand) {
@@ -573,11 +557,6 @@ __global__ void __launch_bounds__(SEL_THREADS) k_topk_rank(u32 *header, const KI
 }
 
 // ---- Pareto ----------------------------------------------------------------------------------------
-
-// does b rule a out?  strictly better in one coordinate and not worse in the other
-__device__ __forceinline__ bool dominates(u64 bx, u64 by, u64 ax, u64 ay) {
-    return bx <= ax && by <= ay && (bx < ax || by < ay);
-}
 
 // lexicographic minimum of (p, q) pairs over the block; every thread gets the result
 __device__ __forceinline__ void block_lex_min(u64 &p, u64 &q, u64 (*scratch)[2]) {
@@ -738,32 +717,6 @@ __global__ void __launch_bounds__(SEL_THREADS) k_pareto_sample(Src<NA> s, Sample
         *reinterpret_cast<ulonglong2 *>(killers + off + __popc(ballot & ((1u << lane) - 1))) = w;
     }
     if (threadIdx.x == 0) header[PH_KILLERS] = total;
-}
-
-struct KillerSet {
-    const P2 *k;      // shared: sorted by x, y strictly falling
-    u32 n;
-    u64 rx[4], ry[4]; // four of them in registers
-    // strictly dominated by a killer?  Only the killer with the largest x <= it.x can do it.
-    __device__ __forceinline__ bool kills(u64 x, u64 y) const {
-        bool dead = false;
-#pragma unroll
-        for (int i = 0; i < 4; i++) dead |= dominates(rx[i], ry[i], x, y);
-        if (dead) return true;
-        u32 lo = 0, hi = n;                           // first killer with x > it.x
-        while (lo < hi) {
-            const u32 mid = (lo + hi) >> 1;
-            if (k[mid].x <= x) lo = mid + 1; else hi = mid;
-        }
-        if (lo == 0) return false;
-        const P2 p = k[lo - 1];
-        return p.y < y || (p.y == y && p.x < x);
-    }
-};
-
-__device__ __forceinline__ void pareto_keep(u64 x, u64 y, u64 idx, u32 *header, P3 *surv) {
-    const u32 pos = atomicAdd(header + PH_COUNT, 1);
-    if (pos < PA_SURV_CAP) { surv[pos].x = x; surv[pos].y = y; surv[pos].idx = idx; }
 }
 
 // Filter pass: passing configs no killer strictly dominates go to the survivor list.
@@ -1025,10 +978,10 @@ int launch_pareto_stream(Range r, const guide_outputs &mat, const guide_constrai
 // the length pair.
 template <int TIME_SUM>
 __global__ void __launch_bounds__(SEL_THREADS) k_fused_sample(DSpace s, int tp_model, Sample sm, Cons c, int m0, int m1,
-                                                              u64 *row_base, uint8_t *pass, double *a0, double *a1) {
+                                                              u64 *row_base, uint8_t *pass, double *a0, double *a1, int beside) {
     grid_dep_launch();
     const u64 slot = (u64)blockIdx.x * (SEL_THREADS / ROW) + threadIdx.x / ROW;
-    if (slot >= sm.n_slots) return;
+    if (slot >= sm.n_slots) { if (beside) grid_dep_wait(); return; }
     const u32 l = threadIdx.x % ROW;
     const u64 first = sm.row(slot) * ROW;
     Metrics m;
@@ -1040,10 +993,9 @@ __global__ void __launch_bounds__(SEL_THREADS) k_fused_sample(DSpace s, int tp_m
     a0[q] = a;
     if (m1 >= 0) a1[q] = b;
     if (l == 0) row_base[slot] = first;
-}
-
-__device__ __forceinline__ bool meets(const Cons &c, double latency, double ttft, double thr, double cost_hr) {
-    return ttft <= c.max_ttft && latency <= c.max_latency && cost_hr <= c.max_cost_hr && thr >= c.min_thr;
+    // Launched beside its predecessor in the stream (another sample), the grid must not be complete
+    // before that one is: whatever follows in the stream waits for this grid only.
+    if (beside) grid_dep_wait();
 }
 
 // Filter pass of the fused top-k: the model walk, with the configs that fit, meet the constraints
@@ -1120,13 +1072,22 @@ static FusedScratch fused_scratch(unsigned char *base) {
 // sample rows of the space -> compact scratch; returns the walk over the scratch (row c of it is slot c)
 template <int TIME_SUM>
 static int fused_sample(const DSpace &s, int tp_model, const Cons &c, int m0, int m1, u32 want_rows, u32 max_r, const FusedScratch &f,
-                        Sample *compact, cudaStream_t st) {
+                        Sample *compact, cudaStream_t st, int phase) {
+    const bool beside = phase == FUSED_SAMPLE_BESIDE;
     const u64 total = (u64)s.n_m * s.n_h * s.n_f * s.n_b * s.n_t * s.n_l;
     Sample sm = make_sample(total / ROW, want_rows, max_r);
     sm.n_slots = std::min<u64>(sm.n_groups, FUSED_ROWS);
     const u32 grid = (u32)((sm.n_slots + SEL_THREADS / ROW - 1) / (SEL_THREADS / ROW));
-    k_fused_sample<TIME_SUM><<<grid, SEL_THREADS, 0, st>>>(s, tp_model, sm, c, m0, m1, f.row_base, f.pass, f.a0, f.a1);
-    GUIDE_CUDA(cudaGetLastError());
+    if (phase == FUSED_BOUND_ONLY) {
+        // the rows were evaluated by an earlier call with the same arguments
+    } else if (beside) {
+        // the stream's previous kernel is the other selection's sample, which lets its dependents start at once
+        GUIDE_CUDA(launch_dependent(k_fused_sample<TIME_SUM>, grid, SEL_THREADS, 0, st, s, tp_model, sm, c, m0, m1, f.row_base, f.pass,
+                                    f.a0, f.a1, 1));
+    } else {
+        k_fused_sample<TIME_SUM><<<grid, SEL_THREADS, 0, st>>>(s, tp_model, sm, c, m0, m1, f.row_base, f.pass, f.a0, f.a1, 0);
+        GUIDE_CUDA(cudaGetLastError());
+    }
     compact->n_groups = sm.n_slots; compact->n_slots = sm.n_slots; compact->mul = 1; compact->r = 1;
     return GUIDE_OK;
 }
@@ -1143,16 +1104,25 @@ static cudaError_t launch_model_dependent_cfg(cudaLaunchConfig_t *cfg, cudaLaunc
 
 template <int TIME_SUM>
 static int topk_fused_t(const DSpace &s, int tp_model, const guide_constraints &gc, int key, u32 k, u32 *header,
-                        unsigned char *region, unsigned *ticket, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st) {
+                        unsigned char *region, unsigned *ticket, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st,
+                        int phase) {
     const Cons c = make_cons(gc);
     const FusedScratch f = fused_scratch(region + TK_OFF_FUSED);
     ulonglong2 *minima = reinterpret_cast<ulonglong2 *>(region);
     ulonglong2 *spairs = reinterpret_cast<ulonglong2 *>(region + TK_OFF_SKEYS);
     KI *cand = reinterpret_cast<KI *>(region + TK_OFF_CAND);
-    GUIDE_CUDA(cudaMemsetAsync(ticket, 0, 4, st));           // the model walk's work counter
+    const size_t smem = (size_t)TK_CAND_SMEM * sizeof(KI);
+    if (phase == FUSED_RANK) {
+        GUIDE_CUDA(cudaFuncSetAttribute(k_topk_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        GUIDE_CUDA(launch_dependent(k_topk_rank, num_sms(), SEL_THREADS, smem, st, header, (const KI *)cand, k,
+                                    key == GUIDE_THROUGHPUT ? 1 : 0, idx_out, key_out, count_out));
+        return GUIDE_OK;
+    }
+    if (phase == FUSED_ALL) GUIDE_CUDA(cudaMemsetAsync(ticket, 0, 4, st));           // the model walk's work counter
     Sample sm;
-    int rc = fused_sample<TIME_SUM>(s, tp_model, c, key, -1, TK_SAMPLE_ROWS, TK_SAMPLE_MAX_R, f, &sm, st);
+    int rc = fused_sample<TIME_SUM>(s, tp_model, c, key, -1, TK_SAMPLE_ROWS, TK_SAMPLE_MAX_R, f, &sm, st, phase);
     if (rc) return rc;
+    if (phase == FUSED_SAMPLE || phase == FUSED_SAMPLE_BESIDE) return GUIDE_OK;
     Src<1> src;
     src.a[0] = Arr{f.a0, 0.0, 0, 0};                         // pick_metric has negated the throughput already
     src.status = f.pass;
@@ -1171,12 +1141,12 @@ static int topk_fused_t(const DSpace &s, int tp_model, const guide_constraints &
         GUIDE_CUDA(cudaGetLastError());
         GUIDE_CUDA(launch_dependent(k_topk_refine<1>, TK_SAMPLE_BLOCKS, SEL_THREADS, 0, st, src, sm, (u64)0, k, header, spairs));
     }
+    if (phase == FUSED_BOUND || phase == FUSED_BOUND_ONLY) return GUIDE_OK;
     const u32 n_chunks = (s.n_h * s.n_f + MODEL_CHUNK - 1) / MODEL_CHUNK;
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute at[1];
     launch_model_dependent_cfg(&cfg, at, st);
     GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_topk_model<TIME_SUM>, s, tp_model, n_chunks, ticket, c, key, header, cand));
-    const size_t smem = (size_t)TK_CAND_SMEM * sizeof(KI);
     GUIDE_CUDA(cudaFuncSetAttribute(k_topk_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     GUIDE_CUDA(launch_dependent(k_topk_rank, num_sms(), SEL_THREADS, smem, st, header, (const KI *)cand, k,
                                 key == GUIDE_THROUGHPUT ? 1 : 0, idx_out, key_out, count_out));
@@ -1184,14 +1154,23 @@ static int topk_fused_t(const DSpace &s, int tp_model, const guide_constraints &
 }
 
 int launch_topk_fused(const DSpace &s, int time_model, int tp_model, const guide_constraints &c, int key, u32 k, u32 *header,
-                      unsigned char *region, unsigned *ticket, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st) {
-    return time_model ? topk_fused_t<1>(s, tp_model, c, key, k, header, region, ticket, idx_out, key_out, count_out, st)
-                      : topk_fused_t<0>(s, tp_model, c, key, k, header, region, ticket, idx_out, key_out, count_out, st);
+                      unsigned char *region, unsigned *ticket, u64 *idx_out, double *key_out, u32 *count_out, cudaStream_t st,
+                      int phase) {
+    return time_model ? topk_fused_t<1>(s, tp_model, c, key, k, header, region, ticket, idx_out, key_out, count_out, st, phase)
+                      : topk_fused_t<0>(s, tp_model, c, key, k, header, region, ticket, idx_out, key_out, count_out, st, phase);
+}
+
+// Where the filter pass of a combined call finds the lists of the two selections' workspaces.
+void fused_lists(unsigned char *topk_region, unsigned char *pareto_region, LineSelect *sel) {
+    sel->cand = reinterpret_cast<KI *>(topk_region + TK_OFF_CAND);
+    sel->killers = reinterpret_cast<const P2 *>(pareto_region + PA_OFF_KILLERS);
+    sel->surv = reinterpret_cast<P3 *>(pareto_region + PA_OFF_SURV);
 }
 
 template <int TIME_SUM>
 static int pareto_fused_t(const DSpace &s, int tp_model, const guide_constraints &gc, int xm, int ym, u32 *header,
-                          unsigned char *region, unsigned *ticket, u64 *idx_out, u32 cap, u32 *count_out, cudaStream_t st) {
+                          unsigned char *region, unsigned *ticket, u64 *idx_out, u32 cap, u32 *count_out, cudaStream_t st,
+                          int phase) {
     const Cons c = make_cons(gc);
     const FusedScratch f = fused_scratch(region + PA_OFF_FUSED);
     P2 *local = reinterpret_cast<P2 *>(region);
@@ -1199,10 +1178,18 @@ static int pareto_fused_t(const DSpace &s, int tp_model, const guide_constraints
     u32 *local_n = reinterpret_cast<u32 *>(region + PA_OFF_LOCAL_N);
     P3 *surv = reinterpret_cast<P3 *>(region + PA_OFF_SURV);
     KI *front = reinterpret_cast<KI *>(region + PA_OFF_FRONT);
-    GUIDE_CUDA(cudaMemsetAsync(ticket, 0, 4, st));
+    const size_t smem = (size_t)PA_SURV_CAP * 16;
+    if (phase == FUSED_RANK) {
+        GUIDE_CUDA(cudaFuncSetAttribute(k_pareto_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        GUIDE_CUDA(launch_dependent(k_pareto_rank, num_sms(), SEL_THREADS, smem, st, header, (const P3 *)surv, front, idx_out, cap,
+                                    count_out));
+        return GUIDE_OK;
+    }
+    if (phase == FUSED_ALL) GUIDE_CUDA(cudaMemsetAsync(ticket, 0, 4, st));
     Sample sm;
-    int rc = fused_sample<TIME_SUM>(s, tp_model, c, xm, ym, PA_SAMPLE_ROWS, 1u << 20, f, &sm, st);
+    int rc = fused_sample<TIME_SUM>(s, tp_model, c, xm, ym, PA_SAMPLE_ROWS, 1u << 20, f, &sm, st, phase);
     if (rc) return rc;
+    if (phase == FUSED_SAMPLE || phase == FUSED_SAMPLE_BESIDE) return GUIDE_OK;
     Src<2> src;
     src.a[0] = Arr{f.a0, 0.0, 0, 0};
     src.a[1] = Arr{f.a1, 0.0, 0, 0};
@@ -1210,13 +1197,13 @@ static int pareto_fused_t(const DSpace &s, int tp_model, const guide_constraints
     src.row_base = f.row_base;
     k_pareto_sample<2><<<PA_SAMPLE_BLOCKS, SEL_THREADS, 0, st>>>(src, sm, header, local, local_n, killers);
     GUIDE_CUDA(cudaGetLastError());
+    if (phase == FUSED_BOUND || phase == FUSED_BOUND_ONLY) return GUIDE_OK;
     const u32 n_chunks = (s.n_h * s.n_f + MODEL_CHUNK - 1) / MODEL_CHUNK;
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute at[1];
     launch_model_dependent_cfg(&cfg, at, st);
     GUIDE_CUDA(cudaLaunchKernelEx(&cfg, k_pareto_model<TIME_SUM>, s, tp_model, n_chunks, ticket, c, xm, ym, header,
                                   (const P2 *)killers, surv));
-    const size_t smem = (size_t)PA_SURV_CAP * 16;
     GUIDE_CUDA(cudaFuncSetAttribute(k_pareto_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     GUIDE_CUDA(launch_dependent(k_pareto_rank, num_sms(), SEL_THREADS, smem, st, header, (const P3 *)surv, front, idx_out, cap,
                                 count_out));
@@ -1224,9 +1211,10 @@ static int pareto_fused_t(const DSpace &s, int tp_model, const guide_constraints
 }
 
 int launch_pareto_fused(const DSpace &s, int time_model, int tp_model, const guide_constraints &c, int xm, int ym, u32 *header,
-                        unsigned char *region, unsigned *ticket, u64 *idx_out, u32 cap, u32 *count_out, cudaStream_t st) {
-    return time_model ? pareto_fused_t<1>(s, tp_model, c, xm, ym, header, region, ticket, idx_out, cap, count_out, st)
-                      : pareto_fused_t<0>(s, tp_model, c, xm, ym, header, region, ticket, idx_out, cap, count_out, st);
+                        unsigned char *region, unsigned *ticket, u64 *idx_out, u32 cap, u32 *count_out, cudaStream_t st,
+                        int phase) {
+    return time_model ? pareto_fused_t<1>(s, tp_model, c, xm, ym, header, region, ticket, idx_out, cap, count_out, st, phase)
+                      : pareto_fused_t<0>(s, tp_model, c, xm, ym, header, region, ticket, idx_out, cap, count_out, st, phase);
 }
 
 }  // namespace guide

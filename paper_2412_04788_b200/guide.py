@@ -32,7 +32,7 @@ ALL_OUTPUTS = F64_OUTPUTS + ("status", "bmax", "n_iters", "n_req_iters")
 EXPORTS = ("guide_last_error", "guide_space_create", "guide_space_destroy", "guide_space_size", "guide_space_decode",
            "guide_trace_load", "guide_trace_destroy", "guide_trace_size", "guide_workspace_bytes", "guide_simulate",
            "guide_select_workspace_bytes", "guide_pareto_workspace_bytes", "guide_select_topk", "guide_pareto",
-           "guide_select_topk_noalloc")
+           "guide_simulate_select", "guide_select_topk_noalloc")
 
 
 class GuideError(RuntimeError):
@@ -86,6 +86,13 @@ class Constraints(C.Structure):
                 ("max_cost_per_hr", C.c_double), ("min_throughput", C.c_double)]
 
 
+class Selection(C.Structure):
+    _fields_ = [("topk_cons", C.POINTER(Constraints)), ("key", C.c_int32), ("k", C.c_uint32), ("topk_idx_dev", C.c_void_p),
+                ("topk_key_dev", C.c_void_p), ("topk_count_dev", C.c_void_p), ("pareto_cons", C.POINTER(Constraints)),
+                ("x_metric", C.c_int32), ("y_metric", C.c_int32), ("front_idx_dev", C.c_void_p), ("front_cap", C.c_uint32),
+                ("front_count_dev", C.c_void_p), ("sweep_begin_event", C.c_void_p), ("sweep_end_event", C.c_void_p)]
+
+
 _lib = None
 
 
@@ -124,6 +131,8 @@ def lib():
                                    C.c_int, C.c_int, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.guide_select_topk_noalloc.argtypes = [C.POINTER(Outputs), C.c_uint64, C.c_uint64, C.POINTER(Constraints), C.c_int,
                                                 C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.guide_simulate_select.argtypes = [C.c_void_p, C.POINTER(SimOpts), C.POINTER(Outputs), C.POINTER(Selection), C.c_void_p,
+                                            C.c_size_t, C.c_void_p, C.c_size_t, C.c_void_p]
         _lib = L
     return _lib
 
@@ -296,6 +305,25 @@ def guide_pareto(space: Space, trace: Trace | None, out: dict | None, cons: dict
                               C.byref(opts), C.byref(cs), METRICS[x], METRICS[y], _ptr(idx_out), idx_out.numel(),
                               _ptr(count_out), _ptr(workspace), workspace.numel() if workspace is not None else 0,
                               _stream_ptr(stream)))
+
+
+def guide_simulate_select(space: Space, out: dict, topk_cons: dict | None, key: str, k: int, topk_idx, topk_key, topk_count,
+                          topk_workspace, pareto_cons: dict | None, x: str, y: str, front_idx, front_count, pareto_workspace,
+                          first=0, count=0, time_model=TIME_MAX, tp_model=TP_EXPLICIT, stream=None, sweep_events=None):
+    """guide_simulate (closed form) + guide_select_topk + guide_pareto in one call: the metrics go to
+    `out`, the two answers to their tensors; on whole spaces the selections cost no pass of their own.
+    sweep_events: optional pair of torch.cuda.Event (already recorded once, so that they exist) that the
+    library records right before and after the kernels that evaluate and store the metrics."""
+    o = _outputs_struct(out)
+    opts = _opts(first, count, time_model, tp_model, 0)
+    ct, cp = _cons(topk_cons), _cons(pareto_cons)
+    sel = Selection(C.pointer(ct), METRICS[key], k, _ptr(topk_idx), _ptr(topk_key), _ptr(topk_count), C.pointer(cp),
+                    METRICS[x], METRICS[y], _ptr(front_idx), front_idx.numel(), _ptr(front_count),
+                    C.c_void_p(sweep_events[0].cuda_event) if sweep_events else None,
+                    C.c_void_p(sweep_events[1].cuda_event) if sweep_events else None)
+    _check(lib().guide_simulate_select(space.handle, C.byref(opts), C.byref(o), C.byref(sel), _ptr(topk_workspace),
+                                       topk_workspace.numel(), _ptr(pareto_workspace), pareto_workspace.numel(),
+                                       _stream_ptr(stream)))
 
 
 def guide_select_topk_noalloc(out: dict, cons: dict | None, key: str, k: int, idx_out, key_out, count_out,

@@ -71,3 +71,28 @@ def run_pareto(sp, out, cons, x, y, cap=guide.PARETO_MAX, tr=None, **kw):
     torch.cuda.synchronize()
     n = int(cnt.cpu().numpy().view(np.uint32)[0])
     return idx.cpu().numpy().view(np.uint64)[:min(n, cap)], n
+
+
+def run_simulate_select(space_np, topk_cons, key, k, pareto_cons, x, y, cap=guide.PARETO_MAX, **kw):
+    """guide_simulate_select on a closed-form space: (host metrics, (idx, val, cnt), (front idx, front size), device arrays, space)"""
+    import torch
+    sp = guide.Space(space_np)
+    first = kw.get("first", 0)
+    count = kw.get("count", 0) or sp.size - first
+    out = guide.alloc_outputs(count, 0)
+    idx = torch.empty(k, dtype=torch.int64, device="cuda")
+    val = torch.empty(k, dtype=torch.float64, device="cuda")
+    cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fidx = torch.empty(cap, dtype=torch.int64, device="cuda")
+    fcnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws_t = torch.empty(guide.guide_select_workspace_bytes(sp, k), dtype=torch.uint8, device="cuda")
+    ws_p = torch.empty(guide.guide_pareto_workspace_bytes(sp), dtype=torch.uint8, device="cuda")
+    guide.guide_simulate_select(sp, out, topk_cons, key, k, idx, val, cnt, ws_t, pareto_cons, x, y, fidx, fcnt, ws_p, **kw)
+    torch.cuda.synchronize()
+    host = {name: v.cpu().numpy() for name, v in out.items()}
+    host["bmax"] = host["bmax"].view(np.uint32)
+    host["n_iters"] = host["n_iters"].view(np.uint64)
+    host["n_req_iters"] = host["n_req_iters"].view(np.uint64)
+    n = int(fcnt.cpu().numpy().view(np.uint32)[0])
+    return (host, (idx.cpu().numpy().view(np.uint64), val.cpu().numpy(), int(cnt.item())),
+            (fidx.cpu().numpy().view(np.uint64)[:min(n, cap)], n), out, sp)

@@ -12,7 +12,7 @@ import pytest
 
 import oracle
 from paper_2412_04788_b200 import guide, inputs as I
-from gpu_util import run_pareto, run_simulate, run_topk
+from gpu_util import run_pareto, run_simulate, run_simulate_select, run_topk
 
 pytestmark = pytest.mark.gpu
 
@@ -233,3 +233,11 @@ def test_workload5_full_size_materialised_selection():
         idx, val, cnt = run_topk(sp5, out_dev, {}, key2, k2)
         w_idx, w_val, w_cnt = oracle.select_topk(want, {}, key2, k2)
         assert cnt == w_cnt and np.array_equal(idx, w_idx)
+    # the same step as one call: the sweep with both selections riding along
+    del out_dev, got
+    got, (idx, val, cnt), (fidx, fcnt), _, _ = run_simulate_select(w["space"], cons, key, k, cons, w["pareto"]["x"], w["pareto"]["y"])
+    for f in ("status", "bmax", "n_iters", "n_req_iters") + tuple(guide.F64_OUTPUTS):
+        assert np.array_equal(got[f].view(np.uint8), want[f].view(np.uint8)), f
+    w_idx, w_val, w_cnt = oracle.select_topk(want, cons, key, k)
+    assert cnt == w_cnt == k and np.array_equal(idx, w_idx) and np.array_equal(val.view(np.uint64), w_val.view(np.uint64))
+    assert fcnt == w_n and np.array_equal(fidx, w_f)
