@@ -22,6 +22,8 @@
 // Per-request results that outlive residency (tokens generated so far, first-token time, time per
 // output token) sit in a per-warp slice of the workspace.  The request trace is the same for every
 // config and is read through the read-only path, so it stays cache resident.
+#include <cstdlib>
+
 #include "guide_internal.cuh"
 #include "trace_fuse.cuh"
 #include "trace_lanes.cuh"
@@ -790,8 +792,12 @@ LaneHints lane_hints(const guide_space &s) {
             if (b >= LANE_CLASSES[c].minb && b <= LANE_CLASSES[c].maxb) all[c] += per_b;
     // Classes are taken from the first one up, without gaps (the warp-per-config kernel leaves out every
     // max batch up to the last launched class's limit), each only when it is large enough to pay.
+    // GUIDE_LANE_MIN_CONFIGS in the environment replaces the thresholds of the first two classes (the
+    // tests set it to 1 so that small spaces reach the lane kernel too); read once per process.
+    static const char *forced = getenv("GUIDE_LANE_MIN_CONFIGS");
     for (u32 c = 0; c < LANE_N_CLASSES; c++) {
-        if (all[c] < LANE_CLASSES[c].min_configs) break;
+        const u64 need = (forced && c < 2) ? strtoull(forced, nullptr, 10) : LANE_CLASSES[c].min_configs;
+        if (all[c] < need || all[c] == 0) break;
         h.class_configs[c] = all[c];
     }
     return h;

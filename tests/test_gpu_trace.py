@@ -87,6 +87,38 @@ def test_memory_pressure_small(seed):
     assert (want["status"] == guide.ST_KV).any() and (want["status"] == 0).any()
 
 
+@pytest.mark.parametrize("policy", ["prefill_first", "split_fuse"])
+def test_block_sizes_and_long_runs(policy):
+    """Runs of several hundred decode iterations (the warp kernels take them 32 at a time) cut short
+    by arrivals, completions and block shortages at every offset; block sizes that are not powers of
+    two, one-token blocks, the largest the histogram covers and one beyond it; idle gaps between
+    bursts of arrivals."""
+    n = 72
+    gaps = I.randint(5, 90, n, 0, 4)
+    arrival = np.cumsum(np.where(gaps == 0, 0.02, 1e-5 * gaps))          # bursts, then a long pause
+    tr = {"arrival": arrival, "in_len": I.randint(5, 91, n, 1, 90).astype(np.uint32),
+          "out_len": I.randint(5, 92, n, 1, 400).astype(np.uint32)}
+    blocks = [1, 3, 12, 64, 100]
+    hw, _ = I.seeded_hw(5, 4, mem_gb=[1] * 4)
+    w_bytes, kv_tok = oracle.weight_bytes_per_gpu(SMALL, 1), oracle.kv_bytes_per_token(SMALL, 1)
+    mem = np.array([w_bytes + tokens * kv_tok + 3 for tokens in (600, 1500, 4000, 10**6)], dtype=np.uint64)
+    fw_f, fw_i = I.seeded_fw(5, len(blocks), kv_block=4, reserve_permille=0)
+    fw_i[:, 1] = blocks
+    kw = {}
+    if policy == "split_fuse":
+        fw_i[:, 3] = guide.GUIDE_POLICY_SPLIT_FUSE
+        kw["fw_chunk"] = [[0, 48]] * len(blocks)
+    sp = I._space(np.array([SMALL]), hw, mem, fw_f, fw_i, [1, 2, 7, 40, 256], [1], [(1, 1)], **kw)
+    want = oracle.simulate(sp, tr, per_request=True)
+    got, *_ = run_simulate(sp, tr, per_request=True)
+    fields = guide.F64_OUTPUTS + ("req_ttft", "req_tpot")
+    assert_parity(got, want, fields=fields)
+    assert sum(bit_mismatches(got, want, fields).values()) == 0
+    ok = want["status"] == 0
+    assert ok.sum() >= 40 and want["n_preempt"][ok].sum() > 0
+    assert (want["n_iters"][ok] > 3000).any()                          # long schedules are in the sample
+
+
 @pytest.mark.parametrize("k", [3, 4])
 def test_workloads_3_and_4_reduced(k):
     """Workloads 3 and 4 with a shortened trace and one hardware profile in eight: same axes,
@@ -98,6 +130,28 @@ def test_workloads_3_and_4_reduced(k):
     assert_parity(got, want, fields=fields)
     assert sum(bit_mismatches(got, want, fields).values()) == 0
     assert (want["status"] == 0).sum() > 50
+
+
+def test_lane_kernel_on_small_spaces():
+    """The one-lane-per-config kernel is launched only for spaces with tens of thousands of configs of
+    small max batch; GUIDE_LANE_MIN_CONFIGS=1 sends every such config of a small space to it.  The
+    library reads the variable once per process, so the cases run in a child process: memory pressure
+    with 4-token blocks, block sizes and long runs, the reduced workloads 3 and 4."""
+    import os
+    import subprocess
+    import sys
+    code = (
+        "import sys; sys.path.insert(0, 'tests')\n"
+        "import test_gpu_trace as t\n"
+        "t.test_memory_pressure_small(2)\n"
+        "t.test_block_sizes_and_long_runs('prefill_first')\n"
+        "t.test_workloads_3_and_4_reduced(3)\n"
+        "t.test_workloads_3_and_4_reduced(4)\n"
+        "print('lane kernel ok')\n")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, "-c", code], cwd=root, env=dict(os.environ, GUIDE_LANE_MIN_CONFIGS="1"),
+                         capture_output=True, text=True, timeout=900)
+    assert res.returncode == 0 and "lane kernel ok" in res.stdout, res.stdout[-2000:] + res.stderr[-2000:]
 
 
 def test_iteration_cap_and_models(golden):
