@@ -39,7 +39,8 @@ namespace guide {
 #endif
 static constexpr u32 SIM_WARPS_PER_BLOCK = 8;
 static constexpr u32 SIM_THREADS = SIM_WARPS_PER_BLOCK * 32;
-static constexpr u32 SIM_MAX_WARPS = 6144;        // workspace is sized for this many resident warps
+static constexpr u32 SIM_MAX_WARPS = 3072;        // workspace is sized for this many resident warps: the warp-per-config kernels
+                                                  // keep two blocks of eight on an SM (148 SMs use 2,368; launches are capped here)
 static constexpr u32 LANE_MAX_WARPS = 148 * 16;   // ... and for this many warps of the lane kernel
 static constexpr u32 SLOTS = GUIDE_TRACE_MAX_BATCH;
 static constexpr u32 HIST = 64;                   // block sizes up to this use the phase histogram
@@ -759,8 +760,8 @@ struct LaneClass { u32 minb, maxb, lanes, round, unroll; u64 min_configs; };
 #ifndef LANE_CLASS0_MIN_WAVES
 #define LANE_CLASS0_MIN_WAVES 8
 #endif
-static const LaneClass LANE_CLASSES[LANE_N_CLASSES] = {{1, 16, 32, 64, 4, (u64)LANE_MAX_WARPS * LANE_CLASS0_MIN_WAVES},
-                                                       {17, 64, 32, 16, 1, (u64)LANE_MAX_WARPS * 32},
+static const LaneClass LANE_CLASSES[LANE_N_CLASSES] = {{1, 16, 32, 128, 4, (u64)LANE_MAX_WARPS * LANE_CLASS0_MIN_WAVES},
+                                                       {17, 64, 32, 32, 1, (u64)LANE_MAX_WARPS * 32},
                                                        {65, GUIDE_TRACE_MAX_BATCH, 8, 8, 1, ~0ull}};
 
 typedef void (*LaneKernel)(DSpace, DTrace, Range, int, u64, guide_outputs, unsigned long long *, unsigned char *, size_t, u32, u32,
