@@ -305,9 +305,9 @@ def extra_workloads(guide, torch, inputs, which, flush, hbm_peak, peak_kind, fra
                             "configs_per_s": n / best * 1e3, "iters_per_s": iters / best * 1e3,
                             "request_iters_per_s": req_iters / best * 1e3, "request_iters": req_iters,
                             "hardware_axis_fraction": scale, "workspace_bytes": ws.numel(),
-                            "kernels": "k_trace_lanes (one lane per config: small max batches, or every config of a small space) + "
-                                       "k_trace_sim (one warp per config: the rest)",
-                            "kernel_launches": {1: 2, 3: 2, 4: 3}[k],
+                            "kernels": "k_trace_sim (one warp per config, 32 iterations of a run at once)" +
+                                       ("" if k == 1 else " + k_trace_lanes (one lane per config: the large classes of small max batch)"),
+                            "kernel_launches": {1: 1, 3: 2, 4: 3}[k],
                             "roofline": alu_roofline(FP64_OPS_PER_ITERATION * iters / best * 1e3,
                                                      f"{FP64_OPS_PER_ITERATION} fp64 operations per simulated iteration x iterations/s"),
                             **extra}
