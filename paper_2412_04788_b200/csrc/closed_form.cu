@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(256, 2) k_closed_form_tiled(DSpace s, Range r,
 // positions, 128 bytes) and k_closed_form_lines takes the model kernel's place: see below.
 
 static constexpr u32 MEM_THREADS = 128;         // x 2 positions = 256 positions of the plane per work item
-static constexpr u32 MEM_BLOCKS_PER_SM = 2;
+static constexpr u32 MEM_BLOCKS_PER_SM = 3;       // 12 warps keep the write path busier than 8 (workload 5: 177.4 against 180.6 us for the pair); 16 do not (181 us)
 static constexpr int SPLIT_MAX_CONST = 10;
 
 // 8-byte arrays that receive a constant for a config that does not fit (+inf, or 0 for throughput and counters)
@@ -225,7 +225,7 @@ static constexpr u32 LINE_KILLERS = 64;          // killers the selecting varian
 // are in registers, and the few that either selection may still want go to its survivor list, so the
 // arrays need not be read back.
 template <int TIME_SUM, bool SELECT>
-__global__ void __launch_bounds__(MODEL_THREADS, LINE_BLOCKS_PER_SM + 1)      // registers: four blocks beside the memory kernel's two
+__global__ void __launch_bounds__(MODEL_THREADS, LINE_BLOCKS_PER_SM + 1)      // registers: four blocks beside the memory kernel's three (3 x 128 x 32 + 4 x 128 x 96 registers fit the file)
 k_closed_form_lines(DSpace s, int tp_model, guide_outputs o, u32 n_chunks, unsigned *ticket, LineSelect sel) {
     extern __shared__ __align__(16) double line_smem[];
     // Four blocks of this kernel fill an SM's shared memory but for a few KB: the filter keeps every
