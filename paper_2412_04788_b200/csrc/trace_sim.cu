@@ -533,7 +533,7 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                     // loop), watching for the arrival of the queue head where it could come in.
                     for (;;) {
                         const u32 nb = min(32u, steps_max - it);
-                        const double t_k = decode_time<TIME_SUM>(cd0 + nd * (double)(it + lane + 1), c_f9, dc_tha, c_kvx, c_f10, c_b10,
+                        const double t_k = decode_time<TIME_SUM>(cd0 + nd * ((double)it + (double)(lane + 1)), c_f9, dc_tha, c_kvx, c_f10, c_b10,
                                                                  icA, imA, dc_fix, dc_comm, dc_head, Nd, rt.tovh, lf);
                         // blocks the residents need before the iteration after lane's, and what is free by then
                         u32 need_k = 0;
