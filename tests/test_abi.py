@@ -154,3 +154,20 @@ def test_null_arguments_are_errors_not_crashes():
     cons = guide._cons({})
     assert L.guide_select_topk(sp.handle, None, None, None, C.byref(cons), 0, 0, None, None, None, None, 0, None) == guide.GUIDE_ERR_INVALID
     assert L.guide_select_topk(sp.handle, tr.handle, None, None, C.byref(cons), 0, 4, None, None, None, None, 0, None) == guide.GUIDE_ERR_UNSUPPORTED
+
+
+def test_simulate_select_refuses_bad_arguments_before_any_gpu_work():
+    L = guide.lib()
+    assert L.guide_simulate_select(None, None, None, None, None, 0, None, 0, None) == guide.GUIDE_ERR_INVALID
+    sp = guide.Space(I.workload(1)["space"])
+    out = guide.Outputs()
+    cons = guide._cons({})
+    sel = guide.Selection(C.pointer(cons), guide.METRICS["latency"], 4, None, None, None, C.pointer(cons),
+                          guide.METRICS["latency"], guide.METRICS["cost_per_hr"], None, 0, None, None, None)
+    # no status array among the outputs: the selections could not fall back on the arrays
+    assert L.guide_simulate_select(sp.handle, None, C.byref(out), C.byref(sel), None, 0, None, 0, None) == guide.GUIDE_ERR_INVALID
+    sel.key = 99
+    assert L.guide_simulate_select(sp.handle, None, C.byref(out), C.byref(sel), None, 0, None, 0, None) == guide.GUIDE_ERR_INVALID
+    opts = guide.SimOpts(0, 0, 0, 0, 0, 1, 0)                          # clamp_seq: the separate calls only
+    assert L.guide_simulate_select(sp.handle, C.byref(opts), C.byref(out), C.byref(sel), None, 0, None, 0, None) == guide.GUIDE_ERR_UNSUPPORTED
+    assert guide.guide_last_error()
