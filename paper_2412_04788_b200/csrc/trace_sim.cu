@@ -83,6 +83,8 @@ __device__ __forceinline__ double decode_time(double ctxd, double c_f9, double t
 struct SlotArrays {
     double tbuf[32];    // times of the 32 iterations a run computes at once
     double dterm[32][4];   // decode terms (fixed tasks, all-reduce, head, activation bytes) of 32 neighbouring resident counts
+    double sc[32];         // the config's task-table factors as doubles (a StageConst), when its counts stay exact in them
+    double rate[10];       // its row of rate10
     u32 req[SLOTS];     // request index
     u32 base[SLOTS];    // resident: cache - D (mod 2^32); waiting for its prompt pass: prompt + recompute tokens
     u32 fin[SLOTS];     // resident: D at which it completes; waiting for its prompt pass: tokens still to emit
@@ -323,8 +325,8 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         const double inv_tt = 1.0 / (double)tt;
         const double icA = rt.inv_c[CLS_ATTN], imA = rt.inv_m[CLS_ATTN];
         // configs the lane kernel was launched for are simulated there
-        if (lanes_take(lane_maxb, lane_hist, b, blk,
-                       lanes_exact(m, tt, b, max(tr.max_tokens, tr.any_zero ? Lin + Lout : 0u)))) continue;
+        const bool sc_ok = lanes_exact(m, tt, b, max(tr.max_tokens, tr.any_zero ? Lin + Lout : 0u));   // stage tables from doubles are exact
+        if (lanes_take(lane_maxb, lane_hist, b, blk, sc_ok)) continue;
 
         // ---- what fits (Sec. 3.2 Step 1) ----
         const u64 blocks_total = rt.usable > mi.w_gpu ? floor_div(rt.usable - mi.w_gpu, (u64)blk * mi.kv_tok) : 0;
@@ -382,6 +384,12 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         };
         if (!st) {
             for (u32 i = lane; i < HIST; i += 32) sl.hist[i] = 0;
+            if (sc_ok) {
+                // what a prompt pass needs, next to the warp: the (model, TP degree) factors and the pair's rates
+                const double *scg = reinterpret_cast<const double *>(s.stage_consts + (size_t)(tp_model ? s.n_t : c.t) * s.n_m + c.m);
+                sl.sc[lane] = scg[lane];
+                if (lane < 10) sl.rate[lane] = s.rate10[(size_t)(c.h * s.n_f + c.f) * 10 + lane];
+            }
             refresh_head();
             __syncwarp();
         }
@@ -422,7 +430,16 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                 const u64 T = pre_T, A = pre_A;          // summed at admission: tokens and tokens squared of the new prompts
                 pre_T = 0; pre_A = 0;
                 double t_iter;
-                {
+                if (sc_ok) {
+                    // the same operations on doubles (exact for this config), the factors read from shared memory as they are used
+                    const StageConst &sc = *reinterpret_cast<const StageConst *>(sl.sc);
+                    const double Td = (double)(long long)T, Ad = (double)(long long)A;
+                    const StageFixed sf = stage_fixed<TIME_SUM>(sc, sl.rate, Td, (double)n_new);
+                    const double xw = rt.flash ? 0.0 : sc.xb;
+                    const double t9 = task_time<TIME_SUM>(Ad * c_f9, ((Td * sc.ha + Td * sc.kv) + Ad * xw) * sc.inv_t, icA, imA);
+                    const double t10 = task_time<TIME_SUM>(Ad * c_f10, Ad * c_b10, icA, imA);
+                    t_iter = combine_phase(sf.fix, (t9 + t10) + t9, sf.comm, sf.head, 1.0, Nd, rt.tovh, lf);
+                } else {
                     TaskTab kt;
                     build_fixed_tasks(m, tt, T, n_new, 1, kt);
                     build_attn_tasks(m, tt, T, A, T, kt);
