@@ -85,6 +85,7 @@ struct SlotArrays {
     double dterm[32][4];   // decode terms (fixed tasks, all-reduce, head, activation bytes) of 32 neighbouring resident counts
     double sc[32];         // the config's task-table factors as doubles (a StageConst), when its counts stay exact in them
     double rate[10];       // its row of rate10
+    double cst[8];         // its attention and stage constants (read where they are used: they need not live in registers)
     u32 req[SLOTS];     // request index
     u32 base[SLOTS];    // resident: cache - D (mod 2^32); waiting for its prompt pass: prompt + recompute tokens
     u32 fin[SLOTS];     // resident: D at which it completes; waiting for its prompt pass: tokens still to emit
@@ -321,9 +322,10 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         const u32 Lin = pr.x, Lout = pr.y, blk = rt.kv_block;
         const MemInfo mi = mem_info(m, t);
         const u32 tt = tp_model ? 1u : t;
-        const double lf = log2_rule_factor(t, tp_model), Nd = (double)m.N;
         const double inv_tt = 1.0 / (double)tt;
-        const double icA = rt.inv_c[CLS_ATTN], imA = rt.inv_m[CLS_ATTN];
+        // per-config constants of the iteration time: kept next to the warp in shared memory
+        const double &lf = sl.cst[0], &Nd = sl.cst[1], &icA = sl.cst[2], &imA = sl.cst[3];
+        const double &c_f9 = sl.cst[4], &c_kvx = sl.cst[5], &c_f10 = sl.cst[6], &c_b10 = sl.cst[7];
         // configs the lane kernel was launched for are simulated there
         const bool sc_ok = lanes_exact(m, tt, b, max(tr.max_tokens, tr.any_zero ? Lin + Lout : 0u));   // stage tables from doubles are exact
         if (lanes_take(lane_maxb, lane_hist, b, blk, sc_ok)) continue;
@@ -345,10 +347,16 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         const u64 xw = rt.flash ? 0ull : (u64)m.nh * m.ab;                 // score-matrix bytes per unit of A
         const bool exact53 = 2 * (u64)m.H * ctx_max < lim53 && 5 * (u64)m.nh * ctx_max < lim53 &&
                              (u64)b * m.H * m.ab + ctx_max * ((u64)m.Dkv * m.kvb + xw) < lim53 && 2 * xw * ctx_max < lim53;
-        const double c_f9 = (double)(2 * (u64)m.H) * inv_tt;               // F9  = ctx * 2H / t
-        const double c_kvx = (double)((u64)m.Dkv * m.kvb + xw) * inv_tt;   // KV read + score bytes per context token / t
-        const double c_f10 = (double)(5 * (u64)m.nh) * inv_tt;             // F10 = ctx * 5 n_h / t
-        const double c_b10 = (double)(2 * xw) * inv_tt;                    // B10 = ctx * 2 n_h a_b / t (0 with flash)
+        __syncwarp();                                                      // the previous config's last reads of the constants
+        if (lane == 0) {
+            sl.cst[0] = log2_rule_factor(t, tp_model); sl.cst[1] = (double)m.N;
+            sl.cst[2] = rt.inv_c[CLS_ATTN]; sl.cst[3] = rt.inv_m[CLS_ATTN];
+            sl.cst[4] = (double)(2 * (u64)m.H) * inv_tt;                   // F9  = ctx * 2H / t
+            sl.cst[5] = (double)((u64)m.Dkv * m.kvb + xw) * inv_tt;        // KV read + score bytes per context token / t
+            sl.cst[6] = (double)(5 * (u64)m.nh) * inv_tt;                  // F10 = ctx * 5 n_h / t
+            sl.cst[7] = (double)(2 * xw) * inv_tt;                         // B10 = ctx * 2 n_h a_b / t (0 with flash)
+        }
+        __syncwarp();
 
         double clock = 0.0, dec_time = 0.0, csum_d = 0.0;   // csum_d mirrors csum when exact53
         u64 dec_tok = 0, n_iters = 0, n_req_iters = 0, free_blocks = blocks_total, csum = 0;
