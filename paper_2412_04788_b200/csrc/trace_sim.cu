@@ -80,12 +80,15 @@ __device__ __forceinline__ double decode_time(double ctxd, double c_f9, double t
     return combine_phase(fix, s_att, comm, head, 1.0, Nd, tovh, lf);
 }
 
+static_assert(sizeof(DModel) <= 128 && sizeof(DRate) <= 128, "a warp copies each of them with one word per lane");
 struct SlotArrays {
     double tbuf[32];    // times of the 32 iterations a run computes at once
     double dterm[32][4];   // decode terms (fixed tasks, all-reduce, head, activation bytes) of 32 neighbouring resident counts
     double sc[32];         // the config's task-table factors as doubles (a StageConst), when its counts stay exact in them
     double rate[10];       // its row of rate10
     double cst[8];         // its attention and stage constants (read where they are used: they need not live in registers)
+    DModel m;              // the config's model and (hardware, framework) rates
+    DRate rt;
     u32 req[SLOTS];     // request index
     u32 base[SLOTS];    // resident: cache - D (mod 2^32); waiting for its prompt pass: prompt + recompute tokens
     u32 fin[SLOTS];     // resident: D at which it completes; waiting for its prompt pass: tokens still to emit
@@ -314,9 +317,15 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
         const u64 idx = reorder ? work_to_index(s, w, true) : r.first + w;
         const u64 j = idx - r.first;
         const Cfg c = decode_index(s, idx);
-        const DModel m = s.models[c.m];
-        const DRate rt = s.rates[c.h * s.n_f + c.f];
-        if (rt.policy != GUIDE_POLICY_PREFILL_FIRST) continue;       // k_trace_fuse simulates those
+        const DRate *rate_g = s.rates + (c.h * s.n_f + c.f);
+        if (rate_g->policy != GUIDE_POLICY_PREFILL_FIRST) continue;  // k_trace_fuse simulates those
+        // the model and the pair's rates next to the warp: their fields are read where they are used
+        __syncwarp();
+        if (lane < sizeof(DModel) / 4) reinterpret_cast<u32 *>(&sl.m)[lane] = reinterpret_cast<const u32 *>(s.models + c.m)[lane];
+        if (lane < sizeof(DRate) / 4) reinterpret_cast<u32 *>(&sl.rt)[lane] = reinterpret_cast<const u32 *>(rate_g)[lane];
+        __syncwarp();
+        const DModel &m = sl.m;
+        const DRate &rt = sl.rt;
         const u32 t = s.tp[c.t], b = s.batch[c.b];
         const uint2 pr = s.pairs[c.l];
         const u32 Lin = pr.x, Lout = pr.y, blk = rt.kv_block;
