@@ -37,7 +37,10 @@ namespace guide {
 #ifndef FUSE_MIN_BLOCKS
 #define FUSE_MIN_BLOCKS 2         // ... and k_trace_fuse (measured 2.5 % faster than 3 blocks of 80 registers)
 #endif
-static constexpr u32 SIM_WARPS_PER_BLOCK = 8;
+#ifndef SIM_BLOCK_WARPS
+#define SIM_BLOCK_WARPS 8
+#endif
+static constexpr u32 SIM_WARPS_PER_BLOCK = SIM_BLOCK_WARPS;
 static constexpr u32 SIM_THREADS = SIM_WARPS_PER_BLOCK * 32;
 static constexpr u32 SIM_MAX_WARPS = 3072;        // workspace is sized for this many resident warps: the warp-per-config kernels
                                                   // keep two blocks of eight on an SM (148 SMs use 2,368; launches are capped here)
