@@ -575,16 +575,27 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                         // blocks the residents need before the iteration after lane's, and what is free by then
                         u32 need_k = 0;
                         if (lane < nb) need_k = blk == 1 ? nrun : sl.hist[hidx >= lmod ? hidx - lmod : hidx + blk - lmod];
-                        u32 incl = need_k;
-                        #pragma unroll
-                        for (int d = 1; d < 32; d <<= 1) {
-                            const u32 up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-                            if (lane >= (u32)d) incl += up;
+                        // Usually the free blocks cover the whole batch and the queue head's need: then only the
+                        // completion count can end the run on integers, and what is free afterwards is one sum.
+                        const u32 total = __reduce_add_sync(0xFFFFFFFFu, need_k);
+                        const bool plenty = (u64)total + need_next <= fb;
+                        u32 fb_k = 0, stops, last, watch;
+                        if (plenty) {
+                            last = nb - 1;
+                            stops = steps_max - it <= 32u ? 1u << last : 0u;
+                            watch = room ? 0xFFFFFFFFu >> (31 - last) : 0u;
+                        } else {
+                            u32 incl = need_k;
+                            #pragma unroll
+                            for (int d = 1; d < 32; d <<= 1) {
+                                const u32 up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                                if (lane >= (u32)d) incl += up;
+                            }
+                            fb_k = fb - (incl - need_k);                  // wraps only behind a lane that already stops
+                            stops = __ballot_sync(0xFFFFFFFFu, lane < nb && (it + lane + 1 == steps_max || need_k > fb_k));
+                            last = stops ? (u32)__ffs(stops) - 1 : 31u;   // a completion, the cap or an eviction follows it
+                            watch = __ballot_sync(0xFFFFFFFFu, room && need_next <= fb_k) & (0xFFFFFFFFu >> (31 - last));
                         }
-                        const u32 fb_k = fb - (incl - need_k);            // wraps only behind a lane that already stops
-                        const u32 stops = __ballot_sync(0xFFFFFFFFu, lane < nb && (it + lane + 1 == steps_max || need_k > fb_k));
-                        const u32 last = stops ? (u32)__ffs(stops) - 1 : 31u;   // a completion, the cap or an eviction follows it
-                        const u32 watch = __ballot_sync(0xFFFFFFFFu, room && need_next <= fb_k) & (0xFFFFFFFFu >> (31 - last));
                         sl.tbuf[lane] = t_k;
                         __syncwarp();
                         // the clock, one iteration after the other: four per trip, the arrival tests of a trip taken together
@@ -622,8 +633,11 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                         }
                         it += k + 1;
                         __syncwarp();
-                        if (stops || arrived) { fb = __shfl_sync(0xFFFFFFFFu, fb_k, k); break; }
-                        fb = __shfl_sync(0xFFFFFFFFu, fb_k - need_k, 31);
+                        if (stops || arrived) {
+                            fb = plenty ? fb - __reduce_add_sync(0xFFFFFFFFu, lane < k ? need_k : 0u) : __shfl_sync(0xFFFFFFFFu, fb_k, k);
+                            break;
+                        }
+                        fb = plenty ? fb - total : __shfl_sync(0xFFFFFFFFu, fb_k - need_k, 31);
                         hidx = hidx >= m32 ? hidx - m32 : hidx + blk - m32;
                     }
                     const double cd = cd0 + nd * (double)it;
