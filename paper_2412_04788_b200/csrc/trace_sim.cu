@@ -602,8 +602,10 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                         u32 k = 0;
                         bool arrived = false;
                         const u32 cnt = last + 1;
+                        double2 va = *(const double2 *)&sl.tbuf[0], vb = *(const double2 *)&sl.tbuf[2];
                         while (k + 4 <= cnt) {
-                            const double2 va = *(const double2 *)&sl.tbuf[k], vb = *(const double2 *)&sl.tbuf[k + 2];
+                            // the next trip's times are loaded ahead of this trip's additions (past the end: wraps, unused)
+                            const double2 na = *(const double2 *)&sl.tbuf[(k + 4) & 31], nb2 = *(const double2 *)&sl.tbuf[(k + 6) & 31];
                             const double c1 = clock + va.x, c2 = c1 + va.y, c3 = c2 + vb.x, c4 = c3 + vb.y;
                             const double d1 = dec_time + va.x, d2 = d1 + va.y, d3 = d2 + vb.x, d4 = d3 + vb.y;
                             const u32 wbits = (watch >> k) & 15u;
@@ -620,6 +622,7 @@ k_trace_sim(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guide
                                 break;
                             }
                             clock = c4; dec_time = d4;
+                            va = na; vb = nb2;
                             k += 4;
                         }
                         if (!arrived) {
