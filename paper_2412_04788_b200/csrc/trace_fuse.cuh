@@ -33,7 +33,7 @@ struct FuseSlots {
     u32 rem[GUIDE_TRACE_MAX_BATCH];     // tokens still to emit
     unsigned char fresh[GUIDE_TRACE_MAX_BATCH];   // no token emitted yet: the first one sets the TTFT
     u32 hist[FUSE_HIST];                // decode-only runs: residents per (cached tokens mod block size)
-    double tbuf[32];                    // decode-only runs: times of the 32 iterations worked out at once
+    alignas(16) double tbuf[32];        // decode-only runs: times of the 32 iterations worked out at once
     double dterm[32][3];                // decode-only runs: fixed-task, all-reduce and head terms of 32 neighbouring resident counts
 };
 
@@ -250,14 +250,40 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
                 const u32 watch = __ballot_sync(0xFFFFFFFFu, room && need_next <= free_k - need_k) & (0xFFFFFFFFu >> (31 - last));
                 sl.tbuf[lane] = t_k;
                 __syncwarp();
+                // the clock, one iteration after the other: four per trip, the arrival tests of a trip taken together
                 u32 k = 0;
                 bool arrived = false;
-                for (;; k++) {
-                    const double v = sl.tbuf[k];
-                    clock = clock + v;
-                    dec_time = dec_time + v;
-                    if (((watch >> k) & 1u) && arr_next <= clock) { arrived = true; break; }   // the queue head can come in
-                    if (k == last) break;
+                const u32 cnt = last + 1;
+                double2 va = *(const double2 *)&sl.tbuf[0], vb = *(const double2 *)&sl.tbuf[2];
+                while (k + 4 <= cnt) {
+                    const double2 na = *(const double2 *)&sl.tbuf[(k + 4) & 31], nb2 = *(const double2 *)&sl.tbuf[(k + 6) & 31];
+                    const double c1 = clock + va.x, c2 = c1 + va.y, c3 = c2 + vb.x, c4 = c3 + vb.y;
+                    const double d1 = dec_time + va.x, d2 = d1 + va.y, d3 = d2 + vb.x, d4 = d3 + vb.y;
+                    const u32 wbits = (watch >> k) & 15u;
+                    u32 hit = 0;
+                    if (wbits)
+                        hit = ((u32)(arr_next <= c1) | ((u32)(arr_next <= c2) << 1) | ((u32)(arr_next <= c3) << 2) |
+                               ((u32)(arr_next <= c4) << 3)) & wbits;
+                    if (hit) {                                             // the queue head can come in after one of the four
+                        const u32 f = (u32)__ffs(hit) - 1;
+                        clock = f == 0 ? c1 : f == 1 ? c2 : f == 2 ? c3 : c4;
+                        dec_time = f == 0 ? d1 : f == 1 ? d2 : f == 2 ? d3 : d4;
+                        k += f;
+                        arrived = true;
+                        break;
+                    }
+                    clock = c4; dec_time = d4;
+                    va = na; vb = nb2;
+                    k += 4;
+                }
+                if (!arrived) {
+                    for (; k < cnt; k++) {
+                        const double v = sl.tbuf[k];
+                        clock = clock + v;
+                        dec_time = dec_time + v;
+                        if (((watch >> k) & 1u) && arr_next <= clock) { arrived = true; break; }
+                    }
+                    if (!arrived) k = last;
                 }
                 free_blocks -= __shfl_sync(0xFFFFFFFFu, incl, k);
                 it += k + 1;
