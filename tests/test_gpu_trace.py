@@ -169,6 +169,31 @@ def test_iteration_cap_and_models(golden):
         assert sum(bit_mismatches(got, want).values()) == 0
 
 
+@pytest.mark.parametrize("policy", ["prefill_first", "split_fuse"])
+def test_iteration_cap_inside_long_runs(policy):
+    """The iteration cap can fall anywhere in a run that the warp kernels take 32 iterations at a time:
+    caps around the batch boundaries, one below the schedule's length and exactly its length."""
+    n = 6
+    tr = {"arrival": np.zeros(n), "in_len": np.full(n, 5, np.uint32), "out_len": np.array([40, 70, 33, 65, 97, 129], np.uint32)}
+    hw, _ = I.seeded_hw(3, 1, mem_gb=[1])
+    fw_f, fw_i = I.seeded_fw(3, 1, kv_block=4, reserve_permille=0)
+    kw = {}
+    if policy == "split_fuse":
+        fw_i[:, 3] = guide.GUIDE_POLICY_SPLIT_FUSE
+        kw["fw_chunk"] = [[0, 16]]
+    sp = I._space(np.array([SMALL]), hw, np.array([10**9], dtype=np.uint64), fw_f, fw_i, [1, 2, 8], [1], [(1, 1)], **kw)
+    full = oracle.simulate(sp, tr)
+    assert (full["status"] == 0).all()
+    caps = sorted({1, 2, 31, 32, 33, 34, 63, 64, 65, 66, 96, 97, 128, 129, 130}
+                  | {int(v) + d for v in full["n_iters"] for d in (-1, 0, 1)})
+    for cap in caps:
+        want = oracle.simulate(sp, tr, max_iters=cap)
+        got, *_ = run_simulate(sp, tr, max_iters=cap)
+        assert np.array_equal(got["status"], want["status"]), cap
+        assert np.array_equal(got["n_iters"], want["n_iters"]), cap
+        assert sum(bit_mismatches(got, want).values()) == 0, cap
+
+
 def test_run_to_run_identical():
     """The same launch twice gives the same bits (no dependence on scheduling order)."""
     w = I.workload(4, scale=1 / 64, trace_scale=1 / 4)
