@@ -33,6 +33,8 @@ struct FuseSlots {
     u32 rem[GUIDE_TRACE_MAX_BATCH];     // tokens still to emit
     unsigned char fresh[GUIDE_TRACE_MAX_BATCH];   // no token emitted yet: the first one sets the TTFT
     u32 hist[FUSE_HIST];                // decode-only runs: residents per (cached tokens mod block size)
+    double sc[32];                      // the config's task-table factors as doubles (a StageConst), when its counts stay exact in them
+    double rate[10];                    // its row of rate10
     alignas(16) double tbuf[32];        // decode-only runs: times of the 32 iterations worked out at once
     double dterm[32][3];                // decode-only runs: fixed-task, all-reduce and head terms of 32 neighbouring resident counts
 };
@@ -66,7 +68,8 @@ struct FuseTrace { const double *arrival; const u32 *in_len, *out_len; };
 template <int TIME_SUM>
 __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, const double *arrival, const u32 *in_len,
                                           const u32 *out_len, u32 n, u32 tt, u32 b, u32 Lin, u32 Lout, u64 blocks_total,
-                                          double lf, u64 max_iters, FuseSlots &sl, u32 *gen, double *first, double *tpot) {
+                                          double lf, u64 max_iters, FuseSlots &sl, u32 *gen, double *first, double *tpot,
+                                          const double *scg, const double *rate_g) {
     const DModel m = *mp;
     const DRate rt = *rp;
     const FuseTrace tr = {arrival, in_len, out_len};
@@ -82,6 +85,24 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
     auto modb = [&](u32 x) { return blk_shift != 0xFFFFFFFFu ? x & (blk - 1) : x % blk; };
     auto blocks_of = [&](u32 tokens) { return divb(tokens + blk - 1); };
 
+    // scg: the (model, TP degree) factors that turn token counts into a task table, as doubles, when the
+    // config's counts stay exact in them (null: the integer table).  Kept next to the warp with the
+    // pair's rates and read where they are used.
+    const bool sc_ok = scg != nullptr;
+    if (sc_ok) {
+        sl.sc[lane] = scg[lane];
+        if (lane < 10) sl.rate[lane] = rate_g[lane];
+        __syncwarp();
+    }
+    const StageConst &sc = *reinterpret_cast<const StageConst *>(sl.sc);
+    const double icA = rt.inv_c[CLS_ATTN], imA = rt.inv_m[CLS_ATTN];
+    // attention tasks of a stage from doubles: the operations of build_attn_tasks and eval_attn on exact values
+    auto attn_d = [&](double Td, double Ad, double Cd) {
+        const double xw = rt.flash ? 0.0 : sc.xb;
+        const double t9 = task_time<TIME_SUM>(Ad * sc.f9, ((Td * sc.ha + Cd * sc.kv) + Ad * xw) * sc.inv_t, icA, imA);
+        const double t10 = task_time<TIME_SUM>(Ad * sc.f10, rt.flash ? 0.0 : (2.0 * (Ad * sc.xb)) * sc.inv_t, icA, imA);
+        return (t9 + t10) + t9;
+    };
     double clock = 0.0, dec_time = 0.0;
     u64 dec_tok = 0, n_iters = 0, n_req_iters = 0, free_blocks = blocks_total;
     u32 next = 0, high_water = 0, nrun = 0, st = 0;
@@ -106,6 +127,16 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
 
     // one stage time from (T, E, A, C); everything but attention is kept while T and E repeat
     auto stage_time = [&](u64 T, u64 E, u64 A, u64 C) {
+        if (sc_ok) {
+            const double Td = (double)(long long)T;
+            if (T != dc_T || E != dc_E) {
+                const StageFixed sf = stage_fixed<TIME_SUM>(sc, sl.rate, Td, (double)(long long)E);
+                dc_T = T; dc_E = E;
+                dc_fix = sf.fix; dc_comm = sf.comm;
+                dc_head = E ? sf.head : 0.0;                       // nobody emits a token: no LM head
+            }
+            return combine_phase(dc_fix, attn_d(Td, (double)(long long)A, (double)(long long)C), dc_comm, dc_head, 1.0, Nd, rt.tovh, lf);
+        }
         if (T != dc_T || E != dc_E) {
             TaskTab kf;
             build_fixed_tasks(m, tt, T, E, 1, kf);
@@ -226,9 +257,16 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
             for (;;) {
                 const u32 nb = min(32u, steps_max - it);
                 const u64 ctx_k = ctx_i + (u64)lane * nrun;
-                TaskTab ka;
-                build_attn_tasks(m, tt, nrun, ctx_k, ctx_k, ka);
-                const double t_k = combine_phase(d_fix, eval_attn<TIME_SUM>(ka, rt), d_comm, d_head, 1.0, Nd, rt.tovh, lf);
+                double s_att;
+                if (sc_ok) {
+                    const double cd = (double)(long long)ctx_k;
+                    s_att = attn_d((double)nrun, cd, cd);
+                } else {
+                    TaskTab ka;
+                    build_attn_tasks(m, tt, nrun, ctx_k, ctx_k, ka);
+                    s_att = eval_attn<TIME_SUM>(ka, rt);
+                }
+                const double t_k = combine_phase(d_fix, s_att, d_comm, d_head, 1.0, Nd, rt.tovh, lf);
                 u32 need_k = 0;                                    // residents whose last block is full before lane's iteration
                 if (lane < nb) {
                     const u32 o = off + lmod >= blk ? off + lmod - blk : off + lmod;
