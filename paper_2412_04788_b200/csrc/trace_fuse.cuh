@@ -14,6 +14,8 @@
 // some request is in its prompt, evaluate one stage time, apply, retire); the non-attention terms
 // of the stage time are kept while the iteration's token counts repeat.
 #pragma once
+#include <cstddef>
+
 #include "guide_internal.cuh"
 
 namespace guide {
@@ -25,6 +27,9 @@ struct FuseResult {
     u64 dec_tok, n_iters, n_req_iters;
 };
 
+static_assert(sizeof(DModel) <= 128 && sizeof(DRate) <= 128, "a warp copies each of them with one word per lane");
+static_assert(offsetof(DRate, inv_m) == 24 && offsetof(DRate, inv_comm) == 48 && offsetof(DRate, clat) == 56 && offsetof(DRate, tovh) == 64,
+              "a rate entry starts like a row of rate10");
 struct FuseSlots {
     FuseResult res;                     // what the schedule hands back to the kernel around it
     u32 req[GUIDE_TRACE_MAX_BATCH];     // request index, ascending
@@ -34,7 +39,8 @@ struct FuseSlots {
     unsigned char fresh[GUIDE_TRACE_MAX_BATCH];   // no token emitted yet: the first one sets the TTFT
     u32 hist[FUSE_HIST];                // decode-only runs: residents per (cached tokens mod block size)
     double sc[32];                      // the config's task-table factors as doubles (a StageConst), when its counts stay exact in them
-    double rate[10];                    // its row of rate10
+    DModel m;                           // the config's model and (hardware, framework) rates
+    DRate rt;
     alignas(16) double tbuf[32];        // decode-only runs: times of the 32 iterations worked out at once
     double dterm[32][3];                // decode-only runs: fixed-task, all-reduce and head terms of 32 neighbouring resident counts
 };
@@ -69,9 +75,15 @@ template <int TIME_SUM>
 __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, const double *arrival, const u32 *in_len,
                                           const u32 *out_len, u32 n, u32 tt, u32 b, u32 Lin, u32 Lout, u64 blocks_total,
                                           double lf, u64 max_iters, FuseSlots &sl, u32 *gen, double *first, double *tpot,
-                                          const double *scg, const double *rate_g) {
-    const DModel m = *mp;
-    const DRate rt = *rp;
+                                          const double *scg) {
+    // the model and the pair's rates next to the warp: their fields are read where they are used
+    const u32 lane0 = threadIdx.x & 31;
+    __syncwarp();
+    if (lane0 < sizeof(DModel) / 4) reinterpret_cast<u32 *>(&sl.m)[lane0] = reinterpret_cast<const u32 *>(mp)[lane0];
+    if (lane0 < sizeof(DRate) / 4) reinterpret_cast<u32 *>(&sl.rt)[lane0] = reinterpret_cast<const u32 *>(rp)[lane0];
+    __syncwarp();
+    const DModel &m = sl.m;
+    const DRate &rt = sl.rt;
     const FuseTrace tr = {arrival, in_len, out_len};
     const double Nd = (double)m.N;
     const u32 lane = threadIdx.x & 31;
@@ -91,7 +103,6 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
     const bool sc_ok = scg != nullptr;
     if (sc_ok) {
         sl.sc[lane] = scg[lane];
-        if (lane < 10) sl.rate[lane] = rate_g[lane];
         __syncwarp();
     }
     const StageConst &sc = *reinterpret_cast<const StageConst *>(sl.sc);
@@ -130,7 +141,7 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
         if (sc_ok) {
             const double Td = (double)(long long)T;
             if (T != dc_T || E != dc_E) {
-                const StageFixed sf = stage_fixed<TIME_SUM>(sc, sl.rate, Td, (double)(long long)E);
+                const StageFixed sf = stage_fixed<TIME_SUM>(sc, rt.inv_c, Td, (double)(long long)E)   /* a rate entry starts like a row of rate10 */;
                 dc_T = T; dc_E = E;
                 dc_fix = sf.fix; dc_comm = sf.comm;
                 dc_head = E ? sf.head : 0.0;                       // nobody emits a token: no LM head

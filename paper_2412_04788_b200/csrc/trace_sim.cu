@@ -774,8 +774,7 @@ k_trace_fuse(DSpace s, DTrace tr, Range r, int tp_model, u64 max_iters_opt, guid
                                     ? reinterpret_cast<const double *>(s.stage_consts + (size_t)(tp_model ? s.n_t : c.t) * s.n_m + c.m)
                                     : nullptr;
             st |= fuse_schedule<TIME_SUM>(mp, rp, tr.arrival, tr.in_len, tr.out_len, n, tp_model ? 1u : t, b, Lin, Lout, blocks_total,
-                                          log2_rule_factor(t, tp_model), max_iters, sh[wib], gen, first, tpot, scg,
-                                          s.rate10 + (size_t)(c.h * s.n_f + c.f) * 10);
+                                          log2_rule_factor(t, tp_model), max_iters, sh[wib], gen, first, tpot, scg);
             fr = sh[wib].res;
         }
         write_trace_results(o, j, n, st, fit, fr.clock, fr.dec_time, fr.dec_tok, fr.n_iters, fr.n_req_iters,
