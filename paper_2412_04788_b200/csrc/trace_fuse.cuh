@@ -398,9 +398,11 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
         u64 T = n_dec, A = ctx, C = ctx;
         u32 E = n_dec, n_chunk = 0, n_finish = 0;
         const bool chunks = n_pre > 0 && left0 > 0;
+        u32 plan_q = 0;                                            // prompt tokens this lane's slot gets (slots 0..31)
         if (chunks) {
             u64 carry = 0, pT = 0, pA = 0, pC = 0;
             u32 pEN = 0;                                           // finishing << 16 | chunks
+            plan_q = 0;
             for (u32 base = 0; base < nrun && carry < left0; base += 32) {
                 const u32 k = base + lane;
                 const u64 td = k < nrun ? sl.todo[k] : 0;
@@ -411,6 +413,7 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
                     const u64 upto = (u64)sl.seen[k] + q;
                     pT += q; pA += q * upto; pC += upto;
                     pEN += 1u + (q == td ? 0x10000u : 0u);
+                    plan_q = (u32)q;                               // with at most 32 residents the pass below needs no second scan
                 }
                 carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
             }
@@ -434,6 +437,27 @@ __device__ __noinline__ u32 fuse_schedule(const DModel *mp, const DRate *rp, con
                     any_done |= rm == 0;
                 }
             }
+        } else if (nrun <= 32) {
+            // one slot per lane: the chunk sizes are those of the plan
+            if (lane < nrun) {
+                const u32 td = sl.todo[lane];
+                if (td == 0) {                                      // decoded one token
+                    sl.seen[lane] += 1;
+                    const u32 rm = sl.rem[lane] - 1;
+                    sl.rem[lane] = rm;
+                    any_done |= rm == 0;
+                } else if (plan_q) {
+                    sl.seen[lane] += plan_q;
+                    sl.todo[lane] = td - plan_q;
+                    if (plan_q == td) {                             // prompt finished: first token
+                        const u32 rm = sl.rem[lane] - 1;
+                        sl.rem[lane] = rm;
+                        any_done |= rm == 0;
+                        if (sl.fresh[lane]) { first[sl.req[lane]] = after; sl.fresh[lane] = 0; }
+                    }
+                }
+            }
+            n_pre -= n_finish;
         } else {
             u64 carry = 0;
             for (u32 base = 0; base < nrun; base += 32) {
