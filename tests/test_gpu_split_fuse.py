@@ -106,3 +106,30 @@ def test_iteration_limit_and_bad_profiles():
         with pytest.raises(guide.GuideError) as e:
             run_simulate(I._space(np.array([SMALL]), hw, np.array([10**9]), fw_f, fw_i, [1], [1], [(4, 3)], fw_chunk=chunk), tr)
         assert e.value.code == guide.GUIDE_ERR_INVALID
+
+
+def test_benchmark_case_sampled():
+    """The case bench.py times: workload 3 on half of its hardware axis (32,768 configs x 4096
+    requests), every framework on the split-and-fuse policy with token budgets 256 .. 8192, in one
+    launch; every 29th config is recomputed by the oracle and must match bit for bit, per-request
+    values included.  GUIDE_TRACE_PARITY_STRIDE overrides the stride."""
+    import os
+    import torch
+    stride = int(os.environ.get("GUIDE_TRACE_PARITY_STRIDE", 29))
+    w = I.workload(3, scale=0.5, trace_scale=1.0)
+    space = fuse_space(w["space"], [256, 512, 2048, 8192])
+    sp, tr = guide.Space(space), guide.Trace(w["trace"])
+    n = sp.size
+    out = guide.alloc_outputs(n, tr.n, per_request=True)
+    ws = torch.empty(guide.guide_workspace_bytes(sp, tr), dtype=torch.uint8, device="cuda")
+    guide.guide_simulate(sp, tr, out, workspace=ws)
+    torch.cuda.synchronize()
+    count = (n + stride - 1) // stride
+    want = oracle.simulate(space, w["trace"], first=0, count=count, stride=stride, per_request=True)
+    for f in guide.F64_OUTPUTS + ("req_ttft", "req_tpot"):
+        got = out[f][::stride].cpu().numpy()
+        assert np.array_equal(got.view(np.uint64), want[f].view(np.uint64)), f
+    assert np.array_equal(out["status"][::stride].cpu().numpy(), want["status"])
+    assert np.array_equal(out["n_iters"][::stride].cpu().numpy().view(np.uint64), want["n_iters"])
+    assert np.array_equal(out["n_req_iters"][::stride].cpu().numpy().view(np.uint64), want["n_req_iters"])
+    assert int((out["status"] == 0).sum()) > n // 2
